@@ -1,0 +1,207 @@
+/*
+ * spark.h -- C ABI of the B200 (sm_100a) Spark Transformer decode library.
+ *
+ * The library implements the per-token, activation-sparse decode step of the
+ * Spark Transformer: statistical top-k (Section 3, Eq. 9-11), Spark FFN
+ * (Section 2.1, Eq. 2) and Spark attention (Section 2.2, Eq. 7), plus the dense
+ * glue a decoder layer needs around them (Section 4, "Implementation details").
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ * - All tensor arguments are DEVICE pointers on the context's device unless a
+ *   comment says "host".  The caller owns every buffer, including the
+ *   workspace handed to spark_create; the library never allocates or frees
+ *   device memory and keeps no pointer beyond a call except that workspace.
+ * - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   Calls only enqueue work; outputs are valid once the stream has been
+ *   synchronised.  Calls that share one context must be issued on one stream
+ *   (they share the workspace); use one context per concurrent stream.
+ * - Return value: 0 (SPARK_OK) or one of the SPARK_ERR_* codes below.  Argument
+ *   errors are detected on the host before anything is enqueued.  Conditions
+ *   only the device can see (a bounded wait that ran out, ...) are recorded in a
+ *   device status word read by spark_device_status.  Nothing aborts or traps.
+ * - Activations (x, q, y, o, h, theta) are fp32.  Weights and KV caches are
+ *   fp32 (SPARK_F32) or bf16 (SPARK_BF16), accumulated in fp32.  Every row of a
+ *   weight / cache tensor must start on a 16-byte boundary: base pointers
+ *   16-byte aligned and row lengths a multiple of 8 elements (bf16) or 4 (fp32),
+ *   otherwise SPARK_ERR_UNSUPPORTED.
+ * - FFN weights are stored neuron-major, i.e. as the transposes of the paper's
+ *   matrices: K1t[d_ff][r] = K1^T, K2t[d_ff][d-r] = K2^T, Vt[d_ff][d] = V^T,
+ *   row-major, so that one neuron's weights are one contiguous run ("we store
+ *   the matrix in row format", Appendix B).
+ * - KV caches are token-major with each key split into its predictor slice and
+ *   the rest (Section 2.2: K1 = first r rows of K, K2 = the others):
+ *   k1c[B][n_kv][cap][r], k2c[B][n_kv][cap][hd-r], vc[B][n_kv][cap][hd].
+ * - Degenerate k (the paper leaves them open): k >= n keeps every entry
+ *   unshifted (theta reported as -inf); k <= 0 is SPARK_ERR_INVALID_ARG.
+ *   Selection is the strict comparison x_i > theta; the number selected is
+ *   whatever exceeds theta (about k, not capped at k).
+ */
+#ifndef SPARK_H_
+#define SPARK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ------------------------------------------------------- */
+enum {
+    SPARK_OK = 0,
+    SPARK_ERR_INVALID_ARG = 1, /* null pointer, k <= 0, r outside (0, d), n_q % n_kv != 0, ...      */
+    SPARK_ERR_UNSUPPORTED = 2, /* misaligned pointer / row length, unknown dtype, size over a limit */
+    SPARK_ERR_WORKSPACE = 3,   /* the context's workspace is too small for this call                */
+    SPARK_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                            */
+    SPARK_ERR_TIMEOUT = 5,     /* device: a bounded wait between thread blocks ran out              */
+    SPARK_ERR_OVERFLOW = 6     /* device: an index list did not fit its capacity (truncated)        */
+};
+
+/* ---- dtypes and flags ----------------------------------------------------- */
+enum { SPARK_F32 = 0, SPARK_BF16 = 1 };
+
+enum {
+    SPARK_FILL_ZERO = 0,   /* Eq. 10: entries not above theta become 0                       */
+    SPARK_FILL_NEGINF = 1  /* the Top_k^(-inf) variant of Section 3 used by Spark attention   */
+};
+
+enum {
+    SPARK_GELU_TANH = 0,     /* tanh form of GELU (the one Gemma uses); the default            */
+    SPARK_GELU_ERF = 1,      /* exact form x * Phi(x)                                          */
+    SPARK_DENSE_LOADS = 2    /* comparator: same result, but every row of K2/V (or of the cache)
+                                is read and multiplied by its (possibly zero) activation       */
+};
+
+typedef struct spark_ctx spark_ctx;
+
+/* ---- context -------------------------------------------------------------- */
+
+/* Bytes of workspace a context needs so that every call with batch <= max_batch,
+ * d_ff <= max_dff, cache capacity <= max_cap, n_q query heads of head_dim hd and model
+ * width <= max_d fits.  Pure host arithmetic. */
+size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap, int64_t n_q,
+                             int64_t hd, int64_t max_d);
+
+/* Create a context on `device` around a caller-owned device workspace (256-byte aligned).
+ * Zeroes the workspace header (a small synchronous memset); queries the SM count.
+ * *out is a host object released by spark_destroy (which leaves the workspace alone). */
+int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_bytes);
+int spark_destroy(spark_ctx* ctx);
+
+/* Synchronise `stream`, copy the device status word to *host_out (host pointer), clear it, and
+ * if it was not SPARK_OK also reset the inter-block barrier state.  Returns SPARK_OK when the
+ * read itself worked (the device status is in *host_out). */
+int spark_device_status(spark_ctx* ctx, void* stream, int* host_out);
+
+/* Static string for a status code (host pointer, never freed). */
+const char* spark_status_string(int status);
+
+/* Number of thread blocks the context launches for its cooperative kernels (= SM count). */
+int spark_grid_size(const spark_ctx* ctx);
+
+/* Gaussian upper quantile used for the threshold: z with P(N(0,1) > z) = p, i.e. Q(1 - p) of
+ * Eq. 11.  Host function (no device work); exported so that it can be checked on its own.
+ * Returns NaN for p outside (0, 1). */
+double spark_normal_upper_quantile(double p);
+
+/* ---- statistical top-k (Section 3, Eq. 9-11) -------------------------------
+ * For each of `rows` rows x[row*ld .. row*ld + n): theta = mean + std * Q(1 - k/n) with the
+ * Bessel-corrected std, active set A = { i : x_i > theta }, values x_i - theta.
+ *   theta  [rows]               fp32, nullable
+ *   count  [rows]               int32, nullable: |A| (the full count even when idx_cap is smaller)
+ *   idx    [rows][idx_cap]      int32, nullable: A in ascending order, first min(|A|, idx_cap)
+ *   val    [rows][idx_cap]      fp32,  nullable: x_i - theta for those entries
+ *   y_dense[rows][ld]           fp32,  nullable: the dense result of Eq. 10 (fill = 0) or of the
+ *                               -inf variant (fill = SPARK_FILL_NEGINF)
+ * If |A| > idx_cap the lists are truncated and SPARK_ERR_OVERFLOW is recorded in the device
+ * status.  x needs 16-byte aligned rows (x aligned, ld % 4 == 0).  n >= 2 unless k >= n. */
+int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, int64_t k,
+                    int fill, float* theta, int32_t* count, int32_t* idx, float* val,
+                    int64_t idx_cap, float* y_dense, void* stream);
+
+/* ---- Spark FFN (Section 2.1, Eq. 2) ------------------------------------------
+ * y_b = V . ( GELU(StatTop_k(K1^T x_b[:r])) * (K2^T x_b[r:]) ) for each of the B tokens, every
+ * token with its own threshold and active set; weight rows are loaded once per call for the
+ * union of the tokens' active sets (Appendix B).
+ *   x [B][d] fp32;  K1t[d_ff][r], K2t[d_ff][d-r], Vt[d_ff][d] of dtype wdtype
+ *   flags: SPARK_GELU_TANH or SPARK_GELU_ERF, optionally | SPARK_DENSE_LOADS
+ *   y     [B][d]     fp32 (overwritten)
+ *   theta [B]        fp32,  nullable
+ *   count [B]        int32, nullable
+ *   idx   [B][d_ff]  int32, nullable: active neurons of token b in unspecified order; entries past
+ *                    count[b] are not written
+ * Limits: 1 <= B <= 64, 0 < r < d, r % 8 == 0, d % 8 == 0, d_ff >= 2. */
+int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const void* K2t,
+                     const void* Vt, int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k,
+                     int flags, float* y, float* theta, int32_t* count, int32_t* idx, void* stream);
+
+/* ---- Spark attention (Section 2.2, Eq. 7) ------------------------------------
+ * For sequence b and query head h (KV head g = h / (n_q / n_kv)), over the tokens t of the window
+ * [max(0, n_b - window), n_b), n_b = ctx_len[b] (window == 0: all n_b tokens):
+ *   s_t = k1c[b][g][t] . q[b][h][:r];  A = StatTop_{k_attn}^{(-inf)}(s);
+ *   o[b][h] = sum_{t in A} softmax_A(s)_t * softplus(k2c[b][g][t] . q[b][h][r:]) * vc[b][g][t]
+ * q is used as given (apply the position encoding and any 1/sqrt(hd) scale before the call).
+ * A window of at most k_attn tokens is attended to densely; an empty A gives o = 0.
+ *   q [B][n_q][hd] fp32;  ctx_len [B] int32 DEVICE array, 1 <= ctx_len[b] <= cap
+ *   flags: 0 or SPARK_DENSE_LOADS
+ *   o     [B][n_q][hd]       fp32 (overwritten)
+ *   theta [B][n_q]           fp32,  nullable
+ *   count [B][n_q]           int32, nullable
+ *   idx   [B][n_q][idx_cap]  int32, nullable: selected token positions, unspecified order,
+ *                            truncated at idx_cap (SPARK_ERR_OVERFLOW recorded)
+ * Limits: hd <= 256, r % 8 == 0, (hd - r) % 8 == 0, 0 < r < hd, n_q / n_kv <= 8. */
+int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c,
+                      const void* vc, int kvdtype, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd,
+                      int64_t r, int64_t cap, const int32_t* ctx_len, int64_t window, int64_t k_attn,
+                      int flags, float* o, float* theta, int32_t* count, int32_t* idx,
+                      int64_t idx_cap, void* stream);
+
+/* ---- dense GEMV (the projections the method leaves dense: Table "FLOPs per token") ----
+ * y[b][n_out] = Wt[n_out][n_in] . x[b][n_in] (+ y_add[b][n_out] if y_add != NULL).
+ * Wt of dtype wdtype, output-major; n_in % 8 == 0; 1 <= B <= 16.  y_add may equal y. */
+int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const void* Wt, int wdtype,
+                     int64_t n_in, int64_t n_out, const float* y_add, float* y, void* stream);
+
+/* ---- one decoder layer (Section 4) ---------------------------------------------
+ * Pre-norm block around the two operators, for one new token per sequence:
+ *   a = RMSNorm(h; norm1);  [q|k|v] = Wqkv a;  rotary position encoding applied separately to
+ *   q[:r], q[r:], k[:r], k[r:] at position ctx_len[b]-1;  q *= 1/sqrt(hd);
+ *   k, v written to row ctx_len[b]-1 of the caches;  h += Wo . SparkAttention;  h += SparkFFN(RMSNorm(h; norm2)).
+ * All pointers inside the structs are device pointers; the structs themselves are host objects. */
+typedef struct spark_layer_weights {
+    const float* norm1;   /* [d]                          */
+    const float* norm2;   /* [d]                          */
+    const void* Wqkv;     /* [(n_q + 2 n_kv) hd][d] bf16  */
+    const void* Wo;       /* [d][n_q hd]            bf16  */
+    const void* K1t;      /* [d_ff][r_ff]           bf16  */
+    const void* K2t;      /* [d_ff][d - r_ff]       bf16  */
+    const void* Vt;       /* [d_ff][d]              bf16  */
+} spark_layer_weights;
+
+typedef struct spark_layer_cfg {
+    int64_t d, d_ff, r_ff, k_ff;
+    int64_t n_q, n_kv, hd, r_attn, k_attn;
+    int64_t window;       /* 0 = global attention, else the local window length          */
+    int64_t cap;          /* cache capacity in tokens                                     */
+    float rms_eps;        /* e.g. 1e-6                                                    */
+    float rope_base;      /* e.g. 10000                                                   */
+    int flags;            /* SPARK_GELU_* | SPARK_DENSE_LOADS (applies to FFN and attention) */
+} spark_layer_cfg;
+
+typedef struct spark_kv_cache {
+    void* k1c;            /* [B][n_kv][cap][r_attn]      bf16, row ctx_len[b]-1 is written */
+    void* k2c;            /* [B][n_kv][cap][hd-r_attn]   bf16                              */
+    void* vc;             /* [B][n_kv][cap][hd]          bf16                              */
+} spark_kv_cache;
+
+/* scratch [B][ (n_q + 2 n_kv) hd + n_q hd + d ] fp32, caller-owned, contents undefined after the call.
+ * h [B][d] fp32 is updated in place.  1 <= B <= 16. */
+int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
+                       const spark_kv_cache* cache, const int32_t* ctx_len, float* h, int64_t B,
+                       float* scratch, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARK_H_ */

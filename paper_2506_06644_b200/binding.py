@@ -1,0 +1,207 @@
+"""ctypes binding of libspark_b200.so: argument marshalling only.
+
+Every function below has the name and the argument order of its C entry point in
+include/spark.h and does nothing but turn torch tensors into device pointers, pass the
+current CUDA stream, and raise on a non-zero status.  torch is used for device memory and
+streams; every step of the computation runs in the library's kernels.  There is no CPU
+fallback: a missing library or a missing GPU is an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspark_b200.so")
+
+SPARK_OK = 0
+SPARK_ERR_INVALID_ARG, SPARK_ERR_UNSUPPORTED, SPARK_ERR_WORKSPACE, SPARK_ERR_CUDA = 1, 2, 3, 4
+SPARK_ERR_TIMEOUT, SPARK_ERR_OVERFLOW = 5, 6
+SPARK_F32, SPARK_BF16 = 0, 1
+SPARK_FILL_ZERO, SPARK_FILL_NEGINF = 0, 1
+SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
+
+EXPORTS = [
+    "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
+    "spark_destroy", "spark_device_status", "spark_grid_size", "spark_stat_topk", "spark_ffn_decode",
+    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode",
+]
+
+
+class SparkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+class _LayerWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("norm1", "norm2", "Wqkv", "Wo", "K1t", "K2t", "Vt")]
+
+
+class _LayerCfg(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("d", "d_ff", "r_ff", "k_ff", "n_q", "n_kv", "hd", "r_attn", "k_attn",
+                                         "window", "cap")] + \
+               [("rms_eps", C.c_float), ("rope_base", C.c_float), ("flags", C.c_int)]
+
+
+class _KvCache(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("k1c", "k2c", "vc")]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the shared library (built in-tree by paper_2506_06644_b200.build); fail loudly if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2506_06644_b200.build` "
+                           "(there is no fallback path)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32, f64 = C.c_void_p, C.c_int64, C.c_int, C.c_double
+    sig = {
+        "spark_status_string": (C.c_char_p, [i32]),
+        "spark_normal_upper_quantile": (f64, [f64]),
+        "spark_workspace_bytes": (C.c_size_t, [i64] * 6),
+        "spark_create": (i32, [C.POINTER(vp), i32, vp, C.c_size_t]),
+        "spark_destroy": (i32, [vp]),
+        "spark_device_status": (i32, [vp, vp, C.POINTER(i32)]),
+        "spark_grid_size": (i32, [vp]),
+        "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
+        "spark_ffn_decode": (i32, [vp, vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
+        "spark_attn_decode": (i32, [vp, vp, vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
+                                    vp, vp, vp, vp, i64, vp]),
+        "spark_dense_gemv": (i32, [vp, vp, i64, vp, i32, i64, i64, vp, vp, vp]),
+        "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
+                                     vp, vp, i64, vp, vp]),
+    }
+    assert sorted(sig) == sorted(EXPORTS)
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name, None)       # a missing symbol surfaces at its first call
+        if fn is not None:
+            fn.restype, fn.argtypes = res, args
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().spark_status_string(status).decode()
+
+
+def spark_normal_upper_quantile(p: float) -> float:
+    return lib().spark_normal_upper_quantile(p)
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensors passed to the library must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _check(status: int, where: str):
+    if status != SPARK_OK:
+        raise SparkError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SPARK_F32
+    if t.dtype == torch.bfloat16:
+        return SPARK_BF16
+    raise ValueError(f"unsupported weight dtype {t.dtype}")
+
+
+def spark_workspace_bytes(max_batch: int, max_dff: int, max_cap: int, n_q: int, hd: int, max_d: int) -> int:
+    return lib().spark_workspace_bytes(max_batch, max_dff, max_cap, n_q, hd, max_d)
+
+
+class SparkContext:
+    """spark_create / spark_destroy around a torch-allocated workspace."""
+
+    def __init__(self, device: int = 0, max_batch: int = 16, max_dff: int = 16384, max_cap: int = 32768,
+                 n_q: int = 16, hd: int = 256, max_d: int = 4096):
+        if not torch.cuda.is_available():
+            raise RuntimeError("the Spark decode library needs a CUDA device (no CPU fallback)")
+        self.device = device
+        nbytes = spark_workspace_bytes(max_batch, max_dff, max_cap, n_q, hd, max_d)
+        with torch.cuda.device(device):
+            self.workspace = torch.zeros(nbytes + 256, dtype=torch.uint8, device=f"cuda:{device}")
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            h = C.c_void_p()
+            _check(lib().spark_create(C.byref(h), device, self._ws_ptr, nbytes), "spark_create")
+        self.handle = h
+
+    def device_status(self) -> int:
+        out = C.c_int(0)
+        _check(lib().spark_device_status(self.handle, _stream(), C.byref(out)), "spark_device_status")
+        return out.value
+
+    @property
+    def grid_size(self) -> int:
+        return lib().spark_grid_size(self.handle)
+
+    def close(self):
+        if self.handle is not None:
+            lib().spark_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def spark_stat_topk(ctx: SparkContext, x, rows, n, ld, k, fill, theta, count, idx, val, idx_cap, y_dense):
+    _check(lib().spark_stat_topk(ctx.handle, _ptr(x), rows, n, ld, k, fill, _ptr(theta), _ptr(count), _ptr(idx),
+                                 _ptr(val), idx_cap, _ptr(y_dense), _stream()), "spark_stat_topk")
+
+
+def spark_ffn_decode(ctx: SparkContext, x, B, K1t, K2t, Vt, wdtype, d, d_ff, r, k, flags, y, theta, count, idx):
+    _check(lib().spark_ffn_decode(ctx.handle, _ptr(x), B, _ptr(K1t), _ptr(K2t), _ptr(Vt), wdtype, d, d_ff, r, k,
+                                  flags, _ptr(y), _ptr(theta), _ptr(count), _ptr(idx), _stream()), "spark_ffn_decode")
+
+
+def spark_attn_decode(ctx: SparkContext, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv, hd, r, cap, ctx_len, window,
+                      k_attn, flags, o, theta, count, idx, idx_cap):
+    _check(lib().spark_attn_decode(ctx.handle, _ptr(q), _ptr(k1c), _ptr(k2c), _ptr(vc), kvdtype, B, n_q, n_kv, hd,
+                                   r, cap, _ptr(ctx_len), window, k_attn, flags, _ptr(o), _ptr(theta), _ptr(count),
+                                   _ptr(idx), idx_cap, _stream()), "spark_attn_decode")
+
+
+def spark_dense_gemv(ctx: SparkContext, x, B, Wt, wdtype, n_in, n_out, y_add, y):
+    _check(lib().spark_dense_gemv(ctx.handle, _ptr(x), B, _ptr(Wt), wdtype, n_in, n_out, _ptr(y_add), _ptr(y),
+                                  _stream()), "spark_dense_gemv")
+
+
+@dataclass
+class LayerHandles:
+    """Host-side structs of spark_layer_decode, built once per layer (they only hold pointers)."""
+    weights: _LayerWeights
+    cfg: _LayerCfg
+    cache: _KvCache
+    keep: tuple            # tensors kept alive
+
+
+def make_layer(weights: dict, cfg: dict, cache: dict) -> LayerHandles:
+    w = _LayerWeights(**{k: _ptr(weights[k]) for k in ("norm1", "norm2", "Wqkv", "Wo", "K1t", "K2t", "Vt")})
+    c = _LayerCfg(**cfg)
+    kv = _KvCache(**{k: _ptr(cache[k]) for k in ("k1c", "k2c", "vc")})
+    return LayerHandles(w, c, kv, (weights, cache))
+
+
+def spark_layer_decode(ctx: SparkContext, layer: LayerHandles, ctx_len, h, B, scratch):
+    _check(lib().spark_layer_decode(ctx.handle, C.byref(layer.weights), C.byref(layer.cfg), C.byref(layer.cache),
+                                    _ptr(ctx_len), _ptr(h), B, _ptr(scratch), _stream()), "spark_layer_decode")

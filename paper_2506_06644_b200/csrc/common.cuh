@@ -1,0 +1,252 @@
+// Shared device/host helpers of the Spark decode library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/spark.h"
+
+namespace spark {
+
+constexpr int kWarp = 32;
+constexpr unsigned kFull = 0xffffffffu;
+
+// ---------------------------------------------------------------------------
+// Context (host object) and workspace header (device)
+// ---------------------------------------------------------------------------
+struct WsHeader {            // lives at the start of the caller's workspace
+    int status;              // device status word (SPARK_OK or a SPARK_ERR_* device code)
+    unsigned bar_count;      // inter-block barrier: arrivals of the current phase
+    unsigned bar_gen;        // inter-block barrier: generation, bumped by the last arriver
+    unsigned pad[61];
+};
+static_assert(sizeof(WsHeader) == 256, "header is one 256-byte line group");
+
+}  // namespace spark
+
+struct spark_ctx {
+    int device;
+    int num_sms;
+    int max_smem_optin;
+    char* ws;                // device workspace base (header first)
+    size_t ws_bytes;
+    spark::WsHeader* hdr;    // == ws
+    char* scratch;           // ws + sizeof(WsHeader)
+    size_t scratch_bytes;
+};
+
+namespace spark {
+
+// ---------------------------------------------------------------------------
+// Loads
+// ---------------------------------------------------------------------------
+// Streaming 16-byte read-only load that does not allocate in L1 (weights and cache rows are
+// touched once per call).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 8 consecutive weights starting at element index `e8*8` of a row, widened to fp32.
+template <typename WT>
+struct Row8;
+
+template <>
+struct Row8<__nv_bfloat16> {
+    uint4 raw;
+    __device__ __forceinline__ void load(const __nv_bfloat16* row, int64_t chunk) {
+        raw = ld_stream16(reinterpret_cast<const uint4*>(row) + chunk);
+    }
+    __device__ __forceinline__ void unpack(float (&f)[8]) const {
+        // bf16 -> fp32 is a 16-bit shift; element 0 sits in the low half of each word
+        f[0] = __uint_as_float(raw.x << 16); f[1] = __uint_as_float(raw.x & 0xffff0000u);
+        f[2] = __uint_as_float(raw.y << 16); f[3] = __uint_as_float(raw.y & 0xffff0000u);
+        f[4] = __uint_as_float(raw.z << 16); f[5] = __uint_as_float(raw.z & 0xffff0000u);
+        f[6] = __uint_as_float(raw.w << 16); f[7] = __uint_as_float(raw.w & 0xffff0000u);
+    }
+};
+
+template <>
+struct Row8<float> {
+    uint4 lo, hi;
+    __device__ __forceinline__ void load(const float* row, int64_t chunk) {
+        lo = ld_stream16(reinterpret_cast<const uint4*>(row) + 2 * chunk);
+        hi = ld_stream16(reinterpret_cast<const uint4*>(row) + 2 * chunk + 1);
+    }
+    __device__ __forceinline__ void unpack(float (&f)[8]) const {
+        f[0] = __uint_as_float(lo.x); f[1] = __uint_as_float(lo.y);
+        f[2] = __uint_as_float(lo.z); f[3] = __uint_as_float(lo.w);
+        f[4] = __uint_as_float(hi.x); f[5] = __uint_as_float(hi.y);
+        f[6] = __uint_as_float(hi.z); f[7] = __uint_as_float(hi.w);
+    }
+};
+
+__device__ __forceinline__ float dot8(const float (&w)[8], const float4& a, const float4& b, float acc) {
+    acc = fmaf(w[0], a.x, acc); acc = fmaf(w[1], a.y, acc);
+    acc = fmaf(w[2], a.z, acc); acc = fmaf(w[3], a.w, acc);
+    acc = fmaf(w[4], b.x, acc); acc = fmaf(w[5], b.y, acc);
+    acc = fmaf(w[6], b.z, acc); acc = fmaf(w[7], b.w, acc);
+    return acc;
+}
+
+// ---------------------------------------------------------------------------
+// Warp reductions
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
+    return v;
+}
+__device__ __forceinline__ int warp_sum_int(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------------------
+// Moments (count, mean, sum of squared deviations) and their pairwise merge
+// ---------------------------------------------------------------------------
+struct Moments {
+    double n, mean, m2;
+};
+__device__ __forceinline__ Moments merge(const Moments& a, const Moments& b) {
+    if (b.n == 0.0) return a;
+    if (a.n == 0.0) return b;
+    Moments o;
+    o.n = a.n + b.n;
+    const double delta = b.mean - a.mean;
+    const double fb = b.n / o.n;
+    o.mean = a.mean + delta * fb;
+    o.m2 = a.m2 + b.m2 + delta * delta * a.n * fb;
+    return o;
+}
+__device__ __forceinline__ Moments warp_merge(Moments m) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Moments other;
+        other.n = __shfl_xor_sync(kFull, m.n, o);
+        other.mean = __shfl_xor_sync(kFull, m.mean, o);
+        other.m2 = __shfl_xor_sync(kFull, m.m2, o);
+        m = merge(m, other);
+    }
+    return m;
+}
+// theta = mean + std * z with the Bessel-corrected std (Eq. 11).
+__device__ __forceinline__ float theta_from(const Moments& m, double z) {
+    const double var = m.n > 1.0 ? m.m2 / (m.n - 1.0) : 0.0;
+    return static_cast<float>(m.mean + sqrt(var) * z);
+}
+
+// ---------------------------------------------------------------------------
+// Activations
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float gelu_tanh(float a) {
+    const float c = 0.7978845608028654f;   // sqrt(2/pi)
+    return 0.5f * a * (1.0f + tanhf(c * (a + 0.044715f * a * a * a)));
+}
+__device__ __forceinline__ float gelu_erf(float a) {
+    return 0.5f * a * (1.0f + erff(a * 0.7071067811865476f));
+}
+__device__ __forceinline__ float softplus(float a) {
+    return fmaxf(a, 0.0f) + log1pf(expf(-fabsf(a)));
+}
+
+// ---------------------------------------------------------------------------
+// Inter-block barrier with a bounded wait
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned atom_add_acqrel_u32(unsigned* p, unsigned v) {
+    unsigned old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// The barrier is split so that independent work can sit between arrival and wait.
+// Every block of a co-resident (cooperative) grid calls arrive once and wait once per phase.
+// Thread 0 of the block does the global traffic; the __syncthreads order the block's other
+// threads around it.  The wait gives up after `limit_ns` and records SPARK_ERR_TIMEOUT.
+struct GridBarrier {
+    WsHeader* hdr;
+    unsigned nblocks;
+    unsigned gen;   // generation observed before arriving (thread 0 only)
+
+    __device__ __forceinline__ void arrive() {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            gen = ld_acquire_u32(&hdr->bar_gen);
+            const unsigned prev = atom_add_acqrel_u32(&hdr->bar_count, 1u);
+            if (prev == nblocks - 1) {
+                hdr->bar_count = 0;                        // ordered before the release below
+                st_release_u32(&hdr->bar_gen, gen + 1);
+            }
+        }
+    }
+    // Returns false if the wait timed out (uniform over the block).
+    __device__ __forceinline__ bool wait(unsigned long long limit_ns = 2000000000ull) {
+        __shared__ int ok_flag;
+        if (threadIdx.x == 0) {
+            int ok = 1;
+            if (ld_acquire_u32(&hdr->bar_gen) == gen) {
+                const unsigned long long t0 = global_ns();
+                while (ld_acquire_u32(&hdr->bar_gen) == gen) {
+                    if (global_ns() - t0 > limit_ns) {
+                        ok = 0;
+                        atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+                        break;
+                    }
+                }
+            }
+            ok_flag = ok;
+        }
+        __syncthreads();
+        const bool ok = ok_flag != 0;
+        __syncthreads();     // ok_flag may be rewritten by the next wait
+        return ok;
+    }
+};
+
+// Vector reduction into global memory: y[0..3] += v (16-byte aligned address).
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
+}
+// Read that bypasses L1 (data written by other SMs earlier in the same kernel).
+__device__ __forceinline__ float4 ld_cg_f4(const float4* p) { return __ldcg(p); }
+
+// ---------------------------------------------------------------------------
+// Host helpers
+// ---------------------------------------------------------------------------
+inline bool on_device(const spark_ctx* ctx) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == ctx->device;
+}
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace spark

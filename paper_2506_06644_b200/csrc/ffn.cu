@@ -1,0 +1,419 @@
+// spark_ffn_decode: Spark FFN (Section 2.1, Eq. 2) for one to a few tokens, one persistent
+// cooperative kernel, one thread block per SM.
+//
+//   phase A  every block streams its contiguous share of K1t once (coalesced 16-byte loads, fp32
+//            accumulate) and forms the predictor scores s = K1^T x[:r] of its neurons;
+//   stats    per-block (count, mean, M2) per token -> workspace; ONE grid-wide barrier (the
+//            threshold of Eq. 11 needs every score); each block merges all partials itself;
+//   phase C  theta, active masks and the union of the tokens' active sets over the block's own
+//            neurons (ballot + prefix-sum compaction in shared memory);
+//   phase D  only the union rows of K2t and Vt are read: a warp per row for t_i = K2[:,i].x[r:],
+//            u_i = GELU(s_i - theta) t_i, then a thread per 8 output columns accumulates
+//            sum_i u_i V[:,i] in registers and adds it to y with vector reductions.
+// Individual masks gate the arithmetic, the union gates the loads (Appendix B).
+#include "kernels.h"
+
+using namespace spark;
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / kWarp;
+constexpr int kRows = 4;          // rows a warp works on at once in phase A
+constexpr int kMaxTB = 16;        // tokens per pass over the weights
+
+struct FfnParams {
+    const float* x;
+    const float* norm_w;
+    float eps;
+    const void* K1t;
+    const void* K2t;
+    const void* Vt;
+    int B, d, d_ff, r, rpc, xw;
+    int dense, erf_form, identity;
+    double z;
+    const float* y_init;
+    float* y;
+    float* theta;
+    int32_t* count;
+    int32_t* idx;
+    float4* stats;                // [2][TB][grid] per-block moments
+    WsHeader* hdr;
+};
+
+template <typename WT, int TB>
+__global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* xs = reinterpret_cast<float*>(smem_raw);                 // [TB][xw]
+    float* s_loc = xs + static_cast<size_t>(TB) * p.xw;             // [TB][rpc]
+    float* u_loc = s_loc + static_cast<size_t>(TB) * p.rpc;         // [TB][rpc]
+    int* ulist = reinterpret_cast<int*>(u_loc + static_cast<size_t>(TB) * p.rpc);   // [rpc]
+    unsigned* amask = reinterpret_cast<unsigned*>(ulist + p.rpc);   // [rpc]
+    __shared__ float rstd[kMaxTB];
+    __shared__ float theta_s[kMaxTB];
+    __shared__ int wcnt[kWarps];
+    __shared__ unsigned tok_any;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grid = gridDim.x, cta = blockIdx.x;
+    const int row0 = static_cast<int>(static_cast<int64_t>(cta) * p.d_ff / grid);
+    const int row1 = static_cast<int>(static_cast<int64_t>(cta + 1) * p.d_ff / grid);
+    const int nloc = row1 - row0;
+    const int d = p.d, r = p.r, d2 = d - r, rpc = p.rpc, xw = p.xw;
+    const WT* K1t = static_cast<const WT*>(p.K1t);
+    const WT* K2t = static_cast<const WT*>(p.K2t);
+    const WT* Vt = static_cast<const WT*>(p.Vt);
+    GridBarrier bar{p.hdr, static_cast<unsigned>(grid), 0u};
+
+    for (int g0 = 0, grp = 0; g0 < p.B; g0 += TB, ++grp) {
+        const int tbv = min(TB, p.B - g0);
+        const float* xg = p.x + static_cast<int64_t>(g0) * d;
+        float* yg = p.y + static_cast<int64_t>(g0) * d;
+
+        // ---- prologue: optional RMSNorm scale, y initialisation, x[:r] into shared memory ------
+        for (int t = warp; t < TB; t += kWarps) {
+            float ss = 0.f;
+            if (p.norm_w != nullptr && t < tbv) {
+                const float4* xr = reinterpret_cast<const float4*>(xg + static_cast<int64_t>(t) * d);
+                for (int i = lane; i < d / 4; i += 32) {
+                    const float4 v = xr[i];
+                    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                }
+                ss = warp_sum(ss);
+            }
+            if (lane == 0) rstd[t] = p.norm_w != nullptr ? rsqrtf(ss / static_cast<float>(d) + p.eps) : 1.f;
+        }
+        {
+            const int64_t total4 = static_cast<int64_t>(tbv) * d / 4;
+            const float4* yi = p.y_init ? reinterpret_cast<const float4*>(p.y_init + static_cast<int64_t>(g0) * d) : nullptr;
+            float4* yo = reinterpret_cast<float4*>(yg);
+            for (int64_t i = static_cast<int64_t>(cta) * kThreads + tid; i < total4; i += static_cast<int64_t>(grid) * kThreads)
+                yo[i] = yi ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (cta == 0 && p.count != nullptr && tid < tbv) p.count[g0 + tid] = 0;
+        if (tid == 0) tok_any = 0u;
+        __syncthreads();
+        auto stage = [&](int col0, int width) {     // xs[t][0:width] = x[t][col0:col0+width] (normalised)
+            const int w4 = width / 4;
+            for (int i = tid; i < TB * w4; i += kThreads) {
+                const int t = i / w4, c = i - t * w4;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (t < tbv) {
+                    v = reinterpret_cast<const float4*>(xg + static_cast<int64_t>(t) * d + col0)[c];
+                    if (p.norm_w != nullptr) {
+                        const float4 w = reinterpret_cast<const float4*>(p.norm_w + col0)[c];
+                        const float sc = rstd[t];
+                        v.x *= sc * w.x; v.y *= sc * w.y; v.z *= sc * w.z; v.w *= sc * w.w;
+                    }
+                }
+                reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * xw)[c] = v;
+            }
+        };
+        stage(0, r);
+        __syncthreads();
+
+        // ---- phase A: predictor scores of this block's neurons ----------------------------------
+        {
+            constexpr int TS = TB >= 16 ? 2 : 1;     // lane groups that split the tokens
+            constexpr int TPL = TB / TS;             // tokens per lane group
+            constexpr int GL = 32 / TS;              // lanes per group
+            const int lg = lane / GL, gl = lane % GL;
+            const int nc1 = r / 8;
+            for (int rg = warp; rg * kRows < nloc; rg += kWarps) {
+                float acc[kRows][TPL];
+#pragma unroll
+                for (int i = 0; i < kRows; ++i)
+#pragma unroll
+                    for (int t = 0; t < TPL; ++t) acc[i][t] = 0.f;
+                const WT* rowp[kRows];
+#pragma unroll
+                for (int i = 0; i < kRows; ++i)
+                    rowp[i] = K1t + static_cast<int64_t>(min(row0 + rg * kRows + i, row1 - 1)) * r;
+#pragma unroll(TB == 1 ? 4 : (TB <= 4 ? 2 : 1))
+                for (int c = gl; c < nc1; c += GL) {
+                    Row8<WT> w[kRows];
+#pragma unroll
+                    for (int i = 0; i < kRows; ++i) w[i].load(rowp[i], c);
+                    float wf[kRows][8];
+#pragma unroll
+                    for (int i = 0; i < kRows; ++i) w[i].unpack(wf[i]);
+#pragma unroll
+                    for (int t = 0; t < TPL; ++t) {
+                        const float4* xr = reinterpret_cast<const float4*>(xs + static_cast<size_t>(lg * TPL + t) * xw) + 2 * c;
+                        const float4 xa = xr[0], xb = xr[1];
+#pragma unroll
+                        for (int i = 0; i < kRows; ++i) acc[i][t] = dot8(wf[i], xa, xb, acc[i][t]);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < kRows; ++i)
+#pragma unroll
+                    for (int t = 0; t < TPL; ++t) {
+                        float v = acc[i][t];
+#pragma unroll
+                        for (int o = GL / 2; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+                        if (gl == 0 && rg * kRows + i < nloc) s_loc[static_cast<size_t>(lg * TPL + t) * rpc + rg * kRows + i] = v;
+                    }
+            }
+        }
+        __syncthreads();
+
+        // ---- per-block moments of the scores, one warp per token (two-pass, in registers) ---------
+        float4* stats = p.stats + static_cast<size_t>(grp & 1) * TB * grid;
+        for (int t = warp; t < tbv; t += kWarps) {
+            const float* sr = s_loc + static_cast<size_t>(t) * rpc;
+            float sum = 0.f;
+            for (int j = lane; j < nloc; j += 32) sum += sr[j];
+            sum = warp_sum(sum);
+            const float mean = nloc > 0 ? sum / static_cast<float>(nloc) : 0.f;
+            float m2 = 0.f;
+            for (int j = lane; j < nloc; j += 32) {
+                const float dl = sr[j] - mean;
+                m2 = fmaf(dl, dl, m2);
+            }
+            m2 = warp_sum(m2);
+            if (lane == 0) stats[static_cast<size_t>(t) * grid + cta] = make_float4(static_cast<float>(nloc), mean, m2, 0.f);
+        }
+        bar.arrive();
+        stage(r, d2);                                   // x[r:] replaces x[:r] while the barrier fills
+        if (!bar.wait()) return;
+
+        // ---- theta per token: every block merges all partial moments itself ----------------------
+        for (int t = warp; t < tbv; t += kWarps) {
+            Moments m{0.0, 0.0, 0.0};
+            for (int c = lane; c < grid; c += 32) {
+                const float4 v = ld_cg_f4(&stats[static_cast<size_t>(t) * grid + c]);
+                m = merge(m, Moments{static_cast<double>(v.x), static_cast<double>(v.y), static_cast<double>(v.z)});
+            }
+            m = warp_merge(m);
+            const float th = p.identity ? -INFINITY : theta_from(m, p.z);
+            if (lane == 0) {
+                theta_s[t] = th;
+                if (cta == 0 && p.theta != nullptr) p.theta[g0 + t] = th;
+            }
+        }
+        __syncthreads();
+
+        // ---- phase C: masks and the ordered union list of this block's neurons --------------------
+        int nU = 0;
+        for (int j0 = 0; j0 < nloc; j0 += kThreads) {
+            const int j = j0 + tid;
+            unsigned m = 0u;
+            if (j < nloc) {
+#pragma unroll
+                for (int t = 0; t < TB; ++t)
+                    if (t < tbv && s_loc[static_cast<size_t>(t) * rpc + j] > theta_s[t]) m |= 1u << t;
+                amask[j] = m;
+            }
+            const bool in = j < nloc && (m != 0u || p.dense);
+            const unsigned bal = __ballot_sync(kFull, in);
+            if (lane == 0) wcnt[warp] = __popc(bal);
+            if (m != 0u) atomicOr(&tok_any, m);
+            __syncthreads();
+            int before = 0, all = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                if (w < warp) before += wcnt[w];
+                all += wcnt[w];
+            }
+            if (in) ulist[nU + before + __popc(bal & ((1u << lane) - 1u))] = j;
+            nU += all;
+            __syncthreads();
+        }
+
+        // ---- optional outputs: per-token count and index list --------------------------------------
+        if (p.count != nullptr) {
+            for (int t = warp; t < tbv; t += kWarps) {
+                int c = 0;
+                for (int j = lane; j < nloc; j += 32) c += (amask[j] >> t) & 1u;
+                c = warp_sum_int(c);
+                int base = 0;
+                if (lane == 0 && c > 0) base = atomicAdd(&p.count[g0 + t], c);
+                base = __shfl_sync(kFull, base, 0);
+                if (p.idx != nullptr && c > 0) {
+                    int32_t* out = p.idx + static_cast<int64_t>(g0 + t) * p.d_ff;
+                    for (int j0 = 0; j0 < nloc; j0 += 32) {
+                        const int j = j0 + lane;
+                        const bool a = j < nloc && ((amask[j] >> t) & 1u);
+                        const unsigned bal = __ballot_sync(kFull, a);
+                        if (a) out[base + __popc(bal & ((1u << lane) - 1u))] = row0 + j;
+                        base += __popc(bal);
+                    }
+                }
+            }
+        }
+
+        // ---- phase D1: t_i = K2[:,i] . x[r:] for union rows, u = GELU(s - theta) * t ---------------
+        {
+            const int nc2 = d2 / 8;
+            const unsigned all_tok = tbv >= 32 ? 0xffffffffu : ((1u << tbv) - 1u);
+            for (int ui = warp; ui < nU; ui += kWarps) {
+                const int j = ulist[ui];
+                const unsigned mask = amask[j];
+                const unsigned cm = p.dense ? all_tok : mask;
+                const WT* krow = K2t + static_cast<int64_t>(row0 + j) * d2;
+                float acc[TB];
+#pragma unroll
+                for (int t = 0; t < TB; ++t) acc[t] = 0.f;
+#pragma unroll 4
+                for (int c = lane; c < nc2; c += 32) {
+                    Row8<WT> w;
+                    w.load(krow, c);
+                    float wf[8];
+                    w.unpack(wf);
+#pragma unroll
+                    for (int t = 0; t < TB; ++t) {
+                        if ((cm >> t) & 1u) {
+                            const float4* xr = reinterpret_cast<const float4*>(xs + static_cast<size_t>(t) * xw) + 2 * c;
+                            acc[t] = dot8(wf, xr[0], xr[1], acc[t]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < TB; ++t) {
+                    float u = 0.f;
+                    if ((cm >> t) & 1u) {
+                        const float tv = warp_sum(acc[t]);
+                        if ((mask >> t) & 1u) {
+                            const float a = s_loc[static_cast<size_t>(t) * rpc + j] - (p.identity ? 0.f : theta_s[t]);
+                            u = (p.erf_form ? gelu_erf(a) : gelu_tanh(a)) * tv;
+                        }
+                    }
+                    if (lane == 0) u_loc[static_cast<size_t>(t) * rpc + ui] = u;
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- phase D2: y += sum_i u_i V[:,i]; a thread owns 8 output columns -----------------------
+        {
+            constexpr int TP = TB < 8 ? TB : 8;          // tokens accumulated in registers at once
+            const int ncd = d / 8;
+            const unsigned anyt = tok_any;
+            for (int cc = tid; cc < ncd; cc += kThreads) {
+#pragma unroll 1
+                for (int tp = 0; tp < TB; tp += TP) {
+                    if (tp >= tbv) break;
+                    if (!p.dense && ((anyt >> tp) & ((1u << TP) - 1u)) == 0u) continue;
+                    float acc[TP][8];
+#pragma unroll
+                    for (int t = 0; t < TP; ++t)
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[t][e] = 0.f;
+#pragma unroll 4
+                    for (int ui = 0; ui < nU; ++ui) {
+                        Row8<WT> w;
+                        w.load(Vt + static_cast<int64_t>(row0 + ulist[ui]) * d, cc);
+                        float wf[8];
+                        w.unpack(wf);
+#pragma unroll
+                        for (int t = 0; t < TP; ++t) {
+                            const float u = u_loc[static_cast<size_t>(tp + t) * rpc + ui];
+                            if (u != 0.f || p.dense) {
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) acc[t][e] = fmaf(u, wf[e], acc[t][e]);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < TP; ++t) {
+                        if (tp + t < tbv && ((anyt >> (tp + t)) & 1u)) {
+                            float* dst = yg + static_cast<int64_t>(tp + t) * d + cc * 8;
+                            red_add_v4(dst, acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+                            red_add_v4(dst + 4, acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();      // shared buffers are reused by the next token group
+    }
+}
+
+template <typename WT, int TB>
+int launch_one(spark_ctx* ctx, FfnParams& p, size_t smem, cudaStream_t stream) {
+    static bool configured[64] = {};
+    auto kern = ffn_kernel<WT, TB>;
+    if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        configured[ctx->device] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctx->num_sms));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, p) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+template <typename WT>
+int launch_tb(spark_ctx* ctx, FfnParams& p, int tb, size_t smem, cudaStream_t stream) {
+    switch (tb) {
+        case 1: return launch_one<WT, 1>(ctx, p, smem, stream);
+        case 4: return launch_one<WT, 4>(ctx, p, smem, stream);
+        case 8: return launch_one<WT, 8>(ctx, p, smem, stream);
+        default: return launch_one<WT, 16>(ctx, p, smem, stream);
+    }
+}
+
+}  // namespace
+
+namespace spark {
+
+int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
+    if (ctx == nullptr || a.x == nullptr || a.K1t == nullptr || a.K2t == nullptr || a.Vt == nullptr || a.y == nullptr)
+        return SPARK_ERR_INVALID_ARG;
+    if (a.B < 1 || a.B > 64 || a.d < 16 || a.d_ff < 2 || a.r <= 0 || a.r >= a.d || a.k <= 0) return SPARK_ERR_INVALID_ARG;
+    if (a.idx != nullptr && a.count == nullptr) return SPARK_ERR_INVALID_ARG;
+    if (a.y_init == a.y && a.y_init != nullptr) return SPARK_ERR_INVALID_ARG;
+    if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
+    if ((a.r & 7) != 0 || (a.d & 7) != 0) return SPARK_ERR_UNSUPPORTED;
+    if (!aligned16(a.x) || !aligned16(a.K1t) || !aligned16(a.K2t) || !aligned16(a.Vt) || !aligned16(a.y) ||
+        !aligned16(a.y_init) || !aligned16(a.norm_w))
+        return SPARK_ERR_UNSUPPORTED;
+    if (a.d > (1 << 20) || a.d_ff > (1 << 24)) return SPARK_ERR_UNSUPPORTED;
+    if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
+
+    const int grid = ctx->num_sms;
+    const int tb = a.B == 1 ? 1 : (a.B <= 4 ? 4 : (a.B <= 8 ? 8 : 16));
+    FfnParams p;
+    p.x = a.x; p.norm_w = a.norm_w; p.eps = a.rms_eps;
+    p.K1t = a.K1t; p.K2t = a.K2t; p.Vt = a.Vt;
+    p.B = static_cast<int>(a.B); p.d = static_cast<int>(a.d); p.d_ff = static_cast<int>(a.d_ff); p.r = static_cast<int>(a.r);
+    p.rpc = static_cast<int>((a.d_ff + grid - 1) / grid);
+    p.xw = static_cast<int>(a.r > a.d - a.r ? a.r : a.d - a.r);
+    p.dense = (a.flags & SPARK_DENSE_LOADS) ? 1 : 0;
+    p.erf_form = (a.flags & SPARK_GELU_ERF) ? 1 : 0;
+    p.identity = a.k >= a.d_ff ? 1 : 0;
+    p.z = p.identity ? 0.0 : spark_normal_upper_quantile(static_cast<double>(a.k) / static_cast<double>(a.d_ff));
+    p.y_init = a.y_init; p.y = a.y; p.theta = a.theta; p.count = a.count; p.idx = a.idx;
+    p.hdr = ctx->hdr;
+    const size_t stats_bytes = static_cast<size_t>(2) * kMaxTB * grid * sizeof(float4);
+    if (stats_bytes > ctx->scratch_bytes) return SPARK_ERR_WORKSPACE;
+    p.stats = reinterpret_cast<float4*>(ctx->scratch);
+
+    const size_t smem = (static_cast<size_t>(tb) * p.xw + static_cast<size_t>(2) * tb * p.rpc) * sizeof(float) +
+                        static_cast<size_t>(p.rpc) * 8;
+    if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_UNSUPPORTED;
+    if (a.wdtype == SPARK_BF16) return launch_tb<__nv_bfloat16>(ctx, p, tb, smem, stream);
+    return launch_tb<float>(ctx, p, tb, smem, stream);
+}
+
+}  // namespace spark
+
+extern "C" int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const void* K2t,
+                                const void* Vt, int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k,
+                                int flags, float* y, float* theta, int32_t* count, int32_t* idx, void* stream) {
+    FfnArgs a;
+    a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
+    a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = wdtype;
+    a.B = B; a.d = d; a.d_ff = d_ff; a.r = r; a.k = k; a.flags = flags;
+    a.y_init = nullptr; a.y = y; a.theta = theta; a.count = count; a.idx = idx;
+    return ffn_launch(ctx, a, static_cast<cudaStream_t>(stream));
+}

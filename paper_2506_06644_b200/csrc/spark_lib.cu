@@ -1,0 +1,116 @@
+// Context management, status handling and host-side helpers of the Spark decode library.
+#include <cmath>
+#include <cstdlib>
+#include <limits>
+#include <new>
+
+#include "common.cuh"
+
+using namespace spark;
+
+extern "C" {
+
+const char* spark_status_string(int status) {
+    switch (status) {
+        case SPARK_OK: return "ok";
+        case SPARK_ERR_INVALID_ARG: return "invalid argument";
+        case SPARK_ERR_UNSUPPORTED: return "unsupported layout, dtype or size";
+        case SPARK_ERR_WORKSPACE: return "workspace too small";
+        case SPARK_ERR_CUDA: return "CUDA runtime or launch failure";
+        case SPARK_ERR_TIMEOUT: return "device: bounded inter-block wait ran out";
+        case SPARK_ERR_OVERFLOW: return "device: index list truncated at its capacity";
+        default: return "unknown status";
+    }
+}
+
+// Q(1 - p) of Eq. 11 for the threshold, as the root of 0.5 * erfc(z / sqrt 2) = p.
+// Start from the classical rational approximation for the normal tail (Abramowitz & Stegun
+// 26.2.23, |error| < 4.5e-4) and polish with Newton steps on the tail function, whose derivative
+// is minus the normal density.  The upper-tail form keeps small p free of cancellation.
+double spark_normal_upper_quantile(double p) {
+    if (!(p > 0.0 && p < 1.0)) return std::numeric_limits<double>::quiet_NaN();
+    if (p > 0.5) return -spark_normal_upper_quantile(1.0 - p);
+    const double t = std::sqrt(-2.0 * std::log(p));
+    double z = t - (2.515517 + t * (0.802853 + t * 0.010328)) /
+                       (1.0 + t * (1.432788 + t * (0.189269 + t * 0.001308)));
+    const double inv_sqrt2 = 0.70710678118654752440;
+    const double inv_sqrt2pi = 0.39894228040143267794;
+    for (int it = 0; it < 60; ++it) {
+        const double tail = 0.5 * std::erfc(z * inv_sqrt2);
+        const double dens = inv_sqrt2pi * std::exp(-0.5 * z * z);
+        const double step = (tail - p) / dens;
+        z += step;
+        if (std::fabs(step) <= 1e-16 * std::fmax(1.0, std::fabs(z))) break;
+    }
+    return z;
+}
+
+size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap, int64_t n_q,
+                             int64_t hd, int64_t max_d) {
+    if (max_batch < 1) max_batch = 1;
+    if (max_dff < 0) max_dff = 0;
+    if (max_cap < 0) max_cap = 0;
+    if (n_q < 1) n_q = 1;
+    if (hd < 8) hd = 8;
+    if (max_d < 0) max_d = 0;
+    const size_t grid_bound = 1024;   // more thread blocks than any device has SMs x residency
+    // FFN: per-token, per-block moments (float4).
+    size_t ffn = round_up(static_cast<size_t>(64) * grid_bound * 16, 256);
+    // attention: predictor scores, per-piece moments and partial outputs, per-segment counters.
+    size_t pieces = grid_bound + static_cast<size_t>(max_batch) * n_q;
+    size_t attn = round_up(static_cast<size_t>(max_batch) * n_q * max_cap * 4, 256) +
+                  round_up(pieces * 8 * 16, 256) +
+                  round_up(pieces * 8 * (static_cast<size_t>(hd) + 8) * 4, 256) +
+                  round_up(static_cast<size_t>(max_batch) * n_q * 16, 256);
+    size_t need = ffn > attn ? ffn : attn;
+    (void)max_dff;
+    (void)max_d;
+    return sizeof(WsHeader) + need + 256;
+}
+
+int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_bytes) {
+    if (out == nullptr || workspace == nullptr) return SPARK_ERR_INVALID_ARG;
+    *out = nullptr;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SPARK_ERR_UNSUPPORTED;
+    if (workspace_bytes < sizeof(WsHeader) + 256) return SPARK_ERR_WORKSPACE;
+    if (cudaSetDevice(device) != cudaSuccess) return SPARK_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SPARK_ERR_CUDA;
+    if (cudaMemset(workspace, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;
+    spark_ctx* c = new (std::nothrow) spark_ctx;
+    if (c == nullptr) return SPARK_ERR_INVALID_ARG;
+    c->device = device;
+    c->num_sms = prop.multiProcessorCount;
+    c->max_smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+    c->ws = static_cast<char*>(workspace);
+    c->ws_bytes = workspace_bytes;
+    c->hdr = reinterpret_cast<WsHeader*>(workspace);
+    c->scratch = c->ws + sizeof(WsHeader);
+    c->scratch_bytes = workspace_bytes - sizeof(WsHeader);
+    *out = c;
+    return SPARK_OK;
+}
+
+int spark_destroy(spark_ctx* ctx) {
+    delete ctx;
+    return SPARK_OK;
+}
+
+int spark_grid_size(const spark_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
+
+int spark_device_status(spark_ctx* ctx, void* stream, int* host_out) {
+    if (ctx == nullptr || host_out == nullptr) return SPARK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPARK_ERR_CUDA;
+    int status = 0;
+    if (cudaMemcpy(&status, &ctx->hdr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    *host_out = status;
+    if (status != SPARK_OK) {
+        // a failed phase may have left arrivals behind: start the barrier afresh
+        if (cudaMemset(ctx->hdr, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;
+    }
+    return SPARK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+"""Comparison rules shared by the GPU parity tests.
+
+Tolerances (written here once, used by every test):
+  * theta: |theta_gpu - theta_oracle| <= 1e-5 * max(|theta_oracle|, std_oracle)  (fp32 threshold)
+  * active sets: identical except for entries with |x_i - theta| <= 1e-4 * std
+  * outputs: max|err| <= 2e-2 * RMS(oracle output) for bf16 weights with fp32 accumulation,
+             max|err| <= 1e-5 * RMS(oracle output) for fp32 weights
+"""
+import numpy as np
+
+THETA_RTOL = 1e-5
+BAND = 1e-4
+OUT_TOL = {"bf16": 2e-2, "f32": 1e-5}
+
+
+def rms(a):
+    a = np.asarray(a, dtype=np.float64)
+    return float(np.sqrt(np.mean(a * a))) if a.size else 0.0
+
+
+def check_theta(theta_gpu, theta_or, std_or, what=""):
+    theta_gpu, theta_or = float(theta_gpu), float(theta_or)
+    if not np.isfinite(theta_or):
+        assert theta_gpu == theta_or, f"{what}: theta {theta_gpu} vs {theta_or}"
+        return
+    err = abs(theta_gpu - theta_or) / max(abs(theta_or), std_or)
+    assert err <= THETA_RTOL, f"{what}: theta {theta_gpu} vs {theta_or} (rel {err:.2e})"
+
+
+def check_set(idx_gpu, mask_or, scores, theta_or, std_or, what=""):
+    """idx_gpu: iterable of selected positions; mask_or: oracle's boolean mask; scores: fp64 values
+    the oracle thresholded.  Returns the symmetric difference (all of it inside the band)."""
+    got = np.zeros(mask_or.shape[0], dtype=bool)
+    idx_gpu = np.asarray(idx_gpu, dtype=np.int64)
+    assert idx_gpu.size == np.unique(idx_gpu).size, f"{what}: duplicate indices"
+    assert idx_gpu.size == 0 or (idx_gpu.min() >= 0 and idx_gpu.max() < mask_or.shape[0]), f"{what}: index out of range"
+    got[idx_gpu] = True
+    diff = np.flatnonzero(got != mask_or)
+    if diff.size:
+        dist = np.abs(np.asarray(scores, dtype=np.float64)[diff] - theta_or)
+        assert np.all(dist <= BAND * std_or), \
+            f"{what}: {diff.size} set differences outside the band (worst {dist.max() / std_or:.2e} std)"
+    return diff
+
+
+def check_output(y_gpu, y_or, kind, what=""):
+    y_gpu = np.asarray(y_gpu, dtype=np.float64)
+    y_or = np.asarray(y_or, dtype=np.float64)
+    assert y_gpu.shape == y_or.shape, f"{what}: shape {y_gpu.shape} vs {y_or.shape}"
+    assert np.all(np.isfinite(y_gpu)), f"{what}: non-finite output"
+    scale = rms(y_or)
+    err = float(np.max(np.abs(y_gpu - y_or))) if y_or.size else 0.0
+    tol = OUT_TOL[kind] * scale if scale > 0 else 1e-30
+    assert err <= tol, f"{what}: max|err| {err:.3e} > {OUT_TOL[kind]:g} * RMS {scale:.3e}"
+    return err / scale if scale > 0 else 0.0
