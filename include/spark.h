@@ -129,8 +129,8 @@ int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int
  *   y     [B][d]     fp32 (overwritten)
  *   theta [B]        fp32,  nullable
  *   count [B]        int32, nullable
- *   idx   [B][d_ff]  int32, nullable: active neurons of token b in unspecified order; entries past
- *                    count[b] are not written
+ *   idx   [B][d_ff]  int32, nullable (needs count): active neurons of token b in unspecified order;
+ *                    entries past count[b] are not written
  * Limits: 1 <= B <= 64, 0 < r < d, r % 8 == 0, d % 8 == 0, d_ff >= 2. */
 int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const void* K2t,
                      const void* Vt, int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k,
@@ -148,9 +148,11 @@ int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t,
  *   o     [B][n_q][hd]       fp32 (overwritten)
  *   theta [B][n_q]           fp32,  nullable
  *   count [B][n_q]           int32, nullable
- *   idx   [B][n_q][idx_cap]  int32, nullable: selected token positions, unspecified order,
+ *   idx   [B][n_q][idx_cap]  int32, nullable (needs count): selected token positions, unspecified order,
  *                            truncated at idx_cap (SPARK_ERR_OVERFLOW recorded)
- * Limits: hd <= 256, r % 8 == 0, (hd - r) % 8 == 0, 0 < r < hd, n_q / n_kv <= 8. */
+ * ctx_len values outside [1, cap] are clamped into it.
+ * Limits: hd <= 256, r and hd - r multiples of 8 and at most 128, n_q / n_kv in {1, 2, 4, 8},
+ * B * n_kv <= 2048. */
 int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c,
                       const void* vc, int kvdtype, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd,
                       int64_t r, int64_t cap, const int32_t* ctx_len, int64_t window, int64_t k_attn,
@@ -195,8 +197,9 @@ typedef struct spark_kv_cache {
     void* vc;             /* [B][n_kv][cap][hd]          bf16                              */
 } spark_kv_cache;
 
-/* scratch [B][ (n_q + 2 n_kv) hd + n_q hd + d ] fp32, caller-owned, contents undefined after the call.
- * h [B][d] fp32 is updated in place.  1 <= B <= 16. */
+/* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d) fp32 values, 16-byte aligned, caller-owned, contents
+ * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 16.  Five kernels are
+ * enqueued: QKV projection, position encoding + cache append, attention, output projection, FFN. */
 int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
                        const spark_kv_cache* cache, const int32_t* ctx_len, float* h, int64_t B,
                        float* scratch, void* stream);

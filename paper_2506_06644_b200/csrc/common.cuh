@@ -15,13 +15,16 @@ constexpr unsigned kFull = 0xffffffffu;
 // ---------------------------------------------------------------------------
 // Context (host object) and workspace header (device)
 // ---------------------------------------------------------------------------
-struct WsHeader {            // lives at the start of the caller's workspace
+constexpr int kMaxSegments = 2048;   // (sequence, KV head) pairs one attention call may cover
+
+struct WsHeader {            // lives at the start of the caller's workspace; zero when idle
     int status;              // device status word (SPARK_OK or a SPARK_ERR_* device code)
     unsigned bar_count;      // inter-block barrier: arrivals of the current phase
     unsigned bar_gen;        // inter-block barrier: generation, bumped by the last arriver
     unsigned pad[61];
+    unsigned seg_done[kMaxSegments];   // attention: finished pieces per segment (self-resetting)
 };
-static_assert(sizeof(WsHeader) == 256, "header is one 256-byte line group");
+static_assert(sizeof(WsHeader) == 256 + 4 * kMaxSegments, "header layout");
 
 }  // namespace spark
 
@@ -51,7 +54,16 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
     return v;
 }
 
-// 8 consecutive weights starting at element index `e8*8` of a row, widened to fp32.
+// Same, but pinned in program order (used to issue loads ahead of a block-wide sync).
+__device__ __forceinline__ uint4 ld_stream16_pinned(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// 8 consecutive weights starting at element index `chunk*8` of a row, widened to fp32.
 template <typename WT>
 struct Row8;
 
@@ -61,6 +73,10 @@ struct Row8<__nv_bfloat16> {
     __device__ __forceinline__ void load(const __nv_bfloat16* row, int64_t chunk) {
         raw = ld_stream16(reinterpret_cast<const uint4*>(row) + chunk);
     }
+    __device__ __forceinline__ void load_pinned(const __nv_bfloat16* row, int64_t chunk) {
+        raw = ld_stream16_pinned(reinterpret_cast<const uint4*>(row) + chunk);
+    }
+    __device__ __forceinline__ void zero() { raw = make_uint4(0u, 0u, 0u, 0u); }
     __device__ __forceinline__ void unpack(float (&f)[8]) const {
         // bf16 -> fp32 is a 16-bit shift; element 0 sits in the low half of each word
         f[0] = __uint_as_float(raw.x << 16); f[1] = __uint_as_float(raw.x & 0xffff0000u);
@@ -77,6 +93,11 @@ struct Row8<float> {
         lo = ld_stream16(reinterpret_cast<const uint4*>(row) + 2 * chunk);
         hi = ld_stream16(reinterpret_cast<const uint4*>(row) + 2 * chunk + 1);
     }
+    __device__ __forceinline__ void load_pinned(const float* row, int64_t chunk) {
+        lo = ld_stream16_pinned(reinterpret_cast<const uint4*>(row) + 2 * chunk);
+        hi = ld_stream16_pinned(reinterpret_cast<const uint4*>(row) + 2 * chunk + 1);
+    }
+    __device__ __forceinline__ void zero() { lo = make_uint4(0u, 0u, 0u, 0u); hi = lo; }
     __device__ __forceinline__ void unpack(float (&f)[8]) const {
         f[0] = __uint_as_float(lo.x); f[1] = __uint_as_float(lo.y);
         f[2] = __uint_as_float(lo.z); f[3] = __uint_as_float(lo.w);

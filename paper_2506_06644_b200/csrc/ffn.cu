@@ -12,6 +12,7 @@
 //            sum_i u_i V[:,i] in registers and adds it to y with vector reductions.
 // Individual masks gate the arithmetic, the union gates the loads (Appendix B).
 #include "kernels.h"
+#include "rowdot.cuh"
 
 using namespace spark;
 
@@ -113,49 +114,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
         __syncthreads();
 
         // ---- phase A: predictor scores of this block's neurons ----------------------------------
-        {
-            constexpr int TS = TB >= 16 ? 2 : 1;     // lane groups that split the tokens
-            constexpr int TPL = TB / TS;             // tokens per lane group
-            constexpr int GL = 32 / TS;              // lanes per group
-            const int lg = lane / GL, gl = lane % GL;
-            const int nc1 = r / 8;
-            for (int rg = warp; rg * kRows < nloc; rg += kWarps) {
-                float acc[kRows][TPL];
-#pragma unroll
-                for (int i = 0; i < kRows; ++i)
-#pragma unroll
-                    for (int t = 0; t < TPL; ++t) acc[i][t] = 0.f;
-                const WT* rowp[kRows];
-#pragma unroll
-                for (int i = 0; i < kRows; ++i)
-                    rowp[i] = K1t + static_cast<int64_t>(min(row0 + rg * kRows + i, row1 - 1)) * r;
-#pragma unroll(TB == 1 ? 4 : (TB <= 4 ? 2 : 1))
-                for (int c = gl; c < nc1; c += GL) {
-                    Row8<WT> w[kRows];
-#pragma unroll
-                    for (int i = 0; i < kRows; ++i) w[i].load(rowp[i], c);
-                    float wf[kRows][8];
-#pragma unroll
-                    for (int i = 0; i < kRows; ++i) w[i].unpack(wf[i]);
-#pragma unroll
-                    for (int t = 0; t < TPL; ++t) {
-                        const float4* xr = reinterpret_cast<const float4*>(xs + static_cast<size_t>(lg * TPL + t) * xw) + 2 * c;
-                        const float4 xa = xr[0], xb = xr[1];
-#pragma unroll
-                        for (int i = 0; i < kRows; ++i) acc[i][t] = dot8(wf[i], xa, xb, acc[i][t]);
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < kRows; ++i)
-#pragma unroll
-                    for (int t = 0; t < TPL; ++t) {
-                        float v = acc[i][t];
-#pragma unroll
-                        for (int o = GL / 2; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-                        if (gl == 0 && rg * kRows + i < nloc) s_loc[static_cast<size_t>(lg * TPL + t) * rpc + rg * kRows + i] = v;
-                    }
-            }
-        }
+        rows_dot<WT, TB, kRows>(K1t, r, row0, nloc, r / 8, xs, xw, [&](int j, int t, float v) {
+            s_loc[static_cast<size_t>(t) * rpc + j] = v;
+        });
         __syncthreads();
 
         // ---- per-block moments of the scores, one warp per token (two-pass, in registers) ---------
@@ -243,54 +204,96 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
             }
         }
 
-        // ---- phase D1: t_i = K2[:,i] . x[r:] for union rows, u = GELU(s - theta) * t ---------------
+        // ---- phase D: only the union rows of K2t and Vt are read -------------------------------------
+        constexpr int RB = 8;                            // union rows a thread holds in flight
+        const int ncd = d / 8;
+        // The first batch of V rows is requested before the K2 dot products so that both gathers
+        // share one trip to HBM; a thread owns 8 output columns.
+        constexpr bool PRE = TB <= 4;                    // larger token groups need the registers
+        Row8<WT> vpre[PRE ? RB : 1];
+#pragma unroll
+        for (int j = 0; j < (PRE ? RB : 1); ++j) {
+            if (PRE && j < nU && tid < ncd) vpre[j].load_pinned(Vt + static_cast<int64_t>(row0 + ulist[j]) * d, tid);
+            else vpre[j].zero();
+        }
+        // ---- D1: t_i = K2[:,i] . x[r:] for union rows (a warp takes one or two rows at a time),
+        //          u = GELU(s - theta) * t
         {
+            constexpr int KU = sizeof(WT) == 4 ? 4 : 8;  // chunks per lane per batch
             const int nc2 = d2 / 8;
-            const unsigned all_tok = tbv >= 32 ? 0xffffffffu : ((1u << tbv) - 1u);
-            for (int ui = warp; ui < nU; ui += kWarps) {
-                const int j = ulist[ui];
-                const unsigned mask = amask[j];
-                const unsigned cm = p.dense ? all_tok : mask;
-                const WT* krow = K2t + static_cast<int64_t>(row0 + j) * d2;
-                float acc[TB];
+            const unsigned all_tok = (1u << tbv) - 1u;
+            constexpr int RR = TB >= 8 ? 1 : 2;          // rows a warp takes at a time
+            for (int ui0 = warp * RR; ui0 < nU; ui0 += kWarps * RR) {
+                int jj[RR];
+                unsigned mask[RR], cm[RR];
+                const WT* krow[RR];
 #pragma unroll
-                for (int t = 0; t < TB; ++t) acc[t] = 0.f;
-#pragma unroll 4
-                for (int c = lane; c < nc2; c += 32) {
-                    Row8<WT> w;
-                    w.load(krow, c);
-                    float wf[8];
-                    w.unpack(wf);
+                for (int rr = 0; rr < RR; ++rr) {
+                    const bool ok = ui0 + rr < nU;
+                    jj[rr] = ulist[ok ? ui0 + rr : ui0];
+                    mask[rr] = ok ? amask[jj[rr]] : 0u;
+                    cm[rr] = ok ? (p.dense ? all_tok : mask[rr]) : 0u;
+                    krow[rr] = K2t + static_cast<int64_t>(row0 + jj[rr]) * d2;
+                }
+                float acc[RR][TB];
 #pragma unroll
-                    for (int t = 0; t < TB; ++t) {
-                        if ((cm >> t) & 1u) {
-                            const float4* xr = reinterpret_cast<const float4*>(xs + static_cast<size_t>(t) * xw) + 2 * c;
-                            acc[t] = dot8(wf, xr[0], xr[1], acc[t]);
+                for (int rr = 0; rr < RR; ++rr)
+#pragma unroll
+                    for (int t = 0; t < TB; ++t) acc[rr][t] = 0.f;
+                for (int c0 = 0; c0 < nc2; c0 += 32 * KU) {
+                    Row8<WT> w[RR][KU];
+#pragma unroll
+                    for (int rr = 0; rr < RR; ++rr)
+#pragma unroll
+                        for (int u = 0; u < KU; ++u) {
+                            const int c = c0 + u * 32 + lane;
+                            if (c < nc2 && cm[rr] != 0u) w[rr][u].load(krow[rr], c);
+                            else w[rr][u].zero();
+                        }
+#pragma unroll
+                    for (int u = 0; u < KU; ++u) {
+                        const int c = c0 + u * 32 + lane;
+                        const int cs = c < nc2 ? c : 0;
+#pragma unroll
+                        for (int rr = 0; rr < RR; ++rr) {
+                            float wf[8];
+                            w[rr][u].unpack(wf);
+#pragma unroll
+                            for (int t = 0; t < TB; ++t) {
+                                if ((cm[rr] >> t) & 1u) {
+                                    const float4* xr = reinterpret_cast<const float4*>(xs + static_cast<size_t>(t) * xw) + 2 * cs;
+                                    acc[rr][t] = dot8(wf, xr[0], xr[1], acc[rr][t]);
+                                }
+                            }
                         }
                     }
                 }
 #pragma unroll
-                for (int t = 0; t < TB; ++t) {
-                    float u = 0.f;
-                    if ((cm >> t) & 1u) {
-                        const float tv = warp_sum(acc[t]);
-                        if ((mask >> t) & 1u) {
-                            const float a = s_loc[static_cast<size_t>(t) * rpc + j] - (p.identity ? 0.f : theta_s[t]);
-                            u = (p.erf_form ? gelu_erf(a) : gelu_tanh(a)) * tv;
+                for (int rr = 0; rr < RR; ++rr) {
+                    if (ui0 + rr >= nU) break;
+#pragma unroll
+                    for (int t = 0; t < TB; ++t) {
+                        float u = 0.f;
+                        if ((cm[rr] >> t) & 1u) {
+                            const float tv = warp_sum(acc[rr][t]);
+                            if ((mask[rr] >> t) & 1u) {
+                                const float a = s_loc[static_cast<size_t>(t) * rpc + jj[rr]] - (p.identity ? 0.f : theta_s[t]);
+                                u = (p.erf_form ? gelu_erf(a) : gelu_tanh(a)) * tv;
+                            }
                         }
+                        if (lane == 0) u_loc[static_cast<size_t>(t) * rpc + ui0 + rr] = u;
                     }
-                    if (lane == 0) u_loc[static_cast<size_t>(t) * rpc + ui] = u;
                 }
             }
         }
         __syncthreads();
 
-        // ---- phase D2: y += sum_i u_i V[:,i]; a thread owns 8 output columns -----------------------
+        // ---- D2: y += sum_i u_i V[:,i]; per-thread register accumulators, vector reductions to y -----
         {
             constexpr int TP = TB < 8 ? TB : 8;          // tokens accumulated in registers at once
-            const int ncd = d / 8;
             const unsigned anyt = tok_any;
-            for (int cc = tid; cc < ncd; cc += kThreads) {
+            for (int cb = 0; cb * kThreads < ncd; ++cb) {
+                const int cc = cb * kThreads + tid;
 #pragma unroll 1
                 for (int tp = 0; tp < TB; tp += TP) {
                     if (tp >= tbv) break;
@@ -300,27 +303,42 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
                     for (int t = 0; t < TP; ++t)
 #pragma unroll
                         for (int e = 0; e < 8; ++e) acc[t][e] = 0.f;
-#pragma unroll 4
-                    for (int ui = 0; ui < nU; ++ui) {
-                        Row8<WT> w;
-                        w.load(Vt + static_cast<int64_t>(row0 + ulist[ui]) * d, cc);
-                        float wf[8];
-                        w.unpack(wf);
+                    for (int ub = 0; ub < nU; ub += RB) {
+                        Row8<WT> w[RB];
+                        if (PRE && cb == 0 && tp == 0 && ub == 0) {
 #pragma unroll
-                        for (int t = 0; t < TP; ++t) {
-                            const float u = u_loc[static_cast<size_t>(tp + t) * rpc + ui];
-                            if (u != 0.f || p.dense) {
+                            for (int j = 0; j < RB; ++j) w[j] = vpre[PRE ? j : 0];
+                        } else {
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) acc[t][e] = fmaf(u, wf[e], acc[t][e]);
+                            for (int j = 0; j < RB; ++j) {
+                                if (ub + j < nU && cc < ncd) w[j].load(Vt + static_cast<int64_t>(row0 + ulist[ub + j]) * d, cc);
+                                else w[j].zero();
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < RB; ++j) {
+                            if (ub + j < nU) {
+                                float wf[8];
+                                w[j].unpack(wf);
+#pragma unroll
+                                for (int t = 0; t < TP; ++t) {
+                                    const float u = u_loc[static_cast<size_t>(tp + t) * rpc + ub + j];
+                                    if (u != 0.f || p.dense) {
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) acc[t][e] = fmaf(u, wf[e], acc[t][e]);
+                                    }
+                                }
                             }
                         }
                     }
+                    if (cc < ncd) {
 #pragma unroll
-                    for (int t = 0; t < TP; ++t) {
-                        if (tp + t < tbv && ((anyt >> (tp + t)) & 1u)) {
-                            float* dst = yg + static_cast<int64_t>(tp + t) * d + cc * 8;
-                            red_add_v4(dst, acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
-                            red_add_v4(dst + 4, acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
+                        for (int t = 0; t < TP; ++t) {
+                            if (tp + t < tbv && ((anyt >> (tp + t)) & 1u)) {
+                                float* dst = yg + static_cast<int64_t>(tp + t) * d + cc * 8;
+                                red_add_v4(dst, acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+                                red_add_v4(dst + 4, acc[t][4], acc[t][5], acc[t][6], acc[t][7]);
+                            }
                         }
                     }
                 }

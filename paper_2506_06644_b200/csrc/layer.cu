@@ -1,0 +1,269 @@
+// Dense glue of a decoder layer (Section 4): GEMV with optional fused RMSNorm / residual, rotary
+// position encoding on each half of q and k with the cache append, and spark_layer_decode, which
+// chains them around Spark attention and Spark FFN.  The projections stay dense: the method does
+// not change them (Table "FLOPs per token").
+#include <cmath>
+
+#include "kernels.h"
+#include "rowdot.cuh"
+
+using namespace spark;
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / kWarp;
+
+struct GemvParams {
+    const float* x;
+    const float* norm_w;
+    float eps;
+    const void* Wt;
+    int B, n_in, n_out;
+    const float* y_add;
+    float* y;
+};
+
+// y[b][o] = Wt[o][:] . xhat[b][:] (+ y_add[b][o]);  xhat = x or RMSNorm(x; norm_w).
+template <typename WT, int TB, int RW>
+__global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
+    extern __shared__ __align__(16) float xs[];       // [TB][n_in]
+    __shared__ float rstd[16];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_in = p.n_in;
+    const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
+    const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
+    const int w4 = n_in / 4;
+    for (int i = tid; i < TB * w4; i += kThreads) {
+        const int t = i / w4, c = i - t * w4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t < p.B) v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
+        reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * n_in)[c] = v;
+    }
+    __syncthreads();
+    if (p.norm_w != nullptr) {
+        for (int t = warp; t < TB; t += kWarps) {
+            float ss = 0.f;
+            for (int i = lane; i < n_in; i += 32) {
+                const float v = xs[static_cast<size_t>(t) * n_in + i];
+                ss = fmaf(v, v, ss);
+            }
+            ss = warp_sum(ss);
+            if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(n_in) + p.eps);
+        }
+        __syncthreads();
+        for (int i = tid; i < TB * n_in; i += kThreads) {
+            const int t = i / n_in, c = i - t * n_in;
+            xs[i] *= rstd[t] * p.norm_w[c];
+        }
+        __syncthreads();
+    }
+    rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in,
+                         [&](int j, int t, float v) {
+                             if (t < p.B) {
+                                 const int64_t o = static_cast<int64_t>(t) * p.n_out + row0 + j;
+                                 p.y[o] = p.y_add != nullptr ? v + p.y_add[o] : v;
+                             }
+                         });
+}
+
+template <typename WT, int TB, int RW>
+int gemv_launch_one(spark_ctx* ctx, GemvParams& p, size_t smem, int grid, cudaStream_t stream) {
+    static bool configured[64] = {};
+    auto kern = gemv_kernel<WT, TB, RW>;
+    if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        configured[ctx->device] = true;
+    }
+    kern<<<grid, kThreads, smem, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+template <typename WT>
+int gemv_dispatch(spark_ctx* ctx, GemvParams& p, int tb, int rw, size_t smem, int grid, cudaStream_t stream) {
+    if (tb == 1) return rw == 1 ? gemv_launch_one<WT, 1, 1>(ctx, p, smem, grid, stream) : gemv_launch_one<WT, 1, 4>(ctx, p, smem, grid, stream);
+    if (tb == 4) return rw == 1 ? gemv_launch_one<WT, 4, 1>(ctx, p, smem, grid, stream) : gemv_launch_one<WT, 4, 4>(ctx, p, smem, grid, stream);
+    return rw == 1 ? gemv_launch_one<WT, 16, 1>(ctx, p, smem, grid, stream) : gemv_launch_one<WT, 16, 4>(ctx, p, smem, grid, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rotary position encoding on each half of q and k, 1/sqrt(hd) on q, cache append (Section 4:
+// the encoding is applied to q[:r], q[r:], and to the columns of K1 and of K2).
+// Part of m dims: pairs (i, i + m/2), pair i turned by pos * base^(-2i/m).
+// ---------------------------------------------------------------------------------------------
+struct RopeParams {
+    const float* qkv;        // [B][(n_q + 2 n_kv) hd]
+    float* q_out;            // [B][n_q][hd]
+    __nv_bfloat16* k1c;
+    __nv_bfloat16* k2c;
+    __nv_bfloat16* vc;
+    const int32_t* ctx_len;
+    int B, n_q, n_kv, hd, r;
+    int64_t cap;
+    float base, q_scale;
+};
+
+__global__ void rope_append_kernel(const RopeParams p) {
+    const int heads = p.n_q + 2 * p.n_kv;
+    const int half_hd = p.hd / 2;
+    const int64_t total = static_cast<int64_t>(p.B) * heads * half_hd;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int pr = static_cast<int>(i % half_hd);
+        const int h = static_cast<int>((i / half_hd) % heads);
+        const int b = static_cast<int>(i / (static_cast<int64_t>(half_hd) * heads));
+        int n = p.ctx_len[b];
+        n = n < 1 ? 1 : (n > p.cap ? static_cast<int>(p.cap) : n);
+        const int pos = n - 1;
+        const float* src = p.qkv + (static_cast<int64_t>(b) * heads + h) * p.hd;
+        if (h >= p.n_q + p.n_kv) {                       // value head: plain copy of two elements
+            const int g = h - p.n_q - p.n_kv;
+            __nv_bfloat16* dst = p.vc + ((static_cast<int64_t>(b) * p.n_kv + g) * p.cap + pos) * p.hd;
+            dst[2 * pr] = __float2bfloat16_rn(src[2 * pr]);
+            dst[2 * pr + 1] = __float2bfloat16_rn(src[2 * pr + 1]);
+            continue;
+        }
+        // pair index inside its part: the first r/2 pairs belong to [0, r), the rest to [r, hd)
+        const int hr = p.r / 2;
+        int part0, m, pi;
+        if (pr < hr) { part0 = 0; m = p.r; pi = pr; }
+        else { part0 = p.r; m = p.hd - p.r; pi = pr - hr; }
+        const int ia = part0 + pi, ib = part0 + pi + m / 2;
+        const double ang = static_cast<double>(pos) * exp2(-2.0 * static_cast<double>(pi) / static_cast<double>(m) * log2(static_cast<double>(p.base)));
+        double sn, cs;
+        sincos(ang, &sn, &cs);
+        const float a = src[ia], bb = src[ib];
+        const float ra = static_cast<float>(a * cs - bb * sn), rb = static_cast<float>(a * sn + bb * cs);
+        if (h < p.n_q) {
+            float* dst = p.q_out + (static_cast<int64_t>(b) * p.n_q + h) * p.hd;
+            dst[ia] = ra * p.q_scale;
+            dst[ib] = rb * p.q_scale;
+        } else {
+            const int g = h - p.n_q;
+            const int64_t rowi = (static_cast<int64_t>(b) * p.n_kv + g) * p.cap + pos;
+            if (part0 == 0) {
+                __nv_bfloat16* dst = p.k1c + rowi * p.r;
+                dst[pi] = __float2bfloat16_rn(ra);
+                dst[pi + m / 2] = __float2bfloat16_rn(rb);
+            } else {
+                __nv_bfloat16* dst = p.k2c + rowi * (p.hd - p.r);
+                dst[pi] = __float2bfloat16_rn(ra);
+                dst[pi + m / 2] = __float2bfloat16_rn(rb);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+namespace spark {
+
+int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
+    if (ctx == nullptr || a.x == nullptr || a.Wt == nullptr || a.y == nullptr) return SPARK_ERR_INVALID_ARG;
+    if (a.B < 1 || a.B > 16 || a.n_in < 8 || a.n_out < 1) return SPARK_ERR_INVALID_ARG;
+    if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
+    if ((a.n_in & 7) != 0 || !aligned16(a.x) || !aligned16(a.Wt) || !aligned16(a.norm_w)) return SPARK_ERR_UNSUPPORTED;
+    if (a.n_out > (1LL << 30) || a.n_in > (1 << 20)) return SPARK_ERR_UNSUPPORTED;
+    if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
+    const size_t limit = static_cast<size_t>(ctx->max_smem_optin - 1024);
+    if (static_cast<size_t>(a.n_in) * 4 > limit) return SPARK_ERR_UNSUPPORTED;
+    // Tokens are processed in sub-batches whose inputs fit in shared memory together.
+    int64_t done = 0;
+    while (done < a.B) {
+        int64_t nb = a.B - done;
+        int tb = nb == 1 ? 1 : (nb <= 4 ? 4 : 16);
+        while (static_cast<size_t>(tb) * a.n_in * 4 > limit) tb = tb == 16 ? 4 : 1;
+        if (nb > tb) nb = tb;
+        const int grid = a.n_out < ctx->num_sms ? static_cast<int>(a.n_out) : ctx->num_sms;
+        const int64_t rows_per_block = (a.n_out + grid - 1) / grid;
+        const int rw = rows_per_block <= kWarps ? 1 : 4;
+        GemvParams p;
+        p.x = a.x + done * a.n_in; p.norm_w = a.norm_w; p.eps = a.rms_eps; p.Wt = a.Wt;
+        p.B = static_cast<int>(nb); p.n_in = static_cast<int>(a.n_in); p.n_out = static_cast<int>(a.n_out);
+        p.y_add = a.y_add ? a.y_add + done * a.n_out : nullptr;
+        p.y = a.y + done * a.n_out;
+        const size_t smem = static_cast<size_t>(tb) * a.n_in * 4;
+        const int st = a.wdtype == SPARK_BF16 ? gemv_dispatch<__nv_bfloat16>(ctx, p, tb, rw, smem, grid, stream)
+                                              : gemv_dispatch<float>(ctx, p, tb, rw, smem, grid, stream);
+        if (st != SPARK_OK) return st;
+        done += nb;
+    }
+    return SPARK_OK;
+}
+
+}  // namespace spark
+
+extern "C" int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const void* Wt, int wdtype, int64_t n_in,
+                                int64_t n_out, const float* y_add, float* y, void* stream) {
+    GemvArgs a;
+    a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f; a.Wt = Wt; a.wdtype = wdtype;
+    a.B = B; a.n_in = n_in; a.n_out = n_out; a.y_add = y_add; a.y = y;
+    return gemv_launch(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
+                                  const spark_kv_cache* cache, const int32_t* ctx_len, float* h, int64_t B,
+                                  float* scratch, void* stream) {
+    if (ctx == nullptr || w == nullptr || cfg == nullptr || cache == nullptr || ctx_len == nullptr || h == nullptr ||
+        scratch == nullptr)
+        return SPARK_ERR_INVALID_ARG;
+    if (B < 1 || B > 16) return SPARK_ERR_INVALID_ARG;
+    if (w->norm1 == nullptr || w->norm2 == nullptr || w->Wqkv == nullptr || w->Wo == nullptr || w->K1t == nullptr ||
+        w->K2t == nullptr || w->Vt == nullptr || cache->k1c == nullptr || cache->k2c == nullptr || cache->vc == nullptr)
+        return SPARK_ERR_INVALID_ARG;
+    if (cfg->hd < 16 || (cfg->hd & 1) || (cfg->r_attn & 1) || ((cfg->hd - cfg->r_attn) & 1) || cfg->n_q < 1 ||
+        cfg->n_kv < 1 || cfg->d < 16)
+        return SPARK_ERR_INVALID_ARG;
+    if (!aligned16(scratch) || !aligned16(h)) return SPARK_ERR_UNSUPPORTED;
+    if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t nqkv = (cfg->n_q + 2 * cfg->n_kv) * cfg->hd, nqo = cfg->n_q * cfg->hd;
+    float* qkv = scratch;                 // [B][nqkv]
+    float* qr = qkv + B * nqkv;           // [B][n_q][hd]  position-encoded, scaled queries
+    float* ao = qr + B * nqo;             // [B][n_q][hd]  attention output
+    float* h2 = ao + B * nqo;             // [B][d]        h + Wo . attention
+
+    // 1. a = RMSNorm(h; norm1); [q|k|v] = Wqkv a
+    GemvArgs g1;
+    g1.x = h; g1.norm_w = w->norm1; g1.rms_eps = cfg->rms_eps; g1.Wt = w->Wqkv; g1.wdtype = SPARK_BF16;
+    g1.B = B; g1.n_in = cfg->d; g1.n_out = nqkv; g1.y_add = nullptr; g1.y = qkv;
+    int rc = gemv_launch(ctx, g1, st);
+    if (rc != SPARK_OK) return rc;
+
+    // 2. rotary encoding per half, query scale, cache append
+    RopeParams rp;
+    rp.qkv = qkv; rp.q_out = qr;
+    rp.k1c = static_cast<__nv_bfloat16*>(cache->k1c); rp.k2c = static_cast<__nv_bfloat16*>(cache->k2c);
+    rp.vc = static_cast<__nv_bfloat16*>(cache->vc);
+    rp.ctx_len = ctx_len; rp.B = static_cast<int>(B); rp.n_q = static_cast<int>(cfg->n_q); rp.n_kv = static_cast<int>(cfg->n_kv);
+    rp.hd = static_cast<int>(cfg->hd); rp.r = static_cast<int>(cfg->r_attn); rp.cap = cfg->cap;
+    rp.base = cfg->rope_base; rp.q_scale = 1.0f / std::sqrt(static_cast<float>(cfg->hd));
+    {
+        const int64_t total = B * (cfg->n_q + 2 * cfg->n_kv) * (cfg->hd / 2);
+        const int blocks = static_cast<int>((total + 255) / 256);
+        rope_append_kernel<<<blocks, 256, 0, st>>>(rp);
+        if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
+    }
+
+    // 3. Spark attention over the cache (the new token included)
+    rc = spark_attn_decode(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd,
+                           cfg->r_attn, cfg->cap, ctx_len, cfg->window, cfg->k_attn, cfg->flags & SPARK_DENSE_LOADS,
+                           ao, nullptr, nullptr, nullptr, 0, stream);
+    if (rc != SPARK_OK) return rc;
+
+    // 4. h2 = h + Wo . attention
+    GemvArgs g2;
+    g2.x = ao; g2.norm_w = nullptr; g2.rms_eps = 0.f; g2.Wt = w->Wo; g2.wdtype = SPARK_BF16;
+    g2.B = B; g2.n_in = nqo; g2.n_out = cfg->d; g2.y_add = h; g2.y = h2;
+    rc = gemv_launch(ctx, g2, st);
+    if (rc != SPARK_OK) return rc;
+
+    // 5. h = h2 + SparkFFN(RMSNorm(h2; norm2))
+    FfnArgs f;
+    f.x = h2; f.norm_w = w->norm2; f.rms_eps = cfg->rms_eps;
+    f.K1t = w->K1t; f.K2t = w->K2t; f.Vt = w->Vt; f.wdtype = SPARK_BF16;
+    f.B = B; f.d = cfg->d; f.d_ff = cfg->d_ff; f.r = cfg->r_ff; f.k = cfg->k_ff; f.flags = cfg->flags;
+    f.y_init = h2; f.y = h; f.theta = nullptr; f.count = nullptr; f.idx = nullptr;
+    return ffn_launch(ctx, f, st);
+}

@@ -1,0 +1,76 @@
+// Streaming "rows times a few vectors" kernel body shared by the Spark FFN predictor and the
+// dense GEMV: out[j][t] = W[row0 + j][:] . xs[t][:] for the nloc rows a block owns.
+#pragma once
+
+#include "common.cuh"
+
+namespace spark {
+
+// W: row-major weights with `ld` elements per row; xs: [TB][xw] fp32 in shared memory holding the
+// first nck*8 elements of every token's input.  A warp works on RW rows at once; every 16-byte
+// load of a batch (CU chunks x RW rows per lane) is issued before the first use so that a block
+// keeps its whole share of the matrix in flight.  With TB >= 16 the two half-warps take eight
+// tokens each.  emit(j, t, value) is called by exactly one lane per (row, token).
+// Must be called by all threads of a 512-thread block.
+template <typename WT, int TB, int RW, typename Emit>
+__device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, int row0, int nloc, int nck,
+                                         const float* xs, int xw, Emit emit) {
+    constexpr int kWarpsPerBlock = 16;
+    constexpr int TS = TB >= 16 ? 2 : 1;     // lane groups that split the tokens
+    constexpr int TPL = TB / TS;             // tokens per lane group
+    constexpr int GL = 32 / TS;              // lanes per group
+    constexpr int CU = (TB == 1 ? (RW >= 4 ? 4 : 8) : 2) / (sizeof(WT) == 4 ? 2 : 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lg = lane / GL, gl = lane % GL;
+    for (int rg = warp; rg * RW < nloc; rg += kWarpsPerBlock) {
+        float acc[RW][TPL];
+#pragma unroll
+        for (int i = 0; i < RW; ++i)
+#pragma unroll
+            for (int t = 0; t < TPL; ++t) acc[i][t] = 0.f;
+        const WT* rowp[RW];
+#pragma unroll
+        for (int i = 0; i < RW; ++i) {
+            const int j = rg * RW + i;
+            rowp[i] = W + static_cast<int64_t>(row0 + (j < nloc ? j : nloc - 1)) * ld;
+        }
+        for (int c0 = 0; c0 < nck; c0 += GL * CU) {
+            Row8<WT> w[CU][RW];
+#pragma unroll
+            for (int u = 0; u < CU; ++u) {
+                const int c = c0 + u * GL + gl;
+#pragma unroll
+                for (int i = 0; i < RW; ++i) {
+                    if (c < nck) w[u][i].load(rowp[i], c);
+                    else w[u][i].zero();
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < CU; ++u) {
+                const int c = c0 + u * GL + gl;
+                const int cs = c < nck ? c : 0;          // zero weights meet a valid x address
+                float wf[RW][8];
+#pragma unroll
+                for (int i = 0; i < RW; ++i) w[u][i].unpack(wf[i]);
+#pragma unroll
+                for (int t = 0; t < TPL; ++t) {
+                    const float4* xr = reinterpret_cast<const float4*>(xs + static_cast<size_t>(lg * TPL + t) * xw) + 2 * cs;
+                    const float4 xa = xr[0], xb = xr[1];
+#pragma unroll
+                    for (int i = 0; i < RW; ++i) acc[i][t] = dot8(wf[i], xa, xb, acc[i][t]);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < RW; ++i)
+#pragma unroll
+            for (int t = 0; t < TPL; ++t) {
+                float v = acc[i][t];
+#pragma unroll
+                for (int o = GL / 2; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+                if (gl == 0 && rg * RW + i < nloc) emit(rg * RW + i, lg * TPL + t, v);
+            }
+    }
+}
+
+}  // namespace spark
