@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the Spark decode hot path on B200.
+
+A step decodes ONE token per sequence through the whole decoder stack: every layer is one
+spark_layer_decode call (RMSNorm + dense QKV projection, rotary encoding + cache append, Spark
+attention with its statistical top-k, output projection, Spark FFN with its statistical top-k).
+Workload (default): Gemma-2-2B shape, 26 layers, bf16 weights and KV caches, context 8192, batch 1,
+random-init weights and synthetic N(0,1) caches (seeded).  The 2.9 GB of weights and 0.9 GB of
+caches are far larger than L2, so every step streams them from HBM.
+
+Prints ONE JSON line (rank 0).  `value` is microseconds per token per layer with all inputs
+resident in HBM; `e2e` is the same through the same C-ABI calls with the token's hidden state
+starting and ending in pinned host memory.  `roofline` is for the dominant kernel (the fused Spark
+FFN kernel): touched bytes (all of K1t plus the active rows of K2t and Vt) over its average
+duration, timed with CUDA events over a loop of the same launches.  `cpu_baseline` times the fp64
+oracle on the host cores on a bounded sample.  `--impl reference` times only that oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from the ncu
+# capture summarised in profiles/ (keyed by shape and batch); None where no capture exists yet.
+NCU_TRAFFIC_BYTES = {}
+
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="spark", choices=["spark", "reference"])
+    ap.add_argument("--shape", default="2b", choices=["2b", "9b", "tiny"])
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--ctx", type=int, default=8192)
+    ap.add_argument("--layers", type=int, default=0, help="0 = the shape's layer count")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense-loads comparator")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    return ap.parse_args()
+
+
+def shape_of(name):
+    from paper_2506_06644_b200 import synth
+    return {"2b": synth.GEMMA2_2B, "9b": synth.GEMMA2_9B, "tiny": synth.TINY}[name]
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for r in self.rows if len(r) >= 6 for i in range(4) if r[2 + i] == "Active"})
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# oracle timing (cpu_baseline and the reference arm)
+# --------------------------------------------------------------------------------------------
+def oracle_sample(shape, ctx_len, n_layers, seed=0):
+    """Host inputs for `n_layers` layers of one token at context ctx_len (bf16-rounded values)."""
+    from paper_2506_06644_b200 import synth
+    layers = []
+    for l in range(n_layers):
+        lw = synth.layer_weights(shape, seed, l)
+        W = {"norm1": lw.norm1, "norm2": lw.norm2, "Wqkv": synth.bf16_bits_to_f32(lw.Wqkv_bits),
+             "Wo": synth.bf16_bits_to_f32(lw.Wo_bits), "K1t": synth.bf16_bits_to_f32(lw.K1t_bits),
+             "K2t": synth.bf16_bits_to_f32(lw.K2t_bits), "Vt": synth.bf16_bits_to_f32(lw.Vt_bits)}
+        kv = synth.attn_inputs(1, shape.n_q, shape.n_kv, shape.hd, shape.r_attn, ctx_len, [ctx_len], "bf16",
+                               seed=seed + 1000 + l)
+        kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+        layers.append((W, kc, kv.vc[0].astype(np.float64)))
+    h = synth.normal_f32((shape.d,), seed, 60).astype(np.float64)
+    return layers, h
+
+
+def oracle_run(shape, layers, h, ctx_len):
+    from oracle import spark_oracle as O
+    for W, kc, vc in layers:
+        h = O.decoder_layer(h, W, kc, vc, ctx_len, n_q=shape.n_q, n_kv=shape.n_kv, hd=shape.hd,
+                            r_attn=shape.r_attn, k_attn=shape.k_attn, r_ff=shape.r_ff, k_ff=shape.k_ff)["h"]
+    return h
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        n = 1
+    try:
+        return min(n, len(os.sched_getaffinity(0)))
+    except Exception:
+        return n
+
+
+def run_reference(args):
+    """The oracle as it stands on the host cores: each step is one layer of one token."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape = shape_of(args.shape)
+    layers, h = oracle_sample(shape, args.ctx, 1)
+    for _ in range(max(args.warmup, 1)):
+        oracle_run(shape, layers, h, args.ctx)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_run(shape, layers, h, args.ctx)
+    dt = time.perf_counter() - t0
+    us = dt / args.steps * 1e6
+    cores = host_threads()
+    line = {
+        "impl": "reference", "metric": "us_per_token_per_layer", "value": us, "unit": "us/token/layer",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args, shape), "sample": "one layer of one token per step"},
+        "cpu_baseline": {"value": us, "unit": "us/token/layer", "cores": cores, "kind": "oracle",
+                         "sample": f"{args.steps} steps of one decoder layer for one token at context {args.ctx}"},
+        "e2e": {"value": us, "unit": "us/token/layer", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(args, shape):
+    n_layers = args.layers or shape.n_layers
+    return (f"gemma2-{args.shape}-shape spark decoder: {n_layers} layers x spark_layer_decode, "
+            f"ctx {args.ctx}, batch {args.batch}, bf16 weights+cache")
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------
+def run_spark(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2506_06644_b200 import binding as S
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    shape = shape_of(args.shape)
+    n_layers = args.layers or shape.n_layers
+    B, ctx_len, d, hd = args.batch, args.ctx, shape.d, shape.hd
+    cap = ctx_len
+    ctx = S.SparkContext(local, max_batch=B, max_dff=shape.d_ff, max_cap=cap, n_q=shape.n_q, hd=hd, max_d=d)
+
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1234 + rank)
+
+    def randw(rows, cols, fan_in):
+        return (torch.randn(rows, cols, device=dev, generator=gen) * (fan_in ** -0.5)).to(torch.bfloat16)
+
+    nqkv = (shape.n_q + 2 * shape.n_kv) * hd
+    layers, keep = [], []
+    for l in range(n_layers):
+        w = dict(norm1=1.0 + 0.1 * torch.randn(d, device=dev, generator=gen),
+                 norm2=1.0 + 0.1 * torch.randn(d, device=dev, generator=gen),
+                 Wqkv=randw(nqkv, d, d), Wo=randw(d, shape.n_q * hd, shape.n_q * hd),
+                 K1t=randw(shape.d_ff, shape.r_ff, d), K2t=randw(shape.d_ff, d - shape.r_ff, d),
+                 Vt=randw(shape.d_ff, d, d))
+        cache = dict(k1c=torch.randn(B, shape.n_kv, cap, shape.r_attn, device=dev, generator=gen).to(torch.bfloat16),
+                     k2c=torch.randn(B, shape.n_kv, cap, hd - shape.r_attn, device=dev, generator=gen).to(torch.bfloat16),
+                     vc=torch.randn(B, shape.n_kv, cap, hd, device=dev, generator=gen).to(torch.bfloat16))
+        window = 4096 if (l % 2 == 0 and ctx_len > 4096) else 0      # local / global layers alternate
+        cfg = dict(d=d, d_ff=shape.d_ff, r_ff=shape.r_ff, k_ff=shape.k_ff, n_q=shape.n_q, n_kv=shape.n_kv, hd=hd,
+                   r_attn=shape.r_attn, k_attn=shape.k_attn, window=window, cap=cap, rms_eps=1e-6,
+                   rope_base=10000.0, flags=0)
+        cfg_dense = dict(cfg, flags=S.SPARK_DENSE_LOADS)
+        layers.append((S.make_layer(w, cfg, cache), S.make_layer(w, cfg_dense, cache), w))
+    h_init = torch.randn(B, d, device=dev, generator=gen)
+    h = torch.empty_like(h_init)
+    cl = torch.full((B,), ctx_len, dtype=torch.int32, device=dev)
+    scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d), device=dev)
+    h_host_in = h_init.cpu().pin_memory()
+    h_host_out = torch.empty_like(h_host_in).pin_memory()
+    kernels_per_layer = 5
+
+    def step(which=0):
+        h.copy_(h_init)                                   # device-to-device copy of the token's input
+        for lay in layers:
+            S.spark_layer_decode(ctx, lay[which], cl, h, B, scratch)
+
+    def step_e2e():
+        h.copy_(h_host_in, non_blocking=True)             # pinned host -> device
+        for lay in layers:
+            S.spark_layer_decode(ctx, lay[0], cl, h, B, scratch)
+        h_host_out.copy_(h, non_blocking=True)            # device -> pinned host
+        torch.cuda.current_stream().synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    W = max(args.warmup, 3)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_total = timed(step, args.steps, W)
+    clocks = sampler.stop()
+    ms_e2e = timed(step_e2e, args.steps, W)
+    ms_dense = None if args.no_dense else timed(lambda: step(1), args.steps, W)
+    status = ctx.device_status()
+    assert status == S.SPARK_OK, f"device status {status}"
+    assert torch.isfinite(h).all()
+
+    # ---- roofline of the dominant kernel: the fused FFN kernel on the same weights ----------------
+    xn = torch.nn.functional.normalize(h_init, dim=1) * (d ** 0.5)
+    y = torch.empty_like(xn)
+    cnt = torch.zeros(B, dtype=torch.int32, device=dev)
+    idx = torch.zeros(B, shape.d_ff, dtype=torch.int32, device=dev)
+    unions = []
+    for lay in layers[: min(4, n_layers)]:
+        w = lay[2]
+        S.spark_ffn_decode(ctx, xn, B, w["K1t"], w["K2t"], w["Vt"], S.SPARK_BF16, d, shape.d_ff, shape.r_ff,
+                           shape.k_ff, 0, y, None, cnt, idx)
+        torch.cuda.synchronize()
+        ids = torch.cat([idx[b, : int(cnt[b])] for b in range(B)])
+        unions.append(int(torch.unique(ids).numel()))
+    union = float(np.mean(unions))
+
+    def ffn_loop():
+        for lay in layers:
+            w = lay[2]
+            S.spark_ffn_decode(ctx, xn, B, w["K1t"], w["K2t"], w["Vt"], S.SPARK_BF16, d, shape.d_ff, shape.r_ff,
+                               shape.k_ff, 0, y, None, None, None)
+
+    ms_ffn = timed(ffn_loop, args.steps, W)
+    ffn_us = ms_ffn * 1e3 / (args.steps * n_layers)
+    touched = shape.d_ff * shape.r_ff * 2 + union * (2 * d - shape.r_ff) * 2       # bytes per launch
+    peak, peak_kind = measured_peak()
+    achieved = touched / (ffn_us * 1e-6) / 1e9
+    traffic = NCU_TRAFFIC_BYTES.get((args.shape, B))
+
+    line = None
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        us_tl = ms_step * 1e3 / (n_layers * B * world)
+        layer_touched = touched_layer_bytes(shape, B, ctx_len, union, n_layers)
+        line = {
+            "metric": "us_per_token_per_layer", "value": us_tl, "unit": "us/token/layer", "n_gpus": world,
+            "steps": args.steps, "warmup": W, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 weights/cache, f32 accumulate", "data": "synthetic",
+            "config": {"workload": workload_name(args, shape), "l2": "weights+caches (>3 GB) exceed L2; no flush needed",
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "local_window": 4096, "k_ff": shape.k_ff, "k_attn": shape.k_attn},
+            "tokens_per_s": B * world * args.steps / (ms_total * 1e-3),
+            "layer_touched_mb": layer_touched / 1e6,
+            "layer_gbs_touched": layer_touched / (ms_step * 1e-3 / n_layers) / 1e9,
+            "layer_frac_of_8tbs": layer_touched / (ms_step * 1e-3 / n_layers) / 8e12,
+            "dense": None if ms_dense is None else {
+                "us_per_token_per_layer": ms_dense / args.steps * 1e3 / (n_layers * B * world),
+                "speedup_spark_vs_dense": ms_dense / ms_total},
+            "e2e": {"value": ms_e2e / args.steps * 1e3 / (n_layers * B * world), "unit": "us/token/layer",
+                    "h2d_bytes_per_step": int(h_host_in.numel() * 4), "d2h_bytes_per_step": int(h_host_out.numel() * 4)},
+            "gpu_launches": args.steps * n_layers * kernels_per_layer,
+            "clocks": clocks,
+            "roofline": {"kernel": "ffn_kernel (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                         "us_per_launch": ffn_us, "touched_bytes_per_launch": touched, "union_rows": union},
+        }
+        if not args.no_cpu and world == 1:
+            line["cpu_baseline"] = cpu_baseline(args, shape)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line), flush=True)
+
+
+def touched_layer_bytes(shape, B, ctx_len, union_ffn, n_layers):
+    """Algorithmic bytes of one layer: dense projections, full predictor slices, active rows."""
+    d, hd = shape.d, shape.hd
+    proj = ((shape.n_q + 2 * shape.n_kv) * hd * d + d * shape.n_q * hd) * 2
+    ffn = shape.d_ff * shape.r_ff * 2 + union_ffn * (2 * d - shape.r_ff) * 2
+    win_local = min(ctx_len, 4096)
+    avg_ctx = (win_local + ctx_len) / 2 if ctx_len > 4096 else ctx_len
+    attn = B * (shape.n_kv * avg_ctx * shape.r_attn * 2 +
+                shape.n_q * min(shape.k_attn, avg_ctx) * ((hd - shape.r_attn) + hd) * 2)
+    return proj + ffn + attn
+
+
+def cpu_baseline(args, shape):
+    n_l = 2
+    layers, h = oracle_sample(shape, args.ctx, n_l)
+    oracle_run(shape, layers[:1], h, args.ctx)            # touch the pages once
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        oracle_run(shape, layers, h, args.ctx)
+        reps += 1
+        if time.perf_counter() - t0 > 10.0 or reps >= 40:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": dt / (reps * n_l) * 1e6, "unit": "us/token/layer", "cores": host_threads(), "kind": "oracle",
+            "sample": f"{reps} x {n_l} decoder layers of one token at context {args.ctx} (fp64 numpy)"}
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_spark(args)
+
+
+if __name__ == "__main__":
+    main()
