@@ -100,6 +100,13 @@ const char* spark_status_string(int status);
 /* Number of thread blocks the context launches for its cooperative kernels (= SM count). */
 int spark_grid_size(const spark_ctx* ctx);
 
+/* Phase tracing (profiling aid; the paper has no counterpart).  With a non-NULL device buffer of
+ * `capacity` uint64 values, the cooperative kernels (FFN, attention) make thread 0 of block b
+ * store its SM's cycle counter at each phase boundary into trace[b * 16 + phase] (phase < 15) and
+ * the GPU-wide nanosecond timer at phase 0 into trace[b * 16 + 15].  `capacity` must cover
+ * 16 entries per block.  NULL switches tracing off (the default). */
+int spark_set_phase_trace(spark_ctx* ctx, uint64_t* trace, int64_t capacity);
+
 /* Gaussian upper quantile used for the threshold: z with P(N(0,1) > z) = p, i.e. Q(1 - p) of
  * Eq. 11.  Host function (no device work); exported so that it can be checked on its own.
  * Returns NaN for p outside (0, 1). */

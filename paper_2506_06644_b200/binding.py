@@ -26,7 +26,7 @@ SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
 
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
-    "spark_destroy", "spark_device_status", "spark_grid_size", "spark_stat_topk", "spark_ffn_decode",
+    "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_stat_topk", "spark_ffn_decode",
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode",
 ]
 
@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
         "spark_destroy": (i32, [vp]),
         "spark_device_status": (i32, [vp, vp, C.POINTER(i32)]),
         "spark_grid_size": (i32, [vp]),
+        "spark_set_phase_trace": (i32, [vp, vp, i64]),
         "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
         "spark_ffn_decode": (i32, [vp, vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
         "spark_attn_decode": (i32, [vp, vp, vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
@@ -147,6 +148,12 @@ class SparkContext:
         out = C.c_int(0)
         _check(lib().spark_device_status(self.handle, _stream(), C.byref(out)), "spark_device_status")
         return out.value
+
+    def set_phase_trace(self, trace):
+        """trace: int64/uint64 CUDA tensor of grid_size * 16 entries, or None to switch tracing off."""
+        n = 0 if trace is None else trace.numel()
+        _check(lib().spark_set_phase_trace(self.handle, _ptr(trace), n), "spark_set_phase_trace")
+        self._trace = trace
 
     @property
     def grid_size(self) -> int:

@@ -45,6 +45,7 @@ struct AttnParams {
     float4* pstats;    // [pieces][GQ]
     float* part;       // [pieces][GQ][hd + kPartPad]
     WsHeader* hdr;
+    PhaseTrace trace;
 };
 
 __device__ __forceinline__ float dot8r(const float (&w)[8], const float (&q)[8]) {
@@ -141,7 +142,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     }
     auto cta_of = [&](int64_t f) -> int { return static_cast<int>(((f + 1) * Gp - 1) / T); };
 
-    GridBarrier bar{p.hdr, static_cast<unsigned>(G), 0u};
+    GridBarrier bar{p.hdr, static_cast<unsigned>(G), 0u, 0u};
+    bar.begin();
+    p.trace.mark(0);
 
     // =============================== pass 1: predictor scores =====================================
     {
@@ -216,8 +219,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             f = sb + te;
         }
     }
+    p.trace.mark(1);
     bar.arrive();
     if (!bar.wait()) return;
+    p.trace.mark(2);
 
     // =============================== pass 2: select, gather, reduce ================================
     {
@@ -418,6 +423,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             f = sb + te;
         }
     }
+    p.trace.mark(3);
 }
 
 template <typename KT, int GQ>
@@ -494,6 +500,7 @@ extern "C" int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c
     p.pstats = reinterpret_cast<float4*>(ctx->scratch + scores_b);
     p.part = reinterpret_cast<float*>(ctx->scratch + scores_b + pstats_b);
     p.hdr = ctx->hdr;
+    p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
 
     const size_t ns_pad = (static_cast<size_t>(B * n_kv) + 1 + 3) & ~static_cast<size_t>(3);
     const size_t smem = ns_pad * 4 + static_cast<size_t>(gq * hd) * 4 + static_cast<size_t>(kCH) * 8 +

@@ -15,16 +15,31 @@ constexpr unsigned kFull = 0xffffffffu;
 // ---------------------------------------------------------------------------
 // Context (host object) and workspace header (device)
 // ---------------------------------------------------------------------------
+// One 32-byte sector that every block adds into and polls: the sum of its scores, the sum of their
+// squares, and the number of blocks that have added both (added last, with release semantics, so a
+// reader that sees the full count sees the full sums).  Reading the sector is one 32-byte load.
+struct __align__(32) SumCell {
+    double s1, s2;
+    unsigned count;
+    unsigned pad[3];
+};
+
+// Blocks spread their additions over this many cells per quantity (block b uses way b % 16): a
+// single cell would serialise 3 x #blocks atomics on one address, which costs microseconds.
+constexpr int kCellWays = 16;
+
 constexpr int kMaxSegments = 2048;   // (sequence, KV head) pairs one attention call may cover
 
 struct WsHeader {            // lives at the start of the caller's workspace; zero when idle
     int status;              // device status word (SPARK_OK or a SPARK_ERR_* device code)
     unsigned bar_count;      // inter-block barrier: arrivals of the current phase
     unsigned bar_gen;        // inter-block barrier: generation, bumped by the last arriver
-    unsigned pad[61];
+    unsigned epoch;          // launches of the FFN kernels so far (selects their accumulator ring slot)
+    unsigned pad[60];
     unsigned seg_done[kMaxSegments];   // attention: finished pieces per segment (self-resetting)
+    SumCell ffn_cells[4][4][16][kCellWays];   // FFN: [epoch & 3][token group][token][way] score sums
 };
-static_assert(sizeof(WsHeader) == 256 + 4 * kMaxSegments, "header layout");
+static_assert(sizeof(WsHeader) == 256 + 4 * kMaxSegments + 32 * 256 * kCellWays, "header layout");
 
 }  // namespace spark
 
@@ -37,6 +52,8 @@ struct spark_ctx {
     spark::WsHeader* hdr;    // == ws
     char* scratch;           // ws + sizeof(WsHeader)
     size_t scratch_bytes;
+    unsigned long long* trace;   // optional phase trace (device), see spark_set_phase_trace
+    long long trace_cap;
 };
 
 namespace spark {
@@ -208,41 +225,67 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 
-// The barrier is split so that independent work can sit between arrival and wait.
-// Every block of a co-resident (cooperative) grid calls arrive once and wait once per phase.
-// Thread 0 of the block does the global traffic; the __syncthreads order the block's other
-// threads around it.  The wait gives up after `limit_ns` and records SPARK_ERR_TIMEOUT.
-struct GridBarrier {
-    WsHeader* hdr;
-    unsigned nblocks;
-    unsigned gen;   // generation observed before arriving (thread 0 only)
-
-    __device__ __forceinline__ void arrive() {
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            gen = ld_acquire_u32(&hdr->bar_gen);
-            const unsigned prev = atom_add_acqrel_u32(&hdr->bar_count, 1u);
-            if (prev == nblocks - 1) {
-                hdr->bar_count = 0;                        // ordered before the release below
-                st_release_u32(&hdr->bar_gen, gen + 1);
+// Optional phase trace: thread 0 of a block stores its SM's cycle counter at a phase boundary
+// (phases 0..14); phase 0 also stores the GPU-wide nanosecond timer in entry 15, which lets a
+// reader line the blocks up.  The cycle counter is cheap to read; the global timer is not.
+struct PhaseTrace {
+    unsigned long long* buf;
+    long long cap;
+    __device__ __forceinline__ void mark(int phase) const {
+        if (buf != nullptr && threadIdx.x == 0) {
+            const long long i = static_cast<long long>(blockIdx.x) * 16 + phase;
+            if (i + 15 < cap) {
+                buf[i] = static_cast<unsigned long long>(clock64());
+                if (phase == 0) buf[i + 15] = global_ns();
             }
         }
     }
-    // Returns false if the wait timed out (uniform over the block).
-    __device__ __forceinline__ bool wait(unsigned long long limit_ns = 2000000000ull) {
+};
+
+// Bound of every spin-wait, in SM cycles (about two seconds at 2 GHz).
+constexpr long long kSpinLimitCycles = 4000000000ll;
+
+// Grid-wide barrier for co-resident (cooperative) grids, split in three so that independent work
+// can sit between the steps and no round trip to L2 is exposed needlessly:
+//   begin()   once per kernel, early: thread 0 requests the current generation;
+//   arrive()  every block, once per phase: block-wide sync, then thread 0 adds its arrival;
+//   wait()    thread 0 of the last block to arrive resets the count and publishes the next
+//             generation; the others poll it.  The poll gives up after about two seconds, records
+//             SPARK_ERR_TIMEOUT and returns false (uniform over the block).
+struct GridBarrier {
+    WsHeader* hdr;
+    unsigned nblocks;
+    unsigned gen;    // generation of the phase in progress (thread 0 only)
+    unsigned prev;   // arrivals before ours (thread 0 only)
+
+    __device__ __forceinline__ void begin() {
+        if (threadIdx.x == 0) gen = ld_acquire_u32(&hdr->bar_gen);
+    }
+    __device__ __forceinline__ void arrive() {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            prev = atom_add_acqrel_u32(&hdr->bar_count, 1u);
+        }
+    }
+    __device__ __forceinline__ bool wait() {
         __shared__ int ok_flag;
         if (threadIdx.x == 0) {
             int ok = 1;
-            if (ld_acquire_u32(&hdr->bar_gen) == gen) {
-                const unsigned long long t0 = global_ns();
+            if (prev == nblocks - 1) {
+                hdr->bar_count = 0;                        // ordered before the release below
+                st_release_u32(&hdr->bar_gen, gen + 1);
+            } else if (ld_acquire_u32(&hdr->bar_gen) == gen) {
+                const long long t0 = clock64();
                 while (ld_acquire_u32(&hdr->bar_gen) == gen) {
-                    if (global_ns() - t0 > limit_ns) {
+                    if (clock64() - t0 > kSpinLimitCycles) {
                         ok = 0;
                         atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
                         break;
                     }
                 }
             }
+            gen += 1;                                      // the next phase of this kernel
             ok_flag = ok;
         }
         __syncthreads();
@@ -251,6 +294,111 @@ struct GridBarrier {
         return ok;
     }
 };
+
+// Sum-cell helpers.
+__device__ __forceinline__ void red_add_f64(double* p, double v) {
+    asm volatile("red.relaxed.gpu.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add_u32(unsigned* p, unsigned v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// One 32-byte read of a cell (sm_100 has 256-bit global loads): {s1, s2, count}.
+__device__ __forceinline__ void ld_cell(const SumCell* c, double& s1, double& s2, unsigned& count) {
+    unsigned long long a, b, d, e;   // e: padding half of the sector
+    asm volatile("ld.acquire.gpu.global.v4.u64 {%0,%1,%2,%3}, [%4];"
+                 : "=l"(a), "=l"(b), "=l"(d), "=l"(e)
+                 : "l"(c)
+                 : "memory");
+    s1 = __longlong_as_double(static_cast<long long>(a));
+    s2 = __longlong_as_double(static_cast<long long>(b));
+    count = static_cast<unsigned>(d & 0xffffffffull);
+    (void)e;
+}
+// Add this block's two sums to its way of a cell group, then its arrival (release: ordered after
+// the sums and after everything the block wrote before).  One thread calls this.
+__device__ __forceinline__ void cells_add(SumCell* ways, int block, double s1, double s2) {
+    SumCell* c = ways + (block % kCellWays);
+    red_add_f64(&c->s1, s1);
+    red_add_f64(&c->s2, s2);
+    red_release_add_u32(&c->count, 1u);
+}
+// Lanes 0..15 of one warp poll the 16 ways (one 32-byte acquire load each) until all `nblocks`
+// blocks have arrived, then every lane of the warp gets the totals.  Called by a full warp.
+// Returns false after about two seconds (SPARK_ERR_TIMEOUT recorded).
+__device__ __forceinline__ bool cells_wait(const SumCell* ways, unsigned nblocks, double& s1, double& s2, WsHeader* hdr) {
+    const int lane = threadIdx.x & 31;
+    const long long t0 = clock64();
+    for (;;) {
+        double a = 0.0, b = 0.0;
+        unsigned cnt = 0u;
+        if (lane < kCellWays) ld_cell(ways + lane, a, b, cnt);
+        unsigned tot = cnt;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) tot += __shfl_xor_sync(kFull, tot, o);
+        tot = __shfl_sync(kFull, tot, 0);
+        if (tot == nblocks) {
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) {
+                a += __shfl_xor_sync(kFull, a, o);
+                b += __shfl_xor_sync(kFull, b, o);
+            }
+            s1 = __shfl_sync(kFull, a, 0);
+            s2 = __shfl_sync(kFull, b, 0);
+            return true;
+        }
+        if (clock64() - t0 > kSpinLimitCycles) {
+            if (lane == 0) atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+// 16-byte accesses that always go to L2 (slots other blocks write or poll).
+__device__ __forceinline__ uint4 ld_volatile16(const void* p) {
+    uint4 v;
+    asm volatile("ld.acquire.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_volatile16(void* p, uint4 v) {
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// Slot exchange between the blocks of a co-resident grid: every block publishes one 16-byte slot
+// {payload x, y, z, tag} per item and every block reads all slots, waiting for the tag of the
+// current launch.  One store and one polled load replace "atomic counter + flag + read-back":
+// the data IS the arrival.  Tags come from a launch epoch kept in the workspace header, read at
+// kernel start and advanced by block 0 once it has seen every slot.  Slot arrays are double
+// buffered by phase parity, so a block that runs ahead never overwrites a slot still being polled.
+// A poll gives up after about two seconds (SPARK_ERR_TIMEOUT is recorded; the caller returns).
+// Waits are bounded in SM cycles: the cycle counter is cheap to read, the global timer is not.
+__device__ __forceinline__ bool poll_slot(const uint4* slot, unsigned tag, uint4& out, WsHeader* hdr) {
+    out = ld_volatile16(slot);
+    if (out.w == tag) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        out = ld_volatile16(slot);
+        if (out.w == tag) return true;
+        if (clock64() - t0 > kSpinLimitCycles) {
+            atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool poll_flag(const unsigned* flag, unsigned tag, WsHeader* hdr) {
+    if (ld_acquire_u32(flag) == tag) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (ld_acquire_u32(flag) == tag) return true;
+        if (clock64() - t0 > kSpinLimitCycles) {
+            atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
 
 // Vector reduction into global memory: y[0..3] += v (16-byte aligned address).
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {

@@ -11,6 +11,7 @@
 //            u_i = GELU(s_i - theta) t_i, then a thread per 8 output columns accumulates
 //            sum_i u_i V[:,i] in registers and adds it to y with vector reductions.
 // Individual masks gate the arithmetic, the union gates the loads (Appendix B).
+#include "ffn_params.h"
 #include "kernels.h"
 #include "rowdot.cuh"
 
@@ -21,26 +22,6 @@ namespace {
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / kWarp;
 constexpr int kRows = 4;          // rows a warp works on at once in phase A
-constexpr int kMaxTB = 16;        // tokens per pass over the weights
-
-struct FfnParams {
-    const float* x;
-    const float* norm_w;
-    float eps;
-    const void* K1t;
-    const void* K2t;
-    const void* Vt;
-    int B, d, d_ff, r, rpc, xw;
-    int dense, erf_form, identity;
-    double z;
-    const float* y_init;
-    float* y;
-    float* theta;
-    int32_t* count;
-    int32_t* idx;
-    float4* stats;                // [2][TB][grid] per-block moments
-    WsHeader* hdr;
-};
 
 template <typename WT, int TB>
 __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
@@ -50,10 +31,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
     float* u_loc = s_loc + static_cast<size_t>(TB) * p.rpc;         // [TB][rpc]
     int* ulist = reinterpret_cast<int*>(u_loc + static_cast<size_t>(TB) * p.rpc);   // [rpc]
     unsigned* amask = reinterpret_cast<unsigned*>(ulist + p.rpc);   // [rpc]
-    __shared__ float rstd[kMaxTB];
-    __shared__ float theta_s[kMaxTB];
+    __shared__ float rstd[kFfnMaxTB];
+    __shared__ float theta_s[kFfnMaxTB];
     __shared__ int wcnt[kWarps];
     __shared__ unsigned tok_any;
+    __shared__ unsigned s_epoch;
+    __shared__ int s_fail;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int grid = gridDim.x, cta = blockIdx.x;
@@ -64,36 +47,23 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
     const WT* K1t = static_cast<const WT*>(p.K1t);
     const WT* K2t = static_cast<const WT*>(p.K2t);
     const WT* Vt = static_cast<const WT*>(p.Vt);
-    GridBarrier bar{p.hdr, static_cast<unsigned>(grid), 0u};
+    if (tid == 0) {
+        s_epoch = ld_acquire_u32(&p.hdr->epoch);      // consumed after phase A
+        s_fail = 0;
+    }
+    if (cta == 0) {
+        // clear the cells the launch after next will use (last used two launches ago)
+        const unsigned e = ld_acquire_u32(&p.hdr->epoch);
+        SumCell* c = &p.hdr->ffn_cells[(e + 2u) & 3u][0][0][0];
+        for (int i = tid; i < 4 * 16 * kCellWays; i += kThreads) { c[i].s1 = 0.0; c[i].s2 = 0.0; c[i].count = 0u; }
+    }
+    p.trace.mark(0);
 
     for (int g0 = 0, grp = 0; g0 < p.B; g0 += TB, ++grp) {
         const int tbv = min(TB, p.B - g0);
         const float* xg = p.x + static_cast<int64_t>(g0) * d;
         float* yg = p.y + static_cast<int64_t>(g0) * d;
 
-        // ---- prologue: optional RMSNorm scale, y initialisation, x[:r] into shared memory ------
-        for (int t = warp; t < TB; t += kWarps) {
-            float ss = 0.f;
-            if (p.norm_w != nullptr && t < tbv) {
-                const float4* xr = reinterpret_cast<const float4*>(xg + static_cast<int64_t>(t) * d);
-                for (int i = lane; i < d / 4; i += 32) {
-                    const float4 v = xr[i];
-                    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-                }
-                ss = warp_sum(ss);
-            }
-            if (lane == 0) rstd[t] = p.norm_w != nullptr ? rsqrtf(ss / static_cast<float>(d) + p.eps) : 1.f;
-        }
-        {
-            const int64_t total4 = static_cast<int64_t>(tbv) * d / 4;
-            const float4* yi = p.y_init ? reinterpret_cast<const float4*>(p.y_init + static_cast<int64_t>(g0) * d) : nullptr;
-            float4* yo = reinterpret_cast<float4*>(yg);
-            for (int64_t i = static_cast<int64_t>(cta) * kThreads + tid; i < total4; i += static_cast<int64_t>(grid) * kThreads)
-                yo[i] = yi ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        if (cta == 0 && p.count != nullptr && tid < tbv) p.count[g0 + tid] = 0;
-        if (tid == 0) tok_any = 0u;
-        __syncthreads();
         auto stage = [&](int col0, int width) {     // xs[t][0:width] = x[t][col0:col0+width] (normalised)
             const int w4 = width / 4;
             for (int i = tid; i < TB * w4; i += kThreads) {
@@ -110,51 +80,84 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
                 reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * xw)[c] = v;
             }
         };
-        stage(0, r);
-        __syncthreads();
+        // Runs once, after the first K1t loads are in flight: optional RMSNorm scale, y
+        // initialisation, x[:r] into shared memory.
+        auto prologue = [&]() {
+            if (p.norm_w != nullptr) {
+                for (int t = warp; t < TB; t += kWarps) {
+                    float ss = 0.f;
+                    if (t < tbv) {
+                        const float4* xr = reinterpret_cast<const float4*>(xg + static_cast<int64_t>(t) * d);
+                        for (int i = lane; i < d / 4; i += 32) {
+                            const float4 v = xr[i];
+                            ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                        }
+                        ss = warp_sum(ss);
+                    }
+                    if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(d) + p.eps);
+                }
+                __syncthreads();
+            }
+            stage(0, r);
+            {
+                const int64_t total4 = static_cast<int64_t>(tbv) * d / 4;
+                const float4* yi = p.y_init ? reinterpret_cast<const float4*>(p.y_init + static_cast<int64_t>(g0) * d) : nullptr;
+                float4* yo = reinterpret_cast<float4*>(yg);
+                for (int64_t i = static_cast<int64_t>(cta) * kThreads + tid; i < total4; i += static_cast<int64_t>(grid) * kThreads)
+                    yo[i] = yi ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (cta == 0 && p.count != nullptr && tid < tbv) p.count[g0 + tid] = 0;
+            if (tid == 0) tok_any = 0u;
+            __syncthreads();
+            p.trace.mark(1);
+        };
 
         // ---- phase A: predictor scores of this block's neurons ----------------------------------
-        rows_dot<WT, TB, kRows>(K1t, r, row0, nloc, r / 8, xs, xw, [&](int j, int t, float v) {
+        rows_dot<WT, TB, kRows>(K1t, r, row0, nloc, r / 8, xs, xw, prologue, [&](int j, int t, float v) {
             s_loc[static_cast<size_t>(t) * rpc + j] = v;
         });
         __syncthreads();
+        p.trace.mark(2);
 
-        // ---- per-block moments of the scores, one warp per token (two-pass, in registers) ---------
-        float4* stats = p.stats + static_cast<size_t>(grp & 1) * TB * grid;
+        // ---- sums of the scores and of their squares (fp64), one warp per token, added to the token's
+        //      grid-wide cell; the arrival follows them with release semantics --------------------------
+        SumCell* cells = &p.hdr->ffn_cells[s_epoch & 3u][grp & 3][0][0];   // [token][way]
         for (int t = warp; t < tbv; t += kWarps) {
             const float* sr = s_loc + static_cast<size_t>(t) * rpc;
-            float sum = 0.f;
-            for (int j = lane; j < nloc; j += 32) sum += sr[j];
-            sum = warp_sum(sum);
-            const float mean = nloc > 0 ? sum / static_cast<float>(nloc) : 0.f;
-            float m2 = 0.f;
+            double s1 = 0.0, s2 = 0.0;
             for (int j = lane; j < nloc; j += 32) {
-                const float dl = sr[j] - mean;
-                m2 = fmaf(dl, dl, m2);
+                const double v = static_cast<double>(sr[j]);
+                s1 += v;
+                s2 = fma(v, v, s2);
             }
-            m2 = warp_sum(m2);
-            if (lane == 0) stats[static_cast<size_t>(t) * grid + cta] = make_float4(static_cast<float>(nloc), mean, m2, 0.f);
+            s1 = warp_sum_f64(s1);
+            s2 = warp_sum_f64(s2);
+            if (lane == 0) cells_add(cells + t * kCellWays, cta, s1, s2);
         }
-        bar.arrive();
-        stage(r, d2);                                   // x[r:] replaces x[:r] while the barrier fills
-        if (!bar.wait()) return;
-
-        // ---- theta per token: every block merges all partial moments itself ----------------------
+        p.trace.mark(3);
+        __syncthreads();
+        stage(r, d2);                                   // x[r:] replaces x[:r] while the cells fill
+        // theta per token (Eq. 11, Bessel-corrected) once every block has added its sums
         for (int t = warp; t < tbv; t += kWarps) {
-            Moments m{0.0, 0.0, 0.0};
-            for (int c = lane; c < grid; c += 32) {
-                const float4 v = ld_cg_f4(&stats[static_cast<size_t>(t) * grid + c]);
-                m = merge(m, Moments{static_cast<double>(v.x), static_cast<double>(v.y), static_cast<double>(v.z)});
-            }
-            m = warp_merge(m);
-            const float th = p.identity ? -INFINITY : theta_from(m, p.z);
+            double sa, sb;
+            const bool ok = cells_wait(cells + t * kCellWays, static_cast<unsigned>(grid), sa, sb, p.hdr);
             if (lane == 0) {
+                float th = -INFINITY;
+                if (!ok) s_fail = 1;
+                if (!p.identity) {
+                    const double mean = sa * p.inv_n;
+                    const float var = static_cast<float>((sb - sa * mean) * p.inv_nm1);
+                    th = static_cast<float>(mean) + sqrtf(fmaxf(var, 0.f)) * static_cast<float>(p.z);
+                }
                 theta_s[t] = th;
                 if (cta == 0 && p.theta != nullptr) p.theta[g0 + t] = th;
             }
         }
         __syncthreads();
+        if (s_fail) return;
+        p.trace.mark(4);
 
+        p.trace.mark(5);
         // ---- phase C: masks and the ordered union list of this block's neurons --------------------
         int nU = 0;
         for (int j0 = 0; j0 < nloc; j0 += kThreads) {
@@ -204,6 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
             }
         }
 
+        p.trace.mark(6);
         // ---- phase D: only the union rows of K2t and Vt are read -------------------------------------
         constexpr int RB = 8;                            // union rows a thread holds in flight
         const int ncd = d / 8;
@@ -216,6 +220,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
             if (PRE && j < nU && tid < ncd) vpre[j].load_pinned(Vt + static_cast<int64_t>(row0 + ulist[j]) * d, tid);
             else vpre[j].zero();
         }
+        p.trace.mark(9);
         // ---- D1: t_i = K2[:,i] . x[r:] for union rows (a warp takes one or two rows at a time),
         //          u = GELU(s - theta) * t
         {
@@ -250,6 +255,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
                             if (c < nc2 && cm[rr] != 0u) w[rr][u].load(krow[rr], c);
                             else w[rr][u].zero();
                         }
+                    p.trace.mark(10);
 #pragma unroll
                     for (int u = 0; u < KU; ++u) {
                         const int c = c0 + u * 32 + lane;
@@ -268,6 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
                         }
                     }
                 }
+                p.trace.mark(11);
 #pragma unroll
                 for (int rr = 0; rr < RR; ++rr) {
                     if (ui0 + rr >= nU) break;
@@ -286,7 +293,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
                 }
             }
         }
+        p.trace.mark(12);
         __syncthreads();
+        p.trace.mark(7);
 
         // ---- D2: y += sum_i u_i V[:,i]; per-thread register accumulators, vector reductions to y -----
         {
@@ -344,8 +353,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
                 }
             }
         }
+        p.trace.mark(8);
         __syncthreads();      // shared buffers are reused by the next token group
     }
+    if (cta == 0 && tid == 0) p.hdr->epoch = s_epoch + 1u;   // every block has read the epoch by now
 }
 
 template <typename WT, int TB>
@@ -411,14 +422,15 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     p.identity = a.k >= a.d_ff ? 1 : 0;
     p.z = p.identity ? 0.0 : spark_normal_upper_quantile(static_cast<double>(a.k) / static_cast<double>(a.d_ff));
     p.y_init = a.y_init; p.y = a.y; p.theta = a.theta; p.count = a.count; p.idx = a.idx;
+    p.ncopy = 0;
+    p.inv_n = 1.0 / static_cast<double>(a.d_ff);
+    p.inv_nm1 = 1.0 / static_cast<double>(a.d_ff - 1);
     p.hdr = ctx->hdr;
-    const size_t stats_bytes = static_cast<size_t>(2) * kMaxTB * grid * sizeof(float4);
-    if (stats_bytes > ctx->scratch_bytes) return SPARK_ERR_WORKSPACE;
-    p.stats = reinterpret_cast<float4*>(ctx->scratch);
-
+    p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
     const size_t smem = (static_cast<size_t>(tb) * p.xw + static_cast<size_t>(2) * tb * p.rpc) * sizeof(float) +
                         static_cast<size_t>(p.rpc) * 8;
     if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_UNSUPPORTED;
+    if (a.B == 1 && grid <= 512 && a.d <= 4096) return ffn1_launch(ctx, p, a.wdtype, stream);
     if (a.wdtype == SPARK_BF16) return launch_tb<__nv_bfloat16>(ctx, p, tb, smem, stream);
     return launch_tb<float>(ctx, p, tb, smem, stream);
 }

@@ -1,0 +1,35 @@
+// Kernel parameters of the Spark FFN kernels (internal).
+#pragma once
+
+#include "common.cuh"
+
+namespace spark {
+
+constexpr int kFfnMaxTB = 16;     // tokens per pass over the weights
+
+struct FfnParams {
+    const float* x;
+    const float* norm_w;
+    float eps;
+    const void* K1t;
+    const void* K2t;
+    const void* Vt;
+    int B, d, d_ff, r, rpc, xw;
+    int ncopy;                    // B == 1 kernel: per-warp copies of y in shared memory
+    int dense, erf_form, identity;
+    double z;
+    double inv_n, inv_nm1;        // 1 / d_ff and 1 / (d_ff - 1)
+    const float* y_init;
+    float* y;
+    float* theta;
+    int32_t* count;
+    int32_t* idx;
+    WsHeader* hdr;
+    PhaseTrace trace;
+};
+
+
+// B == 1 fast path (ffn_b1.cu).
+int ffn1_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream);
+
+}  // namespace spark

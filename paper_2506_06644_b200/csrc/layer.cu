@@ -33,32 +33,34 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
     const int n_in = p.n_in;
     const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
     const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
-    const int w4 = n_in / 4;
-    for (int i = tid; i < TB * w4; i += kThreads) {
-        const int t = i / w4, c = i - t * w4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (t < p.B) v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
-        reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * n_in)[c] = v;
-    }
-    __syncthreads();
-    if (p.norm_w != nullptr) {
-        for (int t = warp; t < TB; t += kWarps) {
-            float ss = 0.f;
-            for (int i = lane; i < n_in; i += 32) {
-                const float v = xs[static_cast<size_t>(t) * n_in + i];
-                ss = fmaf(v, v, ss);
+    auto fill_x = [&]() {       // runs once the first weight loads are in flight
+        const int w4 = n_in / 4;
+        for (int i = tid; i < TB * w4; i += kThreads) {
+            const int t = i / w4, c = i - t * w4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (t < p.B) v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
+            reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * n_in)[c] = v;
+        }
+        __syncthreads();
+        if (p.norm_w != nullptr) {
+            for (int t = warp; t < TB; t += kWarps) {
+                float ss = 0.f;
+                for (int i = lane; i < n_in; i += 32) {
+                    const float v = xs[static_cast<size_t>(t) * n_in + i];
+                    ss = fmaf(v, v, ss);
+                }
+                ss = warp_sum(ss);
+                if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(n_in) + p.eps);
             }
-            ss = warp_sum(ss);
-            if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(n_in) + p.eps);
+            __syncthreads();
+            for (int i = tid; i < TB * n_in; i += kThreads) {
+                const int t = i / n_in, c = i - t * n_in;
+                xs[i] *= rstd[t] * p.norm_w[c];
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        for (int i = tid; i < TB * n_in; i += kThreads) {
-            const int t = i / n_in, c = i - t * n_in;
-            xs[i] *= rstd[t] * p.norm_w[c];
-        }
-        __syncthreads();
-    }
-    rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in,
+    };
+    rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in, fill_x,
                          [&](int j, int t, float v) {
                              if (t < p.B) {
                                  const int64_t o = static_cast<int64_t>(t) * p.n_out + row0 + j;

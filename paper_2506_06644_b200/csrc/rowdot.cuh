@@ -11,10 +11,13 @@ namespace spark {
 // load of a batch (CU chunks x RW rows per lane) is issued before the first use so that a block
 // keeps its whole share of the matrix in flight.  With TB >= 16 the two half-warps take eight
 // tokens each.  emit(j, t, value) is called by exactly one lane per (row, token).
+// before_use() is called exactly once by every thread of the block, after the first batch of
+// weight loads has been issued and before anything is read from xs: the caller fills xs there
+// (and synchronises the block), so that the input's latency hides behind the weights'.
 // Must be called by all threads of a 512-thread block.
-template <typename WT, int TB, int RW, typename Emit>
+template <typename WT, int TB, int RW, typename Hook, typename Emit>
 __device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, int row0, int nloc, int nck,
-                                         const float* xs, int xw, Emit emit) {
+                                         const float* xs, int xw, Hook before_use, Emit emit) {
     constexpr int kWarpsPerBlock = 16;
     constexpr int TS = TB >= 16 ? 2 : 1;     // lane groups that split the tokens
     constexpr int TPL = TB / TS;             // tokens per lane group
@@ -22,7 +25,11 @@ __device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, i
     constexpr int CU = (TB == 1 ? (RW >= 4 ? 4 : 8) : 2) / (sizeof(WT) == 4 ? 2 : 1);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int lg = lane / GL, gl = lane % GL;
-    for (int rg = warp; rg * RW < nloc; rg += kWarpsPerBlock) {
+    bool hooked = false;
+    int rg = warp;
+#pragma unroll 1
+    do {
+        const bool has = rg * RW < nloc;
         float acc[RW][TPL];
 #pragma unroll
         for (int i = 0; i < RW; ++i)
@@ -32,8 +39,9 @@ __device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, i
 #pragma unroll
         for (int i = 0; i < RW; ++i) {
             const int j = rg * RW + i;
-            rowp[i] = W + static_cast<int64_t>(row0 + (j < nloc ? j : nloc - 1)) * ld;
+            rowp[i] = W + static_cast<int64_t>(row0 + (j < nloc ? j : (nloc > 0 ? nloc - 1 : 0))) * ld;
         }
+#pragma unroll 1
         for (int c0 = 0; c0 < nck; c0 += GL * CU) {
             Row8<WT> w[CU][RW];
 #pragma unroll
@@ -41,10 +49,15 @@ __device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, i
                 const int c = c0 + u * GL + gl;
 #pragma unroll
                 for (int i = 0; i < RW; ++i) {
-                    if (c < nck) w[u][i].load(rowp[i], c);
+                    if (has && c < nck) w[u][i].load(rowp[i], c);
                     else w[u][i].zero();
                 }
             }
+            if (!hooked) {
+                before_use();
+                hooked = true;
+            }
+            if (!has) break;
 #pragma unroll
             for (int u = 0; u < CU; ++u) {
                 const int c = c0 + u * GL + gl;
@@ -61,16 +74,19 @@ __device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, i
                 }
             }
         }
+        if (has) {
 #pragma unroll
-        for (int i = 0; i < RW; ++i)
+            for (int i = 0; i < RW; ++i)
 #pragma unroll
-            for (int t = 0; t < TPL; ++t) {
-                float v = acc[i][t];
+                for (int t = 0; t < TPL; ++t) {
+                    float v = acc[i][t];
 #pragma unroll
-                for (int o = GL / 2; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-                if (gl == 0 && rg * RW + i < nloc) emit(rg * RW + i, lg * TPL + t, v);
-            }
-    }
+                    for (int o = GL / 2; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+                    if (gl == 0 && rg * RW + i < nloc) emit(rg * RW + i, lg * TPL + t, v);
+                }
+        }
+        rg += kWarpsPerBlock;
+    } while (rg * RW < nloc);
 }
 
 }  // namespace spark
