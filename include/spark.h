@@ -143,6 +143,33 @@ int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t,
                      const void* Vt, int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k,
                      int flags, float* y, float* theta, int32_t* count, int32_t* idx, void* stream);
 
+/* ---- Spark FFN without any allocation (the paper has no counterpart) ----------------------
+ * Some callers may not call cudaMalloc at all: code that runs where device memory has been
+ * handed out in full up front (an inference server's arena, a plugin inside another runtime), or
+ * that must not touch the allocator because a stream capture or a latency-critical section is
+ * under way elsewhere in the process.  They cannot give spark_create a workspace.  This entry point
+ * computes exactly what spark_ffn_decode computes, with the small amount of inter-block state the
+ * kernel needs (a status word, a launch counter, the cells the blocks add their score sums into)
+ * kept in a fixed array inside the library's device image: about 140 KB on every GPU that loads
+ * the library, held until the process exits.  Inputs and outputs are still the caller's.
+ *   - Limit: B <= SPARK_NOALLOC_MAX_TOKENS; a larger B returns SPARK_ERR_UNSUPPORTED.  All other
+ *     limits and argument checks are those of spark_ffn_decode.  count / idx are not offered.
+ *   - The device is the current one.  The first call on a device looks up the array's device
+ *     address and clears it (a synchronous 140 KB memset); make that first call before any stream
+ *     capture begins.  No call allocates or frees device memory.
+ *   - All calls on a device share the array, and it keeps what the last call left (the kernels
+ *     themselves clear the cells a later call will use).  Two calls whose kernels overlap on the
+ *     GPU -- different streams, or one process-wide array used from two threads -- race on it:
+ *     issue them on one stream, or otherwise order them.  spark_ffn_decode with its own context
+ *     has no such restriction across contexts.
+ *   - A device-side timeout (SPARK_ERR_TIMEOUT) cannot be read back through this entry point; y is
+ *     then incomplete.  It only arises when the launch's blocks cannot all be resident at once,
+ *     which the cooperative launch already refuses with SPARK_ERR_CUDA. */
+#define SPARK_NOALLOC_MAX_TOKENS 16
+int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K1t, const void* K2t, const void* Vt,
+                             int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k, int flags,
+                             float* y, float* theta, void* stream);
+
 /* ---- Spark attention (Section 2.2, Eq. 7) ------------------------------------
  * For sequence b and query head h (KV head g = h / (n_q / n_kv)), over the tokens t of the window
  * [max(0, n_b - window), n_b), n_b = ctx_len[b] (window == 0: all n_b tokens):

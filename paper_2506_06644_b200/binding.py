@@ -27,7 +27,7 @@ SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
     "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_stat_topk", "spark_ffn_decode",
-    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode",
+    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc",
 ]
 
 
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
         "spark_set_phase_trace": (i32, [vp, vp, i64]),
         "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
         "spark_ffn_decode": (i32, [vp, vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
+        "spark_ffn_decode_noalloc": (i32, [vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp]),
         "spark_attn_decode": (i32, [vp, vp, vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
                                     vp, vp, vp, vp, i64, vp]),
         "spark_dense_gemv": (i32, [vp, vp, i64, vp, i32, i64, i64, vp, vp, vp]),
@@ -179,6 +180,13 @@ def spark_stat_topk(ctx: SparkContext, x, rows, n, ld, k, fill, theta, count, id
 def spark_ffn_decode(ctx: SparkContext, x, B, K1t, K2t, Vt, wdtype, d, d_ff, r, k, flags, y, theta, count, idx):
     _check(lib().spark_ffn_decode(ctx.handle, _ptr(x), B, _ptr(K1t), _ptr(K2t), _ptr(Vt), wdtype, d, d_ff, r, k,
                                   flags, _ptr(y), _ptr(theta), _ptr(count), _ptr(idx), _stream()), "spark_ffn_decode")
+
+
+def spark_ffn_decode_noalloc(x, B, K1t, K2t, Vt, wdtype, d, d_ff, r, k, flags, y, theta):
+    """spark_ffn_decode for callers that must not allocate: no context, no workspace; the kernel's
+    inter-block state lives in a fixed array inside the library (see include/spark.h).  B <= 16."""
+    _check(lib().spark_ffn_decode_noalloc(_ptr(x), B, _ptr(K1t), _ptr(K2t), _ptr(Vt), wdtype, d, d_ff, r, k, flags,
+                                          _ptr(y), _ptr(theta), _stream()), "spark_ffn_decode_noalloc")
 
 
 def spark_attn_decode(ctx: SparkContext, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv, hd, r, cap, ctx_len, window,

@@ -447,3 +447,62 @@ extern "C" int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const
     a.y_init = nullptr; a.y = y; a.theta = theta; a.count = count; a.idx = idx;
     return ffn_launch(ctx, a, static_cast<cudaStream_t>(stream));
 }
+
+// ---------------------------------------------------------------------------------------------
+// spark_ffn_decode_noalloc: the same FFN for callers that cannot allocate device memory.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// The inter-block state the FFN kernels need (status word, launch epoch, score-sum cells) lives in
+// this file-scope array instead of a caller-provided workspace.  It is zero when the module is
+// loaded, which is the idle state; every device that loads the library carries its own copy
+// (about 140 KB) until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_state[sizeof(WsHeader)];
+
+struct NoallocDevice {
+    bool ready;
+    WsHeader* state;      // device address of g_noalloc_state on this device
+    int num_sms, max_smem_optin;
+};
+NoallocDevice g_noalloc[64] = {};
+
+}  // namespace
+
+extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K1t, const void* K2t, const void* Vt,
+                                        int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k, int flags,
+                                        float* y, float* theta, void* stream) {
+    if (B > SPARK_NOALLOC_MAX_TOKENS) return SPARK_ERR_UNSUPPORTED;   // beyond what the static state serves
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPARK_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return SPARK_ERR_UNSUPPORTED;
+    NoallocDevice& nd = g_noalloc[dev];
+    if (!nd.ready) {
+        // Once per device, with that device current: in host code the array's name is only a
+        // stand-in for the symbol, so its device address has to be asked for.
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_state) != cudaSuccess || ptr == nullptr) return SPARK_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&nd.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPARK_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&nd.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        if (cudaMemset(ptr, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;   // idle state
+        nd.state = static_cast<WsHeader*>(ptr);
+        nd.ready = true;
+    }
+    spark_ctx local;
+    local.device = dev;
+    local.num_sms = nd.num_sms;
+    local.max_smem_optin = nd.max_smem_optin;
+    local.ws = reinterpret_cast<char*>(nd.state);
+    local.ws_bytes = sizeof(WsHeader);
+    local.hdr = nd.state;
+    local.scratch = nullptr;
+    local.scratch_bytes = 0;
+    local.trace = nullptr;
+    local.trace_cap = 0;
+    FfnArgs a;
+    a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
+    a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = wdtype;
+    a.B = B; a.d = d; a.d_ff = d_ff; a.r = r; a.k = k; a.flags = flags;
+    a.y_init = nullptr; a.y = y; a.theta = theta; a.count = nullptr; a.idx = nullptr;
+    return ffn_launch(&local, a, static_cast<cudaStream_t>(stream));
+}
