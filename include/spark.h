@@ -84,13 +84,13 @@ size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap
                              int64_t hd, int64_t max_d);
 
 /* Create a context on `device` around a caller-owned device workspace (256-byte aligned).
- * Zeroes the workspace header (a small synchronous memset); queries the SM count.
+ * Zeroes the workspace (a synchronous memset: its idle state is all zero); queries the SM count.
  * *out is a host object released by spark_destroy (which leaves the workspace alone). */
 int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_bytes);
 int spark_destroy(spark_ctx* ctx);
 
 /* Synchronise `stream`, copy the device status word to *host_out (host pointer), clear it, and
- * if it was not SPARK_OK also reset the inter-block barrier state.  Returns SPARK_OK when the
+ * if it was not SPARK_OK also reset the workspace to its idle (zero) state.  Returns SPARK_OK when the
  * read itself worked (the device status is in *host_out). */
 int spark_device_status(spark_ctx* ctx, void* stream, int* host_out);
 
@@ -231,7 +231,7 @@ typedef struct spark_kv_cache {
     void* vc;             /* [B][n_kv][cap][hd]          bf16                              */
 } spark_kv_cache;
 
-/* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d) fp32 values, 16-byte aligned, caller-owned, contents
+/* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2) fp32 values, 16-byte aligned, caller-owned, contents
  * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 16.  Five kernels are
  * enqueued: QKV projection, position encoding + cache append, attention, output projection, FFN. */
 int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,

@@ -4,16 +4,22 @@
 // The (sequence, KV head, token) space of all windows is laid out flat and cut into equal
 // contiguous ranges, one per block, so that the predictor slice of the cache is streamed evenly
 // whatever the mix of context lengths.  A range may cross (sequence, KV head) "segments"; the
-// intersection of a block's range with one segment is a "piece".
+// intersection of a block's range with one segment is a "piece"; inside a piece every warp owns a
+// contiguous run of tokens through both passes.
 //
-//   pass 1  per piece: s_t = k1c[t] . q[:r] for the query heads of the KV group (half a warp per
-//           token row, coalesced 16-byte loads), scores to the workspace, per-piece moments;
-//   barrier ONE grid-wide barrier (Eq. 11 needs every score of a window);
-//   pass 2  per piece and query head: theta from the merged moments, ordered compaction of the
-//           selected tokens into shared memory, then only those rows of k2c / vc are read:
-//           gate = softplus(k2c[t] . q[r:]), online softmax over the survivors, value reduction;
-//           piece partials (max, sum, acc) go to the workspace and the block that finishes a
-//           segment last merges its pieces and writes o.
+//   pass 1  s_t = k1c[t] . q[:r] for the query heads of the KV group.  Half a warp reads one token
+//           row (coalesced 16-byte loads, eight rows in flight per lane); the sixteen partial sums
+//           of eight tokens are reduced with a butterfly that leaves one token per lane pair
+//           (one shuffle per token and head instead of four).  Scores stay in shared memory; the
+//           piece's sum and sum of squares (fp64) go to the (sequence, head) cells, followed by the
+//           released arrival.
+//   wait    a warp per head polls that head's cells until every piece of the segment has arrived
+//           and forms theta (Eq. 11); no grid-wide barrier: only the blocks that share a segment
+//           wait for one another.
+//   pass 2  every warp selects among its own tokens (ballot), and only for those reads the k2c and
+//           vc rows: gate = softplus(k2c[t] . q[r:]), online softmax over the survivors, value
+//           reduction; the block combines its warps into a piece partial (max, sum, acc); the
+//           block that completes a segment last merges its pieces and writes o.
 #include "kernels.h"
 
 using namespace spark;
@@ -22,8 +28,6 @@ namespace {
 
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / kWarp;
-constexpr int kHalves = 2 * kWarps;   // half-warps
-constexpr int kCH = 2048;             // tokens per selection list
 constexpr int kZc = 4;                // pieces per block whose quantile is cached between the passes
 constexpr int kPartPad = 8;           // floats in front of a partial accumulator: [0] max, [1] sum
 
@@ -35,14 +39,17 @@ struct AttnParams {
     int B, n_q, n_kv, hd, r;
     int64_t cap;
     const int32_t* ctx_len;
+    const double* zs;  // nullable: Q(1 - k_attn / L_b) per sequence, precomputed by an earlier kernel
     int window, k_attn, dense;
     float* o;
     float* theta;
     int32_t* count;
     int32_t* idx;
     int64_t idx_cap;
-    float* scores;     // [B][n_q][cap]
-    float4* pstats;    // [pieces][GQ]
+    float* scores;     // fallback when a block's scores do not fit in shared memory: [grid][GQ][ntok]
+    int ntok;          // capacity (tokens) of a block's score buffer
+    int sc_smem;       // 1: scores live in shared memory
+    SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
     float* part;       // [pieces][GQ][hd + kPartPad]
     WsHeader* hdr;
     PhaseTrace trace;
@@ -60,23 +67,6 @@ __device__ __forceinline__ float half_sum(float v) {   // sum over the 16 lanes 
     return v;
 }
 
-// Rank of this thread's flag among the block's flags in thread order, and their total.
-__device__ __forceinline__ int block_rank(bool flag, int* wcnt, int& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const unsigned bal = __ballot_sync(kFull, flag);
-    if (lane == 0) wcnt[warp] = __popc(bal);
-    __syncthreads();
-    int before = 0, all = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        if (w < warp) before += wcnt[w];
-        all += wcnt[w];
-    }
-    __syncthreads();
-    total = all;
-    return before + __popc(bal & ((1u << lane) - 1u));
-}
-
 template <typename KT, int GQ>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -84,24 +74,24 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     const int hd = p.hd, r = p.r, d2 = hd - r;
     int* segoff = reinterpret_cast<int*>(smem_raw);                       // [NS + 1], padded
     float* qs = reinterpret_cast<float*>(segoff + ((NS + 1 + 3) & ~3));   // [GQ][hd]
-    int* sel_t = reinterpret_cast<int*>(qs + GQ * hd);                    // [kCH]
-    float* sel_a = reinterpret_cast<float*>(sel_t + kCH);                 // [kCH]
-    float* wpart = sel_a + kCH;                                           // [kWarps][hd + kPartPad]
-    __shared__ float s_mom[kHalves][GQ][3];
+    float* wpart = qs + GQ * hd;                                          // [kWarps][hd + kPartPad]
+    float* sc_s = wpart + kWarps * (hd + kPartPad);                       // [GQ][ntok] when sc_smem
+    __shared__ double red[kWarps][GQ][2];
     __shared__ float theta_s[GQ];
     __shared__ double zcache[kZc];
     __shared__ double s_z;
-    __shared__ int wcnt[kWarps];
-    __shared__ int s_base, s_last;
+    __shared__ int s_last, s_fail;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int half = lane >> 4, hl = lane & 15, hw = warp * 2 + half;
+    const int half = lane >> 4, hl = lane & 15;
     const int G = gridDim.x, cta = blockIdx.x;
     const int nc1 = r / 8, nc2 = d2 / 8, ncv = hd / 8;
     const int pstride = hd + kPartPad;
     const KT* k1c = static_cast<const KT*>(p.k1c);
     const KT* k2c = static_cast<const KT*>(p.k2c);
     const KT* vc = static_cast<const KT*>(p.vc);
+    float* sc = p.sc_smem ? sc_s : p.scores + static_cast<size_t>(cta) * GQ * p.ntok;
+    const int ntok = p.ntok;
 
     auto seq_len = [&](int b) -> int {            // valid tokens of sequence b, clamped into [1, cap]
         int n = p.ctx_len[b];
@@ -111,6 +101,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     auto win_len = [&](int n) -> int { return (p.window > 0 && p.window < n) ? p.window : n; };
 
     // ---- flat layout: prefix sums of the window lengths over the segments -------------------------
+    if (tid == 32) s_fail = 0;
     if (warp == 0) {
         int run = 0;
         for (int s0 = 0; s0 < NS; s0 += 32) {
@@ -127,6 +118,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
         if (lane == 0) segoff[0] = 0;
     }
     __syncthreads();
+    p.trace.mark(0);
+    SumCell* cells = p.cells;
     const int64_t T = segoff[NS];
     const int Gp = T < G ? static_cast<int>(T) : G;        // blocks that own a non-empty range
     const bool has = cta < Gp;
@@ -141,10 +134,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
         seg0 = lo;
     }
     auto cta_of = [&](int64_t f) -> int { return static_cast<int>(((f + 1) * Gp - 1) / T); };
-
-    GridBarrier bar{p.hdr, static_cast<unsigned>(G), 0u, 0u};
-    bar.begin();
-    p.trace.mark(0);
+    // tokens of a piece that warp w owns: [w0, w1), runs of a multiple of 16 tokens
+    auto warp_range = [&](int tb, int te, int& w0, int& w1) {
+        const int n = te - tb;
+        const int cw = (((n + kWarps - 1) / kWarps) + 15) & ~15;
+        w0 = tb + warp * cw;
+        w1 = w0 + cw;
+        if (w0 > te) w0 = te;
+        if (w1 > te) w1 = te;
+    };
 
     // =============================== pass 1: predictor scores =====================================
     {
@@ -155,74 +153,100 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int te = static_cast<int>((f1 < se ? f1 : se) - sb);
             const int b = seg / p.n_kv, g = seg - b * p.n_kv;
             const int lo = seq_len(b) - L;
+            const int off = static_cast<int>(f - f0) - tb;           // score slot of token t: off + t
             for (int i = tid; i < GQ * hd; i += kThreads) qs[i] = p.q[(static_cast<int64_t>(b) * p.n_q + g * GQ) * hd + i];
             if (tb == 0 && p.count != nullptr && tid < GQ) p.count[b * p.n_q + g * GQ + tid] = 0;
             if (tid == kThreads - 1 && ord < kZc)
-                zcache[ord] = p.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L));
+                zcache[ord] = p.k_attn >= L ? 0.0
+                              : (p.zs != nullptr ? p.zs[b] : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
             __syncthreads();
             float qreg[GQ][8];
 #pragma unroll
             for (int hq = 0; hq < GQ; ++hq)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) qreg[hq][e] = hl < nc1 ? qs[hq * hd + hl * 8 + e] : 0.f;
-            float wn = 0.f, wmean[GQ], wm2[GQ];
+            double s1[GQ], s2[GQ];
 #pragma unroll
-            for (int hq = 0; hq < GQ; ++hq) { wmean[hq] = 0.f; wm2[hq] = 0.f; }
+            for (int hq = 0; hq < GQ; ++hq) { s1[hq] = 0.0; s2[hq] = 0.0; }
             const KT* kbase = k1c + (static_cast<int64_t>(seg) * p.cap + lo) * r;
-            float* sbase = p.scores + (static_cast<int64_t>(b) * p.n_q + g * GQ) * p.cap + lo;
-            for (int ib = tb + warp * 2; ib < te; ib += kHalves * 4) {   // warp-uniform trip count
-                const int i0 = ib + half;
-                Row8<KT> w[4];
+            int w0, w1;
+            warp_range(tb, te, w0, w1);
+            const int jidx = ((hl >> 3) & 1) * 4 + ((hl >> 2) & 1) * 2 + ((hl >> 1) & 1);
+#pragma unroll 1
+            for (int base = w0; base < w1; base += 16) {
+                const int tok0 = base + half * 8;
+                Row8<KT> w[8];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * kHalves;
-                    if (i < te && hl < nc1) w[u].load(kbase + static_cast<int64_t>(i) * r, hl);
-                    else w[u].zero();
+                for (int j = 0; j < 8; ++j) {
+                    if (tok0 + j < w1 && hl < nc1) w[j].load(kbase + static_cast<int64_t>(tok0 + j) * r, hl);
+                    else w[j].zero();
                 }
+                float pj[8][GQ];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int i = i0 + u * kHalves;
+                for (int j = 0; j < 8; ++j) {
                     float wf[8];
-                    w[u].unpack(wf);
-                    float sc[GQ];
+                    w[j].unpack(wf);
 #pragma unroll
-                    for (int hq = 0; hq < GQ; ++hq) sc[hq] = half_sum(dot8r(wf, qreg[hq]));
-                    if (hl == 0 && i < te) {
-                        wn += 1.f;
-                        const float inv = 1.f / wn;
+                    for (int hq = 0; hq < GQ; ++hq) pj[j][hq] = dot8r(wf, qreg[hq]);
+                }
+                // butterfly over the 16 lanes of the half-warp: 8 tokens -> 4 -> 2 -> 1 per lane
+                float a4[4][GQ], a2[2][GQ], a1[GQ];
+                const bool b8 = hl & 8, b4 = hl & 4, b2 = hl & 2;
 #pragma unroll
-                        for (int hq = 0; hq < GQ; ++hq) {
-                            sbase[static_cast<int64_t>(hq) * p.cap + i] = sc[hq];
-                            const float dl = sc[hq] - wmean[hq];
-                            wmean[hq] += dl * inv;
-                            wm2[hq] = fmaf(dl, sc[hq] - wmean[hq], wm2[hq]);
-                        }
+                for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                    for (int hq = 0; hq < GQ; ++hq) {
+                        const float keep = b8 ? pj[jj + 4][hq] : pj[jj][hq];
+                        const float send = b8 ? pj[jj][hq] : pj[jj + 4][hq];
+                        a4[jj][hq] = keep + __shfl_xor_sync(kFull, send, 8);
+                    }
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+                    for (int hq = 0; hq < GQ; ++hq) {
+                        const float keep = b4 ? a4[jj + 2][hq] : a4[jj][hq];
+                        const float send = b4 ? a4[jj][hq] : a4[jj + 2][hq];
+                        a2[jj][hq] = keep + __shfl_xor_sync(kFull, send, 4);
+                    }
+#pragma unroll
+                for (int hq = 0; hq < GQ; ++hq) {
+                    const float keep = b2 ? a2[1][hq] : a2[0][hq];
+                    const float send = b2 ? a2[0][hq] : a2[1][hq];
+                    a1[hq] = keep + __shfl_xor_sync(kFull, send, 2);
+                    a1[hq] += __shfl_xor_sync(kFull, a1[hq], 1);
+                }
+                const int t = tok0 + jidx;
+                if ((hl & 1) == 0 && t < w1) {
+#pragma unroll
+                    for (int hq = 0; hq < GQ; ++hq) {
+                        sc[static_cast<size_t>(hq) * ntok + off + t] = a1[hq];
+                        const double v = static_cast<double>(a1[hq]);
+                        s1[hq] += v;
+                        s2[hq] = fma(v, v, s2[hq]);
                     }
                 }
             }
-            if (hl == 0) {
 #pragma unroll
-                for (int hq = 0; hq < GQ; ++hq) {
-                    s_mom[hw][hq][0] = wn; s_mom[hw][hq][1] = wmean[hq]; s_mom[hw][hq][2] = wm2[hq];
-                }
+            for (int hq = 0; hq < GQ; ++hq) {
+                const double a = warp_sum_f64(s1[hq]), c = warp_sum_f64(s2[hq]);
+                if (lane == 0) { red[warp][hq][0] = a; red[warp][hq][1] = c; }
             }
             __syncthreads();
             if (warp < GQ) {
-                Moments m{static_cast<double>(s_mom[lane][warp][0]), static_cast<double>(s_mom[lane][warp][1]),
-                          static_cast<double>(s_mom[lane][warp][2])};
-                m = warp_merge(m);
+                double a = lane < kWarps ? red[lane][warp][0] : 0.0, c = lane < kWarps ? red[lane][warp][1] : 0.0;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) {
+                    a += __shfl_xor_sync(kFull, a, o);
+                    c += __shfl_xor_sync(kFull, c, o);
+                }
                 if (lane == 0)
-                    p.pstats[static_cast<size_t>(cta + seg) * GQ + warp] =
-                        make_float4(static_cast<float>(m.n), static_cast<float>(m.mean), static_cast<float>(m.m2), 0.f);
+                    cells_add_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays, cta, a, c);
             }
             __syncthreads();
             f = sb + te;
         }
     }
     p.trace.mark(1);
-    bar.arrive();
-    if (!bar.wait()) return;
-    p.trace.mark(2);
 
     // =============================== pass 2: select, gather, reduce ================================
     {
@@ -233,119 +257,149 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int te = static_cast<int>((f1 < se ? f1 : se) - sb);
             const int b = seg / p.n_kv, g = seg - b * p.n_kv;
             const int lo = seq_len(b) - L;
+            const int off = static_cast<int>(f - f0) - tb;
             const bool ident = p.k_attn >= L;
             const int c_lo = cta_of(sb), c_hi = cta_of(static_cast<int64_t>(se) - 1);
             const size_t pid = static_cast<size_t>(cta + seg);
             for (int i = tid; i < GQ * hd; i += kThreads) qs[i] = p.q[(static_cast<int64_t>(b) * p.n_q + g * GQ) * hd + i];
             if (ord >= kZc && tid == 0)
-                s_z = ident ? 0.0 : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L));
+                s_z = ident ? 0.0 : (p.zs != nullptr ? p.zs[b] : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
             __syncthreads();
-            if (warp < GQ) {
-                Moments m{0.0, 0.0, 0.0};
-                for (int c = c_lo + lane; c <= c_hi; c += 32) {
-                    const float4 v = ld_cg_f4(&p.pstats[static_cast<size_t>(c + seg) * GQ + warp]);
-                    m = merge(m, Moments{static_cast<double>(v.x), static_cast<double>(v.y), static_cast<double>(v.z)});
-                }
-                m = warp_merge(m);
-                const double z = ord < kZc ? zcache[ord] : s_z;
-                const float th = ident ? -INFINITY : theta_from(m, z);
+            if (warp < GQ) {        // theta of this head once every piece of the segment has arrived
+                double sa, sq;
+                const bool ok = cells_wait_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays,
+                                                        static_cast<unsigned>(c_hi - c_lo + 1), sa, sq, p.hdr);
                 if (lane == 0) {
+                    if (!ok) s_fail = 1;
+                    float th = -INFINITY;
+                    if (!ident) {
+                        const double z = ord < kZc ? zcache[ord] : s_z;
+                        const double n = static_cast<double>(L), mean = sa / n;
+                        double var = (sq - sa * mean) / (n - 1.0);
+                        var = var > 0.0 ? var : 0.0;
+                        th = static_cast<float>(mean + sqrt(var) * z);
+                    }
                     theta_s[warp] = th;
                     if (tb == 0 && p.theta != nullptr) p.theta[b * p.n_q + g * GQ + warp] = th;
                 }
             }
             __syncthreads();
+            if (s_fail) return;
+            if (ord == 0) p.trace.mark(2);
             const KT* k2base = k2c + static_cast<int64_t>(seg) * p.cap * d2;
             const KT* vbase = vc + static_cast<int64_t>(seg) * p.cap * hd;
-
+            // In this pass warp w serves query head w % GQ; the kWarps / GQ warps of a head split the
+            // piece's tokens into contiguous runs (multiples of 32 tokens).
+            constexpr int NSUB = kWarps / GQ;
+            const int hq = warp % GQ, wsub = warp / GQ;
+            int w0, w1;
+            {
+                const int n = te - tb;
+                const int cw = (((n + NSUB - 1) / NSUB) + 31) & ~31;
+                w0 = tb + wsub * cw;
+                w1 = w0 + cw;
+                if (w0 > te) w0 = te;
+                if (w1 > te) w1 = te;
+            }
+            const float th = theta_s[hq];
+            const int bh = b * p.n_q + g * GQ + hq;
+            float q2[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) q2[e] = hl < nc2 ? qs[hq * hd + r + hl * 8 + e] : 0.f;
+            float m_w = -INFINITY, l_w = 0.f, acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+            const float* srow = sc + static_cast<size_t>(hq) * ntok + off;
 #pragma unroll 1
-            for (int hq = 0; hq < GQ; ++hq) {
-                const float th = theta_s[hq];
-                const int bh = b * p.n_q + g * GQ + hq;
-                float q2[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) q2[e] = hl < nc2 ? qs[hq * hd + r + hl * 8 + e] : 0.f;
-                float m_w = -INFINITY, l_w = 0.f, acc[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-                const float* srow = p.scores + static_cast<int64_t>(bh) * p.cap + lo;
-
-                for (int c0 = tb; c0 < te; c0 += kCH) {
-                    const int c1 = te < c0 + kCH ? te : c0 + kCH;
-                    int nlist = 0;
-                    for (int j0 = c0; j0 < c1; j0 += kThreads) {
-                        const int i = j0 + tid;
-                        const bool valid = i < c1;
-                        const float s = valid ? __ldcg(srow + i) : 0.f;
-                        const bool sel = valid && (ident || s > th);
-                        const bool in = valid && (sel || p.dense);
-                        int tot;
-                        const int rank = block_rank(in, wcnt, tot);
-                        if (in) {
-                            sel_t[nlist + rank] = lo + i;
-                            sel_a[nlist + rank] = sel ? (ident ? s : s - th) : -INFINITY;
-                        }
-                        nlist += tot;
-                        if (p.count != nullptr) {
-                            int nt;
-                            const int rk = p.dense ? block_rank(sel, wcnt, nt) : rank;
-                            if (!p.dense) nt = tot;
-                            if (nt > 0) {
-                                if (tid == 0) s_base = atomicAdd(&p.count[bh], nt);
-                                __syncthreads();
-                                const int64_t pos = static_cast<int64_t>(s_base) + rk;
-                                if (sel && p.idx != nullptr) {
-                                    if (pos < p.idx_cap) p.idx[static_cast<int64_t>(bh) * p.idx_cap + pos] = lo + i;
-                                    else atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_OVERFLOW);
-                                }
-                                __syncthreads();
-                            }
-                        }
+            for (int base = w0; base < w1; base += 32) {
+                const int t = base + lane;
+                const bool valid = t < w1;
+                const float s = valid ? srow[t] : 0.f;
+                const bool sel = valid && (ident || s > th);
+                const float a = sel ? (ident ? s : s - th) : -INFINITY;
+                const unsigned bsel = __ballot_sync(kFull, sel);
+                unsigned bal = p.dense ? __ballot_sync(kFull, valid) : bsel;
+                if (p.count != nullptr && bsel != 0u) {
+                    int cbase = 0;
+                    if (lane == 0) cbase = atomicAdd(&p.count[bh], __popc(bsel));
+                    cbase = __shfl_sync(kFull, cbase, 0);
+                    if (sel && p.idx != nullptr) {
+                        const int64_t pos = static_cast<int64_t>(cbase) + __popc(bsel & ((1u << lane) - 1u));
+                        if (pos < p.idx_cap) p.idx[static_cast<int64_t>(bh) * p.idx_cap + pos] = lo + t;
+                        else atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_OVERFLOW);
                     }
-                    __syncthreads();
-                    const int npairs = (nlist + 1) >> 1;
-                    for (int pi = warp; pi < npairs; pi += kWarps) {
-                        const int e0 = 2 * pi, e1 = e0 + 1;
-                        const bool v1 = e1 < nlist;
-                        const int t0 = sel_t[e0], t1 = v1 ? sel_t[e1] : t0;
-                        const float a0 = sel_a[e0], a1 = v1 ? sel_a[e1] : -INFINITY;
-                        const int tm = half ? t1 : t0;
-                        Row8<KT> kw, v0w, v1w;
-                        if ((half == 0 || v1) && hl < nc2) kw.load(k2base + static_cast<int64_t>(tm) * d2, hl);
-                        else kw.zero();
-                        if (lane < ncv) v0w.load(vbase + static_cast<int64_t>(t0) * hd, lane);
-                        else v0w.zero();
-                        if (lane < ncv && v1) v1w.load(vbase + static_cast<int64_t>(t1) * hd, lane);
-                        else v1w.zero();
-                        float wf[8];
-                        kw.unpack(wf);
-                        const float gate = softplus(half_sum(dot8r(wf, q2)));
-                        const float g0 = __shfl_sync(kFull, gate, 0), g1 = __shfl_sync(kFull, gate, 16);
-                        const float mn = fmaxf(m_w, fmaxf(a0, a1));
-                        if (mn != -INFINITY) {
-                            const float sc = m_w == -INFINITY ? 0.f : expf(m_w - mn);
-                            const float p0 = a0 == -INFINITY ? 0.f : expf(a0 - mn);
-                            const float p1 = a1 == -INFINITY ? 0.f : expf(a1 - mn);
-                            l_w = l_w * sc + p0 + p1;
-                            const float w0 = p0 * g0, w1 = p1 * g1;
-                            float f0v[8], f1v[8];
-                            v0w.unpack(f0v);
-                            v1w.unpack(f1v);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w1, f1v[e], fmaf(w0, f0v[e], acc[e] * sc));
-                            m_w = mn;
-                        } else if (p.dense) {
-                            // nothing selected so far: the rows were still read; keep the loads alive
-                            float f0v[8], f1v[8];
-                            v0w.unpack(f0v);
-                            v1w.unpack(f1v);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) acc[e] = fmaf(0.f * g0, f0v[e], fmaf(0.f * g1, f1v[e], acc[e]));
-                        }
-                    }
-                    __syncthreads();
                 }
-                // ---- combine the warps' online-softmax states into the piece partial ---------------
+                while (bal != 0u) {          // four listed tokens per trip: their rows are requested together
+                    int l[4];
+                    bool v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        v[i] = bal != 0u;
+                        l[i] = v[i] ? __ffs(bal) - 1 : 0;
+                        if (v[i]) bal &= bal - 1u;
+                    }
+                    float av[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float x = __shfl_sync(kFull, a, l[i]);
+                        av[i] = v[i] ? x : -INFINITY;
+                    }
+                    Row8<KT> kw[2], vw[4];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {      // half h reads the k2c rows of tokens h and h + 2
+                        const bool vv = half ? v[1 + 2 * i] : v[2 * i];
+                        const int ll = half ? l[1 + 2 * i] : l[2 * i];
+                        if (vv && hl < nc2) kw[i].load(k2base + static_cast<int64_t>(lo + base + ll) * d2, hl);
+                        else kw[i].zero();
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        if (v[i] && lane < ncv) vw[i].load(vbase + static_cast<int64_t>(lo + base + l[i]) * hd, lane);
+                        else vw[i].zero();
+                    }
+                    float gt[4];
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        float wf[8];
+                        kw[i].unpack(wf);
+                        const float gate = softplus(half_sum(dot8r(wf, q2)));
+                        gt[2 * i] = __shfl_sync(kFull, gate, 0);
+                        gt[2 * i + 1] = __shfl_sync(kFull, gate, 16);
+                    }
+                    const float mn = fmaxf(fmaxf(m_w, fmaxf(av[0], av[1])), fmaxf(av[2], av[3]));
+                    float wt[4] = {0.f, 0.f, 0.f, 0.f};
+                    float scl = 1.f;
+                    if (mn != -INFINITY) {
+                        scl = m_w == -INFINITY ? 0.f : expf(m_w - mn);
+                        float add = 0.f;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float pe = av[i] == -INFINITY ? 0.f : expf(av[i] - mn);
+                            add += pe;
+                            wt[i] = pe * gt[i];
+                        }
+                        l_w = l_w * scl + add;
+                        m_w = mn;
+                    } else {
+                        // nothing selected so far: the rows were read (dense comparator); keep the loads alive
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) wt[i] = 0.f * gt[i];
+                    }
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] *= scl;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        float fv[8];
+                        vw[i].unpack(fv);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) acc[e] = fmaf(wt[i], fv[e], acc[e]);
+                    }
+                }
+            }
+            // ---- combine the warps' online-softmax states into one (max, sum, acc) per head --------------
+            // Entry w of wpart belongs to head w % GQ.  `final_out`: normalise and write o; else write the
+            // piece partial to the workspace.
+            auto combine = [&](bool final_out) {
                 float* wp = wpart + warp * pstride;
                 if (lane == 0) { wp[0] = m_w; wp[1] = l_w; }
                 if (lane < ncv) {
@@ -353,71 +407,77 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     for (int e = 0; e < 8; ++e) wp[kPartPad + lane * 8 + e] = acc[e];
                 }
                 __syncthreads();
-                float M = -INFINITY;
+                for (int i = tid; i < GQ * hd; i += kThreads) {
+                    const int h = i / hd, dd = i - h * hd;
+                    float M = -INFINITY;
 #pragma unroll
-                for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wpart[w * pstride]);
-                float* dst = p.part + (pid * GQ + hq) * pstride;
-                for (int dd = tid; dd < hd; dd += kThreads) {
-                    float sum = 0.f;
+                    for (int u = 0; u < NSUB; ++u) M = fmaxf(M, wpart[(u * GQ + h) * pstride]);
+                    float sum = 0.f, l = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kWarps; ++w) {
-                        const float mw = wpart[w * pstride];
-                        if (mw != -INFINITY) sum = fmaf(expf(mw - M), wpart[w * pstride + kPartPad + dd], sum);
+                    for (int u = 0; u < NSUB; ++u) {
+                        const float* e = wpart + (u * GQ + h) * pstride;
+                        if (e[0] != -INFINITY) {
+                            const float w = expf(e[0] - M);
+                            sum = fmaf(w, e[kPartPad + dd], sum);
+                            l = fmaf(w, e[1], l);
+                        }
                     }
-                    dst[kPartPad + dd] = sum;
-                }
-                if (tid == 0) {
-                    float l = 0.f;
-                    for (int w = 0; w < kWarps; ++w) {
-                        const float mw = wpart[w * pstride];
-                        if (mw != -INFINITY) l = fmaf(expf(mw - M), wpart[w * pstride + 1], l);
+                    if (final_out) {
+                        p.o[(static_cast<int64_t>(b) * p.n_q + g * GQ + h) * hd + dd] = l > 0.f ? sum / l : 0.f;
+                    } else {
+                        float* dst = p.part + (pid * GQ + h) * pstride;
+                        dst[kPartPad + dd] = sum;
+                        if (dd == 0) { dst[0] = M; dst[1] = l; }
                     }
-                    dst[0] = M;
-                    dst[1] = l;
                 }
                 __syncthreads();
-            }
+            };
+            const bool single = c_lo == c_hi;       // the whole segment lies in this block: no merge needed
+            combine(single);
 
             // ---- the block that completes a segment last merges its pieces and writes o -------------
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) {
-                const unsigned prev = atom_add_acqrel_u32(&p.hdr->seg_done[seg], 1u);
-                const int last = prev == static_cast<unsigned>(c_hi - c_lo);
-                if (last) p.hdr->seg_done[seg] = 0u;
-                s_last = last;
+            if (!single) {
+                if (tid == 0) {
+                    __threadfence();
+                    const unsigned prev = atom_add_acqrel_u32(&p.hdr->seg_done[seg], 1u);
+                    const int last = prev == static_cast<unsigned>(c_hi - c_lo);
+                    if (last) p.hdr->seg_done[seg] = 0u;
+                    s_last = last;
+                }
+                __syncthreads();
+                if (s_last) {
+                    // warp w merges pieces c_lo + w / GQ, + NSUB, ... of head w % GQ, then the warps combine
+                    m_w = -INFINITY; l_w = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+                    for (int c = c_lo + wsub; c <= c_hi; c += NSUB) {
+                        const float* src = p.part + (static_cast<size_t>(c + seg) * GQ + hq) * pstride;
+                        const float mp = __ldcg(src), lp = __ldcg(src + 1);
+                        float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0;
+                        if (lane < ncv) {
+                            x0 = __ldcg(reinterpret_cast<const float4*>(src + kPartPad + lane * 8));
+                            x1 = __ldcg(reinterpret_cast<const float4*>(src + kPartPad + lane * 8 + 4));
+                        }
+                        if (mp == -INFINITY) continue;
+                        const float mn = fmaxf(m_w, mp);
+                        const float sa = m_w == -INFINITY ? 0.f : expf(m_w - mn), sb2 = expf(mp - mn);
+                        l_w = l_w * sa + lp * sb2;
+                        acc[0] = fmaf(sb2, x0.x, acc[0] * sa); acc[1] = fmaf(sb2, x0.y, acc[1] * sa);
+                        acc[2] = fmaf(sb2, x0.z, acc[2] * sa); acc[3] = fmaf(sb2, x0.w, acc[3] * sa);
+                        acc[4] = fmaf(sb2, x1.x, acc[4] * sa); acc[5] = fmaf(sb2, x1.y, acc[5] * sa);
+                        acc[6] = fmaf(sb2, x1.z, acc[6] * sa); acc[7] = fmaf(sb2, x1.w, acc[7] * sa);
+                        m_w = mn;
+                    }
+                    combine(true);
+                }
+            } else if (tid == 0) {
+                s_last = 1;
             }
             __syncthreads();
-            if (s_last && warp < GQ) {
-                const int hq = warp;
-                float M = -INFINITY;
-                for (int c = c_lo + lane; c <= c_hi; c += 32)
-                    M = fmaxf(M, __ldcg(p.part + (static_cast<size_t>(c + seg) * GQ + hq) * pstride));
-                M = warp_max(M);
-                float Lsum = 0.f, out[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) out[e] = 0.f;
-                for (int c = c_lo; c <= c_hi; ++c) {
-                    const float* src = p.part + (static_cast<size_t>(c + seg) * GQ + hq) * pstride;
-                    const float mp = __ldcg(src);
-                    if (mp == -INFINITY) continue;
-                    const float w = expf(mp - M);
-                    Lsum = fmaf(w, __ldcg(src + 1), Lsum);
-                    if (lane < ncv) {
-                        const float4 a = __ldcg(reinterpret_cast<const float4*>(src + kPartPad + lane * 8));
-                        const float4 c4 = __ldcg(reinterpret_cast<const float4*>(src + kPartPad + lane * 8 + 4));
-                        out[0] = fmaf(w, a.x, out[0]); out[1] = fmaf(w, a.y, out[1]);
-                        out[2] = fmaf(w, a.z, out[2]); out[3] = fmaf(w, a.w, out[3]);
-                        out[4] = fmaf(w, c4.x, out[4]); out[5] = fmaf(w, c4.y, out[5]);
-                        out[6] = fmaf(w, c4.z, out[6]); out[7] = fmaf(w, c4.w, out[7]);
-                    }
-                }
-                const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-                if (lane < ncv) {
-                    float* od = p.o + (static_cast<int64_t>(b) * p.n_q + g * GQ + hq) * hd + lane * 8;
-                    reinterpret_cast<float4*>(od)[0] = make_float4(out[0] * inv, out[1] * inv, out[2] * inv, out[3] * inv);
-                    reinterpret_cast<float4*>(od)[1] = make_float4(out[4] * inv, out[5] * inv, out[6] * inv, out[7] * inv);
-                }
+            // every piece of the segment has read the cells by now: leave them zero for the next launch
+            if (s_last && tid < GQ * kAttnWays) {
+                SumCell* c = cells + static_cast<size_t>(b * p.n_q + g * GQ) * kAttnWays + tid;
+                c->s1 = 0.0; c->s2 = 0.0; c->count = 0u;
             }
             __syncthreads();
             f = sb + te;
@@ -461,11 +521,12 @@ int launch_gq(spark_ctx* ctx, AttnParams& p, int gq, size_t smem, cudaStream_t s
 
 }  // namespace
 
-extern "C" int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc,
-                                 int kvdtype, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd, int64_t r,
-                                 int64_t cap, const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags,
-                                 float* o, float* theta, int32_t* count, int32_t* idx, int64_t idx_cap,
-                                 void* stream) {
+namespace spark {
+
+int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
+                int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
+                int64_t window, int64_t k_attn, int flags, float* o, float* theta, int32_t* count, int32_t* idx,
+                int64_t idx_cap, cudaStream_t st) {
     if (ctx == nullptr || q == nullptr || k1c == nullptr || k2c == nullptr || vc == nullptr || ctx_len == nullptr ||
         o == nullptr)
         return SPARK_ERR_INVALID_ARG;
@@ -482,31 +543,50 @@ extern "C" int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
 
     const int grid = ctx->num_sms;
+    const int64_t span = (window > 0 && window < cap) ? window : cap;          // longest window of a sequence
+    const int64_t ntok = (B * n_kv * span + grid - 1) / grid + 1;            // tokens one block may own
     const size_t pieces = static_cast<size_t>(grid) + static_cast<size_t>(B * n_kv);
-    const size_t scores_b = round_up(static_cast<size_t>(B * n_q * cap) * 4, 256);
-    const size_t pstats_b = round_up(pieces * gq * sizeof(float4), 256);
+    // The cells keep a fixed place and size in the workspace whatever the call's shape: they must be
+    // zero between launches, so nothing else may ever be written there.
+    const size_t cells_b = kAttnCellBytes;
+    if (static_cast<size_t>(B * n_q) * kAttnWays * sizeof(SumCell) > cells_b) return SPARK_ERR_UNSUPPORTED;
     const size_t part_b = round_up(pieces * gq * (hd + kPartPad) * 4, 256);
-    if (scores_b + pstats_b + part_b > ctx->scratch_bytes) return SPARK_ERR_WORKSPACE;
+    const size_t ns_pad = (static_cast<size_t>(B * n_kv) + 1 + 3) & ~static_cast<size_t>(3);
+    const size_t smem_fixed = ns_pad * 4 + static_cast<size_t>(gq * hd) * 4 + static_cast<size_t>(kWarps) * (hd + kPartPad) * 4;
+    const size_t smem_limit = static_cast<size_t>(ctx->max_smem_optin - 8192);
+    if (smem_fixed > smem_limit) return SPARK_ERR_UNSUPPORTED;
+    const size_t sc_bytes = static_cast<size_t>(gq) * ntok * 4;
+    const bool sc_smem = smem_fixed + sc_bytes <= smem_limit;
+    const size_t scores_b = sc_smem ? 0 : round_up(static_cast<size_t>(grid) * sc_bytes, 256);
+    if (cells_b + part_b + scores_b > ctx->scratch_bytes) return SPARK_ERR_WORKSPACE;
 
     AttnParams p;
     p.q = q; p.k1c = k1c; p.k2c = k2c; p.vc = vc;
     p.B = static_cast<int>(B); p.n_q = static_cast<int>(n_q); p.n_kv = static_cast<int>(n_kv);
-    p.hd = static_cast<int>(hd); p.r = static_cast<int>(r); p.cap = cap; p.ctx_len = ctx_len;
+    p.hd = static_cast<int>(hd); p.r = static_cast<int>(r); p.cap = cap; p.ctx_len = ctx_len; p.zs = zs;
     p.window = static_cast<int>(window > 0x7fffffff ? 0x7fffffff : window);
     p.k_attn = static_cast<int>(k_attn > 0x7fffffff ? 0x7fffffff : k_attn);
     p.dense = (flags & SPARK_DENSE_LOADS) ? 1 : 0;
     p.o = o; p.theta = theta; p.count = count; p.idx = idx; p.idx_cap = idx_cap;
-    p.scores = reinterpret_cast<float*>(ctx->scratch);
-    p.pstats = reinterpret_cast<float4*>(ctx->scratch + scores_b);
-    p.part = reinterpret_cast<float*>(ctx->scratch + scores_b + pstats_b);
+    p.cells = reinterpret_cast<SumCell*>(ctx->scratch);
+    p.part = reinterpret_cast<float*>(ctx->scratch + cells_b);
+    p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
+    p.ntok = static_cast<int>(ntok);
+    p.sc_smem = sc_smem ? 1 : 0;
     p.hdr = ctx->hdr;
     p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
-
-    const size_t ns_pad = (static_cast<size_t>(B * n_kv) + 1 + 3) & ~static_cast<size_t>(3);
-    const size_t smem = ns_pad * 4 + static_cast<size_t>(gq * hd) * 4 + static_cast<size_t>(kCH) * 8 +
-                        static_cast<size_t>(kWarps) * (hd + kPartPad) * 4;
-    if (smem > static_cast<size_t>(ctx->max_smem_optin - 8192)) return SPARK_ERR_UNSUPPORTED;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t smem = smem_fixed + (sc_smem ? sc_bytes : 0);
     if (kvdtype == SPARK_BF16) return launch_gq<__nv_bfloat16>(ctx, p, static_cast<int>(gq), smem, st);
     return launch_gq<float>(ctx, p, static_cast<int>(gq), smem, st);
+}
+
+}  // namespace spark
+
+extern "C" int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc,
+                                 int kvdtype, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd, int64_t r,
+                                 int64_t cap, const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags,
+                                 float* o, float* theta, int32_t* count, int32_t* idx, int64_t idx_cap,
+                                 void* stream) {
+    return attn_launch(ctx, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv, hd, r, cap, ctx_len, nullptr, window, k_attn, flags, o,
+                       theta, count, idx, idx_cap, static_cast<cudaStream_t>(stream));
 }

@@ -28,7 +28,11 @@ struct __align__(32) SumCell {
 // single cell would serialise 3 x #blocks atomics on one address, which costs microseconds.
 constexpr int kCellWays = 16;
 
-constexpr int kMaxSegments = 2048;   // (sequence, KV head) pairs one attention call may cover
+constexpr int kMaxSegments = 2048;
+// Attention keeps kAttnWays cells per (sequence, query head) in a fixed region at the start of the
+// workspace scratch (room for 16384 heads).
+constexpr int kAttnWays = 4;
+constexpr size_t kAttnCellBytes = static_cast<size_t>(16384) * kAttnWays * 32;   // (sequence, KV head) pairs one attention call may cover
 
 struct WsHeader {            // lives at the start of the caller's workspace; zero when idle
     int status;              // device status word (SPARK_OK or a SPARK_ERR_* device code)
@@ -316,29 +320,32 @@ __device__ __forceinline__ void ld_cell(const SumCell* c, double& s1, double& s2
 }
 // Add this block's two sums to its way of a cell group, then its arrival (release: ordered after
 // the sums and after everything the block wrote before).  One thread calls this.
-__device__ __forceinline__ void cells_add(SumCell* ways, int block, double s1, double s2) {
-    SumCell* c = ways + (block % kCellWays);
+template <int WAYS>
+__device__ __forceinline__ void cells_add_w(SumCell* ways, int block, double s1, double s2) {
+    SumCell* c = ways + (block % WAYS);
     red_add_f64(&c->s1, s1);
     red_add_f64(&c->s2, s2);
     red_release_add_u32(&c->count, 1u);
 }
-// Lanes 0..15 of one warp poll the 16 ways (one 32-byte acquire load each) until all `nblocks`
+// Lanes 0..WAYS-1 of one warp poll the ways (one 32-byte acquire load each) until all `nblocks`
 // blocks have arrived, then every lane of the warp gets the totals.  Called by a full warp.
 // Returns false after about two seconds (SPARK_ERR_TIMEOUT recorded).
-__device__ __forceinline__ bool cells_wait(const SumCell* ways, unsigned nblocks, double& s1, double& s2, WsHeader* hdr) {
+template <int WAYS>
+__device__ __forceinline__ bool cells_wait_w(const SumCell* ways, unsigned nblocks, double& s1, double& s2, WsHeader* hdr) {
+    static_assert(WAYS == 1 || WAYS == 2 || WAYS == 4 || WAYS == 8 || WAYS == 16, "ways");
     const int lane = threadIdx.x & 31;
     const long long t0 = clock64();
     for (;;) {
         double a = 0.0, b = 0.0;
         unsigned cnt = 0u;
-        if (lane < kCellWays) ld_cell(ways + lane, a, b, cnt);
+        if (lane < WAYS) ld_cell(ways + lane, a, b, cnt);
         unsigned tot = cnt;
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) tot += __shfl_xor_sync(kFull, tot, o);
+        for (int o = WAYS / 2; o > 0; o >>= 1) tot += __shfl_xor_sync(kFull, tot, o);
         tot = __shfl_sync(kFull, tot, 0);
         if (tot == nblocks) {
 #pragma unroll
-            for (int o = 8; o > 0; o >>= 1) {
+            for (int o = WAYS / 2; o > 0; o >>= 1) {
                 a += __shfl_xor_sync(kFull, a, o);
                 b += __shfl_xor_sync(kFull, b, o);
             }
@@ -351,6 +358,12 @@ __device__ __forceinline__ bool cells_wait(const SumCell* ways, unsigned nblocks
             return false;
         }
     }
+}
+__device__ __forceinline__ void cells_add(SumCell* ways, int block, double s1, double s2) {
+    cells_add_w<kCellWays>(ways, block, s1, s2);
+}
+__device__ __forceinline__ bool cells_wait(const SumCell* ways, unsigned nblocks, double& s1, double& s2, WsHeader* hdr) {
+    return cells_wait_w<kCellWays>(ways, nblocks, s1, s2, hdr);
 }
 
 // 16-byte accesses that always go to L2 (slots other blocks write or poll).

@@ -37,4 +37,11 @@ struct GemvArgs {
 };
 int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 
+// Spark attention; zs (nullable) holds Q(1 - k_attn / L_b) per sequence when an earlier kernel of the
+// same stream has already computed it.
+int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
+                int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
+                int64_t window, int64_t k_attn, int flags, float* o, float* theta, int32_t* count, int32_t* idx,
+                int64_t idx_cap, cudaStream_t st);
+
 }  // namespace spark

@@ -104,9 +104,17 @@ struct RopeParams {
     int B, n_q, n_kv, hd, r;
     int64_t cap;
     float base, q_scale;
+    double* zs;              // [B] out: Q(1 - k_attn / L_b) for the attention kernel that follows
+    int window, k_attn;
 };
 
 __global__ void rope_append_kernel(const RopeParams p) {
+    if (blockIdx.x == 0 && threadIdx.x < p.B) {         // the threshold quantile of each sequence's window
+        int n = p.ctx_len[threadIdx.x];
+        n = n < 1 ? 1 : (n > p.cap ? static_cast<int>(p.cap) : n);
+        const int L = (p.window > 0 && p.window < n) ? p.window : n;
+        p.zs[threadIdx.x] = p.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L));
+    }
     const int heads = p.n_q + 2 * p.n_kv;
     const int half_hd = p.hd / 2;
     const int64_t total = static_cast<int64_t>(p.B) * heads * half_hd;
@@ -211,6 +219,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
         scratch == nullptr)
         return SPARK_ERR_INVALID_ARG;
     if (B < 1 || B > 16) return SPARK_ERR_INVALID_ARG;
+    if (((cfg->n_q + 2 * cfg->n_kv) * cfg->hd + 2 * cfg->n_q * cfg->hd + cfg->d) % 2 != 0) return SPARK_ERR_UNSUPPORTED;
     if (w->norm1 == nullptr || w->norm2 == nullptr || w->Wqkv == nullptr || w->Wo == nullptr || w->K1t == nullptr ||
         w->K2t == nullptr || w->Vt == nullptr || cache->k1c == nullptr || cache->k2c == nullptr || cache->vc == nullptr)
         return SPARK_ERR_INVALID_ARG;
@@ -225,6 +234,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     float* qr = qkv + B * nqkv;           // [B][n_q][hd]  position-encoded, scaled queries
     float* ao = qr + B * nqo;             // [B][n_q][hd]  attention output
     float* h2 = ao + B * nqo;             // [B][d]        h + Wo . attention
+    double* zs = reinterpret_cast<double*>(h2 + B * cfg->d);   // [B] threshold quantiles (8-byte aligned: see below)
 
     // 1. a = RMSNorm(h; norm1); [q|k|v] = Wqkv a
     GemvArgs g1;
@@ -241,6 +251,8 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     rp.ctx_len = ctx_len; rp.B = static_cast<int>(B); rp.n_q = static_cast<int>(cfg->n_q); rp.n_kv = static_cast<int>(cfg->n_kv);
     rp.hd = static_cast<int>(cfg->hd); rp.r = static_cast<int>(cfg->r_attn); rp.cap = cfg->cap;
     rp.base = cfg->rope_base; rp.q_scale = 1.0f / std::sqrt(static_cast<float>(cfg->hd));
+    rp.zs = zs; rp.window = static_cast<int>(cfg->window > 0x7fffffff ? 0x7fffffff : cfg->window);
+    rp.k_attn = static_cast<int>(cfg->k_attn > 0x7fffffff ? 0x7fffffff : cfg->k_attn);
     {
         const int64_t total = B * (cfg->n_q + 2 * cfg->n_kv) * (cfg->hd / 2);
         const int blocks = static_cast<int>((total + 255) / 256);
@@ -249,9 +261,9 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     }
 
     // 3. Spark attention over the cache (the new token included)
-    rc = spark_attn_decode(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd,
-                           cfg->r_attn, cfg->cap, ctx_len, cfg->window, cfg->k_attn, cfg->flags & SPARK_DENSE_LOADS,
-                           ao, nullptr, nullptr, nullptr, 0, stream);
+    rc = attn_launch(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd, cfg->r_attn,
+                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & SPARK_DENSE_LOADS, ao, nullptr, nullptr,
+                     nullptr, 0, st);
     if (rc != SPARK_OK) return rc;
 
     // 4. h2 = h + Wo . attention

@@ -54,15 +54,12 @@ size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap
     if (hd < 8) hd = 8;
     if (max_d < 0) max_d = 0;
     const size_t grid_bound = 1024;   // more thread blocks than any device has SMs x residency
-    // FFN: per-token, per-block moments (float4).
-    size_t ffn = round_up(static_cast<size_t>(64) * grid_bound * 16, 256);
-    // attention: predictor scores, per-piece moments and partial outputs, per-segment counters.
-    size_t pieces = grid_bound + static_cast<size_t>(max_batch) * n_q;
-    size_t attn = round_up(static_cast<size_t>(max_batch) * n_q * max_cap * 4, 256) +
-                  round_up(pieces * 8 * 16, 256) +
-                  round_up(pieces * 8 * (static_cast<size_t>(hd) + 8) * 4, 256) +
-                  round_up(static_cast<size_t>(max_batch) * n_q * 16, 256);
-    size_t need = ffn > attn ? ffn : attn;
+    // attention: score-sum cells, per-piece partial outputs, and room for the predictor scores of
+    // blocks whose share does not fit in shared memory.
+    const size_t pieces = grid_bound + static_cast<size_t>(max_batch) * n_q;
+    const size_t need = kAttnCellBytes +
+                        round_up(pieces * 8 * (static_cast<size_t>(hd) + 8) * 4, 256) +
+                        round_up((static_cast<size_t>(max_batch) * n_q * max_cap + grid_bound * 8) * 4, 256);
     (void)max_dff;
     (void)max_d;
     return sizeof(WsHeader) + need + 256;
@@ -76,7 +73,9 @@ int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_
     if (cudaSetDevice(device) != cudaSuccess) return SPARK_ERR_CUDA;
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SPARK_ERR_CUDA;
-    if (cudaMemset(workspace, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;
+    // the whole workspace starts zeroed: header words, score-sum cells and per-segment counters are
+    // idle at zero, and the kernels leave them so
+    if (cudaMemset(workspace, 0, workspace_bytes) != cudaSuccess) return SPARK_ERR_CUDA;
     spark_ctx* c = new (std::nothrow) spark_ctx;
     if (c == nullptr) return SPARK_ERR_INVALID_ARG;
     c->device = device;
@@ -116,8 +115,8 @@ int spark_device_status(spark_ctx* ctx, void* stream, int* host_out) {
         return SPARK_ERR_CUDA;
     *host_out = status;
     if (status != SPARK_OK) {
-        // a failed phase may have left arrivals behind: start the barrier afresh
-        if (cudaMemset(ctx->hdr, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;
+        // a failed phase may have left arrivals or partial sums behind: back to the idle (zero) state
+        if (cudaMemset(ctx->ws, 0, ctx->ws_bytes) != cudaSuccess) return SPARK_ERR_CUDA;
     }
     return SPARK_OK;
 }
