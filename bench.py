@@ -50,6 +50,7 @@ def parse():
     ap.add_argument("--layers", type=int, default=0, help="0 = the shape's layer count")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-loads comparator")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     return ap.parse_args()
 
 
@@ -233,15 +234,38 @@ def run_spark(args):
     h_host_out = torch.empty_like(h_host_in).pin_memory()
     kernels_per_layer = 5
 
-    def step(which=0):
-        h.copy_(h_init)                                   # device-to-device copy of the token's input
+    def stack(which):
         for lay in layers:
             S.spark_layer_decode(ctx, lay[which], cl, h, B, scratch)
 
+    # The library only enqueues kernels on the caller's stream, so a whole decode step can be
+    # captured once into a CUDA graph and replayed per token (what a serving loop would do).
+    graphs = {}
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        for which in ((0,) if args.no_dense else (0, 1)):
+            with torch.cuda.stream(side):
+                stack(which)                               # warm-up outside capture (first-call set-up)
+                side.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    stack(which)
+            graphs[which] = g
+        torch.cuda.synchronize()
+
+    def run_stack(which):
+        if which in graphs:
+            graphs[which].replay()
+        else:
+            stack(which)
+
+    def step(which=0):
+        h.copy_(h_init)                                   # device-to-device copy of the token's input
+        run_stack(which)
+
     def step_e2e():
         h.copy_(h_host_in, non_blocking=True)             # pinned host -> device
-        for lay in layers:
-            S.spark_layer_decode(ctx, lay[0], cl, h, B, scratch)
+        run_stack(0)
         h_host_out.copy_(h, non_blocking=True)            # device -> pinned host
         torch.cuda.current_stream().synchronize()
 
@@ -290,11 +314,27 @@ def run_spark(args):
         unions.append(int(torch.unique(ids).numel()))
     union = float(np.mean(unions))
 
-    def ffn_loop():
+    def ffn_calls():
         for lay in layers:
             w = lay[2]
             S.spark_ffn_decode(ctx, xn, B, w["K1t"], w["K2t"], w["Vt"], S.SPARK_BF16, d, shape.d_ff, shape.r_ff,
                                shape.k_ff, 0, y, None, None, None)
+
+    ffn_graph = None
+    if not args.no_graph:
+        with torch.cuda.stream(side):
+            ffn_calls()
+            side.synchronize()
+            ffn_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(ffn_graph, stream=side):
+                ffn_calls()
+        torch.cuda.synchronize()
+
+    def ffn_loop():
+        if ffn_graph is not None:
+            ffn_graph.replay()
+        else:
+            ffn_calls()
 
     ms_ffn = timed(ffn_loop, args.steps, W)
     ffn_us = ms_ffn * 1e3 / (args.steps * n_layers)
@@ -311,9 +351,10 @@ def run_spark(args):
         line = {
             "metric": "us_per_token_per_layer", "value": us_tl, "unit": "us/token/layer", "n_gpus": world,
             "steps": args.steps, "warmup": W, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 weights/cache, f32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(args, shape), "l2": "weights+caches (>3 GB) exceed L2; no flush needed",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "launch": "host launches" if args.no_graph else "one CUDA graph replay per decode step",
                        "local_window": 4096, "k_ff": shape.k_ff, "k_attn": shape.k_attn},
             "tokens_per_s": B * world * args.steps / (ms_total * 1e-3),
             "layer_touched_mb": layer_touched / 1e6,
