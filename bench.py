@@ -229,7 +229,7 @@ def run_spark(args):
     h_init = torch.randn(B, d, device=dev, generator=gen)
     h = torch.empty_like(h_init)
     cl = torch.full((B,), ctx_len, dtype=torch.int32, device=dev)
-    scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2), device=dev)
+    scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
     kernels_per_layer = 5

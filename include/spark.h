@@ -231,7 +231,7 @@ typedef struct spark_kv_cache {
     void* vc;             /* [B][n_kv][cap][hd]          bf16                              */
 } spark_kv_cache;
 
-/* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2) fp32 values, 16-byte aligned, caller-owned, contents
+/* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2 + n_q) fp32 values, 16-byte aligned, caller-owned, contents
  * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 16.  Five kernels are
  * enqueued: QKV projection, position encoding + cache append, attention, output projection, FFN. */
 int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,

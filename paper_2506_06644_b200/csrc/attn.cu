@@ -17,9 +17,11 @@
 //           and forms theta (Eq. 11); no grid-wide barrier: only the blocks that share a segment
 //           wait for one another.
 //   pass 2  every warp selects among its own tokens (ballot), and only for those reads the k2c and
-//           vc rows: gate = softplus(k2c[t] . q[r:]), online softmax over the survivors, value
-//           reduction; the block combines its warps into a piece partial (max, sum, acc); the
-//           block that completes a segment last merges its pieces and writes o.
+//           vc rows: gate = softplus(k2c[t] . q[r:]), weights exp(s_t - max score) (the cells carry
+//           the head's largest score, so every piece uses the same reference), value reduction;
+//           the block adds its sum of weights and its weighted values to the head's accumulators
+//           with vector reductions; the block that completes a segment last divides.  Inside
+//           spark_layer_decode the division is left to the output projection that follows.
 #include "kernels.h"
 
 using namespace spark;
@@ -50,7 +52,8 @@ struct AttnParams {
     int ntok;          // capacity (tokens) of a block's score buffer
     int sc_smem;       // 1: scores live in shared memory
     SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
-    float* part;       // [pieces][GQ][hd + kPartPad]
+    float* lsum;       // [B][n_q] sum of softmax weights per head (o accumulates the weighted values)
+    int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
     WsHeader* hdr;
     PhaseTrace trace;
 };
@@ -77,7 +80,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     float* wpart = qs + GQ * hd;                                          // [kWarps][hd + kPartPad]
     float* sc_s = wpart + kWarps * (hd + kPartPad);                       // [GQ][ntok] when sc_smem
     __shared__ double red[kWarps][GQ][2];
-    __shared__ float theta_s[GQ];
+    __shared__ float redm[kWarps][GQ];
+    __shared__ float theta_s[GQ], smax_s[GQ];
     __shared__ double zcache[kZc];
     __shared__ double s_z;
     __shared__ int s_last, s_fail;
@@ -156,6 +160,11 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int off = static_cast<int>(f - f0) - tb;           // score slot of token t: off + t
             for (int i = tid; i < GQ * hd; i += kThreads) qs[i] = p.q[(static_cast<int64_t>(b) * p.n_q + g * GQ) * hd + i];
             if (tb == 0 && p.count != nullptr && tid < GQ) p.count[b * p.n_q + g * GQ + tid] = 0;
+            if (tb == 0) {      // the segment's first piece clears the heads' accumulators before it arrives
+                float* ob = p.o + (static_cast<int64_t>(b) * p.n_q + g * GQ) * hd;
+                for (int i = tid; i < GQ * hd; i += kThreads) ob[i] = 0.f;
+                if (tid < GQ) p.lsum[b * p.n_q + g * GQ + tid] = 0.f;
+            }
             if (tid == kThreads - 1 && ord < kZc)
                 zcache[ord] = p.k_attn >= L ? 0.0
                               : (p.zs != nullptr ? p.zs[b] : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
@@ -166,8 +175,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) qreg[hq][e] = hl < nc1 ? qs[hq * hd + hl * 8 + e] : 0.f;
             double s1[GQ], s2[GQ];
+            float mx[GQ];
 #pragma unroll
-            for (int hq = 0; hq < GQ; ++hq) { s1[hq] = 0.0; s2[hq] = 0.0; }
+            for (int hq = 0; hq < GQ; ++hq) { s1[hq] = 0.0; s2[hq] = 0.0; mx[hq] = -INFINITY; }
             const KT* kbase = k1c + (static_cast<int64_t>(seg) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
@@ -223,24 +233,28 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                         const double v = static_cast<double>(a1[hq]);
                         s1[hq] += v;
                         s2[hq] = fma(v, v, s2[hq]);
+                        mx[hq] = fmaxf(mx[hq], a1[hq]);
                     }
                 }
             }
 #pragma unroll
             for (int hq = 0; hq < GQ; ++hq) {
                 const double a = warp_sum_f64(s1[hq]), c = warp_sum_f64(s2[hq]);
-                if (lane == 0) { red[warp][hq][0] = a; red[warp][hq][1] = c; }
+                const float m = warp_max(mx[hq]);
+                if (lane == 0) { red[warp][hq][0] = a; red[warp][hq][1] = c; redm[warp][hq] = m; }
             }
             __syncthreads();
             if (warp < GQ) {
                 double a = lane < kWarps ? red[lane][warp][0] : 0.0, c = lane < kWarps ? red[lane][warp][1] : 0.0;
+                float m = lane < kWarps ? redm[lane][warp] : -INFINITY;
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) {
                     a += __shfl_xor_sync(kFull, a, o);
                     c += __shfl_xor_sync(kFull, c, o);
+                    m = fmaxf(m, __shfl_xor_sync(kFull, m, o));
                 }
                 if (lane == 0)
-                    cells_add_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays, cta, a, c);
+                    cells_add_max_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays, cta, a, c, m);
             }
             __syncthreads();
             f = sb + te;
@@ -267,8 +281,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             __syncthreads();
             if (warp < GQ) {        // theta of this head once every piece of the segment has arrived
                 double sa, sq;
-                const bool ok = cells_wait_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays,
-                                                        static_cast<unsigned>(c_hi - c_lo + 1), sa, sq, p.hdr);
+                float smax;
+                const bool ok = cells_wait_max_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays,
+                                                            static_cast<unsigned>(c_hi - c_lo + 1), sa, sq, smax, p.hdr);
                 if (lane == 0) {
                     if (!ok) s_fail = 1;
                     float th = -INFINITY;
@@ -280,6 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                         th = static_cast<float>(mean + sqrt(var) * z);
                     }
                     theta_s[warp] = th;
+                    smax_s[warp] = smax;
                     if (tb == 0 && p.theta != nullptr) p.theta[b * p.n_q + g * GQ + warp] = th;
                 }
             }
@@ -301,12 +317,12 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 if (w0 > te) w0 = te;
                 if (w1 > te) w1 = te;
             }
-            const float th = theta_s[hq];
+            const float th = theta_s[hq], smax = smax_s[hq];
             const int bh = b * p.n_q + g * GQ + hq;
             float q2[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) q2[e] = hl < nc2 ? qs[hq * hd + r + hl * 8 + e] : 0.f;
-            float m_w = -INFINITY, l_w = 0.f, acc[8];
+            float l_w = 0.f, acc[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = 0.f;
             const float* srow = sc + static_cast<size_t>(hq) * ntok + off;
@@ -316,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 const bool valid = t < w1;
                 const float s = valid ? srow[t] : 0.f;
                 const bool sel = valid && (ident || s > th);
-                const float a = sel ? (ident ? s : s - th) : -INFINITY;
+                const float a = sel ? s - smax : -INFINITY;        // softmax is shift-invariant: the head's largest score is the reference
                 const unsigned bsel = __ballot_sync(kFull, sel);
                 unsigned bal = p.dense ? __ballot_sync(kFull, valid) : bsel;
                 if (p.count != nullptr && bsel != 0u) {
@@ -366,27 +382,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                         gt[2 * i] = __shfl_sync(kFull, gate, 0);
                         gt[2 * i + 1] = __shfl_sync(kFull, gate, 16);
                     }
-                    const float mn = fmaxf(fmaxf(m_w, fmaxf(av[0], av[1])), fmaxf(av[2], av[3]));
-                    float wt[4] = {0.f, 0.f, 0.f, 0.f};
-                    float scl = 1.f;
-                    if (mn != -INFINITY) {
-                        scl = m_w == -INFINITY ? 0.f : expf(m_w - mn);
-                        float add = 0.f;
+                    float wt[4];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float pe = av[i] == -INFINITY ? 0.f : expf(av[i] - mn);
-                            add += pe;
-                            wt[i] = pe * gt[i];
-                        }
-                        l_w = l_w * scl + add;
-                        m_w = mn;
-                    } else {
-                        // nothing selected so far: the rows were read (dense comparator); keep the loads alive
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) wt[i] = 0.f * gt[i];
+                    for (int i = 0; i < 4; ++i) {
+                        const float pe = av[i] == -INFINITY ? 0.f : expf(av[i]);
+                        l_w += pe;
+                        wt[i] = pe * gt[i];         // unselected rows of the dense comparator get weight 0 * gate
                     }
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[e] *= scl;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         float fv[8];
@@ -396,47 +398,36 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     }
                 }
             }
-            // ---- combine the warps' online-softmax states into one (max, sum, acc) per head --------------
-            // Entry w of wpart belongs to head w % GQ.  `final_out`: normalise and write o; else write the
-            // piece partial to the workspace.
-            auto combine = [&](bool final_out) {
+            // ---- add the block's sum of weights and weighted values to the heads' accumulators ----------
+            {
                 float* wp = wpart + warp * pstride;
-                if (lane == 0) { wp[0] = m_w; wp[1] = l_w; }
+                if (lane == 0) wp[1] = l_w;
                 if (lane < ncv) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) wp[kPartPad + lane * 8 + e] = acc[e];
                 }
                 __syncthreads();
-                for (int i = tid; i < GQ * hd; i += kThreads) {
-                    const int h = i / hd, dd = i - h * hd;
-                    float M = -INFINITY;
-#pragma unroll
-                    for (int u = 0; u < NSUB; ++u) M = fmaxf(M, wpart[(u * GQ + h) * pstride]);
-                    float sum = 0.f, l = 0.f;
+                for (int i = tid; i < GQ * (hd / 4); i += kThreads) {
+                    const int h = i / (hd / 4), d4 = i - h * (hd / 4);
+                    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+                    float l = 0.f;
 #pragma unroll
                     for (int u = 0; u < NSUB; ++u) {
                         const float* e = wpart + (u * GQ + h) * pstride;
-                        if (e[0] != -INFINITY) {
-                            const float w = expf(e[0] - M);
-                            sum = fmaf(w, e[kPartPad + dd], sum);
-                            l = fmaf(w, e[1], l);
-                        }
+                        const float4 x = *reinterpret_cast<const float4*>(e + kPartPad + d4 * 4);
+                        sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+                        l += e[1];
                     }
-                    if (final_out) {
-                        p.o[(static_cast<int64_t>(b) * p.n_q + g * GQ + h) * hd + dd] = l > 0.f ? sum / l : 0.f;
-                    } else {
-                        float* dst = p.part + (pid * GQ + h) * pstride;
-                        dst[kPartPad + dd] = sum;
-                        if (dd == 0) { dst[0] = M; dst[1] = l; }
+                    if (l > 0.f || p.dense) {
+                        const int64_t hb = static_cast<int64_t>(b) * p.n_q + g * GQ + h;
+                        red_add_v4(p.o + hb * hd + d4 * 4, sum.x, sum.y, sum.z, sum.w);
+                        if (d4 == 0) atomicAdd(&p.lsum[hb], l);
                     }
                 }
                 __syncthreads();
-            };
-            const bool single = c_lo == c_hi;       // the whole segment lies in this block: no merge needed
-            combine(single);
-
-            // ---- the block that completes a segment last merges its pieces and writes o -------------
-            if (!single) {
+            }
+            // ---- the block that completes a segment last divides by the sum of weights -----------------
+            if (!p.defer) {
                 if (tid == 0) {
                     __threadfence();
                     const unsigned prev = atom_add_acqrel_u32(&p.hdr->seg_done[seg], 1u);
@@ -446,38 +437,23 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 }
                 __syncthreads();
                 if (s_last) {
-                    // warp w merges pieces c_lo + w / GQ, + NSUB, ... of head w % GQ, then the warps combine
-                    m_w = -INFINITY; l_w = 0.f;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-                    for (int c = c_lo + wsub; c <= c_hi; c += NSUB) {
-                        const float* src = p.part + (static_cast<size_t>(c + seg) * GQ + hq) * pstride;
-                        const float mp = __ldcg(src), lp = __ldcg(src + 1);
-                        float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0;
-                        if (lane < ncv) {
-                            x0 = __ldcg(reinterpret_cast<const float4*>(src + kPartPad + lane * 8));
-                            x1 = __ldcg(reinterpret_cast<const float4*>(src + kPartPad + lane * 8 + 4));
-                        }
-                        if (mp == -INFINITY) continue;
-                        const float mn = fmaxf(m_w, mp);
-                        const float sa = m_w == -INFINITY ? 0.f : expf(m_w - mn), sb2 = expf(mp - mn);
-                        l_w = l_w * sa + lp * sb2;
-                        acc[0] = fmaf(sb2, x0.x, acc[0] * sa); acc[1] = fmaf(sb2, x0.y, acc[1] * sa);
-                        acc[2] = fmaf(sb2, x0.z, acc[2] * sa); acc[3] = fmaf(sb2, x0.w, acc[3] * sa);
-                        acc[4] = fmaf(sb2, x1.x, acc[4] * sa); acc[5] = fmaf(sb2, x1.y, acc[5] * sa);
-                        acc[6] = fmaf(sb2, x1.z, acc[6] * sa); acc[7] = fmaf(sb2, x1.w, acc[7] * sa);
-                        m_w = mn;
+                    for (int i = tid; i < GQ * hd; i += kThreads) {
+                        const int h = i / hd;
+                        const int64_t hb = static_cast<int64_t>(b) * p.n_q + g * GQ + h;
+                        const float l = __ldcg(&p.lsum[hb]);
+                        float* od = p.o + hb * hd + (i - h * hd);
+                        const float v = __ldcg(od);
+                        *od = l > 0.f ? v / l : 0.f;
                     }
-                    combine(true);
                 }
             } else if (tid == 0) {
-                s_last = 1;
+                s_last = 0;
             }
             __syncthreads();
             // every piece of the segment has read the cells by now: leave them zero for the next launch
             if (s_last && tid < GQ * kAttnWays) {
                 SumCell* c = cells + static_cast<size_t>(b * p.n_q + g * GQ) * kAttnWays + tid;
-                c->s1 = 0.0; c->s2 = 0.0; c->count = 0u;
+                c->s1 = 0.0; c->s2 = 0.0; c->count = 0u; c->pad[0] = 0u;
             }
             __syncthreads();
             f = sb + te;
@@ -525,7 +501,7 @@ namespace spark {
 
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
-                int64_t window, int64_t k_attn, int flags, float* o, float* theta, int32_t* count, int32_t* idx,
+                int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
                 int64_t idx_cap, cudaStream_t st) {
     if (ctx == nullptr || q == nullptr || k1c == nullptr || k2c == nullptr || vc == nullptr || ctx_len == nullptr ||
         o == nullptr)
@@ -545,12 +521,11 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     const int grid = ctx->num_sms;
     const int64_t span = (window > 0 && window < cap) ? window : cap;          // longest window of a sequence
     const int64_t ntok = (B * n_kv * span + grid - 1) / grid + 1;            // tokens one block may own
-    const size_t pieces = static_cast<size_t>(grid) + static_cast<size_t>(B * n_kv);
     // The cells keep a fixed place and size in the workspace whatever the call's shape: they must be
     // zero between launches, so nothing else may ever be written there.
     const size_t cells_b = kAttnCellBytes;
     if (static_cast<size_t>(B * n_q) * kAttnWays * sizeof(SumCell) > cells_b) return SPARK_ERR_UNSUPPORTED;
-    const size_t part_b = round_up(pieces * gq * (hd + kPartPad) * 4, 256);
+    const size_t part_b = round_up(static_cast<size_t>(B * n_q) * 4, 256);     // sums of weights (standalone calls)
     const size_t ns_pad = (static_cast<size_t>(B * n_kv) + 1 + 3) & ~static_cast<size_t>(3);
     const size_t smem_fixed = ns_pad * 4 + static_cast<size_t>(gq * hd) * 4 + static_cast<size_t>(kWarps) * (hd + kPartPad) * 4;
     const size_t smem_limit = static_cast<size_t>(ctx->max_smem_optin - 8192);
@@ -569,7 +544,8 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.dense = (flags & SPARK_DENSE_LOADS) ? 1 : 0;
     p.o = o; p.theta = theta; p.count = count; p.idx = idx; p.idx_cap = idx_cap;
     p.cells = reinterpret_cast<SumCell*>(ctx->scratch);
-    p.part = reinterpret_cast<float*>(ctx->scratch + cells_b);
+    p.lsum = lsum != nullptr ? lsum : reinterpret_cast<float*>(ctx->scratch + cells_b);
+    p.defer = lsum != nullptr ? 1 : 0;
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;
@@ -588,5 +564,5 @@ extern "C" int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c
                                  float* o, float* theta, int32_t* count, int32_t* idx, int64_t idx_cap,
                                  void* stream) {
     return attn_launch(ctx, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv, hd, r, cap, ctx_len, nullptr, window, k_attn, flags, o,
-                       theta, count, idx, idx_cap, static_cast<cudaStream_t>(stream));
+                       nullptr, theta, count, idx, idx_cap, static_cast<cudaStream_t>(stream));
 }

@@ -306,8 +306,17 @@ __device__ __forceinline__ void red_add_f64(double* p, double v) {
 __device__ __forceinline__ void red_release_add_u32(unsigned* p, unsigned v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-// One 32-byte read of a cell (sm_100 has 256-bit global loads): {s1, s2, count}.
-__device__ __forceinline__ void ld_cell(const SumCell* c, double& s1, double& s2, unsigned& count) {
+// Order-preserving map between fp32 and u32 (for atomic max on floats); 0 decodes below every float.
+__device__ __forceinline__ unsigned f32_to_ordered(float f) {
+    const unsigned u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_f32(unsigned u) {
+    if (u == 0u) return -INFINITY;
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+// One 32-byte read of a cell (sm_100 has 256-bit global loads): {s1, s2, count, pad[0]}.
+__device__ __forceinline__ void ld_cell_x(const SumCell* c, double& s1, double& s2, unsigned& count, unsigned& extra) {
     unsigned long long a, b, d, e;   // e: padding half of the sector
     asm volatile("ld.acquire.gpu.global.v4.u64 {%0,%1,%2,%3}, [%4];"
                  : "=l"(a), "=l"(b), "=l"(d), "=l"(e)
@@ -316,7 +325,12 @@ __device__ __forceinline__ void ld_cell(const SumCell* c, double& s1, double& s2
     s1 = __longlong_as_double(static_cast<long long>(a));
     s2 = __longlong_as_double(static_cast<long long>(b));
     count = static_cast<unsigned>(d & 0xffffffffull);
+    extra = static_cast<unsigned>(d >> 32);
     (void)e;
+}
+__device__ __forceinline__ void ld_cell(const SumCell* c, double& s1, double& s2, unsigned& count) {
+    unsigned extra;
+    ld_cell_x(c, s1, s2, count, extra);
 }
 // Add this block's two sums to its way of a cell group, then its arrival (release: ordered after
 // the sums and after everything the block wrote before).  One thread calls this.
@@ -351,6 +365,47 @@ __device__ __forceinline__ bool cells_wait_w(const SumCell* ways, unsigned nbloc
             }
             s1 = __shfl_sync(kFull, a, 0);
             s2 = __shfl_sync(kFull, b, 0);
+            return true;
+        }
+        if (clock64() - t0 > kSpinLimitCycles) {
+            if (lane == 0) atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+// The same with a running maximum kept in the cell's spare word (attention needs the largest score).
+template <int WAYS>
+__device__ __forceinline__ void cells_add_max_w(SumCell* ways, int block, double s1, double s2, float mx) {
+    SumCell* c = ways + (block % WAYS);
+    red_add_f64(&c->s1, s1);
+    red_add_f64(&c->s2, s2);
+    asm volatile("red.relaxed.gpu.global.max.u32 [%0], %1;" ::"l"(&c->pad[0]), "r"(f32_to_ordered(mx)) : "memory");
+    red_release_add_u32(&c->count, 1u);
+}
+template <int WAYS>
+__device__ __forceinline__ bool cells_wait_max_w(const SumCell* ways, unsigned nblocks, double& s1, double& s2, float& mx,
+                                                 WsHeader* hdr) {
+    const int lane = threadIdx.x & 31;
+    const long long t0 = clock64();
+    for (;;) {
+        double a = 0.0, b = 0.0;
+        unsigned cnt = 0u, ex = 0u;
+        if (lane < WAYS) ld_cell_x(ways + lane, a, b, cnt, ex);
+        unsigned tot = cnt;
+#pragma unroll
+        for (int o = WAYS / 2; o > 0; o >>= 1) tot += __shfl_xor_sync(kFull, tot, o);
+        tot = __shfl_sync(kFull, tot, 0);
+        if (tot == nblocks) {
+#pragma unroll
+            for (int o = WAYS / 2; o > 0; o >>= 1) {
+                a += __shfl_xor_sync(kFull, a, o);
+                b += __shfl_xor_sync(kFull, b, o);
+                const unsigned e2 = __shfl_xor_sync(kFull, ex, o);
+                ex = e2 > ex ? e2 : ex;
+            }
+            s1 = __shfl_sync(kFull, a, 0);
+            s2 = __shfl_sync(kFull, b, 0);
+            mx = ordered_to_f32(__shfl_sync(kFull, ex, 0));
             return true;
         }
         if (clock64() - t0 > kSpinLimitCycles) {

@@ -34,14 +34,20 @@ struct GemvArgs {
     int64_t B, n_in, n_out;
     const float* y_add;      // nullable, may alias y
     float* y;
+    const float* x_div;      // nullable: x[b][i] is divided by x_div[b][i / x_div_group] (0 where that is 0)
+    int64_t x_div_group;
+    void* zero_ptr;          // nullable: this many bytes (multiple of 16) are cleared by the kernel as a side job
+    size_t zero_bytes;
 };
 int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 
 // Spark attention; zs (nullable) holds Q(1 - k_attn / L_b) per sequence when an earlier kernel of the
-// same stream has already computed it.
+// same stream has already computed it.  With lsum != nullptr the kernel leaves o unnormalised (the
+// weighted value sums), writes the sums of weights to lsum[B][n_q] and leaves its score-sum cells
+// for the caller's next kernel to clear (the first B * n_q * kAttnWays cells of the scratch area).
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
-                int64_t window, int64_t k_attn, int flags, float* o, float* theta, int32_t* count, int32_t* idx,
+                int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
                 int64_t idx_cap, cudaStream_t st);
 
 }  // namespace spark

@@ -22,6 +22,10 @@ struct GemvParams {
     int B, n_in, n_out;
     const float* y_add;
     float* y;
+    const float* x_div;
+    int x_div_group;
+    uint4* zero_ptr;
+    int zero_n16;
 };
 
 // y[b][o] = Wt[o][:] . xhat[b][:] (+ y_add[b][o]);  xhat = x or RMSNorm(x; norm_w).
@@ -38,9 +42,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
         for (int i = tid; i < TB * w4; i += kThreads) {
             const int t = i / w4, c = i - t * w4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (t < p.B) v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
+            if (t < p.B) {
+                v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
+                if (p.x_div != nullptr) {
+                    const float dv = p.x_div[static_cast<int64_t>(t) * (n_in / p.x_div_group) + (c * 4) / p.x_div_group];
+                    const float inv = dv > 0.f ? 1.f / dv : 0.f;
+                    v.x *= inv; v.y *= inv; v.z *= inv; v.w *= inv;
+                }
+            }
             reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * n_in)[c] = v;
         }
+        for (int i = blockIdx.x * kThreads + tid; i < p.zero_n16; i += gridDim.x * kThreads)
+            p.zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
         if (p.norm_w != nullptr) {
             for (int t = warp; t < TB; t += kWarps) {
@@ -82,11 +95,18 @@ int gemv_launch_one(spark_ctx* ctx, GemvParams& p, size_t smem, int grid, cudaSt
     return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
+template <typename WT, int TB>
+int gemv_dispatch_rw(spark_ctx* ctx, GemvParams& p, int rw, size_t smem, int grid, cudaStream_t stream) {
+    if (rw == 1) return gemv_launch_one<WT, TB, 1>(ctx, p, smem, grid, stream);
+    if (rw == 2) return gemv_launch_one<WT, TB, 2>(ctx, p, smem, grid, stream);
+    return gemv_launch_one<WT, TB, 4>(ctx, p, smem, grid, stream);
+}
+
 template <typename WT>
 int gemv_dispatch(spark_ctx* ctx, GemvParams& p, int tb, int rw, size_t smem, int grid, cudaStream_t stream) {
-    if (tb == 1) return rw == 1 ? gemv_launch_one<WT, 1, 1>(ctx, p, smem, grid, stream) : gemv_launch_one<WT, 1, 4>(ctx, p, smem, grid, stream);
-    if (tb == 4) return rw == 1 ? gemv_launch_one<WT, 4, 1>(ctx, p, smem, grid, stream) : gemv_launch_one<WT, 4, 4>(ctx, p, smem, grid, stream);
-    return rw == 1 ? gemv_launch_one<WT, 16, 1>(ctx, p, smem, grid, stream) : gemv_launch_one<WT, 16, 4>(ctx, p, smem, grid, stream);
+    if (tb == 1) return gemv_dispatch_rw<WT, 1>(ctx, p, rw, smem, grid, stream);
+    if (tb == 4) return gemv_dispatch_rw<WT, 4>(ctx, p, rw, smem, grid, stream);
+    return gemv_dispatch_rw<WT, 16>(ctx, p, rw, smem, grid, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -106,6 +126,7 @@ struct RopeParams {
     float base, q_scale;
     double* zs;              // [B] out: Q(1 - k_attn / L_b) for the attention kernel that follows
     int window, k_attn;
+    double inv_freq[2][64];  // base^(-2i/m) for the pairs of the first part (m = r) and of the second (m = hd - r)
 };
 
 __global__ void rope_append_kernel(const RopeParams p) {
@@ -140,11 +161,14 @@ __global__ void rope_append_kernel(const RopeParams p) {
         if (pr < hr) { part0 = 0; m = p.r; pi = pr; }
         else { part0 = p.r; m = p.hd - p.r; pi = pr - hr; }
         const int ia = part0 + pi, ib = part0 + pi + m / 2;
-        const double ang = static_cast<double>(pos) * exp2(-2.0 * static_cast<double>(pi) / static_cast<double>(m) * log2(static_cast<double>(p.base)));
-        double sn, cs;
-        sincos(ang, &sn, &cs);
+        // angle = pos * base^(-2i/m): the product and its reduction to one turn in fp64 (positions reach
+        // tens of thousands of radians), sine and cosine of the reduced angle in fp32
+        const double turns = static_cast<double>(pos) * p.inv_freq[part0 ? 1 : 0][pi] * 0.15915494309189533577;
+        const float ang = static_cast<float>((turns - floor(turns)) * 6.28318530717958647692);
+        float sn, cs;
+        sincosf(ang, &sn, &cs);
         const float a = src[ia], bb = src[ib];
-        const float ra = static_cast<float>(a * cs - bb * sn), rb = static_cast<float>(a * sn + bb * cs);
+        const float ra = a * cs - bb * sn, rb = a * sn + bb * cs;
         if (h < p.n_q) {
             float* dst = p.q_out + (static_cast<int64_t>(b) * p.n_q + h) * p.hd;
             dst[ia] = ra * p.q_scale;
@@ -174,6 +198,8 @@ int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
     if (a.B < 1 || a.B > 16 || a.n_in < 8 || a.n_out < 1) return SPARK_ERR_INVALID_ARG;
     if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
     if ((a.n_in & 7) != 0 || !aligned16(a.x) || !aligned16(a.Wt) || !aligned16(a.norm_w)) return SPARK_ERR_UNSUPPORTED;
+    if (a.x_div != nullptr && (a.x_div_group < 4 || (a.x_div_group & 3) != 0 || a.n_in % a.x_div_group != 0)) return SPARK_ERR_UNSUPPORTED;
+    if (a.zero_ptr != nullptr && (!aligned16(a.zero_ptr) || (a.zero_bytes & 15) != 0)) return SPARK_ERR_UNSUPPORTED;
     if (a.n_out > (1LL << 30) || a.n_in > (1 << 20)) return SPARK_ERR_UNSUPPORTED;
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
     const size_t limit = static_cast<size_t>(ctx->max_smem_optin - 1024);
@@ -187,12 +213,17 @@ int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
         if (nb > tb) nb = tb;
         const int grid = a.n_out < ctx->num_sms ? static_cast<int>(a.n_out) : ctx->num_sms;
         const int64_t rows_per_block = (a.n_out + grid - 1) / grid;
-        const int rw = rows_per_block <= kWarps ? 1 : 4;
+        // rows a warp takes at once: as few as keeps all 16 warps of a block busy
+        const int rw = rows_per_block <= kWarps ? 1 : (rows_per_block <= 2 * kWarps ? 2 : 4);
         GemvParams p;
         p.x = a.x + done * a.n_in; p.norm_w = a.norm_w; p.eps = a.rms_eps; p.Wt = a.Wt;
         p.B = static_cast<int>(nb); p.n_in = static_cast<int>(a.n_in); p.n_out = static_cast<int>(a.n_out);
         p.y_add = a.y_add ? a.y_add + done * a.n_out : nullptr;
         p.y = a.y + done * a.n_out;
+        p.x_div = a.x_div ? a.x_div + done * (a.n_in / a.x_div_group) : nullptr;
+        p.x_div_group = static_cast<int>(a.x_div ? a.x_div_group : 1);
+        p.zero_ptr = done == 0 ? static_cast<uint4*>(a.zero_ptr) : nullptr;
+        p.zero_n16 = done == 0 ? static_cast<int>(a.zero_bytes / 16) : 0;
         const size_t smem = static_cast<size_t>(tb) * a.n_in * 4;
         const int st = a.wdtype == SPARK_BF16 ? gemv_dispatch<__nv_bfloat16>(ctx, p, tb, rw, smem, grid, stream)
                                               : gemv_dispatch<float>(ctx, p, tb, rw, smem, grid, stream);
@@ -209,6 +240,7 @@ extern "C" int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const
     GemvArgs a;
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f; a.Wt = Wt; a.wdtype = wdtype;
     a.B = B; a.n_in = n_in; a.n_out = n_out; a.y_add = y_add; a.y = y;
+    a.x_div = nullptr; a.x_div_group = 1; a.zero_ptr = nullptr; a.zero_bytes = 0;
     return gemv_launch(ctx, a, static_cast<cudaStream_t>(stream));
 }
 
@@ -235,11 +267,13 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     float* ao = qr + B * nqo;             // [B][n_q][hd]  attention output
     float* h2 = ao + B * nqo;             // [B][d]        h + Wo . attention
     double* zs = reinterpret_cast<double*>(h2 + B * cfg->d);   // [B] threshold quantiles (8-byte aligned: see below)
+    float* lsum = reinterpret_cast<float*>(zs + B);            // [B][n_q] sums of attention weights
 
     // 1. a = RMSNorm(h; norm1); [q|k|v] = Wqkv a
     GemvArgs g1;
     g1.x = h; g1.norm_w = w->norm1; g1.rms_eps = cfg->rms_eps; g1.Wt = w->Wqkv; g1.wdtype = SPARK_BF16;
     g1.B = B; g1.n_in = cfg->d; g1.n_out = nqkv; g1.y_add = nullptr; g1.y = qkv;
+    g1.x_div = nullptr; g1.x_div_group = 1; g1.zero_ptr = nullptr; g1.zero_bytes = 0;
     int rc = gemv_launch(ctx, g1, st);
     if (rc != SPARK_OK) return rc;
 
@@ -251,6 +285,12 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     rp.ctx_len = ctx_len; rp.B = static_cast<int>(B); rp.n_q = static_cast<int>(cfg->n_q); rp.n_kv = static_cast<int>(cfg->n_kv);
     rp.hd = static_cast<int>(cfg->hd); rp.r = static_cast<int>(cfg->r_attn); rp.cap = cfg->cap;
     rp.base = cfg->rope_base; rp.q_scale = 1.0f / std::sqrt(static_cast<float>(cfg->hd));
+    if (cfg->r_attn > 128 || cfg->hd - cfg->r_attn > 128) return SPARK_ERR_UNSUPPORTED;
+    for (int part = 0; part < 2; ++part) {
+        const int64_t m = part == 0 ? cfg->r_attn : cfg->hd - cfg->r_attn;
+        for (int64_t i = 0; i < m / 2; ++i)
+            rp.inv_freq[part][i] = std::pow(static_cast<double>(cfg->rope_base), -2.0 * static_cast<double>(i) / static_cast<double>(m));
+    }
     rp.zs = zs; rp.window = static_cast<int>(cfg->window > 0x7fffffff ? 0x7fffffff : cfg->window);
     rp.k_attn = static_cast<int>(cfg->k_attn > 0x7fffffff ? 0x7fffffff : cfg->k_attn);
     {
@@ -262,14 +302,17 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
 
     // 3. Spark attention over the cache (the new token included)
     rc = attn_launch(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd, cfg->r_attn,
-                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & SPARK_DENSE_LOADS, ao, nullptr, nullptr,
+                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & SPARK_DENSE_LOADS, ao, lsum, nullptr, nullptr,
                      nullptr, 0, st);
     if (rc != SPARK_OK) return rc;
 
-    // 4. h2 = h + Wo . attention
+    // 4. h2 = h + Wo . (attention sums / sums of weights); the projection kernel also clears the
+    //    attention kernel's score-sum cells for the next call
     GemvArgs g2;
     g2.x = ao; g2.norm_w = nullptr; g2.rms_eps = 0.f; g2.Wt = w->Wo; g2.wdtype = SPARK_BF16;
     g2.B = B; g2.n_in = nqo; g2.n_out = cfg->d; g2.y_add = h; g2.y = h2;
+    g2.x_div = lsum; g2.x_div_group = cfg->hd;
+    g2.zero_ptr = ctx->scratch; g2.zero_bytes = static_cast<size_t>(B * cfg->n_q) * kAttnWays * sizeof(SumCell);
     rc = gemv_launch(ctx, g2, st);
     if (rc != SPARK_OK) return rc;
 

@@ -74,7 +74,7 @@ def run_layer(ctx, sh, B, cap, lens, seed, window=0, flags=0):
     h = torch.from_numpy(h0).cuda()
     cl = torch.tensor(lens, dtype=torch.int32, device="cuda")
     nqkv = (sh.n_q + 2 * sh.n_kv) * sh.hd
-    scratch = torch.empty(B * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2), device="cuda")
+    scratch = torch.empty(B * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device="cuda")
     S.spark_layer_decode(ctx, layer, cl, h, B, scratch)
     torch.cuda.synchronize()
     return lw, kv, h0, h.cpu().numpy(), cache
