@@ -232,7 +232,7 @@ def run_spark(args):
     scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
-    kernels_per_layer = 5
+    kernels_per_layer = 4          # QKV+rotary+append, attention, output projection, FFN
 
     def stack(which):
         for lay in layers:

@@ -28,6 +28,68 @@ struct GemvParams {
     int zero_n16;
 };
 
+// Input staging shared by the GEMV kernels: x (optionally divided per group, optionally RMS-normalised)
+// into shared memory as [TB][n_in]; also the kernel's clear-region side job.  Ends with a block sync.
+// One token: the input is requested into registers BEFORE the weight loads are issued (requests are
+// served in issue order, so this is what puts x in shared memory by the time the first rows land).
+struct EarlyX {
+    float4 v0, v1;
+    bool on;
+};
+__device__ __forceinline__ EarlyX early_x_request(const GemvParams& p) {
+    EarlyX e;
+    e.v0 = make_float4(0.f, 0.f, 0.f, 0.f);
+    e.v1 = e.v0;
+    const int n4 = p.n_in / 4, tid = threadIdx.x;
+    e.on = p.B == 1 && n4 <= 2 * kThreads;
+    if (e.on) {
+        if (tid < n4) e.v0 = reinterpret_cast<const float4*>(p.x)[tid];
+        if (tid + kThreads < n4) e.v1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
+    }
+    return e;
+}
+
+template <int TB>
+__device__ __forceinline__ void stage_input(const GemvParams& p, float* xs, float* rstd, const EarlyX& ex) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_in = p.n_in;
+    const int w4 = n_in / 4;
+    for (int i = tid; i < TB * w4; i += kThreads) {
+        const int t = i / w4, c = i - t * w4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t < p.B) {
+            if (ex.on) v = i < kThreads ? ex.v0 : ex.v1;
+            else v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
+            if (p.x_div != nullptr) {
+                const float dv = p.x_div[static_cast<int64_t>(t) * (n_in / p.x_div_group) + (c * 4) / p.x_div_group];
+                const float inv = dv > 0.f ? 1.f / dv : 0.f;
+                v.x *= inv; v.y *= inv; v.z *= inv; v.w *= inv;
+            }
+        }
+        reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * n_in)[c] = v;
+    }
+    for (int i = blockIdx.x * kThreads + tid; i < p.zero_n16; i += gridDim.x * kThreads)
+        p.zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    if (p.norm_w != nullptr) {
+        for (int t = warp; t < TB; t += kWarps) {
+            float ss = 0.f;
+            for (int i = lane; i < n_in; i += 32) {
+                const float v = xs[static_cast<size_t>(t) * n_in + i];
+                ss = fmaf(v, v, ss);
+            }
+            ss = warp_sum(ss);
+            if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(n_in) + p.eps);
+        }
+        __syncthreads();
+        for (int i = tid; i < TB * n_in; i += kThreads) {
+            const int t = i / n_in, c = i - t * n_in;
+            xs[i] *= rstd[t] * p.norm_w[c];
+        }
+        __syncthreads();
+    }
+}
+
 // y[b][o] = Wt[o][:] . xhat[b][:] (+ y_add[b][o]);  xhat = x or RMSNorm(x; norm_w).
 template <typename WT, int TB, int RW>
 __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
@@ -37,42 +99,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
     const int n_in = p.n_in;
     const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
     const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
-    auto fill_x = [&]() {       // runs once the first weight loads are in flight
-        const int w4 = n_in / 4;
-        for (int i = tid; i < TB * w4; i += kThreads) {
-            const int t = i / w4, c = i - t * w4;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (t < p.B) {
-                v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
-                if (p.x_div != nullptr) {
-                    const float dv = p.x_div[static_cast<int64_t>(t) * (n_in / p.x_div_group) + (c * 4) / p.x_div_group];
-                    const float inv = dv > 0.f ? 1.f / dv : 0.f;
-                    v.x *= inv; v.y *= inv; v.z *= inv; v.w *= inv;
-                }
-            }
-            reinterpret_cast<float4*>(xs + static_cast<size_t>(t) * n_in)[c] = v;
-        }
-        for (int i = blockIdx.x * kThreads + tid; i < p.zero_n16; i += gridDim.x * kThreads)
-            p.zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
-        __syncthreads();
-        if (p.norm_w != nullptr) {
-            for (int t = warp; t < TB; t += kWarps) {
-                float ss = 0.f;
-                for (int i = lane; i < n_in; i += 32) {
-                    const float v = xs[static_cast<size_t>(t) * n_in + i];
-                    ss = fmaf(v, v, ss);
-                }
-                ss = warp_sum(ss);
-                if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(n_in) + p.eps);
-            }
-            __syncthreads();
-            for (int i = tid; i < TB * n_in; i += kThreads) {
-                const int t = i / n_in, c = i - t * n_in;
-                xs[i] *= rstd[t] * p.norm_w[c];
-            }
-            __syncthreads();
-        }
-    };
+    const EarlyX ex = early_x_request(p);
+    auto fill_x = [&]() { stage_input<TB>(p, xs, rstd, ex); };   // runs once the first weight loads are in flight
     rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in, fill_x,
                          [&](int j, int t, float v) {
                              if (t < p.B) {
@@ -189,6 +217,94 @@ __global__ void rope_append_kernel(const RopeParams p) {
     }
 }
 
+// QKV projection with the rotary encoding and the cache append in its epilogue: a warp computes the
+// two output rows of a rotary pair together (rows i and i + m/2 of a head's part), so the pair can be
+// turned and written to q / the caches straight from registers; value rows go to the cache as they
+// are.  Saves the [q|k|v] round trip through memory and one kernel per layer.
+struct QkvRopeParams {
+    GemvParams g;
+    RopeParams r;
+};
+
+template <int TB>
+__global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopeParams p) {
+    extern __shared__ __align__(16) float xs[];       // [TB][n_in]
+    __shared__ float rstd[16];
+    const GemvParams& g = p.g;
+    const RopeParams& rp = p.r;
+    const int tid = threadIdx.x;
+    if (blockIdx.x == gridDim.x - 1 && tid >= kThreads - 32 && tid - (kThreads - 32) < rp.B) {
+        // the threshold quantile of each sequence's window, for the attention kernel that follows
+        const int b = tid - (kThreads - 32);
+        int n = rp.ctx_len[b];
+        n = n < 1 ? 1 : (n > rp.cap ? static_cast<int>(rp.cap) : n);
+        const int L = (rp.window > 0 && rp.window < n) ? rp.window : n;
+        rp.zs[b] = rp.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(rp.k_attn) / static_cast<double>(L));
+    }
+    const int hd = rp.hd, hp = hd / 2, hr = rp.r / 2;
+    const int P = g.n_out / 2;                        // output pairs
+    const int p0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * P / gridDim.x);
+    const int p1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * P / gridDim.x);
+    auto rowmap = [&](int j) -> int {
+        const int pp = p0 + (j >> 1), which = j & 1;
+        const int head = pp / hp, q = pp - head * hp;
+        if (head >= rp.n_q + rp.n_kv) return head * hd + 2 * q + which;
+        if (q < hr) return head * hd + q + which * hr;
+        return head * hd + rp.r + (q - hr) + which * ((hd - rp.r) / 2);
+    };
+    const EarlyX ex = early_x_request(g);
+    auto fill_x = [&]() { stage_input<TB>(g, xs, rstd, ex); };
+    rows_dot_mapped<__nv_bfloat16, TB, 2>(
+        static_cast<const __nv_bfloat16*>(g.Wt), g.n_in, 2 * (p1 - p0), g.n_in / 8, xs, g.n_in, rowmap, fill_x,
+        [&](int rg, int t, const float (&v)[2]) {
+            if (t >= rp.B) return;
+            const int pp = p0 + rg;
+            const int head = pp / hp, q = pp - head * hp;
+            int n = rp.ctx_len[t];
+            n = n < 1 ? 1 : (n > rp.cap ? static_cast<int>(rp.cap) : n);
+            const int pos = n - 1;
+            if (head >= rp.n_q + rp.n_kv) {
+                const int gk = head - rp.n_q - rp.n_kv;
+                __nv_bfloat16* dst = rp.vc + ((static_cast<int64_t>(t) * rp.n_kv + gk) * rp.cap + pos) * hd;
+                dst[2 * q] = __float2bfloat16_rn(v[0]);
+                dst[2 * q + 1] = __float2bfloat16_rn(v[1]);
+                return;
+            }
+            const bool second = q >= hr;
+            const int pi = second ? q - hr : q;
+            const int m = second ? hd - rp.r : rp.r;
+            const double turns = static_cast<double>(pos) * rp.inv_freq[second ? 1 : 0][pi] * 0.15915494309189533577;
+            const float ang = static_cast<float>((turns - floor(turns)) * 6.28318530717958647692);
+            float sn, cs;
+            sincosf(ang, &sn, &cs);
+            const float ra = v[0] * cs - v[1] * sn, rb = v[0] * sn + v[1] * cs;
+            if (head < rp.n_q) {
+                float* dst = rp.q_out + (static_cast<int64_t>(t) * rp.n_q + head) * hd + (second ? rp.r : 0);
+                dst[pi] = ra * rp.q_scale;
+                dst[pi + m / 2] = rb * rp.q_scale;
+            } else {
+                const int gk = head - rp.n_q;
+                const int64_t rowi = (static_cast<int64_t>(t) * rp.n_kv + gk) * rp.cap + pos;
+                __nv_bfloat16* dst = second ? rp.k2c + rowi * (hd - rp.r) : rp.k1c + rowi * rp.r;
+                dst[pi] = __float2bfloat16_rn(ra);
+                dst[pi + m / 2] = __float2bfloat16_rn(rb);
+            }
+        });
+}
+
+template <int TB>
+int qkv_rope_launch_one(spark_ctx* ctx, const QkvRopeParams& p, size_t smem, int grid, cudaStream_t stream) {
+    static bool configured[64] = {};
+    auto kern = qkv_rope_kernel<TB>;
+    if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        configured[ctx->device] = true;
+    }
+    kern<<<grid, kThreads, smem, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
 }  // namespace
 
 namespace spark {
@@ -269,15 +385,8 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     double* zs = reinterpret_cast<double*>(h2 + B * cfg->d);   // [B] threshold quantiles (8-byte aligned: see below)
     float* lsum = reinterpret_cast<float*>(zs + B);            // [B][n_q] sums of attention weights
 
-    // 1. a = RMSNorm(h; norm1); [q|k|v] = Wqkv a
-    GemvArgs g1;
-    g1.x = h; g1.norm_w = w->norm1; g1.rms_eps = cfg->rms_eps; g1.Wt = w->Wqkv; g1.wdtype = SPARK_BF16;
-    g1.B = B; g1.n_in = cfg->d; g1.n_out = nqkv; g1.y_add = nullptr; g1.y = qkv;
-    g1.x_div = nullptr; g1.x_div_group = 1; g1.zero_ptr = nullptr; g1.zero_bytes = 0;
-    int rc = gemv_launch(ctx, g1, st);
-    if (rc != SPARK_OK) return rc;
-
-    // 2. rotary encoding per half, query scale, cache append
+    // 1 + 2. a = RMSNorm(h; norm1); [q|k|v] = Wqkv a; rotary encoding per half, query scale, cache
+    //        append -- one kernel when the batch's inputs fit in shared memory together, else two.
     RopeParams rp;
     rp.qkv = qkv; rp.q_out = qr;
     rp.k1c = static_cast<__nv_bfloat16*>(cache->k1c); rp.k2c = static_cast<__nv_bfloat16*>(cache->k2c);
@@ -293,7 +402,30 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     }
     rp.zs = zs; rp.window = static_cast<int>(cfg->window > 0x7fffffff ? 0x7fffffff : cfg->window);
     rp.k_attn = static_cast<int>(cfg->k_attn > 0x7fffffff ? 0x7fffffff : cfg->k_attn);
-    {
+    int rc;
+    const int tbq = B == 1 ? 1 : (B <= 4 ? 4 : 16);
+    const size_t smem_q = static_cast<size_t>(tbq) * cfg->d * 4;
+    if ((cfg->d & 7) == 0 && smem_q <= static_cast<size_t>(ctx->max_smem_optin - 1024) && nqkv / 2 >= 1 &&
+        aligned16(w->Wqkv) && aligned16(w->norm1)) {
+        QkvRopeParams qp;
+        qp.g.x = h; qp.g.norm_w = w->norm1; qp.g.eps = cfg->rms_eps; qp.g.Wt = w->Wqkv;
+        qp.g.B = static_cast<int>(B); qp.g.n_in = static_cast<int>(cfg->d); qp.g.n_out = static_cast<int>(nqkv);
+        qp.g.y_add = nullptr; qp.g.y = nullptr; qp.g.x_div = nullptr; qp.g.x_div_group = 1;
+        qp.g.zero_ptr = nullptr; qp.g.zero_n16 = 0;
+        qp.r = rp;
+        const int64_t pairs = nqkv / 2;
+        const int gridq = pairs < ctx->num_sms ? static_cast<int>(pairs) : ctx->num_sms;
+        rc = tbq == 1 ? qkv_rope_launch_one<1>(ctx, qp, smem_q, gridq, st)
+                      : (tbq == 4 ? qkv_rope_launch_one<4>(ctx, qp, smem_q, gridq, st)
+                                  : qkv_rope_launch_one<16>(ctx, qp, smem_q, gridq, st));
+        if (rc != SPARK_OK) return rc;
+    } else {
+        GemvArgs g1;
+        g1.x = h; g1.norm_w = w->norm1; g1.rms_eps = cfg->rms_eps; g1.Wt = w->Wqkv; g1.wdtype = SPARK_BF16;
+        g1.B = B; g1.n_in = cfg->d; g1.n_out = nqkv; g1.y_add = nullptr; g1.y = qkv;
+        g1.x_div = nullptr; g1.x_div_group = 1; g1.zero_ptr = nullptr; g1.zero_bytes = 0;
+        rc = gemv_launch(ctx, g1, st);
+        if (rc != SPARK_OK) return rc;
         const int64_t total = B * (cfg->n_q + 2 * cfg->n_kv) * (cfg->hd / 2);
         const int blocks = static_cast<int>((total + 255) / 256);
         rope_append_kernel<<<blocks, 256, 0, st>>>(rp);
