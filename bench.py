@@ -33,7 +33,7 @@ import numpy as np
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from the ncu
 # capture summarised in profiles/ (keyed by shape and batch); None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("2b", 1): 24.23e6}       # profiles/ffn_b1.md
 
 FALLBACK_HBM_GBS = 6650.0
 
@@ -225,7 +225,7 @@ def run_spark(args):
                    r_attn=shape.r_attn, k_attn=shape.k_attn, window=window, cap=cap, rms_eps=1e-6,
                    rope_base=10000.0, flags=0)
         cfg_dense = dict(cfg, flags=S.SPARK_DENSE_LOADS)
-        layers.append((S.make_layer(w, cfg, cache), S.make_layer(w, cfg_dense, cache), w))
+        layers.append((S.make_layer(w, cfg, cache), S.make_layer(w, cfg_dense, cache), w, cache))
     h_init = torch.randn(B, d, device=dev, generator=gen)
     h = torch.empty_like(h_init)
     cl = torch.full((B,), ctx_len, dtype=torch.int32, device=dev)
@@ -337,6 +337,32 @@ def run_spark(args):
             ffn_calls()
 
     ms_ffn = timed(ffn_loop, args.steps, W)
+
+    # ---- the attention kernel alone, same caches (second largest share of the step) ------------------
+    qa = torch.randn(B, shape.n_q, hd, device=dev, generator=gen) / (hd ** 0.5)
+    oa = torch.empty(B, shape.n_q, hd, device=dev)
+
+    def attn_calls():
+        for l, lay in enumerate(layers):
+            c = lay[3]
+            win = 4096 if (l % 2 == 0 and ctx_len > 4096) else 0
+            S.spark_attn_decode(ctx, qa, c["k1c"], c["k2c"], c["vc"], S.SPARK_BF16, B, shape.n_q, shape.n_kv, hd,
+                                shape.r_attn, cap, cl, win, shape.k_attn, 0, oa, None, None, None, 0)
+
+    attn_graph = None
+    if not args.no_graph:
+        with torch.cuda.stream(side):
+            attn_calls()
+            side.synchronize()
+            attn_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(attn_graph, stream=side):
+                attn_calls()
+        torch.cuda.synchronize()
+    ms_attn = timed(lambda: attn_graph.replay() if attn_graph is not None else attn_calls(), args.steps, W)
+    attn_us = ms_attn * 1e3 / (args.steps * n_layers)
+    avg_ctx = (min(ctx_len, 4096) + ctx_len) / 2 if ctx_len > 4096 else ctx_len
+    attn_bytes = B * (shape.n_kv * avg_ctx * shape.r_attn * 2 +
+                      shape.n_q * min(shape.k_attn, avg_ctx) * ((hd - shape.r_attn) + hd) * 2)
     ffn_us = ms_ffn * 1e3 / (args.steps * n_layers)
     touched = shape.d_ff * shape.r_ff * 2 + union * (2 * d - shape.r_ff) * 2       # bytes per launch
     peak, peak_kind = measured_peak()
@@ -370,6 +396,10 @@ def run_spark(args):
             "roofline": {"kernel": "ffn_kernel (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
                          "us_per_launch": ffn_us, "touched_bytes_per_launch": touched, "union_rows": union},
+            "roofline_attention": {"kernel": "attn_kernel (spark_attn_decode)", "bound": "hbm",
+                                   "achieved": attn_bytes / (attn_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
+                                   "frac": attn_bytes / (attn_us * 1e-6) / 1e9 / peak, "us_per_launch": attn_us,
+                                   "touched_bytes_per_launch": attn_bytes, "traffic": None},
         }
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = cpu_baseline(args, shape)

@@ -82,18 +82,31 @@ __global__ void __launch_bounds__(kThreads) stat_topk_kernel(const TopkParams p)
     if (!p.identity) {
         // ---- sweep 1: the only HBM read of the row; sum -> mean --------------------------------
         float s0 = 0.f, s1 = 0.f;
-        for (int v = tid; v < nvec; v += kThreads) {
-            uint4 u = ld_stream16(gsrc + v);
-            float4 f = make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w));
-            const int nv = valid_in(v);
-            if (nv < 4) {
-                if (nv < 2) f.y = 0.f;
-                if (nv < 3) f.z = 0.f;
-                f.w = 0.f;
+        constexpr int LB = 8;                 // 16-byte loads a thread keeps in flight
+        for (int v0 = tid; v0 < nvec; v0 += kThreads * LB) {
+            uint4 u[LB];
+#pragma unroll
+            for (int j = 0; j < LB; ++j) {
+                const int v = v0 + j * kThreads;
+                if (v < nvec) u[j] = ld_stream16(gsrc + v);
+                else u[j] = make_uint4(0u, 0u, 0u, 0u);
             }
-            if (RESIDENT) ssrc[v] = f;
-            s0 += f.x + f.y;
-            s1 += f.z + f.w;
+#pragma unroll
+            for (int j = 0; j < LB; ++j) {
+                const int v = v0 + j * kThreads;
+                if (v < nvec) {
+                    float4 f = make_float4(__uint_as_float(u[j].x), __uint_as_float(u[j].y), __uint_as_float(u[j].z), __uint_as_float(u[j].w));
+                    const int nv = valid_in(v);
+                    if (nv < 4) {
+                        if (nv < 2) f.y = 0.f;
+                        if (nv < 3) f.z = 0.f;
+                        f.w = 0.f;
+                    }
+                    if (RESIDENT) ssrc[v] = f;
+                    s0 += f.x + f.y;
+                    s1 += f.z + f.w;
+                }
+            }
         }
         double bs = block_sum_f64(static_cast<double>(s0) + static_cast<double>(s1), red);
         if (tid == 0) part_sum = bs;
