@@ -1,0 +1,454 @@
+// Spark FFN (Section 2.1, Eq. 2) for 2..16 tokens per pass with bf16 weights: the three products
+// become small GEMMs (neurons x tokens), so they run on the tensor cores while the kernel stays
+// HBM-bound.  One cooperative kernel, one 512-thread block per SM, same phases as the one-token
+// kernel:
+//   A   S = K1t[rows of the block] . X[:, :r]^T         16-row tiles x 8-token tiles, K = r
+//   S   score sums into the grid-wide cells, theta per token (Eq. 11)
+//   C   per-token masks and the union list of the block's neurons (Appendix B: the union gates the
+//       loads, each token's own mask gates what enters its output)
+//   D1  T = K2t[union rows] . X[:, r:]^T, U = mask * GELU(S - theta) * T
+//   D2  Y^T += U . Vt[union rows]                          tokens x 64-column blocks, K = union rows
+// Tensor-core use: mma.sync m16n8k16 bf16 with fp32 accumulation.  The fp32 activations enter as an
+// exact three-way bf16 split (x = hi + mid + lo, one MMA per part), because the scores decide index
+// sets and must keep fp32 accuracy; u enters D2 as a two-way split.  Weight fragments are loaded
+// straight from global memory with 16-byte loads: the k-slots of an MMA may be any permutation of
+// the columns as long as both operands use the same one, so a lane's 8 consecutive bf16 of a row feed
+// two MMAs without any shuffle.  (The contraction is far too small for tcgen05 tiles: M = 16 rows,
+// N = 8 tokens; the kernel's time is the HBM stream.)
+#include "ffn_params.h"
+#include "kernels.h"
+
+using namespace spark;
+
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / kWarp;
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
+                                         unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ unsigned short bf16_bits(float f) { return __bfloat16_as_ushort(__float2bfloat16_rn(f)); }
+__device__ __forceinline__ float bf16_val(unsigned short b) { return __uint_as_float(static_cast<unsigned>(b) << 16); }
+
+// Shared-memory plan of the kernel (element counts), computed the same way on host and device.
+struct Plan {
+    int xs;        // row stride (bf16 elements) of the split activations: = 32 mod 64 keeps 16-byte fragment reads conflict-free
+    int us;        // row stride (bf16 elements) of the split u values: = 8 mod 64
+    __host__ __device__ Plan(int xw, int rpc) {
+        xs = ((xw + 63) / 64) * 64 + 32;
+        us = ((rpc + 15 + 63) / 64) * 64 + 8;
+    }
+};
+
+// S[tile rows][tokens] = W[rows] . X^T for the block's row tiles.  rowptr(i) gives the weight row of
+// the block's i-th row (i < nrows) -- rows beyond nrows contribute zeros.  The split activations
+// xs3[part][token][xs] cover K = 32 * nch columns.  emit(i, token, value) is called once per
+// (row, token) by some thread.  Called by the whole block; ends with a block sync.
+template <int NT, int CB, typename RowPtr, typename Emit>
+__device__ __forceinline__ void mma_rows(RowPtr rowptr, int nrows, int nch, const __nv_bfloat16* xs3, int xs, int tb_stride,
+                                         float4* part, Emit emit) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int MT = (nrows + 15) >> 4;
+    for (int mt0 = 0; mt0 < MT; mt0 += kWarps) {
+        const int mtn = min(kWarps, MT - mt0);                 // tiles in this group
+        int tp = 1;
+        while (tp < mtn) tp <<= 1;
+        const int ks = kWarps / tp;                            // warps that split K for one tile
+        const int tile = warp / ks, kp = warp - tile * ks;
+        const bool active = tile < mtn;
+        const int r_lo = (mt0 + tile) * 16 + g, r_hi = r_lo + 8;
+        const __nv_bfloat16* p_lo = (active && r_lo < nrows) ? rowptr(r_lo) : nullptr;
+        const __nv_bfloat16* p_hi = (active && r_hi < nrows) ? rowptr(r_hi) : nullptr;
+        float acc[NT][4];
+#pragma unroll
+        for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[n][e] = 0.f;
+        // CB chunks per batch: 2 * CB loads of 16 bytes in flight per lane
+#pragma unroll 1
+        for (int c0 = kp; c0 < nch; c0 += ks * CB) {
+            uint4 alo[CB], ahi[CB];
+#pragma unroll
+            for (int u = 0; u < CB; ++u) {
+                const int c = c0 + u * ks;
+                alo[u] = (p_lo != nullptr && c < nch) ? ld_stream16(reinterpret_cast<const uint4*>(p_lo) + 4 * c + t) : make_uint4(0u, 0u, 0u, 0u);
+                ahi[u] = (p_hi != nullptr && c < nch) ? ld_stream16(reinterpret_cast<const uint4*>(p_hi) + 4 * c + t) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < CB; ++u) {
+                const int c = c0 + u * ks;
+                if (c < nch && active) {
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+#pragma unroll
+                        for (int sp = 0; sp < 3; ++sp) {
+                            const uint4 b = *reinterpret_cast<const uint4*>(xs3 + static_cast<size_t>(sp) * tb_stride +
+                                                                            static_cast<size_t>(n * 8 + g) * xs + 32 * c + 8 * t);
+                            mma_bf16(acc[n], alo[u].x, ahi[u].x, alo[u].y, ahi[u].y, b.x, b.y);
+                            mma_bf16(acc[n], alo[u].z, ahi[u].z, alo[u].w, ahi[u].w, b.z, b.w);
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int n = 0; n < NT; ++n) part[(warp * NT + n) * 32 + lane] = make_float4(acc[n][0], acc[n][1], acc[n][2], acc[n][3]);
+        __syncthreads();
+        // sum the K-splits: value index = (tile, n, lane, e)
+        for (int i = tid; i < mtn * NT * 128; i += kThreads) {
+            const int e = i & 3, ln = (i >> 2) & 31, n = (i >> 7) % NT, tl = i / (128 * NT);
+            float v = 0.f;
+            for (int k = 0; k < ks; ++k) v += reinterpret_cast<const float*>(&part[((tl * ks + k) * NT + n) * 32 + ln])[e];
+            const int row = (mt0 + tl) * 16 + (ln >> 2) + ((e & 2) ? 8 : 0);
+            const int tok = n * 8 + (ln & 3) * 2 + (e & 1);
+            if (row < nrows) emit(row, tok, v);
+        }
+        __syncthreads();
+    }
+}
+
+template <int TB>
+__global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p) {
+    constexpr int NT = TB / 8;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const Plan plan(p.xw, p.rpc);
+    const int xs = plan.xs, us = plan.us, rpc = p.rpc;
+    const int tb_stride = TB * xs;                                                   // one split part
+    __nv_bfloat16* xs3 = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [3][TB][xs]
+    __nv_bfloat16* u2 = xs3 + 3 * tb_stride;                                         // [2][16][us]
+    float4* part = reinterpret_cast<float4*>(u2 + 2 * 16 * us);                      // [kWarps][NT][32]
+    float* s_loc = reinterpret_cast<float*>(part + kWarps * NT * 32);                // [TB][rpc]
+    int* ulist = reinterpret_cast<int*>(s_loc + static_cast<size_t>(TB) * rpc);      // [rpc]
+    unsigned* amask = reinterpret_cast<unsigned*>(ulist + rpc);                      // [rpc]
+    __shared__ float rstd[16];
+    __shared__ float theta_s[16];
+    __shared__ int wcnt[kWarps];
+    __shared__ unsigned tok_any;
+    __shared__ unsigned s_epoch;
+    __shared__ int s_fail;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grid = gridDim.x, cta = blockIdx.x;
+    const int row0 = static_cast<int>(static_cast<int64_t>(cta) * p.d_ff / grid);
+    const int row1 = static_cast<int>(static_cast<int64_t>(cta + 1) * p.d_ff / grid);
+    const int nloc = row1 - row0;
+    const int d = p.d, r = p.r, d2 = d - r;
+    const __nv_bfloat16* K1t = static_cast<const __nv_bfloat16*>(p.K1t);
+    const __nv_bfloat16* K2t = static_cast<const __nv_bfloat16*>(p.K2t);
+    const __nv_bfloat16* Vt = static_cast<const __nv_bfloat16*>(p.Vt);
+    if (tid == 0) {
+        s_epoch = ld_acquire_u32(&p.hdr->epoch);
+        s_fail = 0;
+    }
+    if (cta == 0) {      // clear the cells the launch after next will use (last used two launches ago)
+        const unsigned e = ld_acquire_u32(&p.hdr->epoch);
+        SumCell* c = &p.hdr->ffn_cells[(e + 2u) & 3u][0][0][0];
+        for (int i = tid; i < 4 * 16 * kCellWays; i += kThreads) { c[i].s1 = 0.0; c[i].s2 = 0.0; c[i].count = 0u; }
+    }
+    p.trace.mark(0);
+
+    for (int g0 = 0, grp = 0; g0 < p.B; g0 += TB, ++grp) {
+        const int tbv = min(TB, p.B - g0);
+        const float* xg = p.x + static_cast<int64_t>(g0) * d;
+        float* yg = p.y + static_cast<int64_t>(g0) * d;
+
+        // ---- prologue: RMSNorm scale, y initialisation, x[:r] split into shared memory ---------------
+        if (p.norm_w != nullptr) {
+            for (int t = warp; t < TB; t += kWarps) {
+                float ss = 0.f;
+                if (t < tbv) {
+                    const float4* xr = reinterpret_cast<const float4*>(xg + static_cast<int64_t>(t) * d);
+                    for (int i = lane; i < d / 4; i += 32) {
+                        const float4 v = xr[i];
+                        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+                    }
+                    ss = warp_sum(ss);
+                }
+                if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(d) + p.eps);
+            }
+            __syncthreads();
+        }
+        auto stage = [&](int col0, int width) {     // split x[t][col0:col0+width] (normalised) into three bf16 parts
+            const int w4 = width / 4;
+            constexpr int SB = 4;                    // loads a thread keeps in flight
+            for (int i0 = tid; i0 < TB * w4; i0 += kThreads * SB) {
+                float4 v[SB], w[SB];
+                int tt[SB], cc[SB];
+#pragma unroll
+                for (int j = 0; j < SB; ++j) {
+                    const int i = i0 + j * kThreads;
+                    tt[j] = i / w4;
+                    cc[j] = i - tt[j] * w4;
+                    v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    w[j] = make_float4(1.f, 1.f, 1.f, 1.f);
+                    if (i < TB * w4 && tt[j] < tbv) {
+                        v[j] = reinterpret_cast<const float4*>(xg + static_cast<int64_t>(tt[j]) * d + col0)[cc[j]];
+                        if (p.norm_w != nullptr) w[j] = reinterpret_cast<const float4*>(p.norm_w + col0)[cc[j]];
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < SB; ++j) {
+                    const int i = i0 + j * kThreads;
+                    if (i >= TB * w4) break;
+                    const float sc = (p.norm_w != nullptr && tt[j] < tbv) ? rstd[tt[j]] : 1.f;
+                    const float f[4] = {v[j].x * sc * w[j].x, v[j].y * sc * w[j].y, v[j].z * sc * w[j].z, v[j].w * sc * w[j].w};
+                    unsigned short h[4], m[4], l[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        h[e] = bf16_bits(f[e]);
+                        const float r1 = f[e] - bf16_val(h[e]);
+                        m[e] = bf16_bits(r1);
+                        l[e] = bf16_bits(r1 - bf16_val(m[e]));
+                    }
+                    __nv_bfloat16* dst = xs3 + static_cast<size_t>(tt[j]) * xs + 4 * cc[j];
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(h[0] | (static_cast<unsigned>(h[1]) << 16), h[2] | (static_cast<unsigned>(h[3]) << 16));
+                    *reinterpret_cast<uint2*>(dst + tb_stride) = make_uint2(m[0] | (static_cast<unsigned>(m[1]) << 16), m[2] | (static_cast<unsigned>(m[3]) << 16));
+                    *reinterpret_cast<uint2*>(dst + 2 * tb_stride) = make_uint2(l[0] | (static_cast<unsigned>(l[1]) << 16), l[2] | (static_cast<unsigned>(l[3]) << 16));
+                }
+            }
+        };
+        stage(0, r);
+        {
+            const int64_t total4 = static_cast<int64_t>(tbv) * d / 4;
+            const float4* yi = p.y_init ? reinterpret_cast<const float4*>(p.y_init + static_cast<int64_t>(g0) * d) : nullptr;
+            float4* yo = reinterpret_cast<float4*>(yg);
+            for (int64_t i = static_cast<int64_t>(cta) * kThreads + tid; i < total4; i += static_cast<int64_t>(grid) * kThreads)
+                yo[i] = yi ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (cta == 0 && p.count != nullptr && tid < tbv) p.count[g0 + tid] = 0;
+        if (tid == 0) tok_any = 0u;
+        __syncthreads();
+        p.trace.mark(1);
+
+        // ---- phase A: predictor scores of this block's neurons (zero-padded K when r % 32 != 0) ------
+        mma_rows<NT, 8>([&](int i) { return K1t + static_cast<int64_t>(row0 + i) * r; }, nloc, r / 32, xs3, xs, tb_stride, part,
+                     [&](int i, int tok, float v) { s_loc[static_cast<size_t>(tok) * rpc + i] = v; });
+        p.trace.mark(2);
+
+        // ---- score sums into the token's cells, arrival released after them ------------------------------
+        SumCell* cells = &p.hdr->ffn_cells[s_epoch & 3u][grp & 3][0][0];   // [token][way]
+        for (int t = warp; t < tbv; t += kWarps) {
+            const float* sr = s_loc + static_cast<size_t>(t) * rpc;
+            double s1 = 0.0, s2 = 0.0;
+            for (int j = lane; j < nloc; j += 32) {
+                const double v = static_cast<double>(sr[j]);
+                s1 += v;
+                s2 = fma(v, v, s2);
+            }
+            s1 = warp_sum_f64(s1);
+            s2 = warp_sum_f64(s2);
+            if (lane == 0) cells_add(cells + t * kCellWays, cta, s1, s2);
+        }
+        p.trace.mark(3);
+        __syncthreads();
+        stage(r, d2);                                   // x[r:] replaces x[:r] while the cells fill
+        for (int i = tid; i < 2 * 16 * us / 2; i += kThreads) reinterpret_cast<unsigned*>(u2)[i] = 0u;
+        for (int t = warp; t < tbv; t += kWarps) {
+            double sa, sb;
+            const bool ok = cells_wait(cells + t * kCellWays, static_cast<unsigned>(grid), sa, sb, p.hdr);
+            if (lane == 0) {
+                float th = -INFINITY;
+                if (!ok) s_fail = 1;
+                if (!p.identity) {
+                    const double mean = sa * p.inv_n;
+                    const float var = static_cast<float>((sb - sa * mean) * p.inv_nm1);
+                    th = static_cast<float>(mean) + sqrtf(fmaxf(var, 0.f)) * static_cast<float>(p.z);
+                }
+                theta_s[t] = th;
+                if (cta == 0 && p.theta != nullptr) p.theta[g0 + t] = th;
+            }
+        }
+        __syncthreads();
+        if (s_fail) return;
+        p.trace.mark(4);
+
+        // ---- phase C: masks and the ordered union list of this block's neurons --------------------------
+        int nU = 0;
+        for (int j0 = 0; j0 < nloc; j0 += kThreads) {
+            const int j = j0 + tid;
+            unsigned m = 0u;
+            if (j < nloc) {
+#pragma unroll
+                for (int t = 0; t < TB; ++t)
+                    if (t < tbv && s_loc[static_cast<size_t>(t) * rpc + j] > theta_s[t]) m |= 1u << t;
+                amask[j] = m;
+            }
+            const bool in = j < nloc && (m != 0u || p.dense);
+            const unsigned bal = __ballot_sync(kFull, in);
+            if (lane == 0) wcnt[warp] = __popc(bal);
+            if (m != 0u) atomicOr(&tok_any, m);
+            __syncthreads();
+            int before = 0, all = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                if (w < warp) before += wcnt[w];
+                all += wcnt[w];
+            }
+            if (in) ulist[nU + before + __popc(bal & ((1u << lane) - 1u))] = j;
+            nU += all;
+            __syncthreads();
+        }
+        if (p.count != nullptr) {
+            for (int t = warp; t < tbv; t += kWarps) {
+                int c = 0;
+                for (int j = lane; j < nloc; j += 32) c += (amask[j] >> t) & 1u;
+                c = warp_sum_int(c);
+                int base = 0;
+                if (lane == 0 && c > 0) base = atomicAdd(&p.count[g0 + t], c);
+                base = __shfl_sync(kFull, base, 0);
+                if (p.idx != nullptr && c > 0) {
+                    int32_t* out = p.idx + static_cast<int64_t>(g0 + t) * p.d_ff;
+                    for (int j0 = 0; j0 < nloc; j0 += 32) {
+                        const int j = j0 + lane;
+                        const bool a = j < nloc && ((amask[j] >> t) & 1u);
+                        const unsigned bal = __ballot_sync(kFull, a);
+                        if (a) out[base + __popc(bal & ((1u << lane) - 1u))] = row0 + j;
+                        base += __popc(bal);
+                    }
+                }
+            }
+        }
+        p.trace.mark(5);
+
+        // ---- D1: T = K2t[union rows] . X[:, r:]^T; U = mask * GELU(S - theta) * T, split in two bf16 parts
+        mma_rows<NT, 10>([&](int i) { return K2t + static_cast<int64_t>(row0 + ulist[i]) * d2; }, nU, d2 / 32, xs3, xs, tb_stride, part,
+                     [&](int i, int tok, float tv) {
+                         const int j = ulist[i];
+                         float u = 0.f;
+                         if ((amask[j] >> tok) & 1u) {
+                             const float a = s_loc[static_cast<size_t>(tok) * rpc + j] - (p.identity ? 0.f : theta_s[tok]);
+                             u = (p.erf_form ? gelu_erf(a) : gelu_tanh(a)) * tv;
+                         }
+                         const unsigned short h = bf16_bits(u);
+                         u2[static_cast<size_t>(tok) * us + i] = __ushort_as_bfloat16(h);
+                         u2[static_cast<size_t>(16 + tok) * us + i] = __float2bfloat16_rn(u - bf16_val(h));
+                     });
+        p.trace.mark(6);
+
+        // ---- D2: Y^T += U . Vt[union rows]; a warp owns 64-column blocks, K = union rows in steps of 16
+        {
+            const int g = lane >> 2, t = lane & 3;
+            const int ncb = d / 64;                          // full 64-column blocks (d % 64 handled below)
+            const unsigned anyt = tok_any;
+            const int nks = (nU + 15) >> 4;
+            for (int cb = warp; cb * 64 < d; cb += kWarps) {
+                const bool full = cb < ncb;
+                float acc[8][4];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+                constexpr int KB = 4;                        // k-steps per batch: 16 loads of 16 bytes in flight per lane
+#pragma unroll 1
+                for (int k0 = 0; k0 < nks; k0 += KB) {
+                    uint4 rv[KB][4];
+#pragma unroll
+                    for (int kk = 0; kk < KB; ++kk) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int ui = (k0 + kk) * 16 + 2 * t + (q & 1) + (q >> 1) * 8;
+                            const int col = cb * 64 + 8 * g;
+                            rv[kk][q] = (ui < nU && (full || col + 8 <= d))
+                                            ? ld_stream16(reinterpret_cast<const uint4*>(Vt + static_cast<int64_t>(row0 + ulist[ui]) * d + col))
+                                            : make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < KB; ++kk) {
+                        if (k0 + kk < nks) {
+                            const int kb = (k0 + kk) * 16;
+                            unsigned a[2][4];
+#pragma unroll
+                            for (int sp = 0; sp < 2; ++sp) {
+                                const __nv_bfloat16* ub = u2 + static_cast<size_t>(sp * 16) * us + kb + 2 * t;
+                                a[sp][0] = *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g) * us);
+                                a[sp][1] = TB > 8 ? *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g + 8) * us) : 0u;
+                                a[sp][2] = *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g) * us + 8);
+                                a[sp][3] = TB > 8 ? *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g + 8) * us + 8) : 0u;
+                            }
+                            const unsigned wa[4] = {rv[kk][0].x, rv[kk][0].y, rv[kk][0].z, rv[kk][0].w};
+                            const unsigned wb[4] = {rv[kk][1].x, rv[kk][1].y, rv[kk][1].z, rv[kk][1].w};
+                            const unsigned wc[4] = {rv[kk][2].x, rv[kk][2].y, rv[kk][2].z, rv[kk][2].w};
+                            const unsigned wd[4] = {rv[kk][3].x, rv[kk][3].y, rv[kk][3].z, rv[kk][3].w};
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const unsigned sel = (i & 1) ? 0x7632u : 0x5410u;
+                                const unsigned b0 = __byte_perm(wa[i >> 1], wb[i >> 1], sel);
+                                const unsigned b1 = __byte_perm(wc[i >> 1], wd[i >> 1], sel);
+#pragma unroll
+                                for (int sp = 0; sp < 2; ++sp) mma_bf16(acc[i], a[sp][0], a[sp][1], a[sp][2], a[sp][3], b0, b1);
+                            }
+                        }
+                    }
+                }
+                // lane holds, for tokens g and g + 8, columns cb*64 + 16 t + [0, 8) (element 0 of tile i) and + 8 + [0, 8) (element 1)
+                const int colb = cb * 64 + 16 * t;
+#pragma unroll
+                for (int hrow = 0; hrow < 2; ++hrow) {
+                    const int tok = g + 8 * hrow;
+                    if (tok < tbv && ((anyt >> tok) & 1u)) {
+                        float* dst = yg + static_cast<int64_t>(tok) * d + colb;
+                        const int e0 = 2 * hrow;
+                        if (colb + 8 <= d) {
+                            red_add_v4(dst, acc[0][e0], acc[1][e0], acc[2][e0], acc[3][e0]);
+                            red_add_v4(dst + 4, acc[4][e0], acc[5][e0], acc[6][e0], acc[7][e0]);
+                        }
+                        if (colb + 16 <= d) {
+                            red_add_v4(dst + 8, acc[0][e0 + 1], acc[1][e0 + 1], acc[2][e0 + 1], acc[3][e0 + 1]);
+                            red_add_v4(dst + 12, acc[4][e0 + 1], acc[5][e0 + 1], acc[6][e0 + 1], acc[7][e0 + 1]);
+                        }
+                    }
+                }
+            }
+        }
+        p.trace.mark(7);
+        __syncthreads();      // shared buffers are reused by the next token group
+    }
+    if (cta == 0 && tid == 0) p.hdr->epoch = s_epoch + 1u;   // every block has read the epoch by now
+}
+
+template <int TB>
+int launch_mma(spark_ctx* ctx, FfnParams& p, cudaStream_t stream) {
+    static bool configured[64] = {};
+    const Plan plan(p.xw, p.rpc);
+    const size_t smem = static_cast<size_t>(3) * TB * plan.xs * 2 + static_cast<size_t>(2) * 16 * plan.us * 2 +
+                        static_cast<size_t>(kWarps) * (TB / 8) * 32 * 16 + static_cast<size_t>(TB) * p.rpc * 4 +
+                        static_cast<size_t>(p.rpc) * 8 + 64;
+    if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_WORKSPACE;   // caller falls back
+    auto kern = ffn_mma_kernel<TB>;
+    if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        configured[ctx->device] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctx->num_sms));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, p) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+}  // namespace
+
+namespace spark {
+
+// bf16 weights, 2..64 tokens.  Returns SPARK_ERR_WORKSPACE when the shape does not fit this kernel's
+// shared-memory plan or its layout rules (the caller then uses the plain-ALU kernel).
+int ffn_mma_launch(spark_ctx* ctx, FfnParams& p, cudaStream_t stream) {
+    if ((p.r & 31) != 0 || ((p.d - p.r) & 31) != 0 || (p.d & 15) != 0) return SPARK_ERR_WORKSPACE;
+    if (p.B <= 8) return launch_mma<8>(ctx, p, stream);
+    return launch_mma<16>(ctx, p, stream);
+}
+
+}  // namespace spark

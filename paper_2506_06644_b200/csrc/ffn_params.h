@@ -29,6 +29,10 @@ struct FfnParams {
 };
 
 
+// Tensor-core path for bf16 weights and 2..64 tokens (ffn_mma.cu); SPARK_ERR_WORKSPACE = shape not
+// served, use the plain-ALU kernel.
+int ffn_mma_launch(spark_ctx* ctx, FfnParams& p, cudaStream_t stream);
+
 // B == 1 fast path (ffn_b1.cu).
 int ffn1_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream);
 
