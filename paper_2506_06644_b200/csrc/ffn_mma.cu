@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
         }
         auto stage = [&](int col0, int width) {     // split x[t][col0:col0+width] (normalised) into three bf16 parts
             const int w4 = width / 4;
-            constexpr int SB = 4;                    // loads a thread keeps in flight
+            constexpr int SB = 8;                    // loads a thread keeps in flight
             for (int i0 = tid; i0 < TB * w4; i0 += kThreads * SB) {
                 float4 v[SB], w[SB];
                 int tt[SB], cc[SB];
@@ -330,8 +330,105 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
                      });
         p.trace.mark(6);
 
-        // ---- D2: Y^T += U . Vt[union rows]; a warp owns 64-column blocks, K = union rows in steps of 16
+        // ---- D2: Y^T += U . Vt[union rows].  The union rows are staged stripe by stripe into the shared
+        //      memory the activation splits no longer need (cp.async: every thread's requests are in flight
+        //      at once, no registers held), B fragments come out of it with ldmatrix.trans, a warp owns
+        //      64-column blocks, K = union rows in steps of 16.
         {
+            const int g = lane >> 2, t = lane & 3;
+            const unsigned anyt = tok_any;
+            const int nUp = (nU + 15) & ~15, nks = nUp >> 4;
+            unsigned char* vs = smem_raw;                                  // reuses xs3
+            const int sv_bytes = 3 * tb_stride * 2;
+            // two staging buffers: the next stripe's rows are requested while the current one is multiplied
+            int WC = nUp > 0 ? (((sv_bytes / 2 / nUp) - 16) / 2) & ~63 : 0;
+            if (WC > ((d + 63) & ~63)) WC = (d + 63) & ~63;
+            const int RS = WC * 2 + 16;                                    // row stride: 16 mod 128 bytes
+            const unsigned vs_base = static_cast<unsigned>(__cvta_generic_to_shared(vs));
+            if (nU > 0 && WC >= 64) {
+                auto request = [&](int col0, int buf) {
+                    const int wc = min(WC, d - col0), nch8 = wc >> 3;
+                    unsigned char* vb = vs + static_cast<size_t>(buf) * nUp * RS;
+                    const unsigned va = vs_base + buf * nUp * RS;
+                    for (int row = warp; row < nUp; row += kWarps) {       // a warp per row, lanes over 16-byte pieces
+                        if (row < nU) {
+                            const __nv_bfloat16* src = Vt + static_cast<int64_t>(row0 + ulist[row]) * d + col0;
+                            for (int ch = lane; ch < nch8; ch += 32)
+                                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(va + row * RS + ch * 16), "l"(src + ch * 8) : "memory");
+                        } else {
+                            for (int ch = lane; ch < nch8; ch += 32)
+                                *reinterpret_cast<uint4*>(vb + row * RS + ch * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+                    asm volatile("cp.async.commit_group;" ::: "memory");
+                };
+                request(0, 0);
+                int buf = 0;
+                for (int col0 = 0; col0 < d; col0 += WC, buf ^= 1) {
+                    const int wc = min(WC, d - col0);
+                    if (col0 + WC < d) {
+                        request(col0 + WC, buf ^ 1);
+                        asm volatile("cp.async.wait_group 1;" ::: "memory");
+                    } else {
+                        asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    }
+                    __syncthreads();
+                    const unsigned vs_addr = vs_base + buf * nUp * RS;
+                    const int nblk = (wc + 63) >> 6;
+                    for (int cb = warp; cb < nblk; cb += kWarps) {
+                        float acc[8][4];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+#pragma unroll 1
+                        for (int ks = 0; ks < nks; ++ks) {
+                            const int kb = ks * 16;
+                            unsigned a[2][4];
+#pragma unroll
+                            for (int sp = 0; sp < 2; ++sp) {
+                                const __nv_bfloat16* ub = u2 + static_cast<size_t>(sp * 16) * us + kb + 2 * t;
+                                a[sp][0] = *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g) * us);
+                                a[sp][1] = TB > 8 ? *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g + 8) * us) : 0u;
+                                a[sp][2] = *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g) * us + 8);
+                                a[sp][3] = TB > 8 ? *reinterpret_cast<const unsigned*>(ub + static_cast<size_t>(g + 8) * us + 8) : 0u;
+                            }
+                            // lane l addresses row (l & 7) of matrix l >> 3: matrices 0,1 = rows kb.., kb+8.. of
+                            // column tile 2q; matrices 2,3 = the same rows of column tile 2q + 1
+                            const int mrow = kb + ((lane >> 3) & 1) * 8 + (lane & 7);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const int mcol = cb * 64 + (2 * q + (lane >> 4)) * 8;
+                                unsigned b0, b1, b2, b3;
+                                asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                                             : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3)
+                                             : "r"(vs_addr + mrow * RS + mcol * 2));
+#pragma unroll
+                                for (int sp = 0; sp < 2; ++sp) {
+                                    mma_bf16(acc[2 * q], a[sp][0], a[sp][1], a[sp][2], a[sp][3], b0, b1);
+                                    mma_bf16(acc[2 * q + 1], a[sp][0], a[sp][1], a[sp][2], a[sp][3], b2, b3);
+                                }
+                            }
+                        }
+                        // lane holds tokens g and g + 8, columns cb*64 + 8 i + 2 t, + 1 of tile i
+#pragma unroll
+                        for (int hrow = 0; hrow < 2; ++hrow) {
+                            const int tok = g + 8 * hrow;
+                            if (tok < tbv && ((anyt >> tok) & 1u)) {
+                                float* dst = yg + static_cast<int64_t>(tok) * d + col0 + cb * 64 + 2 * t;
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    if (cb * 64 + 8 * i + 2 * t < wc)
+                                        asm volatile("red.global.add.v2.f32 [%0], {%1,%2};" ::"l"(dst + 8 * i), "f"(acc[i][2 * hrow]),
+                                                     "f"(acc[i][2 * hrow + 1])
+                                                     : "memory");
+                                }
+                            }
+                        }
+                    }
+                    __syncthreads();      // this buffer is requested into again two stripes later
+                }
+            } else if (nU > 0) {
             const int g = lane >> 2, t = lane & 3;
             const int ncb = d / 64;                          // full 64-column blocks (d % 64 handled below)
             const unsigned anyt = tok_any;
@@ -404,6 +501,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
                         }
                     }
                 }
+            }
             }
         }
         p.trace.mark(7);
