@@ -1,10 +1,12 @@
 // spark_stat_topk: standalone statistical top-k over many rows (Section 3, Eq. 9-11).
 //
-// One thread-block cluster per row.  Each block of the cluster streams its contiguous part of the
-// row from HBM exactly once into shared memory, and every later sweep (squared deviations around
-// the exact mean, counting, ordered compaction / dense output) reads shared memory.  Partial sums
-// travel between the blocks of a cluster through distributed shared memory.  Rows too long to be
-// held on chip fall back to re-reading global memory in the later sweeps.
+// Two kernels.  Rows of 16K..64K values: one persistent block per SM holds a whole row on chip
+// (stat_topk_row_kernel below).  All other lengths: one thread-block cluster per row; each block
+// of the cluster streams its contiguous part of the row from HBM exactly once into shared memory,
+// and every later sweep (squared deviations around the exact mean, counting, ordered compaction /
+// dense output) reads shared memory.  Partial sums travel between the blocks of a cluster through
+// distributed shared memory.  Rows too long to be held on chip fall back to re-reading global
+// memory in the later sweeps.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
@@ -238,6 +240,377 @@ __global__ void __launch_bounds__(kThreads) stat_topk_kernel(const TopkParams p)
     cluster.sync();   // no block may leave while a peer can still read its shared memory
 }
 
+// ---------------------------------------------------------------------------------------------
+// Rows of 16K..64K values: a persistent 512-thread block per SM keeps one whole row on chip -- the
+// leading part (up to 184 KB) in shared memory, brought in by bulk asynchronous copies that signal
+// one mbarrier per 32 KB piece, and the last (up to) 4608 float4 in registers, nine per thread.  The
+// register part is double-buffered: the next row's is requested as soon as the current row's last
+// piece has landed, so HBM stays busy while the block reduces, counts and writes its lists; the
+// next row's bulk copies start when the last sweep over shared memory is done.  Each row is read
+// from HBM exactly once.  The sums are those of (x - c) and (x - c)^2 around c = the row's first
+// value (shifting keeps the fp32 partial sums accurate when |mean| >> std); they are combined in fp64.
+//
+// Selection: every thread owns a run of 23 consecutive float4 in shared memory (an odd run length
+// keeps the 16-byte reads of a quarter warp on distinct banks); the register part is owned warp by
+// warp, lane-strided, as it was loaded.  The counting sweep leaves one bit per value; scans of the counts
+// give each run its rank; a warp's share of the lists is contiguous and goes through a 256-entry
+// staging window of its own in shared memory, so that it leaves the SM as coalesced stores.
+// ---------------------------------------------------------------------------------------------
+constexpr int kRowThreads = 512;
+constexpr int kRowWarps = kRowThreads / 32;
+constexpr int kRowRegVec = 9;                                    // float4 per thread kept in registers
+constexpr int kRowRunVec = 23;                                   // float4 per thread in shared memory
+constexpr int kRowSmemVec = kRowRunVec * kRowThreads;            // 11776 float4 = 184 KB
+constexpr int kRowPieceVec = 2048;                               // float4 per bulk copy (32 KB)
+constexpr int kRowPieces = (kRowSmemVec + kRowPieceVec - 1) / kRowPieceVec;   // 12 (the last one is half)
+constexpr int kRowMaxVec = kRowSmemVec + kRowRegVec * kRowThreads;   // 16384 float4 = 65536 values
+constexpr int kRowWin = 256;                                     // entries of a warp's staging window
+constexpr int kRowSmemBytes = kRowSmemVec * 16 + kRowWarps * kRowWin * 8;
+constexpr long long kRowSpinLimit = 400000000ll;                 // bound of a wait for one 32 KB copy
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > kRowSpinLimit) return false;
+    return true;
+}
+
+struct RowGeom {
+    int n, nvec, ns, npiece;
+};
+
+// Thread 0: start the bulk copies of one row's shared-memory part.
+__device__ __forceinline__ void row_issue_bulk(const float* xrow, float* srow, unsigned long long* mbar, const RowGeom& g) {
+    for (int c = 0; c < g.npiece; ++c) {
+        const int vec = min(kRowPieceVec, g.ns - c * kRowPieceVec);
+        const uint32_t bytes = static_cast<uint32_t>(vec) * 16u, bar = smem_u32(mbar + c);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(smem_u32(srow + c * kRowPieceVec * 4)), "l"(xrow + static_cast<int64_t>(c) * kRowPieceVec * 4), "r"(bytes), "r"(bar)
+                     : "memory");
+    }
+}
+// All threads: request one row's register part (warp w, lane l: vectors ns + w*288 + i*32 + l).
+__device__ __forceinline__ void row_load_regs(const float* xrow, const RowGeom& g, uint4 (&r)[kRowRegVec]) {
+    const int v0 = g.ns + static_cast<int>(threadIdx.x >> 5) * (kRowRegVec * 32) + static_cast<int>(threadIdx.x & 31);
+    const uint4* gsrc = reinterpret_cast<const uint4*>(xrow);
+#pragma unroll
+    for (int i = 0; i < kRowRegVec; ++i) r[i] = v0 + i * 32 < g.nvec ? ld_stream16_pinned(gsrc + v0 + i * 32) : make_uint4(0u, 0u, 0u, 0u);
+}
+
+struct RowShared {
+    unsigned long long mbar[kRowPieces];
+    double red1[kRowWarps], red2[kRowWarps];
+    int scan[kRowWarps];
+    float theta;
+    int abort;
+};
+
+// One row: cur holds its register part, nxt receives the next row's.  Returns false after a timeout.
+__device__ __forceinline__ bool row_body(const TopkParams& p, const RowGeom& g, float* srow, RowShared& sh, int64_t row, int64_t next_row,
+                                         uint32_t parity, uint4 (&cur)[kRowRegVec], uint4 (&nxt)[kRowRegVec], float c, float& c_next) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float4* ssrc = reinterpret_cast<const float4*>(srow);
+    const int rv0 = g.ns + warp * (kRowRegVec * 32) + lane;           // register vectors: rv0 + 32 * i
+    const int sv0 = tid * kRowRunVec;                                 // first shared-memory vector of its run
+    const int last_nv = g.n - ((g.nvec - 1) << 2);                    // valid values of the last vector (1..4)
+    auto f4 = [](const uint4& u) { return make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w)); };
+
+    float a1 = 0.f, a2 = 0.f;
+    auto accumulate = [&](const float4& f) {
+        const float d0 = f.x - c, d1 = f.y - c, d2 = f.z - c, d3 = f.w - c;
+        a1 += (d0 + d1) + (d2 + d3);
+        a2 = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, fmaf(d3, d3, a2))));
+    };
+    bool ok = true;
+    if (!p.identity) {
+#pragma unroll
+        for (int i = 0; i < kRowRegVec; ++i) {
+            const int v = rv0 + i * 32;
+            if (v < g.nvec) {
+                float4 f = f4(cur[i]);
+                if (v == g.nvec - 1) {                                 // a ragged tail counts as c (adds nothing)
+                    if (last_nv < 2) f.y = c;
+                    if (last_nv < 3) f.z = c;
+                    if (last_nv < 4) f.w = c;
+                }
+                accumulate(f);
+            }
+        }
+    }
+    // the shared-memory part, piece by piece as the copies land
+    for (int pc = 0; pc < g.npiece; ++pc) {
+        ok = mbar_wait(smem_u32(sh.mbar + pc), parity) && ok;
+        if (!p.identity) {
+#pragma unroll
+            for (int h = 0; h < kRowPieceVec / kRowThreads; ++h) {
+                const int v = pc * kRowPieceVec + h * kRowThreads + tid;
+                if (v < g.ns) accumulate(ssrc[v]);
+            }
+        }
+    }
+    // HBM would idle from here to the end of the row: fetch the next row's register part meanwhile
+    if (next_row < p.rows) {
+        const float* xn = p.x + next_row * p.ld;
+        c_next = p.identity ? 0.f : __ldg(xn);
+        row_load_regs(xn, g, nxt);
+    }
+
+    float theta = -INFINITY;
+    {
+        const double w1 = warp_sum_f64(static_cast<double>(a1)), w2 = warp_sum_f64(static_cast<double>(a2));
+        if (lane == 0) { sh.red1[warp] = w1; sh.red2[warp] = w2; }
+        if (!ok) sh.abort = 1;
+        __syncthreads();
+        if (warp == 0) {
+            double t1 = lane < kRowWarps ? sh.red1[lane] : 0.0, t2 = lane < kRowWarps ? sh.red2[lane] : 0.0;
+            t1 = warp_sum_f64(t1);
+            t2 = warp_sum_f64(t2);
+            if (lane == 0) {
+                const double nn = static_cast<double>(g.n);
+                const double mean = static_cast<double>(c) + t1 / nn;
+                double m2 = t2 - t1 * t1 / nn;
+                if (m2 < 0.0) m2 = 0.0;
+                sh.theta = p.identity ? -INFINITY : theta_from(Moments{nn, mean, m2}, p.z);
+            }
+        }
+        __syncthreads();
+        theta = sh.theta;
+        if (sh.abort) return false;
+    }
+    const float shift = p.identity ? 0.f : theta;
+
+    // ---- count: one bit per value of the thread's two runs ------------------------------------------
+    unsigned ms[3] = {0u, 0u, 0u};                                    // 92 bits: shared-memory run
+    unsigned long long mr = 0ull;                                     // 36 bits: register run
+#pragma unroll
+    for (int i = 0; i < kRowRunVec; ++i) {
+        if (sv0 + i < g.ns) {
+            const float4 f = ssrc[sv0 + i];
+            const unsigned nib = (f.x > theta ? 1u : 0u) | (f.y > theta ? 2u : 0u) | (f.z > theta ? 4u : 0u) | (f.w > theta ? 8u : 0u);
+            ms[(4 * i) >> 5] |= nib << ((4 * i) & 31);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kRowRegVec; ++i) {
+        const int v = rv0 + i * 32;
+        if (v < g.nvec) {
+            const float4 f = f4(cur[i]);
+            unsigned nib = (f.x > theta ? 1u : 0u) | (f.y > theta ? 2u : 0u) | (f.z > theta ? 4u : 0u) | (f.w > theta ? 8u : 0u);
+            if (v == g.nvec - 1) nib &= (1u << last_nv) - 1u;
+            mr |= static_cast<unsigned long long>(nib) << (4 * i);
+        }
+    }
+    const int cs = __popc(ms[0]) + __popc(ms[1]) + __popc(ms[2]), cr = __popcll(mr);
+    // block-wide exclusive scan of (cs, cr), packed 16 + 16 bits (the totals stay below 2^16)
+    const int packed = cs | (cr << 16);
+    int inc = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) sh.scan[warp] = inc;
+    __syncthreads();
+    int base = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kRowWarps; ++w) {
+        const int a = sh.scan[w];
+        if (w < warp) base += a;
+        tot += a;
+    }
+    const int excl = base + inc - packed;
+    const int tot_s = tot & 0xffff, total = tot_s + (tot >> 16);
+    const bool want_lists = (p.idx != nullptr) || (p.val != nullptr);
+    if (tid == 0) {
+        if (p.theta) p.theta[row] = theta;
+        if (p.count) p.count[row] = total;
+        if (want_lists && total > p.idx_cap) atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_OVERFLOW);
+    }
+
+    // ---- ordered lists: each warp stages its (contiguous) share in a 256-entry window of its own -------
+    if (want_lists) {
+        int* wi = reinterpret_cast<int*>(srow + kRowSmemVec * 4) + warp * (2 * kRowWin);
+        float* wv = reinterpret_cast<float*>(wi + kRowWin);
+        int32_t* idx_row = p.idx ? p.idx + row * p.idx_cap : nullptr;
+        float* val_row = p.val ? p.val + row * p.idx_cap : nullptr;
+        const int wpacked = sh.scan[warp];
+        auto flush = [&](int first, int cnt) {                         // window -> lists, lanes over consecutive entries
+            __syncwarp();
+            for (int t = lane; t < cnt; t += 32) {
+                const int at = first + t;
+                if (at < p.idx_cap) {
+                    if (idx_row) idx_row[at] = wi[t];
+                    if (val_row) val_row[at] = wv[t];
+                }
+            }
+            __syncwarp();
+        };
+        // shared-memory runs: ranks of this warp start at wbase; a thread's values follow one another
+        {
+            const int wbase = base & 0xffff, wtot = wpacked & 0xffff;
+            int rel = (excl & 0xffff) - wbase;
+            unsigned long long lo = static_cast<unsigned long long>(ms[0]) | (static_cast<unsigned long long>(ms[1]) << 32);
+            unsigned hi = ms[2];
+            const int es = sv0 << 2;
+#pragma unroll 1
+            for (int w0 = 0; w0 < wtot; w0 += kRowWin) {
+                while ((lo != 0ull || hi != 0u) && rel < w0 + kRowWin) {
+                    const bool in_lo = lo != 0ull;
+                    const int bit = in_lo ? __ffsll(static_cast<long long>(lo)) - 1 : 63 + __ffs(hi);
+                    lo &= lo - (in_lo ? 1ull : 0ull);                  // lo == 0 stays 0
+                    hi &= hi - (in_lo ? 0u : 1u);
+                    wi[rel - w0] = es + bit;
+                    wv[rel - w0] = srow[es + bit] - shift;
+                    ++rel;
+                }
+                flush(wbase + w0, min(kRowWin, wtot - w0));
+            }
+        }
+        // register part: a warp owns 288 consecutive vectors, vector i of lane l being number 32 i + l of
+        // them.  Rank inside the warp = totals of the earlier i + the lower lanes' counts in this i + the
+        // lower neighbours in the vector.  The per-i counts (<= 4 per lane, <= 128 per warp) are scanned
+        // across the lanes four to a word.
+        const int wtot_r = wpacked >> 16;
+        if (wtot_r != 0) {
+            const int wbase = tot_s + (base >> 16);
+            unsigned exq[3], offs[5];                                  // lane prefixes (8 bits per i), starts of each i (16 bits)
+            {
+                unsigned q[3] = {0u, 0u, 0u};
+#pragma unroll
+                for (int i = 0; i < kRowRegVec; ++i) q[i >> 2] |= static_cast<unsigned>(__popc(static_cast<unsigned>(mr >> (4 * i)) & 15u)) << (8 * (i & 3));
+                unsigned inc_q[3] = {q[0], q[1], q[2]};
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+                    for (int w = 0; w < 3; ++w) {
+                        const unsigned t = __shfl_up_sync(kFull, inc_q[w], o);
+                        if (lane >= o) inc_q[w] += t;
+                    }
+                }
+                unsigned off = 0u;
+#pragma unroll
+                for (int w = 0; w < 5; ++w) offs[w] = 0u;
+#pragma unroll
+                for (int i = 0; i < kRowRegVec; ++i) {
+                    offs[i >> 1] |= off << (16 * (i & 1));
+                    off += (__shfl_sync(kFull, inc_q[i >> 2], 31) >> (8 * (i & 3))) & 0xffu;
+                }
+#pragma unroll
+                for (int w = 0; w < 3; ++w) exq[w] = inc_q[w] - q[w];
+            }
+#pragma unroll 1
+            for (int w0 = 0; w0 < wtot_r; w0 += kRowWin) {
+                for (unsigned long long m = mr; m != 0ull; m &= m - 1ull) {
+                    const int bit = __ffsll(static_cast<long long>(m)) - 1, i = bit >> 2, j = bit & 3;
+                    const unsigned ew = i < 4 ? exq[0] : (i < 8 ? exq[1] : exq[2]);
+                    const unsigned ow = i < 2 ? offs[0] : (i < 4 ? offs[1] : (i < 6 ? offs[2] : (i < 8 ? offs[3] : offs[4])));
+                    const unsigned nib = static_cast<unsigned>(mr >> (4 * i)) & 15u;
+                    const int rel = static_cast<int>((ow >> (16 * (i & 1))) & 0xffffu) + static_cast<int>((ew >> (8 * (i & 3))) & 0xffu) +
+                                    __popc(nib & ((1u << j) - 1u)) - w0;
+                    if (rel >= 0 && rel < kRowWin) {
+                        uint4 u = cur[0];                                 // registers cannot be indexed: select
+#pragma unroll
+                        for (int t = 1; t < kRowRegVec; ++t)
+                            if (i == t) u = cur[t];
+                        const unsigned bits = j == 0 ? u.x : (j == 1 ? u.y : (j == 2 ? u.z : u.w));
+                        wi[rel] = ((rv0 + 32 * i) << 2) + j;
+                        wv[rel] = __uint_as_float(bits) - shift;
+                    }
+                }
+                flush(wbase + w0, min(kRowWin, wtot_r - w0));
+            }
+        }
+    }
+    // ---- dense output -----------------------------------------------------------------------------
+    if (p.y_dense != nullptr) {
+        const float fillv = p.fill == SPARK_FILL_NEGINF ? -INFINITY : 0.f;
+        float* yrow = p.y_dense + row * p.ld;
+        auto emit4 = [&](const float4& f, int v, int nv) {
+            float4 o;
+            o.x = f.x > theta ? f.x - shift : fillv; o.y = f.y > theta ? f.y - shift : fillv;
+            o.z = f.z > theta ? f.z - shift : fillv; o.w = f.w > theta ? f.w - shift : fillv;
+            if (nv == 4) {
+                __stcs(reinterpret_cast<float4*>(yrow) + v, o);
+            } else {
+                float* t = yrow + (v << 2);
+                t[0] = o.x;
+                if (nv > 1) t[1] = o.y;
+                if (nv > 2) t[2] = o.z;
+            }
+        };
+        for (int v = tid; v < g.ns; v += kRowThreads) emit4(ssrc[v], v, 4);
+#pragma unroll
+        for (int i = 0; i < kRowRegVec; ++i) {
+            const int v = rv0 + i * 32;
+            if (v < g.nvec) emit4(f4(cur[i]), v, v == g.nvec - 1 ? last_nv : 4);
+        }
+    }
+    // shared memory is free again: start the next row's copies
+    __syncthreads();
+    if (tid == 0 && next_row < p.rows) row_issue_bulk(p.x + next_row * p.ld, srow, sh.mbar, g);
+    return true;
+}
+
+__global__ void __launch_bounds__(kRowThreads, 1) stat_topk_row_kernel(const TopkParams p) {
+    extern __shared__ __align__(128) float srow[];
+    __shared__ RowShared sh;
+    const int tid = threadIdx.x;
+    RowGeom g;
+    g.n = static_cast<int>(p.n);
+    g.nvec = (g.n + 3) >> 2;
+    const int nr = min(g.nvec, kRowRegVec * kRowThreads);
+    g.ns = g.nvec - nr;
+    g.npiece = (g.ns + kRowPieceVec - 1) / kRowPieceVec;
+
+    int64_t row = blockIdx.x;
+    if (row >= p.rows) return;
+    if (tid == 0) {
+        for (int c = 0; c < kRowPieces; ++c)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(sh.mbar + c)) : "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        sh.abort = 0;
+        row_issue_bulk(p.x + row * p.ld, srow, sh.mbar, g);
+    }
+    uint4 ra[kRowRegVec], rb[kRowRegVec];
+    float ca = p.identity ? 0.f : __ldg(p.x + row * p.ld), cb = 0.f;
+    row_load_regs(p.x + row * p.ld, g, ra);
+    __syncthreads();                                                  // barrier objects visible to every thread
+    const int64_t step = gridDim.x;
+    bool ok = true;
+    uint32_t parity = 0;
+#pragma unroll 1
+    for (;;) {
+        ok = row_body(p, g, srow, sh, row, row + step, parity, ra, rb, ca, cb);
+        row += step;
+        if (!ok || row >= p.rows) break;
+        parity ^= 1u;
+        ok = row_body(p, g, srow, sh, row, row + step, parity, rb, ra, cb, ca);
+        row += step;
+        if (!ok || row >= p.rows) break;
+        parity ^= 1u;
+    }
+    if (!ok) {
+        // a copy did not land in time: report it, then give copies still in flight one more bounded wait
+        if (tid == 0) {
+            atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+            for (int c = 0; c < g.npiece; ++c) {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(smem_u32(sh.mbar + c), parity))
+                    if (clock64() - t0 > kRowSpinLimit) break;
+            }
+        }
+    }
+}
+
 bool g_attr_done[64] = {};   // per device: opt-in shared memory configured
 
 }  // namespace
@@ -275,6 +648,19 @@ extern "C" int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int
                                  static_cast<int>(hard * 4)) != cudaSuccess)
             return SPARK_ERR_CUDA;
         g_attr_done[ctx->device] = true;
+    }
+
+    if (n > 16384 && (n + 3) / 4 <= kRowMaxVec) {      // the whole row fits one block: no cluster needed
+        static bool row_attr_done[64] = {};
+        if (ctx->device >= 0 && ctx->device < 64 && !row_attr_done[ctx->device]) {
+            if (cudaFuncSetAttribute(stat_topk_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowSmemBytes) != cudaSuccess)
+                return SPARK_ERR_CUDA;
+            row_attr_done[ctx->device] = true;
+        }
+        const size_t smem = kRowSmemBytes;
+        const int64_t grid = rows < ctx->num_sms ? rows : ctx->num_sms;
+        stat_topk_row_kernel<<<static_cast<unsigned>(grid), kRowThreads, smem, static_cast<cudaStream_t>(stream)>>>(p);
+        return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
     }
 
     cudaLaunchConfig_t cfg = {};

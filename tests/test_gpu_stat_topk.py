@@ -155,3 +155,25 @@ def test_full_size_workload_sampled(ctx):
             sd = 44.1
             assert np.all(np.abs(ct - k) < 6 * sd) and abs(ct.mean() - k) < 0.5 * sd
         del xd, idx, val
+
+
+@pytest.mark.parametrize("n,k,rows", [(65536, 1311, 450), (40004, 9000, 320), (28670, 500, 160), (65533, 70000, 150)])
+def test_rows_held_on_chip_by_a_persistent_block(ctx, n, k, rows):
+    # 16K < n <= 64K: one block per SM walks over several rows, part of each row in shared memory and part in
+    # registers (n = 28670: registers only after the first 8190 values; n = 65533: ragged tail; k >= n: identity).
+    # Every row is compared on theta and count, a sample of rows on sets, values and the dense output.
+    X = synth.rows_f32("laplace", rows, n, seed=11) * 0.8 + 25.0      # mean far from zero
+    ld = (n + 3) // 4 * 4
+    out = run_topk(ctx, X, k, ld=ld)
+    theta, count = out[0], out[1]
+    x64 = X.astype(np.float64)
+    if k < n:
+        mean = x64.mean(axis=1)
+        std = x64.std(axis=1, ddof=1)
+        th = mean + std * O.gaussian_upper_quantile(k / n)
+        assert np.all(np.abs(theta - th) <= parity.THETA_RTOL * np.maximum(np.abs(th), std))
+        near = (np.abs(x64 - th[:, None]) <= parity.BAND * std[:, None]).sum(axis=1)
+        assert np.all(np.abs(count - (x64 > th[:, None]).sum(axis=1)) <= near)
+    else:
+        assert np.all(np.isneginf(theta)) and np.all(count == n)
+    compare_rows(X, k, S.SPARK_FILL_ZERO, out, rows=[0, 1, 147, 148, 149, rows - 1])
