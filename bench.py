@@ -50,6 +50,7 @@ def parse():
     ap.add_argument("--layers", type=int, default=0, help="0 = the shape's layer count")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-loads comparator")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
+    ap.add_argument("--overlap", type=int, default=1, help="1 = launch kernels with programmatic stream serialization")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     return ap.parse_args()
 
@@ -202,6 +203,7 @@ def run_spark(args):
     B, ctx_len, d, hd = args.batch, args.ctx, shape.d, shape.hd
     cap = ctx_len
     ctx = S.SparkContext(local, max_batch=B, max_dff=shape.d_ff, max_cap=cap, n_q=shape.n_q, hd=hd, max_d=d)
+    ctx.set_launch_overlap(bool(args.overlap))
 
     gen = torch.Generator(device=dev)
     gen.manual_seed(1234 + rank)
@@ -380,7 +382,8 @@ def run_spark(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(args, shape), "l2": "weights+caches (>3 GB) exceed L2; no flush needed",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                       "launch": "host launches" if args.no_graph else "one CUDA graph replay per decode step",
+                       "launch": ("host launches" if args.no_graph else "one CUDA graph replay per decode step") +
+                                 (", programmatic dependent launches (spark_set_launch_overlap)" if args.overlap else ""),
                        "local_window": 4096, "k_ff": shape.k_ff, "k_attn": shape.k_attn},
             "tokens_per_s": B * world * args.steps / (ms_total * 1e-3),
             "layer_touched_mb": layer_touched / 1e6,

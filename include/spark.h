@@ -107,6 +107,17 @@ int spark_grid_size(const spark_ctx* ctx);
  * 16 entries per block.  NULL switches tracing off (the default). */
 int spark_set_phase_trace(spark_ctx* ctx, uint64_t* trace, int64_t capacity);
 
+/* Launch overlap (scheduling aid; the paper has no counterpart).  With on != 0 every kernel of
+ * this context is launched with the programmatic stream-serialization attribute: it may start
+ * while the kernel before it in the stream still runs, requests its first weights, and only then
+ * waits for that kernel to complete.  The caller promises that (1) the work placed in the stream
+ * directly before a call does not write the WEIGHT buffers of that call (everything else is read
+ * after the wait), and (2) the GPU runs no other kernels meanwhile: the inter-block exchanges rely
+ * on all blocks being resident, which the cooperative launch used otherwise (on == 0, the default)
+ * guarantees and this mode only obtains from an otherwise idle GPU; a block that waits in vain
+ * gives up after its limit and the device status becomes SPARK_ERR_TIMEOUT.  Host-only setting. */
+int spark_set_launch_overlap(spark_ctx* ctx, int on);
+
 /* Gaussian upper quantile used for the threshold: z with P(N(0,1) > z) = p, i.e. Q(1 - p) of
  * Eq. 11.  Host function (no device work); exported so that it can be checked on its own.
  * Returns NaN for p outside (0, 1). */

@@ -26,7 +26,7 @@ SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
 
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
-    "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_stat_topk", "spark_ffn_decode",
+    "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_set_launch_overlap", "spark_stat_topk", "spark_ffn_decode",
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc",
 ]
 
@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
         "spark_device_status": (i32, [vp, vp, C.POINTER(i32)]),
         "spark_grid_size": (i32, [vp]),
         "spark_set_phase_trace": (i32, [vp, vp, i64]),
+        "spark_set_launch_overlap": (i32, [vp, i32]),
         "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
         "spark_ffn_decode": (i32, [vp, vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
         "spark_ffn_decode_noalloc": (i32, [vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp]),
@@ -155,6 +156,10 @@ class SparkContext:
         n = 0 if trace is None else trace.numel()
         _check(lib().spark_set_phase_trace(self.handle, _ptr(trace), n), "spark_set_phase_trace")
         self._trace = trace
+
+    def set_launch_overlap(self, on: bool):
+        """Launch every kernel of this context so that it may start under the tail of the kernel before it."""
+        _check(lib().spark_set_launch_overlap(self.handle, 1 if on else 0), "spark_set_launch_overlap")
 
     @property
     def grid_size(self) -> int:

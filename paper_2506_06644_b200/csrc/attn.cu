@@ -104,6 +104,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     };
     auto win_len = [&](int n) -> int { return (p.window > 0 && p.window < n) ? p.window : n; };
 
+    dep_wait();        // lengths, queries and the newest cache rows all come from the kernels before this one
+    dep_trigger();
     // ---- flat layout: prefix sums of the window lengths over the segments -------------------------
     if (tid == 32) s_fail = 0;
     if (warp == 0) {
@@ -471,17 +473,9 @@ int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) 
             return SPARK_ERR_CUDA;
         configured[ctx->device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ctx->num_sms));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, p) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    void* args[] = {&p};
+    return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(ctx->num_sms), kThreads, smem, stream, true, args) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 template <typename KT>

@@ -58,9 +58,47 @@ struct spark_ctx {
     size_t scratch_bytes;
     unsigned long long* trace;   // optional phase trace (device), see spark_set_phase_trace
     long long trace_cap;
+    int overlap;             // launch with programmatic stream serialization, see spark_set_launch_overlap
 };
 
 namespace spark {
+
+// ---------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel launched with the stream-serialization attribute may
+// start while the kernel before it in the stream still runs; dep_wait() returns once that kernel
+// has completed and its writes are visible.  Only immutable data (weights) may be touched before
+// it.  dep_trigger() lets the kernel after this one be scheduled as blocks of this one leave; it
+// is called right after dep_wait(), so that a dependent never starts before the grid two places
+// back has completed.  Both are no-ops in a kernel launched the ordinary way.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Host: one launch.  `cooperative` asks for the co-residency guarantee; with ctx->overlap the
+// launch carries the programmatic attribute instead (the two cannot be combined), and co-residency
+// rests on the grid being one block per SM on a GPU that runs nothing else (a block that waits in
+// vain gives up after its spin limit and reports SPARK_ERR_TIMEOUT).
+inline cudaError_t launch_kernel(const spark_ctx* ctx, const void* kern, unsigned grid, unsigned block, size_t smem,
+                                 cudaStream_t stream, bool cooperative, void** args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    cfg.attrs = attr;
+    cfg.numAttrs = 0;
+    if (ctx->overlap) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 1;
+    } else if (cooperative) {
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.numAttrs = 1;
+    }
+    return cudaLaunchKernelExC(&cfg, kern, args);
+}
 
 // ---------------------------------------------------------------------------
 // Loads

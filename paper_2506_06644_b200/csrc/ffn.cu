@@ -47,6 +47,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
     const WT* K1t = static_cast<const WT*>(p.K1t);
     const WT* K2t = static_cast<const WT*>(p.K2t);
     const WT* Vt = static_cast<const WT*>(p.Vt);
+    dep_wait();        // these kernels read the batch's inputs first: nothing to do ahead of the dependency
+    dep_trigger();
     if (tid == 0) {
         s_epoch = ld_acquire_u32(&p.hdr->epoch);      // consumed after phase A
         s_fail = 0;
@@ -368,17 +370,10 @@ int launch_one(spark_ctx* ctx, FfnParams& p, size_t smem, cudaStream_t stream) {
             return SPARK_ERR_CUDA;
         configured[ctx->device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ctx->num_sms));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, p) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    p.overlap = ctx->overlap;
+    void* args[] = {&p};
+    return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(ctx->num_sms), kThreads, smem, stream, true, args) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 template <typename WT>
@@ -503,6 +498,7 @@ extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K
     local.scratch_bytes = 0;
     local.trace = nullptr;
     local.trace_cap = 0;
+    local.overlap = 0;
     FfnArgs a;
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
     a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = wdtype;

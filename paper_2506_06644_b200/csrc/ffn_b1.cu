@@ -51,31 +51,38 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     const WT* Vt = static_cast<const WT*>(p.Vt);
     const int d4 = d / 4;
     const int n_init = (d4 + kThreads - 1) / kThreads;          // blocks that initialise y
-    if (tid == 0) {
-        s_epoch = ld_acquire_u32(&p.hdr->epoch);                // consumed after phase A
-        s_nact = 0;
-        s_fail = 0;
-    }
-    if (cta == 0) {
-        // clear the cells the launch after next will use (last used two launches ago)
-        const unsigned e = ld_acquire_u32(&p.hdr->epoch);
-        SumCell* c = &p.hdr->ffn_cells[(e + 2u) & 3u][0][0][0];
-        for (int i = tid; i < 4 * 16 * kCellWays; i += kThreads) { c[i].s1 = 0.0; c[i].s2 = 0.0; c[i].count = 0u; }
-    }
-    p.trace.mark(0);
-
-    // The token's input is requested before anything else so that it is in shared memory when the
-    // first K1t rows arrive (requests are served in issue order).
+    // Everything that another kernel may have written is read in after_dependency(): with launch overlap
+    // that is after the first K1t loads have been issued (they fly while the kernel before this one in the
+    // stream drains); otherwise before them, so that the token's input is in shared memory when the first
+    // rows arrive (requests are served in issue order).
     const bool has0 = tid < d4, has1 = tid + kThreads < d4;
     float4 xv0 = make_float4(0.f, 0.f, 0.f, 0.f), xv1 = xv0, nw0 = make_float4(1.f, 1.f, 1.f, 1.f), nw1 = nw0;
-    if (has0) xv0 = reinterpret_cast<const float4*>(p.x)[tid];
-    if (has1) xv1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
-    if (p.norm_w != nullptr) {
-        if (has0) nw0 = reinterpret_cast<const float4*>(p.norm_w)[tid];
-        if (has1) nw1 = reinterpret_cast<const float4*>(p.norm_w)[tid + kThreads];
-    }
+    auto after_dependency = [&]() {
+        dep_wait();
+        dep_trigger();
+        if (has0) xv0 = reinterpret_cast<const float4*>(p.x)[tid];
+        if (has1) xv1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
+        if (p.norm_w != nullptr) {
+            if (has0) nw0 = reinterpret_cast<const float4*>(p.norm_w)[tid];
+            if (has1) nw1 = reinterpret_cast<const float4*>(p.norm_w)[tid + kThreads];
+        }
+        if (tid == 0) {
+            s_epoch = ld_acquire_u32(&p.hdr->epoch);            // consumed after phase A
+            s_nact = 0;
+            s_fail = 0;
+        }
+        if (cta == 0) {
+            // clear the cells the launch after next will use (last used two launches ago)
+            const unsigned e = ld_acquire_u32(&p.hdr->epoch);
+            SumCell* c = &p.hdr->ffn_cells[(e + 2u) & 3u][0][0][0];
+            for (int i = tid; i < 4 * 16 * kCellWays; i += kThreads) { c[i].s1 = 0.0; c[i].s2 = 0.0; c[i].count = 0u; }
+        }
+        p.trace.mark(0);
+    };
+    if (!p.overlap) after_dependency();
     // Runs once the first K1t loads are in flight: y initialisation, optional RMSNorm, x to shared memory.
     auto prologue = [&]() {
+        if (p.overlap) after_dependency();
         if (cta < n_init) {
             const int i = cta * kThreads + tid;
             if (i < d4)
@@ -284,18 +291,9 @@ int ffn1_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream) {
             return SPARK_ERR_CUDA;
         configured[wi][ctx->device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ctx->num_sms));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    p.overlap = ctx->overlap;
     void* args[] = {&p};
-    return cudaLaunchKernelExC(&cfg, kern, args) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    return launch_kernel(ctx, kern, static_cast<unsigned>(ctx->num_sms), kThreads, smem, stream, true, args) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 }  // namespace spark

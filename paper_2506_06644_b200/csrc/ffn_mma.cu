@@ -141,6 +141,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
     const __nv_bfloat16* K1t = static_cast<const __nv_bfloat16*>(p.K1t);
     const __nv_bfloat16* K2t = static_cast<const __nv_bfloat16*>(p.K2t);
     const __nv_bfloat16* Vt = static_cast<const __nv_bfloat16*>(p.Vt);
+    dep_wait();        // these kernels read the batch's inputs first: nothing to do ahead of the dependency
+    dep_trigger();
     if (tid == 0) {
         s_epoch = ld_acquire_u32(&p.hdr->epoch);
         s_fail = 0;
@@ -524,17 +526,10 @@ int launch_mma(spark_ctx* ctx, FfnParams& p, cudaStream_t stream) {
             return SPARK_ERR_CUDA;
         configured[ctx->device] = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ctx->num_sms));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, p) == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    p.overlap = ctx->overlap;
+    void* args[] = {&p};
+    return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(ctx->num_sms), kThreads, smem, stream, true, args) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 }  // namespace

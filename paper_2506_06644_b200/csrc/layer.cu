@@ -26,6 +26,7 @@ struct GemvParams {
     int x_div_group;
     uint4* zero_ptr;
     int zero_n16;
+    int overlap;             // launched with the programmatic attribute: weights first, then dep_wait()
 };
 
 // Input staging shared by the GEMV kernels: x (optionally divided per group, optionally RMS-normalised)
@@ -41,7 +42,7 @@ __device__ __forceinline__ EarlyX early_x_request(const GemvParams& p) {
     e.v0 = make_float4(0.f, 0.f, 0.f, 0.f);
     e.v1 = e.v0;
     const int n4 = p.n_in / 4, tid = threadIdx.x;
-    e.on = p.B == 1 && n4 <= 2 * kThreads;
+    e.on = !p.overlap && p.B == 1 && n4 <= 2 * kThreads;
     if (e.on) {
         if (tid < n4) e.v0 = reinterpret_cast<const float4*>(p.x)[tid];
         if (tid + kThreads < n4) e.v1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
@@ -100,7 +101,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
     const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
     const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
     const EarlyX ex = early_x_request(p);
-    auto fill_x = [&]() { stage_input<TB>(p, xs, rstd, ex); };   // runs once the first weight loads are in flight
+    auto fill_x = [&]() {                                         // runs once the first weight loads are in flight
+        if (p.overlap) { dep_wait(); dep_trigger(); }
+        stage_input<TB>(p, xs, rstd, ex);
+    };
     rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in, fill_x,
                          [&](int j, int t, float v) {
                              if (t < p.B) {
@@ -119,8 +123,10 @@ int gemv_launch_one(spark_ctx* ctx, GemvParams& p, size_t smem, int grid, cudaSt
             return SPARK_ERR_CUDA;
         configured[ctx->device] = true;
     }
-    kern<<<grid, kThreads, smem, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    p.overlap = ctx->overlap;
+    void* args[] = {&p};
+    return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(grid), kThreads, smem, stream, false, args) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 template <typename WT, int TB>
@@ -233,14 +239,6 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
     const GemvParams& g = p.g;
     const RopeParams& rp = p.r;
     const int tid = threadIdx.x;
-    if (blockIdx.x == gridDim.x - 1 && tid >= kThreads - 32 && tid - (kThreads - 32) < rp.B) {
-        // the threshold quantile of each sequence's window, for the attention kernel that follows
-        const int b = tid - (kThreads - 32);
-        int n = rp.ctx_len[b];
-        n = n < 1 ? 1 : (n > rp.cap ? static_cast<int>(rp.cap) : n);
-        const int L = (rp.window > 0 && rp.window < n) ? rp.window : n;
-        rp.zs[b] = rp.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(rp.k_attn) / static_cast<double>(L));
-    }
     const int hd = rp.hd, hp = hd / 2, hr = rp.r / 2;
     const int P = g.n_out / 2;                        // output pairs
     const int p0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * P / gridDim.x);
@@ -253,7 +251,18 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
         return head * hd + rp.r + (q - hr) + which * ((hd - rp.r) / 2);
     };
     const EarlyX ex = early_x_request(g);
-    auto fill_x = [&]() { stage_input<TB>(g, xs, rstd, ex); };
+    auto fill_x = [&]() {
+        if (g.overlap) { dep_wait(); dep_trigger(); }
+        if (blockIdx.x == gridDim.x - 1 && tid >= kThreads - 32 && tid - (kThreads - 32) < rp.B) {
+            // the threshold quantile of each sequence's window, for the attention kernel that follows
+            const int b = tid - (kThreads - 32);
+            int n = rp.ctx_len[b];
+            n = n < 1 ? 1 : (n > rp.cap ? static_cast<int>(rp.cap) : n);
+            const int L = (rp.window > 0 && rp.window < n) ? rp.window : n;
+            rp.zs[b] = rp.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(rp.k_attn) / static_cast<double>(L));
+        }
+        stage_input<TB>(g, xs, rstd, ex);
+    };
     rows_dot_mapped<__nv_bfloat16, TB, 2>(
         static_cast<const __nv_bfloat16*>(g.Wt), g.n_in, 2 * (p1 - p0), g.n_in / 8, xs, g.n_in, rowmap, fill_x,
         [&](int rg, int t, const float (&v)[2]) {
@@ -301,8 +310,11 @@ int qkv_rope_launch_one(spark_ctx* ctx, const QkvRopeParams& p, size_t smem, int
             return SPARK_ERR_CUDA;
         configured[ctx->device] = true;
     }
-    kern<<<grid, kThreads, smem, stream>>>(p);
-    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+    QkvRopeParams q = p;
+    q.g.overlap = ctx->overlap;
+    void* args[] = {&q};
+    return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(grid), kThreads, smem, stream, false, args) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 }  // namespace

@@ -88,6 +88,7 @@ int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_
     c->scratch_bytes = workspace_bytes - sizeof(WsHeader);
     c->trace = nullptr;
     c->trace_cap = 0;
+    c->overlap = 0;
     *out = c;
     return SPARK_OK;
 }
@@ -101,6 +102,12 @@ int spark_set_phase_trace(spark_ctx* ctx, uint64_t* trace, int64_t capacity) {
     if (ctx == nullptr || (trace != nullptr && capacity < 16)) return SPARK_ERR_INVALID_ARG;
     ctx->trace = reinterpret_cast<unsigned long long*>(trace);
     ctx->trace_cap = trace != nullptr ? capacity : 0;
+    return SPARK_OK;
+}
+
+int spark_set_launch_overlap(spark_ctx* ctx, int on) {
+    if (ctx == nullptr) return SPARK_ERR_INVALID_ARG;
+    ctx->overlap = on ? 1 : 0;
     return SPARK_OK;
 }
 

@@ -1,0 +1,90 @@
+"""GPU parity with launch overlap on: every kernel carries the programmatic stream-serialization
+attribute, requests its first weights under the tail of the kernel before it and only then waits for
+that kernel.  Results must not change: against the oracle for one call, against the ordinary launch
+mode for chains of calls placed back to back in the stream (where a stale read would show)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_06644_b200 import binding as S
+from paper_2506_06644_b200 import synth
+from tests import parity
+from tests.test_gpu_ffn import compare as compare_ffn, upload
+from tests.test_gpu_layer import make_layer, oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx_pair():
+    plain = S.SparkContext(0, max_batch=16, max_cap=16384, n_q=16, hd=256)
+    over = S.SparkContext(0, max_batch=16, max_cap=16384, n_q=16, hd=256)
+    over.set_launch_overlap(True)
+    yield plain, over
+    assert plain.device_status() == S.SPARK_OK
+    assert over.device_status() == S.SPARK_OK
+    plain.close()
+    over.close()
+
+
+def chain(ctx, sh, B, cap, lens, window, calls, seed=4):
+    """`calls` decoder-layer calls back to back on one stream (the same layer: h feeds the next call)."""
+    lw, kv, h0, layer, cache = make_layer(sh, B, cap, lens, seed, window)
+    h = torch.from_numpy(h0).cuda()
+    cl = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    nqkv = (sh.n_q + 2 * sh.n_kv) * sh.hd
+    scratch = torch.empty(B * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device="cuda")
+    torch.cuda.synchronize()
+    for _ in range(calls):
+        S.spark_layer_decode(ctx, layer, cl, h, B, scratch)
+    torch.cuda.synchronize()
+    return lw, kv, h0, h.cpu().numpy()
+
+
+@pytest.mark.parametrize("shape,B,cap,lens,window", [
+    (synth.TINY, 3, 128, [128, 1, 17], 0),
+    (synth.GEMMA2_2B, 1, 2048, [2048], 0),
+    (synth.GEMMA2_2B, 2, 1024, [700, 1024], 512),
+])
+def test_one_layer_call_against_oracle(ctx_pair, shape, B, cap, lens, window):
+    _, over = ctx_pair
+    lw, kv, h0, h = chain(over, shape, B, cap, lens, window, calls=1)
+    for b in range(B):
+        ref, _, _ = oracle_layer(shape, lw, kv, h0, b, lens[b], window)
+        parity.check_output(h[b], ref["h"], "bf16", f"seq {b}")
+        parity.check_output(h[b] - h0[b], ref["h"] - h0[b], "bf16", f"seq {b} (update only)")
+
+
+@pytest.mark.parametrize("shape,B,cap,lens", [(synth.TINY, 2, 128, [100, 90]), (synth.GEMMA2_2B, 1, 4096, [4096]),
+                                               (synth.GEMMA2_2B, 4, 512, [512, 300, 77, 1])])
+def test_chain_of_calls_matches_ordinary_launches(ctx_pair, shape, B, cap, lens):
+    plain, over = ctx_pair
+    a = chain(plain, shape, B, cap, lens, 0, calls=6)[3]
+    for _ in range(3):                                    # timing between kernels differs from run to run
+        b = chain(over, shape, B, cap, lens, 0, calls=6)[3]
+        assert np.all(np.isfinite(b))
+        # six chained layers amplify the last-bit differences of the atomic reductions' order
+        np.testing.assert_allclose(b, a, rtol=0, atol=2e-4 * parity.rms(a))
+
+
+@pytest.mark.parametrize("B", [1, 4])
+def test_ffn_calls_back_to_back(ctx_pair, B):
+    # FFN launches in a row use different accumulator ring slots: a launch must not pick its slot
+    # before the one before it has advanced the launch count
+    _, over = ctx_pair
+    p = synth.ffn_inputs(2304, 9216, 1024, 737, B, "bf16", seed=21)
+    K1t, K2t, Vt = upload(p)
+    x = torch.from_numpy(p.x).cuda()
+    outs = []
+    for _ in range(5):
+        y = torch.full((B, p.d), float("nan"), device="cuda")
+        theta = torch.full((B,), 77.0, device="cuda")
+        count = torch.full((B,), -5, dtype=torch.int32, device="cuda")
+        idx = torch.full((B, p.d_ff), -1, dtype=torch.int32, device="cuda")
+        outs.append((y, theta, count, idx))
+    torch.cuda.synchronize()
+    for y, theta, count, idx in outs:                     # no synchronisation between the launches
+        S.spark_ffn_decode(over, x, B, K1t, K2t, Vt, S.SPARK_BF16, p.d, p.d_ff, p.r, p.k, 0, y, theta, count, idx)
+    torch.cuda.synchronize()
+    for out in outs:
+        compare_ffn(p, tuple(t.cpu().numpy() for t in out))
