@@ -54,6 +54,8 @@ struct AttnParams {
     SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
     float* lsum;       // [B][n_q] sum of softmax weights per head (o accumulates the weighted values)
     int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
+    int pre_stable;    // 1: the kernel directly before this one writes neither ctx_len nor cache rows other than each
+                       //    sequence's newest, so lengths and older rows may be read before dep_wait()
     WsHeader* hdr;
     PhaseTrace trace;
 };
@@ -104,8 +106,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     };
     auto win_len = [&](int n) -> int { return (p.window > 0 && p.window < n) ? p.window : n; };
 
-    dep_wait();        // lengths, queries and the newest cache rows all come from the kernels before this one
-    dep_trigger();
+    if (!p.pre_stable) {   // lengths, queries and cache rows may all come from the kernel before this one
+        dep_wait();
+        dep_trigger();
+    }
     // ---- flat layout: prefix sums of the window lengths over the segments -------------------------
     if (tid == 32) s_fail = 0;
     if (warp == 0) {
@@ -124,7 +128,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
         if (lane == 0) segoff[0] = 0;
     }
     __syncthreads();
-    p.trace.mark(0);
     SumCell* cells = p.cells;
     const int64_t T = segoff[NS];
     const int Gp = T < G ? static_cast<int>(T) : G;        // blocks that own a non-empty range
@@ -149,6 +152,45 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
         if (w0 > te) w0 = te;
         if (w1 > te) w1 = te;
     };
+
+    // The first batch of predictor rows is requested before anything else is waited for: before the
+    // query is staged and, when the lengths are known to be stable, before the kernel ahead of this one
+    // has finished (its newest cache row is held back until it has).
+    Row8<KT> wpre[8];
+    bool have_pre = false;
+    {
+        int held = -1;
+        const KT* held_row = nullptr;
+        if (has) {
+            const int sb = segoff[seg0], se = segoff[seg0 + 1], L = se - sb;
+            const int tb = static_cast<int>(f0 - sb);
+            const int te = static_cast<int>((f1 < se ? f1 : se) - sb);
+            const int lo = seq_len(seg0 / p.n_kv) - L;
+            const KT* kbase = k1c + (static_cast<int64_t>(seg0) * p.cap + lo) * r;
+            int w0, w1;
+            warp_range(tb, te, w0, w1);
+            if (w0 < w1) {
+                const int tok0 = w0 + half * 8;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int t = tok0 + j;
+                    const bool newest = p.pre_stable && t == L - 1;
+                    if (t < w1 && hl < nc1 && !newest) wpre[j].load(kbase + static_cast<int64_t>(t) * r, hl);
+                    else wpre[j].zero();
+                    if (newest && t < w1 && hl < nc1) { held = j; held_row = kbase + static_cast<int64_t>(t) * r; }
+                }
+                have_pre = true;
+            }
+        }
+        if (p.pre_stable) {
+            dep_wait();
+            dep_trigger();
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j == held) wpre[j].load(held_row, hl);
+        }
+    }
+    p.trace.mark(0);
 
     // =============================== pass 1: predictor scores =====================================
     {
@@ -188,10 +230,15 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             for (int base = w0; base < w1; base += 16) {
                 const int tok0 = base + half * 8;
                 Row8<KT> w[8];
+                if (have_pre && ord == 0 && base == w0) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (tok0 + j < w1 && hl < nc1) w[j].load(kbase + static_cast<int64_t>(tok0 + j) * r, hl);
-                    else w[j].zero();
+                    for (int j = 0; j < 8; ++j) w[j] = wpre[j];
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (tok0 + j < w1 && hl < nc1) w[j].load(kbase + static_cast<int64_t>(tok0 + j) * r, hl);
+                        else w[j].zero();
+                    }
                 }
                 float pj[8][GQ];
 #pragma unroll
@@ -540,6 +587,7 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.cells = reinterpret_cast<SumCell*>(ctx->scratch);
     p.lsum = lsum != nullptr ? lsum : reinterpret_cast<float*>(ctx->scratch + cells_b);
     p.defer = lsum != nullptr ? 1 : 0;
+    p.pre_stable = p.defer;
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;

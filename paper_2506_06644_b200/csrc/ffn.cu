@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_kernel(const FfnParams p) {
         };
 
         // ---- phase A: predictor scores of this block's neurons ----------------------------------
-        rows_dot<WT, TB, kRows>(K1t, r, row0, nloc, r / 8, xs, xw, prologue, [&](int j, int t, float v) {
+        rows_dot<WT, TB, kRows>(K1t, r, row0, nloc, r / 8, xs, xw, [] {}, prologue, [&](int j, int t, float v) {
             s_loc[static_cast<size_t>(t) * rpc + j] = v;
         });
         __syncthreads();

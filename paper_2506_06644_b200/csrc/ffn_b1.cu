@@ -52,9 +52,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     const int d4 = d / 4;
     const int n_init = (d4 + kThreads - 1) / kThreads;          // blocks that initialise y
     // Everything that another kernel may have written is read in after_dependency(): with launch overlap
-    // that is after the first K1t loads have been issued (they fly while the kernel before this one in the
-    // stream drains); otherwise before them, so that the token's input is in shared memory when the first
-    // rows arrive (requests are served in issue order).
+    // that is after the first batch of K1t loads has been issued (they fly while the kernel before
+    // this one in the stream drains); otherwise before them, so that the token's input is in shared memory
+    // when the first rows arrive (requests are served in issue order).
     const bool has0 = tid < d4, has1 = tid + kThreads < d4;
     float4 xv0 = make_float4(0.f, 0.f, 0.f, 0.f), xv1 = xv0, nw0 = make_float4(1.f, 1.f, 1.f, 1.f), nw1 = nw0;
     auto after_dependency = [&]() {
@@ -82,7 +82,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     if (!p.overlap) after_dependency();
     // Runs once the first K1t loads are in flight: y initialisation, optional RMSNorm, x to shared memory.
     auto prologue = [&]() {
-        if (p.overlap) after_dependency();
         if (cta < n_init) {
             const int i = cta * kThreads + tid;
             if (i < d4)
@@ -111,7 +110,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     };
 
     // ---- A: predictor scores s = K1^T x[:r] of this block's neurons ---------------------------------
-    rows_dot<WT, 1, kRows>(K1t, r, row0, nloc, r / 8, xs, 0, prologue,
+    rows_dot<WT, 1, kRows>(K1t, r, row0, nloc, r / 8, xs, 0, [&]() { if (p.overlap) after_dependency(); }, prologue,
                            [&](int j, int, float v) { s_loc[j] = v; });
     __syncthreads();
     p.trace.mark(2);

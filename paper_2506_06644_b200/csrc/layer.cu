@@ -37,13 +37,13 @@ struct EarlyX {
     float4 v0, v1;
     bool on;
 };
-__device__ __forceinline__ EarlyX early_x_request(const GemvParams& p) {
+__device__ __forceinline__ EarlyX early_x_request(const GemvParams& p, bool after_dependency) {
     EarlyX e;
     e.v0 = make_float4(0.f, 0.f, 0.f, 0.f);
     e.v1 = e.v0;
     const int n4 = p.n_in / 4, tid = threadIdx.x;
-    e.on = !p.overlap && p.B == 1 && n4 <= 2 * kThreads;
-    if (e.on) {
+    e.on = p.B == 1 && n4 <= 2 * kThreads;
+    if (e.on && (!p.overlap || after_dependency)) {
         if (tid < n4) e.v0 = reinterpret_cast<const float4*>(p.x)[tid];
         if (tid + kThreads < n4) e.v1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
     }
@@ -100,12 +100,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
     const int n_in = p.n_in;
     const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
     const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
-    const EarlyX ex = early_x_request(p);
-    auto fill_x = [&]() {                                         // runs once the first weight loads are in flight
-        if (p.overlap) { dep_wait(); dep_trigger(); }
-        stage_input<TB>(p, xs, rstd, ex);
+    EarlyX ex = early_x_request(p, false);
+    auto dependency = [&]() {                                     // runs once the first slice of weight loads is in flight
+        if (p.overlap) {
+            dep_wait();
+            dep_trigger();
+            ex = early_x_request(p, true);
+        }
     };
-    rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in, fill_x,
+    auto fill_x = [&]() { stage_input<TB>(p, xs, rstd, ex); };   // runs once the first batch is in flight
+    rows_dot<WT, TB, RW>(static_cast<const WT*>(p.Wt), n_in, row0, row1 - row0, n_in / 8, xs, n_in, dependency, fill_x,
                          [&](int j, int t, float v) {
                              if (t < p.B) {
                                  const int64_t o = static_cast<int64_t>(t) * p.n_out + row0 + j;
@@ -250,9 +254,15 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
         if (q < hr) return head * hd + q + which * hr;
         return head * hd + rp.r + (q - hr) + which * ((hd - rp.r) / 2);
     };
-    const EarlyX ex = early_x_request(g);
+    EarlyX ex = early_x_request(g, false);
+    auto dependency = [&]() {
+        if (g.overlap) {
+            dep_wait();
+            dep_trigger();
+            ex = early_x_request(g, true);
+        }
+    };
     auto fill_x = [&]() {
-        if (g.overlap) { dep_wait(); dep_trigger(); }
         if (blockIdx.x == gridDim.x - 1 && tid >= kThreads - 32 && tid - (kThreads - 32) < rp.B) {
             // the threshold quantile of each sequence's window, for the attention kernel that follows
             const int b = tid - (kThreads - 32);
@@ -264,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
         stage_input<TB>(g, xs, rstd, ex);
     };
     rows_dot_mapped<__nv_bfloat16, TB, 2>(
-        static_cast<const __nv_bfloat16*>(g.Wt), g.n_in, 2 * (p1 - p0), g.n_in / 8, xs, g.n_in, rowmap, fill_x,
+        static_cast<const __nv_bfloat16*>(g.Wt), g.n_in, 2 * (p1 - p0), g.n_in / 8, xs, g.n_in, rowmap, dependency, fill_x,
         [&](int rg, int t, const float (&v)[2]) {
             if (t >= rp.B) return;
             const int pp = p0 + rg;

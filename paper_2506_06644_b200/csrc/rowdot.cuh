@@ -14,12 +14,16 @@ namespace spark {
 // before_use() is called exactly once by every thread of the block, after the first batch of
 // weight loads has been issued and before anything is read from xs: the caller fills xs there
 // (and synchronises the block), so that the input's latency hides behind the weights'.
+// after_first() is called exactly once by every thread as well, just before: a kernel that may
+// start under the tail of the kernel before it waits for that kernel there and requests its input.
+// (Waiting earlier, after the first quarter of the batch, so that the input queues behind fewer
+// weight requests, measured slower: the rest of the batch then cannot fly during the wait.)
 // Must be called by all threads of a 512-thread block.  rows_dot_mapped takes the row of the weight
 // matrix for each of the block's nloc logical rows from rowmap(j) and hands the RW values of a
 // warp's row group to emit_group(group, token, values) together.
-template <typename WT, int TB, int RW, typename RowMap, typename Hook, typename EmitGroup>
+template <typename WT, int TB, int RW, typename RowMap, typename Pre, typename Hook, typename EmitGroup>
 __device__ __forceinline__ void rows_dot_mapped(const WT* __restrict__ W, int64_t ld, int nloc, int nck, const float* xs,
-                                                int xw, RowMap rowmap, Hook before_use, EmitGroup emit_group) {
+                                                int xw, RowMap rowmap, Pre after_first, Hook before_use, EmitGroup emit_group) {
     constexpr int kWarpsPerBlock = 16;
     constexpr int TS = TB >= 16 ? 2 : 1;     // lane groups that split the tokens
     constexpr int TPL = TB / TS;             // tokens per lane group
@@ -55,9 +59,10 @@ __device__ __forceinline__ void rows_dot_mapped(const WT* __restrict__ W, int64_
                 const int c = c0 + u * GL + gl;
 #pragma unroll
                 for (int i = 0; i < RW; ++i) {
-                    if (has && u < cu && c < nck) w[u][i].load(rowp[i], c);
+                    if (has && u < cu && c < nck) w[u][i].load_pinned(rowp[i], c);
                     else w[u][i].zero();
                 }
+                if (u == CU - 1 && !hooked) after_first();
             }
             if (!hooked) {
                 before_use();
@@ -99,11 +104,11 @@ __device__ __forceinline__ void rows_dot_mapped(const WT* __restrict__ W, int64_
 
 // The common case: the block owns the contiguous rows [row0, row0 + nloc); emit(j, t, value) is
 // called by exactly one lane per (row, token).
-template <typename WT, int TB, int RW, typename Hook, typename Emit>
+template <typename WT, int TB, int RW, typename Pre, typename Hook, typename Emit>
 __device__ __forceinline__ void rows_dot(const WT* __restrict__ W, int64_t ld, int row0, int nloc, int nck,
-                                         const float* xs, int xw, Hook before_use, Emit emit) {
+                                         const float* xs, int xw, Pre after_first, Hook before_use, Emit emit) {
     rows_dot_mapped<WT, TB, RW>(
-        W, ld, nloc, nck, xs, xw, [&](int j) { return row0 + j; }, before_use,
+        W, ld, nloc, nck, xs, xw, [&](int j) { return row0 + j; }, after_first, before_use,
         [&](int rg, int t, const float (&v)[RW]) {
 #pragma unroll
             for (int i = 0; i < RW; ++i)
