@@ -51,6 +51,7 @@ struct AttnParams {
     float* scores;     // fallback when a block's scores do not fit in shared memory: [grid][GQ][ntok]
     int ntok;          // capacity (tokens) of a block's score buffer
     int sc_smem;       // 1: scores live in shared memory
+    int sel_list;      // 1: pass 2 first compacts a piece's survivors into a shared-memory list per head
     SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
     float* lsum;       // [B][n_q] sum of softmax weights per head (o accumulates the weighted values)
     int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
@@ -81,6 +82,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     float* qs = reinterpret_cast<float*>(segoff + ((NS + 1 + 3) & ~3));   // [GQ][hd]
     float* wpart = qs + GQ * hd;                                          // [kWarps][hd + kPartPad]
     float* sc_s = wpart + kWarps * (hd + kPartPad);                       // [GQ][ntok] when sc_smem
+    int* sel_tok = reinterpret_cast<int*>(sc_s + GQ * p.ntok);            // [GQ][ntok] when sel_list: surviving tokens
+    float* sel_a = reinterpret_cast<float*>(sel_tok + GQ * p.ntok);       // [GQ][ntok]              their s - s_max
+    __shared__ int sel_n[GQ];
     __shared__ double red[kWarps][GQ][2];
     __shared__ float redm[kWarps][GQ];
     __shared__ float theta_s[GQ], smax_s[GQ];
@@ -325,6 +329,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int c_lo = cta_of(sb), c_hi = cta_of(static_cast<int64_t>(se) - 1);
             const size_t pid = static_cast<size_t>(cta + seg);
             for (int i = tid; i < GQ * hd; i += kThreads) qs[i] = p.q[(static_cast<int64_t>(b) * p.n_q + g * GQ) * hd + i];
+            if (tid < GQ) sel_n[tid] = 0;
             if (ord >= kZc && tid == 0)
                 s_z = ident ? 0.0 : (p.zs != nullptr ? p.zs[b] : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
             __syncthreads();
@@ -375,6 +380,47 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = 0.f;
             const float* srow = sc + static_cast<size_t>(hq) * ntok + off;
+            // the k2c and vc rows of up to four surviving tokens (tk: token inside the window), requested together
+            auto gather4 = [&](const int (&tk)[4], const bool (&v)[4], const float (&av)[4]) {
+                Row8<KT> kw[2], vw[4];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {      // half h reads the k2c rows of entries h and h + 2
+                    const bool vv = half ? v[1 + 2 * i] : v[2 * i];
+                    const int tt = half ? tk[1 + 2 * i] : tk[2 * i];
+                    if (vv && hl < nc2) kw[i].load(k2base + static_cast<int64_t>(lo + tt) * d2, hl);
+                    else kw[i].zero();
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (v[i] && lane < ncv) vw[i].load(vbase + static_cast<int64_t>(lo + tk[i]) * hd, lane);
+                    else vw[i].zero();
+                }
+                float gt[4];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    float wf[8];
+                    kw[i].unpack(wf);
+                    const float gate = softplus(half_sum(dot8r(wf, q2)));
+                    gt[2 * i] = __shfl_sync(kFull, gate, 0);
+                    gt[2 * i + 1] = __shfl_sync(kFull, gate, 16);
+                }
+                float wt[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float pe = av[i] == -INFINITY ? 0.f : expf(av[i]);
+                    l_w += pe;
+                    wt[i] = pe * gt[i];         // unselected rows of the dense comparator get weight 0 * gate
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    float fv[8];
+                    vw[i].unpack(fv);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) acc[e] = fmaf(wt[i], fv[e], acc[e]);
+                }
+            };
+            int* ltok = sel_tok + static_cast<size_t>(hq) * ntok;
+            float* la = sel_a + static_cast<size_t>(hq) * ntok;
 #pragma unroll 1
             for (int base = w0; base < w1; base += 32) {
                 const int t = base + lane;
@@ -394,57 +440,53 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                         else atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_OVERFLOW);
                     }
                 }
-                while (bal != 0u) {          // four listed tokens per trip: their rows are requested together
-                    int l[4];
-                    bool v[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        v[i] = bal != 0u;
-                        l[i] = v[i] ? __ffs(bal) - 1 : 0;
-                        if (v[i]) bal &= bal - 1u;
+                if (p.sel_list) {
+                    // The survivors of the whole piece go to one list per head, from which the head's warps
+                    // then take four entries each: a warp that found many does not make the block wait for a
+                    // second round of loads while others found none.
+                    if (bal != 0u) {
+                        int pos0 = 0;
+                        if (lane == 0) pos0 = atomicAdd(&sel_n[hq], __popc(bal));
+                        pos0 = __shfl_sync(kFull, pos0, 0);
+                        if ((bal >> lane) & 1u) {
+                            const int pos = pos0 + __popc(bal & ((1u << lane) - 1u));
+                            ltok[pos] = t;
+                            la[pos] = a;
+                        }
                     }
+                    continue;
+                }
+                while (bal != 0u) {          // four listed tokens per trip: their rows are requested together
+                    int tk[4];
+                    bool v[4];
                     float av[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const float x = __shfl_sync(kFull, a, l[i]);
+                        v[i] = bal != 0u;
+                        const int l = v[i] ? __ffs(bal) - 1 : 0;
+                        if (v[i]) bal &= bal - 1u;
+                        const float x = __shfl_sync(kFull, a, l);
                         av[i] = v[i] ? x : -INFINITY;
+                        tk[i] = base + l;
                     }
-                    Row8<KT> kw[2], vw[4];
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {      // half h reads the k2c rows of tokens h and h + 2
-                        const bool vv = half ? v[1 + 2 * i] : v[2 * i];
-                        const int ll = half ? l[1 + 2 * i] : l[2 * i];
-                        if (vv && hl < nc2) kw[i].load(k2base + static_cast<int64_t>(lo + base + ll) * d2, hl);
-                        else kw[i].zero();
-                    }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        if (v[i] && lane < ncv) vw[i].load(vbase + static_cast<int64_t>(lo + base + l[i]) * hd, lane);
-                        else vw[i].zero();
-                    }
-                    float gt[4];
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        float wf[8];
-                        kw[i].unpack(wf);
-                        const float gate = softplus(half_sum(dot8r(wf, q2)));
-                        gt[2 * i] = __shfl_sync(kFull, gate, 0);
-                        gt[2 * i + 1] = __shfl_sync(kFull, gate, 16);
-                    }
-                    float wt[4];
+                    gather4(tk, v, av);
+                }
+            }
+            if (p.sel_list) {
+                __syncthreads();
+                const int n = sel_n[hq];
+#pragma unroll 1
+                for (int e0 = wsub * 4; e0 < n; e0 += NSUB * 4) {
+                    int tk[4];
+                    bool v[4];
+                    float av[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const float pe = av[i] == -INFINITY ? 0.f : expf(av[i]);
-                        l_w += pe;
-                        wt[i] = pe * gt[i];         // unselected rows of the dense comparator get weight 0 * gate
+                        v[i] = e0 + i < n;
+                        tk[i] = v[i] ? ltok[e0 + i] : 0;
+                        av[i] = v[i] ? la[e0 + i] : -INFINITY;
                     }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        float fv[8];
-                        vw[i].unpack(fv);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[e] = fmaf(wt[i], fv[e], acc[e]);
-                    }
+                    gather4(tk, v, av);
                 }
             }
             // ---- add the block's sum of weights and weighted values to the heads' accumulators ----------
@@ -591,9 +633,11 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;
+    const bool sel_list = sc_smem && smem_fixed + 3 * sc_bytes <= smem_limit;
+    p.sel_list = sel_list ? 1 : 0;
     p.hdr = ctx->hdr;
     p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
-    const size_t smem = smem_fixed + (sc_smem ? sc_bytes : 0);
+    const size_t smem = smem_fixed + (sel_list ? 3 * sc_bytes : (sc_smem ? sc_bytes : 0));
     if (kvdtype == SPARK_BF16) return launch_gq<__nv_bfloat16>(ctx, p, static_cast<int>(gq), smem, st);
     return launch_gq<float>(ctx, p, static_cast<int>(gq), smem, st);
 }
