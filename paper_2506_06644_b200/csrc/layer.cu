@@ -34,18 +34,32 @@ struct GemvParams {
 // One token: the input is requested into registers BEFORE the weight loads are issued (requests are
 // served in issue order, so this is what puts x in shared memory by the time the first rows land).
 struct EarlyX {
-    float4 v0, v1;
+    float4 v0, v1;           // the thread's two float4 of x
+    float4 w0, w1;           // the norm weights at the same places
+    float d0, d1;            // the divisors of their groups
     bool on;
 };
 __device__ __forceinline__ EarlyX early_x_request(const GemvParams& p, bool after_dependency) {
     EarlyX e;
     e.v0 = make_float4(0.f, 0.f, 0.f, 0.f);
     e.v1 = e.v0;
+    e.w0 = make_float4(1.f, 1.f, 1.f, 1.f);
+    e.w1 = e.w0;
+    e.d0 = e.d1 = 1.f;
     const int n4 = p.n_in / 4, tid = threadIdx.x;
     e.on = p.B == 1 && n4 <= 2 * kThreads;
     if (e.on && (!p.overlap || after_dependency)) {
-        if (tid < n4) e.v0 = reinterpret_cast<const float4*>(p.x)[tid];
-        if (tid + kThreads < n4) e.v1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
+        const bool h0 = tid < n4, h1 = tid + kThreads < n4;
+        if (h0) e.v0 = reinterpret_cast<const float4*>(p.x)[tid];
+        if (h1) e.v1 = reinterpret_cast<const float4*>(p.x)[tid + kThreads];
+        if (p.x_div != nullptr) {
+            if (h0) e.d0 = p.x_div[(tid * 4) / p.x_div_group];
+            if (h1) e.d1 = p.x_div[((tid + kThreads) * 4) / p.x_div_group];
+        }
+        if (p.norm_w != nullptr) {
+            if (h0) e.w0 = reinterpret_cast<const float4*>(p.norm_w)[tid];
+            if (h1) e.w1 = reinterpret_cast<const float4*>(p.norm_w)[tid + kThreads];
+        }
     }
     return e;
 }
@@ -55,12 +69,39 @@ __device__ __forceinline__ void stage_input(const GemvParams& p, float* xs, floa
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_in = p.n_in;
     const int w4 = n_in / 4;
+    if (ex.on) {
+        // one token, everything already in registers: divide, normalise, store -- one block-wide sum
+        for (int i = blockIdx.x * kThreads + tid; i < p.zero_n16; i += gridDim.x * kThreads)
+            p.zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
+        float4 v0 = ex.v0, v1 = ex.v1;
+        if (p.x_div != nullptr) {
+            const float i0 = ex.d0 > 0.f ? 1.f / ex.d0 : 0.f, i1 = ex.d1 > 0.f ? 1.f / ex.d1 : 0.f;
+            v0.x *= i0; v0.y *= i0; v0.z *= i0; v0.w *= i0;
+            v1.x *= i1; v1.y *= i1; v1.z *= i1; v1.w *= i1;
+        }
+        if (p.norm_w != nullptr) {
+            float ss = v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w + v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;
+            ss = warp_sum(ss);
+            if (lane == 0) rstd[warp] = ss;
+            __syncthreads();
+            float tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) tot += rstd[w];
+            const float sc = rsqrtf(tot / static_cast<float>(n_in) + p.eps);
+            v0.x *= sc * ex.w0.x; v0.y *= sc * ex.w0.y; v0.z *= sc * ex.w0.z; v0.w *= sc * ex.w0.w;
+            v1.x *= sc * ex.w1.x; v1.y *= sc * ex.w1.y; v1.z *= sc * ex.w1.z; v1.w *= sc * ex.w1.w;
+        }
+        if (tid < w4) reinterpret_cast<float4*>(xs)[tid] = v0;
+        if (tid + kThreads < w4) reinterpret_cast<float4*>(xs)[tid + kThreads] = v1;
+        for (int i = w4 + tid; i < TB * w4; i += kThreads) reinterpret_cast<float4*>(xs)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncthreads();
+        return;
+    }
     for (int i = tid; i < TB * w4; i += kThreads) {
         const int t = i / w4, c = i - t * w4;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (t < p.B) {
-            if (ex.on) v = i < kThreads ? ex.v0 : ex.v1;
-            else v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
+            v = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in)[c];
             if (p.x_div != nullptr) {
                 const float dv = p.x_div[static_cast<int64_t>(t) * (n_in / p.x_div_group) + (c * 4) / p.x_div_group];
                 const float inv = dv > 0.f ? 1.f / dv : 0.f;
