@@ -33,7 +33,7 @@ import numpy as np
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from the ncu
 # capture summarised in profiles/ (keyed by shape and batch); None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {("2b", 1): 24.23e6}       # profiles/ffn_b1.md
+NCU_TRAFFIC_BYTES = {("2b", 1): 24.34e6, ("2b", 16): 68.07e6}       # profiles/ffn_b1.md, profiles/ffn_mma_b16.md
 
 FALLBACK_HBM_GBS = 6650.0
 
@@ -396,7 +396,7 @@ def run_spark(args):
                     "h2d_bytes_per_step": int(h_host_in.numel() * 4), "d2h_bytes_per_step": int(h_host_out.numel() * 4)},
             "gpu_launches": args.steps * n_layers * kernels_per_layer,
             "clocks": clocks,
-            "roofline": {"kernel": "ffn_kernel (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": ("ffn1_kernel" if B == 1 else "ffn_mma_kernel") + " (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
                          "us_per_launch": ffn_us, "touched_bytes_per_launch": touched, "union_rows": union},
             "roofline_attention": {"kernel": "attn_kernel (spark_attn_decode)", "bound": "hbm",
