@@ -51,6 +51,7 @@ def parse():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense-loads comparator")
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--overlap", type=int, default=1, help="1 = launch kernels with programmatic stream serialization")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other configurations (batched FFN, long-context attention, top-k)")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     return ap.parse_args()
 
@@ -404,6 +405,10 @@ def run_spark(args):
                                    "frac": attn_bytes / (attn_us * 1e-6) / 1e9 / peak, "us_per_launch": attn_us,
                                    "touched_bytes_per_launch": attn_bytes, "traffic": None},
         }
+        if not args.no_extra and world == 1 and args.shape == "2b" and B == 1:
+            del layers, graphs, ffn_graph, attn_graph
+            torch.cuda.empty_cache()
+            line["other_workloads"] = other_workloads(torch, S, peak, max(args.steps // 4, 4), W)
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = cpu_baseline(args, shape)
     if world > 1:
@@ -411,6 +416,117 @@ def run_spark(args):
         dist.destroy_process_group()
     if line is not None:
         print(json.dumps(line), flush=True)
+
+
+def other_workloads(torch, S, peak, steps, warmup):
+    """The other configurations of the method, each timed alone with CUDA events around a CUDA graph of
+    back-to-back launches that cycle over more data than L2 holds.  GB/s are touched bytes."""
+    from paper_2506_06644_b200 import synth
+    dev = torch.device("cuda", torch.cuda.current_device())
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(99)
+    sh = synth.GEMMA2_2B
+    out = []
+
+    def time_graph(calls, n_launch):
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            calls()
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                calls()
+        torch.cuda.synchronize()
+        for _ in range(warmup):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (steps * n_launch)
+
+    def entry(name, us, nbytes, dense_us=None):
+        e = {"workload": name, "us_per_launch": us, "touched_mb": nbytes / 1e6, "gbs_touched": nbytes / us / 1e3,
+             "frac_of_measured_peak": nbytes / us / 1e3 / peak}
+        if dense_us is not None:
+            e["dense_loads_us_per_launch"] = dense_us
+            e["speedup_vs_dense_loads"] = dense_us / us
+        out.append(e)
+
+    # -- Spark FFN, 4 and 16 tokens, Gemma-2-2B shape, 8 weight sets (580 MB)
+    def w(rows, cols):
+        return (torch.randn(rows, cols, device=dev, generator=gen) * sh.d ** -0.5).to(torch.bfloat16)
+    sets = [(w(sh.d_ff, sh.r_ff), w(sh.d_ff, sh.d - sh.r_ff), w(sh.d_ff, sh.d)) for _ in range(8)]
+    for B in (4, 16):
+        ctx = S.SparkContext(dev.index, max_batch=B, max_dff=sh.d_ff, max_d=sh.d)
+        ctx.set_launch_overlap(True)
+        x = torch.randn(B, sh.d, device=dev, generator=gen)
+        y = torch.empty(B, sh.d, device=dev)
+        cnt = torch.zeros(B, dtype=torch.int32, device=dev)
+        idx = torch.zeros(B, sh.d_ff, dtype=torch.int32, device=dev)
+        S.spark_ffn_decode(ctx, x, B, *sets[0], S.SPARK_BF16, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, 0, y, None, cnt, idx)
+        torch.cuda.synchronize()
+        union = int(torch.unique(torch.cat([idx[b, : int(cnt[b])] for b in range(B)])).numel())
+        res = []
+        for flags in (0, S.SPARK_DENSE_LOADS):
+            def calls():
+                for k1, k2, v in sets:
+                    S.spark_ffn_decode(ctx, x, B, k1, k2, v, S.SPARK_BF16, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, flags, y, None, None, None)
+            res.append(time_graph(calls, len(sets)))
+        assert ctx.device_status() == S.SPARK_OK
+        entry(f"spark_ffn_decode gemma2-2b shape, {B} tokens (union of active sets {union} of {sh.d_ff})", res[0],
+              sh.d_ff * sh.r_ff * 2 + union * (2 * sh.d - sh.r_ff) * 2, res[1])
+        ctx.close()
+    del sets
+
+    # -- Spark attention, long contexts
+    for B, L, nsets in ((1, 16384, 6), (8, 32768, 2)):
+        ctx = S.SparkContext(dev.index, max_batch=B, max_cap=L, n_q=sh.n_q, hd=sh.hd)
+        ctx.set_launch_overlap(True)
+        caches = [tuple(torch.randn(B, sh.n_kv, L, wd, device=dev, generator=gen).to(torch.bfloat16)
+                        for wd in (sh.r_attn, sh.hd - sh.r_attn, sh.hd)) for _ in range(nsets)]
+        q = torch.randn(B, sh.n_q, sh.hd, device=dev, generator=gen) * sh.hd ** -0.5
+        o = torch.empty(B, sh.n_q, sh.hd, device=dev)
+        cl = torch.full((B,), L, dtype=torch.int32, device=dev)
+        res = []
+        for flags in (0, S.SPARK_DENSE_LOADS):
+            def calls():
+                for rep in range(2):
+                    for k1c, k2c, vc in caches:
+                        S.spark_attn_decode(ctx, q, k1c, k2c, vc, S.SPARK_BF16, B, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, L, cl, 0,
+                                            sh.k_attn, flags, o, None, None, None, 0)
+            res.append(time_graph(calls, 2 * nsets))
+        assert ctx.device_status() == S.SPARK_OK
+        nbytes = B * (sh.n_kv * L * sh.r_attn * 2 + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn) * 2)
+        entry(f"spark_attn_decode 8q/4kv heads hd 256, context {L}, batch {B}, k_attn {sh.k_attn}", res[0], nbytes, res[1])
+        ctx.close()
+        del caches
+
+    # -- statistical top-k, 4096 rows x 65536 (1.07 GB read per launch)
+    ctx = S.SparkContext(dev.index)
+    rows, n = 4096, 65536
+    xs = torch.randn(rows, n, device=dev, generator=gen)
+    theta = torch.empty(rows, device=dev)
+    count = torch.empty(rows, dtype=torch.int32, device=dev)
+    yd = torch.empty(rows, n, device=dev)
+    for kk in (1311, 5243):
+        us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, kk, S.SPARK_FILL_ZERO, theta, count, None, None, 0, None), 1)
+        entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = {kk / n:.0%}, theta + count", us, rows * n * 4)
+    us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, 5243, S.SPARK_FILL_ZERO, theta, count, None, None, 0, yd), 1)
+    entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = 8%, dense output (Eq. 10)", us, 2 * rows * n * 4)
+    cap = 4 * 1311
+    idx = torch.empty(rows, cap, dtype=torch.int32, device=dev)
+    val = torch.empty(rows, cap, device=dev)
+    us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, 1311, S.SPARK_FILL_ZERO, theta, count, idx, val, cap, None), 1)
+    entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = 2%, ordered index and value lists", us,
+          rows * n * 4 + int(count.sum().item()) * 8)
+    assert ctx.device_status() == S.SPARK_OK
+    ctx.close()
+    return out
+
 
 
 def touched_layer_bytes(shape, B, ctx_len, union_ffn, n_layers):

@@ -411,6 +411,40 @@ __device__ __forceinline__ bool cells_wait_w(const SumCell* ways, unsigned nbloc
         }
     }
 }
+// Group protocol for several cell sets that fill together (the tokens of a batch): every block adds its
+// sums to each set without an arrival (cells_add_sums_w, any thread), then -- after a block-wide sync --
+// ONE thread releases one arrival on the first set (cells_arrive_w); a single warp waits for the arrivals
+// (cells_wait_arrivals_w) and, after another block-wide sync, the sets are read once each (cells_read_w).
+// Polling one set instead of all of them keeps the poll traffic independent of the batch size.
+template <int WAYS>
+__device__ __forceinline__ void cells_add_sums_w(SumCell* ways, int block, double s1, double s2) {
+    SumCell* c = ways + (block % WAYS);
+    red_add_f64(&c->s1, s1);
+    red_add_f64(&c->s2, s2);
+}
+template <int WAYS>
+__device__ __forceinline__ void cells_arrive_w(SumCell* ways, int block) {
+    red_release_add_u32(&ways[block % WAYS].count, 1u);
+}
+template <int WAYS>
+__device__ __forceinline__ bool cells_wait_arrivals_w(const SumCell* ways, unsigned nblocks, WsHeader* hdr) {
+    double a, b;
+    return cells_wait_w<WAYS>(ways, nblocks, a, b, hdr);
+}
+template <int WAYS>
+__device__ __forceinline__ void cells_read_w(const SumCell* ways, double& s1, double& s2) {
+    const int lane = threadIdx.x & 31;
+    double a = 0.0, b = 0.0;
+    unsigned cnt = 0u;
+    if (lane < WAYS) ld_cell(ways + lane, a, b, cnt);
+#pragma unroll
+    for (int o = WAYS / 2; o > 0; o >>= 1) {
+        a += __shfl_xor_sync(kFull, a, o);
+        b += __shfl_xor_sync(kFull, b, o);
+    }
+    s1 = __shfl_sync(kFull, a, 0);
+    s2 = __shfl_sync(kFull, b, 0);
+}
 // The same with a running maximum kept in the cell's spare word (attention needs the largest score).
 template <int WAYS>
 __device__ __forceinline__ void cells_add_max_w(SumCell* ways, int block, double s1, double s2, float mx) {

@@ -244,18 +244,24 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
             }
             s1 = warp_sum_f64(s1);
             s2 = warp_sum_f64(s2);
-            if (lane == 0) cells_add(cells + t * kCellWays, cta, s1, s2);
+            if (lane == 0) cells_add_sums_w<kCellWays>(cells + t * kCellWays, cta, s1, s2);
         }
         p.trace.mark(3);
         __syncthreads();
+        if (tid == 0) cells_arrive_w<kCellWays>(cells, cta);      // one arrival for the group, after every token's sums
         stage(r, d2);                                   // x[r:] replaces x[:r] while the cells fill
         for (int i = tid; i < 2 * 16 * us / 2; i += kThreads) reinterpret_cast<unsigned*>(u2)[i] = 0u;
+        if (warp == 0) {
+            const bool ok = cells_wait_arrivals_w<kCellWays>(cells, static_cast<unsigned>(grid), p.hdr);
+            if (lane == 0 && !ok) s_fail = 1;
+        }
+        __syncthreads();
+        if (s_fail) return;
         for (int t = warp; t < tbv; t += kWarps) {
             double sa, sb;
-            const bool ok = cells_wait(cells + t * kCellWays, static_cast<unsigned>(grid), sa, sb, p.hdr);
+            cells_read_w<kCellWays>(cells + t * kCellWays, sa, sb);
             if (lane == 0) {
                 float th = -INFINITY;
-                if (!ok) s_fail = 1;
                 if (!p.identity) {
                     const double mean = sa * p.inv_n;
                     const float var = static_cast<float>((sb - sa * mean) * p.inv_nm1);
