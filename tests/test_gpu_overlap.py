@@ -63,8 +63,11 @@ def test_chain_of_calls_matches_ordinary_launches(ctx_pair, shape, B, cap, lens)
     for _ in range(3):                                    # timing between kernels differs from run to run
         b = chain(over, shape, B, cap, lens, 0, calls=6)[3]
         assert np.all(np.isfinite(b))
-        # six chained layers amplify the last-bit differences of the atomic reductions' order
-        np.testing.assert_allclose(b, a, rtol=0, atol=2e-4 * parity.rms(a))
+        # The order of the atomic reductions differs from run to run; over six chained layers a last-bit
+        # difference can move a score across a threshold, and the attention's hard threshold then changes
+        # the result by that token's weight.  A stale read (what this test is after) gives errors of order 1.
+        err = np.abs(b - a).max() / parity.rms(a)
+        assert err <= parity.OUT_TOL["bf16"], f"chain differs by {err:.2e} of the RMS"
 
 
 @pytest.mark.parametrize("B", [1, 4])
