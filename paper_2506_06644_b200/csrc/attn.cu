@@ -33,6 +33,9 @@ constexpr int kWarps = kThreads / kWarp;
 constexpr int kZc = 4;                // pieces per block whose quantile is cached between the passes
 constexpr int kPartPad = 8;           // floats in front of a partial accumulator: [0] max, [1] sum
 
+constexpr int kMaxAlignedSegs = 256;   // segment-aligned cut of the token space: at most this many segments ...
+constexpr int kMinAlignedSegs = 8;     // ... and at least this many (below, the set-up costs more than it saves)
+
 struct AttnParams {
     const float* q;
     const void* k1c;
@@ -51,6 +54,7 @@ struct AttnParams {
     float* scores;     // fallback when a block's scores do not fit in shared memory: [grid][GQ][ntok]
     int ntok;          // capacity (tokens) of a block's score buffer
     int sc_smem;       // 1: scores live in shared memory
+    int al_ok;         // host: the even share of a block is short enough for the segment-aligned cut to pay
     int sel_list;      // 1: pass 2 first compacts a piece's survivors into a shared-memory list per head
     SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
     float* lsum;       // [B][n_q] sum of softmax weights per head (o accumulates the weighted values)
@@ -73,7 +77,8 @@ __device__ __forceinline__ float half_sum(float v) {   // sum over the 16 lanes 
     return v;
 }
 
-template <typename KT, int GQ>
+// AL: the segment-aligned cut is available (the host asks for it when the batch has enough segments).
+template <typename KT, int GQ, bool AL>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int NS = p.B * p.n_kv;
@@ -90,7 +95,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     __shared__ float theta_s[GQ], smax_s[GQ];
     __shared__ double zcache[kZc];
     __shared__ double s_z;
-    __shared__ int s_last, s_fail;
+    __shared__ int s_last, s_fail, s_aligned;
+    __shared__ int segblk[AL ? kMaxAlignedSegs + 1 : 1];   // first block of every segment (aligned cut)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int half = lane >> 4, hl = lane & 15;
@@ -130,15 +136,60 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             run += __shfl_sync(kFull, incl, 31);
         }
         if (lane == 0) segoff[0] = 0;
+        // Two ways to cut the flat token space.  With a batch (many segments, yet no more than blocks) every
+        // segment gets a whole number of blocks in proportion to its length, so that no block works on two
+        // segments one after the other: such a block arrives late at both thresholds, holds up every block of
+        // both segments and finishes last.  Otherwise: equal flat ranges, which may span segments.  The
+        // aligned cut is taken only if every block's share fits the score buffer (sized by the host from the
+        // capacity, not from the lengths).
+        bool ok = AL && NS >= kMinAlignedSegs && NS <= G && NS <= kMaxAlignedSegs;
+        if (AL && ok) {
+            __syncwarp();
+            const int64_t Tw = run;
+            int carry = -(1 << 29);
+            for (int s0 = 0; s0 < NS; s0 += 32) {
+                const int s = s0 + lane;
+                // first block: proportional, at least one block per segment before it, room for those after it
+                int key = s < NS ? static_cast<int>(static_cast<int64_t>(G) * segoff[s] / Tw) - s : -(1 << 29);
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int t = __shfl_up_sync(kFull, key, o);
+                    if (lane >= o) key = max(key, t);
+                }
+                key = max(key, carry);
+                carry = __shfl_sync(kFull, key, 31);
+                if (s < NS) segblk[s] = min(key + s, G - NS + s);
+            }
+            if (lane == 0) segblk[NS] = G;
+            __syncwarp();
+            bool fits = true;
+            for (int s = lane; s < NS; s += 32) {
+                const int nb = segblk[s + 1] - segblk[s], L = segoff[s + 1] - segoff[s];
+                fits = fits && (L + nb - 1) / nb <= p.ntok;
+            }
+            ok = __all_sync(kFull, fits);
+        }
+        if (AL && lane == 0) s_aligned = ok ? 1 : 0;
     }
     __syncthreads();
     SumCell* cells = p.cells;
     const int64_t T = segoff[NS];
-    const int Gp = T < G ? static_cast<int>(T) : G;        // blocks that own a non-empty range
-    const bool has = cta < Gp;
-    const int64_t f0 = has ? T * cta / Gp : 0, f1 = has ? T * (cta + 1) / Gp : 0;
+    const bool aligned = AL && s_aligned != 0;
+    const int Gp = T < G ? static_cast<int>(T) : G;        // flat cut: blocks that own a non-empty range
+    int64_t f0 = 0, f1 = 0;
     int seg0 = 0;
-    {
+    if (aligned) {
+        int lo = 0, hi = NS - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (segblk[mid] <= cta) lo = mid; else hi = mid - 1;
+        }
+        seg0 = lo;
+        const int64_t i = cta - segblk[lo], nb = segblk[lo + 1] - segblk[lo], L = segoff[lo + 1] - segoff[lo];
+        f0 = segoff[lo] + L * i / nb;
+        f1 = segoff[lo] + L * (i + 1) / nb;
+    } else {
+        if (cta < Gp) { f0 = T * cta / Gp; f1 = T * (cta + 1) / Gp; }
         int lo = 0, hi = NS - 1;
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
@@ -146,7 +197,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
         }
         seg0 = lo;
     }
-    auto cta_of = [&](int64_t f) -> int { return static_cast<int>(((f + 1) * Gp - 1) / T); };
+    const bool has = f1 > f0;
+    // pieces (non-empty block ranges) of a segment: the arrivals its threshold waits for
+    auto pieces_of = [&](int seg) -> int {
+        if (aligned) {
+            const int nb = segblk[seg + 1] - segblk[seg], L = segoff[seg + 1] - segoff[seg];
+            return nb < L ? nb : L;
+        }
+        const int64_t a = segoff[seg], b = static_cast<int64_t>(segoff[seg + 1]) - 1;
+        return static_cast<int>(((b + 1) * Gp - 1) / T) - static_cast<int>(((a + 1) * Gp - 1) / T) + 1;
+    };
     // tokens of a piece that warp w owns: [w0, w1), runs of a multiple of 16 tokens
     auto warp_range = [&](int tb, int te, int& w0, int& w1) {
         const int n = te - tb;
@@ -326,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int lo = seq_len(b) - L;
             const int off = static_cast<int>(f - f0) - tb;
             const bool ident = p.k_attn >= L;
-            const int c_lo = cta_of(sb), c_hi = cta_of(static_cast<int64_t>(se) - 1);
+            const int npieces = pieces_of(seg);
             const size_t pid = static_cast<size_t>(cta + seg);
             for (int i = tid; i < GQ * hd; i += kThreads) qs[i] = p.q[(static_cast<int64_t>(b) * p.n_q + g * GQ) * hd + i];
             if (tid < GQ) sel_n[tid] = 0;
@@ -337,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 double sa, sq;
                 float smax;
                 const bool ok = cells_wait_max_w<kAttnWays>(cells + static_cast<size_t>(b * p.n_q + g * GQ + warp) * kAttnWays,
-                                                            static_cast<unsigned>(c_hi - c_lo + 1), sa, sq, smax, p.hdr);
+                                                            static_cast<unsigned>(npieces), sa, sq, smax, p.hdr);
                 if (lane == 0) {
                     if (!ok) s_fail = 1;
                     float th = -INFINITY;
@@ -522,7 +582,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 if (tid == 0) {
                     __threadfence();
                     const unsigned prev = atom_add_acqrel_u32(&p.hdr->seg_done[seg], 1u);
-                    const int last = prev == static_cast<unsigned>(c_hi - c_lo);
+                    const int last = prev == static_cast<unsigned>(npieces - 1);
                     if (last) p.hdr->seg_done[seg] = 0u;
                     s_last = last;
                 }
@@ -553,10 +613,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     p.trace.mark(3);
 }
 
-template <typename KT, int GQ>
-int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
+template <typename KT, int GQ, bool AL>
+int launch_al(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
     static bool configured[64] = {};
-    auto kern = attn_kernel<KT, GQ>;
+    auto kern = attn_kernel<KT, GQ, AL>;
     if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 8192) != cudaSuccess)
             return SPARK_ERR_CUDA;
@@ -565,6 +625,17 @@ int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) 
     void* args[] = {&p};
     return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(ctx->num_sms), kThreads, smem, stream, true, args) == cudaSuccess
                ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+template <typename KT, int GQ>
+int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
+    // The aligned cut removes the blocks that work on two segments in turn (about one pass-2 round, 5-6 us) but
+    // gives the segments 1/(blocks per segment) uneven shares of the streaming pass: worth it while a block's
+    // share of that pass is short.
+    const int ns = p.B * p.n_kv;
+    if (p.al_ok && ns >= kMinAlignedSegs && ns <= ctx->num_sms && ns <= kMaxAlignedSegs)
+        return launch_al<KT, GQ, true>(ctx, p, smem, stream);
+    return launch_al<KT, GQ, false>(ctx, p, smem, stream);
 }
 
 template <typename KT>
@@ -603,7 +674,7 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
 
     const int grid = ctx->num_sms;
     const int64_t span = (window > 0 && window < cap) ? window : cap;          // longest window of a sequence
-    const int64_t ntok = (B * n_kv * span + grid - 1) / grid + 1;            // tokens one block may own
+    int64_t ntok = (B * n_kv * span + grid - 1) / grid + 1;                  // tokens one block may own (equal flat ranges)
     // The cells keep a fixed place and size in the workspace whatever the call's shape: they must be
     // zero between launches, so nothing else may ever be written there.
     const size_t cells_b = kAttnCellBytes;
@@ -613,6 +684,18 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     const size_t smem_fixed = ns_pad * 4 + static_cast<size_t>(gq * hd) * 4 + static_cast<size_t>(kWarps) * (hd + kPartPad) * 4;
     const size_t smem_limit = static_cast<size_t>(ctx->max_smem_optin - 8192);
     if (smem_fixed > smem_limit) return SPARK_ERR_UNSUPPORTED;
+    // room for the segment-aligned cut, whose shares are uneven, when everything still fits shared memory
+    const bool al_ok = B * n_kv >= kMinAlignedSegs && ntok <= 6144;    // measured: pays at 3500 tokens a block, a tie at 7000
+    if (al_ok) {
+        const int64_t flat = ntok;
+        for (int num : {12, 9, 8, 7}) {      // 2, 1.5, 1.33, 1.17 times the even share
+            const int64_t cand = flat * num / 6 + 16;
+            if (smem_fixed + 3 * static_cast<size_t>(gq) * cand * 4 <= smem_limit) {
+                ntok = cand;
+                break;
+            }
+        }
+    }
     const size_t sc_bytes = static_cast<size_t>(gq) * ntok * 4;
     const bool sc_smem = smem_fixed + sc_bytes <= smem_limit;
     const size_t scores_b = sc_smem ? 0 : round_up(static_cast<size_t>(grid) * sc_bytes, 256);
@@ -633,6 +716,7 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;
+    p.al_ok = al_ok ? 1 : 0;
     const bool sel_list = sc_smem && smem_fixed + 3 * sc_bytes <= smem_limit;
     p.sel_list = sel_list ? 1 : 0;
     p.hdr = ctx->hdr;
