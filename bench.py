@@ -183,6 +183,24 @@ def workload_name(args, shape):
 
 
 # --------------------------------------------------------------------------------------------
+# N > 1: independent replicas, one process per GPU.  The step time is the slowest rank's; the
+# whole-job figure counts every rank's tokens.
+def max_over_ranks(ms, world, device):
+    """The largest of the ranks' times (every rank gets it).  `device`: where the process group reduces."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def us_per_token_per_layer(ms_total, steps, n_layers, batch, world):
+    """Time of one decoder layer for one token, whole job: `world` replicas each step `batch` tokens."""
+    return ms_total / steps * 1e3 / (n_layers * batch * world)
+
+
+# --------------------------------------------------------------------------------------------
 # the CUDA arm
 # --------------------------------------------------------------------------------------------
 def run_spark(args):
@@ -286,10 +304,7 @@ def run_spark(args):
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     W = max(args.warmup, 3)
     sampler = ClockSampler(local)
@@ -375,7 +390,7 @@ def run_spark(args):
     line = None
     if rank == 0:
         ms_step = ms_total / args.steps
-        us_tl = ms_step * 1e3 / (n_layers * B * world)
+        us_tl = us_per_token_per_layer(ms_total, args.steps, n_layers, B, world)
         layer_touched = touched_layer_bytes(shape, B, ctx_len, union, n_layers)
         line = {
             "metric": "us_per_token_per_layer", "value": us_tl, "unit": "us/token/layer", "n_gpus": world,
