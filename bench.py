@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="spark", choices=["spark", "reference"])
     ap.add_argument("--shape", default="2b", choices=["2b", "9b", "tiny"])
@@ -178,8 +178,8 @@ def run_reference(args):
 
 def workload_name(args, shape):
     n_layers = args.layers or shape.n_layers
-    return (f"gemma2-{args.shape}-shape spark decoder: {n_layers} layers x spark_layer_decode, "
-            f"ctx {args.ctx}, batch {args.batch}, bf16 weights+cache")
+    return (f"gemma2-{args.shape}-shape spark decoder: {n_layers} layers x spark_layer_decode, decode of "
+            f"{args.steps} tokens after a {args.ctx}-token prompt (synthetic cache), batch {args.batch}, bf16 weights+cache")
 
 
 # --------------------------------------------------------------------------------------------
@@ -220,7 +220,8 @@ def run_spark(args):
     shape = shape_of(args.shape)
     n_layers = args.layers or shape.n_layers
     B, ctx_len, d, hd = args.batch, args.ctx, shape.d, shape.hd
-    cap = ctx_len
+    W = max(args.warmup, 3)
+    cap = ctx_len + args.steps + W + 8                  # the prompt plus every token decoded in one timed loop
     ctx = S.SparkContext(local, max_batch=B, max_dff=shape.d_ff, max_cap=cap, n_q=shape.n_q, hd=hd, max_d=d)
     ctx.set_launch_overlap(bool(args.overlap))
 
@@ -249,7 +250,7 @@ def run_spark(args):
         layers.append((S.make_layer(w, cfg, cache), S.make_layer(w, cfg_dense, cache), w, cache))
     h_init = torch.randn(B, d, device=dev, generator=gen)
     h = torch.empty_like(h_init)
-    cl = torch.full((B,), ctx_len, dtype=torch.int32, device=dev)
+    cl = torch.full((B,), ctx_len + 1, dtype=torch.int32, device=dev)   # valid tokens, the one being decoded included
     scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
@@ -280,17 +281,22 @@ def run_spark(args):
         else:
             stack(which)
 
+    # One step decodes one token per sequence: the context grows by one (the lengths live on the device,
+    # so the replayed graph follows them); every timed loop starts again right after the prompt.
     def step(which=0):
         h.copy_(h_init)                                   # device-to-device copy of the token's input
         run_stack(which)
+        cl.add_(1)
 
     def step_e2e():
         h.copy_(h_host_in, non_blocking=True)             # pinned host -> device
         run_stack(0)
+        cl.add_(1)
         h_host_out.copy_(h, non_blocking=True)            # device -> pinned host
         torch.cuda.current_stream().synchronize()
 
     def timed(fn, steps, warmup):
+        cl.fill_(ctx_len + 1)
         for _ in range(warmup):
             fn()
         if world > 1:
@@ -306,7 +312,6 @@ def run_spark(args):
             dist.barrier()
         return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
-    W = max(args.warmup, 3)
     sampler = ClockSampler(local)
     sampler.start()
     ms_total = timed(step, args.steps, W)
