@@ -387,7 +387,6 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int off = static_cast<int>(f - f0) - tb;
             const bool ident = p.k_attn >= L;
             const int npieces = pieces_of(seg);
-            const size_t pid = static_cast<size_t>(cta + seg);
             for (int i = tid; i < GQ * hd; i += kThreads) qs[i] = p.q[(static_cast<int64_t>(b) * p.n_q + g * GQ) * hd + i];
             if (tid < GQ) sel_n[tid] = 0;
             if (ord >= kZc && tid == 0)

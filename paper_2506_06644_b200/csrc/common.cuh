@@ -36,8 +36,7 @@ constexpr size_t kAttnCellBytes = static_cast<size_t>(16384) * kAttnWays * 32;  
 
 struct WsHeader {            // lives at the start of the caller's workspace; zero when idle
     int status;              // device status word (SPARK_OK or a SPARK_ERR_* device code)
-    unsigned bar_count;      // inter-block barrier: arrivals of the current phase
-    unsigned bar_gen;        // inter-block barrier: generation, bumped by the last arriver
+    unsigned reserved[2];
     unsigned epoch;          // launches of the FFN kernels so far (selects their accumulator ring slot)
     unsigned pad[60];
     unsigned seg_done[kMaxSegments];   // attention: finished pieces per segment (self-resetting)
@@ -287,56 +286,6 @@ struct PhaseTrace {
 // Bound of every spin-wait, in SM cycles (about two seconds at 2 GHz).
 constexpr long long kSpinLimitCycles = 4000000000ll;
 
-// Grid-wide barrier for co-resident (cooperative) grids, split in three so that independent work
-// can sit between the steps and no round trip to L2 is exposed needlessly:
-//   begin()   once per kernel, early: thread 0 requests the current generation;
-//   arrive()  every block, once per phase: block-wide sync, then thread 0 adds its arrival;
-//   wait()    thread 0 of the last block to arrive resets the count and publishes the next
-//             generation; the others poll it.  The poll gives up after about two seconds, records
-//             SPARK_ERR_TIMEOUT and returns false (uniform over the block).
-struct GridBarrier {
-    WsHeader* hdr;
-    unsigned nblocks;
-    unsigned gen;    // generation of the phase in progress (thread 0 only)
-    unsigned prev;   // arrivals before ours (thread 0 only)
-
-    __device__ __forceinline__ void begin() {
-        if (threadIdx.x == 0) gen = ld_acquire_u32(&hdr->bar_gen);
-    }
-    __device__ __forceinline__ void arrive() {
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            __threadfence();
-            prev = atom_add_acqrel_u32(&hdr->bar_count, 1u);
-        }
-    }
-    __device__ __forceinline__ bool wait() {
-        __shared__ int ok_flag;
-        if (threadIdx.x == 0) {
-            int ok = 1;
-            if (prev == nblocks - 1) {
-                hdr->bar_count = 0;                        // ordered before the release below
-                st_release_u32(&hdr->bar_gen, gen + 1);
-            } else if (ld_acquire_u32(&hdr->bar_gen) == gen) {
-                const long long t0 = clock64();
-                while (ld_acquire_u32(&hdr->bar_gen) == gen) {
-                    if (clock64() - t0 > kSpinLimitCycles) {
-                        ok = 0;
-                        atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
-                        break;
-                    }
-                }
-            }
-            gen += 1;                                      // the next phase of this kernel
-            ok_flag = ok;
-        }
-        __syncthreads();
-        const bool ok = ok_flag != 0;
-        __syncthreads();     // ok_flag may be rewritten by the next wait
-        return ok;
-    }
-};
-
 // Sum-cell helpers.
 __device__ __forceinline__ void red_add_f64(double* p, double v) {
     asm volatile("red.relaxed.gpu.global.add.f64 [%0], %1;" ::"l"(p), "d"(v) : "memory");
@@ -355,7 +304,8 @@ __device__ __forceinline__ float ordered_to_f32(unsigned u) {
 }
 // One 32-byte read of a cell (sm_100 has 256-bit global loads): {s1, s2, count, pad[0]}.
 __device__ __forceinline__ void ld_cell_x(const SumCell* c, double& s1, double& s2, unsigned& count, unsigned& extra) {
-    unsigned long long a, b, d, e;   // e: padding half of the sector
+    unsigned long long a, b, d;
+    [[maybe_unused]] unsigned long long e;   // padding half of the sector: loaded with the rest, not used
     asm volatile("ld.acquire.gpu.global.v4.u64 {%0,%1,%2,%3}, [%4];"
                  : "=l"(a), "=l"(b), "=l"(d), "=l"(e)
                  : "l"(c)
@@ -491,53 +441,6 @@ __device__ __forceinline__ void cells_add(SumCell* ways, int block, double s1, d
 }
 __device__ __forceinline__ bool cells_wait(const SumCell* ways, unsigned nblocks, double& s1, double& s2, WsHeader* hdr) {
     return cells_wait_w<kCellWays>(ways, nblocks, s1, s2, hdr);
-}
-
-// 16-byte accesses that always go to L2 (slots other blocks write or poll).
-__device__ __forceinline__ uint4 ld_volatile16(const void* p) {
-    uint4 v;
-    asm volatile("ld.acquire.gpu.global.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p)
-                 : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_volatile16(void* p, uint4 v) {
-    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
-                 : "memory");
-}
-
-// Slot exchange between the blocks of a co-resident grid: every block publishes one 16-byte slot
-// {payload x, y, z, tag} per item and every block reads all slots, waiting for the tag of the
-// current launch.  One store and one polled load replace "atomic counter + flag + read-back":
-// the data IS the arrival.  Tags come from a launch epoch kept in the workspace header, read at
-// kernel start and advanced by block 0 once it has seen every slot.  Slot arrays are double
-// buffered by phase parity, so a block that runs ahead never overwrites a slot still being polled.
-// A poll gives up after about two seconds (SPARK_ERR_TIMEOUT is recorded; the caller returns).
-// Waits are bounded in SM cycles: the cycle counter is cheap to read, the global timer is not.
-__device__ __forceinline__ bool poll_slot(const uint4* slot, unsigned tag, uint4& out, WsHeader* hdr) {
-    out = ld_volatile16(slot);
-    if (out.w == tag) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        out = ld_volatile16(slot);
-        if (out.w == tag) return true;
-        if (clock64() - t0 > kSpinLimitCycles) {
-            atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ bool poll_flag(const unsigned* flag, unsigned tag, WsHeader* hdr) {
-    if (ld_acquire_u32(flag) == tag) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        if (ld_acquire_u32(flag) == tag) return true;
-        if (clock64() - t0 > kSpinLimitCycles) {
-            atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
-            return false;
-        }
-    }
 }
 
 // Vector reduction into global memory: y[0..3] += v (16-byte aligned address).

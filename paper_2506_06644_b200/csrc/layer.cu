@@ -137,7 +137,6 @@ template <typename WT, int TB, int RW>
 __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
     extern __shared__ __align__(16) float xs[];       // [TB][n_in]
     __shared__ float rstd[16];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_in = p.n_in;
     const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
     const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);

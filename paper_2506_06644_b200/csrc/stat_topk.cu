@@ -561,7 +561,7 @@ __device__ __forceinline__ bool row_body(const TopkParams& p, const RowGeom& g, 
 }
 
 __global__ void __launch_bounds__(kRowThreads, 1) stat_topk_row_kernel(const TopkParams p) {
-    extern __shared__ __align__(128) float srow[];
+    extern __shared__ __align__(16) float srow[];
     __shared__ RowShared sh;
     const int tid = threadIdx.x;
     RowGeom g;
