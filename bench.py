@@ -263,8 +263,12 @@ def run_spark(args):
     # The library only enqueues kernels on the caller's stream, so a whole decode step can be
     # captured once into a CUDA graph and replayed per token (what a serving loop would do).
     graphs = {}
-    if not args.no_graph:
-        side = torch.cuda.Stream()
+    side = torch.cuda.Stream()
+
+    def capture():
+        graphs.clear()
+        if args.no_graph:
+            return
         for which in ((0,) if args.no_dense else (0, 1)):
             with torch.cuda.stream(side):
                 stack(which)                               # warm-up outside capture (first-call set-up)
@@ -274,6 +278,19 @@ def run_spark(args):
                     stack(which)
             graphs[which] = g
         torch.cuda.synchronize()
+
+    capture()
+    overlap_on = bool(args.overlap)
+    if overlap_on:
+        # Launch overlap needs the GPU to itself (its blocks must all become resident).  Try it once; if a
+        # block gave up waiting, go back to ordinary cooperative launches and say so in the result.
+        for g in graphs.values():
+            g.replay()
+        stack(0)
+        if ctx.device_status() != S.SPARK_OK:
+            overlap_on = False
+            ctx.set_launch_overlap(False)
+            capture()
 
     def run_stack(which):
         if which in graphs:
@@ -404,7 +421,7 @@ def run_spark(args):
             "config": {"workload": workload_name(args, shape), "l2": "weights+caches (>3 GB) exceed L2; no flush needed",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "launch": ("host launches" if args.no_graph else "one CUDA graph replay per decode step") +
-                                 (", programmatic dependent launches (spark_set_launch_overlap)" if args.overlap else ""),
+                                 (", programmatic dependent launches (spark_set_launch_overlap)" if overlap_on else ""),
                        "local_window": 4096, "k_ff": shape.k_ff, "k_attn": shape.k_attn},
             "tokens_per_s": B * world * args.steps / (ms_total * 1e-3),
             "layer_touched_mb": layer_touched / 1e6,
