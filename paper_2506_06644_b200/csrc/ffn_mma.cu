@@ -9,8 +9,11 @@
 //   D1  T = K2t[union rows] . X[:, r:]^T, U = mask * GELU(S - theta) * T
 //   D2  Y^T += U . Vt[union rows]                          tokens x 64-column blocks, K = union rows
 // Tensor-core use: mma.sync m16n8k16 bf16 with fp32 accumulation.  The fp32 activations enter as an
-// exact three-way bf16 split (x = hi + mid + lo, one MMA per part), because the scores decide index
-// sets and must keep fp32 accuracy; u enters D2 as a two-way split.  Weight fragments are loaded
+// error-compensated two-term bf16 split (x = hi + lo, 16 mantissa bits, one MMA per term): the scores
+// decide index sets, and a bare bf16 rounding of x (2^-9 relative) would move them far outside the
+// band in which the sets may differ, whereas the two-term split moves them by about 1e-5 of their
+// spread, a tenth of that band; u enters D2 the same way.  Both halves of the split input, x[:r] and
+// x[r:], are staged once at the start when they fit side by side.  Weight fragments are loaded
 // straight from global memory with 16-byte loads: the k-slots of an MMA may be any permutation of
 // the columns as long as both operands use the same one, so a lane's 8 consecutive bf16 of a row feed
 // two MMAs without any shuffle.  (The contraction is far too small for tcgen05 tiles: M = 16 rows,
@@ -39,14 +42,20 @@ struct Plan {
     int xs;        // row stride (bf16 elements) of the split activations: = 32 mod 64 keeps 16-byte fragment reads conflict-free
     int us;        // row stride (bf16 elements) of the split u values: = 8 mod 64
     __host__ __device__ Plan(int xw, int rpc) {
-        xs = ((xw + 63) / 64) * 64 + 32;
+        xs = pad(xw);
         us = ((rpc + 15 + 63) / 64) * 64 + 8;
+    }
+    __host__ __device__ static int pad(int w) { return ((w + 63) / 64) * 64 + 32; }
+    // bf16 elements of the activation region (two split parts).  Resident: x[:r] and x[r:] side by side, staged
+    // once; otherwise one area that x[r:] takes over from x[:r] between the phases.
+    __host__ __device__ static size_t region(bool resident, int tb, int r, int d2) {
+        return resident ? static_cast<size_t>(2) * tb * (pad(r) + pad(d2)) : static_cast<size_t>(2) * tb * pad(r > d2 ? r : d2);
     }
 };
 
 // S[tile rows][tokens] = W[rows] . X^T for the block's row tiles.  rowptr(i) gives the weight row of
 // the block's i-th row (i < nrows) -- rows beyond nrows contribute zeros.  The split activations
-// xs3[part][token][xs] cover K = 32 * nch columns.  emit(i, token, value) is called once per
+// xs3[part][token][xs] (two parts) cover K = 32 * nch columns.  emit(i, token, value) is called once per
 // (row, token) by some thread.  Called by the whole block; ends with a block sync.
 template <int NT, int CB, typename RowPtr, typename Emit>
 __device__ __forceinline__ void mma_rows(RowPtr rowptr, int nrows, int nch, const __nv_bfloat16* xs3, int xs, int tb_stride,
@@ -86,7 +95,7 @@ __device__ __forceinline__ void mma_rows(RowPtr rowptr, int nrows, int nch, cons
 #pragma unroll
                     for (int n = 0; n < NT; ++n) {
 #pragma unroll
-                        for (int sp = 0; sp < 3; ++sp) {
+                        for (int sp = 0; sp < 2; ++sp) {
                             const uint4 b = *reinterpret_cast<const uint4*>(xs3 + static_cast<size_t>(sp) * tb_stride +
                                                                             static_cast<size_t>(n * 8 + g) * xs + 32 * c + 8 * t);
                             mma_bf16(acc[n], alo[u].x, ahi[u].x, alo[u].y, ahi[u].y, b.x, b.y);
@@ -118,9 +127,13 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const Plan plan(p.xw, p.rpc);
     const int xs = plan.xs, us = plan.us, rpc = p.rpc;
-    const int tb_stride = TB * xs;                                                   // one split part
-    __nv_bfloat16* xs3 = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [3][TB][xs]
-    __nv_bfloat16* u2 = xs3 + 3 * tb_stride;                                         // [2][16][us]
+    const bool xres = p.xres != 0;
+    const int xs1 = xres ? Plan::pad(p.r) : xs, xs2 = xres ? Plan::pad(p.d - p.r) : xs;   // row strides of x[:r] and x[r:]
+    const int tb_stride = TB * xs1, tb_stride2 = TB * xs2;                           // one split part of each
+    const size_t region = Plan::region(xres, TB, p.r, p.d - p.r);
+    __nv_bfloat16* xs3 = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [2][TB][xs1]: x[:r]
+    __nv_bfloat16* xr2 = xres ? xs3 + 2 * tb_stride : xs3;                           // [2][TB][xs2]: x[r:]
+    __nv_bfloat16* u2 = xs3 + region;                                                // [2][16][us]
     float4* part = reinterpret_cast<float4*>(u2 + 2 * 16 * us);                      // [kWarps][NT][32]
     float* s_loc = reinterpret_cast<float*>(part + kWarps * NT * 32);                // [TB][rpc]
     int* ulist = reinterpret_cast<int*>(s_loc + static_cast<size_t>(TB) * rpc);      // [rpc]
@@ -175,8 +188,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
             }
             __syncthreads();
         }
-        auto stage = [&](int col0, int width) {     // split x[t][col0:col0+width] (normalised) into three bf16 parts
+        // split x[t][col0:col0+width] (normalised) into two bf16 parts (hi + lo carry 16 mantissa bits: scores move by
+        // about 1e-5 of their spread, a tenth of the band inside which the index sets may differ)
+        auto stage = [&](int col0, int width, __nv_bfloat16* dst0, int stride) {
             const int w4 = width / 4;
+            const int part_stride = TB * stride;
             constexpr int SB = 8;                    // loads a thread keeps in flight
             for (int i0 = tid; i0 < TB * w4; i0 += kThreads * SB) {
                 float4 v[SB], w[SB];
@@ -199,22 +215,20 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
                     if (i >= TB * w4) break;
                     const float sc = (p.norm_w != nullptr && tt[j] < tbv) ? rstd[tt[j]] : 1.f;
                     const float f[4] = {v[j].x * sc * w[j].x, v[j].y * sc * w[j].y, v[j].z * sc * w[j].z, v[j].w * sc * w[j].w};
-                    unsigned short h[4], m[4], l[4];
+                    unsigned short h[4], m[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         h[e] = bf16_bits(f[e]);
-                        const float r1 = f[e] - bf16_val(h[e]);
-                        m[e] = bf16_bits(r1);
-                        l[e] = bf16_bits(r1 - bf16_val(m[e]));
+                        m[e] = bf16_bits(f[e] - bf16_val(h[e]));
                     }
-                    __nv_bfloat16* dst = xs3 + static_cast<size_t>(tt[j]) * xs + 4 * cc[j];
+                    __nv_bfloat16* dst = dst0 + static_cast<size_t>(tt[j]) * stride + 4 * cc[j];
                     *reinterpret_cast<uint2*>(dst) = make_uint2(h[0] | (static_cast<unsigned>(h[1]) << 16), h[2] | (static_cast<unsigned>(h[3]) << 16));
-                    *reinterpret_cast<uint2*>(dst + tb_stride) = make_uint2(m[0] | (static_cast<unsigned>(m[1]) << 16), m[2] | (static_cast<unsigned>(m[3]) << 16));
-                    *reinterpret_cast<uint2*>(dst + 2 * tb_stride) = make_uint2(l[0] | (static_cast<unsigned>(l[1]) << 16), l[2] | (static_cast<unsigned>(l[3]) << 16));
+                    *reinterpret_cast<uint2*>(dst + part_stride) = make_uint2(m[0] | (static_cast<unsigned>(m[1]) << 16), m[2] | (static_cast<unsigned>(m[3]) << 16));
                 }
             }
         };
-        stage(0, r);
+        stage(0, r, xs3, xs1);
+        if (xres) stage(r, d2, xr2, xs2);
         {
             const int64_t total4 = static_cast<int64_t>(tbv) * d / 4;
             const float4* yi = p.y_init ? reinterpret_cast<const float4*>(p.y_init + static_cast<int64_t>(g0) * d) : nullptr;
@@ -228,7 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
         p.trace.mark(1);
 
         // ---- phase A: predictor scores of this block's neurons (zero-padded K when r % 32 != 0) ------
-        mma_rows<NT, 8>([&](int i) { return K1t + static_cast<int64_t>(row0 + i) * r; }, nloc, r / 32, xs3, xs, tb_stride, part,
+        mma_rows<NT, 8>([&](int i) { return K1t + static_cast<int64_t>(row0 + i) * r; }, nloc, r / 32, xs3, xs1, tb_stride, part,
                      [&](int i, int tok, float v) { s_loc[static_cast<size_t>(tok) * rpc + i] = v; });
         p.trace.mark(2);
 
@@ -249,7 +263,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
         p.trace.mark(3);
         __syncthreads();
         if (tid == 0) cells_arrive_w<kCellWays>(cells, cta);      // one arrival for the group, after every token's sums
-        stage(r, d2);                                   // x[r:] replaces x[:r] while the cells fill
+        if (!xres) stage(r, d2, xr2, xs2);              // x[r:] replaces x[:r] while the cells fill
         for (int i = tid; i < 2 * 16 * us / 2; i += kThreads) reinterpret_cast<unsigned*>(u2)[i] = 0u;
         if (warp == 0) {
             const bool ok = cells_wait_arrivals_w<kCellWays>(cells, static_cast<unsigned>(grid), p.hdr);
@@ -324,7 +338,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
         p.trace.mark(5);
 
         // ---- D1: T = K2t[union rows] . X[:, r:]^T; U = mask * GELU(S - theta) * T, split in two bf16 parts
-        mma_rows<NT, 10>([&](int i) { return K2t + static_cast<int64_t>(row0 + ulist[i]) * d2; }, nU, d2 / 32, xs3, xs, tb_stride, part,
+        mma_rows<NT, 10>([&](int i) { return K2t + static_cast<int64_t>(row0 + ulist[i]) * d2; }, nU, d2 / 32, xr2, xs2, tb_stride2, part,
                      [&](int i, int tok, float tv) {
                          const int j = ulist[i];
                          float u = 0.f;
@@ -347,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
             const unsigned anyt = tok_any;
             const int nUp = (nU + 15) & ~15, nks = nUp >> 4;
             unsigned char* vs = smem_raw;                                  // reuses xs3
-            const int sv_bytes = 3 * tb_stride * 2;
+            const int sv_bytes = static_cast<int>(region) * 2;
             // two staging buffers: the next stripe's rows are requested while the current one is multiplied
             int WC = nUp > 0 ? (((sv_bytes / 2 / nUp) - 16) / 2) & ~63 : 0;
             if (WC > ((d + 63) & ~63)) WC = (d + 63) & ~63;
@@ -522,10 +536,12 @@ template <int TB>
 int launch_mma(spark_ctx* ctx, FfnParams& p, cudaStream_t stream) {
     static bool configured[64] = {};
     const Plan plan(p.xw, p.rpc);
-    const size_t smem = static_cast<size_t>(3) * TB * plan.xs * 2 + static_cast<size_t>(2) * 16 * plan.us * 2 +
-                        static_cast<size_t>(kWarps) * (TB / 8) * 32 * 16 + static_cast<size_t>(TB) * p.rpc * 4 +
-                        static_cast<size_t>(p.rpc) * 8 + 64;
-    if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_WORKSPACE;   // caller falls back
+    const size_t rest = static_cast<size_t>(2) * 16 * plan.us * 2 + static_cast<size_t>(kWarps) * (TB / 8) * 32 * 16 +
+                        static_cast<size_t>(TB) * p.rpc * 4 + static_cast<size_t>(p.rpc) * 8 + 64;
+    const size_t limit = static_cast<size_t>(ctx->max_smem_optin - 1024);
+    p.xres = Plan::region(true, TB, p.r, p.d - p.r) * 2 + rest <= limit ? 1 : 0;
+    const size_t smem = Plan::region(p.xres != 0, TB, p.r, p.d - p.r) * 2 + rest;
+    if (smem > limit) return SPARK_ERR_WORKSPACE;   // caller falls back
     auto kern = ffn_mma_kernel<TB>;
     if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)

@@ -17,6 +17,7 @@ struct FfnParams {
     int B, d, d_ff, r, rpc, xw;
     int ncopy;                    // B == 1 kernel: per-warp copies of y in shared memory
     int dense, erf_form, identity;
+    int xres;                     // tensor-core kernel: both halves of the split input stay in shared memory
     int overlap;                  // launched with the programmatic attribute: weights first, then dep_wait()
     double z;
     double inv_n, inv_nm1;        // 1 / d_ff and 1 / (d_ff - 1)
