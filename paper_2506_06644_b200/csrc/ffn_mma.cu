@@ -34,6 +34,11 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], unsigned a0, unsigned a1
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {      // {bf16(lo) in bits 0-15, bf16(hi) in bits 16-31}
+    unsigned r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 __device__ __forceinline__ unsigned short bf16_bits(float f) { return __bfloat16_as_ushort(__float2bfloat16_rn(f)); }
 __device__ __forceinline__ float bf16_val(unsigned short b) { return __uint_as_float(static_cast<unsigned>(b) << 16); }
 
@@ -215,15 +220,13 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_mma_kernel(const FfnParams p)
                     if (i >= TB * w4) break;
                     const float sc = (p.norm_w != nullptr && tt[j] < tbv) ? rstd[tt[j]] : 1.f;
                     const float f[4] = {v[j].x * sc * w[j].x, v[j].y * sc * w[j].y, v[j].z * sc * w[j].z, v[j].w * sc * w[j].w};
-                    unsigned short h[4], m[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        h[e] = bf16_bits(f[e]);
-                        m[e] = bf16_bits(f[e] - bf16_val(h[e]));
-                    }
+                    // two values per conversion: hi = bf16x2(f), lo = bf16x2(f - hi); a bf16 widens by a 16-bit shift
+                    const unsigned h01 = pack_bf16x2(f[0], f[1]), h23 = pack_bf16x2(f[2], f[3]);
+                    const unsigned m01 = pack_bf16x2(f[0] - __uint_as_float(h01 << 16), f[1] - __uint_as_float(h01 & 0xffff0000u));
+                    const unsigned m23 = pack_bf16x2(f[2] - __uint_as_float(h23 << 16), f[3] - __uint_as_float(h23 & 0xffff0000u));
                     __nv_bfloat16* dst = dst0 + static_cast<size_t>(tt[j]) * stride + 4 * cc[j];
-                    *reinterpret_cast<uint2*>(dst) = make_uint2(h[0] | (static_cast<unsigned>(h[1]) << 16), h[2] | (static_cast<unsigned>(h[3]) << 16));
-                    *reinterpret_cast<uint2*>(dst + part_stride) = make_uint2(m[0] | (static_cast<unsigned>(m[1]) << 16), m[2] | (static_cast<unsigned>(m[3]) << 16));
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(h01, h23);
+                    *reinterpret_cast<uint2*>(dst + part_stride) = make_uint2(m01, m23);
                 }
             }
         };
