@@ -426,6 +426,10 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
                         static_cast<size_t>(p.rpc) * 8;
     if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_UNSUPPORTED;
     if (a.B == 1 && grid <= 512 && a.d <= 4096) return ffn1_launch(ctx, p, a.wdtype, stream);
+    if (a.B >= 2 && a.B <= 4 && grid <= 512) {
+        const int rc = ffn_few_launch(ctx, p, a.wdtype, stream);
+        if (rc != SPARK_ERR_WORKSPACE) return rc;
+    }
     if (a.B >= 2 && a.wdtype == SPARK_BF16) {
         const int rc = ffn_mma_launch(ctx, p, stream);
         if (rc != SPARK_ERR_WORKSPACE) return rc;

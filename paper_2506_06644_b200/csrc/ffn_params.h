@@ -18,6 +18,7 @@ struct FfnParams {
     int ncopy;                    // B == 1 kernel: per-warp copies of y in shared memory
     int dense, erf_form, identity;
     int xres;                     // tensor-core kernel: both halves of the split input stay in shared memory
+    int vrows, vstage_off;        // few-token kernel: rows of V per round and the byte offset of their staging area
     int overlap;                  // launched with the programmatic attribute: weights first, then dep_wait()
     double z;
     double inv_n, inv_nm1;        // 1 / d_ff and 1 / (d_ff - 1)
@@ -34,6 +35,9 @@ struct FfnParams {
 // Tensor-core path for bf16 weights and 2..64 tokens (ffn_mma.cu); SPARK_ERR_WORKSPACE = shape not
 // served, use the plain-ALU kernel.
 int ffn_mma_launch(spark_ctx* ctx, FfnParams& p, cudaStream_t stream);
+
+// 2..4 tokens without tensor cores (ffn_few.cu); SPARK_ERR_WORKSPACE = shape not served.
+int ffn_few_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream);
 
 // B == 1 fast path (ffn_b1.cu).
 int ffn1_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream);

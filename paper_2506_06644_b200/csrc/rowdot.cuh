@@ -29,7 +29,7 @@ __device__ __forceinline__ void rows_dot_mapped(const WT* __restrict__ W, int64_
     constexpr int TPL = TB / TS;             // tokens per lane group
     constexpr int GL = 32 / TS;              // lanes per group
     // chunks per lane held in flight per batch (upper bound); the batches of a row are made equal
-    constexpr int CU = (TB == 1 ? (RW >= 4 ? 4 : (RW == 2 ? 10 : 8)) : 2) / (sizeof(WT) == 4 ? 2 : 1);
+    constexpr int CU = (TB == 1 ? (RW >= 4 ? 4 : (RW == 2 ? 10 : 8)) : (TB <= 4 && RW == 4 && sizeof(WT) == 2 ? 4 : 2)) / (sizeof(WT) == 4 ? 2 : 1);
     const int per_lane = (nck + GL - 1) / GL;
     const int nbatch = (per_lane + CU - 1) / CU;
     const int cu = nbatch > 0 ? (per_lane + nbatch - 1) / nbatch : 1;      // <= CU
