@@ -5,6 +5,7 @@
 #include <cmath>
 
 #include "kernels.h"
+#include "mma_rows.cuh"
 #include "rowdot.cuh"
 
 using namespace spark;
@@ -156,6 +157,110 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
                                  p.y[o] = p.y_add != nullptr ? v + p.y_add[o] : v;
                              }
                          });
+}
+
+// The same product for 5..16 tokens on the tensor cores: with that many tokens the plain-ALU kernel is bound by
+// the shared-memory reads of the inputs (every 16 bytes of weights meet 16 x 32 bytes of activations).  The
+// inputs (divided, normalised) are staged once as a two-term bf16 split; the block's rows go through mma_rows.
+template <int TB>
+__global__ void __launch_bounds__(kThreads, 1) gemv_mma_kernel(const GemvParams p) {
+    using namespace spark::mma;
+    constexpr int NT = TB / 8;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int n_in = p.n_in, xsd = Plan::pad(n_in), tb_stride = TB * xsd;
+    __nv_bfloat16* xs2 = reinterpret_cast<__nv_bfloat16*>(smem_raw);                 // [2][TB][xsd]
+    float4* part = reinterpret_cast<float4*>(xs2 + 2 * tb_stride);                   // [kWarps][NT][32]
+    __shared__ float rstd[16];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * p.n_out / gridDim.x);
+    const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
+    dep_wait();
+    dep_trigger();
+    for (int i = blockIdx.x * kThreads + tid; i < p.zero_n16; i += gridDim.x * kThreads) p.zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
+    const int w4 = n_in / 4;
+    auto divisor = [&](int t, int c4) -> float {
+        if (p.x_div == nullptr) return 1.f;
+        const float dv = p.x_div[static_cast<int64_t>(t) * (n_in / p.x_div_group) + (c4 * 4) / p.x_div_group];
+        return dv > 0.f ? 1.f / dv : 0.f;
+    };
+    if (p.norm_w != nullptr) {                        // a warp per token: sum of squares of the (divided) input
+        for (int t = warp; t < TB; t += kWarps) {
+            float ss = 0.f;
+            if (t < p.B) {
+                const float4* xr = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(t) * n_in);
+                for (int i = lane; i < w4; i += 32) {
+                    const float4 v = xr[i];
+                    const float iv = divisor(t, i);
+                    ss += (v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w) * iv * iv;
+                }
+                ss = warp_sum(ss);
+            }
+            if (lane == 0) rstd[t] = rsqrtf(ss / static_cast<float>(n_in) + p.eps);
+        }
+        __syncthreads();
+    }
+    constexpr int SB = 8;                             // loads a thread keeps in flight
+    for (int i0 = tid; i0 < TB * w4; i0 += kThreads * SB) {
+        float4 v[SB];
+        float sc[SB];
+        int tt[SB], cc[SB];
+#pragma unroll
+        for (int j = 0; j < SB; ++j) {
+            const int i = i0 + j * kThreads;
+            tt[j] = i / w4;
+            cc[j] = i - tt[j] * w4;
+            v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            sc[j] = 1.f;
+            if (i < TB * w4 && tt[j] < p.B) {
+                v[j] = reinterpret_cast<const float4*>(p.x + static_cast<int64_t>(tt[j]) * n_in)[cc[j]];
+                sc[j] = divisor(tt[j], cc[j]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < SB; ++j) {
+            const int i = i0 + j * kThreads;
+            if (i >= TB * w4) break;
+            float4 w = make_float4(1.f, 1.f, 1.f, 1.f);
+            float s = sc[j];
+            if (p.norm_w != nullptr) {
+                w = __ldg(reinterpret_cast<const float4*>(p.norm_w) + cc[j]);
+                s *= tt[j] < p.B ? rstd[tt[j]] : 0.f;
+            }
+            const float f[4] = {v[j].x * s * w.x, v[j].y * s * w.y, v[j].z * s * w.z, v[j].w * s * w.w};
+            const unsigned h01 = pack_bf16x2(f[0], f[1]), h23 = pack_bf16x2(f[2], f[3]);
+            const unsigned m01 = pack_bf16x2(f[0] - __uint_as_float(h01 << 16), f[1] - __uint_as_float(h01 & 0xffff0000u));
+            const unsigned m23 = pack_bf16x2(f[2] - __uint_as_float(h23 << 16), f[3] - __uint_as_float(h23 & 0xffff0000u));
+            __nv_bfloat16* dst = xs2 + static_cast<size_t>(tt[j]) * xsd + 4 * cc[j];
+            *reinterpret_cast<uint2*>(dst) = make_uint2(h01, h23);
+            *reinterpret_cast<uint2*>(dst + tb_stride) = make_uint2(m01, m23);
+        }
+    }
+    __syncthreads();
+    const __nv_bfloat16* Wt = static_cast<const __nv_bfloat16*>(p.Wt);
+    mma_rows<NT, 8>([&](int i) { return Wt + static_cast<int64_t>(row0 + i) * n_in; }, row1 - row0, n_in / 32, xs2, xsd, tb_stride, part,
+                    [&](int i, int tok, float v) {
+                        if (tok < p.B) {
+                            const int64_t o = static_cast<int64_t>(tok) * p.n_out + row0 + i;
+                            p.y[o] = p.y_add != nullptr ? v + p.y_add[o] : v;
+                        }
+                    });
+}
+
+template <int TB>
+int gemv_mma_launch(spark_ctx* ctx, GemvParams& p, int grid, cudaStream_t stream) {
+    static bool configured[64] = {};
+    const size_t smem = static_cast<size_t>(2) * TB * spark::mma::Plan::pad(p.n_in) * 2 + static_cast<size_t>(kWarps) * (TB / 8) * 32 * 16;
+    if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_WORKSPACE;
+    auto kern = gemv_mma_kernel<TB>;
+    if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        configured[ctx->device] = true;
+    }
+    p.overlap = ctx->overlap;
+    void* args[] = {&p};
+    return launch_kernel(ctx, reinterpret_cast<const void*>(kern), static_cast<unsigned>(grid), kThreads, smem, stream, false, args) == cudaSuccess
+               ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
 template <typename WT, int TB, int RW>
@@ -402,6 +507,14 @@ int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
         p.x_div_group = static_cast<int>(a.x_div ? a.x_div_group : 1);
         p.zero_ptr = done == 0 ? static_cast<uint4*>(a.zero_ptr) : nullptr;
         p.zero_n16 = done == 0 ? static_cast<int>(a.zero_bytes / 16) : 0;
+        if (nb >= 5 && a.wdtype == SPARK_BF16 && (a.n_in & 31) == 0 && a.n_out >= 16) {      // tensor cores
+            const int rc = nb <= 8 ? gemv_mma_launch<8>(ctx, p, grid, stream) : gemv_mma_launch<16>(ctx, p, grid, stream);
+            if (rc == SPARK_OK) {
+                done += nb;
+                continue;
+            }
+            if (rc != SPARK_ERR_WORKSPACE) return rc;
+        }
         const size_t smem = static_cast<size_t>(tb) * a.n_in * 4;
         const int st = a.wdtype == SPARK_BF16 ? gemv_dispatch<__nv_bfloat16>(ctx, p, tb, rw, smem, grid, stream)
                                               : gemv_dispatch<float>(ctx, p, tb, rw, smem, grid, stream);
@@ -467,7 +580,9 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     int rc;
     const int tbq = B == 1 ? 1 : (B <= 4 ? 4 : 16);
     const size_t smem_q = static_cast<size_t>(tbq) * cfg->d * 4;
-    if ((cfg->d & 7) == 0 && smem_q <= static_cast<size_t>(ctx->max_smem_optin - 1024) && nqkv / 2 >= 1 &&
+    // up to four tokens: projection, rotary encoding and cache append in one kernel; more: the tensor-core GEMV,
+    // then a small kernel for the rotary encoding and the append
+    if (B <= 4 && (cfg->d & 7) == 0 && smem_q <= static_cast<size_t>(ctx->max_smem_optin - 1024) && nqkv / 2 >= 1 &&
         aligned16(w->Wqkv) && aligned16(w->norm1)) {
         QkvRopeParams qp;
         qp.g.x = h; qp.g.norm_w = w->norm1; qp.g.eps = cfg->rms_eps; qp.g.Wt = w->Wqkv;

@@ -86,6 +86,8 @@ def run_layer(ctx, sh, B, cap, lens, seed, window=0, flags=0):
     (synth.TINY, 2, 128, [100, 90], 32),
     (synth.GEMMA2_2B, 1, 2048, [2048], 0),
     (synth.GEMMA2_2B, 2, 1024, [700, 1024], 512),
+    (synth.TINY, 5, 64, [64, 3, 40, 17, 1], 0),                    # five and more tokens: tensor-core projections
+    (synth.GEMMA2_2B, 6, 512, [512, 300, 77, 1, 450, 260], 0),
 ])
 def test_layer_against_oracle(ctx, shape, B, cap, lens, window):
     lw, kv, h0, h, cache = run_layer(ctx, shape, B, cap, lens, seed=4, window=window)
@@ -95,10 +97,13 @@ def test_layer_against_oracle(ctx, shape, B, cap, lens, window):
     for b in range(B):
         n = lens[b]
         ref, kc, vc = oracle_layer(shape, lw, kv, h0, b, n, window)
-        # the appended cache row: equal up to one bf16 rounding step of an fp32-vs-fp64 difference
+        # the appended cache row: equal up to one bf16 rounding step of an fp32-vs-fp64 difference; with five or
+        # more tokens the projection's inputs are a two-term bf16 split (16 mantissa bits), an absolute error of
+        # about 1e-5 of the row's scale before the rounding
         got_k = np.concatenate([k1[b, :, n - 1], k2[b, :, n - 1]], axis=-1)
-        np.testing.assert_allclose(got_k, kc[:, n - 1], rtol=2 ** -7, atol=1e-6)
-        np.testing.assert_allclose(v[b, :, n - 1], vc[:, n - 1], rtol=2 ** -7, atol=1e-6)
+        atol = 1e-6 if B < 5 else 1e-4 * parity.rms(kc[:, n - 1])
+        np.testing.assert_allclose(got_k, kc[:, n - 1], rtol=2 ** -7, atol=atol)
+        np.testing.assert_allclose(v[b, :, n - 1], vc[:, n - 1], rtol=2 ** -7, atol=atol)
         # untouched rows stay untouched
         if n > 1:
             assert np.array_equal(k1[b, :, : n - 1], kv.k1c[b, :, : n - 1])
