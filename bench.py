@@ -542,6 +542,47 @@ def other_workloads(torch, S, peak, steps, warmup):
         ctx.close()
         del caches
 
+    # -- eight layers of the decoder at batch 8 (eight sequences, 8192-token synthetic caches each)
+    B, L, nl = 8, 8192, 8
+    ctx = S.SparkContext(dev.index, max_batch=B, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
+    ctx.set_launch_overlap(True)
+    nqkv = (sh.n_q + 2 * sh.n_kv) * sh.hd
+
+    def wm(rows, cols, fan_in):
+        return (torch.randn(rows, cols, device=dev, generator=gen) * fan_in ** -0.5).to(torch.bfloat16)
+    stacks = {0: [], S.SPARK_DENSE_LOADS: []}
+    for l in range(nl):
+        wts = dict(norm1=torch.ones(sh.d, device=dev), norm2=torch.ones(sh.d, device=dev), Wqkv=wm(nqkv, sh.d, sh.d),
+                   Wo=wm(sh.d, sh.n_q * sh.hd, sh.n_q * sh.hd), K1t=wm(sh.d_ff, sh.r_ff, sh.d), K2t=wm(sh.d_ff, sh.d - sh.r_ff, sh.d),
+                   Vt=wm(sh.d_ff, sh.d, sh.d))
+        cache = dict(k1c=torch.randn(B, sh.n_kv, L, sh.r_attn, device=dev, generator=gen).to(torch.bfloat16),
+                     k2c=torch.randn(B, sh.n_kv, L, sh.hd - sh.r_attn, device=dev, generator=gen).to(torch.bfloat16),
+                     vc=torch.randn(B, sh.n_kv, L, sh.hd, device=dev, generator=gen).to(torch.bfloat16))
+        for flags in stacks:
+            cfg = dict(d=sh.d, d_ff=sh.d_ff, r_ff=sh.r_ff, k_ff=sh.k_ff, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+                       k_attn=sh.k_attn, window=4096 if l % 2 == 0 else 0, cap=L, rms_eps=1e-6, rope_base=10000.0, flags=flags)
+            stacks[flags].append((S.make_layer(wts, cfg, cache), wts, cache))
+    h = torch.randn(B, sh.d, device=dev, generator=gen)
+    cl = torch.full((B,), L, dtype=torch.int32, device=dev)
+    scratch = torch.empty(B * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device=dev)
+    res = []
+    for flags in (0, S.SPARK_DENSE_LOADS):
+        def calls():
+            for lay in stacks[flags]:
+                S.spark_layer_decode(ctx, lay[0], cl, h, B, scratch)
+        res.append(time_graph(calls, nl))
+    assert ctx.device_status() == S.SPARK_OK
+    lens = [4096 if l % 2 == 0 else L for l in range(nl)]
+    nbytes = sum((nqkv * sh.d + sh.d * sh.n_q * sh.hd + sh.d_ff * sh.r_ff) * 2 +
+                 B * (sh.n_kv * n * sh.r_attn * 2 + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn) * 2) for n in lens) / nl
+    out.append({"workload": f"spark_layer_decode gemma2-2b shape, batch {B}, context {L} (local 4096 / global), {nl} layers: "
+                            "per layer; touched bytes without the FFN's gathered rows",
+                "us_per_launch": res[0], "us_per_token_per_layer": res[0] / B, "touched_mb": nbytes / 1e6,
+                "gbs_touched": nbytes / res[0] / 1e3, "frac_of_measured_peak": nbytes / res[0] / 1e3 / peak,
+                "dense_loads_us_per_launch": res[1], "speedup_vs_dense_loads": res[1] / res[0]})
+    ctx.close()
+    del stacks
+
     # -- statistical top-k, 4096 rows x 65536 (1.07 GB read per launch)
     ctx = S.SparkContext(dev.index)
     rows, n = 4096, 65536
