@@ -254,7 +254,7 @@ def run_spark(args):
     scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
-    kernels_per_layer = 4          # QKV+rotary+append, attention, output projection, FFN
+    kernels_per_layer = 4 if B <= 4 else 5     # QKV (+ rotary, append: a kernel of their own for B >= 5), attention, output projection, FFN
 
     def stack(which):
         for lay in layers:

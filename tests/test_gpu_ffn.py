@@ -69,7 +69,7 @@ def test_tiny_fp32_layer(ctx):
         compare(p, run_ffn(ctx, p, flags=flags), form=form)
 
 
-@pytest.mark.parametrize("B", [1, 4, 16])
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 8, 16])     # 1: one-token kernel; 2-4: few-token kernel; 5-16: tensor cores
 def test_gemma2_2b_shape_bf16(ctx, B):
     p = synth.ffn_inputs(2304, 9216, 1024, 737, B, "bf16", seed=0)
     w = upload(p)
