@@ -519,6 +519,32 @@ def other_workloads(torch, S, peak, steps, warmup):
         ctx.close()
     del sets
 
+    # -- Spark FFN, one token, at the paper's iso-parameter width (Section 4: d_ff 13824, k 1106), 6 weight sets (600 MB)
+    dffw, kw = 13824, 1106
+
+    def ww(rows, cols):
+        return (torch.randn(rows, cols, device=dev, generator=gen) * sh.d ** -0.5).to(torch.bfloat16)
+    sets = [(ww(dffw, sh.r_ff), ww(dffw, sh.d - sh.r_ff), ww(dffw, sh.d)) for _ in range(6)]
+    ctx = S.SparkContext(dev.index, max_batch=1, max_dff=dffw, max_d=sh.d)
+    ctx.set_launch_overlap(True)
+    x = torch.randn(1, sh.d, device=dev, generator=gen)
+    y = torch.empty(1, sh.d, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    S.spark_ffn_decode(ctx, x, 1, *sets[0], S.SPARK_BF16, sh.d, dffw, sh.r_ff, kw, 0, y, None, cnt, None)
+    torch.cuda.synchronize()
+    nact = int(cnt[0])
+    res = []
+    for flags in (0, S.SPARK_DENSE_LOADS):
+        def calls():
+            for k1, k2, v in sets:
+                S.spark_ffn_decode(ctx, x, 1, k1, k2, v, S.SPARK_BF16, sh.d, dffw, sh.r_ff, kw, flags, y, None, None, None)
+        res.append(time_graph(calls, len(sets)))
+    assert ctx.device_status() == S.SPARK_OK
+    entry(f"spark_ffn_decode at the paper's width: d {sh.d}, d_ff {dffw}, r {sh.r_ff}, k {kw}, 1 token ({nact} active)", res[0],
+          dffw * sh.r_ff * 2 + nact * (2 * sh.d - sh.r_ff) * 2, res[1])
+    ctx.close()
+    del sets
+
     # -- Spark attention, long contexts
     for B, L, nsets in ((1, 16384, 6), (8, 32768, 2)):
         ctx = S.SparkContext(dev.index, max_batch=B, max_cap=L, n_q=sh.n_q, hd=sh.hd)
