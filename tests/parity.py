@@ -10,7 +10,10 @@ import numpy as np
 
 THETA_RTOL = 1e-5
 BAND = 1e-4
-OUT_TOL = {"bf16": 2e-2, "f32": 1e-5}
+# "split2": exact (bf16-representable) weights met by activations that the tensor-core kernels feed as a two-term
+# bf16 split (16 mantissa bits): every product carries a relative error of up to 2^-17 = 7.6e-6, the largest of
+# tens of thousands of outputs lands near 1e-5 of the RMS; 4e-5 leaves a factor of four.
+OUT_TOL = {"bf16": 2e-2, "f32": 1e-5, "split2": 4e-5}
 
 
 def rms(a):
