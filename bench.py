@@ -545,6 +545,33 @@ def other_workloads(torch, S, peak, steps, warmup):
     ctx.close()
     del sets
 
+    # -- Spark FFN, one token, FP8 E4M3 weights with one scale per neuron (quantisation on top of sparsity), 12 sets
+    def q8(rows, cols):
+        wf = torch.randn(rows, cols, device=dev, generator=gen) * sh.d ** -0.5
+        sc = wf.abs().amax(dim=1) / 448.0
+        return (wf / sc[:, None]).to(torch.float8_e4m3fn).view(torch.uint8), sc
+    sets = [(q8(sh.d_ff, sh.r_ff), q8(sh.d_ff, sh.d - sh.r_ff), q8(sh.d_ff, sh.d)) for _ in range(12)]
+    ctx = S.SparkContext(dev.index, max_batch=1, max_dff=sh.d_ff, max_d=sh.d)
+    ctx.set_launch_overlap(True)
+    x = torch.randn(1, sh.d, device=dev, generator=gen)
+    y = torch.empty(1, sh.d, device=dev)
+    cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+    (a, a_s), (b, b_s), (c, c_s) = sets[0]
+    S.spark_ffn_decode_fp8(ctx, x, 1, a, a_s, b, b_s, c, c_s, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, 0, y, None, cnt, None)
+    torch.cuda.synchronize()
+    nact = int(cnt[0])
+    res = []
+    for flags in (0, S.SPARK_DENSE_LOADS):
+        def calls():
+            for (a, a_s), (b, b_s), (c, c_s) in sets:
+                S.spark_ffn_decode_fp8(ctx, x, 1, a, a_s, b, b_s, c, c_s, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, flags, y, None, None, None)
+        res.append(time_graph(calls, len(sets)))
+    assert ctx.device_status() == S.SPARK_OK
+    entry(f"spark_ffn_decode_fp8 gemma2-2b shape, 1 token, FP8 E4M3 weights + per-neuron scales ({nact} active)", res[0],
+          sh.d_ff * sh.r_ff + nact * (2 * sh.d - sh.r_ff) + sh.d_ff * 4 + nact * 8, res[1])
+    ctx.close()
+    del sets
+
     # -- Spark attention, long contexts
     for B, L, nsets in ((1, 16384, 6), (8, 32768, 2)):
         ctx = S.SparkContext(dev.index, max_batch=B, max_cap=L, n_q=sh.n_q, hd=sh.hd)

@@ -59,7 +59,7 @@ enum {
 };
 
 /* ---- dtypes and flags ----------------------------------------------------- */
-enum { SPARK_F32 = 0, SPARK_BF16 = 1 };
+enum { SPARK_F32 = 0, SPARK_BF16 = 1, SPARK_FP8_E4M3 = 2 /* spark_ffn_decode_fp8 only */ };
 
 enum {
     SPARK_FILL_ZERO = 0,   /* Eq. 10: entries not above theta become 0                       */
@@ -153,6 +153,16 @@ int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int
 int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const void* K2t,
                      const void* Vt, int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k,
                      int flags, float* y, float* theta, int32_t* count, int32_t* idx, void* stream);
+
+/* The same FFN with the three matrices stored as FP8 E4M3 (1-4-3 bits, bias 7, largest finite 448) and one
+ * fp32 scale per neuron: row i of K1t / K2t / Vt stands for K1s[i] / K2s[i] / Vs[i] times its stored values
+ * (quantised weights are named in the paper's closing section as the natural companion of activation sparsity;
+ * the format and the per-neuron scales are this library's choice).  K1t [d_ff][r], K2t [d_ff][d-r], Vt [d_ff][d]
+ * uint8 device buffers, 16-byte aligned, r and d multiples of 8; K1s, K2s, Vs [d_ff] fp32.  One token only
+ * (B == 1, d <= 4096): SPARK_ERR_UNSUPPORTED otherwise.  Everything else as spark_ffn_decode. */
+int spark_ffn_decode_fp8(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const float* K1s, const void* K2t,
+                         const float* K2s, const void* Vt, const float* Vs, int64_t d, int64_t d_ff, int64_t r, int64_t k,
+                         int flags, float* y, float* theta, int32_t* count, int32_t* idx, void* stream);
 
 /* ---- Spark FFN without any allocation (the paper has no counterpart) ----------------------
  * Some callers may not call cudaMalloc at all: code that runs where device memory has been

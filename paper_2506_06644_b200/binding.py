@@ -20,14 +20,14 @@ LIB_PATH = os.path.join(_HERE, "libspark_b200.so")
 SPARK_OK = 0
 SPARK_ERR_INVALID_ARG, SPARK_ERR_UNSUPPORTED, SPARK_ERR_WORKSPACE, SPARK_ERR_CUDA = 1, 2, 3, 4
 SPARK_ERR_TIMEOUT, SPARK_ERR_OVERFLOW = 5, 6
-SPARK_F32, SPARK_BF16 = 0, 1
+SPARK_F32, SPARK_BF16, SPARK_FP8_E4M3 = 0, 1, 2
 SPARK_FILL_ZERO, SPARK_FILL_NEGINF = 0, 1
 SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
 
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
     "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_set_launch_overlap", "spark_stat_topk", "spark_ffn_decode",
-    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc",
+    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8",
 ]
 
 
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
         "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
         "spark_ffn_decode": (i32, [vp, vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
         "spark_ffn_decode_noalloc": (i32, [vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp]),
+        "spark_ffn_decode_fp8": (i32, [vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
         "spark_attn_decode": (i32, [vp, vp, vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
                                     vp, vp, vp, vp, i64, vp]),
         "spark_dense_gemv": (i32, [vp, vp, i64, vp, i32, i64, i64, vp, vp, vp]),
@@ -185,6 +186,11 @@ def spark_stat_topk(ctx: SparkContext, x, rows, n, ld, k, fill, theta, count, id
 def spark_ffn_decode(ctx: SparkContext, x, B, K1t, K2t, Vt, wdtype, d, d_ff, r, k, flags, y, theta, count, idx):
     _check(lib().spark_ffn_decode(ctx.handle, _ptr(x), B, _ptr(K1t), _ptr(K2t), _ptr(Vt), wdtype, d, d_ff, r, k,
                                   flags, _ptr(y), _ptr(theta), _ptr(count), _ptr(idx), _stream()), "spark_ffn_decode")
+
+
+def spark_ffn_decode_fp8(ctx: SparkContext, x, B, K1t, K1s, K2t, K2s, Vt, Vs, d, d_ff, r, k, flags, y, theta, count, idx):
+    _check(lib().spark_ffn_decode_fp8(ctx.handle, _ptr(x), B, _ptr(K1t), _ptr(K1s), _ptr(K2t), _ptr(K2s), _ptr(Vt), _ptr(Vs), d,
+                                      d_ff, r, k, flags, _ptr(y), _ptr(theta), _ptr(count), _ptr(idx), _stream()), "spark_ffn_decode_fp8")
 
 
 def spark_ffn_decode_noalloc(x, B, K1t, K2t, Vt, wdtype, d, d_ff, r, k, flags, y, theta):

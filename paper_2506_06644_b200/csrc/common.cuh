@@ -3,6 +3,7 @@
 
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <stdint.h>
 
 #include "../../include/spark.h"
@@ -141,6 +142,32 @@ struct Row8<__nv_bfloat16> {
         f[2] = __uint_as_float(raw.y << 16); f[3] = __uint_as_float(raw.y & 0xffff0000u);
         f[4] = __uint_as_float(raw.z << 16); f[5] = __uint_as_float(raw.z & 0xffff0000u);
         f[6] = __uint_as_float(raw.w << 16); f[7] = __uint_as_float(raw.w & 0xffff0000u);
+    }
+};
+
+// FP8 E4M3 storage (per-row scales are applied by the caller): eight values = eight bytes.
+template <>
+struct Row8<__nv_fp8_e4m3> {
+    uint2 raw;
+    __device__ __forceinline__ void load(const __nv_fp8_e4m3* row, int64_t chunk) {
+        asm("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(raw.x), "=r"(raw.y) : "l"(reinterpret_cast<const uint2*>(row) + chunk));
+    }
+    __device__ __forceinline__ void load_pinned(const __nv_fp8_e4m3* row, int64_t chunk) {
+        asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(raw.x), "=r"(raw.y) : "l"(reinterpret_cast<const uint2*>(row) + chunk));
+    }
+    __device__ __forceinline__ void zero() { raw = make_uint2(0u, 0u); }
+    __device__ __forceinline__ void unpack(float (&f)[8]) const {
+        // two e4m3 -> two f16 in one conversion, then f16 -> f32; element 0 sits in the lowest byte
+        const unsigned w[2] = {raw.x, raw.y};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            unsigned h01, h23;
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"(static_cast<unsigned short>(w[i] & 0xffffu)));
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"(static_cast<unsigned short>(w[i] >> 16)));
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+            f[4 * i] = a.x; f[4 * i + 1] = a.y; f[4 * i + 2] = b.x; f[4 * i + 3] = b.y;
+        }
     }
 };
 

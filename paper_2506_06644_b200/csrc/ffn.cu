@@ -396,7 +396,9 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     if (a.B < 1 || a.B > 64 || a.d < 16 || a.d_ff < 2 || a.r <= 0 || a.r >= a.d || a.k <= 0) return SPARK_ERR_INVALID_ARG;
     if (a.idx != nullptr && a.count == nullptr) return SPARK_ERR_INVALID_ARG;
     if (a.y_init == a.y && a.y_init != nullptr) return SPARK_ERR_INVALID_ARG;
-    if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
+    if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16 && a.wdtype != SPARK_FP8_E4M3) return SPARK_ERR_UNSUPPORTED;
+    if (a.wdtype == SPARK_FP8_E4M3 && (a.K1s == nullptr || a.K2s == nullptr || a.Vs == nullptr)) return SPARK_ERR_INVALID_ARG;
+    if (a.wdtype == SPARK_FP8_E4M3 && (a.B != 1 || a.d > 4096)) return SPARK_ERR_UNSUPPORTED;      // one token only
     if ((a.r & 7) != 0 || (a.d & 7) != 0) return SPARK_ERR_UNSUPPORTED;
     if (!aligned16(a.x) || !aligned16(a.K1t) || !aligned16(a.K2t) || !aligned16(a.Vt) || !aligned16(a.y) ||
         !aligned16(a.y_init) || !aligned16(a.norm_w))
@@ -409,6 +411,9 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     FfnParams p;
     p.x = a.x; p.norm_w = a.norm_w; p.eps = a.rms_eps;
     p.K1t = a.K1t; p.K2t = a.K2t; p.Vt = a.Vt;
+    p.K1s = a.wdtype == SPARK_FP8_E4M3 ? a.K1s : nullptr;
+    p.K2s = a.wdtype == SPARK_FP8_E4M3 ? a.K2s : nullptr;
+    p.Vs = a.wdtype == SPARK_FP8_E4M3 ? a.Vs : nullptr;
     p.B = static_cast<int>(a.B); p.d = static_cast<int>(a.d); p.d_ff = static_cast<int>(a.d_ff); p.r = static_cast<int>(a.r);
     p.rpc = static_cast<int>((a.d_ff + grid - 1) / grid);
     p.xw = static_cast<int>(a.r > a.d - a.r ? a.r : a.d - a.r);
@@ -425,6 +430,7 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     const size_t smem = (static_cast<size_t>(tb) * p.xw + static_cast<size_t>(2) * tb * p.rpc) * sizeof(float) +
                         static_cast<size_t>(p.rpc) * 8;
     if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_UNSUPPORTED;
+    if (a.wdtype == SPARK_FP8_E4M3) return grid <= 512 ? ffn1_launch(ctx, p, a.wdtype, stream) : SPARK_ERR_UNSUPPORTED;
     if (a.B == 1 && grid <= 512 && a.d <= 4096) return ffn1_launch(ctx, p, a.wdtype, stream);
     if (a.B >= 2 && a.B <= 4 && grid <= 512) {
         const int rc = ffn_few_launch(ctx, p, a.wdtype, stream);
@@ -446,6 +452,22 @@ extern "C" int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const
     FfnArgs a;
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
     a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = wdtype;
+    a.K1s = nullptr; a.K2s = nullptr; a.Vs = nullptr;
+    a.B = B; a.d = d; a.d_ff = d_ff; a.r = r; a.k = k; a.flags = flags;
+    a.y_init = nullptr; a.y = y; a.theta = theta; a.count = count; a.idx = idx;
+    return ffn_launch(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+// FP8 storage of the three matrices with one fp32 scale per neuron (the paper's closing section expects
+// quantisation to compound with activation sparsity: it halves the bytes of what is still read).
+extern "C" int spark_ffn_decode_fp8(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const float* K1s,
+                                    const void* K2t, const float* K2s, const void* Vt, const float* Vs, int64_t d,
+                                    int64_t d_ff, int64_t r, int64_t k, int flags, float* y, float* theta, int32_t* count,
+                                    int32_t* idx, void* stream) {
+    FfnArgs a;
+    a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
+    a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = SPARK_FP8_E4M3;
+    a.K1s = K1s; a.K2s = K2s; a.Vs = Vs;
     a.B = B; a.d = d; a.d_ff = d_ff; a.r = r; a.k = k; a.flags = flags;
     a.y_init = nullptr; a.y = y; a.theta = theta; a.count = count; a.idx = idx;
     return ffn_launch(ctx, a, static_cast<cudaStream_t>(stream));
@@ -506,6 +528,7 @@ extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K
     FfnArgs a;
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
     a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = wdtype;
+    a.K1s = nullptr; a.K2s = nullptr; a.Vs = nullptr;
     a.B = B; a.d = d; a.d_ff = d_ff; a.r = r; a.k = k; a.flags = flags;
     a.y_init = nullptr; a.y = y; a.theta = theta; a.count = nullptr; a.idx = nullptr;
     return ffn_launch(&local, a, static_cast<cudaStream_t>(stream));

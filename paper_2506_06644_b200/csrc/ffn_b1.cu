@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     float* s_loc = ys + static_cast<size_t>(p.ncopy) * p.d;                                    // [rpc]  scores of this block's neurons
     int* lst_j = reinterpret_cast<int*>(s_loc + p.rpc);         // [rpc]  active neurons (local index)
     float* lst_a = reinterpret_cast<float*>(lst_j + p.rpc);     // [rpc]  s - theta (or -inf: read, not used)
+    float* ksc = lst_a + p.rpc;                                 // [rpc]  scales of this block's K1t rows (1 without)
     __shared__ double red_a[kWarps];
     __shared__ float s_theta;
     __shared__ unsigned s_epoch;
@@ -51,6 +52,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     const WT* Vt = static_cast<const WT*>(p.Vt);
     const int d4 = d / 4;
     const int n_init = (d4 + kThreads - 1) / kThreads;          // blocks that initialise y
+    for (int j = tid; j < nloc; j += kThreads) ksc[j] = p.K1s != nullptr ? __ldg(p.K1s + row0 + j) : 1.f;   // weights: never written
     // Everything that another kernel may have written is read in after_dependency(): with launch overlap
     // that is after the first batch of K1t loads has been issued (they fly while the kernel before
     // this one in the stream drains); otherwise before them, so that the token's input is in shared memory
@@ -111,7 +113,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
 
     // ---- A: predictor scores s = K1^T x[:r] of this block's neurons ---------------------------------
     rows_dot<WT, 1, kRows>(K1t, r, row0, nloc, r / 8, xs, 0, [&]() { if (p.overlap) after_dependency(); }, prologue,
-                           [&](int j, int, float v) { s_loc[j] = v; });
+                           [&](int j, int, float v) { s_loc[j] = v * ksc[j]; });
     __syncthreads();
     p.trace.mark(2);
 
@@ -187,6 +189,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
         const float aj = lst_a[e];
         const WT* krow = K2t + static_cast<int64_t>(row0 + j) * d2;
         const WT* vrow = Vt + static_cast<int64_t>(row0 + j) * d;
+        const float rsc = (p.K2s != nullptr ? __ldg(p.K2s + row0 + j) : 1.f) * (p.Vs != nullptr ? __ldg(p.Vs + row0 + j) : 1.f);
         Row8<WT> kw[kKB], vw[kVB];
 #pragma unroll
         for (int u = 0; u < kKB; ++u) {
@@ -219,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
             }
         }
         t = warp_sum(t);
-        const float uval = aj == -INFINITY ? 0.f : (p.erf_form ? gelu_erf(aj) : gelu_tanh(aj)) * t;
+        const float uval = aj == -INFINITY ? 0.f : (p.erf_form ? gelu_erf(aj) : gelu_tanh(aj)) * t * rsc;
 #pragma unroll 1
         for (int c0 = 0;;) {
 #pragma unroll
@@ -272,9 +275,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
 namespace spark {
 
 int ffn1_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream) {
-    static bool configured[2][64] = {};
+    static bool configured[3][64] = {};
     if (p.d / 4 > 2 * kThreads) return SPARK_ERR_UNSUPPORTED;    // the input is held in two float4 per thread
-    const size_t fixed = (static_cast<size_t>(p.d) + 3 * static_cast<size_t>(p.rpc)) * 4 + 16;
+    const size_t fixed = (static_cast<size_t>(p.d) + 4 * static_cast<size_t>(p.rpc)) * 4 + 16;
     const size_t limit = static_cast<size_t>(ctx->max_smem_optin - 2048);
     if (fixed + static_cast<size_t>(p.d) * 4 > limit) return SPARK_ERR_UNSUPPORTED;
     size_t ncopy = (limit - fixed) / (static_cast<size_t>(p.d) * 4);
@@ -283,8 +286,9 @@ int ffn1_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream) {
     const size_t smem = fixed + ncopy * p.d * 4;
     if ((p.d / 4 + kThreads - 1) / kThreads > ctx->num_sms) return SPARK_ERR_UNSUPPORTED;
     const void* kern = wdtype == SPARK_BF16 ? reinterpret_cast<const void*>(ffn1_kernel<__nv_bfloat16>)
-                                            : reinterpret_cast<const void*>(ffn1_kernel<float>);
-    const int wi = wdtype == SPARK_BF16 ? 1 : 0;
+                     : (wdtype == SPARK_FP8_E4M3 ? reinterpret_cast<const void*>(ffn1_kernel<__nv_fp8_e4m3>)
+                                                 : reinterpret_cast<const void*>(ffn1_kernel<float>));
+    const int wi = wdtype == SPARK_BF16 ? 1 : (wdtype == SPARK_FP8_E4M3 ? 2 : 0);
     if (ctx->device >= 0 && ctx->device < 64 && !configured[wi][ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
             return SPARK_ERR_CUDA;

@@ -14,6 +14,9 @@ struct FfnParams {
     const void* K1t;
     const void* K2t;
     const void* Vt;
+    const float* K1s;             // nullable: per-neuron scales of the three matrices (FP8 storage), [d_ff] each
+    const float* K2s;
+    const float* Vs;
     int B, d, d_ff, r, rpc, xw;
     int ncopy;                    // B == 1 kernel: per-warp copies of y in shared memory
     int dense, erf_form, identity;

@@ -14,6 +14,9 @@ struct FfnArgs {
     const void* K2t;
     const void* Vt;
     int wdtype;
+    const float* K1s;        // per-neuron scales [d_ff] of K1t, K2t, Vt: required for SPARK_FP8_E4M3, nullptr otherwise
+    const float* K2s;
+    const float* Vs;
     int64_t B, d, d_ff, r, k;
     int flags;
     const float* y_init;     // nullable: y = y_init + FFN(x) (y_init must not alias y)

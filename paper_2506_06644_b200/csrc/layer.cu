@@ -629,6 +629,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     FfnArgs f;
     f.x = h2; f.norm_w = w->norm2; f.rms_eps = cfg->rms_eps;
     f.K1t = w->K1t; f.K2t = w->K2t; f.Vt = w->Vt; f.wdtype = SPARK_BF16;
+    f.K1s = nullptr; f.K2s = nullptr; f.Vs = nullptr;
     f.B = B; f.d = cfg->d; f.d_ff = cfg->d_ff; f.r = cfg->r_ff; f.k = cfg->k_ff; f.flags = cfg->flags;
     f.y_init = h2; f.y = h; f.theta = nullptr; f.count = nullptr; f.idx = nullptr;
     return ffn_launch(ctx, f, st);

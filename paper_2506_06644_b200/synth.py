@@ -41,6 +41,47 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
 
 
+def f32_to_e4m3_bits(a: np.ndarray) -> np.ndarray:
+    """Round fp32 to FP8 E4M3 (1-4-3 bits, bias 7, largest finite 448, no infinities; nearest, ties to even,
+    magnitudes beyond 448 saturate); returns the uint8 patterns.  NaN -> 0x7f."""
+    a = np.ascontiguousarray(a, dtype=np.float32).astype(np.float64)
+    sign = np.signbit(a).astype(np.uint8) << np.uint8(7)
+    mag = np.minimum(np.abs(a), 448.0)
+    # subnormal codes (and zero): multiples of 2^-9 below 2^-6
+    sub = np.rint(mag * 512.0)
+    m, e = np.frexp(np.where(mag > 0, mag, 1.0))                  # mag = m * 2^e, m in [0.5, 1)
+    expo = e - 1
+    mant = np.rint((2.0 * m - 1.0) * 8.0)
+    carry = mant >= 8
+    mant = np.where(carry, 0, mant)
+    expo = np.where(carry, expo + 1, expo)
+    code = np.where(mag < 2.0 ** -6, sub, (expo + 7) * 8 + mant)
+    code = np.minimum(code, 0x7E).astype(np.uint8)
+    out = sign | code
+    return np.where(np.isnan(a), np.uint8(0x7F), out).astype(np.uint8)
+
+
+def e4m3_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """Widen FP8 E4M3 bit patterns to fp32 (exact); 0x7f / 0xff are NaN."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint8)
+    codes = np.arange(256)
+    e, m = (codes >> 3) & 15, codes & 7
+    val = np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * 2.0 ** (e - 7.0))
+    val = np.where(codes & 0x80, -val, val)
+    val[[0x7F, 0xFF]] = np.nan
+    return val.astype(np.float32)[bits]
+
+
+def quantize_rows_e4m3(W: np.ndarray):
+    """Per-row scaled FP8 storage of a weight matrix: W[i, :] ~ scale[i] * e4m3(bits[i, :]) with
+    scale[i] = max|W[i, :]| / 448 (1 for an all-zero row).  Returns (bits uint8, scale float32)."""
+    W = np.ascontiguousarray(W, dtype=np.float32)
+    amax = np.abs(W).max(axis=1)
+    scale = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+    bits = f32_to_e4m3_bits(W / scale[:, None])
+    return bits, scale
+
+
 def _rng(seed: int, stream: int) -> np.random.Generator:
     # One independent stream per tensor, so that adding a tensor to a workload
     # does not change the others.

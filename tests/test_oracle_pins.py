@@ -403,3 +403,44 @@ def test_decoder_layer_composition_against_library_ops():
     act = torch.nn.functional.gelu(T(W["K1t"]) @ b[: sh.r_ff])
     h = h + T(W["Vt"]).T @ (act * (T(W["K2t"]) @ b[sh.r_ff:]))
     np.testing.assert_allclose(out["h"], h.numpy(), rtol=1e-11, atol=1e-13)
+
+
+# ---- storage rounding to FP8 E4M3 (used by the quantised-weight FFN; a library routine is the pin) ----------------
+def test_e4m3_rounding_matches_the_library_cast_and_known_codes():
+    import torch
+    from paper_2506_06644_b200 import synth
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.standard_normal(50000).astype(np.float32) * s for s in (1e-3, 2e-2, 1.0, 40.0, 200.0)])
+    x = np.clip(x, -448.0, 448.0)                      # the library cast does not saturate; the generator does
+    ref = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(synth.f32_to_e4m3_bits(x), ref)
+    # known codes: 1 = 0x38, largest finite 448 = 0x7e, smallest subnormal 2^-9 = 0x01, smallest normal 2^-6 = 0x08
+    known = {1.0: 0x38, 448.0: 0x7E, 2.0 ** -9: 0x01, 2.0 ** -6: 0x08, -2.0: 0xC0, 0.0: 0x00, 1.5: 0x3C}
+    got = synth.f32_to_e4m3_bits(np.array(list(known), dtype=np.float32))
+    assert got.tolist() == list(known.values())
+    # ties go to the even mantissa; beyond the range the value saturates
+    ties = synth.f32_to_e4m3_bits(np.array([1.0625, 1.1875, 2.0 ** -10, 3 * 2.0 ** -10, 1000.0, -1e9], dtype=np.float32))
+    assert ties.tolist() == [0x38, 0x3A, 0x00, 0x02, 0x7E, 0xFE]
+    # decoding all 254 finite codes agrees with the library, and encode(decode(code)) is the identity
+    codes = np.arange(256, dtype=np.uint8)
+    val = synth.e4m3_bits_to_f32(codes)
+    lib = torch.from_numpy(codes).view(torch.float8_e4m3fn).float().numpy()
+    fin = ~np.isnan(lib)
+    assert fin.sum() == 254 and np.array_equal(val[fin], lib[fin]) and np.all(np.isnan(val[~fin]))
+    back = synth.f32_to_e4m3_bits(val[fin])
+    assert np.array_equal(back & 0x7F, codes[fin] & 0x7F) and np.array_equal(back[val[fin] != 0], codes[fin][val[fin] != 0])
+
+
+def test_row_scaled_e4m3_quantisation_error_bound():
+    from paper_2506_06644_b200 import synth
+    W = synth.normal_f32((64, 512), 9, 1, 0.02)
+    W[3] = 0.0
+    bits, scale = synth.quantize_rows_e4m3(W)
+    deq = synth.e4m3_bits_to_f32(bits) * scale[:, None]
+    assert scale[3] == 1.0 and np.all(deq[3] == 0)
+    amax = np.abs(W).max(axis=1, keepdims=True)
+    # three mantissa bits: relative error <= 2^-4 for normal values; absolute error <= half a subnormal step (scaled) below
+    err = np.abs(deq - W)
+    bound = np.maximum(np.abs(W) * 2.0 ** -4, (amax / 448.0) * 2.0 ** -10)
+    assert np.all(err <= bound * (1 + 1e-6))
+    assert np.all(np.abs(deq).max(axis=1) <= amax[:, 0] * (1 + 1e-6))
