@@ -592,8 +592,25 @@ def other_workloads(torch, S, peak, steps, warmup):
         assert ctx.device_status() == S.SPARK_OK
         nbytes = B * (sh.n_kv * L * sh.r_attn * 2 + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn) * 2)
         entry(f"spark_attn_decode 8q/4kv heads hd 256, context {L}, batch {B}, k_attn {sh.k_attn}", res[0], nbytes, res[1])
+        # the same with the predictor slice of the cache in FP8 E4M3 (one scale per cached row)
+        q8c = []
+        for k1c, k2c, vc in caches:
+            kf = k1c.float()
+            sc = kf.abs().amax(dim=-1).clamp_min(1e-30) / 448.0
+            q8c.append(((kf / sc[..., None]).to(torch.float8_e4m3fn).view(torch.uint8), sc, k2c, vc))
+            del kf
+
+        def calls8():
+            for rep in range(2):
+                for k1q, k1s, k2c, vc in q8c:
+                    S.spark_attn_decode_fp8k(ctx, q, k1q, k1s, k2c, vc, B, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, L, cl, 0, sh.k_attn, 0,
+                                             o, None, None, None, 0)
+        us8 = time_graph(calls8, 2 * nsets)
+        assert ctx.device_status() == S.SPARK_OK
+        nbytes8 = B * (sh.n_kv * L * (sh.r_attn + 4) + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn) * 2)
+        entry(f"spark_attn_decode_fp8k (FP8 predictor slice), context {L}, batch {B}, k_attn {sh.k_attn}", us8, nbytes8)
         ctx.close()
-        del caches
+        del caches, q8c
 
     # -- eight layers of the decoder at batch 8 (eight sequences, 8192-token synthetic caches each)
     B, L, nl = 8, 8192, 8

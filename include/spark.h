@@ -214,6 +214,16 @@ int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c, const voi
                       int flags, float* o, float* theta, int32_t* count, int32_t* idx,
                       int64_t idx_cap, void* stream);
 
+/* The same attention with the predictor slice of the cache stored as FP8 E4M3: k1c [B][n_kv][cap][r] uint8 and
+ * k1s [B][n_kv][cap] fp32, cached row t of a head standing for k1s[t] times its stored values; k2c and vc stay
+ * bf16.  The predictor slice is all that a long context streams, so this halves the bytes read there (the paper's
+ * closing section names quantisation as the companion of activation sparsity; format and per-row scales are this
+ * library's choice).  Everything else as spark_attn_decode. */
+int spark_attn_decode_fp8k(spark_ctx* ctx, const float* q, const void* k1c, const float* k1s, const void* k2c,
+                           const void* vc, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap,
+                           const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags, float* o, float* theta,
+                           int32_t* count, int32_t* idx, int64_t idx_cap, void* stream);
+
 /* ---- dense GEMV (the projections the method leaves dense: Table "FLOPs per token") ----
  * y[b][n_out] = Wt[n_out][n_in] . x[b][n_in] (+ y_add[b][n_out] if y_add != NULL).
  * Wt of dtype wdtype, output-major; n_in % 8 == 0; 1 <= B <= 16.  y_add may equal y. */

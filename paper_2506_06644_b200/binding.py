@@ -27,7 +27,7 @@ SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
     "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_set_launch_overlap", "spark_stat_topk", "spark_ffn_decode",
-    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8",
+    "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
 ]
 
 
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         "spark_ffn_decode_fp8": (i32, [vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
         "spark_attn_decode": (i32, [vp, vp, vp, vp, vp, i32, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
                                     vp, vp, vp, vp, i64, vp]),
+        "spark_attn_decode_fp8k": (i32, [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
+                                         vp, vp, vp, vp, i64, vp]),
         "spark_dense_gemv": (i32, [vp, vp, i64, vp, i32, i64, i64, vp, vp, vp]),
         "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
                                      vp, vp, i64, vp, vp]),
@@ -205,6 +207,13 @@ def spark_attn_decode(ctx: SparkContext, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv,
     _check(lib().spark_attn_decode(ctx.handle, _ptr(q), _ptr(k1c), _ptr(k2c), _ptr(vc), kvdtype, B, n_q, n_kv, hd,
                                    r, cap, _ptr(ctx_len), window, k_attn, flags, _ptr(o), _ptr(theta), _ptr(count),
                                    _ptr(idx), idx_cap, _stream()), "spark_attn_decode")
+
+
+def spark_attn_decode_fp8k(ctx: SparkContext, q, k1c, k1s, k2c, vc, B, n_q, n_kv, hd, r, cap, ctx_len, window, k_attn, flags,
+                           o, theta, count, idx, idx_cap):
+    _check(lib().spark_attn_decode_fp8k(ctx.handle, _ptr(q), _ptr(k1c), _ptr(k1s), _ptr(k2c), _ptr(vc), B, n_q, n_kv, hd, r, cap,
+                                        _ptr(ctx_len), window, k_attn, flags, _ptr(o), _ptr(theta), _ptr(count), _ptr(idx), idx_cap,
+                                        _stream()), "spark_attn_decode_fp8k")
 
 
 def spark_dense_gemv(ctx: SparkContext, x, B, Wt, wdtype, n_in, n_out, y_add, y):

@@ -44,6 +44,7 @@ struct AttnParams {
     int B, n_q, n_kv, hd, r;
     int64_t cap;
     const int32_t* ctx_len;
+    const float* k1s;  // nullable: k1c is FP8 E4M3 and k1s[B][n_kv][cap] holds one scale per cached row
     const double* zs;  // nullable: Q(1 - k_attn / L_b) per sequence, precomputed by an earlier kernel
     int window, k_attn, dense;
     float* o;
@@ -78,7 +79,8 @@ __device__ __forceinline__ float half_sum(float v) {   // sum over the 16 lanes 
 }
 
 // AL: the segment-aligned cut is available (the host asks for it when the batch has enough segments).
-template <typename KT, int GQ, bool AL>
+// K1T: storage of the predictor slice k1c (KT, or FP8 E4M3 with one fp32 scale per cached row in p.k1s).
+template <typename KT, typename K1T, int GQ, bool AL>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int NS = p.B * p.n_kv;
@@ -103,7 +105,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     const int G = gridDim.x, cta = blockIdx.x;
     const int nc1 = r / 8, nc2 = d2 / 8, ncv = hd / 8;
     const int pstride = hd + kPartPad;
-    const KT* k1c = static_cast<const KT*>(p.k1c);
+    const K1T* k1c = static_cast<const K1T*>(p.k1c);
     const KT* k2c = static_cast<const KT*>(p.k2c);
     const KT* vc = static_cast<const KT*>(p.vc);
     float* sc = p.sc_smem ? sc_s : p.scores + static_cast<size_t>(cta) * GQ * p.ntok;
@@ -220,17 +222,17 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     // The first batch of predictor rows is requested before anything else is waited for: before the
     // query is staged and, when the lengths are known to be stable, before the kernel ahead of this one
     // has finished (its newest cache row is held back until it has).
-    Row8<KT> wpre[8];
+    Row8<K1T> wpre[8];
     bool have_pre = false;
     {
         int held = -1;
-        const KT* held_row = nullptr;
+        const K1T* held_row = nullptr;
         if (has) {
             const int sb = segoff[seg0], se = segoff[seg0 + 1], L = se - sb;
             const int tb = static_cast<int>(f0 - sb);
             const int te = static_cast<int>((f1 < se ? f1 : se) - sb);
             const int lo = seq_len(seg0 / p.n_kv) - L;
-            const KT* kbase = k1c + (static_cast<int64_t>(seg0) * p.cap + lo) * r;
+            const K1T* kbase = k1c + (static_cast<int64_t>(seg0) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
             if (w0 < w1) {
@@ -286,14 +288,20 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             float mx[GQ];
 #pragma unroll
             for (int hq = 0; hq < GQ; ++hq) { s1[hq] = 0.0; s2[hq] = 0.0; mx[hq] = -INFINITY; }
-            const KT* kbase = k1c + (static_cast<int64_t>(seg) * p.cap + lo) * r;
+            const K1T* kbase = k1c + (static_cast<int64_t>(seg) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
             const int jidx = ((hl >> 3) & 1) * 4 + ((hl >> 2) & 1) * 2 + ((hl >> 1) & 1);
 #pragma unroll 1
             for (int base = w0; base < w1; base += 16) {
                 const int tok0 = base + half * 8;
-                Row8<KT> w[8];
+                Row8<K1T> w[8];
+                // the scale of the row whose score this lane ends up with (FP8 predictor slice), requested with the rows
+                [[maybe_unused]] float ksc = 1.f;
+                if constexpr (sizeof(K1T) == 1) {
+                    const int tsc = tok0 + jidx;
+                    if ((hl & 1) == 0 && tsc < w1) ksc = p.k1s[static_cast<int64_t>(seg) * p.cap + lo + tsc];
+                }
                 if (have_pre && ord == 0 && base == w0) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) w[j] = wpre[j];
@@ -337,6 +345,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     const float send = b2 ? a2[0][hq] : a2[1][hq];
                     a1[hq] = keep + __shfl_xor_sync(kFull, send, 2);
                     a1[hq] += __shfl_xor_sync(kFull, a1[hq], 1);
+                    if constexpr (sizeof(K1T) == 1) a1[hq] *= ksc;
                 }
                 const int t = tok0 + jidx;
                 if ((hl & 1) == 0 && t < w1) {
@@ -612,10 +621,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     p.trace.mark(3);
 }
 
-template <typename KT, int GQ, bool AL>
+template <typename KT, typename K1T, int GQ, bool AL>
 int launch_al(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
     static bool configured[64] = {};
-    auto kern = attn_kernel<KT, GQ, AL>;
+    auto kern = attn_kernel<KT, K1T, GQ, AL>;
     if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 8192) != cudaSuccess)
             return SPARK_ERR_CUDA;
@@ -626,24 +635,24 @@ int launch_al(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
                ? SPARK_OK : SPARK_ERR_CUDA;
 }
 
-template <typename KT, int GQ>
+template <typename KT, typename K1T, int GQ>
 int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
     // The aligned cut removes the blocks that work on two segments in turn (about one pass-2 round, 5-6 us) but
     // gives the segments 1/(blocks per segment) uneven shares of the streaming pass: worth it while a block's
     // share of that pass is short.
     const int ns = p.B * p.n_kv;
     if (p.al_ok && ns >= kMinAlignedSegs && ns <= ctx->num_sms && ns <= kMaxAlignedSegs)
-        return launch_al<KT, GQ, true>(ctx, p, smem, stream);
-    return launch_al<KT, GQ, false>(ctx, p, smem, stream);
+        return launch_al<KT, K1T, GQ, true>(ctx, p, smem, stream);
+    return launch_al<KT, K1T, GQ, false>(ctx, p, smem, stream);
 }
 
-template <typename KT>
+template <typename KT, typename K1T>
 int launch_gq(spark_ctx* ctx, AttnParams& p, int gq, size_t smem, cudaStream_t stream) {
     switch (gq) {
-        case 1: return launch_one<KT, 1>(ctx, p, smem, stream);
-        case 2: return launch_one<KT, 2>(ctx, p, smem, stream);
-        case 4: return launch_one<KT, 4>(ctx, p, smem, stream);
-        case 8: return launch_one<KT, 8>(ctx, p, smem, stream);
+        case 1: return launch_one<KT, K1T, 1>(ctx, p, smem, stream);
+        case 2: return launch_one<KT, K1T, 2>(ctx, p, smem, stream);
+        case 4: return launch_one<KT, K1T, 4>(ctx, p, smem, stream);
+        case 8: return launch_one<KT, K1T, 8>(ctx, p, smem, stream);
         default: return SPARK_ERR_UNSUPPORTED;
     }
 }
@@ -655,7 +664,7 @@ namespace spark {
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
-                int64_t idx_cap, cudaStream_t st) {
+                int64_t idx_cap, const float* k1s, cudaStream_t st) {
     if (ctx == nullptr || q == nullptr || k1c == nullptr || k2c == nullptr || vc == nullptr || ctx_len == nullptr ||
         o == nullptr)
         return SPARK_ERR_INVALID_ARG;
@@ -664,6 +673,7 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
         return SPARK_ERR_INVALID_ARG;
     if (idx != nullptr && (count == nullptr || idx_cap < 1)) return SPARK_ERR_INVALID_ARG;
     if (kvdtype != SPARK_F32 && kvdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
+    if (k1s != nullptr && kvdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;      // FP8 predictor slice: beside bf16 k2c / vc
     const int64_t gq = n_q / n_kv;
     if (hd > 256 || (r & 7) != 0 || ((hd - r) & 7) != 0 || r > 128 || hd - r > 128) return SPARK_ERR_UNSUPPORTED;
     if (gq != 1 && gq != 2 && gq != 4 && gq != 8) return SPARK_ERR_UNSUPPORTED;
@@ -721,8 +731,10 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.hdr = ctx->hdr;
     p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
     const size_t smem = smem_fixed + (sel_list ? 3 * sc_bytes : (sc_smem ? sc_bytes : 0));
-    if (kvdtype == SPARK_BF16) return launch_gq<__nv_bfloat16>(ctx, p, static_cast<int>(gq), smem, st);
-    return launch_gq<float>(ctx, p, static_cast<int>(gq), smem, st);
+    p.k1s = k1s;
+    if (k1s != nullptr) return launch_gq<__nv_bfloat16, __nv_fp8_e4m3>(ctx, p, static_cast<int>(gq), smem, st);
+    if (kvdtype == SPARK_BF16) return launch_gq<__nv_bfloat16, __nv_bfloat16>(ctx, p, static_cast<int>(gq), smem, st);
+    return launch_gq<float, float>(ctx, p, static_cast<int>(gq), smem, st);
 }
 
 }  // namespace spark
@@ -733,5 +745,15 @@ extern "C" int spark_attn_decode(spark_ctx* ctx, const float* q, const void* k1c
                                  float* o, float* theta, int32_t* count, int32_t* idx, int64_t idx_cap,
                                  void* stream) {
     return attn_launch(ctx, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv, hd, r, cap, ctx_len, nullptr, window, k_attn, flags, o,
-                       nullptr, theta, count, idx, idx_cap, static_cast<cudaStream_t>(stream));
+                       nullptr, theta, count, idx, idx_cap, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+// The predictor slice of the cache in FP8 E4M3 with one fp32 scale per cached row; k2c and vc stay bf16.
+extern "C" int spark_attn_decode_fp8k(spark_ctx* ctx, const float* q, const void* k1c, const float* k1s, const void* k2c,
+                                      const void* vc, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap,
+                                      const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags, float* o, float* theta,
+                                      int32_t* count, int32_t* idx, int64_t idx_cap, void* stream) {
+    if (k1s == nullptr) return SPARK_ERR_INVALID_ARG;
+    return attn_launch(ctx, q, k1c, k2c, vc, SPARK_BF16, B, n_q, n_kv, hd, r, cap, ctx_len, nullptr, window, k_attn, flags, o,
+                       nullptr, theta, count, idx, idx_cap, k1s, static_cast<cudaStream_t>(stream));
 }

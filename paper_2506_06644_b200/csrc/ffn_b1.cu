@@ -52,7 +52,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     const WT* Vt = static_cast<const WT*>(p.Vt);
     const int d4 = d / 4;
     const int n_init = (d4 + kThreads - 1) / kThreads;          // blocks that initialise y
-    for (int j = tid; j < nloc; j += kThreads) ksc[j] = p.K1s != nullptr ? __ldg(p.K1s + row0 + j) : 1.f;   // weights: never written
+    constexpr bool kScaled = sizeof(WT) == 1;                   // FP8 storage: one scale per neuron and matrix
+    if constexpr (kScaled)
+        for (int j = tid; j < nloc; j += kThreads) ksc[j] = __ldg(p.K1s + row0 + j);   // weights: never written
     // Everything that another kernel may have written is read in after_dependency(): with launch overlap
     // that is after the first batch of K1t loads has been issued (they fly while the kernel before
     // this one in the stream drains); otherwise before them, so that the token's input is in shared memory
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
 
     // ---- A: predictor scores s = K1^T x[:r] of this block's neurons ---------------------------------
     rows_dot<WT, 1, kRows>(K1t, r, row0, nloc, r / 8, xs, 0, [&]() { if (p.overlap) after_dependency(); }, prologue,
-                           [&](int j, int, float v) { s_loc[j] = v * ksc[j]; });
+                           [&](int j, int, float v) { s_loc[j] = kScaled ? v * ksc[j] : v; });
     __syncthreads();
     p.trace.mark(2);
 
@@ -189,7 +191,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
         const float aj = lst_a[e];
         const WT* krow = K2t + static_cast<int64_t>(row0 + j) * d2;
         const WT* vrow = Vt + static_cast<int64_t>(row0 + j) * d;
-        const float rsc = (p.K2s != nullptr ? __ldg(p.K2s + row0 + j) : 1.f) * (p.Vs != nullptr ? __ldg(p.Vs + row0 + j) : 1.f);
+        float rsc = 1.f;
+        if constexpr (kScaled) rsc = __ldg(p.K2s + row0 + j) * __ldg(p.Vs + row0 + j);
         Row8<WT> kw[kKB], vw[kVB];
 #pragma unroll
         for (int u = 0; u < kKB; ++u) {
@@ -222,7 +225,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
             }
         }
         t = warp_sum(t);
-        const float uval = aj == -INFINITY ? 0.f : (p.erf_form ? gelu_erf(aj) : gelu_tanh(aj)) * t * rsc;
+        float uval = aj == -INFINITY ? 0.f : (p.erf_form ? gelu_erf(aj) : gelu_tanh(aj)) * t;
+        if constexpr (kScaled) uval *= rsc;
 #pragma unroll 1
         for (int c0 = 0;;) {
 #pragma unroll

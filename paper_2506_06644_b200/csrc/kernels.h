@@ -47,10 +47,11 @@ int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 // Spark attention; zs (nullable) holds Q(1 - k_attn / L_b) per sequence when an earlier kernel of the
 // same stream has already computed it.  With lsum != nullptr the kernel leaves o unnormalised (the
 // weighted value sums), writes the sums of weights to lsum[B][n_q] and leaves its score-sum cells
-// for the caller's next kernel to clear (the first B * n_q * kAttnWays cells of the scratch area).
+// for the caller's next kernel to clear (the first B * n_q * kAttnWays cells of the scratch area).  With k1s !=
+// nullptr the predictor slice k1c is FP8 E4M3 and k1s[B][n_kv][cap] holds one scale per cached row (bf16 k2c / vc).
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
-                int64_t idx_cap, cudaStream_t st);
+                int64_t idx_cap, const float* k1s, cudaStream_t st);
 
 }  // namespace spark
