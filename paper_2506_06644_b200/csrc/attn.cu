@@ -33,6 +33,23 @@ constexpr int kWarps = kThreads / kWarp;
 constexpr int kZc = 4;                // pieces per block whose quantile is cached between the passes
 constexpr int kPartPad = 8;           // floats in front of a partial accumulator: [0] max, [1] sum
 
+// FP8 predictor slice on the tensor cores (r = 128, one or two query heads per KV head): a warp takes 16 cached
+// rows as the M dimension of mma.m16n8k32 e4m3 tiles -- the stored bytes are the A operand as they are, nothing
+// is unpacked -- and the query as four e4m3 terms per head in the eight columns (term i of head h in column
+// 4 h + i, scaled by qsc[4 h + i]; each term carries four significant bits, 16 in all).  q8 row stride 160 bytes:
+// the 8-byte fragment reads of a half warp fall on distinct banks.
+constexpr int kQ8Stride = 160;
+__device__ __forceinline__ void mma_e4m3_16832(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint2 raw8_of(const Row8<__nv_fp8_e4m3>& w) { return w.raw; }
+template <typename T>
+__device__ __forceinline__ uint2 raw8_of(const Row8<T>&) { return make_uint2(0u, 0u); }          // never used: other storage types
+__device__ __forceinline__ unsigned char to_e4m3(float x) { return static_cast<unsigned char>(__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3)); }
+__device__ __forceinline__ float from_e4m3(unsigned char b) { return __half2float(__half(__nv_cvt_fp8_to_halfraw(b, __NV_E4M3))); }
+
 constexpr int kMaxAlignedSegs = 256;   // segment-aligned cut of the token space: at most this many segments ...
 constexpr int kMinAlignedSegs = 8;     // ... and at least this many (below, the set-up costs more than it saves)
 
@@ -98,6 +115,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     __shared__ double zcache[kZc];
     __shared__ double s_z;
     __shared__ int s_last, s_fail, s_aligned;
+    __shared__ __align__(16) unsigned char q8[sizeof(K1T) == 1 ? 8 * kQ8Stride : 16];   // FP8 tensor-core pass 1: query terms
+    __shared__ float qsc[8];                                                             //   and their scales, per column
     __shared__ int segblk[AL ? kMaxAlignedSegs + 1 : 1];   // first block of every segment (aligned cut)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -105,6 +124,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     const int G = gridDim.x, cta = blockIdx.x;
     const int nc1 = r / 8, nc2 = d2 / 8, ncv = hd / 8;
     const int pstride = hd + kPartPad;
+    const bool mma8 = sizeof(K1T) == 1 && GQ <= 2 && r == 128;          // FP8 tensor-core pass 1
+    const int mg = lane >> 2, mt = lane & 3;                            // fragment row group and column pair
     const K1T* k1c = static_cast<const K1T*>(p.k1c);
     const KT* k2c = static_cast<const KT*>(p.k2c);
     const KT* vc = static_cast<const KT*>(p.vc);
@@ -124,6 +145,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     }
     // ---- flat layout: prefix sums of the window lengths over the segments -------------------------
     if (tid == 32) s_fail = 0;
+    if constexpr (sizeof(K1T) == 1)
+        for (int i = tid; i < 8 * kQ8Stride / 4; i += kThreads) reinterpret_cast<unsigned*>(q8)[i] = 0u;
     if (warp == 0) {
         int run = 0;
         for (int s0 = 0; s0 < NS; s0 += 32) {
@@ -235,7 +258,18 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const K1T* kbase = k1c + (static_cast<int64_t>(seg0) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
-            if (w0 < w1) {
+            if (w0 < w1 && mma8) {          // rows w0 + mg and w0 + mg + 8, pieces 4 c + mt of their four 32-column chunks
+#pragma unroll
+                for (int hrow = 0; hrow < 2; ++hrow) {
+                    const int t = w0 + mg + 8 * hrow;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        if (t < w1) wpre[4 * hrow + c].load(kbase + static_cast<int64_t>(t) * r, 4 * c + mt);
+                        else wpre[4 * hrow + c].zero();
+                    }
+                }
+                have_pre = true;
+            } else if (w0 < w1) {
                 const int tok0 = w0 + half * 8;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -279,6 +313,37 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 zcache[ord] = p.k_attn >= L ? 0.0
                               : (p.zs != nullptr ? p.zs[b] : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
             __syncthreads();
+            if constexpr (sizeof(K1T) == 1) {
+                if (mma8) {
+                    // The query as four e4m3 terms per head: term i holds what the terms before it left, at a scale 16
+                    // times finer (an e4m3 value carries four significant bits).  A warp per head, four values per lane.
+                    if (warp < GQ) {
+                        float v[4], amax = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            v[e] = qs[warp * hd + lane * 4 + e];
+                            amax = fmaxf(amax, fabsf(v[e]));
+                        }
+                        amax = warp_max(amax);
+                        float scale = amax > 0.f ? amax * (1.f / 448.f) : 1.f;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float inv = 1.f / scale;
+                            unsigned packed = 0u;
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const unsigned char code = to_e4m3(v[e] * inv);
+                                v[e] -= scale * from_e4m3(code);
+                                packed |= static_cast<unsigned>(code) << (8 * e);
+                            }
+                            *reinterpret_cast<unsigned*>(q8 + (4 * warp + i) * kQ8Stride + lane * 4) = packed;
+                            if (lane == 0) qsc[4 * warp + i] = scale;
+                            scale *= 0.0625f;
+                        }
+                    }
+                    __syncthreads();
+                }
+            }
             float qreg[GQ][8];
 #pragma unroll
             for (int hq = 0; hq < GQ; ++hq)
@@ -292,6 +357,71 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             int w0, w1;
             warp_range(tb, te, w0, w1);
             const int jidx = ((hl >> 3) & 1) * 4 + ((hl >> 2) & 1) * 2 + ((hl >> 1) & 1);
+            if (mma8) {
+                const int myh = mt >> 1;                                  // the head whose terms this lane's two columns hold
+                const bool owner = (mt & 1) == 0 && myh < GQ;              // ... and the lane that ends up with its scores
+                const float c0 = qsc[2 * mt], c1 = qsc[2 * mt + 1];
+                double t1 = 0.0, t2 = 0.0;
+                float tm = -INFINITY;
+#pragma unroll 1
+                for (int base = w0; base < w1; base += 32) {               // two 16-row tiles per trip: 16 loads in flight per lane
+                    Row8<K1T> w[2][8];
+                    float rs[2][2];
+#pragma unroll
+                    for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+                        for (int hrow = 0; hrow < 2; ++hrow) {
+                            const int t = base + 16 * nb + mg + 8 * hrow;
+                            rs[nb][hrow] = (owner && t < w1) ? p.k1s[static_cast<int64_t>(seg) * p.cap + lo + t] : 0.f;
+                            if (nb == 0 && have_pre && ord == 0 && base == w0) {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) w[0][4 * hrow + c] = wpre[4 * hrow + c];
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) {
+                                    if (t < w1) w[nb][4 * hrow + c].load(kbase + static_cast<int64_t>(t) * r, 4 * c + mt);
+                                    else w[nb][4 * hrow + c].zero();
+                                }
+                            }
+                        }
+#pragma unroll
+                    for (int nb = 0; nb < 2; ++nb) {
+                        float dd[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const uint2 qb = *reinterpret_cast<const uint2*>(q8 + mg * kQ8Stride + 32 * c + 8 * mt);
+                            const uint2 a_lo = raw8_of(w[nb][c]), a_hi = raw8_of(w[nb][4 + c]);
+                            mma_e4m3_16832(dd, a_lo.x, a_hi.x, a_lo.y, a_hi.y, qb.x, qb.y);
+                        }
+                        float sa = c0 * dd[0] + c1 * dd[1], sb2 = c0 * dd[2] + c1 * dd[3];
+                        sa += __shfl_xor_sync(kFull, sa, 1);
+                        sb2 += __shfl_xor_sync(kFull, sb2, 1);
+                        if (owner) {
+                            const int ta = base + 16 * nb + mg, tb2 = ta + 8;
+                            if (ta < w1) {
+                                const float v32 = sa * rs[nb][0];
+                                sc[static_cast<size_t>(myh) * ntok + off + ta] = v32;
+                                const double v = static_cast<double>(v32);
+                                t1 += v; t2 = fma(v, v, t2); tm = fmaxf(tm, v32);
+                            }
+                            if (tb2 < w1) {
+                                const float v32 = sb2 * rs[nb][1];
+                                sc[static_cast<size_t>(myh) * ntok + off + tb2] = v32;
+                                const double v = static_cast<double>(v32);
+                                t1 += v; t2 = fma(v, v, t2); tm = fmaxf(tm, v32);
+                            }
+                        }
+                    }
+                }
+                // sums over the eight row groups (lane bits 2..4); lanes with mg == 0 hold a head's totals
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) {
+                    t1 += __shfl_xor_sync(kFull, t1, o);
+                    t2 += __shfl_xor_sync(kFull, t2, o);
+                    tm = fmaxf(tm, __shfl_xor_sync(kFull, tm, o));
+                }
+                if (owner && mg == 0) { red[warp][myh][0] = t1; red[warp][myh][1] = t2; redm[warp][myh] = tm; }
+            } else {
 #pragma unroll 1
             for (int base = w0; base < w1; base += 16) {
                 const int tok0 = base + half * 8;
@@ -364,6 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 const double a = warp_sum_f64(s1[hq]), c = warp_sum_f64(s2[hq]);
                 const float m = warp_max(mx[hq]);
                 if (lane == 0) { red[warp][hq][0] = a; red[warp][hq][1] = c; redm[warp][hq] = m; }
+            }
             }
             __syncthreads();
             if (warp < GQ) {
