@@ -246,6 +246,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     // query is staged and, when the lengths are known to be stable, before the kernel ahead of this one
     // has finished (its newest cache row is held back until it has).
     Row8<K1T> wpre[8];
+    [[maybe_unused]] uint4 wq[sizeof(K1T) == 1 ? 4 : 1];      // FP8 tensor-core pass: the first tile's rows, 16-byte pieces
     bool have_pre = false;
     {
         int held = -1;
@@ -258,15 +259,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const K1T* kbase = k1c + (static_cast<int64_t>(seg0) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
-            if (w0 < w1 && mma8) {          // rows w0 + mg and w0 + mg + 8, pieces 4 c + mt of their four 32-column chunks
+            if (w0 < w1 && mma8) {          // rows w0 + mg and w0 + mg + 8, their 16-byte pieces mt and mt + 4
 #pragma unroll
                 for (int hrow = 0; hrow < 2; ++hrow) {
                     const int t = w0 + mg + 8 * hrow;
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (t < w1) wpre[4 * hrow + c].load(kbase + static_cast<int64_t>(t) * r, 4 * c + mt);
-                        else wpre[4 * hrow + c].zero();
-                    }
+                    for (int j = 0; j < 2; ++j)
+                        wq[2 * hrow + j] = t < w1 ? ld_stream16(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(t) * r) + mt + 4 * j)
+                                                  : make_uint4(0u, 0u, 0u, 0u);
                 }
                 have_pre = true;
             } else if (w0 < w1) {
@@ -364,8 +364,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 double t1 = 0.0, t2 = 0.0;
                 float tm = -INFINITY;
 #pragma unroll 1
-                for (int base = w0; base < w1; base += 32) {               // two 16-row tiles per trip: 16 loads in flight per lane
-                    Row8<K1T> w[2][8];
+                for (int base = w0; base < w1; base += 32) {               // two 16-row tiles per trip: eight 16-byte loads in flight per lane
+                    // A lane takes the 16-byte pieces mt and mt + 4 of rows mg and mg + 8: the k-slots of an MMA may be any
+                    // permutation of the columns as long as both operands use it, so a piece feeds two MMAs (its two halves).
+                    uint4 w[2][4];
                     float rs[2][2];
 #pragma unroll
                     for (int nb = 0; nb < 2; ++nb)
@@ -373,25 +375,22 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                         for (int hrow = 0; hrow < 2; ++hrow) {
                             const int t = base + 16 * nb + mg + 8 * hrow;
                             rs[nb][hrow] = (owner && t < w1) ? p.k1s[static_cast<int64_t>(seg) * p.cap + lo + t] : 0.f;
-                            if (nb == 0 && have_pre && ord == 0 && base == w0) {
 #pragma unroll
-                                for (int c = 0; c < 4; ++c) w[0][4 * hrow + c] = wpre[4 * hrow + c];
-                            } else {
-#pragma unroll
-                                for (int c = 0; c < 4; ++c) {
-                                    if (t < w1) w[nb][4 * hrow + c].load(kbase + static_cast<int64_t>(t) * r, 4 * c + mt);
-                                    else w[nb][4 * hrow + c].zero();
-                                }
+                            for (int j = 0; j < 2; ++j) {
+                                if (nb == 0 && have_pre && ord == 0 && base == w0) w[0][2 * hrow + j] = wq[2 * hrow + j];
+                                else w[nb][2 * hrow + j] = t < w1 ? ld_stream16(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(t) * r) + mt + 4 * j)
+                                                                  : make_uint4(0u, 0u, 0u, 0u);
                             }
                         }
 #pragma unroll
                     for (int nb = 0; nb < 2; ++nb) {
                         float dd[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const uint2 qb = *reinterpret_cast<const uint2*>(q8 + mg * kQ8Stride + 32 * c + 8 * mt);
-                            const uint2 a_lo = raw8_of(w[nb][c]), a_hi = raw8_of(w[nb][4 + c]);
+                        for (int j = 0; j < 2; ++j) {
+                            const uint4 qb = *reinterpret_cast<const uint4*>(q8 + mg * kQ8Stride + 16 * (mt + 4 * j));
+                            const uint4 a_lo = w[nb][j], a_hi = w[nb][2 + j];
                             mma_e4m3_16832(dd, a_lo.x, a_hi.x, a_lo.y, a_hi.y, qb.x, qb.y);
+                            mma_e4m3_16832(dd, a_lo.z, a_hi.z, a_lo.w, a_hi.w, qb.z, qb.w);
                         }
                         float sa = c0 * dd[0] + c1 * dd[1], sb2 = c0 * dd[2] + c1 * dd[3];
                         sa += __shfl_xor_sync(kFull, sa, 1);

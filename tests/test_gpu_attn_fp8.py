@@ -45,7 +45,9 @@ def run(ctx, a, k_attn, window=0, flags=0):
     (1, 8, 4, 256, 128, 4096, [4096], 256, 0),
     (3, 8, 4, 256, 128, 2048, [2048, 700, 33], 256, 512),
     (8, 16, 8, 256, 128, 1024, [1024, 1000, 900, 512, 300, 100, 17, 1], 64, 0),       # aligned cut
-    (2, 4, 4, 64, 32, 300, [300, 150], 16, 0),
+    (2, 4, 4, 64, 32, 300, [300, 150], 16, 0),                                          # r = 32: plain-ALU first pass
+    (1, 4, 4, 256, 128, 700, [650], 64, 0),                                             # one query head per KV head
+    (2, 16, 4, 256, 128, 500, [500, 77], 32, 128),                                      # four per KV head: plain-ALU first pass
 ])
 def test_fp8_predictor_slice_against_oracle(ctx, B, n_q, n_kv, hd, r, cap, lens, k_attn, window):
     a = synth.attn_inputs(B, n_q, n_kv, hd, r, cap, lens, "bf16", seed=13)
