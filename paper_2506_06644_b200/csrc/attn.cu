@@ -44,9 +44,6 @@ __device__ __forceinline__ void mma_e4m3_16832(float (&d)[4], unsigned a0, unsig
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint2 raw8_of(const Row8<__nv_fp8_e4m3>& w) { return w.raw; }
-template <typename T>
-__device__ __forceinline__ uint2 raw8_of(const Row8<T>&) { return make_uint2(0u, 0u); }          // never used: other storage types
 __device__ __forceinline__ unsigned char to_e4m3(float x) { return static_cast<unsigned char>(__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3)); }
 __device__ __forceinline__ float from_e4m3(unsigned char b) { return __half2float(__half(__nv_cvt_fp8_to_halfraw(b, __NV_E4M3))); }
 

@@ -11,6 +11,8 @@
 //            u_i = GELU(s_i - theta) t_i, then a thread per 8 output columns accumulates
 //            sum_i u_i V[:,i] in registers and adds it to y with vector reductions.
 // Individual masks gate the arithmetic, the union gates the loads (Appendix B).
+#include <cstdlib>
+
 #include "ffn_params.h"
 #include "kernels.h"
 #include "rowdot.cuh"
@@ -390,6 +392,11 @@ int launch_tb(spark_ctx* ctx, FfnParams& p, int tb, size_t smem, cudaStream_t st
 
 namespace spark {
 
+static int tc_min_tokens() {
+    static const int v = []() { const char* e = getenv("SPARK_TC_MIN"); return e ? atoi(e) : 17; }();
+    return v;
+}
+
 int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     if (ctx == nullptr || a.x == nullptr || a.K1t == nullptr || a.K2t == nullptr || a.Vt == nullptr || a.y == nullptr)
         return SPARK_ERR_INVALID_ARG;
@@ -434,6 +441,10 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     if (a.B == 1 && grid <= 512 && a.d <= 4096) return ffn1_launch(ctx, p, a.wdtype, stream);
     if (a.B >= 2 && a.B <= 4 && grid <= 512) {
         const int rc = ffn_few_launch(ctx, p, a.wdtype, stream);
+        if (rc != SPARK_ERR_WORKSPACE) return rc;
+    }
+    if (a.B >= tc_min_tokens() && a.B <= 64 && a.wdtype == SPARK_BF16) {      // reads every row: SPARK_DENSE_LOADS changes nothing here
+        const int rc = ffn_tc_launch(ctx, p, stream);
         if (rc != SPARK_ERR_WORKSPACE) return rc;
     }
     if (a.B >= 2 && a.wdtype == SPARK_BF16) {

@@ -39,6 +39,11 @@ struct FfnParams {
 // served, use the plain-ALU kernel.
 int ffn_mma_launch(spark_ctx* ctx, FfnParams& p, cudaStream_t stream);
 
+// Chunks of up to 64 tokens on tcgen05 tensor cores, every weight row read (ffn_tc.cu); SPARK_ERR_WORKSPACE =
+// shape or workspace not served.
+int ffn_tc_launch(spark_ctx* ctx, FfnParams& p, cudaStream_t stream);
+size_t ffn_tc_workspace_bytes(int64_t d, int64_t d_ff);
+
 // 2..4 tokens without tensor cores (ffn_few.cu); SPARK_ERR_WORKSPACE = shape not served.
 int ffn_few_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream);
 

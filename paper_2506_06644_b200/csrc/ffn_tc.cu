@@ -1,0 +1,693 @@
+// Spark FFN (Section 2.1, Eq. 2) for a chunk of 5..64 tokens with bf16 weights, on the fifth-generation
+// tensor cores.  With this many tokens the union of the tokens' active sets (Appendix B) covers most
+// neurons, every weight row is read anyway, and the three products are real GEMMs with the tokens as
+// the N dimension.  Four kernels, ordered by the stream (no block waits on another block):
+//   prep    RMSNorm scale (optional), x -> two bf16 terms (x = hi + lo), y = y_init, sums cleared
+//   scores  S^T = K1t . X[:, :r]^T and T^T = K2t . X[:, r:]^T: TMA-fed tcgen05.mma, M = 128 neurons,
+//           N = tokens, accumulators in tensor memory; two blocks per 128 neurons split the K range;
+//           per-token score sums for Eq. 11 leave with the epilogue
+//   act     theta per token (Eq. 10/11), U = [S > theta] . GELU(S - theta) . T as two bf16 terms,
+//           counts and index lists
+//   out     Y^T += Vt^T . U: M = 128 model columns (Vt enters MN-major, as it is stored), N = tokens,
+//           K = neurons split over blocks, fp32 vector reductions into y
+// The fp32 activations enter every product as an error-compensated two-term bf16 split (one MMA per
+// term): the scores decide index sets, so a bare bf16 rounding (2^-9) is not enough, and the two
+// terms carry 16 mantissa bits.  The weight streams are requested before the kernel waits for the
+// one ahead of it, so they overlap its tail.
+#include <cuda.h>      // CUtensorMap and its enums; the encoder itself is looked up through the runtime
+
+#include "ffn_params.h"
+#include "kernels.h"
+
+using namespace spark;
+
+namespace {
+
+constexpr int kTok = 64;              // token rows of the padded operands
+constexpr int kChunk = 64;            // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int kTcThreads = 192;       // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
+constexpr int kSumWays = 16;
+constexpr long long kTcSpinLimit = 2000000000ll;
+
+// ---- layout of the chunk path's part of the workspace ----------------------------------------------
+struct TcRegion {
+    double* sums;                 // [kSumWays][kTok][2]
+    __nv_bfloat16* xhi;           // [kTok][d]
+    __nv_bfloat16* xlo;
+    float* S;                     // [kTok][d_ff] scores, token-major
+    float* T0;                    // [kTok][d_ff] K2 products, first K half
+    float* T1;                    // second K half
+    __nv_bfloat16* uhi;           // [kTok][d_ff]
+    __nv_bfloat16* ulo;
+};
+inline size_t tc_region_bytes(int64_t d, int64_t d_ff) {
+    return round_up(sizeof(double) * kSumWays * kTok * 2, 1024) + 2 * round_up(static_cast<size_t>(kTok) * d * 2, 1024) +
+           3 * round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024) + 2 * round_up(static_cast<size_t>(kTok) * d_ff * 2, 1024);
+}
+inline TcRegion tc_region(char* base, int64_t d, int64_t d_ff) {
+    TcRegion g;
+    char* p = base;
+    g.sums = reinterpret_cast<double*>(p); p += round_up(sizeof(double) * kSumWays * kTok * 2, 1024);
+    g.xhi = reinterpret_cast<__nv_bfloat16*>(p); p += round_up(static_cast<size_t>(kTok) * d * 2, 1024);
+    g.xlo = reinterpret_cast<__nv_bfloat16*>(p); p += round_up(static_cast<size_t>(kTok) * d * 2, 1024);
+    g.S = reinterpret_cast<float*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
+    g.T0 = reinterpret_cast<float*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
+    g.T1 = reinterpret_cast<float*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
+    g.uhi = reinterpret_cast<__nv_bfloat16*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 2, 1024);
+    g.ulo = reinterpret_cast<__nv_bfloat16*>(p);
+    return g;
+}
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after about a second, or as soon as another role of the block has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity)) {
+        if (*abort_flag != 0) return false;
+        if (clock64() - t0 > kTcSpinLimit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {      // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_free(uint32_t taddr, uint32_t cols) {           // whole warp
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] . B[smem], bf16 operands, fp32 accumulation; one thread issues.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's tensor-memory lane (warp w reads lanes 32 (w % 4) ..).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                   "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+                   "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+                   "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory operand descriptor, 128-byte swizzle (the layout a TMA box with 128-byte rows and
+// CU_TENSOR_MAP_SWIZZLE_128B leaves): start address, leading and stride byte offsets in 16-byte
+// units, descriptor version 1 in bits 46..47, layout type 2 in bits 61..63.
+//   K-major operand (rows of 64 K-elements): groups of 8 rows are `sbo` bytes apart; lbo unused.
+//   MN-major operand (rows = K, 64 MN-elements per row): groups of 8 K-rows are `sbo` bytes apart,
+//   the next 64 MN-elements `lbo` bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (static_cast<uint64_t>((lbo >> 4) & 0x3fffu) << 16) |
+           (static_cast<uint64_t>((sbo >> 4) & 0x3fffu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator (bits 4..5 = 1), bf16 A and B (bits 7..9 and
+// 10..12 = 1), A MN-major (bit 15), N / 8 in bits 17..22, M / 16 in bits 24..28.
+__host__ __device__ constexpr uint32_t instr_desc(int m, int n, bool a_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+__device__ __forceinline__ unsigned pack2_bf16(float lo, float hi) {
+    unsigned r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+struct TcParams {
+    FfnParams f;
+    TcRegion g;
+    int ntok;            // MMA N: B rounded up to a multiple of 16
+    int cs;              // K chunks of the predictor (r / 64)
+    int call;            // K chunks of both products (d / 64)
+    int chalf;           // chunks of the first block of a pair
+    int ksplit;          // out kernel: blocks per column block
+};
+
+// ---- prep: one block per (padded) token --------------------------------------------------------------
+__global__ void __launch_bounds__(256) ffn_tc_prep_kernel(const TcParams p) {
+    __shared__ float red[8];
+    const int n = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d = p.f.d;
+    dep_wait();
+    dep_trigger();
+    if (n == 0) {
+        for (int i = tid; i < kSumWays * kTok * 2; i += 256) p.g.sums[i] = 0.0;
+        if (p.f.count != nullptr && tid < p.f.B) p.f.count[tid] = 0;
+    }
+    __nv_bfloat16* hi = p.g.xhi + static_cast<int64_t>(n) * d;
+    __nv_bfloat16* lo = p.g.xlo + static_cast<int64_t>(n) * d;
+    if (n >= p.f.B) {              // padding rows of the operands
+        for (int i = tid; i < d / 8; i += 256) {
+            reinterpret_cast<uint4*>(hi)[i] = make_uint4(0u, 0u, 0u, 0u);
+            reinterpret_cast<uint4*>(lo)[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        return;
+    }
+    const float4* xr = reinterpret_cast<const float4*>(p.f.x + static_cast<int64_t>(n) * d);
+    float sc = 1.f;
+    if (p.f.norm_w != nullptr) {
+        float ss = 0.f;
+        for (int i = tid; i < d / 4; i += 256) {
+            const float4 v = xr[i];
+            ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) red[warp] = ss;
+        __syncthreads();
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot += red[w];
+        sc = rsqrtf(tot / static_cast<float>(d) + p.f.eps);
+    }
+    const float4* yi = p.f.y_init ? reinterpret_cast<const float4*>(p.f.y_init + static_cast<int64_t>(n) * d) : nullptr;
+    float4* yo = reinterpret_cast<float4*>(p.f.y + static_cast<int64_t>(n) * d);
+    for (int i = tid; i < d / 4; i += 256) {
+        float4 v = xr[i];
+        if (p.f.norm_w != nullptr) {
+            const float4 w = reinterpret_cast<const float4*>(p.f.norm_w)[i];
+            v = make_float4(v.x * sc * w.x, v.y * sc * w.y, v.z * sc * w.z, v.w * sc * w.w);
+        }
+        const unsigned h01 = pack2_bf16(v.x, v.y), h23 = pack2_bf16(v.z, v.w);
+        const unsigned l01 = pack2_bf16(v.x - __uint_as_float(h01 << 16), v.y - __uint_as_float(h01 & 0xffff0000u));
+        const unsigned l23 = pack2_bf16(v.z - __uint_as_float(h23 << 16), v.w - __uint_as_float(h23 & 0xffff0000u));
+        reinterpret_cast<uint2*>(hi)[i] = make_uint2(h01, h23);
+        reinterpret_cast<uint2*>(lo)[i] = make_uint2(l01, l23);
+        yo[i] = yi ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+
+// ---- block-level pieces shared by the two tensor-core kernels ------------------------------------------
+struct TcShared {
+    unsigned long long full[8];     // stage filled (TMA transaction bytes)
+    unsigned long long empty[8];    // stage drained (tcgen05.commit)
+    unsigned long long accum;       // accumulators final
+    uint32_t tmem;                  // tensor-memory base address written by tcgen05.alloc
+    int abort_flag;                 // a bounded wait of some role ran out
+    double colsum[4][kTok][2];
+};
+
+template <int STAGES>
+__device__ __forceinline__ uint32_t tc_setup(TcShared& sh, unsigned char* raw, uint32_t tmem_cols) {
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_addr(&sh.full[s]), 1u);
+            mbar_init(smem_addr(&sh.empty[s]), 1u);
+        }
+        mbar_init(smem_addr(&sh.accum), 1u);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_addr(&sh.tmem), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    return (smem_addr(raw) + 1023u) & ~1023u;         // operand tiles need 1024-byte alignment (swizzle atom)
+}
+
+// After a wait ran out: the producer thread gives its copies in flight a bounded time to land, so
+// that none writes into the shared memory of a block that has gone.
+template <int STAGES>
+__device__ __forceinline__ void tc_drain(TcShared& sh, int issued) {
+    for (int i = max(0, issued - STAGES); i < issued; ++i) {
+        const uint32_t bar = smem_addr(&sh.full[i % STAGES]), parity = static_cast<uint32_t>(i / STAGES) & 1u;
+        const long long t0 = clock64();
+        while (!mbar_try(bar, parity))
+            if (clock64() - t0 > kTcSpinLimit) break;
+    }
+}
+
+__device__ __forceinline__ void tc_finish(TcShared& sh, uint32_t tmem_cols, WsHeader* hdr) {
+    tc_fence_before();
+    __syncthreads();
+    if ((threadIdx.x >> 5) == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_free(sh.tmem, tmem_cols);
+    }
+    if (threadIdx.x == 0 && sh.abort_flag != 0) atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+}
+
+// ---- scores: S^T and T^T tiles of 128 neurons, two blocks per tile splitting the K range ---------------------
+constexpr int kScoreStages = 6;
+constexpr int kScoreStageBytes = 128 * kChunk * 2 + 2 * kTok * kChunk * 2;      // weights 16 KB, x hi 8 KB, x lo 8 KB
+constexpr uint32_t kScoreCols = 128;                                            // tensor-memory columns: S at 0, T at 64
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k1, const __grid_constant__ CUtensorMap map_k2,
+                     const __grid_constant__ CUtensorMap map_xhi, const __grid_constant__ CUtensorMap map_xlo) {
+    extern __shared__ unsigned char tc_raw[];
+    __shared__ TcShared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tile = blockIdx.x >> 1, half = blockIdx.x & 1;
+    const int c0 = half == 0 ? 0 : p.chalf, c1 = half == 0 ? p.chalf : p.call, nch = c1 - c0;
+    const int row0 = tile * 128;
+    const uint32_t base = tc_setup<kScoreStages>(sh, tc_raw, kScoreCols);
+    const uint32_t tmem = sh.tmem;
+    volatile int* abort_flag = &sh.abort_flag;
+    dep_trigger();          // the kernel behind (act) holds next to nothing while it waits for this one
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&map_k1);
+            tma_prefetch_desc(&map_k2);
+            tma_prefetch_desc(&map_xhi);
+            tma_prefetch_desc(&map_xlo);
+            auto load_w = [&](int i) {
+                const int c = c0 + i, s = i % kScoreStages;
+                const uint32_t bar = smem_addr(&sh.full[s]);
+                mbar_expect_tx(bar, kScoreStageBytes);
+                if (c < p.cs) tma_load_2d(base + s * kScoreStageBytes, &map_k1, bar, c * kChunk, row0);
+                else tma_load_2d(base + s * kScoreStageBytes, &map_k2, bar, (c - p.cs) * kChunk, row0);
+            };
+            auto load_x = [&](int i) {
+                const int c = c0 + i, s = i % kScoreStages;
+                const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kScoreStageBytes + 128 * kChunk * 2;
+                tma_load_2d(dst, &map_xhi, bar, c * kChunk, 0);
+                tma_load_2d(dst + kTok * kChunk * 2, &map_xlo, bar, c * kChunk, 0);
+            };
+            const int pre = min(nch, kScoreStages);
+            for (int i = 0; i < pre; ++i) load_w(i);      // the weights do not depend on the kernel ahead
+            dep_wait();
+            for (int i = 0; i < pre; ++i) load_x(i);
+            int issued = pre;
+            for (int i = pre; i < nch; ++i) {
+                if (!mbar_wait(smem_addr(&sh.empty[i % kScoreStages]), ((i / kScoreStages) & 1) ^ 1, abort_flag)) break;
+                load_w(i);
+                load_x(i);
+                issued = i + 1;
+            }
+            if (*abort_flag != 0) tc_drain<kScoreStages>(sh, issued);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(128, p.ntok, false);
+            bool ok = true;
+            for (int i = 0; i < nch && ok; ++i) {
+                const int s = i % kScoreStages, c = c0 + i;
+                ok = mbar_wait(smem_addr(&sh.full[s]), (i / kScoreStages) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a0 = base + s * kScoreStageBytes, bh = a0 + 128 * kChunk * 2, bl = bh + kTok * kChunk * 2;
+                const uint32_t dcol = tmem + (c < p.cs ? 0u : 64u);
+                const bool fresh = i == 0 || c == p.cs;             // first chunk of this accumulator in this block
+#pragma unroll
+                for (int j = 0; j < kChunk / 16; ++j) {
+                    const uint64_t ad = smem_desc(a0 + 32 * j, 0u, 1024u);
+                    umma_bf16(dcol, ad, smem_desc(bh + 32 * j, 0u, 1024u), idesc, (fresh && j == 0) ? 0u : 1u);
+                    umma_bf16(dcol, ad, smem_desc(bl + 32 * j, 0u, 1024u), idesc, 1u);
+                }
+                umma_commit(smem_addr(&sh.empty[s]));
+            }
+            if (ok) umma_commit(smem_addr(&sh.accum));
+        }
+    } else {
+        const int q = warp & 3;                                    // tensor-memory lanes 32 q .. 32 q + 31
+        const int row = row0 + q * 32 + lane, B = p.f.B;
+        const int64_t dff = p.f.d_ff;
+        dep_wait();
+        const bool ok = __all_sync(kFull, mbar_wait(smem_addr(&sh.accum), 0u, abort_flag));   // warp-uniform: tcgen05.ld is warp-wide
+        const bool has_t0 = p.chalf > p.cs;                        // else the first block of the pair has no K2 chunk
+        if (ok) {
+            tc_fence_after();
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16);
+            float v[32];
+            if (half == 0) {
+                // the stages are idle now: a 32 x 33 transposition window per warp for the per-token sums
+                float* win = reinterpret_cast<float*>(tc_raw + (base - smem_addr(tc_raw))) + (warp - 2) * (32 * 33);
+                for (int hb = 0; hb * 32 < B; ++hb) {
+                    tmem_ld32(taddr + hb * 32, v);
+#pragma unroll
+                    for (int n = 0; n < 32; ++n) {
+                        if (hb * 32 + n < B) p.g.S[(hb * 32 + n) * dff + row] = v[n];
+                        win[n * 33 + lane] = v[n];
+                    }
+                    __syncwarp();
+                    double s1 = 0.0, s2 = 0.0;
+#pragma unroll 8
+                    for (int i = 0; i < 32; ++i) {
+                        const double x = static_cast<double>(win[lane * 33 + i]);
+                        s1 += x;
+                        s2 = fma(x, x, s2);
+                    }
+                    sh.colsum[q][hb * 32 + lane][0] = s1;
+                    sh.colsum[q][hb * 32 + lane][1] = s2;
+                    __syncwarp();
+                }
+                for (int hb = 0; hb * 32 < B; ++hb) {
+                    if (has_t0) tmem_ld32(taddr + 64 + hb * 32, v);
+#pragma unroll
+                    for (int n = 0; n < 32; ++n)
+                        if (hb * 32 + n < B) p.g.T0[(hb * 32 + n) * dff + row] = has_t0 ? v[n] : 0.f;
+                }
+            } else {
+                for (int hb = 0; hb * 32 < B; ++hb) {
+                    tmem_ld32(taddr + 64 + hb * 32, v);
+#pragma unroll
+                    for (int n = 0; n < 32; ++n)
+                        if (hb * 32 + n < B) p.g.T1[(hb * 32 + n) * dff + row] = v[n];
+                }
+            }
+        }
+        if (half == 0) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");               // the four epilogue warps
+            const int n = tid - 64;
+            if (ok && n < B) {
+                double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    s1 += sh.colsum[w][n][0];
+                    s2 += sh.colsum[w][n][1];
+                }
+                double* cell = p.g.sums + (static_cast<size_t>(tile % kSumWays) * kTok + n) * 2;
+                red_add_f64(cell, s1);
+                red_add_f64(cell + 1, s2);
+            }
+        }
+    }
+    tc_finish(sh, kScoreCols, p.f.hdr);
+}
+
+// ---- act: theta, masks, U = [S > theta] . GELU(S - theta) . T in two bf16 terms -----------------------------
+constexpr int kActThreads = 512;
+constexpr int kActSpan = kActThreads * 8;        // neurons per block, eight per thread
+
+__global__ void __launch_bounds__(kActThreads) ffn_tc_act_kernel(const TcParams p, int blocks_per_token) {
+    __shared__ float theta_s;
+    __shared__ int wsum[kActThreads / 32];
+    __shared__ int base_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = blockIdx.x / blocks_per_token, bx = blockIdx.x - n * blocks_per_token;
+    const int64_t dff = p.f.d_ff;
+    dep_trigger();          // the kernel behind (out) starts on its weight stream while this one runs
+    dep_wait();
+    if (warp == 0) {
+        double s1 = 0.0, s2 = 0.0;
+        if (lane < kSumWays) {
+            const double* cell = p.g.sums + (static_cast<size_t>(lane) * kTok + n) * 2;
+            s1 = cell[0];
+            s2 = cell[1];
+        }
+        s1 = warp_sum_f64(s1);
+        s2 = warp_sum_f64(s2);
+        if (lane == 0) {
+            float th = -INFINITY;
+            if (!p.f.identity) {
+                const double mean = s1 * p.f.inv_n;
+                const float var = static_cast<float>((s2 - s1 * mean) * p.f.inv_nm1);
+                th = static_cast<float>(mean) + sqrtf(fmaxf(var, 0.f)) * static_cast<float>(p.f.z);
+            }
+            theta_s = th;
+            if (bx == 0 && p.f.theta != nullptr) p.f.theta[n] = th;
+        }
+    }
+    __syncthreads();
+    const float th = theta_s, shift = p.f.identity ? 0.f : th;
+    const int j0 = bx * kActSpan + tid * 8;
+    unsigned mask = 0u;
+    if (j0 < dff) {
+        const int64_t off = static_cast<int64_t>(n) * dff + j0;
+        float s[8], t[8], t1[8];
+        *reinterpret_cast<float4*>(s) = __ldcg(reinterpret_cast<const float4*>(p.g.S + off));
+        *reinterpret_cast<float4*>(s + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.S + off) + 1);
+        *reinterpret_cast<float4*>(t) = __ldcg(reinterpret_cast<const float4*>(p.g.T0 + off));
+        *reinterpret_cast<float4*>(t + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.T0 + off) + 1);
+        *reinterpret_cast<float4*>(t1) = __ldcg(reinterpret_cast<const float4*>(p.g.T1 + off));
+        *reinterpret_cast<float4*>(t1 + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.T1 + off) + 1);
+        float u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const bool on = s[i] > th;
+            const float a = s[i] - shift;
+            u[i] = on ? (p.f.erf_form ? gelu_erf(a) : gelu_tanh(a)) * (t[i] + t1[i]) : 0.f;
+            mask |= on ? 1u << i : 0u;
+        }
+        unsigned h[4], l[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            h[i] = pack2_bf16(u[2 * i], u[2 * i + 1]);
+            l[i] = pack2_bf16(u[2 * i] - __uint_as_float(h[i] << 16), u[2 * i + 1] - __uint_as_float(h[i] & 0xffff0000u));
+        }
+        *reinterpret_cast<uint4*>(p.g.uhi + off) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4*>(p.g.ulo + off) = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+    if (p.f.count != nullptr) {
+        // the block's share of the token's list is contiguous and ascending; blocks take their places in
+        // the order in which they get here
+        const int c = __popc(mask);
+        int incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(kFull, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        int before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kActThreads / 32; ++w) {
+            if (w < warp) before += wsum[w];
+            total += wsum[w];
+        }
+        if (tid == 0) base_s = total > 0 ? atomicAdd(&p.f.count[n], total) : 0;
+        __syncthreads();
+        if (p.f.idx != nullptr && c > 0) {
+            int32_t* out = p.f.idx + static_cast<int64_t>(n) * dff + base_s + before + incl - c;
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if ((mask >> i) & 1u) *out++ = j0 + i;
+        }
+    }
+}
+
+// ---- out: Y^T[256 columns of the block] += Vt[neurons of the block]^T . U ------------------------------------
+constexpr int kOutStages = 4;
+constexpr int kOutVBytes = 4 * kChunk * 128;                                  // four boxes of 64 neurons x 64 columns
+constexpr int kOutStageBytes = kOutVBytes + 2 * kTok * kChunk * 2;            // + u hi, u lo
+constexpr uint32_t kOutCols = 128;                                            // two accumulators of 128 columns x 64 tokens
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_uhi,
+                  const __grid_constant__ CUtensorMap map_ulo) {
+    extern __shared__ unsigned char tc_raw[];
+    __shared__ TcShared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nb = blockIdx.x / p.ksplit, ks = blockIdx.x - nb * p.ksplit;
+    const int cn = p.f.d_ff / kChunk;
+    const int c0 = static_cast<int>(static_cast<int64_t>(ks) * cn / p.ksplit), c1 = static_cast<int>(static_cast<int64_t>(ks + 1) * cn / p.ksplit);
+    const int nch = c1 - c0, col0 = nb * 256;
+    const uint32_t base = tc_setup<kOutStages>(sh, tc_raw, kOutCols);
+    const uint32_t tmem = sh.tmem;
+    volatile int* abort_flag = &sh.abort_flag;
+    dep_trigger();
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&map_v);
+            tma_prefetch_desc(&map_uhi);
+            tma_prefetch_desc(&map_ulo);
+            auto load_v = [&](int i) {
+                const int s = i % kOutStages;
+                const uint32_t bar = smem_addr(&sh.full[s]);
+                mbar_expect_tx(bar, kOutStageBytes);
+#pragma unroll
+                for (int b = 0; b < 4; ++b) tma_load_2d(base + s * kOutStageBytes + b * (kChunk * 128), &map_v, bar, col0 + 64 * b, (c0 + i) * kChunk);
+            };
+            auto load_u = [&](int i) {
+                const int s = i % kOutStages;
+                const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kOutStageBytes + kOutVBytes;
+                tma_load_2d(dst, &map_uhi, bar, (c0 + i) * kChunk, 0);
+                tma_load_2d(dst + kTok * kChunk * 2, &map_ulo, bar, (c0 + i) * kChunk, 0);
+            };
+            const int pre = min(nch, kOutStages);
+            for (int i = 0; i < pre; ++i) load_v(i);      // the rows of V do not depend on the kernels ahead
+            dep_wait();
+            for (int i = 0; i < pre; ++i) load_u(i);
+            int issued = pre;
+            for (int i = pre; i < nch; ++i) {
+                if (!mbar_wait(smem_addr(&sh.empty[i % kOutStages]), ((i / kOutStages) & 1) ^ 1, abort_flag)) break;
+                load_v(i);
+                load_u(i);
+                issued = i + 1;
+            }
+            if (*abort_flag != 0) tc_drain<kOutStages>(sh, issued);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(128, p.ntok, true);
+            bool ok = true;
+            for (int i = 0; i < nch && ok; ++i) {
+                const int s = i % kOutStages;
+                ok = mbar_wait(smem_addr(&sh.full[s]), (i / kOutStages) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t v0 = base + s * kOutStageBytes, bh = v0 + kOutVBytes, bl = bh + kTok * kChunk * 2;
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+#pragma unroll
+                    for (int j = 0; j < kChunk / 16; ++j) {
+                        // A: 16 neurons (K) x 128 columns (M) of V, MN-major: 8-neuron groups 1024 bytes apart, the
+                        // second 64 columns in the next box (8192 bytes on)
+                        const uint64_t ad = smem_desc(v0 + mt * (2 * kChunk * 128) + j * 2048, kChunk * 128, 1024u);
+                        umma_bf16(tmem + mt * 64, ad, smem_desc(bh + 32 * j, 0u, 1024u), idesc, (i == 0 && j == 0) ? 0u : 1u);
+                        umma_bf16(tmem + mt * 64, ad, smem_desc(bl + 32 * j, 0u, 1024u), idesc, 1u);
+                    }
+                }
+                umma_commit(smem_addr(&sh.empty[s]));
+            }
+            if (ok) umma_commit(smem_addr(&sh.accum));
+        }
+    } else {
+        const int q = warp & 3, B = p.f.B;
+        const int64_t d = p.f.d;
+        dep_wait();
+        if (nch > 0 && __all_sync(kFull, mbar_wait(smem_addr(&sh.accum), 0u, abort_flag))) {
+            tc_fence_after();
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16);
+            float v[32];
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                float* ycol = p.f.y + col0 + mt * 128 + q * 32 + lane;
+                for (int hb = 0; hb * 32 < B; ++hb) {
+                    tmem_ld32(taddr + mt * 64 + hb * 32, v);
+#pragma unroll
+                    for (int n = 0; n < 32; ++n)
+                        if (hb * 32 + n < B) atomicAdd(ycol + (hb * 32 + n) * d, v[n]);
+                }
+            }
+        }
+    }
+    tc_finish(sh, kOutCols, p.f.hdr);
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(sym);
+    }();
+    return fn;
+}
+
+// Row-major bf16 matrix [rows][cols] (row stride ld elements), boxes of 64 columns x box_rows rows, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows, bool streamed) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kChunk), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, streamed ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+namespace spark {
+
+size_t ffn_tc_workspace_bytes(int64_t d, int64_t d_ff) { return tc_region_bytes(d, d_ff); }
+
+// SPARK_ERR_WORKSPACE = shape or workspace not served by this path (the caller falls back).
+int ffn_tc_launch(spark_ctx* ctx, FfnParams& f, cudaStream_t stream) {
+    const int d = f.d, r = f.r, d_ff = f.d_ff, B = f.B;
+    if (B < 1 || B > kTok || d % 256 != 0 || r % kChunk != 0 || r <= 0 || r >= d || d_ff % 128 != 0 || f.K1s != nullptr) return SPARK_ERR_WORKSPACE;
+    const int call = d / kChunk, cs = r / kChunk, chalf = (call + 1) / 2;
+    if (cs > chalf) return SPARK_ERR_WORKSPACE;
+    if (ctx->scratch == nullptr || ctx->scratch_bytes < kAttnCellBytes + tc_region_bytes(d, d_ff)) return SPARK_ERR_WORKSPACE;
+    const size_t smem_scores = static_cast<size_t>(kScoreStages) * kScoreStageBytes + 1024;
+    const size_t smem_out = static_cast<size_t>(kOutStages) * kOutStageBytes + 1024;
+    if (smem_scores + sizeof(TcShared) + 64 > static_cast<size_t>(ctx->max_smem_optin) ||
+        smem_out + sizeof(TcShared) + 64 > static_cast<size_t>(ctx->max_smem_optin))
+        return SPARK_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(f.K1t) | reinterpret_cast<uintptr_t>(f.K2t) | reinterpret_cast<uintptr_t>(f.Vt)) & 15u) return SPARK_ERR_WORKSPACE;
+
+    TcParams p;
+    p.f = f;
+    p.g = tc_region(ctx->scratch + kAttnCellBytes, d, d_ff);       // behind the attention's persistent cells
+    p.ntok = (B + 15) & ~15;
+    p.cs = cs;
+    p.call = call;
+    p.chalf = chalf;
+    const int nbk = d / 256;
+    p.ksplit = ctx->num_sms / nbk > 0 ? ctx->num_sms / nbk : 1;
+    if (p.ksplit > d_ff / kChunk) p.ksplit = d_ff / kChunk;
+
+    CUtensorMap m_k1, m_k2, m_xhi, m_xlo, m_v, m_uhi, m_ulo;
+    if (!make_map(&m_k1, f.K1t, d_ff, r, r, 128, true) || !make_map(&m_k2, f.K2t, d_ff, d - r, d - r, 128, true) ||
+        !make_map(&m_xhi, p.g.xhi, kTok, d, d, kTok, false) || !make_map(&m_xlo, p.g.xlo, kTok, d, d, kTok, false) ||
+        !make_map(&m_v, f.Vt, d_ff, d, d, kChunk, true) || !make_map(&m_uhi, p.g.uhi, kTok, d_ff, d_ff, kTok, false) ||
+        !make_map(&m_ulo, p.g.ulo, kTok, d_ff, d_ff, kTok, false))
+        return SPARK_ERR_WORKSPACE;
+
+    if (cudaFuncSetAttribute(ffn_tc_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_scores)) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_tc_out_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_out)) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    {
+        void* args[] = {&p};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_prep_kernel), kTok, 256, 0, stream, false, args) != cudaSuccess) return SPARK_ERR_CUDA;
+    }
+    {
+        void* args[] = {&p, &m_k1, &m_k2, &m_xhi, &m_xlo};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_scores_kernel), 2 * (d_ff / 128), kTcThreads, smem_scores, stream, false, args) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+    {
+        int bpt = (d_ff + kActSpan - 1) / kActSpan;
+        void* args[] = {&p, &bpt};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_act_kernel), static_cast<unsigned>(bpt * B), kActThreads, 0, stream, false, args) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+    {
+        void* args[] = {&p, &m_v, &m_uhi, &m_ulo};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_out_kernel), static_cast<unsigned>(nbk * p.ksplit), kTcThreads, smem_out, stream, false, args) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+    return SPARK_OK;
+}
+
+}  // namespace spark

@@ -84,6 +84,20 @@ def test_gemma2_2b_shape_bf16(ctx, B):
     np.testing.assert_allclose(again[0], out[0], rtol=0, atol=1e-5 * parity.rms(out[0]))
 
 
+@pytest.mark.parametrize("d,d_ff,r,k,B,form", [(2304, 9216, 1024, 737, 17, "tanh"), (2304, 9216, 1152, 737, 40, "tanh"),
+                                              (2304, 9216, 1024, 737, 64, "erf"), (3584, 14336, 1792, 1147, 24, "tanh"),
+                                              (256, 1024, 128, 82, 33, "tanh"), (512, 2048, 64, 164, 20, "tanh")])
+def test_token_chunks_on_the_tensor_cores(ctx, d, d_ff, r, k, B, form):
+    # 17..64 tokens: TMA-fed tcgen05 kernels that read every weight row (the union of the active sets covers most)
+    p = synth.ffn_inputs(d, d_ff, r, k, B, "bf16", seed=B)
+    w = upload(p)
+    out = run_ffn(ctx, p, weights=w, flags=S.SPARK_GELU_ERF if form == "erf" else S.SPARK_GELU_TANH)
+    assert compare(p, out, form=form) < 5e-3
+    again = run_ffn(ctx, p, weights=w, want_idx=False, flags=S.SPARK_GELU_ERF if form == "erf" else S.SPARK_GELU_TANH)
+    np.testing.assert_allclose(again[0], out[0], rtol=0, atol=1e-5 * parity.rms(out[0]))
+    assert np.array_equal(again[1], out[1])
+
+
 def test_gemma2_9b_shape_bf16(ctx):
     p = synth.ffn_inputs(3584, 14336, 1792, 1147, 2, "bf16", seed=1)
     compare(p, run_ffn(ctx, p))
