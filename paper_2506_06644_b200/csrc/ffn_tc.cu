@@ -27,6 +27,7 @@ constexpr int kTok = 64;              // token rows of the padded operands
 constexpr int kChunk = 64;            // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kTcThreads = 192;       // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
 constexpr int kSumWays = 16;
+constexpr int kMaxTParts = 2;         // blocks that share the K range of the K2 product of one row tile
 constexpr long long kTcSpinLimit = 2000000000ll;
 
 // ---- layout of the chunk path's part of the workspace ----------------------------------------------
@@ -35,14 +36,13 @@ struct TcRegion {
     __nv_bfloat16* xhi;           // [kTok][d]
     __nv_bfloat16* xlo;
     float* S;                     // [kTok][d_ff] scores, token-major
-    float* T0;                    // [kTok][d_ff] K2 products, first K half
-    float* T1;                    // second K half
+    float* T;                     // [kMaxTParts][kTok][d_ff] K2 products, one per K part
     __nv_bfloat16* uhi;           // [kTok][d_ff]
     __nv_bfloat16* ulo;
 };
 inline size_t tc_region_bytes(int64_t d, int64_t d_ff) {
     return round_up(sizeof(double) * kSumWays * kTok * 2, 1024) + 2 * round_up(static_cast<size_t>(kTok) * d * 2, 1024) +
-           3 * round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024) + 2 * round_up(static_cast<size_t>(kTok) * d_ff * 2, 1024);
+           (1 + kMaxTParts) * round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024) + 2 * round_up(static_cast<size_t>(kTok) * d_ff * 2, 1024);
 }
 inline TcRegion tc_region(char* base, int64_t d, int64_t d_ff) {
     TcRegion g;
@@ -51,8 +51,7 @@ inline TcRegion tc_region(char* base, int64_t d, int64_t d_ff) {
     g.xhi = reinterpret_cast<__nv_bfloat16*>(p); p += round_up(static_cast<size_t>(kTok) * d * 2, 1024);
     g.xlo = reinterpret_cast<__nv_bfloat16*>(p); p += round_up(static_cast<size_t>(kTok) * d * 2, 1024);
     g.S = reinterpret_cast<float*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
-    g.T0 = reinterpret_cast<float*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
-    g.T1 = reinterpret_cast<float*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
+    g.T = reinterpret_cast<float*>(p); p += kMaxTParts * round_up(static_cast<size_t>(kTok) * d_ff * 4, 1024);
     g.uhi = reinterpret_cast<__nv_bfloat16*>(p); p += round_up(static_cast<size_t>(kTok) * d_ff * 2, 1024);
     g.ulo = reinterpret_cast<__nv_bfloat16*>(p);
     return g;
@@ -154,33 +153,36 @@ struct TcParams {
     int ntok;            // MMA N: B rounded up to a multiple of 16
     int cs;              // K chunks of the predictor (r / 64)
     int call;            // K chunks of both products (d / 64)
-    int chalf;           // chunks of the first block of a pair
+    int chalf;           // chunks of the first block of a pair (it holds all of the predictor's)
+    int tfirst;          // first partial K2 product that exists (0, or 1 when the first block has none)
     int ksplit;          // out kernel: blocks per column block
 };
 
-// ---- prep: one block per (padded) token --------------------------------------------------------------
+// ---- prep: four blocks per (padded) token row, a quarter of the row each -----------------------------------
+constexpr int kPrepSplit = 4;
 __global__ void __launch_bounds__(256) ffn_tc_prep_kernel(const TcParams p) {
     __shared__ float red[8];
-    const int n = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int d = p.f.d;
+    const int n = blockIdx.x / kPrepSplit, qr = blockIdx.x % kPrepSplit, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d = p.f.d, q4 = d / 4 / kPrepSplit;          // float4 per quarter row (d is a multiple of 256)
     dep_wait();
     dep_trigger();
-    if (n == 0) {
+    if (blockIdx.x == 0) {
         for (int i = tid; i < kSumWays * kTok * 2; i += 256) p.g.sums[i] = 0.0;
         if (p.f.count != nullptr && tid < p.f.B) p.f.count[tid] = 0;
     }
-    __nv_bfloat16* hi = p.g.xhi + static_cast<int64_t>(n) * d;
-    __nv_bfloat16* lo = p.g.xlo + static_cast<int64_t>(n) * d;
+    if (n >= p.ntok) return;       // rows the operand boxes never touch
+    uint2* hi = reinterpret_cast<uint2*>(p.g.xhi + static_cast<int64_t>(n) * d) + qr * q4;
+    uint2* lo = reinterpret_cast<uint2*>(p.g.xlo + static_cast<int64_t>(n) * d) + qr * q4;
     if (n >= p.f.B) {              // padding rows of the operands
-        for (int i = tid; i < d / 8; i += 256) {
-            reinterpret_cast<uint4*>(hi)[i] = make_uint4(0u, 0u, 0u, 0u);
-            reinterpret_cast<uint4*>(lo)[i] = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = tid; i < q4; i += 256) {
+            hi[i] = make_uint2(0u, 0u);
+            lo[i] = make_uint2(0u, 0u);
         }
         return;
     }
     const float4* xr = reinterpret_cast<const float4*>(p.f.x + static_cast<int64_t>(n) * d);
     float sc = 1.f;
-    if (p.f.norm_w != nullptr) {
+    if (p.f.norm_w != nullptr) {   // every quarter sums the whole row (9 KB out of L2)
         float ss = 0.f;
         for (int i = tid; i < d / 4; i += 256) {
             const float4 v = xr[i];
@@ -194,20 +196,17 @@ __global__ void __launch_bounds__(256) ffn_tc_prep_kernel(const TcParams p) {
         for (int w = 0; w < 8; ++w) tot += red[w];
         sc = rsqrtf(tot / static_cast<float>(d) + p.f.eps);
     }
-    const float4* yi = p.f.y_init ? reinterpret_cast<const float4*>(p.f.y_init + static_cast<int64_t>(n) * d) : nullptr;
-    float4* yo = reinterpret_cast<float4*>(p.f.y + static_cast<int64_t>(n) * d);
-    for (int i = tid; i < d / 4; i += 256) {
-        float4 v = xr[i];
+    for (int i = tid; i < q4; i += 256) {
+        float4 v = xr[qr * q4 + i];
         if (p.f.norm_w != nullptr) {
-            const float4 w = reinterpret_cast<const float4*>(p.f.norm_w)[i];
+            const float4 w = reinterpret_cast<const float4*>(p.f.norm_w)[qr * q4 + i];
             v = make_float4(v.x * sc * w.x, v.y * sc * w.y, v.z * sc * w.z, v.w * sc * w.w);
         }
         const unsigned h01 = pack2_bf16(v.x, v.y), h23 = pack2_bf16(v.z, v.w);
         const unsigned l01 = pack2_bf16(v.x - __uint_as_float(h01 << 16), v.y - __uint_as_float(h01 & 0xffff0000u));
         const unsigned l23 = pack2_bf16(v.z - __uint_as_float(h23 << 16), v.w - __uint_as_float(h23 & 0xffff0000u));
-        reinterpret_cast<uint2*>(hi)[i] = make_uint2(h01, h23);
-        reinterpret_cast<uint2*>(lo)[i] = make_uint2(l01, l23);
-        yo[i] = yi ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        hi[i] = make_uint2(h01, h23);
+        lo[i] = make_uint2(l01, l23);
     }
 }
 
@@ -264,10 +263,18 @@ __device__ __forceinline__ void tc_finish(TcShared& sh, uint32_t tmem_cols, WsHe
     if (threadIdx.x == 0 && sh.abort_flag != 0) atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
 }
 
-// ---- scores: S^T and T^T tiles of 128 neurons, two blocks per tile splitting the K range ---------------------
+// ---- scores: S^T and T^T tiles of 128 neurons; the two blocks of a tile split the K range ----------------
+// The first block of a pair takes the predictor's chunks (its scores are complete, so their sums can
+// leave with the epilogue) and the first chunks of the K2 product, the second block the rest; the
+// activation kernel adds the partial products.  Both terms of X sit in one operand tile (hi rows, then
+// lo rows), so one MMA of N = 2 ntok serves both and the weight tile is read from shared memory once;
+// the epilogue adds the two halves of the accumulator.  (Shared-memory bandwidth -- TMA writes plus
+// operand reads -- is what bounds the main loop, not HBM.)
+constexpr int kScoreRows = 128;
 constexpr int kScoreStages = 6;
-constexpr int kScoreStageBytes = 128 * kChunk * 2 + 2 * kTok * kChunk * 2;      // weights 16 KB, x hi 8 KB, x lo 8 KB
-constexpr uint32_t kScoreCols = 128;                                            // tensor-memory columns: S at 0, T at 64
+constexpr int kScoreWBytes = kScoreRows * kChunk * 2;                           // 16 KB of weights per stage
+constexpr int kScoreStageBytes = kScoreWBytes + 2 * kTok * kChunk * 2;          // + x hi, x lo (8 KB each at 64 tokens)
+constexpr uint32_t kScoreCols = 256;                                            // S: columns 0..127 (hi | lo), T: 128..255
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k1, const __grid_constant__ CUtensorMap map_k2,
@@ -275,9 +282,11 @@ ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k
     extern __shared__ unsigned char tc_raw[];
     __shared__ TcShared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int tile = blockIdx.x >> 1, half = blockIdx.x & 1;
-    const int c0 = half == 0 ? 0 : p.chalf, c1 = half == 0 ? p.chalf : p.call, nch = c1 - c0;
-    const int row0 = tile * 128;
+    const int tile = blockIdx.x >> 1, part = blockIdx.x & 1;
+    // chunk range over the combined index (predictor chunks first, then the K2 product's)
+    const int c0 = part == 0 ? 0 : p.chalf, c1 = part == 0 ? p.chalf : p.call, nch = c1 - c0;
+    const int row0 = tile * kScoreRows;
+    const uint32_t xbytes = static_cast<uint32_t>(p.ntok) * kChunk * 2;         // one term of one chunk of X
     const uint32_t base = tc_setup<kScoreStages>(sh, tc_raw, kScoreCols);
     const uint32_t tmem = sh.tmem;
     volatile int* abort_flag = &sh.abort_flag;
@@ -291,16 +300,16 @@ ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k
             tma_prefetch_desc(&map_xlo);
             auto load_w = [&](int i) {
                 const int c = c0 + i, s = i % kScoreStages;
-                const uint32_t bar = smem_addr(&sh.full[s]);
-                mbar_expect_tx(bar, kScoreStageBytes);
-                if (c < p.cs) tma_load_2d(base + s * kScoreStageBytes, &map_k1, bar, c * kChunk, row0);
-                else tma_load_2d(base + s * kScoreStageBytes, &map_k2, bar, (c - p.cs) * kChunk, row0);
+                const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kScoreStageBytes;
+                mbar_expect_tx(bar, kScoreWBytes + 2 * xbytes);
+                if (c < p.cs) tma_load_2d(dst, &map_k1, bar, c * kChunk, row0);
+                else tma_load_2d(dst, &map_k2, bar, (c - p.cs) * kChunk, row0);
             };
             auto load_x = [&](int i) {
                 const int c = c0 + i, s = i % kScoreStages;
-                const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kScoreStageBytes + 128 * kChunk * 2;
+                const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kScoreStageBytes + kScoreWBytes;
                 tma_load_2d(dst, &map_xhi, bar, c * kChunk, 0);
-                tma_load_2d(dst + kTok * kChunk * 2, &map_xlo, bar, c * kChunk, 0);
+                tma_load_2d(dst + xbytes, &map_xlo, bar, c * kChunk, 0);        // lo rows right behind the hi rows
             };
             const int pre = min(nch, kScoreStages);
             for (int i = 0; i < pre; ++i) load_w(i);      // the weights do not depend on the kernel ahead
@@ -317,46 +326,52 @@ ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc(128, p.ntok, false);
+            const uint32_t idesc = instr_desc(128, 2 * p.ntok, false);
             bool ok = true;
             for (int i = 0; i < nch && ok; ++i) {
                 const int s = i % kScoreStages, c = c0 + i;
                 ok = mbar_wait(smem_addr(&sh.full[s]), (i / kScoreStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a0 = base + s * kScoreStageBytes, bh = a0 + 128 * kChunk * 2, bl = bh + kTok * kChunk * 2;
-                const uint32_t dcol = tmem + (c < p.cs ? 0u : 64u);
+                const uint32_t a0 = base + s * kScoreStageBytes, b0 = a0 + kScoreWBytes;
+                const uint32_t dcol = tmem + (c < p.cs ? 0u : 128u);
                 const bool fresh = i == 0 || c == p.cs;             // first chunk of this accumulator in this block
 #pragma unroll
-                for (int j = 0; j < kChunk / 16; ++j) {
-                    const uint64_t ad = smem_desc(a0 + 32 * j, 0u, 1024u);
-                    umma_bf16(dcol, ad, smem_desc(bh + 32 * j, 0u, 1024u), idesc, (fresh && j == 0) ? 0u : 1u);
-                    umma_bf16(dcol, ad, smem_desc(bl + 32 * j, 0u, 1024u), idesc, 1u);
-                }
+                for (int j = 0; j < kChunk / 16; ++j)
+                    umma_bf16(dcol, smem_desc(a0 + 32 * j, 0u, 1024u), smem_desc(b0 + 32 * j, 0u, 1024u), idesc, (fresh && j == 0) ? 0u : 1u);
                 umma_commit(smem_addr(&sh.empty[s]));
             }
             if (ok) umma_commit(smem_addr(&sh.accum));
         }
     } else {
         const int q = warp & 3;                                    // tensor-memory lanes 32 q .. 32 q + 31
-        const int row = row0 + q * 32 + lane, B = p.f.B;
+        const int B = p.f.B, row = row0 + q * 32 + lane;
         const int64_t dff = p.f.d_ff;
         dep_wait();
+        {   // y = y_init (or 0) while the weights stream: the output kernel adds into it
+            const int64_t total4 = static_cast<int64_t>(B) * p.f.d / 4;
+            const float4* yi = reinterpret_cast<const float4*>(p.f.y_init);
+            float4* yo = reinterpret_cast<float4*>(p.f.y);
+            for (int64_t i = static_cast<int64_t>(blockIdx.x) * 128 + (tid - 64); i < total4; i += static_cast<int64_t>(gridDim.x) * 128)
+                yo[i] = yi != nullptr ? yi[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         const bool ok = __all_sync(kFull, mbar_wait(smem_addr(&sh.accum), 0u, abort_flag));   // warp-uniform: tcgen05.ld is warp-wide
-        const bool has_t0 = p.chalf > p.cs;                        // else the first block of the pair has no K2 chunk
+        const bool has_s = c0 < p.cs, has_t = c1 > p.cs;
         if (ok) {
             tc_fence_after();
             const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16);
-            float v[32];
-            if (half == 0) {
+            float v[32], w[32];
+            if (has_s) {
                 // the stages are idle now: a 32 x 33 transposition window per warp for the per-token sums
                 float* win = reinterpret_cast<float*>(tc_raw + (base - smem_addr(tc_raw))) + (warp - 2) * (32 * 33);
                 for (int hb = 0; hb * 32 < B; ++hb) {
                     tmem_ld32(taddr + hb * 32, v);
+                    tmem_ld32(taddr + p.ntok + hb * 32, w);
 #pragma unroll
                     for (int n = 0; n < 32; ++n) {
-                        if (hb * 32 + n < B) p.g.S[(hb * 32 + n) * dff + row] = v[n];
-                        win[n * 33 + lane] = v[n];
+                        const float sv = v[n] + w[n];
+                        if (hb * 32 + n < B) p.g.S[(hb * 32 + n) * dff + row] = sv;
+                        win[n * 33 + lane] = sv;
                     }
                     __syncwarp();
                     double s1 = 0.0, s2 = 0.0;
@@ -370,30 +385,27 @@ ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k
                     sh.colsum[q][hb * 32 + lane][1] = s2;
                     __syncwarp();
                 }
+            }
+            if (has_t) {
+                float* T = p.g.T + static_cast<int64_t>(part) * kTok * dff;
                 for (int hb = 0; hb * 32 < B; ++hb) {
-                    if (has_t0) tmem_ld32(taddr + 64 + hb * 32, v);
+                    tmem_ld32(taddr + 128 + hb * 32, v);
+                    tmem_ld32(taddr + 128 + p.ntok + hb * 32, w);
 #pragma unroll
                     for (int n = 0; n < 32; ++n)
-                        if (hb * 32 + n < B) p.g.T0[(hb * 32 + n) * dff + row] = has_t0 ? v[n] : 0.f;
-                }
-            } else {
-                for (int hb = 0; hb * 32 < B; ++hb) {
-                    tmem_ld32(taddr + 64 + hb * 32, v);
-#pragma unroll
-                    for (int n = 0; n < 32; ++n)
-                        if (hb * 32 + n < B) p.g.T1[(hb * 32 + n) * dff + row] = v[n];
+                        if (hb * 32 + n < B) T[(hb * 32 + n) * dff + row] = v[n] + w[n];
                 }
             }
         }
-        if (half == 0) {
+        if (has_s) {
             asm volatile("bar.sync 1, 128;" ::: "memory");               // the four epilogue warps
             const int n = tid - 64;
             if (ok && n < B) {
                 double s1 = 0.0, s2 = 0.0;
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    s1 += sh.colsum[w][n][0];
-                    s2 += sh.colsum[w][n][1];
+                for (int w4 = 0; w4 < 4; ++w4) {
+                    s1 += sh.colsum[w4][n][0];
+                    s2 += sh.colsum[w4][n][1];
                 }
                 double* cell = p.g.sums + (static_cast<size_t>(tile % kSumWays) * kTok + n) * 2;
                 red_add_f64(cell, s1);
@@ -405,7 +417,7 @@ ffn_tc_scores_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k
 }
 
 // ---- act: theta, masks, U = [S > theta] . GELU(S - theta) . T in two bf16 terms -----------------------------
-constexpr int kActThreads = 512;
+constexpr int kActThreads = 256;
 constexpr int kActSpan = kActThreads * 8;        // neurons per block, eight per thread
 
 __global__ void __launch_bounds__(kActThreads) ffn_tc_act_kernel(const TcParams p, int blocks_per_token) {
@@ -417,6 +429,22 @@ __global__ void __launch_bounds__(kActThreads) ffn_tc_act_kernel(const TcParams 
     const int64_t dff = p.f.d_ff;
     dep_trigger();          // the kernel behind (out) starts on its weight stream while this one runs
     dep_wait();
+    // the block's scores and products are requested before theta is known
+    const int j0 = bx * kActSpan + tid * 8;
+    const int64_t off = static_cast<int64_t>(n) * dff + j0;
+    float s[8], t[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = t[i] = 0.f;
+    if (j0 < dff) {
+        *reinterpret_cast<float4*>(s) = __ldcg(reinterpret_cast<const float4*>(p.g.S + off));
+        *reinterpret_cast<float4*>(s + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.S + off) + 1);
+        for (int tp = p.tfirst; tp < kMaxTParts; ++tp) {
+            const float4* src = reinterpret_cast<const float4*>(p.g.T + static_cast<int64_t>(tp) * kTok * dff + off);
+            const float4 a = __ldcg(src), b = __ldcg(src + 1);
+            t[0] += a.x; t[1] += a.y; t[2] += a.z; t[3] += a.w;
+            t[4] += b.x; t[5] += b.y; t[6] += b.z; t[7] += b.w;
+        }
+    }
     if (warp == 0) {
         double s1 = 0.0, s2 = 0.0;
         if (lane < kSumWays) {
@@ -439,23 +467,14 @@ __global__ void __launch_bounds__(kActThreads) ffn_tc_act_kernel(const TcParams 
     }
     __syncthreads();
     const float th = theta_s, shift = p.f.identity ? 0.f : th;
-    const int j0 = bx * kActSpan + tid * 8;
     unsigned mask = 0u;
     if (j0 < dff) {
-        const int64_t off = static_cast<int64_t>(n) * dff + j0;
-        float s[8], t[8], t1[8];
-        *reinterpret_cast<float4*>(s) = __ldcg(reinterpret_cast<const float4*>(p.g.S + off));
-        *reinterpret_cast<float4*>(s + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.S + off) + 1);
-        *reinterpret_cast<float4*>(t) = __ldcg(reinterpret_cast<const float4*>(p.g.T0 + off));
-        *reinterpret_cast<float4*>(t + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.T0 + off) + 1);
-        *reinterpret_cast<float4*>(t1) = __ldcg(reinterpret_cast<const float4*>(p.g.T1 + off));
-        *reinterpret_cast<float4*>(t1 + 4) = __ldcg(reinterpret_cast<const float4*>(p.g.T1 + off) + 1);
         float u[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const bool on = s[i] > th;
             const float a = s[i] - shift;
-            u[i] = on ? (p.f.erf_form ? gelu_erf(a) : gelu_tanh(a)) * (t[i] + t1[i]) : 0.f;
+            u[i] = on ? (p.f.erf_form ? gelu_erf(a) : gelu_tanh(a)) * t[i] : 0.f;
             mask |= on ? 1u << i : 0u;
         }
         unsigned h[4], l[4];
@@ -500,7 +519,7 @@ __global__ void __launch_bounds__(kActThreads) ffn_tc_act_kernel(const TcParams 
 constexpr int kOutStages = 4;
 constexpr int kOutVBytes = 4 * kChunk * 128;                                  // four boxes of 64 neurons x 64 columns
 constexpr int kOutStageBytes = kOutVBytes + 2 * kTok * kChunk * 2;            // + u hi, u lo
-constexpr uint32_t kOutCols = 128;                                            // two accumulators of 128 columns x 64 tokens
+constexpr uint32_t kOutCols = 256;                                            // two accumulators of 128 model columns x (hi | lo) tokens
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_uhi,
@@ -525,7 +544,7 @@ ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, c
             auto load_v = [&](int i) {
                 const int s = i % kOutStages;
                 const uint32_t bar = smem_addr(&sh.full[s]);
-                mbar_expect_tx(bar, kOutStageBytes);
+                mbar_expect_tx(bar, kOutVBytes + 2 * static_cast<uint32_t>(p.ntok) * kChunk * 2);
 #pragma unroll
                 for (int b = 0; b < 4; ++b) tma_load_2d(base + s * kOutStageBytes + b * (kChunk * 128), &map_v, bar, col0 + 64 * b, (c0 + i) * kChunk);
             };
@@ -533,7 +552,7 @@ ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, c
                 const int s = i % kOutStages;
                 const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kOutStageBytes + kOutVBytes;
                 tma_load_2d(dst, &map_uhi, bar, (c0 + i) * kChunk, 0);
-                tma_load_2d(dst + kTok * kChunk * 2, &map_ulo, bar, (c0 + i) * kChunk, 0);
+                tma_load_2d(dst + static_cast<uint32_t>(p.ntok) * kChunk * 2, &map_ulo, bar, (c0 + i) * kChunk, 0);   // lo rows behind the hi rows
             };
             const int pre = min(nch, kOutStages);
             for (int i = 0; i < pre; ++i) load_v(i);      // the rows of V do not depend on the kernels ahead
@@ -550,14 +569,14 @@ ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, c
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc(128, p.ntok, true);
+            const uint32_t idesc = instr_desc(128, 2 * p.ntok, true);
             bool ok = true;
             for (int i = 0; i < nch && ok; ++i) {
                 const int s = i % kOutStages;
                 ok = mbar_wait(smem_addr(&sh.full[s]), (i / kOutStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t v0 = base + s * kOutStageBytes, bh = v0 + kOutVBytes, bl = bh + kTok * kChunk * 2;
+                const uint32_t v0 = base + s * kOutStageBytes, b0 = v0 + kOutVBytes;
 #pragma unroll
                 for (int mt = 0; mt < 2; ++mt) {
 #pragma unroll
@@ -565,8 +584,7 @@ ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, c
                         // A: 16 neurons (K) x 128 columns (M) of V, MN-major: 8-neuron groups 1024 bytes apart, the
                         // second 64 columns in the next box (8192 bytes on)
                         const uint64_t ad = smem_desc(v0 + mt * (2 * kChunk * 128) + j * 2048, kChunk * 128, 1024u);
-                        umma_bf16(tmem + mt * 64, ad, smem_desc(bh + 32 * j, 0u, 1024u), idesc, (i == 0 && j == 0) ? 0u : 1u);
-                        umma_bf16(tmem + mt * 64, ad, smem_desc(bl + 32 * j, 0u, 1024u), idesc, 1u);
+                        umma_bf16(tmem + mt * 128, ad, smem_desc(b0 + 32 * j, 0u, 1024u), idesc, (i == 0 && j == 0) ? 0u : 1u);
                     }
                 }
                 umma_commit(smem_addr(&sh.empty[s]));
@@ -580,15 +598,16 @@ ffn_tc_out_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_v, c
         if (nch > 0 && __all_sync(kFull, mbar_wait(smem_addr(&sh.accum), 0u, abort_flag))) {
             tc_fence_after();
             const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16);
-            float v[32];
+            float v[32], w[32];
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
                 float* ycol = p.f.y + col0 + mt * 128 + q * 32 + lane;
                 for (int hb = 0; hb * 32 < B; ++hb) {
-                    tmem_ld32(taddr + mt * 64 + hb * 32, v);
+                    tmem_ld32(taddr + mt * 128 + hb * 32, v);
+                    tmem_ld32(taddr + mt * 128 + p.ntok + hb * 32, w);
 #pragma unroll
                     for (int n = 0; n < 32; ++n)
-                        if (hb * 32 + n < B) atomicAdd(ycol + (hb * 32 + n) * d, v[n]);
+                        if (hb * 32 + n < B) atomicAdd(ycol + (hb * 32 + n) * d, v[n] + w[n]);
                 }
             }
         }
@@ -636,8 +655,8 @@ size_t ffn_tc_workspace_bytes(int64_t d, int64_t d_ff) { return tc_region_bytes(
 int ffn_tc_launch(spark_ctx* ctx, FfnParams& f, cudaStream_t stream) {
     const int d = f.d, r = f.r, d_ff = f.d_ff, B = f.B;
     if (B < 1 || B > kTok || d % 256 != 0 || r % kChunk != 0 || r <= 0 || r >= d || d_ff % 128 != 0 || f.K1s != nullptr) return SPARK_ERR_WORKSPACE;
-    const int call = d / kChunk, cs = r / kChunk, chalf = (call + 1) / 2;
-    if (cs > chalf) return SPARK_ERR_WORKSPACE;
+    const int call = d / kChunk, cs = r / kChunk, chalf = cs > (call + 1) / 2 ? cs : (call + 1) / 2;
+    if (chalf >= call) return SPARK_ERR_WORKSPACE;
     if (ctx->scratch == nullptr || ctx->scratch_bytes < kAttnCellBytes + tc_region_bytes(d, d_ff)) return SPARK_ERR_WORKSPACE;
     const size_t smem_scores = static_cast<size_t>(kScoreStages) * kScoreStageBytes + 1024;
     const size_t smem_out = static_cast<size_t>(kOutStages) * kOutStageBytes + 1024;
@@ -653,15 +672,16 @@ int ffn_tc_launch(spark_ctx* ctx, FfnParams& f, cudaStream_t stream) {
     p.cs = cs;
     p.call = call;
     p.chalf = chalf;
+    p.tfirst = chalf > cs ? 0 : 1;
     const int nbk = d / 256;
     p.ksplit = ctx->num_sms / nbk > 0 ? ctx->num_sms / nbk : 1;
     if (p.ksplit > d_ff / kChunk) p.ksplit = d_ff / kChunk;
 
     CUtensorMap m_k1, m_k2, m_xhi, m_xlo, m_v, m_uhi, m_ulo;
     if (!make_map(&m_k1, f.K1t, d_ff, r, r, 128, true) || !make_map(&m_k2, f.K2t, d_ff, d - r, d - r, 128, true) ||
-        !make_map(&m_xhi, p.g.xhi, kTok, d, d, kTok, false) || !make_map(&m_xlo, p.g.xlo, kTok, d, d, kTok, false) ||
-        !make_map(&m_v, f.Vt, d_ff, d, d, kChunk, true) || !make_map(&m_uhi, p.g.uhi, kTok, d_ff, d_ff, kTok, false) ||
-        !make_map(&m_ulo, p.g.ulo, kTok, d_ff, d_ff, kTok, false))
+        !make_map(&m_xhi, p.g.xhi, kTok, d, d, p.ntok, false) || !make_map(&m_xlo, p.g.xlo, kTok, d, d, p.ntok, false) ||
+        !make_map(&m_v, f.Vt, d_ff, d, d, kChunk, true) || !make_map(&m_uhi, p.g.uhi, kTok, d_ff, d_ff, p.ntok, false) ||
+        !make_map(&m_ulo, p.g.ulo, kTok, d_ff, d_ff, p.ntok, false))
         return SPARK_ERR_WORKSPACE;
 
     if (cudaFuncSetAttribute(ffn_tc_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_scores)) != cudaSuccess ||
@@ -669,11 +689,11 @@ int ffn_tc_launch(spark_ctx* ctx, FfnParams& f, cudaStream_t stream) {
         return SPARK_ERR_CUDA;
     {
         void* args[] = {&p};
-        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_prep_kernel), kTok, 256, 0, stream, false, args) != cudaSuccess) return SPARK_ERR_CUDA;
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_prep_kernel), kTok * kPrepSplit, 256, 0, stream, false, args) != cudaSuccess) return SPARK_ERR_CUDA;
     }
     {
         void* args[] = {&p, &m_k1, &m_k2, &m_xhi, &m_xlo};
-        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_scores_kernel), 2 * (d_ff / 128), kTcThreads, smem_scores, stream, false, args) != cudaSuccess)
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(ffn_tc_scores_kernel), static_cast<unsigned>(2 * (d_ff / kScoreRows)), kTcThreads, smem_scores, stream, false, args) != cudaSuccess)
             return SPARK_ERR_CUDA;
     }
     {

@@ -2,7 +2,8 @@
 
     python -m paper_2506_06644_b200.profile_cases ffn     # one-token Spark FFN, Gemma-2-2B shape
     python -m paper_2506_06644_b200.profile_cases ffn4    # four tokens (few-token kernel)
-    python -m paper_2506_06644_b200.profile_cases ffn16   # sixteen tokens (tensor-core kernel)
+    python -m paper_2506_06644_b200.profile_cases ffn16   # sixteen tokens (tensor-core kernel, mma.sync)
+    python -m paper_2506_06644_b200.profile_cases ffn64   # a chunk of 64 tokens (tcgen05 kernels)
     python -m paper_2506_06644_b200.profile_cases attn    # Spark attention, batch 1, context 8192
     python -m paper_2506_06644_b200.profile_cases topk    # statistical top-k, 512 rows x 65536
     python -m paper_2506_06644_b200.profile_cases layer   # four decoder layers, one token
@@ -107,7 +108,7 @@ def case_layer(n_layers=4, B=1, ctx_len=8192, steps=3, overlap=True):
     assert ctx.device_status() == S.SPARK_OK
 
 
-CASES = {"ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
+CASES = {"ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
 
 if __name__ == "__main__":
     name = sys.argv[1] if len(sys.argv) > 1 else ""
