@@ -11,8 +11,6 @@
 //            u_i = GELU(s_i - theta) t_i, then a thread per 8 output columns accumulates
 //            sum_i u_i V[:,i] in registers and adds it to y with vector reductions.
 // Individual masks gate the arithmetic, the union gates the loads (Appendix B).
-#include <cstdlib>
-
 #include "ffn_params.h"
 #include "kernels.h"
 #include "rowdot.cuh"
@@ -392,10 +390,9 @@ int launch_tb(spark_ctx* ctx, FfnParams& p, int tb, size_t smem, cudaStream_t st
 
 namespace spark {
 
-static int tc_min_tokens() {
-    static const int v = []() { const char* e = getenv("SPARK_TC_MIN"); return e ? atoi(e) : 17; }();
-    return v;
-}
+// From this many tokens on the chunk path on the tcgen05 tensor cores (reads every weight row) is at least as
+// fast as the union-gather kernels, measured at the Gemma-2 shapes with independent and with correlated tokens.
+constexpr int kTcMinTokens = 5;
 
 int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     if (ctx == nullptr || a.x == nullptr || a.K1t == nullptr || a.K2t == nullptr || a.Vt == nullptr || a.y == nullptr)
@@ -443,7 +440,7 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
         const int rc = ffn_few_launch(ctx, p, a.wdtype, stream);
         if (rc != SPARK_ERR_WORKSPACE) return rc;
     }
-    if (a.B >= tc_min_tokens() && a.B <= 64 && a.wdtype == SPARK_BF16) {      // reads every row: SPARK_DENSE_LOADS changes nothing here
+    if (a.B >= kTcMinTokens && a.B <= 64 && a.wdtype == SPARK_BF16) {      // reads every row: SPARK_DENSE_LOADS changes nothing here
         const int rc = ffn_tc_launch(ctx, p, stream);
         if (rc != SPARK_ERR_WORKSPACE) return rc;
     }

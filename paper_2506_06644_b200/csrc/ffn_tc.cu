@@ -655,8 +655,19 @@ size_t ffn_tc_workspace_bytes(int64_t d, int64_t d_ff) { return tc_region_bytes(
 int ffn_tc_launch(spark_ctx* ctx, FfnParams& f, cudaStream_t stream) {
     const int d = f.d, r = f.r, d_ff = f.d_ff, B = f.B;
     if (B < 1 || B > kTok || d % 256 != 0 || r % kChunk != 0 || r <= 0 || r >= d || d_ff % 128 != 0 || f.K1s != nullptr) return SPARK_ERR_WORKSPACE;
-    const int call = d / kChunk, cs = r / kChunk, chalf = cs > (call + 1) / 2 ? cs : (call + 1) / 2;
-    if (chalf >= call) return SPARK_ERR_WORKSPACE;
+    // The first block of a pair takes all of the predictor's chunks (its sums must be complete) and, where that
+    // leaves it short, some of the K2 product's.  Epilogues in units of a chunk's time (measured): scores
+    // and sums about eight, a partial K2 product about four.
+    const int call = d / kChunk, cs = r / kChunk;
+    if (cs >= call) return SPARK_ERR_WORKSPACE;
+    int chalf = cs, best = 1 << 30;
+    for (int c = cs; c < call; ++c) {
+        const int first = c + 8 + (c > cs ? 4 : 0), second = call - c + 4, worst = first > second ? first : second;
+        if (worst < best) {
+            best = worst;
+            chalf = c;
+        }
+    }
     if (ctx->scratch == nullptr || ctx->scratch_bytes < kAttnCellBytes + tc_region_bytes(d, d_ff)) return SPARK_ERR_WORKSPACE;
     const size_t smem_scores = static_cast<size_t>(kScoreStages) * kScoreStageBytes + 1024;
     const size_t smem_out = static_cast<size_t>(kOutStages) * kOutStageBytes + 1024;

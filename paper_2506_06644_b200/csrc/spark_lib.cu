@@ -60,10 +60,10 @@ size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap
     const size_t need = kAttnCellBytes +
                         round_up(pieces * 8 * (static_cast<size_t>(hd) + 8) * 4, 256) +
                         round_up((static_cast<size_t>(max_batch) * n_q * max_cap + grid_bound * 8) * 4, 256);
-    // FFN over chunks of more than 16 tokens: split inputs, scores and activations of the tensor-core path,
+    // FFN over chunks of five and more tokens: split inputs, scores and activations of the tensor-core path,
     // placed behind the attention's cells (the two never run at the same time on one context)
     size_t need_ffn = 0;
-    if (max_batch > 16 && max_dff > 0 && max_d > 0) need_ffn = kAttnCellBytes + ffn_tc_workspace_bytes(max_d, max_dff);
+    if (max_batch >= 5 && max_dff > 0 && max_d > 0) need_ffn = kAttnCellBytes + ffn_tc_workspace_bytes(max_d, max_dff);
     return sizeof(WsHeader) + (need > need_ffn ? need : need_ffn) + 256;
 }
 
