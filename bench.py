@@ -33,7 +33,7 @@ import numpy as np
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from the ncu
 # capture summarised in profiles/ (keyed by shape and batch); None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {("2b", 1): 24.34e6, ("2b", 16): 68.07e6}       # profiles/ffn_b1.md, profiles/ffn_mma_b16.md
+NCU_TRAFFIC_BYTES = {("2b", 1): 24.34e6}       # profiles/ffn_b1.md
 
 FALLBACK_HBM_GBS = 6650.0
 
@@ -254,7 +254,9 @@ def run_spark(args):
     scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
-    kernels_per_layer = 4 if B <= 4 else 5     # QKV (+ rotary, append: a kernel of their own for B >= 5), attention, output projection, FFN
+    # QKV (+ rotary, append: a kernel of their own for B >= 5), attention, output projection, FFN (four kernels on the
+    # tcgen05 chunk path for B >= 5: prep, scores, activation, output)
+    kernels_per_layer = 4 if B <= 4 else 8
 
     def stack(which):
         for lay in layers:
@@ -434,7 +436,7 @@ def run_spark(args):
                     "h2d_bytes_per_step": int(h_host_in.numel() * 4), "d2h_bytes_per_step": int(h_host_out.numel() * 4)},
             "gpu_launches": args.steps * n_layers * kernels_per_layer,
             "clocks": clocks,
-            "roofline": {"kernel": ("ffn1_kernel" if B == 1 else "ffn_mma_kernel") + " (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
+            "roofline": {"kernel": ("ffn1_kernel" if B == 1 else "ffn_few_kernel" if B <= 4 else "ffn_tc_{prep,scores,act,out}_kernel") + " (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
                          "us_per_launch": ffn_us, "touched_bytes_per_launch": touched, "union_rows": union},
             "roofline_attention": {"kernel": "attn_kernel (spark_attn_decode)", "bound": "hbm",
@@ -493,11 +495,12 @@ def other_workloads(torch, S, peak, steps, warmup):
             e["speedup_vs_dense_loads"] = dense_us / us
         out.append(e)
 
-    # -- Spark FFN, 4 and 16 tokens, Gemma-2-2B shape, 8 weight sets (580 MB)
+    # -- Spark FFN, 4, 16 and 64 tokens, Gemma-2-2B shape, 8 weight sets (580 MB); from five tokens on the path reads every
+    #    weight row (tcgen05 chunk kernels), so SPARK_DENSE_LOADS is the same run and the bytes are all of the weights
     def w(rows, cols):
         return (torch.randn(rows, cols, device=dev, generator=gen) * sh.d ** -0.5).to(torch.bfloat16)
     sets = [(w(sh.d_ff, sh.r_ff), w(sh.d_ff, sh.d - sh.r_ff), w(sh.d_ff, sh.d)) for _ in range(8)]
-    for B in (4, 16):
+    for B in (4, 16, 64):
         ctx = S.SparkContext(dev.index, max_batch=B, max_dff=sh.d_ff, max_d=sh.d)
         ctx.set_launch_overlap(True)
         x = torch.randn(B, sh.d, device=dev, generator=gen)
@@ -508,14 +511,16 @@ def other_workloads(torch, S, peak, steps, warmup):
         torch.cuda.synchronize()
         union = int(torch.unique(torch.cat([idx[b, : int(cnt[b])] for b in range(B)])).numel())
         res = []
-        for flags in (0, S.SPARK_DENSE_LOADS):
+        for flags in (0, S.SPARK_DENSE_LOADS) if B <= 4 else (0,):
             def calls():
                 for k1, k2, v in sets:
                     S.spark_ffn_decode(ctx, x, B, k1, k2, v, S.SPARK_BF16, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, flags, y, None, None, None)
             res.append(time_graph(calls, len(sets)))
         assert ctx.device_status() == S.SPARK_OK
-        entry(f"spark_ffn_decode gemma2-2b shape, {B} tokens (union of active sets {union} of {sh.d_ff})", res[0],
-              sh.d_ff * sh.r_ff * 2 + union * (2 * sh.d - sh.r_ff) * 2, res[1])
+        rows_read = union if B <= 4 else sh.d_ff
+        entry(f"spark_ffn_decode gemma2-2b shape, {B} tokens (union of active sets {union} of {sh.d_ff}" +
+              (")" if B <= 4 else "; every row read)"), res[0],
+              sh.d_ff * sh.r_ff * 2 + rows_read * (2 * sh.d - sh.r_ff) * 2, res[1] if B <= 4 else None)
         ctx.close()
     del sets
 

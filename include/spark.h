@@ -141,7 +141,11 @@ int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int
 /* ---- Spark FFN (Section 2.1, Eq. 2) ------------------------------------------
  * y_b = V . ( GELU(StatTop_k(K1^T x_b[:r])) * (K2^T x_b[r:]) ) for each of the B tokens, every
  * token with its own threshold and active set; weight rows are loaded once per call for the
- * union of the tokens' active sets (Appendix B).
+ * union of the tokens' active sets (Appendix B).  Chunks of 5 to 64 tokens with bf16 weights, where
+ * that union covers most rows, read every row instead and run the three products as GEMMs on the
+ * tensor cores (same results; SPARK_DENSE_LOADS changes nothing there); this needs d % 256 == 0,
+ * r % 64 == 0, d_ff % 128 == 0 and a workspace sized by spark_workspace_bytes for max_batch >= 5,
+ * max_dff >= d_ff and max_d >= d -- any other call with 5..64 tokens takes the union-gather kernels.
  *   x [B][d] fp32;  K1t[d_ff][r], K2t[d_ff][d-r], Vt[d_ff][d] of dtype wdtype
  *   flags: SPARK_GELU_TANH or SPARK_GELU_ERF, optionally | SPARK_DENSE_LOADS
  *   y     [B][d]     fp32 (overwritten)

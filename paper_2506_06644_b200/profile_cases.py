@@ -2,7 +2,7 @@
 
     python -m paper_2506_06644_b200.profile_cases ffn     # one-token Spark FFN, Gemma-2-2B shape
     python -m paper_2506_06644_b200.profile_cases ffn4    # four tokens (few-token kernel)
-    python -m paper_2506_06644_b200.profile_cases ffn16   # sixteen tokens (tensor-core kernel, mma.sync)
+    python -m paper_2506_06644_b200.profile_cases ffn16   # sixteen tokens (tcgen05 chunk kernels)
     python -m paper_2506_06644_b200.profile_cases ffn64   # a chunk of 64 tokens (tcgen05 kernels)
     python -m paper_2506_06644_b200.profile_cases attn    # Spark attention, batch 1, context 8192
     python -m paper_2506_06644_b200.profile_cases topk    # statistical top-k, 512 rows x 65536

@@ -69,7 +69,7 @@ def test_tiny_fp32_layer(ctx):
         compare(p, run_ffn(ctx, p, flags=flags), form=form)
 
 
-@pytest.mark.parametrize("B", [1, 2, 3, 4, 8, 16])     # 1: one-token kernel; 2-4: few-token kernel; 5-16: tensor cores
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 8, 16])     # 1: one-token kernel; 2-4: few-token kernel; 8, 16: tcgen05 chunk kernels
 def test_gemma2_2b_shape_bf16(ctx, B):
     p = synth.ffn_inputs(2304, 9216, 1024, 737, B, "bf16", seed=0)
     w = upload(p)
@@ -88,7 +88,8 @@ def test_gemma2_2b_shape_bf16(ctx, B):
                                               (2304, 9216, 1024, 737, 64, "erf"), (3584, 14336, 1792, 1147, 24, "tanh"),
                                               (256, 1024, 128, 82, 33, "tanh"), (512, 2048, 64, 164, 20, "tanh")])
 def test_token_chunks_on_the_tensor_cores(ctx, d, d_ff, r, k, B, form):
-    # 17..64 tokens: TMA-fed tcgen05 kernels that read every weight row (the union of the active sets covers most)
+    # TMA-fed tcgen05 kernels that read every weight row (the union of the active sets covers most); shapes with one and
+    # two partial K2 products, 9B shape, token counts that fill 2, 3 and 4 sixteen-token groups
     p = synth.ffn_inputs(d, d_ff, r, k, B, "bf16", seed=B)
     w = upload(p)
     out = run_ffn(ctx, p, weights=w, flags=S.SPARK_GELU_ERF if form == "erf" else S.SPARK_GELU_TANH)
