@@ -138,6 +138,29 @@ int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int
                     int fill, float* theta, int32_t* count, int32_t* idx, float* val,
                     int64_t idx_cap, float* y_dense, void* stream);
 
+/* ---- statistical top-k of a row sharded over several devices (Appendix, "global statistical top-k") ----
+ * Each device holds a contiguous part of every row.  The global form needs one small exchange: every
+ * device takes the moments of its part (spark_stat_moments), the parts' moments are gathered (the
+ * caller's collective; 24 bytes per row and device), merged into theta of the whole row
+ * (spark_stat_merge; the same on every device), and each device selects from its part with that
+ * threshold (spark_stat_select).  The result equals spark_stat_topk on the concatenated row.  The local
+ * form of the same appendix needs no exchange: spark_stat_topk on the part with k / m.
+ *
+ * spark_stat_moments: moments[row] = (n, mean, sum of squared deviations from the mean) of
+ *   x[row*ld .. row*ld + n) as three doubles, [rows][3].  n >= 2.
+ * spark_stat_merge: parts [m][rows][3] (device memory, part after part as gathered); theta[rows] =
+ *   mean + std * Q(1 - k / n_total) of the merged moments, Bessel-corrected (Eq. 11), -inf for
+ *   k >= n_total; merged [rows][3] nullable.  The parts' counts must add up to n_total.
+ * spark_stat_select: like spark_stat_topk with the thresholds given (theta_in [rows], device): count,
+ *   idx (indices within the part), val, y_dense as there; survivors are shifted by theta_in. */
+int spark_stat_moments(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, double* moments,
+                       void* stream);
+int spark_stat_merge(spark_ctx* ctx, const double* parts, int64_t m, int64_t rows, int64_t k, int64_t n_total,
+                     float* theta, double* merged, void* stream);
+int spark_stat_select(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, const float* theta_in,
+                      int fill, int32_t* count, int32_t* idx, float* val, int64_t idx_cap, float* y_dense,
+                      void* stream);
+
 /* ---- Spark FFN (Section 2.1, Eq. 2) ------------------------------------------
  * y_b = V . ( GELU(StatTop_k(K1^T x_b[:r])) * (K2^T x_b[r:]) ) for each of the B tokens, every
  * token with its own threshold and active set; weight rows are loaded once per call for the

@@ -100,6 +100,51 @@ def stat_topk(x: np.ndarray, k: int, fill: str = "zero"):
 
 
 # ----------------------------------------------------------------------------
+# statistical top-k of a vector sharded over m devices (appendix on distributed
+# training: "global" and "local" statistical top-k)
+# ----------------------------------------------------------------------------
+def shard_moments(x: np.ndarray) -> tuple[float, float, float]:
+    """What one device computes of its part: (count, mean, sum of squared deviations from its mean).
+
+    Reading: the paper has the devices exchange "mean and variance"; the count is carried along so
+    that parts of unequal length combine correctly, and the sum of squared deviations stands for
+    the variance (variance x count) so that no convention about its divisor is needed."""
+    x = np.asarray(x, dtype=F64).reshape(-1)
+    mean = float(np.sum(x) / x.size)
+    return float(x.size), mean, float(np.sum((x - mean) ** 2))
+
+
+def combine_moments(parts) -> tuple[float, float, float]:
+    """Moments of the whole vector from the parts' moments: the weighted mean, and the law of total
+    variance (within-part deviations plus the parts' squared distances to the global mean)."""
+    n = sum(p[0] for p in parts)
+    mean = sum(p[0] * p[1] for p in parts) / n
+    m2 = sum(p[2] + p[0] * (p[1] - mean) ** 2 for p in parts)
+    return n, mean, m2
+
+
+def stat_topk_sharded_global(shards, k: int, fill: str = "zero"):
+    """Global statistical top-k: every device combines all parts' moments into mean and Bessel-corrected
+    std of the whole vector, forms theta (Eq. 11 with d = total length) and thresholds its own part.
+    Returns (theta, [mask per shard], [out per shard])."""
+    shards = [np.asarray(s, dtype=F64).reshape(-1) for s in shards]
+    n, mean, m2 = combine_moments([shard_moments(s) for s in shards])
+    off = 0.0 if fill == "zero" else -np.inf
+    if k >= n:
+        return -np.inf, [np.ones(s.size, dtype=bool) for s in shards], [s.copy() for s in shards]
+    theta = mean + math.sqrt(m2 / (n - 1)) * gaussian_upper_quantile(k / n)
+    masks = [s > theta for s in shards]
+    return theta, masks, [np.where(m, s - theta, off) for s, m in zip(shards, masks)]
+
+
+def stat_topk_sharded_local(shards, k: int, fill: str = "zero"):
+    """Local statistical top-k: each device applies the operator to its own part with k' = k / m
+    (reading: integer division, at least 1).  Returns a list of (theta, mask, out) per shard."""
+    kk = max(1, k // len(shards))
+    return [stat_topk(s, kk, fill) for s in shards]
+
+
+# ----------------------------------------------------------------------------
 # activations
 # ----------------------------------------------------------------------------
 _erf = np.vectorize(math.erf, otypes=[F64])

@@ -28,6 +28,7 @@ EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
     "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_set_launch_overlap", "spark_stat_topk", "spark_ffn_decode",
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
+    "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
 ]
 
 
@@ -75,6 +76,9 @@ def lib() -> C.CDLL:
         "spark_set_phase_trace": (i32, [vp, vp, i64]),
         "spark_set_launch_overlap": (i32, [vp, i32]),
         "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
+        "spark_stat_moments": (i32, [vp, vp, i64, i64, i64, vp, vp]),
+        "spark_stat_merge": (i32, [vp, vp, i64, i64, i64, i64, vp, vp, vp]),
+        "spark_stat_select": (i32, [vp, vp, i64, i64, i64, vp, i32, vp, vp, vp, i64, vp, vp]),
         "spark_ffn_decode": (i32, [vp, vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
         "spark_ffn_decode_noalloc": (i32, [vp, i64, vp, vp, vp, i32, i64, i64, i64, i64, i32, vp, vp, vp]),
         "spark_ffn_decode_fp8": (i32, [vp, vp, i64, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, vp]),
@@ -178,6 +182,20 @@ class SparkContext:
             self.close()
         except Exception:
             pass
+
+
+def spark_stat_moments(ctx: SparkContext, x, rows, n, ld, moments):
+    _check(lib().spark_stat_moments(ctx.handle, _ptr(x), rows, n, ld, _ptr(moments), _stream()), "spark_stat_moments")
+
+
+def spark_stat_merge(ctx: SparkContext, parts, m, rows, k, n_total, theta, merged):
+    _check(lib().spark_stat_merge(ctx.handle, _ptr(parts), m, rows, k, n_total, _ptr(theta), _ptr(merged), _stream()),
+           "spark_stat_merge")
+
+
+def spark_stat_select(ctx: SparkContext, x, rows, n, ld, theta_in, fill, count, idx, val, idx_cap, y_dense):
+    _check(lib().spark_stat_select(ctx.handle, _ptr(x), rows, n, ld, _ptr(theta_in), fill, _ptr(count), _ptr(idx), _ptr(val),
+                                   idx_cap, _ptr(y_dense), _stream()), "spark_stat_select")
 
 
 def spark_stat_topk(ctx: SparkContext, x, rows, n, ld, k, fill, theta, count, idx, val, idx_cap, y_dense):

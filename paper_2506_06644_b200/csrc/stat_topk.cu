@@ -32,6 +32,8 @@ struct TopkParams {
     float* val;
     int64_t idx_cap;
     float* y_dense;
+    const float* theta_in;   // nullable: thresholds given by the caller (sharded rows: theta of the whole row); no statistics
+    double* moments_out;     // nullable: [rows][3] = (n, mean, sum of squared deviations) of each row; nothing else is produced
     WsHeader* hdr;
 };
 
@@ -81,7 +83,7 @@ __global__ void __launch_bounds__(kThreads) stat_topk_kernel(const TopkParams p)
     };
 
     float theta = -INFINITY;
-    if (!p.identity) {
+    if (!p.identity && p.theta_in == nullptr) {
         // ---- sweep 1: the only HBM read of the row; sum -> mean --------------------------------
         float s0 = 0.f, s1 = 0.f;
         constexpr int LB = 8;                 // 16-byte loads a thread keeps in flight
@@ -141,6 +143,15 @@ __global__ void __launch_bounds__(kThreads) stat_topk_kernel(const TopkParams p)
         for (unsigned c = 0; c < cl; ++c) m2 += *cluster.map_shared_rank(&part_m2, c);
         if (m2 < 0.0) m2 = 0.0;
         Moments m{static_cast<double>(p.n), mean, m2};
+        if (p.moments_out != nullptr) {      // a shard's moments for the caller to merge (Appendix: global statistical top-k)
+            if (rank == 0 && tid == 0) {
+                p.moments_out[row * 3 + 0] = m.n;
+                p.moments_out[row * 3 + 1] = m.mean;
+                p.moments_out[row * 3 + 2] = m.m2;
+            }
+            cluster.sync();   // no block may leave while a peer can still read its shared memory
+            return;
+        }
         theta = theta_from(m, p.z);
     } else if (RESIDENT) {
         for (int v = tid; v < nvec; v += kThreads) {
@@ -149,6 +160,7 @@ __global__ void __launch_bounds__(kThreads) stat_topk_kernel(const TopkParams p)
         }
         __syncthreads();
     }
+    if (p.theta_in != nullptr) theta = p.theta_in[row];
     const float shift = p.identity ? 0.f : theta;
     const bool want_lists = (p.idx != nullptr) || (p.val != nullptr);
 
@@ -615,9 +627,9 @@ bool g_attr_done[64] = {};   // per device: opt-in shared memory configured
 
 }  // namespace
 
-extern "C" int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld,
-                               int64_t k, int fill, float* theta, int32_t* count, int32_t* idx,
-                               float* val, int64_t idx_cap, float* y_dense, void* stream) {
+// theta_in / moments_out: the two halves of the sharded form (see spark_stat_moments, spark_stat_select).
+static int topk_launch(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, int64_t k, int fill, float* theta, int32_t* count,
+                int32_t* idx, float* val, int64_t idx_cap, float* y_dense, const float* theta_in, double* moments_out, void* stream) {
     if (ctx == nullptr || x == nullptr) return SPARK_ERR_INVALID_ARG;
     if (rows < 0 || n < 1 || ld < n || k <= 0) return SPARK_ERR_INVALID_ARG;
     if (fill != SPARK_FILL_ZERO && fill != SPARK_FILL_NEGINF) return SPARK_ERR_INVALID_ARG;
@@ -641,6 +653,7 @@ extern "C" int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int
     p.identity = k >= n ? 1 : 0;
     p.z = p.identity ? 0.0 : spark_normal_upper_quantile(static_cast<double>(k) / static_cast<double>(n));
     p.theta = theta; p.count = count; p.idx = idx; p.val = val; p.idx_cap = idx_cap; p.y_dense = y_dense;
+    p.theta_in = theta_in; p.moments_out = moments_out;
     p.hdr = ctx->hdr;
 
     if (ctx->device >= 0 && ctx->device < 64 && !g_attr_done[ctx->device]) {
@@ -650,7 +663,7 @@ extern "C" int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int
         g_attr_done[ctx->device] = true;
     }
 
-    if (n > 16384 && (n + 3) / 4 <= kRowMaxVec) {      // the whole row fits one block: no cluster needed
+    if (n > 16384 && (n + 3) / 4 <= kRowMaxVec && theta_in == nullptr && moments_out == nullptr) {      // the whole row fits one block: no cluster needed
         static bool row_attr_done[64] = {};
         if (ctx->device >= 0 && ctx->device < 64 && !row_attr_done[ctx->device]) {
             if (cudaFuncSetAttribute(stat_topk_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowSmemBytes) != cudaSuccess)
@@ -678,4 +691,58 @@ extern "C" int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int
     cudaError_t e = resident ? cudaLaunchKernelEx(&cfg, stat_topk_kernel<true>, p)
                              : cudaLaunchKernelEx(&cfg, stat_topk_kernel<false>, p);
     return e == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+extern "C" int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld,
+                               int64_t k, int fill, float* theta, int32_t* count, int32_t* idx,
+                               float* val, int64_t idx_cap, float* y_dense, void* stream) {
+    return topk_launch(ctx, x, rows, n, ld, k, fill, theta, count, idx, val, idx_cap, y_dense, nullptr, nullptr, stream);
+}
+
+extern "C" int spark_stat_moments(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, double* moments, void* stream) {
+    if (moments == nullptr || n < 1) return SPARK_ERR_INVALID_ARG;
+    // k = 1 < n keeps the statistics branch; for n == 1 the row is its own mean
+    if (n == 1) return SPARK_ERR_UNSUPPORTED;
+    return topk_launch(ctx, x, rows, n, ld, 1, SPARK_FILL_ZERO, nullptr, nullptr, nullptr, nullptr, 0, nullptr, nullptr, moments, stream);
+}
+
+extern "C" int spark_stat_select(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, const float* theta_in, int fill,
+                                 int32_t* count, int32_t* idx, float* val, int64_t idx_cap, float* y_dense, void* stream) {
+    if (theta_in == nullptr) return SPARK_ERR_INVALID_ARG;
+    // k = 1 < n: not the identity case, so survivors are shifted by the given threshold
+    if (n < 2) return SPARK_ERR_UNSUPPORTED;
+    return topk_launch(ctx, x, rows, n, ld, 1, fill, nullptr, count, idx, val, idx_cap, y_dense, theta_in, nullptr, stream);
+}
+
+namespace {
+
+// One thread per row: merge the m shards' moments (pairwise update of count, mean and sum of squared deviations) and
+// form theta = mean + std * Q(1 - k/n) of the whole row (Eq. 10/11 on the merged moments).
+__global__ void stat_merge_kernel(const double* parts, int64_t m, int64_t rows, double z, int identity, float* theta, double* merged) {
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    Moments acc{0.0, 0.0, 0.0};
+    for (int64_t s = 0; s < m; ++s) {
+        const double* q = parts + (s * rows + row) * 3;
+        acc = merge(acc, Moments{q[0], q[1], q[2]});
+    }
+    if (merged != nullptr) {
+        merged[row * 3 + 0] = acc.n;
+        merged[row * 3 + 1] = acc.mean;
+        merged[row * 3 + 2] = acc.m2;
+    }
+    theta[row] = identity ? -INFINITY : theta_from(acc, z);
+}
+
+}  // namespace
+
+extern "C" int spark_stat_merge(spark_ctx* ctx, const double* parts, int64_t m, int64_t rows, int64_t k, int64_t n_total, float* theta,
+                                double* merged, void* stream) {
+    if (ctx == nullptr || parts == nullptr || theta == nullptr || m < 1 || rows < 0 || k <= 0 || n_total < 1) return SPARK_ERR_INVALID_ARG;
+    if (k < n_total && n_total < 2) return SPARK_ERR_INVALID_ARG;
+    if (rows == 0) return SPARK_OK;
+    const int identity = k >= n_total ? 1 : 0;
+    const double z = identity ? 0.0 : spark_normal_upper_quantile(static_cast<double>(k) / static_cast<double>(n_total));
+    stat_merge_kernel<<<static_cast<unsigned>((rows + 127) / 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(parts, m, rows, z, identity, theta, merged);
+    return cudaGetLastError() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
 }

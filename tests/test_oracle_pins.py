@@ -444,3 +444,50 @@ def test_row_scaled_e4m3_quantisation_error_bound():
     bound = np.maximum(np.abs(W) * 2.0 ** -4, (amax / 448.0) * 2.0 ** -10)
     assert np.all(err <= bound * (1 + 1e-6))
     assert np.all(np.abs(deq).max(axis=1) <= amax[:, 0] * (1 + 1e-6))
+
+
+# ---- sharded statistical top-k (appendix on distributed training) ----------------------------------------
+def test_combined_moments_hand_example_and_library():
+    # parts [1, 2, 3] and [4 .. 8]: eight values, mean 4.5, sum of squared deviations 42 (by hand)
+    parts = [O.shard_moments(np.array([1.0, 2.0, 3.0])), O.shard_moments(np.array([4.0, 5.0, 6.0, 7.0, 8.0]))]
+    assert parts[0] == (3.0, 2.0, 2.0) and parts[1] == (5.0, 6.0, 10.0)
+    assert O.combine_moments(parts) == (8.0, 4.5, 42.0)
+    rng = np.random.default_rng(11)
+    x = rng.normal(3.0, 2.0, size=5000)
+    cuts = [0, 17, 1200, 1201, 4000, 5000]
+    n, mean, m2 = O.combine_moments([O.shard_moments(x[a:b]) for a, b in zip(cuts[:-1], cuts[1:])])
+    assert n == 5000 and mean == pytest.approx(np.mean(x), rel=1e-13)
+    assert m2 / (n - 1) == pytest.approx(np.var(x, ddof=1), rel=1e-12)
+
+
+@pytest.mark.parametrize("m", [2, 3, 8])
+def test_global_sharded_topk_equals_the_unsharded_operator(m):
+    # the appendix's claim: the output is exactly that of statistical top-k without sharding
+    rng = np.random.default_rng(m)
+    x = rng.normal(size=4096) + np.repeat(rng.normal(size=m), -(-4096 // m))[:4096]      # parts with different means
+    cuts = np.concatenate([[0], np.sort(rng.choice(np.arange(1, 4096), size=m - 1, replace=False)), [4096]])
+    shards = [x[a:b] for a, b in zip(cuts[:-1], cuts[1:])]
+    for fill in ("zero", "neginf"):
+        theta, masks, outs = O.stat_topk_sharded_global(shards, 300, fill)
+        ref_theta, ref_mask, ref_out = O.stat_topk(x, 300, fill)
+        assert theta == pytest.approx(ref_theta, rel=1e-12)
+        assert np.array_equal(np.concatenate(masks), ref_mask)
+        np.testing.assert_allclose(np.concatenate(outs), ref_out, rtol=0, atol=1e-12)
+    theta, masks, _ = O.stat_topk_sharded_global(shards, 4096)
+    assert theta == -np.inf and all(mk.all() for mk in masks)
+
+
+def test_local_sharded_topk_is_the_operator_per_part_and_differs_from_global():
+    rng = np.random.default_rng(5)
+    lo, hi = rng.normal(0.0, 1.0, size=2048), rng.normal(6.0, 1.0, size=2048)       # the second part holds the largest values
+    local = O.stat_topk_sharded_local([lo, hi], 200)
+    for part, (theta, mask, out) in zip((lo, hi), local):
+        ref = O.stat_topk(part, 100)
+        assert theta == ref[0] and np.array_equal(mask, ref[1])
+    # each part keeps about k / m; the global form takes everything from the part with the larger values
+    assert abs(int(local[0][1].sum()) - 100) < 40 and abs(int(local[1][1].sum()) - 100) < 40
+    _, gmasks, _ = O.stat_topk_sharded_global([lo, hi], 200)
+    assert gmasks[0].sum() == 0 and gmasks[1].sum() > 150
+    # k not divisible by m: k' = floor(k / m), never below one
+    assert O.stat_topk_sharded_local([lo, hi], 201)[0][0] == local[0][0]
+    assert O.stat_topk_sharded_local([lo, hi, lo, hi], 3)[0][0] == O.stat_topk(lo, 1)[0]
