@@ -27,7 +27,7 @@ def gather_parts(local: torch.Tensor, group=None) -> torch.Tensor:
     """All-gather the ranks' [rows, 3] moments into [world, rows, 3], part r from rank r."""
     world = dist.get_world_size(group)
     out = torch.empty((world,) + tuple(local.shape), dtype=local.dtype, device=local.device)
-    dist.all_gather_into_tensor(out, local.contiguous(), group=group)
+    dist.all_gather(list(out.unbind(0)), local.contiguous(), group=group)      # views of one buffer: part r lands in out[r]
     return out
 
 

@@ -484,10 +484,11 @@ def test_local_sharded_topk_is_the_operator_per_part_and_differs_from_global():
     for part, (theta, mask, out) in zip((lo, hi), local):
         ref = O.stat_topk(part, 100)
         assert theta == ref[0] and np.array_equal(mask, ref[1])
-    # each part keeps about k / m; the global form takes everything from the part with the larger values
+    # each part keeps about k / m; the global form takes nothing from the part with the smaller values (how many it
+    # takes from the other is no longer about k: the mixture is far from Gaussian)
     assert abs(int(local[0][1].sum()) - 100) < 40 and abs(int(local[1][1].sum()) - 100) < 40
     _, gmasks, _ = O.stat_topk_sharded_global([lo, hi], 200)
-    assert gmasks[0].sum() == 0 and gmasks[1].sum() > 150
+    assert gmasks[0].sum() == 0 and gmasks[1].sum() > 0 and local[0][1].sum() > 0
     # k not divisible by m: k' = floor(k / m), never below one
     assert O.stat_topk_sharded_local([lo, hi], 201)[0][0] == local[0][0]
     assert O.stat_topk_sharded_local([lo, hi, lo, hi], 3)[0][0] == O.stat_topk(lo, 1)[0]
