@@ -69,8 +69,13 @@ enum {
 enum {
     SPARK_GELU_TANH = 0,     /* tanh form of GELU (the one Gemma uses); the default            */
     SPARK_GELU_ERF = 1,      /* exact form x * Phi(x)                                          */
-    SPARK_DENSE_LOADS = 2    /* comparator: same result, but every row of K2/V (or of the cache)
+    SPARK_DENSE_LOADS = 2,   /* comparator: same result, but every row of K2/V (or of the cache)
                                 is read and multiplied by its (possibly zero) activation       */
+    SPARK_SHARED_CACHE = 4   /* attention and layer: the B tokens are consecutive tokens of ONE
+                                sequence (a chunk of its prompt) and share one cache
+                                [n_kv][cap][.]; token b is the sequence's token number ctx_len[b]
+                                (1-based) and sees rows [0, ctx_len[b]), so with ctx_len[b] =
+                                L0 + b + 1 the chunk is causal; caches lose their [B] dimension  */
 };
 
 typedef struct spark_ctx spark_ctx;
@@ -262,6 +267,10 @@ int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const void* Wt, 
  *   a = RMSNorm(h; norm1);  [q|k|v] = Wqkv a;  rotary position encoding applied separately to
  *   q[:r], q[r:], k[:r], k[r:] at position ctx_len[b]-1;  q *= 1/sqrt(hd);
  *   k, v written to row ctx_len[b]-1 of the caches;  h += Wo . SparkAttention;  h += SparkFFN(RMSNorm(h; norm2)).
+ * With SPARK_SHARED_CACHE in cfg->flags the B tokens are consecutive tokens of one sequence (a chunk of
+ * its prompt): the caches are [n_kv][cap][.], token b is appended at row ctx_len[b]-1 and attends to rows
+ * [0, ctx_len[b]); ctx_len[b] = L0 + b + 1 gives what decoding the chunk token by token gives (n_kv a
+ * power of two).  1 <= B <= 16 either way.
  * All pointers inside the structs are device pointers; the structs themselves are host objects. */
 typedef struct spark_layer_weights {
     const float* norm1;   /* [d]                          */

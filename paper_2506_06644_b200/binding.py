@@ -22,7 +22,7 @@ SPARK_ERR_INVALID_ARG, SPARK_ERR_UNSUPPORTED, SPARK_ERR_WORKSPACE, SPARK_ERR_CUD
 SPARK_ERR_TIMEOUT, SPARK_ERR_OVERFLOW = 5, 6
 SPARK_F32, SPARK_BF16, SPARK_FP8_E4M3 = 0, 1, 2
 SPARK_FILL_ZERO, SPARK_FILL_NEGINF = 0, 1
-SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS = 0, 1, 2
+SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS, SPARK_SHARED_CACHE = 0, 1, 2, 4
 
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",

@@ -61,6 +61,8 @@ struct AttnParams {
     const float* k1s;  // nullable: k1c is FP8 E4M3 and k1s[B][n_kv][cap] holds one scale per cached row
     const double* zs;  // nullable: Q(1 - k_attn / L_b) per sequence, precomputed by an earlier kernel
     int window, k_attn, dense;
+    int seg_mask;      // cache segment of (sequence b, KV head g) = (b n_kv + g) & seg_mask: all ones, or n_kv - 1 when the B
+                       // queries belong to one sequence and read one cache [n_kv][cap][.] (a chunk of a prompt; n_kv a power of two)
     float* o;
     float* theta;
     int32_t* count;
@@ -92,10 +94,13 @@ __device__ __forceinline__ float half_sum(float v) {   // sum over the 16 lanes 
     return v;
 }
 
-// AL: the segment-aligned cut is available (the host asks for it when the batch has enough segments).
+// MODE 0: flat cut of the token space; 1: segment-aligned cut (the host asks for it when the batch has enough segments);
+// 2: flat cut, all queries read one shared cache (a chunk of a prompt).
 // K1T: storage of the predictor slice k1c (KT, or FP8 E4M3 with one fp32 scale per cached row in p.k1s).
-template <typename KT, typename K1T, int GQ, bool AL>
+template <typename KT, typename K1T, int GQ, int MODE>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
+    constexpr bool AL = MODE == 1;      // segment-aligned cut
+    constexpr bool SH = MODE == 2;      // one cache shared by all queries (flat cut)
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int NS = p.B * p.n_kv;
     const int hd = p.hd, r = p.r, d2 = hd - r;
@@ -135,6 +140,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
         return n > p.cap ? static_cast<int>(p.cap) : n;
     };
     auto win_len = [&](int n) -> int { return (p.window > 0 && p.window < n) ? p.window : n; };
+    // cache rows of segment (sequence b, KV head g): sequence b's own cache, or the one cache all queries share
+    auto cseg = [&](int seg) -> int64_t { return static_cast<int64_t>(SH ? (seg & p.seg_mask) : seg); };
 
     if (!p.pre_stable) {   // lengths, queries and cache rows may all come from the kernel before this one
         dep_wait();
@@ -253,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             const int tb = static_cast<int>(f0 - sb);
             const int te = static_cast<int>((f1 < se ? f1 : se) - sb);
             const int lo = seq_len(seg0 / p.n_kv) - L;
-            const K1T* kbase = k1c + (static_cast<int64_t>(seg0) * p.cap + lo) * r;
+            const K1T* kbase = k1c + (cseg(seg0) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
             if (w0 < w1 && mma8) {          // rows w0 + mg and w0 + mg + 8, their 16-byte pieces mt and mt + 4
@@ -350,7 +357,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             float mx[GQ];
 #pragma unroll
             for (int hq = 0; hq < GQ; ++hq) { s1[hq] = 0.0; s2[hq] = 0.0; mx[hq] = -INFINITY; }
-            const K1T* kbase = k1c + (static_cast<int64_t>(seg) * p.cap + lo) * r;
+            const K1T* kbase = k1c + (cseg(seg) * p.cap + lo) * r;
             int w0, w1;
             warp_range(tb, te, w0, w1);
             const int jidx = ((hl >> 3) & 1) * 4 + ((hl >> 2) & 1) * 2 + ((hl >> 1) & 1);
@@ -371,7 +378,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
 #pragma unroll
                         for (int hrow = 0; hrow < 2; ++hrow) {
                             const int t = base + 16 * nb + mg + 8 * hrow;
-                            rs[nb][hrow] = (owner && t < w1) ? p.k1s[static_cast<int64_t>(seg) * p.cap + lo + t] : 0.f;
+                            rs[nb][hrow] = (owner && t < w1) ? p.k1s[cseg(seg) * p.cap + lo + t] : 0.f;
 #pragma unroll
                             for (int j = 0; j < 2; ++j) {
                                 if (nb == 0 && have_pre && ord == 0 && base == w0) w[0][2 * hrow + j] = wq[2 * hrow + j];
@@ -426,7 +433,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 [[maybe_unused]] float ksc = 1.f;
                 if constexpr (sizeof(K1T) == 1) {
                     const int tsc = tok0 + jidx;
-                    if ((hl & 1) == 0 && tsc < w1) ksc = p.k1s[static_cast<int64_t>(seg) * p.cap + lo + tsc];
+                    if ((hl & 1) == 0 && tsc < w1) ksc = p.k1s[cseg(seg) * p.cap + lo + tsc];
                 }
                 if (have_pre && ord == 0 && base == w0) {
 #pragma unroll
@@ -551,8 +558,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             __syncthreads();
             if (s_fail) return;
             if (ord == 0) p.trace.mark(2);
-            const KT* k2base = k2c + static_cast<int64_t>(seg) * p.cap * d2;
-            const KT* vbase = vc + static_cast<int64_t>(seg) * p.cap * hd;
+            const KT* k2base = k2c + cseg(seg) * p.cap * d2;
+            const KT* vbase = vc + cseg(seg) * p.cap * hd;
             // In this pass warp w serves query head w % GQ; the kWarps / GQ warps of a head split the
             // piece's tokens into contiguous runs (multiples of 32 tokens).
             constexpr int NSUB = kWarps / GQ;
@@ -748,10 +755,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     p.trace.mark(3);
 }
 
-template <typename KT, typename K1T, int GQ, bool AL>
+template <typename KT, typename K1T, int GQ, int MODE>
 int launch_al(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
     static bool configured[64] = {};
-    auto kern = attn_kernel<KT, K1T, GQ, AL>;
+    auto kern = attn_kernel<KT, K1T, GQ, MODE>;
     if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 8192) != cudaSuccess)
             return SPARK_ERR_CUDA;
@@ -768,9 +775,10 @@ int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) 
     // gives the segments 1/(blocks per segment) uneven shares of the streaming pass: worth it while a block's
     // share of that pass is short.
     const int ns = p.B * p.n_kv;
+    if (p.seg_mask != -1) return launch_al<KT, K1T, GQ, 2>(ctx, p, smem, stream);
     if (p.al_ok && ns >= kMinAlignedSegs && ns <= ctx->num_sms && ns <= kMaxAlignedSegs)
-        return launch_al<KT, K1T, GQ, true>(ctx, p, smem, stream);
-    return launch_al<KT, K1T, GQ, false>(ctx, p, smem, stream);
+        return launch_al<KT, K1T, GQ, 1>(ctx, p, smem, stream);
+    return launch_al<KT, K1T, GQ, 0>(ctx, p, smem, stream);
 }
 
 template <typename KT, typename K1T>
@@ -844,11 +852,14 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.window = static_cast<int>(window > 0x7fffffff ? 0x7fffffff : window);
     p.k_attn = static_cast<int>(k_attn > 0x7fffffff ? 0x7fffffff : k_attn);
     p.dense = (flags & SPARK_DENSE_LOADS) ? 1 : 0;
+    const bool shared = (flags & SPARK_SHARED_CACHE) != 0;
+    if (shared && (n_kv & (n_kv - 1)) != 0) return SPARK_ERR_UNSUPPORTED;
+    p.seg_mask = shared ? static_cast<int>(n_kv - 1) : -1;
     p.o = o; p.theta = theta; p.count = count; p.idx = idx; p.idx_cap = idx_cap;
     p.cells = reinterpret_cast<SumCell*>(ctx->scratch);
     p.lsum = lsum != nullptr ? lsum : reinterpret_cast<float*>(ctx->scratch + cells_b);
     p.defer = lsum != nullptr ? 1 : 0;
-    p.pre_stable = p.defer;
+    p.pre_stable = p.defer && !shared;      // a chunk's rows are all fresh from the kernel ahead
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;

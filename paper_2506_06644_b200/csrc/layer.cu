@@ -305,6 +305,7 @@ struct RopeParams {
     __nv_bfloat16* vc;
     const int32_t* ctx_len;
     int B, n_q, n_kv, hd, r;
+    int shared;              // 1: one cache [n_kv][cap][.] for all B tokens (consecutive tokens of one sequence)
     int64_t cap;
     float base, q_scale;
     double* zs;              // [B] out: Q(1 - k_attn / L_b) for the attention kernel that follows
@@ -333,7 +334,7 @@ __global__ void rope_append_kernel(const RopeParams p) {
         const float* src = p.qkv + (static_cast<int64_t>(b) * heads + h) * p.hd;
         if (h >= p.n_q + p.n_kv) {                       // value head: plain copy of two elements
             const int g = h - p.n_q - p.n_kv;
-            __nv_bfloat16* dst = p.vc + ((static_cast<int64_t>(b) * p.n_kv + g) * p.cap + pos) * p.hd;
+            __nv_bfloat16* dst = p.vc + ((static_cast<int64_t>(p.shared ? 0 : b) * p.n_kv + g) * p.cap + pos) * p.hd;
             dst[2 * pr] = __float2bfloat16_rn(src[2 * pr]);
             dst[2 * pr + 1] = __float2bfloat16_rn(src[2 * pr + 1]);
             continue;
@@ -358,7 +359,7 @@ __global__ void rope_append_kernel(const RopeParams p) {
             dst[ib] = rb * p.q_scale;
         } else {
             const int g = h - p.n_q;
-            const int64_t rowi = (static_cast<int64_t>(b) * p.n_kv + g) * p.cap + pos;
+            const int64_t rowi = (static_cast<int64_t>(p.shared ? 0 : b) * p.n_kv + g) * p.cap + pos;
             if (part0 == 0) {
                 __nv_bfloat16* dst = p.k1c + rowi * p.r;
                 dst[pi] = __float2bfloat16_rn(ra);
@@ -429,7 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
             const int pos = n - 1;
             if (head >= rp.n_q + rp.n_kv) {
                 const int gk = head - rp.n_q - rp.n_kv;
-                __nv_bfloat16* dst = rp.vc + ((static_cast<int64_t>(t) * rp.n_kv + gk) * rp.cap + pos) * hd;
+                __nv_bfloat16* dst = rp.vc + ((static_cast<int64_t>(rp.shared ? 0 : t) * rp.n_kv + gk) * rp.cap + pos) * hd;
                 dst[2 * q] = __float2bfloat16_rn(v[0]);
                 dst[2 * q + 1] = __float2bfloat16_rn(v[1]);
                 return;
@@ -448,7 +449,7 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
                 dst[pi + m / 2] = rb * rp.q_scale;
             } else {
                 const int gk = head - rp.n_q;
-                const int64_t rowi = (static_cast<int64_t>(t) * rp.n_kv + gk) * rp.cap + pos;
+                const int64_t rowi = (static_cast<int64_t>(rp.shared ? 0 : t) * rp.n_kv + gk) * rp.cap + pos;
                 __nv_bfloat16* dst = second ? rp.k2c + rowi * (hd - rp.r) : rp.k1c + rowi * rp.r;
                 dst[pi] = __float2bfloat16_rn(ra);
                 dst[pi + m / 2] = __float2bfloat16_rn(rb);
@@ -568,6 +569,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     rp.vc = static_cast<__nv_bfloat16*>(cache->vc);
     rp.ctx_len = ctx_len; rp.B = static_cast<int>(B); rp.n_q = static_cast<int>(cfg->n_q); rp.n_kv = static_cast<int>(cfg->n_kv);
     rp.hd = static_cast<int>(cfg->hd); rp.r = static_cast<int>(cfg->r_attn); rp.cap = cfg->cap;
+    rp.shared = (cfg->flags & SPARK_SHARED_CACHE) ? 1 : 0;
     rp.base = cfg->rope_base; rp.q_scale = 1.0f / std::sqrt(static_cast<float>(cfg->hd));
     if (cfg->r_attn > 128 || cfg->hd - cfg->r_attn > 128) return SPARK_ERR_UNSUPPORTED;
     for (int part = 0; part < 2; ++part) {
@@ -611,7 +613,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
 
     // 3. Spark attention over the cache (the new token included)
     rc = attn_launch(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd, cfg->r_attn,
-                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & SPARK_DENSE_LOADS, ao, lsum, nullptr, nullptr,
+                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & (SPARK_DENSE_LOADS | SPARK_SHARED_CACHE), ao, lsum, nullptr, nullptr,
                      nullptr, 0, nullptr, st);
     if (rc != SPARK_OK) return rc;
 

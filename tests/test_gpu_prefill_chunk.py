@@ -1,0 +1,89 @@
+"""GPU parity of the shared-cache mode (SPARK_SHARED_CACHE): the B tokens of a call are consecutive tokens of
+one sequence -- a chunk of its prompt -- appended to one cache, token b attending to the prompt and to the
+chunk's tokens up to itself.  The oracle is the decoder layer applied token by token."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spark_oracle as O
+from paper_2506_06644_b200 import binding as S
+from paper_2506_06644_b200 import synth
+from tests import parity
+from tests.test_gpu_layer import bf16_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = S.SparkContext(0, max_batch=64)
+    yield c
+    assert c.device_status() == S.SPARK_OK
+    c.close()
+
+
+@pytest.mark.parametrize("shape,T,L0,cap,window", [
+    (synth.TINY, 3, 40, 64, 0),                 # fused projection + rotary + append kernel (up to four tokens)
+    (synth.TINY, 7, 20, 64, 0),                 # five and more tokens: separate append kernel
+    (synth.TINY, 6, 50, 64, 16),                # local window sliding over the chunk
+    (synth.GEMMA2_2B, 8, 300, 512, 0),          # FFN of the chunk on the tcgen05 path
+    (synth.GEMMA2_2B, 16, 0, 64, 0),            # the largest chunk a layer call takes, starting the sequence (empty cache)
+])
+def test_chunk_of_a_prompt_equals_token_by_token_decoding(ctx, shape, T, L0, cap, window):
+    sh = shape
+    lw = synth.layer_weights(sh, 21, 0)
+    kv = synth.attn_inputs(1, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, cap, [max(L0, 1)], "bf16", seed=22)
+    h0 = synth.normal_f32((T, sh.d), 23, 60)
+    dev = dict(norm1=torch.from_numpy(lw.norm1).cuda(), norm2=torch.from_numpy(lw.norm2).cuda(),
+               Wqkv=bf16_dev(lw.Wqkv_bits), Wo=bf16_dev(lw.Wo_bits), K1t=bf16_dev(lw.K1t_bits),
+               K2t=bf16_dev(lw.K2t_bits), Vt=bf16_dev(lw.Vt_bits))
+    cache = dict(k1c=bf16_dev(kv.k1c_bits[0]), k2c=bf16_dev(kv.k2c_bits[0]), vc=bf16_dev(kv.vc_bits[0]))     # [n_kv][cap][.]
+    cfg = dict(d=sh.d, d_ff=sh.d_ff, r_ff=sh.r_ff, k_ff=sh.k_ff, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+               k_attn=sh.k_attn, window=window, cap=cap, rms_eps=1e-6, rope_base=10000.0, flags=S.SPARK_SHARED_CACHE)
+    layer = S.make_layer(dev, cfg, cache)
+    h = torch.from_numpy(h0).cuda()
+    cl = torch.tensor([L0 + t + 1 for t in range(T)], dtype=torch.int32, device="cuda")
+    nqkv = (sh.n_q + 2 * sh.n_kv) * sh.hd
+    scratch = torch.empty(T * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device="cuda")
+    S.spark_layer_decode(ctx, layer, cl, h, T, scratch)
+    torch.cuda.synchronize()
+    got = h.cpu().numpy()
+
+    W = {"norm1": lw.norm1, "norm2": lw.norm2, "Wqkv": synth.bf16_bits_to_f32(lw.Wqkv_bits),
+         "Wo": synth.bf16_bits_to_f32(lw.Wo_bits), "K1t": synth.bf16_bits_to_f32(lw.K1t_bits),
+         "K2t": synth.bf16_bits_to_f32(lw.K2t_bits), "Vt": synth.bf16_bits_to_f32(lw.Vt_bits)}
+    kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+    vc = kv.vc[0].astype(np.float64)
+    for t in range(T):                           # the oracle appends token t's row before token t + 1 reads the cache
+        ref = O.decoder_layer(h0[t], W, kc, vc, L0 + t + 1, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+                              k_attn=sh.k_attn, r_ff=sh.r_ff, k_ff=sh.k_ff, window=window)
+        parity.check_output(got[t], ref["h"], "bf16", f"token {t}")
+        parity.check_output(got[t] - h0[t], ref["h"] - h0[t], "bf16", f"token {t} (update only)")
+    # the chunk's rows are in the one cache, the prompt's rows untouched
+    k1 = cache["k1c"].float().cpu().numpy()
+    v = cache["vc"].float().cpu().numpy()
+    for t in range(T):
+        n = L0 + t + 1
+        np.testing.assert_allclose(k1[:, n - 1], kc[:, n - 1, : sh.r_attn], rtol=2 ** -7, atol=1e-4 * parity.rms(kc[:, n - 1]))
+        np.testing.assert_allclose(v[:, n - 1], vc[:, n - 1], rtol=2 ** -7, atol=1e-4 * parity.rms(vc[:, n - 1]))
+    if L0 > 0:
+        assert np.array_equal(k1[:, :L0], kv.k1c[0][:, :L0])
+
+
+def test_attention_queries_sharing_one_cache(ctx):
+    # spark_attn_decode alone: eight queries over one cache, query b seeing the first L0 + b + 1 rows
+    B, n_q, n_kv, hd, r, cap, L0, k_attn = 8, 8, 4, 64, 32, 256, 200, 24
+    kv = synth.attn_inputs(1, n_q, n_kv, hd, r, cap, [cap], "bf16", seed=31)
+    q = synth.normal_f32((B, n_q, hd), 32, 0) * hd ** -0.5
+    lens = [L0 + b + 1 for b in range(B)]
+    o = torch.empty(B, n_q, hd, device="cuda")
+    theta = torch.empty(B, n_q, device="cuda")
+    S.spark_attn_decode(ctx, torch.from_numpy(q).cuda(), bf16_dev(kv.k1c_bits[0]), bf16_dev(kv.k2c_bits[0]), bf16_dev(kv.vc_bits[0]),
+                        S.SPARK_BF16, B, n_q, n_kv, hd, r, cap, torch.tensor(lens, dtype=torch.int32, device="cuda"), 0, k_attn,
+                        S.SPARK_SHARED_CACHE, o, theta, None, None, 0)
+    torch.cuda.synchronize()
+    kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+    vc = kv.vc[0].astype(np.float64)
+    for b in range(B):
+        ref = O.spark_attention(q[b].astype(np.float64), kc, vc, lens[b], k_attn, r)
+        parity.check_output(o[b].cpu().numpy().reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"query {b}")
