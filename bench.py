@@ -254,9 +254,9 @@ def run_spark(args):
     scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
-    # QKV (+ rotary, append: a kernel of their own for B >= 5), attention, output projection, FFN (four kernels on the
-    # tcgen05 chunk path for B >= 5: prep, scores, activation, output)
-    kernels_per_layer = 4 if B <= 4 else 8
+    # QKV (+ rotary, append: a kernel of their own for B >= 5), attention, output projection, FFN; for B >= 5 the projections
+    # are two kernels each (prep, tcgen05 GEMM) and the FFN four (prep, scores, activation, output)
+    kernels_per_layer = 4 if B <= 4 else 10
 
     def stack(which):
         for lay in layers:

@@ -43,6 +43,9 @@ struct GemvArgs {
     size_t zero_bytes;
 };
 int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
+// The same product for 5..16 tokens and bf16 weights as a TMA-fed tcgen05 GEMM (gemm_tc.cu); SPARK_ERR_WORKSPACE = shape or
+// workspace not served (n_in % 64, n_out % 128, room for the split input behind the attention's cells).
+int gemm_tc_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 
 // Spark attention; zs (nullable) holds Q(1 - k_attn / L_b) per sequence when an earlier kernel of the
 // same stream has already computed it.  With lsum != nullptr the kernel leaves o unnormalised (the

@@ -488,6 +488,10 @@ int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
     const size_t limit = static_cast<size_t>(ctx->max_smem_optin - 1024);
     if (static_cast<size_t>(a.n_in) * 4 > limit) return SPARK_ERR_UNSUPPORTED;
+    if (a.B >= 5 && a.wdtype == SPARK_BF16) {      // five and more tokens: a real GEMM, on the tcgen05 tensor cores when the shape allows
+        const int rc = gemm_tc_launch(ctx, a, stream);
+        if (rc != SPARK_ERR_WORKSPACE) return rc;
+    }
     // Tokens are processed in sub-batches whose inputs fit in shared memory together.
     int64_t done = 0;
     while (done < a.B) {
