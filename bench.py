@@ -657,10 +657,9 @@ def other_workloads(torch, S, peak, steps, warmup):
                 "dense_loads_us_per_launch": res[1], "speedup_vs_dense_loads": res[1] / res[0]})
     ctx.close()
 
-    # -- the same eight layers over chunks of a prompt: 16 consecutive tokens of ONE sequence per call (SPARK_SHARED_CACHE),
-    #    appended behind 8192 - 16 cached tokens, every token attending causally; per-layer caches [n_kv][L][.]
-    T = 16
-    ctx = S.SparkContext(dev.index, max_batch=T, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
+    # -- the same eight layers over chunks of a prompt: T consecutive tokens of ONE sequence per call (SPARK_SHARED_CACHE),
+    #    appended behind 8192 - T cached tokens, every token attending causally; per-layer caches [n_kv][L][.]
+    ctx = S.SparkContext(dev.index, max_batch=64, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
     ctx.set_launch_overlap(True)
     chunk_layers = []
     for l, (_, wts, cache) in enumerate(stacks[0]):
@@ -669,18 +668,19 @@ def other_workloads(torch, S, peak, steps, warmup):
                    k_attn=sh.k_attn, window=4096 if l % 2 == 0 else 0, cap=L, rms_eps=1e-6, rope_base=10000.0,
                    flags=S.SPARK_SHARED_CACHE)
         chunk_layers.append((S.make_layer(wts, cfg, one), wts, one))
-    hc = torch.randn(T, sh.d, device=dev, generator=gen)
-    clc = torch.arange(L - T + 1, L + 1, dtype=torch.int32, device=dev)
-    scratch_c = torch.empty(T * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device=dev)
+    for T in (16, 64):
+        hc = torch.randn(T, sh.d, device=dev, generator=gen)
+        clc = torch.arange(L - T + 1, L + 1, dtype=torch.int32, device=dev)
+        scratch_c = torch.empty(T * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device=dev)
 
-    def chunk_calls():
-        for lay in chunk_layers:
-            S.spark_layer_decode(ctx, lay[0], clc, hc, T, scratch_c)
-    us_chunk = time_graph(chunk_calls, nl)
-    assert ctx.device_status() == S.SPARK_OK
-    out.append({"workload": f"spark_layer_decode over a chunk of a prompt: {T} consecutive tokens of one sequence per call "
-                            f"(shared cache, causal), context {L}, {nl} layers: per layer",
-                "us_per_launch": us_chunk, "us_per_token_per_layer": us_chunk / T})
+        def chunk_calls():
+            for lay in chunk_layers:
+                S.spark_layer_decode(ctx, lay[0], clc, hc, T, scratch_c)
+        us_chunk = time_graph(chunk_calls, nl)
+        assert ctx.device_status() == S.SPARK_OK
+        out.append({"workload": f"spark_layer_decode over a chunk of a prompt: {T} consecutive tokens of one sequence per call "
+                                f"(shared cache, causal), context {L}, {nl} layers: per layer",
+                    "us_per_launch": us_chunk, "us_per_token_per_layer": us_chunk / T})
     ctx.close()
     del stacks, chunk_layers
 

@@ -258,7 +258,7 @@ int spark_attn_decode_fp8k(spark_ctx* ctx, const float* q, const void* k1c, cons
 
 /* ---- dense GEMV (the projections the method leaves dense: Table "FLOPs per token") ----
  * y[b][n_out] = Wt[n_out][n_in] . x[b][n_in] (+ y_add[b][n_out] if y_add != NULL).
- * Wt of dtype wdtype, output-major; n_in % 8 == 0; 1 <= B <= 16.  y_add may equal y. */
+ * Wt of dtype wdtype, output-major; n_in % 8 == 0; 1 <= B <= 64.  y_add may equal y. */
 int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const void* Wt, int wdtype,
                      int64_t n_in, int64_t n_out, const float* y_add, float* y, void* stream);
 
@@ -270,7 +270,7 @@ int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const void* Wt, 
  * With SPARK_SHARED_CACHE in cfg->flags the B tokens are consecutive tokens of one sequence (a chunk of
  * its prompt): the caches are [n_kv][cap][.], token b is appended at row ctx_len[b]-1 and attends to rows
  * [0, ctx_len[b]); ctx_len[b] = L0 + b + 1 gives what decoding the chunk token by token gives (n_kv a
- * power of two).  1 <= B <= 16 either way.
+ * power of two).  1 <= B <= 64 either way.
  * All pointers inside the structs are device pointers; the structs themselves are host objects. */
 typedef struct spark_layer_weights {
     const float* norm1;   /* [d]                          */
@@ -299,7 +299,7 @@ typedef struct spark_kv_cache {
 } spark_kv_cache;
 
 /* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2 + n_q) fp32 values, 16-byte aligned, caller-owned, contents
- * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 16.  Four kernels are
+ * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 64.  Four kernels are
  * enqueued for B <= 4: QKV projection with position encoding and cache append, attention, output projection,
  * FFN; five for B >= 5, where the position encoding and the append follow the projection as a kernel of
  * their own. */

@@ -1,9 +1,9 @@
-// Dense projection for 5..16 tokens with bf16 weights on the fifth-generation tensor cores:
+// Dense projection for 5..64 tokens with bf16 weights on the fifth-generation tensor cores:
 // y[b][:] = Wt . f(x[b][:]) (+ y_add[b][:]), f = optional division per group, optional RMSNorm -- the
 // decoder layer's QKV and output projections for a batch or a chunk of a prompt.  Two kernels:
-//   prep   f(x) -> two bf16 terms (x = hi + lo, 16 mantissa bits) in the workspace, padded to 16 tokens;
+//   prep   f(x) -> two bf16 terms (x = hi + lo, 16 mantissa bits) in the workspace, padded to a multiple of 16 tokens;
 //          y = y_add (or 0); the caller's clear-region side job
-//   gemm   M = 128 output rows per tile, N = 2 x 16 (hi rows, lo rows of the token operand), K split over
+//   gemm   M = 128 output rows per tile, N = 2 x tokens (hi rows, lo rows of the token operand), K split over
 //          the blocks of a tile so that every SM has one block; TMA-fed tcgen05.mma, accumulator in tensor
 //          memory, epilogue adds the two halves and reduces into y (fp32 reductions)
 // The weights do not depend on the kernel ahead: their first stages are requested before
@@ -16,14 +16,16 @@ using namespace spark::tc;
 
 namespace {
 
-constexpr int kGemmTok = 16;                                   // token rows of the padded operand
+constexpr int kGemmMaxTok = 64;
 constexpr int kGemmRows = 128;
-constexpr int kGemmStages = 8;
 constexpr int kGemmWBytes = kGemmRows * kChunk * 2;            // 16 KB of weights per stage
-constexpr int kGemmXBytes = kGemmTok * kChunk * 2;             // 2 KB per term of X per stage
-constexpr int kGemmStageBytes = kGemmWBytes + 2 * kGemmXBytes; // 20 KB
-constexpr uint32_t kGemmCols = 32;                             // tensor-memory columns: hi | lo
 constexpr int kGemmPrepSplit = 4;
+// TOK = token rows of the operand tile a stage has room for (16: 8 stages of 20 KB; 64: 6 stages of 32 KB)
+template <int TOK> struct GemmCfg {
+    static constexpr int kStages = TOK <= 16 ? 8 : 6;
+    static constexpr int kStageBytes = kGemmWBytes + 2 * TOK * kChunk * 2;
+    static constexpr uint32_t kCols = TOK <= 16 ? 32 : 128;    // tensor-memory columns: hi | lo
+};
 
 struct GemmParams {
     const float* x;
@@ -36,7 +38,8 @@ struct GemmParams {
     int x_div_group;
     uint4* zero_ptr;
     int zero_n16;
-    __nv_bfloat16* xhi;      // [kGemmTok][n_in]
+    int ntok;                // B rounded up to a multiple of 16: rows of the operand boxes, half of the MMA's N
+    __nv_bfloat16* xhi;      // [ntok][n_in]
     __nv_bfloat16* xlo;
     int ksplit, nchunks;
     WsHeader* hdr;
@@ -106,6 +109,7 @@ __global__ void __launch_bounds__(256) gemm_tc_prep_kernel(const GemmParams p) {
     }
 }
 
+template <int TOK>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_xhi,
                const __grid_constant__ CUtensorMap map_xlo) {
@@ -115,6 +119,9 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_w, co
     const int tile = blockIdx.x / p.ksplit, ks = blockIdx.x - tile * p.ksplit;
     const int c0 = static_cast<int>(static_cast<int64_t>(ks) * p.nchunks / p.ksplit), c1 = static_cast<int>(static_cast<int64_t>(ks + 1) * p.nchunks / p.ksplit);
     const int nch = c1 - c0, row0 = tile * kGemmRows;
+    constexpr int kGemmStages = GemmCfg<TOK>::kStages, kGemmStageBytes = GemmCfg<TOK>::kStageBytes;
+    constexpr uint32_t kGemmCols = GemmCfg<TOK>::kCols;
+    const uint32_t xbytes = static_cast<uint32_t>(p.ntok) * kChunk * 2;         // one term of one chunk of X
     const uint32_t base = tc_setup<kGemmStages>(sh, tc_raw, kGemmCols);
     const uint32_t tmem = sh.tmem;
     volatile int* abort_flag = &sh.abort_flag;
@@ -128,14 +135,14 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_w, co
             auto load_w = [&](int i) {
                 const int s = i % kGemmStages;
                 const uint32_t bar = smem_addr(&sh.full[s]);
-                mbar_expect_tx(bar, kGemmStageBytes);
+                mbar_expect_tx(bar, kGemmWBytes + 2 * xbytes);
                 tma_load_2d(base + s * kGemmStageBytes, &map_w, bar, (c0 + i) * kChunk, row0);
             };
             auto load_x = [&](int i) {
                 const int s = i % kGemmStages;
                 const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kGemmStageBytes + kGemmWBytes;
                 tma_load_2d(dst, &map_xhi, bar, (c0 + i) * kChunk, 0);
-                tma_load_2d(dst + kGemmXBytes, &map_xlo, bar, (c0 + i) * kChunk, 0);     // lo rows right behind the hi rows
+                tma_load_2d(dst + xbytes, &map_xlo, bar, (c0 + i) * kChunk, 0);          // lo rows right behind the hi rows
             };
             const int pre = min(nch, kGemmStages);
             for (int i = 0; i < pre; ++i) load_w(i);      // the weights do not depend on the kernel ahead
@@ -152,7 +159,7 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_w, co
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc(128, 2 * kGemmTok, false);
+            const uint32_t idesc = instr_desc(128, 2 * p.ntok, false);
             bool ok = true;
             for (int i = 0; i < nch && ok; ++i) {
                 const int s = i % kGemmStages;
@@ -172,12 +179,24 @@ gemm_tc_kernel(const GemmParams p, const __grid_constant__ CUtensorMap map_w, co
         dep_wait();
         if (nch > 0 && __all_sync(kFull, mbar_wait(smem_addr(&sh.accum), 0u, abort_flag))) {
             tc_fence_after();
-            float v[32];
-            tmem_ld32(tmem + (static_cast<uint32_t>(q * 32) << 16), v);       // columns 0..15 hi, 16..31 lo
+            const uint32_t taddr = tmem + (static_cast<uint32_t>(q * 32) << 16);
             float* ycol = p.y + row0 + q * 32 + lane;
+            float v[32];
+            if (TOK <= 16) {
+                tmem_ld32(taddr, v);                                              // columns 0..15 hi, 16..31 lo
 #pragma unroll
-            for (int n = 0; n < kGemmTok; ++n)
-                if (n < p.B) atomicAdd(ycol + static_cast<int64_t>(n) * p.n_out, v[n] + v[kGemmTok + n]);
+                for (int n = 0; n < 16; ++n)
+                    if (n < p.B) atomicAdd(ycol + static_cast<int64_t>(n) * p.n_out, v[n] + v[16 + n]);
+            } else {
+                float w[32];
+                for (int hb = 0; hb * 32 < p.B; ++hb) {
+                    tmem_ld32(taddr + hb * 32, v);
+                    tmem_ld32(taddr + p.ntok + hb * 32, w);
+#pragma unroll
+                    for (int n = 0; n < 32; ++n)
+                        if (hb * 32 + n < p.B) atomicAdd(ycol + static_cast<int64_t>(hb * 32 + n) * p.n_out, v[n] + w[n]);
+                }
+            }
         }
     }
     tc_finish(sh, kGemmCols, p.hdr);
@@ -189,14 +208,16 @@ namespace spark {
 
 // SPARK_ERR_WORKSPACE = shape or workspace not served by this path (the caller falls back).
 int gemm_tc_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
-    if (a.wdtype != SPARK_BF16 || a.B < 5 || a.B > kGemmTok || a.n_in % kChunk != 0 || a.n_out % kGemmRows != 0) return SPARK_ERR_WORKSPACE;
+    if (a.wdtype != SPARK_BF16 || a.B < 5 || a.B > kGemmMaxTok || a.n_in % kChunk != 0 || a.n_out % kGemmRows != 0) return SPARK_ERR_WORKSPACE;
+    const int ntok = static_cast<int>((a.B + 15) & ~15);
     if ((reinterpret_cast<uintptr_t>(a.Wt) & 15u) != 0 || (reinterpret_cast<uintptr_t>(a.y) & 15u) != 0 ||
         (a.y_add != nullptr && (reinterpret_cast<uintptr_t>(a.y_add) & 15u) != 0))
         return SPARK_ERR_WORKSPACE;
     // the split input sits behind the attention's cells, where the FFN chunk path keeps its own (neither outlives its call)
-    const size_t xb = round_up(static_cast<size_t>(kGemmTok) * a.n_in * 2, 1024);
+    const size_t xb = round_up(static_cast<size_t>(ntok) * a.n_in * 2, 1024);
     if (ctx->scratch == nullptr || ctx->scratch_bytes < kAttnCellBytes + 2 * xb) return SPARK_ERR_WORKSPACE;
-    const size_t smem = static_cast<size_t>(kGemmStages) * kGemmStageBytes + 1024;
+    const size_t smem = (ntok <= 16 ? static_cast<size_t>(GemmCfg<16>::kStages) * GemmCfg<16>::kStageBytes
+                                    : static_cast<size_t>(GemmCfg<64>::kStages) * GemmCfg<64>::kStageBytes) + 1024;
     if (smem + sizeof(TcShared) + 64 > static_cast<size_t>(ctx->max_smem_optin)) return SPARK_ERR_WORKSPACE;
 
     GemmParams p;
@@ -205,6 +226,7 @@ int gemm_tc_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
     p.y_add = a.y_add; p.y = a.y;
     p.x_div = a.x_div; p.x_div_group = static_cast<int>(a.x_div ? a.x_div_group : 1);
     p.zero_ptr = static_cast<uint4*>(a.zero_ptr); p.zero_n16 = static_cast<int>(a.zero_bytes / 16);
+    p.ntok = ntok;
     p.xhi = reinterpret_cast<__nv_bfloat16*>(ctx->scratch + kAttnCellBytes);
     p.xlo = reinterpret_cast<__nv_bfloat16*>(ctx->scratch + kAttnCellBytes + xb);
     const int tiles = static_cast<int>(a.n_out / kGemmRows);
@@ -214,18 +236,19 @@ int gemm_tc_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
     p.hdr = ctx->hdr;
 
     CUtensorMap m_w, m_xhi, m_xlo;
-    if (!make_map(&m_w, a.Wt, a.n_out, a.n_in, a.n_in, kGemmRows, true) || !make_map(&m_xhi, p.xhi, kGemmTok, a.n_in, a.n_in, kGemmTok, false) ||
-        !make_map(&m_xlo, p.xlo, kGemmTok, a.n_in, a.n_in, kGemmTok, false))
+    if (!make_map(&m_w, a.Wt, a.n_out, a.n_in, a.n_in, kGemmRows, true) || !make_map(&m_xhi, p.xhi, ntok, a.n_in, a.n_in, ntok, false) ||
+        !make_map(&m_xlo, p.xlo, ntok, a.n_in, a.n_in, ntok, false))
         return SPARK_ERR_WORKSPACE;
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return SPARK_ERR_CUDA;
+    const void* kern = ntok <= 16 ? reinterpret_cast<const void*>(gemm_tc_kernel<16>) : reinterpret_cast<const void*>(gemm_tc_kernel<64>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess) return SPARK_ERR_CUDA;
     {
         void* args[] = {&p};
-        if (launch_kernel(ctx, reinterpret_cast<const void*>(gemm_tc_prep_kernel), kGemmTok * kGemmPrepSplit, 256, 0, stream, false, args) != cudaSuccess)
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(gemm_tc_prep_kernel), static_cast<unsigned>(ntok * kGemmPrepSplit), 256, 0, stream, false, args) != cudaSuccess)
             return SPARK_ERR_CUDA;
     }
     {
         void* args[] = {&p, &m_w, &m_xhi, &m_xlo};
-        if (launch_kernel(ctx, reinterpret_cast<const void*>(gemm_tc_kernel), static_cast<unsigned>(tiles * p.ksplit), kTcThreads, smem, stream, false, args) != cudaSuccess)
+        if (launch_kernel(ctx, kern, static_cast<unsigned>(tiles * p.ksplit), kTcThreads, smem, stream, false, args) != cudaSuccess)
             return SPARK_ERR_CUDA;
     }
     return SPARK_OK;

@@ -479,7 +479,7 @@ namespace spark {
 
 int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
     if (ctx == nullptr || a.x == nullptr || a.Wt == nullptr || a.y == nullptr) return SPARK_ERR_INVALID_ARG;
-    if (a.B < 1 || a.B > 16 || a.n_in < 8 || a.n_out < 1) return SPARK_ERR_INVALID_ARG;
+    if (a.B < 1 || a.B > 64 || a.n_in < 8 || a.n_out < 1) return SPARK_ERR_INVALID_ARG;
     if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16) return SPARK_ERR_UNSUPPORTED;
     if ((a.n_in & 7) != 0 || !aligned16(a.x) || !aligned16(a.Wt) || !aligned16(a.norm_w)) return SPARK_ERR_UNSUPPORTED;
     if (a.x_div != nullptr && (a.x_div_group < 4 || (a.x_div_group & 3) != 0 || a.n_in % a.x_div_group != 0)) return SPARK_ERR_UNSUPPORTED;
@@ -546,7 +546,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     if (ctx == nullptr || w == nullptr || cfg == nullptr || cache == nullptr || ctx_len == nullptr || h == nullptr ||
         scratch == nullptr)
         return SPARK_ERR_INVALID_ARG;
-    if (B < 1 || B > 16) return SPARK_ERR_INVALID_ARG;
+    if (B < 1 || B > 64) return SPARK_ERR_INVALID_ARG;
     if (((cfg->n_q + 2 * cfg->n_kv) * cfg->hd + 2 * cfg->n_q * cfg->hd + cfg->d) % 2 != 0) return SPARK_ERR_UNSUPPORTED;
     if (w->norm1 == nullptr || w->norm2 == nullptr || w->Wqkv == nullptr || w->Wo == nullptr || w->K1t == nullptr ||
         w->K2t == nullptr || w->Vt == nullptr || cache->k1c == nullptr || cache->k2c == nullptr || cache->vc == nullptr)

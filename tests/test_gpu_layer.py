@@ -26,7 +26,9 @@ def bf16_dev(bits):
 @pytest.mark.parametrize("wd", ["bf16", "f32"])
 @pytest.mark.parametrize("B,n_in,n_out", [(1, 2304, 4096), (1, 2048, 2304), (4, 256, 1000), (16, 3584, 300),
                                           (7, 64, 5), (2, 1024, 20000),
-                                          (5, 2304, 4096), (12, 2048, 2304),      # five and more tokens: tensor cores
+                                          (5, 2304, 4096), (12, 2048, 2304),      # five and more tokens: tensor cores (tcgen05 GEMM)
+                                          (20, 2304, 4096), (64, 2048, 2304),     # more than one sixteen-token group
+                                          (9, 96, 200), (40, 96, 200),            # shapes the GEMM does not take: mma.sync kernel
                                           (8, 264, 500)])                          # ... unless n_in % 32 != 0
 def test_dense_gemv(ctx, wd, B, n_in, n_out):
     W = synth.normal_f32((n_out, n_in), 3, 1, 1 / np.sqrt(n_in))
@@ -92,6 +94,7 @@ def run_layer(ctx, sh, B, cap, lens, seed, window=0, flags=0):
     (synth.GEMMA2_2B, 2, 1024, [700, 1024], 512),
     (synth.TINY, 5, 64, [64, 3, 40, 17, 1], 0),                    # five and more tokens: tensor-core projections
     (synth.GEMMA2_2B, 6, 512, [512, 300, 77, 1, 450, 260], 0),
+    (synth.GEMMA2_2B, 20, 256, [256, 200, 77, 1, 150, 60, 3, 90, 256, 17, 100, 101, 102, 33, 64, 65, 128, 129, 250, 5], 128),   # more than sixteen sequences
     (synth.GEMMA2_9B, 1, 1024, [1024], 0),                         # 16 query / 8 KV heads, d_ff 14336
     (synth.GEMMA2_9B, 2, 512, [512, 100], 256),
 ])

@@ -27,7 +27,9 @@ def ctx():
     (synth.TINY, 7, 20, 64, 0),                 # five and more tokens: separate append kernel
     (synth.TINY, 6, 50, 64, 16),                # local window sliding over the chunk
     (synth.GEMMA2_2B, 8, 300, 512, 0),          # FFN of the chunk on the tcgen05 path
-    (synth.GEMMA2_2B, 16, 0, 64, 0),            # the largest chunk a layer call takes, starting the sequence (empty cache)
+    (synth.GEMMA2_2B, 16, 0, 64, 0),            # a chunk that starts the sequence (empty cache)
+    (synth.GEMMA2_2B, 64, 100, 256, 0),         # the largest chunk a layer call takes
+    (synth.TINY, 20, 10, 64, 0),                # more than sixteen tokens on the fallback kernels (shape not served by the GEMMs)
 ])
 def test_chunk_of_a_prompt_equals_token_by_token_decoding(ctx, shape, T, L0, cap, window):
     sh = shape
