@@ -816,6 +816,12 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     if (!aligned16(q) || !aligned16(k1c) || !aligned16(k2c) || !aligned16(vc) || !aligned16(o)) return SPARK_ERR_UNSUPPORTED;
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
 
+    if ((flags & SPARK_SHARED_CACHE) && !(flags & SPARK_DENSE_LOADS) && B >= 32 && kvdtype == SPARK_BF16 && k1s == nullptr && idx == nullptr) {
+        // a long chunk of a prompt: the predictor scores of all its queries as one GEMM per KV head (measured: pays from
+        // about 32 tokens on; shorter chunks stream the slice per query out of L2 as fast)
+        const int rc = attn_chunk_launch(ctx, q, k1c, k2c, vc, B, n_q, n_kv, hd, r, cap, ctx_len, zs, window, k_attn, o, lsum, theta, count, st);
+        if (rc != SPARK_ERR_WORKSPACE) return rc;
+    }
     const int grid = ctx->num_sms;
     const int64_t span = (window > 0 && window < cap) ? window : cap;          // longest window of a sequence
     int64_t ntok = (B * n_kv * span + grid - 1) / grid + 1;                  // tokens one block may own (equal flat ranges)

@@ -1,0 +1,540 @@
+// Spark attention (Section 2.2, Eq. 7) for a chunk of a prompt: T consecutive tokens of one sequence, all
+// reading one cache, token t seeing rows [lo_t, n_t).  Here the predictor scores of all of the chunk's queries
+// against a cached row are one row of a GEMM -- S[j][(t, head)] = k1c[j] . q1[t, head] -- so every cached row of
+// the predictor slice is read once for the whole chunk instead of once per query, and the product runs on the
+// fifth-generation tensor cores.  Three kernels, ordered by the stream (no block waits on another block):
+//   prep    q[:, :, :r] -> two bf16 terms (hi + lo) as operand rows per KV head; Q(1 - k/L_t), row ranges
+//   scores  per KV head: S = k1c . Q1^T, M = 128 cached rows per tile, N = 2 x (tokens x heads per KV head), K = r;
+//           TMA-fed tcgen05.mma into double-buffered tensor-memory accumulators; eight epilogue warps add the two
+//           halves of the accumulator and write S column-major
+//   select  one block per (token, query head): sums of its column over the rows it may see -> theta (Eq. 10/11),
+//           survivors, softmax over the survivors, softplus gate from the k2c rows, weighted sum of the vc rows
+//           (only the survivors' rows are read)
+// Same pipeline skeleton and bounded waits as the other tensor-core kernels (tc_common.cuh).
+#include "kernels.h"
+#include "tc_common.cuh"
+
+using namespace spark;
+using namespace spark::tc;
+
+namespace {
+
+constexpr int kColMax = 128;          // (token, head-in-group) columns per KV head
+constexpr int kSelThreads = 256;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kListCap = 512;         // survivors a warp of the select kernel lists before it gathers them
+
+struct ChunkParams {
+    const float* q;            // [T][n_q][hd]
+    const __nv_bfloat16* k2c;  // [n_kv][cap][hd - r]
+    const __nv_bfloat16* vc;   // [n_kv][cap][hd]
+    const int32_t* ctx_len;    // [T]
+    const double* zs_in;       // nullable: Q(1 - k_attn / L_t) per token from an earlier kernel
+    int T, n_q, n_kv, gq, hd, r, window, k_attn;
+    int ncol, ncolp;           // T * gq, rounded up to a multiple of 16
+    int64_t cap;
+    float* o;                  // [T][n_q][hd], normalised
+    float* lsum;               // nullable: [T][n_q] = 1 (0 for an empty selection): the caller divides by it
+    float* theta;              // nullable [T][n_q]
+    int32_t* count;            // nullable [T][n_q]
+    // workspace
+    double* zt;                // [T]
+    int* range;                // [T][2] = lo_t, n_t
+    __nv_bfloat16* qhi;        // [n_kv][kColMax][r]
+    __nv_bfloat16* qlo;
+    float* S;                  // [n_kv][kColMax][scap]
+    int64_t scap;              // column stride of S: cap + 32, so that the columns' lines do not all fall on the same slices
+    WsHeader* hdr;
+};
+
+__device__ __forceinline__ void token_range(const ChunkParams& p, int t, int& lo, int& n) {
+    n = p.ctx_len[t];
+    n = n < 1 ? 1 : (n > p.cap ? static_cast<int>(p.cap) : n);
+    lo = (p.window > 0 && p.window < n) ? n - p.window : 0;
+}
+
+// ---- prep: one block per (KV head, column) ---------------------------------------------------------------------
+__global__ void __launch_bounds__(128) attn_chunk_prep_kernel(const ChunkParams p) {
+    const int g = blockIdx.x / kColMax, col = blockIdx.x % kColMax, tid = threadIdx.x;
+    dep_wait();
+    dep_trigger();
+    if (blockIdx.x == 0) {
+        for (int t = tid; t < p.T; t += 128) {
+            int lo, n;
+            token_range(p, t, lo, n);
+            p.range[2 * t] = lo;
+            p.range[2 * t + 1] = n;
+            const int L = n - lo;
+            p.zt[t] = p.zs_in != nullptr ? p.zs_in[t]
+                                         : (p.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
+        }
+    }
+    if (col >= p.ncolp) return;                 // rows the operand boxes never touch
+    __nv_bfloat16* hi = p.qhi + (static_cast<int64_t>(g) * kColMax + col) * p.r;
+    __nv_bfloat16* lo = p.qlo + (static_cast<int64_t>(g) * kColMax + col) * p.r;
+    const int t = col / p.gq, hq = col - t * p.gq;
+    for (int i = tid; i < p.r; i += 128) {
+        float v = 0.f;
+        if (col < p.ncol) v = p.q[(static_cast<int64_t>(t) * p.n_q + g * p.gq + hq) * p.hd + i];
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi[i] = h;
+        lo[i] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+}
+
+// ---- scores: S = k1c . Q1^T per KV head, 128 cached rows per tile ------------------------------------------------------
+constexpr int kChunkStages = 2;
+constexpr int kChunkABytes = 2 * 128 * kChunk * 2;           // up to two K chunks of 128 rows x 128 bytes
+constexpr int kChunkBBytes = 2 * 2 * kColMax * kChunk * 2;   // per K chunk: hi rows, lo rows of the query operand
+constexpr int kChunkStageBytes = kChunkABytes + kChunkBBytes;
+constexpr uint32_t kChunkCols = 512;                         // two accumulators of 128 rows x (hi | lo) columns
+
+struct ChunkShared {
+    unsigned long long full[kChunkStages], empty[kChunkStages];
+    unsigned long long acc_full[2], acc_empty[2];
+    uint32_t tmem;
+    int abort_flag;
+    int n_max;
+};
+constexpr int kChunkThreads = 64 + 8 * 32;      // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..9: epilogue
+
+__global__ void __launch_bounds__(kChunkThreads, 1)
+attn_chunk_scores_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap map_k1, const __grid_constant__ CUtensorMap map_qhi,
+                         const __grid_constant__ CUtensorMap map_qlo) {
+    extern __shared__ unsigned char tc_raw[];
+    __shared__ ChunkShared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nkc = p.r / kChunk;
+    if (tid == 0) {
+        for (int s = 0; s < kChunkStages; ++s) {
+            mbar_init(smem_addr(&sh.full[s]), 1u);
+            mbar_init(smem_addr(&sh.empty[s]), 1u);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_addr(&sh.acc_full[b]), 1u);
+            mbar_init(smem_addr(&sh.acc_empty[b]), 1u);
+        }
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_addr(&sh.tmem), kChunkCols);
+    dep_wait();                  // everything this kernel reads comes from the kernels ahead (cache rows, queries, ranges)
+    dep_trigger();
+    if (tid == 0) {
+        int m = 1;
+        for (int t = 0; t < p.T; ++t) m = max(m, p.range[2 * t + 1]);
+        sh.n_max = m;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t base = (smem_addr(tc_raw) + 1023u) & ~1023u;
+    const uint32_t tmem = sh.tmem;
+    volatile int* abort_flag = &sh.abort_flag;
+    const int n_max = sh.n_max;
+    const int tiles_h = (n_max + 127) / 128, total = p.n_kv * tiles_h;
+    const int t0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * total / gridDim.x);
+    const int t1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * total / gridDim.x);
+    const uint32_t qbytes = static_cast<uint32_t>(p.ncolp) * kChunk * 2;          // one term of one K chunk of the queries
+    const uint32_t stage_tx = static_cast<uint32_t>(nkc) * (128 * kChunk * 2 + 2 * qbytes);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&map_k1);
+            tma_prefetch_desc(&map_qhi);
+            tma_prefetch_desc(&map_qlo);
+            int issued = 0;
+            for (int tile = t0; tile < t1; ++tile) {
+                const int i = tile - t0, s = i % kChunkStages;
+                if (i >= kChunkStages && !mbar_wait(smem_addr(&sh.empty[s]), ((i / kChunkStages) & 1) ^ 1, abort_flag)) break;
+                const int g = tile / tiles_h, rb = tile - g * tiles_h;
+                const uint32_t bar = smem_addr(&sh.full[s]), dst = base + s * kChunkStageBytes;
+                mbar_expect_tx(bar, stage_tx);
+                for (int kc = 0; kc < nkc; ++kc) {
+                    tma_load_2d(dst + kc * (128 * kChunk * 2), &map_k1, bar, kc * kChunk, static_cast<int>(g * p.cap + rb * 128));
+                    const uint32_t qd = dst + kChunkABytes + kc * (2 * kColMax * kChunk * 2);
+                    tma_load_2d(qd, &map_qhi, bar, kc * kChunk, g * kColMax);
+                    tma_load_2d(qd + qbytes, &map_qlo, bar, kc * kChunk, g * kColMax);    // lo rows right behind the hi rows
+                }
+                issued = i + 1;
+            }
+            if (*abort_flag != 0) {
+                for (int i = max(0, issued - kChunkStages); i < issued; ++i) {
+                    const long long c0 = clock64();
+                    while (!mbar_try(smem_addr(&sh.full[i % kChunkStages]), (i / kChunkStages) & 1))
+                        if (clock64() - c0 > kTcSpinLimit) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(128, 2 * p.ncolp, false);
+            for (int tile = t0; tile < t1; ++tile) {
+                const int i = tile - t0, s = i % kChunkStages, b = i & 1;
+                if (i >= 2 && !mbar_wait(smem_addr(&sh.acc_empty[b]), ((i >> 1) & 1) ^ 1, abort_flag)) break;
+                if (!mbar_wait(smem_addr(&sh.full[s]), (i / kChunkStages) & 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t a0 = base + s * kChunkStageBytes, q0 = a0 + kChunkABytes;
+                for (int kc = 0; kc < nkc; ++kc)
+#pragma unroll
+                    for (int j = 0; j < kChunk / 16; ++j)
+                        umma_bf16(tmem + b * 256, smem_desc(a0 + kc * (128 * kChunk * 2) + 32 * j, 0u, 1024u),
+                                  smem_desc(q0 + kc * (2 * kColMax * kChunk * 2) + 32 * j, 0u, 1024u), idesc, (kc == 0 && j == 0) ? 0u : 1u);
+                umma_commit(smem_addr(&sh.empty[s]));
+                umma_commit(smem_addr(&sh.acc_full[b]));
+            }
+        }
+    } else {
+        // eight warps: two per tensor-memory lane quadrant, each taking half of the columns
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        bool ok = true;
+        for (int tile = t0; tile < t1 && ok; ++tile) {
+            const int i = tile - t0, b = i & 1;
+            const int g = tile / tiles_h, rb = tile - g * tiles_h;
+            ok = __all_sync(kFull, mbar_wait(smem_addr(&sh.acc_full[b]), (i >> 1) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const int j = rb * 128 + q * 32 + lane;
+            const uint32_t tacc = tmem + b * 256 + (static_cast<uint32_t>(q * 32) << 16);
+            float* scol = p.S + static_cast<int64_t>(g) * kColMax * p.scap + j;
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+                const int cb = 2 * half + cc;
+                if (cb * 32 < p.ncol) {
+                    float v[32], w[32];
+                    tmem_ld32(tacc + cb * 32, v);
+                    tmem_ld32(tacc + p.ncolp + cb * 32, w);
+                    if (j < n_max) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (cb * 32 + c < p.ncol) scol[static_cast<int64_t>(cb * 32 + c) * p.scap] = v[c] + w[c];
+                    }
+                }
+            }
+            tc_fence_before();
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (tid == 64) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&sh.acc_empty[b])) : "memory");
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_free(tmem, kChunkCols);
+    }
+    if (tid == 0 && sh.abort_flag != 0) atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+}
+
+// ---- select: one block per (token, query head) ---------------------------------------------------------------------------
+// The column's visible scores are swept once: every warp compacts the survivors of its slice into a list in shared
+// memory (index, score) and tracks their maximum; after the block-wide maximum is known each warp walks its list
+// four survivors at a time (three blocks per SM matter more than loads in flight: the gather is bound by what L2
+// delivers): the k2c rows give the softplus gates, the vc rows are accumulated with weight
+// exp(s - max) . gate, eight columns of the output per lane.  The sum of exp(s - max) normalises the result.
+struct SelShared {
+    int idx[kSelWarps][kListCap];
+    float sc[kSelWarps][kListCap];
+    float q2[128];
+    float red[kSelWarps];
+    float acc[kSelWarps][256];
+    float esum[kSelWarps];
+    int cnt[kSelWarps];
+    double part[kSelWarps][2];
+    float theta;
+};
+
+__global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const ChunkParams p) {
+    extern __shared__ __align__(16) unsigned char sel_raw[];
+    SelShared& sh = *reinterpret_cast<SelShared*>(sel_raw);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t = blockIdx.x / p.n_q, h = blockIdx.x - t * p.n_q;
+    const int g = h / p.gq, col = t * p.gq + (h - g * p.gq);
+    const int d2 = p.hd - p.r;
+    dep_wait();
+    dep_trigger();
+    const int lo = p.range[2 * t], n = p.range[2 * t + 1], L = n - lo;
+    if (tid < d2) sh.q2[tid] = p.q[(static_cast<int64_t>(t) * p.n_q + h) * p.hd + p.r + tid];
+    const float* scol = p.S + (static_cast<int64_t>(g) * kColMax + col) * p.scap;
+    // slices of the visible range, one per warp
+    const int per = (L + kSelWarps - 1) / kSelWarps;
+    const int w0 = lo + warp * per, w1 = min(n, w0 + per);
+    // A slice of up to 1024 rows stays in registers (32 per lane) between the statistics and the selection, so
+    // the column is read once; longer slices are read again.
+    constexpr int kKeep = 32;
+    const bool kept = per <= 32 * kKeep;
+    float keep[kKeep];
+    if (kept) {
+#pragma unroll
+        for (int u = 0; u < kKeep; ++u) {
+            const int j = w0 + 32 * u + lane;
+            keep[u] = j < w1 ? __ldcg(scol + j) : -INFINITY;
+        }
+    }
+    if (p.k_attn < L) {
+        // sums of the column over the rows this query may see, around the column's first value (keeps the fp32
+        // partial sums accurate when |mean| >> std); combined in fp64
+        const float c0 = __ldcg(scol + lo);
+        float f1 = 0.f, f2 = 0.f;
+        if (kept) {
+#pragma unroll
+            for (int u = 0; u < kKeep; ++u) {
+                const float d = w0 + 32 * u + lane < w1 ? keep[u] - c0 : 0.f;
+                f1 += d;
+                f2 = fmaf(d, d, f2);
+            }
+        } else {
+            for (int j0 = w0; j0 < w1; j0 += 32 * 16) {
+                float sv[16];
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    const int j = j0 + 32 * u + lane;
+                    sv[u] = j < w1 ? __ldcg(scol + j) - c0 : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 16; ++u) {
+                    f1 += sv[u];
+                    f2 = fmaf(sv[u], sv[u], f2);
+                }
+            }
+        }
+        const double s1 = warp_sum_f64(static_cast<double>(f1)), s2 = warp_sum_f64(static_cast<double>(f2));
+        if (lane == 0) {
+            sh.part[warp][0] = s1;
+            sh.part[warp][1] = s2;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float th = -INFINITY;
+        if (p.k_attn < L) {
+            double s1 = 0.0, s2 = 0.0;
+#pragma unroll
+            for (int w = 0; w < kSelWarps; ++w) {
+                s1 += sh.part[w][0];
+                s2 += sh.part[w][1];
+            }
+            const double dm = s1 / static_cast<double>(L);                 // mean - c0
+            const double var = (s2 - s1 * dm) / static_cast<double>(L - 1);
+            th = static_cast<float>(static_cast<double>(__ldcg(scol + lo)) + dm + sqrt(var > 0.0 ? var : 0.0) * p.zt[t]);
+        }
+        sh.theta = th;
+        if (p.theta != nullptr) p.theta[blockIdx.x] = th;
+    }
+    __syncthreads();
+    const float th = sh.theta;
+    const __nv_bfloat16* k2 = p.k2c + static_cast<int64_t>(g) * p.cap * d2;
+    const __nv_bfloat16* vv = p.vc + static_cast<int64_t>(g) * p.cap * p.hd;
+    const int nc2 = d2 / 8, ncv = p.hd / 8;          // 16-byte pieces of a k2c row and of a vc row
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    float run_max = -INFINITY, esum = 0.f;           // of this warp so far: weights are exp(s - run_max)
+    int total = 0;
+    // The warp's list is drained (its survivors gathered) when the slice is done, or earlier when it is about to overflow.
+    auto drain = [&](int cnt, float mx) {
+        mx = warp_max(mx);
+        __syncwarp();
+        if (cnt == 0) return;
+        total += cnt;
+        if (mx > run_max) {              // rescale what has been accumulated to the new reference
+            const float f = run_max == -INFINITY ? 0.f : __expf(run_max - mx);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] *= f;
+            esum *= f;
+            run_max = mx;
+        }
+        for (int i0 = 0; i0 < cnt; i0 += 4) {
+            uint4 kr[2], vr[4];
+            // k2c rows: half a warp per survivor, two loads for four survivors; vc rows: a warp per survivor
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int i = i0 + 2 * u + (lane >> 4);
+                kr[u] = (i < cnt && (lane & 15) < nc2) ? ld_stream16(reinterpret_cast<const uint4*>(k2 + static_cast<int64_t>(sh.idx[warp][i]) * d2) + (lane & 15))
+                                                       : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u;
+                vr[u] = (i < cnt && lane < ncv) ? ld_stream16(reinterpret_cast<const uint4*>(vv + static_cast<int64_t>(sh.idx[warp][i]) * p.hd) + lane)
+                                                : make_uint4(0u, 0u, 0u, 0u);
+            }
+            float gate[4];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const unsigned wds[4] = {kr[u].x, kr[u].y, kr[u].z, kr[u].w};
+                const float* qq = sh.q2 + 8 * (lane & 15);
+                float d = 0.f;
+                if ((lane & 15) < nc2) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        d = fmaf(__uint_as_float(wds[e] << 16), qq[2 * e], d);
+                        d = fmaf(__uint_as_float(wds[e] & 0xffff0000u), qq[2 * e + 1], d);
+                    }
+                }
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) d += __shfl_xor_sync(kFull, d, o);       // within each half-warp
+                gate[2 * u] = __shfl_sync(kFull, d, 0);
+                gate[2 * u + 1] = __shfl_sync(kFull, d, 16);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u;
+                if (i < cnt) {
+                    const float e = __expf(sh.sc[warp][i] - run_max);
+                    const float wgt = e * softplus(gate[u]);
+                    esum += e;
+                    const unsigned wds[4] = {vr[u].x, vr[u].y, vr[u].z, vr[u].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        acc[2 * k] = fmaf(wgt, __uint_as_float(wds[k] << 16), acc[2 * k]);
+                        acc[2 * k + 1] = fmaf(wgt, __uint_as_float(wds[k] & 0xffff0000u), acc[2 * k + 1]);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    };
+    {
+        int cnt = 0;
+        float mx = -INFINITY;
+        auto take = [&](int j, float sv, bool in_range) {      // one 32-row step: the survivors join the list
+            const bool on = in_range && sv > th;
+            const unsigned bal = __ballot_sync(kFull, on);
+            if (cnt + 32 > kListCap) {
+                drain(cnt, mx);
+                cnt = 0;
+                mx = -INFINITY;
+            }
+            if (on) {
+                const int at = cnt + __popc(bal & ((1u << lane) - 1u));
+                sh.idx[warp][at] = j;
+                sh.sc[warp][at] = sv;
+                mx = fmaxf(mx, sv);
+            }
+            cnt += __popc(bal);
+        };
+        if (kept) {
+#pragma unroll
+            for (int u = 0; u < kKeep; ++u) {
+                const int j = w0 + 32 * u + lane;
+                if (w0 + 32 * u < w1) take(j, keep[u], j < w1);
+            }
+        } else {
+            for (int j0 = w0; j0 < w1; j0 += 32 * 8) {          // eight loads per lane in flight
+                float sv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int j = j0 + 32 * u + lane;
+                    sv[u] = j < w1 ? __ldcg(scol + j) : -INFINITY;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int j = j0 + 32 * u + lane;
+                    if (j0 + 32 * u < w1) take(j, sv[u], j < w1);
+                }
+            }
+        }
+        drain(cnt, mx);
+    }
+    // merge the warps: common reference = the block's maximum
+    if (lane == 0) {
+        sh.red[warp] = run_max;
+        sh.cnt[warp] = total;
+    }
+    __syncthreads();
+    float bmax = -INFINITY;
+    int btotal = 0;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+        bmax = fmaxf(bmax, sh.red[w]);
+        btotal += sh.cnt[w];
+    }
+    const float f = (run_max == -INFINITY) ? 0.f : __expf(run_max - bmax);
+    if (lane < ncv) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sh.acc[warp][8 * lane + e] = acc[e] * f;
+    }
+    if (lane == 0) sh.esum[warp] = esum * f;
+    __syncthreads();
+    float es = 0.f;
+#pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) es += sh.esum[w];
+    float* orow = p.o + static_cast<int64_t>(blockIdx.x) * p.hd;
+    for (int c = tid; c < p.hd; c += kSelThreads) {
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < kSelWarps; ++w) v += sh.acc[w][c];
+        orow[c] = btotal > 0 ? v / es : 0.f;
+    }
+    if (tid == 0) {
+        if (p.lsum != nullptr) p.lsum[blockIdx.x] = btotal > 0 ? 1.f : 0.f;
+        if (p.count != nullptr) p.count[blockIdx.x] = btotal;
+    }
+}
+
+}  // namespace
+
+namespace spark {
+
+// SPARK_ERR_WORKSPACE = shape or workspace not served by this path (the caller falls back to the per-query kernel).
+int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int64_t T, int64_t n_q,
+                      int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs, int64_t window,
+                      int64_t k_attn, float* o, float* lsum, float* theta, int32_t* count, cudaStream_t stream) {
+    const int64_t gq = n_q / n_kv, d2 = hd - r;
+    if (T < 1 || T > 64 || T * gq > kColMax || (gq != 1 && gq != 2 && gq != 4 && gq != 8)) return SPARK_ERR_WORKSPACE;
+    if ((r != 64 && r != 128) || d2 < 8 || d2 > 128 || (d2 & 7) != 0 || hd > 256 || (hd & 7) != 0) return SPARK_ERR_WORKSPACE;
+    if (n_kv * cap >= (1LL << 31) || ((reinterpret_cast<uintptr_t>(k1c) | reinterpret_cast<uintptr_t>(k2c) | reinterpret_cast<uintptr_t>(vc)) & 15u) != 0)
+        return SPARK_ERR_WORKSPACE;
+    const size_t small_b = round_up(static_cast<size_t>(T) * (sizeof(double) + 2 * sizeof(int)), 1024);
+    const size_t q_b = round_up(static_cast<size_t>(n_kv) * kColMax * r * 2, 1024);
+    const size_t s_b = round_up(static_cast<size_t>(n_kv) * kColMax * (cap + 32) * 4, 1024);
+    if (ctx->scratch == nullptr || ctx->scratch_bytes < kAttnCellBytes + small_b + 2 * q_b + s_b) return SPARK_ERR_WORKSPACE;
+    const size_t smem_scores = static_cast<size_t>(kChunkStages) * kChunkStageBytes + 1024;
+    if (smem_scores + sizeof(ChunkShared) + 64 > static_cast<size_t>(ctx->max_smem_optin)) return SPARK_ERR_WORKSPACE;
+
+    ChunkParams p;
+    p.q = q; p.k2c = static_cast<const __nv_bfloat16*>(k2c); p.vc = static_cast<const __nv_bfloat16*>(vc);
+    p.ctx_len = ctx_len; p.zs_in = zs;
+    p.T = static_cast<int>(T); p.n_q = static_cast<int>(n_q); p.n_kv = static_cast<int>(n_kv); p.gq = static_cast<int>(gq);
+    p.hd = static_cast<int>(hd); p.r = static_cast<int>(r);
+    p.window = static_cast<int>(window > 0x7fffffff ? 0x7fffffff : window);
+    p.k_attn = static_cast<int>(k_attn > 0x7fffffff ? 0x7fffffff : k_attn);
+    p.ncol = static_cast<int>(T * gq);
+    p.ncolp = (p.ncol + 15) & ~15;
+    p.cap = cap;
+    p.scap = cap + 32;
+    p.o = o; p.lsum = lsum; p.theta = theta; p.count = count;
+    char* w = ctx->scratch + kAttnCellBytes;
+    p.zt = reinterpret_cast<double*>(w);
+    p.range = reinterpret_cast<int*>(w + static_cast<size_t>(T) * sizeof(double)); w += small_b;
+    p.qhi = reinterpret_cast<__nv_bfloat16*>(w); w += q_b;
+    p.qlo = reinterpret_cast<__nv_bfloat16*>(w); w += q_b;
+    p.S = reinterpret_cast<float*>(w);
+    p.hdr = ctx->hdr;
+
+    CUtensorMap m_k1, m_qhi, m_qlo;
+    if (!make_map(&m_k1, k1c, n_kv * cap, r, r, 128, true) || !make_map(&m_qhi, p.qhi, n_kv * kColMax, r, r, p.ncolp, false) ||
+        !make_map(&m_qlo, p.qlo, n_kv * kColMax, r, r, p.ncolp, false))
+        return SPARK_ERR_WORKSPACE;
+    if (cudaFuncSetAttribute(attn_chunk_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_scores)) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_chunk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(SelShared))) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    {
+        void* args[] = {&p};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_prep_kernel), static_cast<unsigned>(n_kv * kColMax), 128, 0, stream, false, args) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+    {
+        void* args[] = {&p, &m_k1, &m_qhi, &m_qlo};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_scores_kernel), static_cast<unsigned>(ctx->num_sms), kChunkThreads, smem_scores, stream, false, args) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+    {
+        void* args[] = {&p};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_select_kernel), static_cast<unsigned>(T * n_q), kSelThreads, sizeof(SelShared), stream, false, args) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+    return SPARK_OK;
+}
+
+}  // namespace spark

@@ -57,4 +57,11 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
                 int64_t idx_cap, const float* k1s, cudaStream_t st);
 
+// Spark attention for a chunk of a prompt (T consecutive tokens of one sequence over one cache, bf16): predictor scores of
+// the whole chunk as one tcgen05 GEMM per KV head (attn_chunk.cu).  o is written normalised; lsum (nullable) receives 1 per
+// head (0 for an empty selection).  SPARK_ERR_WORKSPACE = shape or workspace not served.
+int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int64_t T, int64_t n_q,
+                      int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs, int64_t window,
+                      int64_t k_attn, float* o, float* lsum, float* theta, int32_t* count, cudaStream_t stream);
+
 }  // namespace spark

@@ -7,6 +7,7 @@
     python -m paper_2506_06644_b200.profile_cases attn    # Spark attention, batch 1, context 8192
     python -m paper_2506_06644_b200.profile_cases topk    # statistical top-k, 512 rows x 65536
     python -m paper_2506_06644_b200.profile_cases layer   # four decoder layers, one token
+    python -m paper_2506_06644_b200.profile_cases chunk64 # four decoder layers over a 64-token chunk of a prompt
 
 Every case cycles over enough distinct weight sets / caches / rows to exceed the 126 MB L2, holds at
 most about 1 GB on the device and launches a dozen kernels, so that a capture of two or three of
@@ -108,7 +109,37 @@ def case_layer(n_layers=4, B=1, ctx_len=8192, steps=3, overlap=True):
     assert ctx.device_status() == S.SPARK_OK
 
 
-CASES = {"ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
+def case_chunk(n_layers=4, T=64, ctx_len=8192, steps=2):
+    """Chunks of a prompt: T consecutive tokens of one sequence per layer call, behind ctx_len - T cached tokens."""
+    sh = synth.GEMMA2_2B
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4)
+    ctx = S.SparkContext(0, max_batch=T, max_dff=sh.d_ff, max_cap=ctx_len, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
+    ctx.set_launch_overlap(True)
+    nqkv = (sh.n_q + 2 * sh.n_kv) * sh.hd
+    layers = []
+    for _ in range(n_layers):
+        w = dict(norm1=torch.ones(sh.d, device="cuda"), norm2=torch.ones(sh.d, device="cuda"),
+                 Wqkv=_w(gen, nqkv, sh.d, sh.d), Wo=_w(gen, sh.d, sh.n_q * sh.hd, sh.n_q * sh.hd),
+                 K1t=_w(gen, sh.d_ff, sh.r_ff, sh.d), K2t=_w(gen, sh.d_ff, sh.d - sh.r_ff, sh.d), Vt=_w(gen, sh.d_ff, sh.d, sh.d))
+        cache = dict(k1c=torch.randn(sh.n_kv, ctx_len, sh.r_attn, device="cuda", generator=gen).to(torch.bfloat16),
+                     k2c=torch.randn(sh.n_kv, ctx_len, sh.hd - sh.r_attn, device="cuda", generator=gen).to(torch.bfloat16),
+                     vc=torch.randn(sh.n_kv, ctx_len, sh.hd, device="cuda", generator=gen).to(torch.bfloat16))
+        cfg = dict(d=sh.d, d_ff=sh.d_ff, r_ff=sh.r_ff, k_ff=sh.k_ff, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+                   k_attn=sh.k_attn, window=0, cap=ctx_len, rms_eps=1e-6, rope_base=10000.0, flags=S.SPARK_SHARED_CACHE)
+        layers.append((S.make_layer(w, cfg, cache), w, cache))
+    h = torch.randn(T, sh.d, device="cuda", generator=gen)
+    cl = torch.arange(ctx_len - T + 1, ctx_len + 1, dtype=torch.int32, device="cuda")
+    scratch = torch.empty(T * (nqkv + 2 * sh.n_q * sh.hd + sh.d + 2 + sh.n_q), device="cuda")
+    torch.cuda.synchronize()
+    for _ in range(steps):
+        for lay in layers:
+            S.spark_layer_decode(ctx, lay[0], cl, h, T, scratch)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == S.SPARK_OK
+
+
+CASES = {"chunk64": case_chunk, "ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
 
 if __name__ == "__main__":
     name = sys.argv[1] if len(sys.argv) > 1 else ""

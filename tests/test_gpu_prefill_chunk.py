@@ -89,3 +89,36 @@ def test_attention_queries_sharing_one_cache(ctx):
     for b in range(B):
         ref = O.spark_attention(q[b].astype(np.float64), kc, vc, lens[b], k_attn, r)
         parity.check_output(o[b].cpu().numpy().reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"query {b}")
+
+
+@pytest.mark.parametrize("T,n_q,n_kv,hd,r,cap,L0,k_attn,window", [
+    (33, 8, 4, 256, 128, 1024, 700, 64, 0),          # two query heads per KV head, tensor-core scores for the whole chunk
+    (64, 8, 4, 256, 128, 640, 500, 32, 0),           # the largest chunk: 128 columns per KV head
+    (40, 4, 4, 128, 64, 512, 300, 40, 100),          # one head per KV head, r = 64, a window sliding over the chunk
+    (32, 8, 2, 256, 128, 256, 0, 16, 0),             # four heads per KV head; the chunk starts the sequence (identity for short rows)
+    (12, 8, 4, 256, 128, 512, 400, 64, 0),           # a short chunk: per-query kernel over the shared cache
+])
+def test_chunk_attention_on_the_tensor_cores(ctx, T, n_q, n_kv, hd, r, cap, L0, k_attn, window):
+    kv = synth.attn_inputs(1, n_q, n_kv, hd, r, cap, [cap], "bf16", seed=41)
+    q = synth.normal_f32((T, n_q, hd), 42, 0) * hd ** -0.5
+    lens = [L0 + t + 1 for t in range(T)]
+    o = torch.full((T, n_q, hd), float("nan"), device="cuda")
+    theta = torch.empty(T, n_q, device="cuda")
+    count = torch.empty(T, n_q, dtype=torch.int32, device="cuda")
+    S.spark_attn_decode(ctx, torch.from_numpy(q).cuda(), bf16_dev(kv.k1c_bits[0]), bf16_dev(kv.k2c_bits[0]), bf16_dev(kv.vc_bits[0]),
+                        S.SPARK_BF16, T, n_q, n_kv, hd, r, cap, torch.tensor(lens, dtype=torch.int32, device="cuda"), window, k_attn,
+                        S.SPARK_SHARED_CACHE, o, theta, count, None, 0)
+    torch.cuda.synchronize()
+    kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+    vc = kv.vc[0].astype(np.float64)
+    og, thg, cg = o.cpu().numpy(), theta.cpu().numpy(), count.cpu().numpy()
+    for t in range(T):
+        ref = O.spark_attention(q[t].astype(np.float64), kc, vc, lens[t], k_attn, r, window)
+        for h in range(n_q):
+            lo = 0 if window <= 0 else max(0, lens[t] - window)
+            s = kc[h // (n_q // n_kv), lo:lens[t], :r] @ q[t, h, :r].astype(np.float64)
+            std = float(np.std(s, ddof=1)) if s.size > 1 else 1.0
+            parity.check_theta(thg[t, h], ref["theta"][h], std, f"token {t} head {h}")
+            near = int(np.sum(np.abs(s - ref["theta"][h]) <= 1e-4 * std)) if np.isfinite(ref["theta"][h]) else 0
+            assert abs(int(cg[t, h]) - int(ref["mask"][h].sum())) <= near
+        parity.check_output(og[t].reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"token {t}")
