@@ -376,12 +376,18 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
                 gate[2 * u] = __shfl_sync(kFull, d, 0);
                 gate[2 * u + 1] = __shfl_sync(kFull, d, 16);
             }
+            // lane u < 4 evaluates survivor u's exponential and gate once; the others receive them
+            float e_l = 0.f, w_l = 0.f;
+            if (lane < 4 && i0 + lane < cnt) {
+                const float gl = lane == 0 ? gate[0] : (lane == 1 ? gate[1] : (lane == 2 ? gate[2] : gate[3]));
+                e_l = __expf(sh.sc[warp][i0 + lane] - run_max);
+                w_l = e_l * softplus(gl);
+            }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int i = i0 + u;
+                const float e = __shfl_sync(kFull, e_l, u), wgt = __shfl_sync(kFull, w_l, u);
                 if (i < cnt) {
-                    const float e = __expf(sh.sc[warp][i] - run_max);
-                    const float wgt = e * softplus(gate[u]);
                     esum += e;
                     const unsigned wds[4] = {vr[u].x, vr[u].y, vr[u].z, vr[u].w};
 #pragma unroll
@@ -413,7 +419,38 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
             }
             cnt += __popc(bal);
         };
+        bool listed = false;
         if (kept) {
+            // the order of the list does not matter: every lane counts its own survivors, a scan of the counts gives it
+            // a place, and it writes them there -- no ballot per 32 rows
+            int mine = 0;
+#pragma unroll
+            for (int u = 0; u < kKeep; ++u) mine += (keep[u] > th) ? 1 : 0;          // rows past the slice hold -inf
+            int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const int all = __shfl_sync(kFull, incl, 31);
+            if (all <= kListCap) {
+                int at = incl - mine;
+#pragma unroll
+                for (int u = 0; u < kKeep; ++u) {
+                    if (keep[u] > th) {
+                        sh.idx[warp][at] = w0 + 32 * u + lane;
+                        sh.sc[warp][at] = keep[u];
+                        mx = fmaxf(mx, keep[u]);
+                        ++at;
+                    }
+                }
+                cnt = all;
+                listed = true;
+            }
+        }
+        if (listed) {
+            // done
+        } else if (kept) {
 #pragma unroll
             for (int u = 0; u < kKeep; ++u) {
                 const int j = w0 + 32 * u + lane;
