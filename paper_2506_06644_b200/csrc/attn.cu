@@ -816,9 +816,9 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     if (!aligned16(q) || !aligned16(k1c) || !aligned16(k2c) || !aligned16(vc) || !aligned16(o)) return SPARK_ERR_UNSUPPORTED;
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
 
-    if ((flags & SPARK_SHARED_CACHE) && !(flags & SPARK_DENSE_LOADS) && B >= 32 && kvdtype == SPARK_BF16 && k1s == nullptr && idx == nullptr) {
-        // a long chunk of a prompt: the predictor scores of all its queries as one GEMM per KV head (measured: pays from
-        // about 32 tokens on; shorter chunks stream the slice per query out of L2 as fast)
+    if ((flags & SPARK_SHARED_CACHE) && !(flags & SPARK_DENSE_LOADS) && B >= 16 && kvdtype == SPARK_BF16 && k1s == nullptr && idx == nullptr) {
+        // a chunk of a prompt: the predictor scores of all its queries as one GEMM per KV head (measured: pays from
+        // about 16 tokens on; shorter chunks stream the slice per query out of L2 as fast)
         const int rc = attn_chunk_launch(ctx, q, k1c, k2c, vc, B, n_q, n_kv, hd, r, cap, ctx_len, zs, window, k_attn, o, lsum, theta, count, st);
         if (rc != SPARK_ERR_WORKSPACE) return rc;
     }
