@@ -92,7 +92,7 @@ def test_attention_queries_sharing_one_cache(ctx):
 
 
 @pytest.mark.parametrize("T,n_q,n_kv,hd,r,cap,L0,k_attn,window", [
-    (33, 8, 4, 256, 128, 1024, 700, 64, 0),          # two query heads per KV head, tensor-core scores for the whole chunk
+    (17, 8, 4, 256, 128, 1024, 700, 64, 0),          # two query heads per KV head, tensor-core scores for the whole chunk
     (64, 8, 4, 256, 128, 640, 500, 32, 0),           # the largest chunk: 128 columns per KV head
     (40, 4, 4, 128, 64, 512, 300, 40, 100),          # one head per KV head, r = 64, a window sliding over the chunk
     (32, 8, 2, 256, 128, 256, 0, 16, 0),             # four heads per KV head; the chunk starts the sequence (identity for short rows)
