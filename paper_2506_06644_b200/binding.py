@@ -258,3 +258,32 @@ def make_layer(weights: dict, cfg: dict, cache: dict) -> LayerHandles:
 def spark_layer_decode(ctx: SparkContext, layer: LayerHandles, ctx_len, h, B, scratch):
     _check(lib().spark_layer_decode(ctx.handle, C.byref(layer.weights), C.byref(layer.cfg), C.byref(layer.cache),
                                     _ptr(ctx_len), _ptr(h), B, _ptr(scratch), _stream()), "spark_layer_decode")
+
+
+def layer_scratch_floats(cfg: dict, B: int) -> int:
+    """fp32 elements of scratch spark_layer_decode needs for B tokens."""
+    nqkv = (cfg["n_q"] + 2 * cfg["n_kv"]) * cfg["hd"]
+    return B * (nqkv + 2 * cfg["n_q"] * cfg["hd"] + cfg["d"] + 2 + cfg["n_q"])
+
+
+def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64):
+    """Run a prompt through a stack of layers chunk by chunk (host loop only: every step is spark_layer_decode).
+
+    layers: LayerHandles made with SPARK_SHARED_CACHE in cfg["flags"] and caches [n_kv][cap][.]; h [N][d] fp32 holds the
+    prompt's N embeddings and is replaced in place by the stack's outputs; the tokens are appended to each layer's
+    cache at rows start .. start + N - 1 (start = tokens already cached).  chunk <= 64 tokens go through the stack
+    together; later chunks see the earlier ones through the caches."""
+    if not 1 <= chunk <= 64:
+        raise ValueError("chunk must be 1..64")
+    N = h.shape[0]
+    cfg = {k: getattr(layers[0].cfg, k) for k in ("n_q", "n_kv", "hd", "d")}
+    scratch = torch.empty(layer_scratch_floats(cfg, min(chunk, N)), dtype=torch.float32, device=h.device)
+    for c0 in range(0, N, chunk):
+        T = min(chunk, N - c0)
+        lens = torch.arange(start + c0 + 1, start + c0 + T + 1, dtype=torch.int32, device=h.device)
+        part = h[c0 : c0 + T]
+        for layer in layers:
+            if not (layer.cfg.flags & SPARK_SHARED_CACHE):
+                raise ValueError("spark_prefill needs layers configured with SPARK_SHARED_CACHE")
+            spark_layer_decode(ctx, layer, lens, part, T, scratch)
+    return h

@@ -122,3 +122,38 @@ def test_chunk_attention_on_the_tensor_cores(ctx, T, n_q, n_kv, hd, r, cap, L0, 
             near = int(np.sum(np.abs(s - ref["theta"][h]) <= 1e-4 * std)) if np.isfinite(ref["theta"][h]) else 0
             assert abs(int(cg[t, h]) - int(ref["mask"][h].sum())) <= near
         parity.check_output(og[t].reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"token {t}")
+
+
+def test_prefill_loop_over_two_layers_and_ragged_chunks(ctx):
+    # 100 tokens in chunks of 64 (64 + 36) through two layers behind 30 cached tokens, against token-by-token decoding
+    sh, N, L0, cap = synth.GEMMA2_2B, 100, 30, 256
+    lws = [synth.layer_weights(sh, 51 + l, 0) for l in range(2)]
+    kvs = [synth.attn_inputs(1, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, cap, [L0], "bf16", seed=61 + l) for l in range(2)]
+    h0 = synth.normal_f32((N, sh.d), 71, 60)
+    layers, keep = [], []
+    for lw, kv in zip(lws, kvs):
+        dev = dict(norm1=torch.from_numpy(lw.norm1).cuda(), norm2=torch.from_numpy(lw.norm2).cuda(),
+                   Wqkv=bf16_dev(lw.Wqkv_bits), Wo=bf16_dev(lw.Wo_bits), K1t=bf16_dev(lw.K1t_bits),
+                   K2t=bf16_dev(lw.K2t_bits), Vt=bf16_dev(lw.Vt_bits))
+        cache = dict(k1c=bf16_dev(kv.k1c_bits[0]), k2c=bf16_dev(kv.k2c_bits[0]), vc=bf16_dev(kv.vc_bits[0]))
+        cfg = dict(d=sh.d, d_ff=sh.d_ff, r_ff=sh.r_ff, k_ff=sh.k_ff, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+                   k_attn=sh.k_attn, window=0, cap=cap, rms_eps=1e-6, rope_base=10000.0, flags=S.SPARK_SHARED_CACHE)
+        layers.append(S.make_layer(dev, cfg, cache))
+        keep.append((dev, cache))
+    h = torch.from_numpy(h0).cuda()
+    S.spark_prefill(ctx, layers, h, L0, chunk=64)
+    torch.cuda.synchronize()
+    got = h.cpu().numpy()
+    caches = [(np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64), kv.vc[0].astype(np.float64)) for kv in kvs]
+    Ws = [{"norm1": lw.norm1, "norm2": lw.norm2, "Wqkv": synth.bf16_bits_to_f32(lw.Wqkv_bits), "Wo": synth.bf16_bits_to_f32(lw.Wo_bits),
+           "K1t": synth.bf16_bits_to_f32(lw.K1t_bits), "K2t": synth.bf16_bits_to_f32(lw.K2t_bits), "Vt": synth.bf16_bits_to_f32(lw.Vt_bits)}
+          for lw in lws]
+    ref = np.zeros_like(got, dtype=np.float64)
+    for t in range(N):
+        x = h0[t].astype(np.float64)
+        for W, (kc, vc) in zip(Ws, caches):
+            x = O.decoder_layer(x, W, kc, vc, L0 + t + 1, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn, k_attn=sh.k_attn,
+                                r_ff=sh.r_ff, k_ff=sh.k_ff, window=0)["h"]
+        ref[t] = x
+    for t in range(N):
+        parity.check_output(got[t], ref[t], "bf16", f"token {t}")
