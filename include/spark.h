@@ -301,8 +301,10 @@ typedef struct spark_kv_cache {
 /* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2 + n_q) fp32 values, 16-byte aligned, caller-owned, contents
  * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 64.  Four kernels are
  * enqueued for B <= 4: QKV projection with position encoding and cache append, attention, output projection,
- * FFN; five for B >= 5, where the position encoding and the append follow the projection as a kernel of
- * their own. */
+ * FFN.  For B >= 5 the position encoding and the append follow the projection as a kernel of their own, and
+ * where the shapes allow (see spark_ffn_decode; projections: inputs % 64 == 0, outputs % 128 == 0) the
+ * projections and the FFN run as tensor-core GEMMs of two and four kernels each, and the attention of a
+ * chunk (SPARK_SHARED_CACHE, B >= 16) as three: up to thirteen kernels per call. */
 int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
                        const spark_kv_cache* cache, const int32_t* ctx_len, float* h, int64_t B,
                        float* scratch, void* stream);
