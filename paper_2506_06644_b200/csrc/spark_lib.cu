@@ -64,7 +64,15 @@ size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap
     // placed behind the attention's cells (the two never run at the same time on one context)
     size_t need_ffn = 0;
     if (max_batch >= 5 && max_dff > 0 && max_d > 0) need_ffn = kAttnCellBytes + ffn_tc_workspace_bytes(max_d, max_dff);
-    return sizeof(WsHeader) + (need > need_ffn ? need : need_ffn) + 256;
+    // attention over a chunk of a prompt (16 and more tokens sharing one cache): split queries and the score matrix of the
+    // tensor-core path, at most n_q KV heads x 128 columns x (max_cap + 32) scores
+    size_t need_chunk = 0;
+    if (max_batch >= 16)
+        need_chunk = kAttnCellBytes + 4096 + 2 * round_up(static_cast<size_t>(n_q) * 128 * 128 * 2, 1024) +
+                     round_up(static_cast<size_t>(n_q) * 128 * (static_cast<size_t>(max_cap) + 32) * 4, 1024);
+    size_t most = need > need_ffn ? need : need_ffn;
+    if (need_chunk > most) most = need_chunk;
+    return sizeof(WsHeader) + most + 256;
 }
 
 int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_bytes) {
