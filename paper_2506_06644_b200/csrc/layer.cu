@@ -314,6 +314,8 @@ struct RopeParams {
 };
 
 __global__ void rope_append_kernel(const RopeParams p) {
+    dep_wait();        // the projections come from the kernel ahead
+    dep_trigger();
     if (blockIdx.x == 0 && threadIdx.x < p.B) {         // the threshold quantile of each sequence's window
         int n = p.ctx_len[threadIdx.x];
         n = n < 1 ? 1 : (n > p.cap ? static_cast<int>(p.cap) : n);
@@ -611,8 +613,9 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
         if (rc != SPARK_OK) return rc;
         const int64_t total = B * (cfg->n_q + 2 * cfg->n_kv) * (cfg->hd / 2);
         const int blocks = static_cast<int>((total + 255) / 256);
-        rope_append_kernel<<<blocks, 256, 0, st>>>(rp);
-        if (cudaGetLastError() != cudaSuccess) return SPARK_ERR_CUDA;
+        void* rargs[] = {&rp};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(rope_append_kernel), static_cast<unsigned>(blocks), 256, 0, st, false, rargs) != cudaSuccess)
+            return SPARK_ERR_CUDA;
     }
 
     // 3. Spark attention over the cache (the new token included)
