@@ -30,6 +30,7 @@ def ctx():
     (synth.GEMMA2_2B, 16, 0, 64, 0),            # a chunk that starts the sequence (empty cache)
     (synth.GEMMA2_2B, 64, 100, 256, 0),         # the largest chunk a layer call takes
     (synth.TINY, 20, 10, 64, 0),                # more than sixteen tokens on the fallback kernels (shape not served by the GEMMs)
+    (synth.GEMMA2_9B, 16, 40, 128, 0),          # 9B shape: 16 query / 8 KV heads, d 3584, d_ff 14336 on every tensor-core path
 ])
 def test_chunk_of_a_prompt_equals_token_by_token_decoding(ctx, shape, T, L0, cap, window):
     sh = shape
