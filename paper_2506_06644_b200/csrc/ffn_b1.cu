@@ -119,6 +119,35 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     __syncthreads();
     p.trace.mark(2);
 
+    // While warp 0 exchanges the sums, the other warps ask L2 for the rows this block will most likely gather: the
+    // neurons above the threshold estimated from the block's own scores alone.  The gather then finds most of its
+    // rows in L2 instead of waiting for DRAM after the exchange (a lower estimate, which catches more of them, measured
+    // slower: the extra requests delay the exchange).
+    if (warp > 0 && !p.identity && !p.dense && nloc >= 8) {
+        float a1 = 0.f, a2 = 0.f;
+        for (int j = lane; j < nloc; j += 32) {
+            const float v = s_loc[j];
+            a1 += v;
+            a2 = fmaf(v, v, a2);
+        }
+        a1 = warp_sum(a1);
+        a2 = warp_sum(a2);
+        const float mean = a1 / nloc, var = fmaxf((a2 - a1 * mean) / (nloc - 1), 0.f);
+        const float guess = mean + sqrtf(var) * static_cast<float>(p.z);
+        int seen = 0;
+        for (int j0 = 0; j0 < nloc; j0 += 32) {
+            const int j = j0 + lane;
+            const unsigned bal = __ballot_sync(kFull, j < nloc && s_loc[j] > guess);
+            for (unsigned m = bal; m != 0u; m &= m - 1u) {
+                if (seen++ % (kWarps - 1) != warp - 1) continue;
+                const int jj = j0 + __ffs(m) - 1;
+                const char* krow = reinterpret_cast<const char*>(K2t + static_cast<int64_t>(row0 + jj) * d2);
+                const char* vrow = reinterpret_cast<const char*>(Vt + static_cast<int64_t>(row0 + jj) * d);
+                for (int o = lane * 128; o < d2 * static_cast<int>(sizeof(WT)); o += 32 * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(krow + o));
+                for (int o = lane * 128; o < d * static_cast<int>(sizeof(WT)); o += 32 * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(vrow + o));
+            }
+        }
+    }
     // ---- S: add this block's sums to the grid-wide cell, wait for everybody's, theta ------------------
     if (warp == 0) {
         SumCell* ways = &p.hdr->ffn_cells[s_epoch & 3u][0][0][0];
