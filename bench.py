@@ -33,7 +33,7 @@ import numpy as np
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from the ncu
 # capture summarised in profiles/ (keyed by shape and batch); None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {("2b", 1): 24.34e6}       # profiles/ffn_b1.md
+NCU_TRAFFIC_BYTES = {("2b", 1): 25.04e6}       # profiles/ffn_b1.md
 
 FALLBACK_HBM_GBS = 6650.0
 
