@@ -681,6 +681,23 @@ def other_workloads(torch, S, peak, steps, warmup):
         out.append({"workload": f"spark_layer_decode over a chunk of a prompt: {T} consecutive tokens of one sequence per call "
                                 f"(shared cache, causal), context {L}, {nl} layers: per layer",
                     "us_per_launch": us_chunk, "us_per_token_per_layer": us_chunk / T})
+    # -- a whole prompt: 4096 tokens from an empty cache through the eight layers in 64-token chunks (binding.spark_prefill:
+    #    host loop, 64 x 8 layer calls of 13 kernels), timed with events around the loop
+    Np = 4096
+    hp = torch.randn(Np, sh.d, device=dev, generator=gen)
+    lay_only = [c[0] for c in chunk_layers]
+    S.spark_prefill(ctx, lay_only, hp[:256].clone(), 0, chunk=64)          # warm-up
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    S.spark_prefill(ctx, lay_only, hp, 0, chunk=64)
+    e1.record()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == S.SPARK_OK
+    ms_pre = e0.elapsed_time(e1)
+    out.append({"workload": f"spark_prefill: {Np} tokens from an empty cache through {nl} layers in 64-token chunks (host launches)",
+                "us_per_launch": ms_pre * 1e3 / (Np // 64 * nl), "us_per_token_per_layer": ms_pre * 1e3 / (Np * nl),
+                "prompt_tokens_per_s_per_layer_stack": Np / (ms_pre * 1e-3)})
     ctx.close()
     del stacks, chunk_layers
 
