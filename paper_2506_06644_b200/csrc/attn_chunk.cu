@@ -22,7 +22,8 @@ namespace {
 constexpr int kColMax = 128;          // (token, head-in-group) columns per KV head
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kListCap = 512;         // survivors a warp of the select kernel lists before it gathers them
+constexpr int kListCap = 128;         // survivors a warp of the select kernel lists before it gathers them
+constexpr int kColRows = 8192;        // visible rows of a column the select kernel keeps in shared memory
 
 struct ChunkParams {
     const float* q;            // [T][n_q][hd]
@@ -228,12 +229,13 @@ attn_chunk_scores_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
 }
 
 // ---- select: one block per (token, query head) ---------------------------------------------------------------------------
-// The column's visible scores are swept once: every warp compacts the survivors of its slice into a list in shared
-// memory (index, score) and tracks their maximum; after the block-wide maximum is known each warp walks its list
-// four survivors at a time (three blocks per SM matter more than loads in flight: the gather is bound by what L2
-// delivers): the k2c rows give the softplus gates, the vc rows are accumulated with weight
+// The column's visible scores are read once into shared memory: every warp compacts the survivors of its slice into a
+// list (index, score) and tracks their maximum; after the block-wide maximum is known each warp walks its list
+// four survivors at a time (four blocks per SM -- all 512 (token, head) pairs of a 64-token chunk resident at once --
+// matter more than loads in flight: the gather is bound by what L2 delivers): the k2c rows give the softplus gates, the vc rows are accumulated with weight
 // exp(s - max) . gate, eight columns of the output per lane.  The sum of exp(s - max) normalises the result.
 struct SelShared {
+    float col[kColRows];
     int idx[kSelWarps][kListCap];
     float sc[kSelWarps][kListCap];
     float q2[128];
@@ -245,7 +247,7 @@ struct SelShared {
     float theta;
 };
 
-__global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const ChunkParams p) {
+__global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const ChunkParams p) {
     extern __shared__ __align__(16) unsigned char sel_raw[];
     SelShared& sh = *reinterpret_cast<SelShared*>(sel_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -260,17 +262,24 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
     // slices of the visible range, one per warp
     const int per = (L + kSelWarps - 1) / kSelWarps;
     const int w0 = lo + warp * per, w1 = min(n, w0 + per);
-    // A slice of up to 1024 rows stays in registers (32 per lane) between the statistics and the selection, so
-    // the column is read once; longer slices are read again.
-    constexpr int kKeep = 32;
-    const bool kept = per <= 32 * kKeep;
-    float keep[kKeep];
+    // A column of up to 8192 visible rows stays in shared memory between the statistics and the selection, so it is
+    // read once; longer columns are read again.
+    const bool kept = L <= kColRows;
     if (kept) {
+        for (int j0 = w0; j0 < w1; j0 += 32 * 8) {          // eight loads per lane in flight
+            float sv[8];
 #pragma unroll
-        for (int u = 0; u < kKeep; ++u) {
-            const int j = w0 + 32 * u + lane;
-            keep[u] = j < w1 ? __ldcg(scol + j) : -INFINITY;
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + 32 * u + lane;
+                sv[u] = j < w1 ? __ldcg(scol + j) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + 32 * u + lane;
+                if (j < w1) sh.col[j - lo] = sv[u];
+            }
         }
+        __syncwarp();
     }
     if (p.k_attn < L) {
         // sums of the column over the rows this query may see, around the column's first value (keeps the fp32
@@ -278,9 +287,8 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
         const float c0 = __ldcg(scol + lo);
         float f1 = 0.f, f2 = 0.f;
         if (kept) {
-#pragma unroll
-            for (int u = 0; u < kKeep; ++u) {
-                const float d = w0 + 32 * u + lane < w1 ? keep[u] - c0 : 0.f;
+            for (int j = w0 + lane; j < w1; j += 32) {
+                const float d = sh.col[j - lo] - c0;
                 f1 += d;
                 f2 = fmaf(d, d, f2);
             }
@@ -424,8 +432,7 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
             // the order of the list does not matter: every lane counts its own survivors, a scan of the counts gives it
             // a place, and it writes them there -- no ballot per 32 rows
             int mine = 0;
-#pragma unroll
-            for (int u = 0; u < kKeep; ++u) mine += (keep[u] > th) ? 1 : 0;          // rows past the slice hold -inf
+            for (int j = w0 + lane; j < w1; j += 32) mine += (sh.col[j - lo] > th) ? 1 : 0;
             int incl = mine;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -435,12 +442,12 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
             const int all = __shfl_sync(kFull, incl, 31);
             if (all <= kListCap) {
                 int at = incl - mine;
-#pragma unroll
-                for (int u = 0; u < kKeep; ++u) {
-                    if (keep[u] > th) {
-                        sh.idx[warp][at] = w0 + 32 * u + lane;
-                        sh.sc[warp][at] = keep[u];
-                        mx = fmaxf(mx, keep[u]);
+                for (int j = w0 + lane; j < w1; j += 32) {
+                    const float v = sh.col[j - lo];
+                    if (v > th) {
+                        sh.idx[warp][at] = j;
+                        sh.sc[warp][at] = v;
+                        mx = fmaxf(mx, v);
                         ++at;
                     }
                 }
@@ -451,10 +458,9 @@ __global__ void __launch_bounds__(kSelThreads, 3) attn_chunk_select_kernel(const
         if (listed) {
             // done
         } else if (kept) {
-#pragma unroll
-            for (int u = 0; u < kKeep; ++u) {
-                const int j = w0 + 32 * u + lane;
-                if (w0 + 32 * u < w1) take(j, keep[u], j < w1);
+            for (int j0 = w0; j0 < w1; j0 += 32) {
+                const int j = j0 + lane;
+                take(j, j < w1 ? sh.col[j - lo] : -INFINITY, j < w1);
             }
         } else {
             for (int j0 = w0; j0 < w1; j0 += 32 * 8) {          // eight loads per lane in flight
