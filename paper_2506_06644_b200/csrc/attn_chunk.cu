@@ -11,6 +11,8 @@
 //           survivors, softmax over the survivors, softplus gate from the k2c rows, weighted sum of the vc rows
 //           (only the survivors' rows are read)
 // Same pipeline skeleton and bounded waits as the other tensor-core kernels (tc_common.cuh).
+#include <cstddef>
+
 #include "kernels.h"
 #include "tc_common.cuh"
 
@@ -22,7 +24,6 @@ namespace {
 constexpr int kColMax = 128;          // (token, head-in-group) columns per KV head
 constexpr int kSelThreads = 256;
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kListCap = 128;         // survivors a warp of the select kernel lists before it gathers them
 constexpr int kColRows = 8192;        // visible rows of a column the select kernel keeps in shared memory
 
 struct ChunkParams {
@@ -234,8 +235,10 @@ attn_chunk_scores_kernel(const ChunkParams p, const __grid_constant__ CUtensorMa
 // four survivors at a time (four blocks per SM -- all 512 (token, head) pairs of a 64-token chunk resident at once --
 // matter more than loads in flight: the gather is bound by what L2 delivers): the k2c rows give the softplus gates, the vc rows are accumulated with weight
 // exp(s - max) . gate, eight columns of the output per lane.  The sum of exp(s - max) normalises the result.
+// REGS: see the kernel below (the list capacity and the column buffer differ between its two variants)
+template <bool REGS>
 struct SelShared {
-    float col[kColRows];
+    static constexpr int kListCap = REGS ? 512 : 192;      // survivors a warp lists before it gathers them
     int idx[kSelWarps][kListCap];
     float sc[kSelWarps][kListCap];
     float q2[128];
@@ -245,11 +248,16 @@ struct SelShared {
     int cnt[kSelWarps];
     double part[kSelWarps][2];
     float theta;
+    __align__(16) float col[REGS ? 4 : kColRows + 4];
 };
 
-__global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const ChunkParams p) {
+// REGS: a slice of up to 1024 rows per warp stays in registers (three blocks per SM; the faster block when all blocks
+// are resident anyway); otherwise the column is staged in shared memory (64 registers, four blocks per SM).
+template <bool REGS>
+__global__ void __launch_bounds__(kSelThreads, REGS ? 3 : 4) attn_chunk_select_kernel(const ChunkParams p) {
     extern __shared__ __align__(16) unsigned char sel_raw[];
-    SelShared& sh = *reinterpret_cast<SelShared*>(sel_raw);
+    SelShared<REGS>& sh = *reinterpret_cast<SelShared<REGS>*>(sel_raw);
+    constexpr int kListCap = SelShared<REGS>::kListCap;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int t = blockIdx.x / p.n_q, h = blockIdx.x - t * p.n_q;
     const int g = h / p.gq, col = t * p.gq + (h - g * p.gq);
@@ -259,26 +267,31 @@ __global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const
     const int lo = p.range[2 * t], n = p.range[2 * t + 1], L = n - lo;
     if (tid < d2) sh.q2[tid] = p.q[(static_cast<int64_t>(t) * p.n_q + h) * p.hd + p.r + tid];
     const float* scol = p.S + (static_cast<int64_t>(g) * kColMax + col) * p.scap;
-    // slices of the visible range, one per warp
-    const int per = (L + kSelWarps - 1) / kSelWarps;
-    const int w0 = lo + warp * per, w1 = min(n, w0 + per);
-    // A column of up to 8192 visible rows stays in shared memory between the statistics and the selection, so it is
-    // read once; longer columns are read again.
-    const bool kept = L <= kColRows;
-    if (kept) {
-        for (int j0 = w0; j0 < w1; j0 += 32 * 8) {          // eight loads per lane in flight
-            float sv[8];
+    // slices of the visible range, one per warp; with the column in shared memory they start on 16-byte boundaries
+    // of the column (lo4 <= lo)
+    const int lo4 = REGS ? lo : (lo & ~3);
+    const int per = REGS ? (L + kSelWarps - 1) / kSelWarps : ((((n - lo4) + kSelWarps - 1) / kSelWarps + 3) & ~3);
+    const int w0 = max(lo, lo4 + warp * per), w1 = min(n, lo4 + (warp + 1) * per);
+    constexpr int kKeep = REGS ? 32 : 1;
+    const bool kept = REGS ? per <= 32 * kKeep : n - lo4 <= kColRows;
+    [[maybe_unused]] float keep[kKeep];
+    if constexpr (REGS) {
+        if (kept) {      // up to 1024 rows of the slice in registers, all loads in flight at once
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int j = j0 + 32 * u + lane;
-                sv[u] = j < w1 ? __ldcg(scol + j) : 0.f;
-            }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int j = j0 + 32 * u + lane;
-                if (j < w1) sh.col[j - lo] = sv[u];
+            for (int u = 0; u < kKeep; ++u) {
+                const int j = w0 + 32 * u + lane;
+                keep[u] = j < w1 ? __ldcg(scol + j) : -INFINITY;
             }
         }
+    } else if (kept) {
+        // asynchronous 16-byte copies straight into shared memory: the whole slice is in flight at once and no
+        // registers are held (rows past n inside the last 16 bytes are copied too and never looked at)
+        const int c0 = lo4 + warp * per, c1 = min((n + 3) & ~3, c0 + per);
+        const unsigned dst0 = static_cast<unsigned>(__cvta_generic_to_shared(sh.col));
+        for (int j = c0 + 4 * lane; j < c1; j += 128)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + 4u * static_cast<unsigned>(j - lo4)), "l"(scol + j) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncwarp();
     }
     if (p.k_attn < L) {
@@ -287,10 +300,19 @@ __global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const
         const float c0 = __ldcg(scol + lo);
         float f1 = 0.f, f2 = 0.f;
         if (kept) {
-            for (int j = w0 + lane; j < w1; j += 32) {
-                const float d = sh.col[j - lo] - c0;
-                f1 += d;
-                f2 = fmaf(d, d, f2);
+            if constexpr (REGS) {
+#pragma unroll
+                for (int u = 0; u < kKeep; ++u) {
+                    const float d = w0 + 32 * u + lane < w1 ? keep[u] - c0 : 0.f;
+                    f1 += d;
+                    f2 = fmaf(d, d, f2);
+                }
+            } else {
+                for (int j = w0 + lane; j < w1; j += 32) {
+                    const float d = sh.col[j - lo4] - c0;
+                    f1 += d;
+                    f2 = fmaf(d, d, f2);
+                }
             }
         } else {
             for (int j0 = w0; j0 < w1; j0 += 32 * 16) {
@@ -432,7 +454,12 @@ __global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const
             // the order of the list does not matter: every lane counts its own survivors, a scan of the counts gives it
             // a place, and it writes them there -- no ballot per 32 rows
             int mine = 0;
-            for (int j = w0 + lane; j < w1; j += 32) mine += (sh.col[j - lo] > th) ? 1 : 0;
+            if constexpr (REGS) {
+#pragma unroll
+                for (int u = 0; u < kKeep; ++u) mine += (keep[u] > th) ? 1 : 0;          // rows past the slice hold -inf
+            } else {
+                for (int j = w0 + lane; j < w1; j += 32) mine += (sh.col[j - lo4] > th) ? 1 : 0;
+            }
             int incl = mine;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -442,13 +469,25 @@ __global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const
             const int all = __shfl_sync(kFull, incl, 31);
             if (all <= kListCap) {
                 int at = incl - mine;
-                for (int j = w0 + lane; j < w1; j += 32) {
-                    const float v = sh.col[j - lo];
-                    if (v > th) {
-                        sh.idx[warp][at] = j;
-                        sh.sc[warp][at] = v;
-                        mx = fmaxf(mx, v);
-                        ++at;
+                if constexpr (REGS) {
+#pragma unroll
+                    for (int u = 0; u < kKeep; ++u) {
+                        if (keep[u] > th) {
+                            sh.idx[warp][at] = w0 + 32 * u + lane;
+                            sh.sc[warp][at] = keep[u];
+                            mx = fmaxf(mx, keep[u]);
+                            ++at;
+                        }
+                    }
+                } else {
+                    for (int j = w0 + lane; j < w1; j += 32) {
+                        const float v = sh.col[j - lo4];
+                        if (v > th) {
+                            sh.idx[warp][at] = j;
+                            sh.sc[warp][at] = v;
+                            mx = fmaxf(mx, v);
+                            ++at;
+                        }
                     }
                 }
                 cnt = all;
@@ -458,9 +497,17 @@ __global__ void __launch_bounds__(kSelThreads, 4) attn_chunk_select_kernel(const
         if (listed) {
             // done
         } else if (kept) {
-            for (int j0 = w0; j0 < w1; j0 += 32) {
-                const int j = j0 + lane;
-                take(j, j < w1 ? sh.col[j - lo] : -INFINITY, j < w1);
+            if constexpr (REGS) {
+#pragma unroll
+                for (int u = 0; u < kKeep; ++u) {
+                    const int j = w0 + 32 * u + lane;
+                    if (w0 + 32 * u < w1) take(j, keep[u], j < w1);
+                }
+            } else {
+                for (int j0 = w0; j0 < w1; j0 += 32) {
+                    const int j = j0 + lane;
+                    take(j, j < w1 ? sh.col[j - lo4] : -INFINITY, j < w1);
+                }
             }
         } else {
             for (int j0 = w0; j0 < w1; j0 += 32 * 8) {          // eight loads per lane in flight
@@ -526,6 +573,7 @@ int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const voi
     const int64_t gq = n_q / n_kv, d2 = hd - r;
     if (T < 1 || T > 64 || T * gq > kColMax || (gq != 1 && gq != 2 && gq != 4 && gq != 8)) return SPARK_ERR_WORKSPACE;
     if ((r != 64 && r != 128) || d2 < 8 || d2 > 128 || (d2 & 7) != 0 || hd > 256 || (hd & 7) != 0) return SPARK_ERR_WORKSPACE;
+    if ((cap & 3) != 0) return SPARK_ERR_WORKSPACE;          // 16-byte copies out of the score columns
     if (n_kv * cap >= (1LL << 31) || ((reinterpret_cast<uintptr_t>(k1c) | reinterpret_cast<uintptr_t>(k2c) | reinterpret_cast<uintptr_t>(vc)) & 15u) != 0)
         return SPARK_ERR_WORKSPACE;
     const size_t small_b = round_up(static_cast<size_t>(T) * (sizeof(double) + 2 * sizeof(int)), 1024);
@@ -560,7 +608,8 @@ int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const voi
         !make_map(&m_qlo, p.qlo, n_kv * kColMax, r, r, p.ncolp, false))
         return SPARK_ERR_WORKSPACE;
     if (cudaFuncSetAttribute(attn_chunk_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_scores)) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_chunk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(SelShared))) != cudaSuccess)
+        cudaFuncSetAttribute(attn_chunk_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(SelShared<true>))) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_chunk_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(SelShared<false>))) != cudaSuccess)
         return SPARK_ERR_CUDA;
     {
         void* args[] = {&p};
@@ -574,7 +623,11 @@ int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const voi
     }
     {
         void* args[] = {&p};
-        if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_select_kernel), static_cast<unsigned>(T * n_q), kSelThreads, sizeof(SelShared), stream, false, args) != cudaSuccess)
+        // all blocks resident at three per SM: the register variant; more blocks than that: four per SM
+        const bool regs = T * n_q <= 3 * static_cast<int64_t>(ctx->num_sms);
+        const size_t sel_smem = regs ? sizeof(SelShared<true>) : sizeof(SelShared<false>);
+        const void* sel = regs ? reinterpret_cast<const void*>(attn_chunk_select_kernel<true>) : reinterpret_cast<const void*>(attn_chunk_select_kernel<false>);
+        if (launch_kernel(ctx, sel, static_cast<unsigned>(T * n_q), kSelThreads, sel_smem, stream, false, args) != cudaSuccess)
             return SPARK_ERR_CUDA;
     }
     return SPARK_OK;
