@@ -175,3 +175,14 @@ def test_argument_errors(ctx):
         assert e.value.status == code, bad
     call()
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_seeded_random_shapes_of_the_chunk_path(ctx, seed):
+    # widths, predictor splits (r close to 0 and close to d), neuron counts, token counts and k from a seeded generator
+    rng = np.random.default_rng(500 + seed)
+    d = 256 * int(rng.integers(1, 4)); r = 64 * int(rng.integers(1, d // 64)); d_ff = 128 * int(rng.integers(2, 24)); B = int(rng.integers(5, 65))
+    k = max(1, int(d_ff * float(rng.choice([0.02, 0.08, 0.3]))))
+    p = synth.ffn_inputs(d, d_ff, r, k, B, "bf16", seed=600 + seed)
+    out = run_ffn(ctx, p, weights=upload(p))
+    assert compare(p, out) < 5e-3

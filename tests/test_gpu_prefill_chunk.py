@@ -158,3 +158,32 @@ def test_prefill_loop_over_two_layers_and_ragged_chunks(ctx):
         ref[t] = x
     for t in range(N):
         parity.check_output(got[t], ref[t], "bf16", f"token {t}")
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_seeded_random_shapes_of_the_chunk_attention(ctx, seed):
+    # head layouts, chunk lengths, cache fill, k and windows drawn from a seeded generator (shapes the tensor-core path serves)
+    rng = np.random.default_rng(1000 + seed)
+    gq = int(rng.choice([1, 2, 4])); n_kv = int(rng.choice([1, 2, 4])); n_q = gq * n_kv
+    hd, r = [(256, 128), (128, 64), (192, 128)][int(rng.integers(3))]
+    T = int(rng.integers(16, min(64, 128 // gq) + 1)); cap = 4 * int(rng.integers(40, 160))
+    L0 = int(rng.integers(0, cap - T + 1)); k_attn = int(rng.choice([8, 40, 200])); window = int(rng.choice([0, 0, 37, 300]))
+    kv = synth.attn_inputs(1, n_q, n_kv, hd, r, cap, [cap], "bf16", seed=2000 + seed)
+    q = synth.normal_f32((T, n_q, hd), 3000 + seed, 0) * hd ** -0.5
+    lens = [L0 + t + 1 for t in range(T)]
+    o = torch.full((T, n_q, hd), float("nan"), device="cuda")
+    theta = torch.empty(T, n_q, device="cuda")
+    S.spark_attn_decode(ctx, torch.from_numpy(q).cuda(), bf16_dev(kv.k1c_bits[0]), bf16_dev(kv.k2c_bits[0]), bf16_dev(kv.vc_bits[0]),
+                        S.SPARK_BF16, T, n_q, n_kv, hd, r, cap, torch.tensor(lens, dtype=torch.int32, device="cuda"), window, k_attn,
+                        S.SPARK_SHARED_CACHE, o, theta, None, None, 0)
+    torch.cuda.synchronize()
+    kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+    vc = kv.vc[0].astype(np.float64)
+    og, thg = o.cpu().numpy(), theta.cpu().numpy()
+    for t in range(T):
+        ref = O.spark_attention(q[t].astype(np.float64), kc, vc, lens[t], k_attn, r, window)
+        for h in range(n_q):
+            lo = 0 if window <= 0 else max(0, lens[t] - window)
+            s = kc[h // gq, lo:lens[t], :r] @ q[t, h, :r].astype(np.float64)
+            parity.check_theta(thg[t, h], ref["theta"][h], float(np.std(s, ddof=1)) if s.size > 1 else 1.0, f"token {t} head {h}")
+        parity.check_output(og[t].reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"token {t}")
