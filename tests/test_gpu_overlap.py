@@ -45,6 +45,7 @@ def chain(ctx, sh, B, cap, lens, window, calls, seed=4):
     (synth.TINY, 3, 128, [128, 1, 17], 0),
     (synth.GEMMA2_2B, 1, 2048, [2048], 0),
     (synth.GEMMA2_2B, 2, 1024, [700, 1024], 512),
+    (synth.GEMMA2_2B, 8, 256, [256, 200, 77, 1, 150, 60, 3, 90], 0),      # projections and FFN on the tcgen05 kernels
 ])
 def test_one_layer_call_against_oracle(ctx_pair, shape, B, cap, lens, window):
     _, over = ctx_pair
@@ -56,7 +57,8 @@ def test_one_layer_call_against_oracle(ctx_pair, shape, B, cap, lens, window):
 
 
 @pytest.mark.parametrize("shape,B,cap,lens", [(synth.TINY, 2, 128, [100, 90]), (synth.GEMMA2_2B, 1, 4096, [4096]),
-                                               (synth.GEMMA2_2B, 4, 512, [512, 300, 77, 1])])
+                                               (synth.GEMMA2_2B, 4, 512, [512, 300, 77, 1]),
+                                               (synth.GEMMA2_2B, 8, 256, [256, 200, 77, 1, 150, 60, 3, 90])])     # tcgen05 kernels in the chain
 def test_chain_of_calls_matches_ordinary_launches(ctx_pair, shape, B, cap, lens):
     plain, over = ctx_pair
     a = chain(plain, shape, B, cap, lens, 0, calls=6)[3]
@@ -70,7 +72,7 @@ def test_chain_of_calls_matches_ordinary_launches(ctx_pair, shape, B, cap, lens)
         assert err <= parity.OUT_TOL["bf16"], f"chain differs by {err:.2e} of the RMS"
 
 
-@pytest.mark.parametrize("B", [1, 4])
+@pytest.mark.parametrize("B", [1, 4, 12])
 def test_ffn_calls_back_to_back(ctx_pair, B):
     # FFN launches in a row use different accumulator ring slots: a launch must not pick its slot
     # before the one before it has advanced the launch count
