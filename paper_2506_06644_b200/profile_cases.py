@@ -8,6 +8,7 @@
     python -m paper_2506_06644_b200.profile_cases topk    # statistical top-k, 512 rows x 65536
     python -m paper_2506_06644_b200.profile_cases layer   # four decoder layers, one token
     python -m paper_2506_06644_b200.profile_cases chunk64 # four decoder layers over a 64-token chunk of a prompt
+    python -m paper_2506_06644_b200.profile_cases layer8  # four decoder layers, eight sequences
 
 Every case cycles over enough distinct weight sets / caches / rows to exceed the 126 MB L2, holds at
 most about 1 GB on the device and launches a dozen kernels, so that a capture of two or three of
@@ -139,7 +140,7 @@ def case_chunk(n_layers=4, T=64, ctx_len=8192, steps=2):
     assert ctx.device_status() == S.SPARK_OK
 
 
-CASES = {"chunk64": case_chunk, "ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
+CASES = {"chunk64": case_chunk, "layer8": lambda: case_layer(n_layers=4, B=8, steps=2), "ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
 
 if __name__ == "__main__":
     name = sys.argv[1] if len(sys.argv) > 1 else ""
