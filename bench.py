@@ -14,6 +14,9 @@ starting and ending in pinned host memory.  `roofline` is for the dominant kerne
 FFN kernel): touched bytes (all of K1t plus the active rows of K2t and Vt) over its average
 duration, timed with CUDA events over a loop of the same launches.  `cpu_baseline` times the fp64
 oracle on the host cores on a bounded sample.  `--impl reference` times only that oracle.
+The default run (2B shape, batch 1) also measures, under `stacks`, the 42-layer 9B-shape stack at
+batch 1 and the 2B-shape stack at batch 8, and under `other_workloads` the remaining configurations
+(batched FFN, attention at 4096 to 32768 tokens, the LM head, statistical top-k on three distributions).
 """
 from __future__ import annotations
 
@@ -31,9 +34,9 @@ if ROOT not in sys.path:
 
 import numpy as np
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from the ncu
-# capture summarised in profiles/ (keyed by shape and batch); None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {("2b", 1): 25.04e6}       # profiles/ffn_b1.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel, from one ncu
+# capture of that kernel (keyed by shape and batch); None where no capture exists.
+NCU_TRAFFIC_BYTES = {("2b", 1): 25.04e6}
 
 FALLBACK_HBM_GBS = 6650.0
 
@@ -203,28 +206,22 @@ def us_per_token_per_layer(ms_total, steps, n_layers, batch, world):
 # --------------------------------------------------------------------------------------------
 # the CUDA arm
 # --------------------------------------------------------------------------------------------
-def run_spark(args):
-    import torch
-    import torch.distributed as dist
+def step_stats(events, torch):
+    """Per-step times (ms) from the events recorded around every step of a timed loop."""
+    per = np.array([events[i].elapsed_time(events[i + 1]) for i in range(len(events) - 1)])
+    return {"mean": float(per.mean()), "median": float(np.median(per)), "min": float(per.min())}
 
-    from paper_2506_06644_b200 import binding as S
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    shape = shape_of(args.shape)
-    n_layers = args.layers or shape.n_layers
-    B, ctx_len, d, hd = args.batch, args.ctx, shape.d, shape.hd
-    W = max(args.warmup, 3)
-    cap = ctx_len + args.steps + W + 8                  # the prompt plus every token decoded in one timed loop
-    ctx = S.SparkContext(local, max_batch=B, max_dff=shape.d_ff, max_cap=cap, n_q=shape.n_q, hd=hd, max_d=d)
-    ctx.set_launch_overlap(bool(args.overlap))
-
+def measure_stack(torch, S, dist, dev, rank, world, shape_name, B, ctx_len, n_layers, steps, W, overlap, no_graph, no_dense,
+                  with_e2e, with_kernels):
+    """Build the decoder stack of `shape_name` for B sequences behind ctx_len cached tokens, time `steps` decode steps of
+    the whole stack (plus its dense-loads comparator, the end-to-end variant and the per-kernel loops), free it, and
+    return the figures.  One step decodes one token per sequence through every layer."""
+    shape = shape_of(shape_name)
+    d, hd = shape.d, shape.hd
+    cap = ctx_len + steps + W + 8                       # the prompt plus every token decoded in one timed loop
+    ctx = S.SparkContext(dev.index, max_batch=B, max_dff=shape.d_ff, max_cap=cap, n_q=shape.n_q, hd=hd, max_d=d)
+    ctx.set_launch_overlap(bool(overlap))
     gen = torch.Generator(device=dev)
     gen.manual_seed(1234 + rank)
 
@@ -232,7 +229,7 @@ def run_spark(args):
         return (torch.randn(rows, cols, device=dev, generator=gen) * (fan_in ** -0.5)).to(torch.bfloat16)
 
     nqkv = (shape.n_q + 2 * shape.n_kv) * hd
-    layers, keep = [], []
+    layers = []
     for l in range(n_layers):
         w = dict(norm1=1.0 + 0.1 * torch.randn(d, device=dev, generator=gen),
                  norm2=1.0 + 0.1 * torch.randn(d, device=dev, generator=gen),
@@ -251,7 +248,7 @@ def run_spark(args):
     h_init = torch.randn(B, d, device=dev, generator=gen)
     h = torch.empty_like(h_init)
     cl = torch.full((B,), ctx_len + 1, dtype=torch.int32, device=dev)   # valid tokens, the one being decoded included
-    scratch = torch.empty(B * (nqkv + 2 * shape.n_q * hd + d + 2 + shape.n_q), device=dev)
+    scratch = torch.empty(S.layer_scratch_floats(dict(n_q=shape.n_q, n_kv=shape.n_kv, hd=hd, d=d), B), device=dev)
     h_host_in = h_init.cpu().pin_memory()
     h_host_out = torch.empty_like(h_host_in).pin_memory()
     # QKV (+ rotary, append: a kernel of their own for B >= 5), attention, output projection, FFN; for B >= 5 the projections
@@ -267,22 +264,25 @@ def run_spark(args):
     graphs = {}
     side = torch.cuda.Stream()
 
+    def capture_of(calls):
+        with torch.cuda.stream(side):
+            calls()                                        # warm-up outside capture (first-call set-up)
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                calls()
+        torch.cuda.synchronize()
+        return g
+
     def capture():
         graphs.clear()
-        if args.no_graph:
+        if no_graph:
             return
-        for which in ((0,) if args.no_dense else (0, 1)):
-            with torch.cuda.stream(side):
-                stack(which)                               # warm-up outside capture (first-call set-up)
-                side.synchronize()
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=side):
-                    stack(which)
-            graphs[which] = g
-        torch.cuda.synchronize()
+        for which in ((0,) if no_dense else (0, 1)):
+            graphs[which] = capture_of(lambda: stack(which))
 
     capture()
-    overlap_on = bool(args.overlap)
+    overlap_on = bool(overlap)
     if overlap_on:
         # Launch overlap needs the GPU to itself (its blocks must all become resident).  Try it once; if a
         # block gave up waiting, go back to ordinary cooperative launches and say so in the result.
@@ -314,34 +314,42 @@ def run_spark(args):
         h_host_out.copy_(h, non_blocking=True)            # device -> pinned host
         torch.cuda.current_stream().synchronize()
 
-    def timed(fn, steps, warmup):
-        cl.fill_(ctx_len + 1)
+    def timed(fn, nsteps, warmup, reset=True):
+        """Total ms of nsteps calls of fn (max over ranks) and the per-step statistics of this rank."""
+        if reset:
+            cl.fill_(ctx_len + 1)
         for _ in range(warmup):
             fn()
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(nsteps + 1)]
+        ev[0].record()
+        for i in range(nsteps):
             fn()
-        e1.record()
+            ev[i + 1].record()
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)
+        return max_over_ranks(ev[0].elapsed_time(ev[-1]), world, dev), step_stats(ev, torch)
 
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(dev.index)
     sampler.start()
-    ms_total = timed(step, args.steps, W)
+    ms_total, st_total = timed(step, steps, W)
     clocks = sampler.stop()
-    ms_e2e = timed(step_e2e, args.steps, W)
-    ms_dense = None if args.no_dense else timed(lambda: step(1), args.steps, W)
+    ms_e2e = timed(step_e2e, steps, W)[0] if with_e2e else None
+    ms_dense, st_dense = (None, None) if no_dense else timed(lambda: step(1), steps, W)
     status = ctx.device_status()
     assert status == S.SPARK_OK, f"device status {status}"
     assert torch.isfinite(h).all()
 
-    # ---- roofline of the dominant kernel: the fused FFN kernel on the same weights ----------------
+    # ---- the kernels of a layer one by one, each as a CUDA graph of n_layers launches over the layers' own weights and
+    #      caches (more data than L2 holds): FFN, attention, the two projections ------------------------------------
+    peak, peak_kind = measured_peak()
+    out = {"shape": shape_name, "batch": B, "ctx": ctx_len, "n_layers": n_layers, "kernels_per_layer": kernels_per_layer,
+           "overlap_on": overlap_on, "ms_total": ms_total, "steps_ms": st_total, "ms_e2e": ms_e2e, "ms_dense": ms_dense,
+           "steps_ms_dense": st_dense, "clocks": clocks,
+           "h2d_bytes_per_step": int(h_host_in.numel() * 4), "d2h_bytes_per_step": int(h_host_out.numel() * 4)}
     xn = torch.nn.functional.normalize(h_init, dim=1) * (d ** 0.5)
     y = torch.empty_like(xn)
     cnt = torch.zeros(B, dtype=torch.int32, device=dev)
@@ -355,99 +363,157 @@ def run_spark(args):
         ids = torch.cat([idx[b, : int(cnt[b])] for b in range(B)])
         unions.append(int(torch.unique(ids).numel()))
     union = float(np.mean(unions))
+    out["union_rows"] = union
+    out["layer_touched_bytes"] = touched_layer_bytes(shape, B, ctx_len, union if B <= 4 else shape.d_ff, n_layers)
+    if with_kernels:
+        def loop_us(calls):
+            g = None if no_graph else capture_of(calls)
+            ms, st = timed(lambda: g.replay() if g is not None else calls(), steps, W, reset=False)
+            return {"us_per_launch": ms * 1e3 / (steps * n_layers), "median_us": st["median"] * 1e3 / n_layers,
+                    "min_us": st["min"] * 1e3 / n_layers}
 
-    def ffn_calls():
-        for lay in layers:
-            w = lay[2]
-            S.spark_ffn_decode(ctx, xn, B, w["K1t"], w["K2t"], w["Vt"], S.SPARK_BF16, d, shape.d_ff, shape.r_ff,
-                               shape.k_ff, 0, y, None, None, None)
+        def entry(name, t, nbytes):
+            t.update({"kernel": name, "bound": "hbm", "touched_bytes_per_launch": nbytes, "unit": "GB/s", "peak": peak,
+                      "achieved": nbytes / (t["us_per_launch"] * 1e-6) / 1e9,
+                      "frac": nbytes / (t["us_per_launch"] * 1e-6) / 1e9 / peak, "peak_kind": f"of {peak_kind}"})
+            return t
 
-    ffn_graph = None
-    if not args.no_graph:
-        with torch.cuda.stream(side):
-            ffn_calls()
-            side.synchronize()
-            ffn_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(ffn_graph, stream=side):
-                ffn_calls()
-        torch.cuda.synchronize()
+        def ffn_calls():
+            for lay in layers:
+                w = lay[2]
+                S.spark_ffn_decode(ctx, xn, B, w["K1t"], w["K2t"], w["Vt"], S.SPARK_BF16, d, shape.d_ff, shape.r_ff,
+                                   shape.k_ff, 0, y, None, None, None)
+        cl.fill_(ctx_len + 1)
+        rows_read = union if B <= 4 else shape.d_ff
+        out["ffn"] = entry(("ffn1_kernel" if B == 1 else "ffn_few_kernel" if B <= 4 else "ffn_tc_{prep,scores,act,out}_kernel") +
+                           " (spark_ffn_decode)", loop_us(ffn_calls), shape.d_ff * shape.r_ff * 2 + rows_read * (2 * d - shape.r_ff) * 2)
 
-    def ffn_loop():
-        if ffn_graph is not None:
-            ffn_graph.replay()
-        else:
-            ffn_calls()
+        qa = torch.randn(B, shape.n_q, hd, device=dev, generator=gen) / (hd ** 0.5)
+        oa = torch.empty(B, shape.n_q, hd, device=dev)
 
-    ms_ffn = timed(ffn_loop, args.steps, W)
+        def attn_calls():
+            for l, lay in enumerate(layers):
+                c = lay[3]
+                win = 4096 if (l % 2 == 0 and ctx_len > 4096) else 0
+                S.spark_attn_decode(ctx, qa, c["k1c"], c["k2c"], c["vc"], S.SPARK_BF16, B, shape.n_q, shape.n_kv, hd,
+                                    shape.r_attn, cap, cl, win, shape.k_attn, 0, oa, None, None, None, 0)
+        avg_ctx = (min(ctx_len, 4096) + ctx_len) / 2 if ctx_len > 4096 else ctx_len
+        attn_bytes = B * (shape.n_kv * avg_ctx * shape.r_attn * 2 +
+                          shape.n_q * min(shape.k_attn, avg_ctx) * ((hd - shape.r_attn) + hd) * 2)
+        out["attn"] = entry("attn_kernel (spark_attn_decode)", loop_us(attn_calls), attn_bytes)
 
-    # ---- the attention kernel alone, same caches (second largest share of the step) ------------------
-    qa = torch.randn(B, shape.n_q, hd, device=dev, generator=gen) / (hd ** 0.5)
-    oa = torch.empty(B, shape.n_q, hd, device=dev)
+        yq = torch.empty(B, nqkv, device=dev)
+        yo = torch.empty(B, d, device=dev)
+        xo = torch.randn(B, shape.n_q * hd, device=dev, generator=gen)
 
-    def attn_calls():
-        for l, lay in enumerate(layers):
-            c = lay[3]
-            win = 4096 if (l % 2 == 0 and ctx_len > 4096) else 0
-            S.spark_attn_decode(ctx, qa, c["k1c"], c["k2c"], c["vc"], S.SPARK_BF16, B, shape.n_q, shape.n_kv, hd,
-                                shape.r_attn, cap, cl, win, shape.k_attn, 0, oa, None, None, None, 0)
+        def qkv_calls():
+            for lay in layers:
+                S.spark_dense_gemv(ctx, xn, B, lay[2]["Wqkv"], S.SPARK_BF16, d, nqkv, None, yq)
 
-    attn_graph = None
-    if not args.no_graph:
-        with torch.cuda.stream(side):
-            attn_calls()
-            side.synchronize()
-            attn_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(attn_graph, stream=side):
-                attn_calls()
-        torch.cuda.synchronize()
-    ms_attn = timed(lambda: attn_graph.replay() if attn_graph is not None else attn_calls(), args.steps, W)
-    attn_us = ms_attn * 1e3 / (args.steps * n_layers)
-    avg_ctx = (min(ctx_len, 4096) + ctx_len) / 2 if ctx_len > 4096 else ctx_len
-    attn_bytes = B * (shape.n_kv * avg_ctx * shape.r_attn * 2 +
-                      shape.n_q * min(shape.k_attn, avg_ctx) * ((hd - shape.r_attn) + hd) * 2)
-    ffn_us = ms_ffn * 1e3 / (args.steps * n_layers)
-    touched = shape.d_ff * shape.r_ff * 2 + union * (2 * d - shape.r_ff) * 2       # bytes per launch
+        def wo_calls():
+            for lay in layers:
+                S.spark_dense_gemv(ctx, xo, B, lay[2]["Wo"], S.SPARK_BF16, shape.n_q * hd, d, None, yo)
+        out["qkv_proj"] = entry("gemv_kernel / gemm_tc_kernel on Wqkv (spark_dense_gemv; the layer fuses norm, rotary, append)",
+                                loop_us(qkv_calls), nqkv * d * 2)
+        out["o_proj"] = entry("gemv_kernel / gemm_tc_kernel on Wo (spark_dense_gemv)", loop_us(wo_calls), d * shape.n_q * hd * 2)
+        assert ctx.device_status() == S.SPARK_OK
+    ctx.close()
+    del layers, graphs
+    torch.cuda.empty_cache()
+    return out
+
+
+def stack_summary(m, world, peak):
+    """The reported figures of one measured stack (see measure_stack)."""
+    steps_ms = m["steps_ms"]
+    per = 1e3 / (m["n_layers"] * m["batch"] * world)          # ms per step -> us per token per layer
+    n = m["n_layers"]
+    us_layer_call = steps_ms["mean"] * 1e3 / n
+    touched = m["layer_touched_bytes"]
+    s = {"workload": f"gemma2-{m['shape']}-shape spark decoder, {n} layers, batch {m['batch']}, context {m['ctx']} "
+                     "(local 4096 / global layers alternate), one CUDA graph replay per decode step",
+         "us_per_token_per_layer": steps_ms["mean"] * per, "median_us_per_token_per_layer": steps_ms["median"] * per,
+         "min_us_per_token_per_layer": steps_ms["min"] * per, "ms_per_step": steps_ms["mean"],
+         "tokens_per_s": m["batch"] * world / (steps_ms["mean"] * 1e-3),
+         "layer_touched_mb": touched / 1e6, "layer_gbs_touched": touched / (us_layer_call * 1e-6) / 1e9,
+         "layer_frac_of_measured_peak": touched / (us_layer_call * 1e-6) / 1e9 / peak,
+         "layer_frac_of_8tbs": touched / (us_layer_call * 1e-6) / 8e12,
+         "union_rows_ffn": m["union_rows"], "launch_overlap": m["overlap_on"]}
+    if m["ms_dense"] is not None:
+        s["dense_loads"] = {"us_per_token_per_layer": m["steps_ms_dense"]["mean"] * per,
+                            "median_us_per_token_per_layer": m["steps_ms_dense"]["median"] * per,
+                            "speedup_spark_vs_dense_loads": m["ms_dense"] / m["ms_total"]}
+    for k in ("ffn", "attn", "qkv_proj", "o_proj"):
+        if k in m:
+            s[k] = m[k]
+    return s
+
+
+def run_spark(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2506_06644_b200 import binding as S
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    shape = shape_of(args.shape)
+    n_layers = args.layers or shape.n_layers
+    B, ctx_len = args.batch, args.ctx
+    W = max(args.warmup, 3)
+    m = measure_stack(torch, S, dist, dev, rank, world, args.shape, B, ctx_len, n_layers, args.steps, W, args.overlap,
+                      args.no_graph, args.no_dense, with_e2e=True, with_kernels=True)
     peak, peak_kind = measured_peak()
-    achieved = touched / (ffn_us * 1e-6) / 1e9
-    traffic = NCU_TRAFFIC_BYTES.get((args.shape, B))
-
     line = None
     if rank == 0:
-        ms_step = ms_total / args.steps
-        us_tl = us_per_token_per_layer(ms_total, args.steps, n_layers, B, world)
-        layer_touched = touched_layer_bytes(shape, B, ctx_len, union, n_layers)
+        s = stack_summary(m, world, peak)
+        per = 1e3 / (n_layers * B * world)
+        ffn = m["ffn"]
         line = {
-            "metric": "us_per_token_per_layer", "value": us_tl, "unit": "us/token/layer", "n_gpus": world,
-            "steps": args.steps, "warmup": W, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "metric": "us_per_token_per_layer", "value": us_per_token_per_layer(m["ms_total"], args.steps, n_layers, B, world),
+            "unit": "us/token/layer", "n_gpus": world, "steps": args.steps, "warmup": W, "ms_per_step": m["ms_total"] / args.steps,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(args, shape), "l2": "weights+caches (>3 GB) exceed L2; no flush needed",
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                        "launch": ("host launches" if args.no_graph else "one CUDA graph replay per decode step") +
-                                 (", programmatic dependent launches (spark_set_launch_overlap)" if overlap_on else ""),
+                                 (", programmatic dependent launches (spark_set_launch_overlap)" if m["overlap_on"] else ""),
                        "local_window": 4096, "k_ff": shape.k_ff, "k_attn": shape.k_attn},
-            "tokens_per_s": B * world * args.steps / (ms_total * 1e-3),
-            "layer_touched_mb": layer_touched / 1e6,
-            "layer_gbs_touched": layer_touched / (ms_step * 1e-3 / n_layers) / 1e9,
-            "layer_frac_of_8tbs": layer_touched / (ms_step * 1e-3 / n_layers) / 8e12,
-            "dense": None if ms_dense is None else {
-                "us_per_token_per_layer": ms_dense / args.steps * 1e3 / (n_layers * B * world),
-                "speedup_spark_vs_dense": ms_dense / ms_total},
-            "e2e": {"value": ms_e2e / args.steps * 1e3 / (n_layers * B * world), "unit": "us/token/layer",
-                    "h2d_bytes_per_step": int(h_host_in.numel() * 4), "d2h_bytes_per_step": int(h_host_out.numel() * 4)},
-            "gpu_launches": args.steps * n_layers * kernels_per_layer,
-            "clocks": clocks,
-            "roofline": {"kernel": ("ffn1_kernel" if B == 1 else "ffn_few_kernel" if B <= 4 else "ffn_tc_{prep,scores,act,out}_kernel") + " (spark_ffn_decode)", "bound": "hbm", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                         "us_per_launch": ffn_us, "touched_bytes_per_launch": touched, "union_rows": union},
-            "roofline_attention": {"kernel": "attn_kernel (spark_attn_decode)", "bound": "hbm",
-                                   "achieved": attn_bytes / (attn_us * 1e-6) / 1e9, "peak": peak, "unit": "GB/s",
-                                   "frac": attn_bytes / (attn_us * 1e-6) / 1e9 / peak, "us_per_launch": attn_us,
-                                   "touched_bytes_per_launch": attn_bytes, "traffic": None},
+            "median_us_per_token_per_layer": s["median_us_per_token_per_layer"],
+            "min_us_per_token_per_layer": s["min_us_per_token_per_layer"],
+            "tokens_per_s": B * world * args.steps / (m["ms_total"] * 1e-3),
+            "layer_touched_mb": s["layer_touched_mb"], "layer_gbs_touched": s["layer_gbs_touched"],
+            "layer_frac_of_measured_peak": s["layer_frac_of_measured_peak"], "layer_frac_of_8tbs": s["layer_frac_of_8tbs"],
+            "dense": None if m["ms_dense"] is None else {
+                "us_per_token_per_layer": m["ms_dense"] / args.steps * per,
+                "median_us_per_token_per_layer": m["steps_ms_dense"]["median"] * per,
+                "speedup_spark_vs_dense": m["ms_dense"] / m["ms_total"]},
+            "e2e": {"value": m["ms_e2e"] / args.steps * per, "unit": "us/token/layer",
+                    "h2d_bytes_per_step": m["h2d_bytes_per_step"], "d2h_bytes_per_step": m["d2h_bytes_per_step"]},
+            "gpu_launches": args.steps * n_layers * m["kernels_per_layer"],
+            "clocks": m["clocks"],
+            "roofline": {"kernel": ffn["kernel"], "bound": "hbm", "achieved": ffn["achieved"], "peak": peak, "unit": "GB/s",
+                         "frac": ffn["frac"], "traffic": NCU_TRAFFIC_BYTES.get((args.shape, B)), "peak_kind": f"of {peak_kind}",
+                         "us_per_launch": ffn["us_per_launch"], "median_us": ffn["median_us"], "min_us": ffn["min_us"],
+                         "touched_bytes_per_launch": ffn["touched_bytes_per_launch"], "union_rows": m["union_rows"]},
+            "roofline_attention": dict(m["attn"], traffic=None),
+            "kernels": {k: m[k] for k in ("qkv_proj", "attn", "o_proj", "ffn")},
         }
         if not args.no_extra and world == 1 and args.shape == "2b" and B == 1:
-            del layers, graphs, ffn_graph, attn_graph
-            torch.cuda.empty_cache()
-            line["other_workloads"] = other_workloads(torch, S, peak, max(args.steps // 4, 4), W)
+            # the other halves of the target, in the same run: the 9B-shape stack at batch 1 and the 2B-shape stack at
+            # batch 8 (eight sequences with their own 8192-token caches), each with its dense-loads comparator
+            ex_steps = max(min(args.steps, 24), 4)
+            line["stacks"] = []
+            for shp, bb in (("9b", 1), ("2b", 8)):
+                mm = measure_stack(torch, S, dist, dev, rank, world, shp, bb, ctx_len, shape_of(shp).n_layers, ex_steps, W,
+                                   args.overlap, args.no_graph, False, with_e2e=False, with_kernels=True)
+                line["stacks"].append(stack_summary(mm, world, peak))
+            line["other_workloads"] = other_workloads(torch, S, peak, max(args.steps // 4, 4), W, with_oracle=not args.no_cpu)
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = cpu_baseline(args, shape)
     if world > 1:
@@ -457,7 +523,7 @@ def run_spark(args):
         print(json.dumps(line), flush=True)
 
 
-def other_workloads(torch, S, peak, steps, warmup):
+def other_workloads(torch, S, peak, steps, warmup, with_oracle=True):
     """The other configurations of the method, each timed alone with CUDA events around a CUDA graph of
     back-to-back launches that cycle over more data than L2 holds.  GB/s are touched bytes."""
     from paper_2506_06644_b200 import synth
@@ -578,7 +644,7 @@ def other_workloads(torch, S, peak, steps, warmup):
     del sets
 
     # -- Spark attention, long contexts
-    for B, L, nsets in ((1, 16384, 6), (8, 32768, 2)):
+    for B, L, nsets in ((1, 4096, 24), (1, 16384, 6), (1, 32768, 4), (8, 32768, 2)):
         ctx = S.SparkContext(dev.index, max_batch=B, max_cap=L, n_q=sh.n_q, hd=sh.hd)
         ctx.set_launch_overlap(True)
         caches = [tuple(torch.randn(B, sh.n_kv, L, wd, device=dev, generator=gen).to(torch.bfloat16)
@@ -597,6 +663,10 @@ def other_workloads(torch, S, peak, steps, warmup):
         assert ctx.device_status() == S.SPARK_OK
         nbytes = B * (sh.n_kv * L * sh.r_attn * 2 + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn) * 2)
         entry(f"spark_attn_decode 8q/4kv heads hd 256, context {L}, batch {B}, k_attn {sh.k_attn}", res[0], nbytes, res[1])
+        if (B, L) not in ((1, 16384), (8, 32768)):
+            ctx.close()
+            del caches
+            continue
         # the same with the predictor slice of the cache in FP8 E4M3 (one scale per cached row)
         q8c = []
         for k1c, k2c, vc in caches:
@@ -701,24 +771,68 @@ def other_workloads(torch, S, peak, steps, warmup):
     ctx.close()
     del stacks, chunk_layers
 
-    # -- statistical top-k, 4096 rows x 65536 (1.07 GB read per launch)
+    # -- the LM head as a plain GEMV over the tied embedding (256000 x d, bf16: 1.18 GB at the 2B shape, 1.84 GB at 9B), one token
+    for name, dm in (("2b", synth.GEMMA2_2B.d), ("9b", synth.GEMMA2_9B.d)):
+        vocab = synth.GEMMA2_2B.vocab
+        ctx = S.SparkContext(dev.index, max_batch=1, max_d=dm)
+        ctx.set_launch_overlap(True)
+        E = torch.randn(vocab, dm, device=dev, generator=gen).to(torch.bfloat16)
+        xh = torch.randn(1, dm, device=dev, generator=gen)
+        logits = torch.empty(1, vocab, device=dev)
+        us = time_graph(lambda: [S.spark_dense_gemv(ctx, xh, 1, E, S.SPARK_BF16, dm, vocab, None, logits) for _ in range(2)], 2)
+        assert ctx.device_status() == S.SPARK_OK
+        entry(f"LM head: spark_dense_gemv {vocab} x {dm} bf16 (gemma2-{name} shape), one token", us, vocab * dm * 2)
+        ctx.close()
+        del E
+
+    # -- statistical top-k, 4096 rows x 65536 (1.07 GB read per launch): three distributions x k/n in {2, 8, 25} %
     ctx = S.SparkContext(dev.index)
     rows, n = 4096, 65536
-    xs = torch.randn(rows, n, device=dev, generator=gen)
     theta = torch.empty(rows, device=dev)
     count = torch.empty(rows, dtype=torch.int32, device=dev)
-    yd = torch.empty(rows, n, device=dev)
-    for kk in (1311, 5243):
-        us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, kk, S.SPARK_FILL_ZERO, theta, count, None, None, 0, None), 1)
-        entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = {kk / n:.0%}, theta + count", us, rows * n * 4)
-    us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, 5243, S.SPARK_FILL_ZERO, theta, count, None, None, 0, yd), 1)
-    entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = 8%, dense output (Eq. 10)", us, 2 * rows * n * 4)
-    cap = 4 * 1311
-    idx = torch.empty(rows, cap, dtype=torch.int32, device=dev)
-    val = torch.empty(rows, cap, device=dev)
-    us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, 1311, S.SPARK_FILL_ZERO, theta, count, idx, val, cap, None), 1)
-    entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = 2%, ordered index and value lists", us,
-          rows * n * 4 + int(count.sum().item()) * 8)
+
+    def draw(dist):
+        if dist == "N(0,1)":
+            return torch.randn(rows, n, device=dev, generator=gen)
+        if dist == "Laplace(0,1)":
+            u = torch.rand(rows, n, device=dev, generator=gen)
+            return torch.where(u < 0.5, torch.log(2 * u), -torch.log(2 * (1 - u))).clamp_(-80, 80)
+        z = torch.randn(rows, n, device=dev, generator=gen)                  # Student-t(4) = Z / sqrt(chi2_4 / 4)
+        chi = torch.zeros(rows, n, device=dev)
+        for _ in range(4):
+            chi += torch.randn(rows, n, device=dev, generator=gen) ** 2
+        return z / torch.sqrt(chi / 4)
+
+    for dist in ("N(0,1)", "Laplace(0,1)", "Student-t(4)"):
+        xs = draw(dist)
+        for kk in (1311, 5243, 16384):
+            us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, kk, S.SPARK_FILL_ZERO, theta, count, None, None, 0, None), 1)
+            entry(f"spark_stat_topk {rows} x {n} fp32 {dist}, k/n = {kk / n:.0%}, theta + count", us, rows * n * 4)
+            c = count.float()
+            out[-1].update({"k": kk, "selected_mean": float(c.mean()), "selected_std": float(c.std()),
+                            "selected_min": int(count.min()), "selected_max": int(count.max())})
+            if with_oracle:          # theta of eight sampled rows against the oracle (relative to max(|theta|, std) of the row)
+                from oracle import spark_oracle as O
+                worst = 0.0
+                for rr in range(0, rows, rows // 8):
+                    xr = xs[rr].cpu().numpy()
+                    th, mask, _ = O.stat_topk(xr, kk)
+                    worst = max(worst, abs(float(theta[rr]) - th) / max(abs(th), float(np.std(xr.astype(np.float64), ddof=1))))
+                    assert abs(int(count[rr]) - int(mask.sum())) <= 2
+                out[-1]["theta_max_rel_err_vs_oracle_8_rows"] = worst
+        if dist == "N(0,1)":
+            yd = torch.empty(rows, n, device=dev)
+            us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, 5243, S.SPARK_FILL_ZERO, theta, count, None, None, 0, yd), 1)
+            entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = 8%, dense output (Eq. 10)", us, 2 * rows * n * 4)
+            del yd
+            cap = 4 * 1311
+            idx = torch.empty(rows, cap, dtype=torch.int32, device=dev)
+            val = torch.empty(rows, cap, device=dev)
+            us = time_graph(lambda: S.spark_stat_topk(ctx, xs, rows, n, n, 1311, S.SPARK_FILL_ZERO, theta, count, idx, val, cap, None), 1)
+            entry(f"spark_stat_topk {rows} x {n} fp32 N(0,1), k/n = 2%, ordered index and value lists", us,
+                  rows * n * 4 + int(count.sum().item()) * 8)
+            del idx, val
+        del xs
     assert ctx.device_status() == S.SPARK_OK
     ctx.close()
     return out
@@ -738,18 +852,32 @@ def touched_layer_bytes(shape, B, ctx_len, union_ffn, n_layers):
 
 
 def cpu_baseline(args, shape):
+    """The oracle as it stands on the host cores: all the threads its numpy build uses, and pinned to one thread."""
     n_l = 2
     layers, h = oracle_sample(shape, args.ctx, n_l)
     oracle_run(shape, layers[:1], h, args.ctx)            # touch the pages once
-    reps, t0 = 0, time.perf_counter()
-    while True:
-        oracle_run(shape, layers, h, args.ctx)
-        reps += 1
-        if time.perf_counter() - t0 > 10.0 or reps >= 40:
-            break
-    dt = time.perf_counter() - t0
-    return {"value": dt / (reps * n_l) * 1e6, "unit": "us/token/layer", "cores": host_threads(), "kind": "oracle",
-            "sample": f"{reps} x {n_l} decoder layers of one token at context {args.ctx} (fp64 numpy)"}
+
+    def timed_reps(budget_s, max_reps):
+        reps, t0 = 0, time.perf_counter()
+        while True:
+            oracle_run(shape, layers, h, args.ctx)
+            reps += 1
+            if time.perf_counter() - t0 > budget_s or reps >= max_reps:
+                break
+        return (time.perf_counter() - t0) / (reps * n_l) * 1e6, reps
+
+    us_all, reps = timed_reps(10.0, 40)
+    out = {"value": us_all, "unit": "us/token/layer", "cores": host_threads(), "kind": "oracle",
+           "sample": f"{reps} x {n_l} decoder layers of one token at context {args.ctx} (fp64 numpy)"}
+    try:
+        from threadpoolctl import threadpool_limits
+        with threadpool_limits(limits=1):
+            us_one, reps1 = timed_reps(6.0, 10)
+        out["single_thread"] = {"value": us_one, "unit": "us/token/layer", "cores": 1,
+                                "sample": f"{reps1} x {n_l} decoder layers, numpy limited to one thread"}
+    except Exception:
+        pass
+    return out
 
 
 def main():

@@ -55,7 +55,9 @@ enum {
     SPARK_ERR_WORKSPACE = 3,   /* the context's workspace is too small for this call                */
     SPARK_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                            */
     SPARK_ERR_TIMEOUT = 5,     /* device: a bounded wait between thread blocks ran out              */
-    SPARK_ERR_OVERFLOW = 6     /* device: an index list did not fit its capacity (truncated)        */
+    SPARK_ERR_OVERFLOW = 6,    /* device: an index list did not fit its capacity (truncated)        */
+    SPARK_ERR_NONFINITE = 7    /* device: the score statistics of a call made with SPARK_CHECK_FINITE
+                                  were not finite (a NaN or infinity in its inputs or weights)     */
 };
 
 /* ---- dtypes and flags ----------------------------------------------------- */
@@ -71,11 +73,17 @@ enum {
     SPARK_GELU_ERF = 1,      /* exact form x * Phi(x)                                          */
     SPARK_DENSE_LOADS = 2,   /* comparator: same result, but every row of K2/V (or of the cache)
                                 is read and multiplied by its (possibly zero) activation       */
-    SPARK_SHARED_CACHE = 4   /* attention and layer: the B tokens are consecutive tokens of ONE
+    SPARK_SHARED_CACHE = 4,  /* attention and layer: the B tokens are consecutive tokens of ONE
                                 sequence (a chunk of its prompt) and share one cache
                                 [n_kv][cap][.]; token b is the sequence's token number ctx_len[b]
                                 (1-based) and sees rows [0, ctx_len[b]), so with ctx_len[b] =
                                 L0 + b + 1 the chunk is causal; caches lose their [B] dimension  */
+    SPARK_CHECK_FINITE = 8   /* debugging aid: a threshold whose score sums are not finite (a NaN or an
+                                infinity reached the predictor) records SPARK_ERR_NONFINITE in the
+                                device status.  Honoured by the one-token FFN kernel and by the
+                                per-query attention kernel, also inside spark_layer_decode; the
+                                other kernels ignore it.  The paper leaves non-finite inputs
+                                undefined; outputs are then undefined here too                     */
 };
 
 typedef struct spark_ctx spark_ctx;
@@ -89,14 +97,16 @@ size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap
                              int64_t hd, int64_t max_d);
 
 /* Create a context on `device` around a caller-owned device workspace (256-byte aligned).
- * Zeroes the workspace (a synchronous memset: its idle state is all zero); queries the SM count.
+ * Zeroes the workspace (its idle state is all zero) and waits for the device, so that the first
+ * call may go to any stream; queries the SM count.
  * *out is a host object released by spark_destroy (which leaves the workspace alone). */
 int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_bytes);
 int spark_destroy(spark_ctx* ctx);
 
 /* Synchronise `stream`, copy the device status word to *host_out (host pointer), clear it, and
- * if it was not SPARK_OK also reset the workspace to its idle (zero) state.  Returns SPARK_OK when the
- * read itself worked (the device status is in *host_out). */
+ * if it was not SPARK_OK also reset the workspace to its idle (zero) state (synchronously: the
+ * context is usable again when the call returns).  Returns SPARK_OK when the read itself worked
+ * (the device status is in *host_out). */
 int spark_device_status(spark_ctx* ctx, void* stream, int* host_out);
 
 /* Static string for a status code (host pointer, never freed). */
@@ -122,6 +132,21 @@ int spark_set_phase_trace(spark_ctx* ctx, uint64_t* trace, int64_t capacity);
  * guarantees and this mode only obtains from an otherwise idle GPU; a block that waits in vain
  * gives up after its limit and the device status becomes SPARK_ERR_TIMEOUT.  Host-only setting. */
 int spark_set_launch_overlap(spark_ctx* ctx, int on);
+
+/* Bound of the waits between thread blocks (failure detection; the paper has no counterpart).  The
+ * kernels that exchange score sums between blocks (FFN, attention, the fused one-token layer) poll
+ * until every block has arrived; a block that has waited `cycles` SM cycles gives up, records
+ * SPARK_ERR_TIMEOUT in the device status and returns, the kernel ends by itself and the outputs of
+ * that call are incomplete.  spark_device_status then reports the code and resets the workspace,
+ * after which the context is usable again.  cycles == 0 restores the default (about two seconds).
+ * Synchronises `stream` and the device: call it between steps, not during a stream capture.  The
+ * tensor-core chunk kernels and the top-k row kernel keep their own fixed bounds. */
+int spark_set_wait_limit(spark_ctx* ctx, void* stream, int64_t cycles);
+
+/* Test hook for that path (host-only setting; 0 = off, the default): the one-token FFN kernel waits
+ * for `extra` more arrivals than its grid has blocks, so its wait runs out exactly as it would if a
+ * block never became resident.  Nothing faults: the kernel returns after the wait limit. */
+int spark_debug_expect_arrivals(spark_ctx* ctx, int extra);
 
 /* Gaussian upper quantile used for the threshold: z with P(N(0,1) > z) = p, i.e. Q(1 - p) of
  * Eq. 11.  Host function (no device work); exported so that it can be checked on its own.
@@ -157,7 +182,8 @@ int spark_stat_topk(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int
  *   mean + std * Q(1 - k / n_total) of the merged moments, Bessel-corrected (Eq. 11), -inf for
  *   k >= n_total; merged [rows][3] nullable.  The parts' counts must add up to n_total.
  * spark_stat_select: like spark_stat_topk with the thresholds given (theta_in [rows], device): count,
- *   idx (indices within the part), val, y_dense as there; survivors are shifted by theta_in. */
+ *   idx (indices within the part), val, y_dense as there; survivors are shifted by theta_in, except that
+ *   theta_in = -inf (what spark_stat_merge gives for k >= n_total) keeps every entry unshifted. */
 int spark_stat_moments(spark_ctx* ctx, const float* x, int64_t rows, int64_t n, int64_t ld, double* moments,
                        void* stream);
 int spark_stat_merge(spark_ctx* ctx, const double* parts, int64_t m, int64_t rows, int64_t k, int64_t n_total,
@@ -201,27 +227,33 @@ int spark_ffn_decode_fp8(spark_ctx* ctx, const float* x, int64_t B, const void* 
  * handed out in full up front (an inference server's arena, a plugin inside another runtime), or
  * that must not touch the allocator because a stream capture or a latency-critical section is
  * under way elsewhere in the process.  They cannot give spark_create a workspace.  This entry point
- * computes exactly what spark_ffn_decode computes, with the small amount of inter-block state the
- * kernel needs (a status word, a launch counter, the cells the blocks add their score sums into)
- * kept in a fixed array inside the library's device image: about 140 KB on every GPU that loads
- * the library, held until the process exits.  Inputs and outputs are still the caller's.
+ * computes what spark_ffn_decode computes, within the library's stated tolerances (for 5 to 16
+ * tokens it takes the union-gather kernels, where spark_ffn_decode with a workspace may take the
+ * tensor-core chunk kernels), with the small amount of inter-block state the kernels need (a status
+ * word, a launch counter, the cells the blocks add their score sums into) kept in a fixed array
+ * inside the library's device image: about 140 KB on every GPU that loads the library, held until
+ * the process exits.  Inputs and outputs are still the caller's.
  *   - Limit: B <= SPARK_NOALLOC_MAX_TOKENS; a larger B returns SPARK_ERR_UNSUPPORTED.  All other
  *     limits and argument checks are those of spark_ffn_decode.  count / idx are not offered.
  *   - The device is the current one.  The first call on a device looks up the array's device
- *     address and clears it (a synchronous 140 KB memset); make that first call before any stream
- *     capture begins.  No call allocates or frees device memory.
+ *     address (the array is zero, its idle state, from the moment the library is loaded; nothing
+ *     is cleared and nothing is enqueued besides the kernel, so the first call may go to any
+ *     stream); make that first call before any stream capture begins.  No call allocates or frees
+ *     device memory.
  *   - All calls on a device share the array, and it keeps what the last call left (the kernels
  *     themselves clear the cells a later call will use).  Two calls whose kernels overlap on the
  *     GPU -- different streams, or one process-wide array used from two threads -- race on it:
  *     issue them on one stream, or otherwise order them.  spark_ffn_decode with its own context
  *     has no such restriction across contexts.
- *   - A device-side timeout (SPARK_ERR_TIMEOUT) cannot be read back through this entry point; y is
- *     then incomplete.  It only arises when the launch's blocks cannot all be resident at once,
- *     which the cooperative launch already refuses with SPARK_ERR_CUDA. */
+ *   - spark_noalloc_status plays the part of spark_device_status: it synchronises `stream`, copies
+ *     the array's status word to *host_out (host pointer) and, if that is not SPARK_OK (a bounded
+ *     wait ran out: y of that call is incomplete), puts the array back into its idle state so that
+ *     later calls work again.  It allocates nothing either. */
 #define SPARK_NOALLOC_MAX_TOKENS 16
 int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K1t, const void* K2t, const void* Vt,
                              int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k, int flags,
                              float* y, float* theta, void* stream);
+int spark_noalloc_status(void* stream, int* host_out);
 
 /* ---- Spark attention (Section 2.2, Eq. 7) ------------------------------------
  * For sequence b and query head h (KV head g = h / (n_q / n_kv)), over the tokens t of the window

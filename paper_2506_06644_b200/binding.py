@@ -19,16 +19,17 @@ LIB_PATH = os.path.join(_HERE, "libspark_b200.so")
 
 SPARK_OK = 0
 SPARK_ERR_INVALID_ARG, SPARK_ERR_UNSUPPORTED, SPARK_ERR_WORKSPACE, SPARK_ERR_CUDA = 1, 2, 3, 4
-SPARK_ERR_TIMEOUT, SPARK_ERR_OVERFLOW = 5, 6
+SPARK_ERR_TIMEOUT, SPARK_ERR_OVERFLOW, SPARK_ERR_NONFINITE = 5, 6, 7
 SPARK_F32, SPARK_BF16, SPARK_FP8_E4M3 = 0, 1, 2
 SPARK_FILL_ZERO, SPARK_FILL_NEGINF = 0, 1
-SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS, SPARK_SHARED_CACHE = 0, 1, 2, 4
+SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS, SPARK_SHARED_CACHE, SPARK_CHECK_FINITE = 0, 1, 2, 4, 8
 
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
     "spark_destroy", "spark_device_status", "spark_grid_size", "spark_set_phase_trace", "spark_set_launch_overlap", "spark_stat_topk", "spark_ffn_decode",
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
     "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
+    "spark_set_wait_limit", "spark_debug_expect_arrivals", "spark_noalloc_status",
 ]
 
 
@@ -75,6 +76,9 @@ def lib() -> C.CDLL:
         "spark_grid_size": (i32, [vp]),
         "spark_set_phase_trace": (i32, [vp, vp, i64]),
         "spark_set_launch_overlap": (i32, [vp, i32]),
+        "spark_set_wait_limit": (i32, [vp, vp, i64]),
+        "spark_debug_expect_arrivals": (i32, [vp, i32]),
+        "spark_noalloc_status": (i32, [vp, C.POINTER(i32)]),
         "spark_stat_topk": (i32, [vp, vp, i64, i64, i64, i64, i32, vp, vp, vp, vp, i64, vp, vp]),
         "spark_stat_moments": (i32, [vp, vp, i64, i64, i64, vp, vp]),
         "spark_stat_merge": (i32, [vp, vp, i64, i64, i64, i64, vp, vp, vp]),
@@ -168,6 +172,14 @@ class SparkContext:
         """Launch every kernel of this context so that it may start under the tail of the kernel before it."""
         _check(lib().spark_set_launch_overlap(self.handle, 1 if on else 0), "spark_set_launch_overlap")
 
+    def set_wait_limit(self, cycles: int):
+        """Bound of the waits between thread blocks in SM cycles (0 = the default of about two seconds)."""
+        _check(lib().spark_set_wait_limit(self.handle, _stream(), cycles), "spark_set_wait_limit")
+
+    def debug_expect_arrivals(self, extra: int):
+        """Test hook: the one-token FFN kernel waits for `extra` arrivals that never come (0 = off)."""
+        _check(lib().spark_debug_expect_arrivals(self.handle, extra), "spark_debug_expect_arrivals")
+
     @property
     def grid_size(self) -> int:
         return lib().spark_grid_size(self.handle)
@@ -218,6 +230,13 @@ def spark_ffn_decode_noalloc(x, B, K1t, K2t, Vt, wdtype, d, d_ff, r, k, flags, y
     inter-block state lives in a fixed array inside the library (see include/spark.h).  B <= 16."""
     _check(lib().spark_ffn_decode_noalloc(_ptr(x), B, _ptr(K1t), _ptr(K2t), _ptr(Vt), wdtype, d, d_ff, r, k, flags,
                                           _ptr(y), _ptr(theta), _stream()), "spark_ffn_decode_noalloc")
+
+
+def spark_noalloc_status() -> int:
+    """Device status of the no-allocation entry point on the current device (resets its state after an error)."""
+    out = C.c_int(0)
+    _check(lib().spark_noalloc_status(_stream(), C.byref(out)), "spark_noalloc_status")
+    return out.value
 
 
 def spark_attn_decode(ctx: SparkContext, q, k1c, k2c, vc, kvdtype, B, n_q, n_kv, hd, r, cap, ctx_len, window,

@@ -76,6 +76,7 @@ struct AttnParams {
     SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
     float* lsum;       // [B][n_q] sum of softmax weights per head (o accumulates the weighted values)
     int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
+    int check_finite;  // SPARK_CHECK_FINITE: non-finite score sums are reported in the device status
     int pre_stable;    // 1: the kernel directly before this one writes neither ctx_len nor cache rows other than each
                        //    sequence's newest, so lengths and older rows may be read before dep_wait()
     WsHeader* hdr;
@@ -542,6 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                                                             static_cast<unsigned>(npieces), sa, sq, smax, p.hdr);
                 if (lane == 0) {
                     if (!ok) s_fail = 1;
+                    if (ok && p.check_finite && !(isfinite(sa) && isfinite(sq))) atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_NONFINITE);
                     float th = -INFINITY;
                     if (!ident) {
                         const double z = ord < kZc ? zcache[ord] : s_z;
@@ -858,6 +860,7 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.window = static_cast<int>(window > 0x7fffffff ? 0x7fffffff : window);
     p.k_attn = static_cast<int>(k_attn > 0x7fffffff ? 0x7fffffff : k_attn);
     p.dense = (flags & SPARK_DENSE_LOADS) ? 1 : 0;
+    p.check_finite = (flags & SPARK_CHECK_FINITE) ? 1 : 0;
     const bool shared = (flags & SPARK_SHARED_CACHE) != 0;
     if (shared && (n_kv & (n_kv - 1)) != 0) return SPARK_ERR_UNSUPPORTED;
     p.seg_mask = shared ? static_cast<int>(n_kv - 1) : -1;

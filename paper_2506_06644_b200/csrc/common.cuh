@@ -37,7 +37,8 @@ constexpr size_t kAttnCellBytes = static_cast<size_t>(16384) * kAttnWays * 32;  
 
 struct WsHeader {            // lives at the start of the caller's workspace; zero when idle
     int status;              // device status word (SPARK_OK or a SPARK_ERR_* device code)
-    unsigned reserved[2];
+    unsigned wait_kcycles;   // bound of the inter-block waits in units of 1024 SM cycles; 0 = kSpinLimitCycles (spark_set_wait_limit)
+    unsigned reserved;
     unsigned epoch;          // launches of the FFN kernels so far (selects their accumulator ring slot)
     unsigned pad[60];
     unsigned seg_done[kMaxSegments];   // attention: finished pieces per segment (self-resetting)
@@ -59,6 +60,8 @@ struct spark_ctx {
     unsigned long long* trace;   // optional phase trace (device), see spark_set_phase_trace
     long long trace_cap;
     int overlap;             // launch with programmatic stream serialization, see spark_set_launch_overlap
+    unsigned wait_kcycles;   // host copy of the header's wait bound (restored after a workspace reset)
+    int debug_extra_arrivals;   // test hook: the one-token kernels wait for this many arrivals more than blocks exist
 };
 
 namespace spark {
@@ -310,8 +313,12 @@ struct PhaseTrace {
     }
 };
 
-// Bound of every spin-wait, in SM cycles (about two seconds at 2 GHz).
+// Bound of every spin-wait, in SM cycles (about two seconds at 2 GHz), unless the workspace header carries another.
 constexpr long long kSpinLimitCycles = 4000000000ll;
+__device__ __forceinline__ long long spin_limit(const WsHeader* hdr) {
+    const unsigned k = __ldg(&hdr->wait_kcycles);      // constant while kernels run: written by the host only
+    return k != 0u ? static_cast<long long>(k) << 10 : kSpinLimitCycles;
+}
 
 // Sum-cell helpers.
 __device__ __forceinline__ void red_add_f64(double* p, double v) {
@@ -363,7 +370,7 @@ template <int WAYS>
 __device__ __forceinline__ bool cells_wait_w(const SumCell* ways, unsigned nblocks, double& s1, double& s2, WsHeader* hdr) {
     static_assert(WAYS == 1 || WAYS == 2 || WAYS == 4 || WAYS == 8 || WAYS == 16, "ways");
     const int lane = threadIdx.x & 31;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = spin_limit(hdr);
     for (;;) {
         double a = 0.0, b = 0.0;
         unsigned cnt = 0u;
@@ -382,7 +389,7 @@ __device__ __forceinline__ bool cells_wait_w(const SumCell* ways, unsigned nbloc
             s2 = __shfl_sync(kFull, b, 0);
             return true;
         }
-        if (clock64() - t0 > kSpinLimitCycles) {
+        if (clock64() - t0 > limit) {
             if (lane == 0) atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
             return false;
         }
@@ -435,7 +442,7 @@ template <int WAYS>
 __device__ __forceinline__ bool cells_wait_max_w(const SumCell* ways, unsigned nblocks, double& s1, double& s2, float& mx,
                                                  WsHeader* hdr) {
     const int lane = threadIdx.x & 31;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = spin_limit(hdr);
     for (;;) {
         double a = 0.0, b = 0.0;
         unsigned cnt = 0u, ex = 0u;
@@ -457,7 +464,7 @@ __device__ __forceinline__ bool cells_wait_max_w(const SumCell* ways, unsigned n
             mx = ordered_to_f32(__shfl_sync(kFull, ex, 0));
             return true;
         }
-        if (clock64() - t0 > kSpinLimitCycles) {
+        if (clock64() - t0 > limit) {
             if (lane == 0) atomicCAS(&hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
             return false;
         }

@@ -11,6 +11,9 @@
 //            u_i = GELU(s_i - theta) t_i, then a thread per 8 output columns accumulates
 //            sum_i u_i V[:,i] in registers and adds it to y with vector reductions.
 // Individual masks gate the arithmetic, the union gates the loads (Appendix B).
+#include <atomic>
+#include <mutex>
+
 #include "ffn_params.h"
 #include "kernels.h"
 #include "rowdot.cuh"
@@ -431,6 +434,8 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     p.inv_nm1 = 1.0 / static_cast<double>(a.d_ff - 1);
     p.hdr = ctx->hdr;
     p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
+    p.extra_arrivals = ctx->debug_extra_arrivals;
+    p.check_finite = (a.flags & SPARK_CHECK_FINITE) ? 1 : 0;
     const size_t smem = (static_cast<size_t>(tb) * p.xw + static_cast<size_t>(2) * tb * p.rpc) * sizeof(float) +
                         static_cast<size_t>(p.rpc) * 8;
     if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_UNSUPPORTED;
@@ -488,16 +493,40 @@ namespace {
 
 // The inter-block state the FFN kernels need (status word, launch epoch, score-sum cells) lives in
 // this file-scope array instead of a caller-provided workspace.  It is zero when the module is
-// loaded, which is the idle state; every device that loads the library carries its own copy
-// (about 140 KB) until the process exits.
+// loaded, which is the idle state (so the first call has nothing to clear); every device that loads
+// the library carries its own copy (about 140 KB) until the process exits.
 static __device__ __align__(256) unsigned char g_noalloc_state[sizeof(WsHeader)];
 
 struct NoallocDevice {
-    bool ready;
-    WsHeader* state;      // device address of g_noalloc_state on this device
-    int num_sms, max_smem_optin;
+    std::atomic<bool> ready{false};
+    WsHeader* state = nullptr;      // device address of g_noalloc_state on this device
+    int num_sms = 0, max_smem_optin = 0;
 };
-NoallocDevice g_noalloc[64] = {};
+NoallocDevice g_noalloc[64];
+std::mutex g_noalloc_mutex;         // first calls from several host threads: one of them does the set-up
+
+// Once per device, with that device current: in host code the array's name is only a stand-in for
+// the symbol, so its device address has to be asked for.  Allocates nothing.
+int noalloc_device(NoallocDevice** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SPARK_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return SPARK_ERR_UNSUPPORTED;
+    NoallocDevice& nd = g_noalloc[dev];
+    if (!nd.ready.load(std::memory_order_acquire)) {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!nd.ready.load(std::memory_order_relaxed)) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_noalloc_state) != cudaSuccess || ptr == nullptr) return SPARK_ERR_CUDA;
+            if (cudaDeviceGetAttribute(&nd.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPARK_ERR_CUDA;
+            if (cudaDeviceGetAttribute(&nd.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+                return SPARK_ERR_CUDA;
+            nd.state = static_cast<WsHeader*>(ptr);
+            nd.ready.store(true, std::memory_order_release);
+        }
+    }
+    *out = &nd;
+    return SPARK_OK;
+}
 
 }  // namespace
 
@@ -505,34 +534,25 @@ extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K
                                         int wdtype, int64_t d, int64_t d_ff, int64_t r, int64_t k, int flags,
                                         float* y, float* theta, void* stream) {
     if (B > SPARK_NOALLOC_MAX_TOKENS) return SPARK_ERR_UNSUPPORTED;   // beyond what the static state serves
+    NoallocDevice* nd = nullptr;
+    const int rc = noalloc_device(&nd);
+    if (rc != SPARK_OK) return rc;
     int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess) return SPARK_ERR_CUDA;
-    if (dev < 0 || dev >= 64) return SPARK_ERR_UNSUPPORTED;
-    NoallocDevice& nd = g_noalloc[dev];
-    if (!nd.ready) {
-        // Once per device, with that device current: in host code the array's name is only a
-        // stand-in for the symbol, so its device address has to be asked for.
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_noalloc_state) != cudaSuccess || ptr == nullptr) return SPARK_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&nd.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SPARK_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&nd.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-            return SPARK_ERR_CUDA;
-        if (cudaMemset(ptr, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;   // idle state
-        nd.state = static_cast<WsHeader*>(ptr);
-        nd.ready = true;
-    }
+    cudaGetDevice(&dev);
     spark_ctx local;
     local.device = dev;
-    local.num_sms = nd.num_sms;
-    local.max_smem_optin = nd.max_smem_optin;
-    local.ws = reinterpret_cast<char*>(nd.state);
+    local.num_sms = nd->num_sms;
+    local.max_smem_optin = nd->max_smem_optin;
+    local.ws = reinterpret_cast<char*>(nd->state);
     local.ws_bytes = sizeof(WsHeader);
-    local.hdr = nd.state;
+    local.hdr = nd->state;
     local.scratch = nullptr;
     local.scratch_bytes = 0;
     local.trace = nullptr;
     local.trace_cap = 0;
     local.overlap = 0;
+    local.wait_kcycles = 0;
+    local.debug_extra_arrivals = 0;
     FfnArgs a;
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;
     a.K1t = K1t; a.K2t = K2t; a.Vt = Vt; a.wdtype = wdtype;
@@ -540,4 +560,22 @@ extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K
     a.B = B; a.d = d; a.d_ff = d_ff; a.r = r; a.k = k; a.flags = flags;
     a.y_init = nullptr; a.y = y; a.theta = theta; a.count = nullptr; a.idx = nullptr;
     return ffn_launch(&local, a, static_cast<cudaStream_t>(stream));
+}
+
+// The device status of the no-allocation entry point: what spark_device_status is for a context.
+extern "C" int spark_noalloc_status(void* stream, int* host_out) {
+    if (host_out == nullptr) return SPARK_ERR_INVALID_ARG;
+    NoallocDevice* nd = nullptr;
+    const int rc = noalloc_device(&nd);
+    if (rc != SPARK_OK) return rc;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SPARK_ERR_CUDA;
+    int status = 0;
+    if (cudaMemcpy(&status, &nd->state->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SPARK_ERR_CUDA;
+    *host_out = status;
+    if (status != SPARK_OK) {
+        // a wait that ran out left arrivals and partial sums behind: back to the idle (zero) state
+        if (cudaMemset(nd->state, 0, sizeof(WsHeader)) != cudaSuccess) return SPARK_ERR_CUDA;
+        if (cudaDeviceSynchronize() != cudaSuccess) return SPARK_ERR_CUDA;
+    }
+    return SPARK_OK;
 }

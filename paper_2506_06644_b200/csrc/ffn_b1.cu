@@ -162,10 +162,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
         if (lane == 0) cells_add(ways, cta, s1, s2);    // also orders y's initialisation before the arrival
         p.trace.mark(3);
         double sa, sb;
-        const bool ok = cells_wait(ways, static_cast<unsigned>(grid), sa, sb, p.hdr);
+        const bool ok = cells_wait(ways, static_cast<unsigned>(grid + p.extra_arrivals), sa, sb, p.hdr);
         if (lane == 0) {
             float th = -INFINITY;
             if (!ok) s_fail = 1;
+            if (ok && p.check_finite && !(isfinite(sa) && isfinite(sb))) atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_NONFINITE);
             if (!p.identity) {
                 const double mean = sa * p.inv_n;
                 const float var = static_cast<float>((sb - sa * mean) * p.inv_nm1);

@@ -23,6 +23,8 @@ struct FfnParams {
     int xres;                     // tensor-core kernel: both halves of the split input stay in shared memory
     int vrows, vstage_off;        // few-token kernel: rows of V per round and the byte offset of their staging area
     int overlap;                  // launched with the programmatic attribute: weights first, then dep_wait()
+    int extra_arrivals;           // test hook (one-token kernel): arrivals waited for beyond the grid's blocks
+    int check_finite;             // SPARK_CHECK_FINITE: non-finite score sums are reported in the device status
     double z;
     double inv_n, inv_nm1;        // 1 / d_ff and 1 / (d_ff - 1)
     const float* y_init;

@@ -620,7 +620,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
 
     // 3. Spark attention over the cache (the new token included)
     rc = attn_launch(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd, cfg->r_attn,
-                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & (SPARK_DENSE_LOADS | SPARK_SHARED_CACHE), ao, lsum, nullptr, nullptr,
+                     cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & (SPARK_DENSE_LOADS | SPARK_SHARED_CACHE | SPARK_CHECK_FINITE), ao, lsum, nullptr, nullptr,
                      nullptr, 0, nullptr, st);
     if (rc != SPARK_OK) return rc;
 

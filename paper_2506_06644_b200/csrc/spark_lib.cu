@@ -19,6 +19,7 @@ const char* spark_status_string(int status) {
         case SPARK_ERR_CUDA: return "CUDA runtime or launch failure";
         case SPARK_ERR_TIMEOUT: return "device: bounded inter-block wait ran out";
         case SPARK_ERR_OVERFLOW: return "device: index list truncated at its capacity";
+        case SPARK_ERR_NONFINITE: return "device: non-finite score statistics (SPARK_CHECK_FINITE)";
         default: return "unknown status";
     }
 }
@@ -85,7 +86,10 @@ int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SPARK_ERR_CUDA;
     // the whole workspace starts zeroed: header words, score-sum cells and per-segment counters are
     // idle at zero, and the kernels leave them so
+    // (the memset runs on the legacy default stream and may still be in flight when it returns; kernels the caller
+    // then launches on a non-blocking stream are not ordered behind it, hence the synchronisation)
     if (cudaMemset(workspace, 0, workspace_bytes) != cudaSuccess) return SPARK_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return SPARK_ERR_CUDA;
     spark_ctx* c = new (std::nothrow) spark_ctx;
     if (c == nullptr) return SPARK_ERR_INVALID_ARG;
     c->device = device;
@@ -99,6 +103,8 @@ int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_
     c->trace = nullptr;
     c->trace_cap = 0;
     c->overlap = 0;
+    c->wait_kcycles = 0;
+    c->debug_extra_arrivals = 0;
     *out = c;
     return SPARK_OK;
 }
@@ -123,6 +129,25 @@ int spark_set_launch_overlap(spark_ctx* ctx, int on) {
 
 int spark_grid_size(const spark_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
 
+int spark_set_wait_limit(spark_ctx* ctx, void* stream, int64_t cycles) {
+    if (ctx == nullptr || cycles < 0) return SPARK_ERR_INVALID_ARG;
+    if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
+    int64_t k = (cycles + 1023) >> 10;
+    if (k > 0xffffffffll) k = 0xffffffffll;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return SPARK_ERR_CUDA;      // no kernel of this context reads the word meanwhile
+    ctx->wait_kcycles = static_cast<unsigned>(k);
+    if (cudaMemcpy(&ctx->hdr->wait_kcycles, &ctx->wait_kcycles, sizeof(unsigned), cudaMemcpyHostToDevice) != cudaSuccess)
+        return SPARK_ERR_CUDA;
+    return cudaDeviceSynchronize() == cudaSuccess ? SPARK_OK : SPARK_ERR_CUDA;
+}
+
+int spark_debug_expect_arrivals(spark_ctx* ctx, int extra) {
+    if (ctx == nullptr || extra < 0) return SPARK_ERR_INVALID_ARG;
+    ctx->debug_extra_arrivals = extra;
+    return SPARK_OK;
+}
+
 int spark_device_status(spark_ctx* ctx, void* stream, int* host_out) {
     if (ctx == nullptr || host_out == nullptr) return SPARK_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -134,6 +159,10 @@ int spark_device_status(spark_ctx* ctx, void* stream, int* host_out) {
     if (status != SPARK_OK) {
         // a failed phase may have left arrivals or partial sums behind: back to the idle (zero) state
         if (cudaMemset(ctx->ws, 0, ctx->ws_bytes) != cudaSuccess) return SPARK_ERR_CUDA;
+        if (ctx->wait_kcycles != 0u &&
+            cudaMemcpy(&ctx->hdr->wait_kcycles, &ctx->wait_kcycles, sizeof(unsigned), cudaMemcpyHostToDevice) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        if (cudaDeviceSynchronize() != cudaSuccess) return SPARK_ERR_CUDA;      // the reset is complete before the next launch, on any stream
     }
     return SPARK_OK;
 }

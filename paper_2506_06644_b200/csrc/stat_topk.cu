@@ -161,7 +161,8 @@ __global__ void __launch_bounds__(kThreads) stat_topk_kernel(const TopkParams p)
         __syncthreads();
     }
     if (p.theta_in != nullptr) theta = p.theta_in[row];
-    const float shift = p.identity ? 0.f : theta;
+    // a given threshold of -inf is spark_stat_merge's "k >= n_total": everything survives, unshifted
+    const float shift = (p.identity || theta == -INFINITY) ? 0.f : theta;
     const bool want_lists = (p.idx != nullptr) || (p.val != nullptr);
 
     // ---- sweep 3: count the active entries; each warp owns a contiguous run of vectors ----------

@@ -79,6 +79,21 @@ def test_k_at_least_the_total_length_keeps_everything_unshifted(ctx):
     theta = steps.merge(moms, 1024, 1024)
     torch.cuda.synchronize()
     assert torch.isneginf(theta).all()
+    # the selection with that threshold keeps every entry as it is (no shift by -inf), lists and dense form alike
+    for fill, fillc in (("zero", S.SPARK_FILL_ZERO), ("neginf", S.SPARK_FILL_NEGINF)):
+        steps = sharded.gpu_steps(ctx, fillc, idx_cap=724)
+        for r in range(2):
+            _, masks, outs = O.stat_topk_sharded_global([p[r] for p in parts], 1024, fill)
+            for i, x in enumerate(dev):
+                count, idx, val = (t.cpu().numpy() for t in steps.select(x, theta))
+                y = torch.full_like(x, float("nan"))
+                S.spark_stat_select(ctx, x, 2, x.shape[1], x.stride(0), theta, fillc, None, None, None, 0, y)
+                torch.cuda.synchronize()
+                n = parts[i].shape[1]
+                assert count[r] == n == int(masks[i].sum())
+                assert np.array_equal(idx[r, :n], np.arange(n))
+                assert np.array_equal(val[r, :n], parts[i][r])
+                assert np.array_equal(y.cpu().numpy()[r], outs[i].astype(np.float32))
 
 
 def test_argument_errors(ctx):

@@ -34,8 +34,8 @@ def test_every_declared_symbol_is_exported(built):
 
 
 def test_status_strings(built):
-    seen = {S.status_string(c) for c in range(7)}
-    assert len(seen) == 7 and "ok" in seen
+    seen = {S.status_string(c) for c in range(8)}
+    assert len(seen) == 8 and "ok" in seen
     assert S.status_string(99) == "unknown status"
 
 

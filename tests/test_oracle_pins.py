@@ -312,6 +312,42 @@ def test_attention_grouped_heads_and_window():
     assert np.array_equal(one["o"], loc["o"][3])
 
 
+def test_attention_mask_override_branch():
+    # the parity harness hands the oracle a selected set of its own when an entry sits within rounding distance of
+    # theta: (i) its own set changes nothing; (ii) any other set gives softmax over that set x gate, by library ops
+    q, K, V, r = _attn_case(400, seed=7)
+    base = O.spark_attention_head(q, K, V, 40, r)
+    same = O.spark_attention_head(q, K, V, 40, r, mask_override=base["mask"].copy())
+    assert np.array_equal(same["o"], base["o"]) and same["theta"] == base["theta"]
+    hand = np.zeros(400, dtype=bool)
+    hand[[3, 17, 250, 399]] = True                      # a hand-made set, unrelated to the scores
+    got = O.spark_attention_head(q, K, V, 40, r, mask_override=hand)
+    tq, tK, tV = (torch.from_numpy(a) for a in (q, K, V))
+    logits = (tK[:r].T @ tq[:r]).masked_fill(~torch.from_numpy(hand), float("-inf"))
+    w = torch.softmax(logits, 0) * torch.nn.functional.softplus(tK[r:].T @ tq[r:])
+    np.testing.assert_allclose(got["o"], (tV @ w).numpy(), rtol=1e-11, atol=1e-13)
+    assert np.array_equal(got["mask"], hand) and got["theta"] == base["theta"]
+    # one flipped entry moves the output (the override is really used), an empty override attends to nothing
+    flip = base["mask"].copy()
+    flip[np.flatnonzero(~flip)[0]] = True
+    assert not np.array_equal(O.spark_attention_head(q, K, V, 40, r, mask_override=flip)["o"], base["o"])
+    assert np.all(O.spark_attention_head(q, K, V, 40, r, mask_override=np.zeros(400, dtype=bool))["o"] == 0.0)
+    # short context (k >= n, theta = -inf): the override still restricts the softmax
+    q2, K2, V2, _ = _attn_case(30, seed=8)
+    m = np.arange(30) % 2 == 0
+    got = O.spark_attention_head(q2, K2, V2, 64, r, mask_override=m)
+    tq, tK, tV = (torch.from_numpy(a) for a in (q2, K2, V2))
+    logits = (tK[:r].T @ tq[:r]).masked_fill(~torch.from_numpy(m), float("-inf"))
+    w = torch.softmax(logits, 0) * torch.nn.functional.softplus(tK[r:].T @ tq[r:])
+    np.testing.assert_allclose(got["o"], (tV @ w).numpy(), rtol=1e-11, atol=1e-13)
+    # through the grouped-head wrapper: per-head overrides over the whole context, cut to the window inside
+    a = synth.attn_inputs(1, 4, 2, 64, 32, 256, [200], "f32", seed=3)
+    kc = np.concatenate([a.k1c[0], a.k2c[0]], axis=-1)
+    loc = O.spark_attention(a.q[0], kc, a.vc[0], 200, 16, 32, window=50)
+    again = O.spark_attention(a.q[0], kc, a.vc[0], 200, 16, 32, window=50, mask_override=loc["mask"])
+    assert np.array_equal(again["o"], loc["o"])
+
+
 # ----------------------------------------------------------------------------- FLOP counts the paper prints
 def test_flop_counts_match_the_papers_closed_forms():
     d, d_ff, r, k = 2304, 13824, 1024, 1106
