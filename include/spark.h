@@ -331,15 +331,36 @@ typedef struct spark_kv_cache {
 } spark_kv_cache;
 
 /* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2 + n_q) fp32 values, 16-byte aligned, caller-owned, contents
- * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 64.  Four kernels are
- * enqueued for B <= 4: QKV projection with position encoding and cache append, attention, output projection,
- * FFN.  For B >= 5 the position encoding and the append follow the projection as a kernel of their own, and
- * where the shapes allow (see spark_ffn_decode; projections: inputs % 64 == 0, outputs % 128 == 0) the
- * projections and the FFN run as tensor-core GEMMs of two and four kernels each, and the attention of a
- * chunk (SPARK_SHARED_CACHE, B >= 16) as three: up to thirteen kernels per call. */
+ * undefined after the call.  h [B][d] fp32 is updated in place.  1 <= B <= 64.
+ * Four kernels are enqueued for B <= 4: QKV projection with position encoding and cache
+ * append, attention, output projection, FFN.  For B >= 5 the position encoding and the append follow the projection as a
+ * kernel of their own, and where the shapes allow (see spark_ffn_decode; projections: inputs % 64 == 0, outputs % 128 == 0)
+ * the projections and the FFN run as tensor-core GEMMs of two and four kernels each, and the attention of a chunk
+ * (SPARK_SHARED_CACHE, B >= 16) as three: up to thirteen kernels per call. */
 int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
                        const spark_kv_cache* cache, const int32_t* ctx_len, float* h, int64_t B,
                        float* scratch, void* stream);
+
+/* The same for a stack of n_layers layers applied one after the other to the same tokens (Section 4: the decoder is a stack
+ * of such layers; local and global attention layers alternate, so the layers' configurations may differ in `window`):
+ * w, cfg and cache are HOST arrays of n_layers structs, h and scratch as for one layer.  With one token and equal
+ * configurations but for the window, the fused kernel takes up to 64 layers per launch, so that its weight stream runs on
+ * across the layer boundaries; every other call is the loop over spark_layer_decode. */
+int spark_stack_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
+                       const spark_kv_cache* cache, int64_t n_layers, const int32_t* ctx_len, float* h, int64_t B,
+                       float* scratch, void* stream);
+
+/* Scheduling option (the paper has no counterpart; default off): in layer calls of one to four tokens every kernel asks L2,
+ * with a few bulk-prefetch instructions per block, for the weights the NEXT kernel will stream (QKV kernel: Wo; attention:
+ * K1t; FFN, inside spark_stack_decode: the next layer's Wqkv).  Measured on B200 it LOSES (2B layer 30.8 -> 32.0 us, 9B
+ * 57.8 -> 61-63 us): the prefetch traffic delays the few loads the step's critical path waits for by more than the L2-resident
+ * stream saves.  Kept as a switch so that the comparison can be repeated.  Host-only setting. */
+int spark_set_l2_prefetch(spark_ctx* ctx, int on);
+
+/* Scheduling option (the paper has no counterpart): on != 0 makes one-token layer calls take the fused persistent kernel
+ * where it serves the shape; the default (0) is the kernel-per-step path, which measures faster on B200 (the fused kernel's
+ * critical path is bound by serial bookkeeping and grid-wide barriers).  Host-only setting. */
+int spark_set_fused_layer(spark_ctx* ctx, int on);
 
 #ifdef __cplusplus
 }

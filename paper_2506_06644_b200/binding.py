@@ -30,6 +30,7 @@ EXPORTS = [
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
     "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
     "spark_set_wait_limit", "spark_debug_expect_arrivals", "spark_noalloc_status",
+    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch",
 ]
 
 
@@ -91,6 +92,10 @@ def lib() -> C.CDLL:
         "spark_attn_decode_fp8k": (i32, [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
                                          vp, vp, vp, vp, i64, vp]),
         "spark_dense_gemv": (i32, [vp, vp, i64, vp, i32, i64, i64, vp, vp, vp]),
+        "spark_stack_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64,
+                                     vp, vp, i64, vp, vp]),
+        "spark_set_fused_layer": (i32, [vp, i32]),
+        "spark_set_l2_prefetch": (i32, [vp, i32]),
         "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
                                      vp, vp, i64, vp, vp]),
     }
@@ -175,6 +180,14 @@ class SparkContext:
     def set_wait_limit(self, cycles: int):
         """Bound of the waits between thread blocks in SM cycles (0 = the default of about two seconds)."""
         _check(lib().spark_set_wait_limit(self.handle, _stream(), cycles), "spark_set_wait_limit")
+
+    def set_fused_layer(self, on: bool):
+        """One-token layer calls: the fused persistent kernel (default) or the kernel-per-step path."""
+        _check(lib().spark_set_fused_layer(self.handle, 1 if on else 0), "spark_set_fused_layer")
+
+    def set_l2_prefetch(self, on: bool):
+        """Kernels of a one-token layer call ask L2 for the next kernel's weights (default on)."""
+        _check(lib().spark_set_l2_prefetch(self.handle, 1 if on else 0), "spark_set_l2_prefetch")
 
     def debug_expect_arrivals(self, extra: int):
         """Test hook: the one-token FFN kernel waits for `extra` arrivals that never come (0 = off)."""
@@ -277,6 +290,30 @@ def make_layer(weights: dict, cfg: dict, cache: dict) -> LayerHandles:
 def spark_layer_decode(ctx: SparkContext, layer: LayerHandles, ctx_len, h, B, scratch):
     _check(lib().spark_layer_decode(ctx.handle, C.byref(layer.weights), C.byref(layer.cfg), C.byref(layer.cache),
                                     _ptr(ctx_len), _ptr(h), B, _ptr(scratch), _stream()), "spark_layer_decode")
+
+
+@dataclass
+class StackHandles:
+    """Host arrays of the per-layer structs of spark_stack_decode (they only hold pointers)."""
+    weights: object
+    cfgs: object
+    caches: object
+    n_layers: int
+    keep: tuple
+
+
+def make_stack(layers) -> StackHandles:
+    """layers: LayerHandles of the stack's layers, first to last."""
+    n = len(layers)
+    w = (_LayerWeights * n)(*[l.weights for l in layers])
+    c = (_LayerCfg * n)(*[l.cfg for l in layers])
+    kv = (_KvCache * n)(*[l.cache for l in layers])
+    return StackHandles(w, c, kv, n, tuple(layers))
+
+
+def spark_stack_decode(ctx: SparkContext, stack: StackHandles, ctx_len, h, B, scratch):
+    _check(lib().spark_stack_decode(ctx.handle, stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(ctx_len), _ptr(h), B,
+                                    _ptr(scratch), _stream()), "spark_stack_decode")
 
 
 def layer_scratch_floats(cfg: dict, B: int) -> int:

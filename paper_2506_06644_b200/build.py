@@ -18,7 +18,7 @@ LIB = os.path.join(HERE, "libspark_b200.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC",
-    "-Xptxas", "-v",
+    "-Xptxas", "-v", *(["-DSPARK_L1_DEBUG"] if os.environ.get("SPARK_L1_DEBUG") else []),
 ]
 
 

@@ -76,6 +76,7 @@ struct AttnParams {
     SumCell* cells;    // [B * n_q][kAttnWays], zero between launches (the block that merges a segment clears its cells)
     float* lsum;       // [B][n_q] sum of softmax weights per head (o accumulates the weighted values)
     int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
+    PrefetchSpec pf;   // weights of the kernel after this one, asked into L2 once the first predictor rows are in flight
     int check_finite;  // SPARK_CHECK_FINITE: non-finite score sums are reported in the device status
     int pre_stable;    // 1: the kernel directly before this one writes neither ctx_len nor cache rows other than each
                        //    sequence's newest, so lengths and older rows may be read before dep_wait()
@@ -287,6 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                 have_pre = true;
             }
         }
+        if (tid == kThreads - 1) prefetch_l2_share(p.pf, cta, G);
         if (p.pre_stable) {
             dep_wait();
             dep_trigger();
@@ -801,7 +803,7 @@ namespace spark {
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
-                int64_t idx_cap, const float* k1s, cudaStream_t st) {
+                int64_t idx_cap, const float* k1s, cudaStream_t st, PrefetchSpec pf) {
     if (ctx == nullptr || q == nullptr || k1c == nullptr || k2c == nullptr || vc == nullptr || ctx_len == nullptr ||
         o == nullptr)
         return SPARK_ERR_INVALID_ARG;
@@ -861,6 +863,7 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.k_attn = static_cast<int>(k_attn > 0x7fffffff ? 0x7fffffff : k_attn);
     p.dense = (flags & SPARK_DENSE_LOADS) ? 1 : 0;
     p.check_finite = (flags & SPARK_CHECK_FINITE) ? 1 : 0;
+    p.pf = pf;
     const bool shared = (flags & SPARK_SHARED_CACHE) != 0;
     if (shared && (n_kv & (n_kv - 1)) != 0) return SPARK_ERR_UNSUPPORTED;
     p.seg_mask = shared ? static_cast<int>(n_kv - 1) : -1;

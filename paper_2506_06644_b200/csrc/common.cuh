@@ -43,8 +43,13 @@ struct WsHeader {            // lives at the start of the caller's workspace; ze
     unsigned pad[60];
     unsigned seg_done[kMaxSegments];   // attention: finished pieces per segment (self-resetting)
     SumCell ffn_cells[4][4][16][kCellWays];   // FFN: [epoch & 3][token group][token][way] score sums
+    // fused one-token layer kernel: grid-wide barriers as arrival counters that only ever grow (one 32-byte sector per way);
+    // barrier number j since the workspace was last reset is complete when the ways add up to j x blocks (modulo 2^32)
+    unsigned l1_gen;         // barriers completed by the launches so far
+    unsigned l1_pad[63];      // keeps the header a multiple of 256 bytes
+    struct { unsigned count; unsigned pad[7]; } l1_ways[kCellWays];
 };
-static_assert(sizeof(WsHeader) == 256 + 4 * kMaxSegments + 32 * 256 * kCellWays, "header layout");
+static_assert(sizeof(WsHeader) == 256 + 4 * kMaxSegments + 32 * 256 * kCellWays + 256 + 32 * kCellWays && sizeof(WsHeader) % 256 == 0, "header layout");
 
 }  // namespace spark
 
@@ -61,6 +66,9 @@ struct spark_ctx {
     long long trace_cap;
     int overlap;             // launch with programmatic stream serialization, see spark_set_launch_overlap
     unsigned wait_kcycles;   // host copy of the header's wait bound (restored after a workspace reset)
+    const void* next_wqkv;   // set by spark_stack_decode around a layer call: the QKV matrix of the layer after it (or nullptr)
+    int l2_prefetch;         // one-token layer calls ask L2 for the next kernel's weights (spark_set_l2_prefetch)
+    int fused;               // one token: take the fused layer kernel when it serves the shape (spark_set_fused_layer)
     int debug_extra_arrivals;   // test hook: the one-token kernels wait for this many arrivals more than blocks exist
 };
 
@@ -101,6 +109,34 @@ inline cudaError_t launch_kernel(const spark_ctx* ctx, const void* kern, unsigne
         cfg.numAttrs = 1;
     }
     return cudaLaunchKernelExC(&cfg, kern, args);
+}
+
+// ---------------------------------------------------------------------------
+// L2 prefetch of data a LATER kernel of the stream will read (weights: never written).  At one token the steps are
+// latency-bound and HBM idles most of the time; asking L2 for the next kernel's weights meanwhile turns that kernel's
+// streaming phase from an HBM stream into an L2 stream.  One bulk-prefetch instruction covers up to 32 KB, so a block's
+// share (tens of KB) costs one thread a handful of instructions -- unlike a per-line prefetch it does not compete for issue
+// slots or load/store queue entries with the loads on the critical path.
+// ---------------------------------------------------------------------------
+struct PrefetchSpec {
+    const void* ptr;         // nullptr: nothing to prefetch
+    unsigned long long bytes;
+};
+// Called by ONE thread of every block: the block's 1/nparts of the range, in 16-byte aligned pieces.
+__device__ __forceinline__ void prefetch_l2_share(const PrefetchSpec& sp, int part, int nparts) {
+    if (sp.ptr == nullptr) return;
+    const unsigned long long per = ((sp.bytes / nparts) + 127ull) & ~127ull;
+    unsigned long long off = per * part;
+    if (off >= sp.bytes) return;
+    unsigned long long n = sp.bytes - off < per ? sp.bytes - off : per;
+    n &= ~15ull;
+    const char* q = static_cast<const char*>(sp.ptr) + off;
+    while (n > 0) {
+        const unsigned piece = n > 32768ull ? 32768u : static_cast<unsigned>(n);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(q), "r"(piece) : "memory");
+        q += piece;
+        n -= piece;
+    }
 }
 
 // ---------------------------------------------------------------------------

@@ -435,6 +435,7 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     p.hdr = ctx->hdr;
     p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
     p.extra_arrivals = ctx->debug_extra_arrivals;
+    p.pf = a.pf;
     p.check_finite = (a.flags & SPARK_CHECK_FINITE) ? 1 : 0;
     const size_t smem = (static_cast<size_t>(tb) * p.xw + static_cast<size_t>(2) * tb * p.rpc) * sizeof(float) +
                         static_cast<size_t>(p.rpc) * 8;
@@ -552,6 +553,9 @@ extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K
     local.trace_cap = 0;
     local.overlap = 0;
     local.wait_kcycles = 0;
+    local.fused = 0;
+    local.l2_prefetch = 0;
+    local.next_wqkv = nullptr;
     local.debug_extra_arrivals = 0;
     FfnArgs a;
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f;

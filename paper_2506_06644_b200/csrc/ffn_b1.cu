@@ -123,6 +123,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn1_kernel(const FfnParams p) {
     // neurons above the threshold estimated from the block's own scores alone.  The gather then finds most of its
     // rows in L2 instead of waiting for DRAM after the exchange (a lower estimate, which catches more of them, measured
     // slower: the extra requests delay the exchange).
+    if (tid == kThreads - 1) prefetch_l2_share(p.pf, cta, grid);      // the next kernel's weights: HBM idles during the exchange
     if (warp > 0 && !p.identity && !p.dense && nloc >= 8) {
         float a1 = 0.f, a2 = 0.f;
         for (int j = lane; j < nloc; j += 32) {

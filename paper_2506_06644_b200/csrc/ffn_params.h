@@ -24,6 +24,7 @@ struct FfnParams {
     int vrows, vstage_off;        // few-token kernel: rows of V per round and the byte offset of their staging area
     int overlap;                  // launched with the programmatic attribute: weights first, then dep_wait()
     int extra_arrivals;           // test hook (one-token kernel): arrivals waited for beyond the grid's blocks
+    PrefetchSpec pf;              // one-token kernel: weights of the kernel after this one, asked into L2 during the exchange
     int check_finite;             // SPARK_CHECK_FINITE: non-finite score sums are reported in the device status
     double z;
     double inv_n, inv_nm1;        // 1 / d_ff and 1 / (d_ff - 1)

@@ -24,6 +24,7 @@ struct FfnArgs {
     float* theta;
     int32_t* count;
     int32_t* idx;
+    PrefetchSpec pf = PrefetchSpec{nullptr, 0};      // weights of the kernel after this one, asked into L2 (one token)
 };
 int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream);
 
@@ -41,6 +42,8 @@ struct GemvArgs {
     int64_t x_div_group;
     void* zero_ptr;          // nullable: this many bytes (multiple of 16) are cleared by the kernel as a side job
     size_t zero_bytes;
+    const void* pf_ptr;      // nullable: weights of the kernel after this one, asked into L2 (one token)
+    unsigned long long pf_bytes;
 };
 int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 // The same product for 5..16 tokens and bf16 weights as a TMA-fed tcgen05 GEMM (gemm_tc.cu); SPARK_ERR_WORKSPACE = shape or
@@ -55,7 +58,7 @@ int gemm_tc_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
-                int64_t idx_cap, const float* k1s, cudaStream_t st);
+                int64_t idx_cap, const float* k1s, cudaStream_t st, PrefetchSpec pf = PrefetchSpec{nullptr, 0});
 
 // Spark attention for a chunk of a prompt (T consecutive tokens of one sequence over one cache, bf16): predictor scores of
 // the whole chunk as one tcgen05 GEMM per KV head (attn_chunk.cu).  o is written normalised; lsum (nullable) receives 1 per
@@ -63,5 +66,10 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
 int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int64_t T, int64_t n_q,
                       int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs, int64_t window,
                       int64_t k_attn, float* o, float* lsum, float* theta, int32_t* count, cudaStream_t stream);
+
+// One token through n_layers decoder layers in one launch of the fused persistent kernel (layer1.cu); the layers' configurations
+// are equal but for the attention window.  SPARK_ERR_WORKSPACE = shape, flags or sizes not served.
+int layer1_launch(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg, const spark_kv_cache* cache, int n_layers,
+                  const int32_t* ctx_len, float* h, float* scratch, cudaStream_t stream);
 
 }  // namespace spark

@@ -28,6 +28,7 @@ struct GemvParams {
     uint4* zero_ptr;
     int zero_n16;
     int overlap;             // launched with the programmatic attribute: weights first, then dep_wait()
+    PrefetchSpec pf;         // weights of the kernel after this one: asked into L2 once this kernel's own loads are in flight
 };
 
 // Input staging shared by the GEMV kernels: x (optionally divided per group, optionally RMS-normalised)
@@ -143,6 +144,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_kernel(const GemvParams p) {
     const int row1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * p.n_out / gridDim.x);
     EarlyX ex = early_x_request(p, false);
     auto dependency = [&]() {                                     // runs once the first slice of weight loads is in flight
+        if (threadIdx.x == kThreads - 1) prefetch_l2_share(p.pf, blockIdx.x, gridDim.x);
         if (p.overlap) {
             dep_wait();
             dep_trigger();
@@ -404,6 +406,7 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
     };
     EarlyX ex = early_x_request(g, false);
     auto dependency = [&]() {
+        if (tid == kThreads - 1) prefetch_l2_share(g.pf, blockIdx.x, gridDim.x);
         if (g.overlap) {
             dep_wait();
             dep_trigger();
@@ -514,6 +517,7 @@ int gemv_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream) {
         p.x_div_group = static_cast<int>(a.x_div ? a.x_div_group : 1);
         p.zero_ptr = done == 0 ? static_cast<uint4*>(a.zero_ptr) : nullptr;
         p.zero_n16 = done == 0 ? static_cast<int>(a.zero_bytes / 16) : 0;
+        p.pf = PrefetchSpec{done == 0 ? a.pf_ptr : nullptr, a.pf_bytes};
         if (nb >= 5 && a.wdtype == SPARK_BF16 && (a.n_in & 31) == 0 && a.n_out >= 16) {      // tensor cores
             const int rc = nb <= 8 ? gemv_mma_launch<8>(ctx, p, grid, stream) : gemv_mma_launch<16>(ctx, p, grid, stream);
             if (rc == SPARK_OK) {
@@ -539,6 +543,7 @@ extern "C" int spark_dense_gemv(spark_ctx* ctx, const float* x, int64_t B, const
     a.x = x; a.norm_w = nullptr; a.rms_eps = 0.f; a.Wt = Wt; a.wdtype = wdtype;
     a.B = B; a.n_in = n_in; a.n_out = n_out; a.y_add = y_add; a.y = y;
     a.x_div = nullptr; a.x_div_group = 1; a.zero_ptr = nullptr; a.zero_bytes = 0;
+    a.pf_ptr = nullptr; a.pf_bytes = 0;
     return gemv_launch(ctx, a, static_cast<cudaStream_t>(stream));
 }
 
@@ -559,7 +564,12 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     if (!aligned16(scratch) || !aligned16(h)) return SPARK_ERR_UNSUPPORTED;
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (B == 1 && ctx->fused) {           // one token: the whole layer as one persistent kernel when it serves the shape
+        const int rc1 = layer1_launch(ctx, w, cfg, cache, 1, ctx_len, h, scratch, st);
+        if (rc1 != SPARK_ERR_WORKSPACE) return rc1;
+    }
     const int64_t nqkv = (cfg->n_q + 2 * cfg->n_kv) * cfg->hd, nqo = cfg->n_q * cfg->hd;
+    const bool pf_on = ctx->l2_prefetch && B <= 4;      // the latency-bound case
     float* qkv = scratch;                 // [B][nqkv]
     float* qr = qkv + B * nqkv;           // [B][n_q][hd]  position-encoded, scaled queries
     float* ao = qr + B * nqo;             // [B][n_q][hd]  attention output
@@ -597,6 +607,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
         qp.g.B = static_cast<int>(B); qp.g.n_in = static_cast<int>(cfg->d); qp.g.n_out = static_cast<int>(nqkv);
         qp.g.y_add = nullptr; qp.g.y = nullptr; qp.g.x_div = nullptr; qp.g.x_div_group = 1;
         qp.g.zero_ptr = nullptr; qp.g.zero_n16 = 0;
+        qp.g.pf = PrefetchSpec{pf_on ? w->Wo : nullptr, static_cast<unsigned long long>(cfg->d) * nqo * 2ull};
         qp.r = rp;
         const int64_t pairs = nqkv / 2;
         const int gridq = pairs < ctx->num_sms ? static_cast<int>(pairs) : ctx->num_sms;
@@ -609,6 +620,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
         g1.x = h; g1.norm_w = w->norm1; g1.rms_eps = cfg->rms_eps; g1.Wt = w->Wqkv; g1.wdtype = SPARK_BF16;
         g1.B = B; g1.n_in = cfg->d; g1.n_out = nqkv; g1.y_add = nullptr; g1.y = qkv;
         g1.x_div = nullptr; g1.x_div_group = 1; g1.zero_ptr = nullptr; g1.zero_bytes = 0;
+        g1.pf_ptr = nullptr; g1.pf_bytes = 0;
         rc = gemv_launch(ctx, g1, st);
         if (rc != SPARK_OK) return rc;
         const int64_t total = B * (cfg->n_q + 2 * cfg->n_kv) * (cfg->hd / 2);
@@ -621,7 +633,8 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     // 3. Spark attention over the cache (the new token included)
     rc = attn_launch(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd, cfg->r_attn,
                      cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & (SPARK_DENSE_LOADS | SPARK_SHARED_CACHE | SPARK_CHECK_FINITE), ao, lsum, nullptr, nullptr,
-                     nullptr, 0, nullptr, st);
+                     nullptr, 0, nullptr, st,
+                     PrefetchSpec{pf_on ? w->K1t : nullptr, static_cast<unsigned long long>(cfg->d_ff) * cfg->r_ff * 2ull});
     if (rc != SPARK_OK) return rc;
 
     // 4. h2 = h + Wo . (attention sums / sums of weights); the projection kernel also clears the
@@ -631,6 +644,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     g2.B = B; g2.n_in = nqo; g2.n_out = cfg->d; g2.y_add = h; g2.y = h2;
     g2.x_div = lsum; g2.x_div_group = cfg->hd;
     g2.zero_ptr = ctx->scratch; g2.zero_bytes = static_cast<size_t>(B * cfg->n_q) * kAttnWays * sizeof(SumCell);
+    g2.pf_ptr = nullptr; g2.pf_bytes = 0;
     rc = gemv_launch(ctx, g2, st);
     if (rc != SPARK_OK) return rc;
 
@@ -641,5 +655,37 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     f.K1s = nullptr; f.K2s = nullptr; f.Vs = nullptr;
     f.B = B; f.d = cfg->d; f.d_ff = cfg->d_ff; f.r = cfg->r_ff; f.k = cfg->k_ff; f.flags = cfg->flags;
     f.y_init = h2; f.y = h; f.theta = nullptr; f.count = nullptr; f.idx = nullptr;
+    f.pf = PrefetchSpec{pf_on ? ctx->next_wqkv : nullptr, static_cast<unsigned long long>(nqkv) * cfg->d * 2ull};
     return ffn_launch(ctx, f, st);
+}
+
+// A stack of layers for the same tokens: one launch of the fused kernel per 64 layers when it serves the call (one token,
+// equal configurations but for the window), otherwise one spark_layer_decode per layer.
+extern "C" int spark_stack_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg, const spark_kv_cache* cache,
+                                  int64_t n_layers, const int32_t* ctx_len, float* h, int64_t B, float* scratch, void* stream) {
+    if (ctx == nullptr || w == nullptr || cfg == nullptr || cache == nullptr || ctx_len == nullptr || h == nullptr || scratch == nullptr)
+        return SPARK_ERR_INVALID_ARG;
+    if (n_layers < 1 || B < 1 || B > 64) return SPARK_ERR_INVALID_ARG;
+    if (!aligned16(scratch) || !aligned16(h)) return SPARK_ERR_UNSUPPORTED;
+    if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int64_t done = 0;
+    while (done < n_layers) {
+        const int64_t n = n_layers - done < 64 ? n_layers - done : 64;
+        int rc = SPARK_ERR_WORKSPACE;
+        if (B == 1 && ctx->fused) rc = layer1_launch(ctx, w + done, cfg + done, cache + done, static_cast<int>(n), ctx_len, h, scratch, st);
+        if (rc == SPARK_ERR_WORKSPACE) {
+            for (int64_t l = 0; l < n; ++l) {
+                // the FFN kernel of layer l asks L2 for the QKV matrix of layer l + 1 while its blocks exchange their sums
+                ctx->next_wqkv = done + l + 1 < n_layers ? w[done + l + 1].Wqkv : nullptr;
+                rc = spark_layer_decode(ctx, w + done + l, cfg + done + l, cache + done + l, ctx_len, h, B, scratch, stream);
+                ctx->next_wqkv = nullptr;
+                if (rc != SPARK_OK) return rc;
+            }
+        } else if (rc != SPARK_OK) {
+            return rc;
+        }
+        done += n;
+    }
+    return SPARK_OK;
 }

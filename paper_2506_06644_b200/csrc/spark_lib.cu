@@ -104,6 +104,9 @@ int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_
     c->trace_cap = 0;
     c->overlap = 0;
     c->wait_kcycles = 0;
+    c->fused = 0;
+    c->l2_prefetch = 0;
+    c->next_wqkv = nullptr;
     c->debug_extra_arrivals = 0;
     *out = c;
     return SPARK_OK;
@@ -128,6 +131,18 @@ int spark_set_launch_overlap(spark_ctx* ctx, int on) {
 }
 
 int spark_grid_size(const spark_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
+
+int spark_set_l2_prefetch(spark_ctx* ctx, int on) {
+    if (ctx == nullptr) return SPARK_ERR_INVALID_ARG;
+    ctx->l2_prefetch = on ? 1 : 0;
+    return SPARK_OK;
+}
+
+int spark_set_fused_layer(spark_ctx* ctx, int on) {
+    if (ctx == nullptr) return SPARK_ERR_INVALID_ARG;
+    ctx->fused = on ? 1 : 0;
+    return SPARK_OK;
+}
 
 int spark_set_wait_limit(spark_ctx* ctx, void* stream, int64_t cycles) {
     if (ctx == nullptr || cycles < 0) return SPARK_ERR_INVALID_ARG;

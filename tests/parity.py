@@ -56,3 +56,28 @@ def check_output(y_gpu, y_or, kind, what=""):
     tol = OUT_TOL[kind] * scale if scale > 0 else 1e-30
     assert err <= tol, f"{what}: max|err| {err:.3e} > {OUT_TOL[kind]:g} * RMS {scale:.3e}"
     return err / scale if scale > 0 else 0.0
+
+
+def layer_refs_within_band(O, h_in, W, kc, vc, n, window, **shape_kw):
+    """The oracle's decoder layer, then -- lazily -- its variants in which attended tokens whose predictor score lies within
+    BAND * std of their head's threshold are toggled (at most four such tokens: sixteen variants).  The -inf threshold of the
+    attention is discontinuous, so either side of the band is a correct result; a GPU output must match one of them."""
+    ref = O.decoder_layer(h_in, W, kc, vc, n, window=window, **shape_kw)
+    yield ref
+    n_q, n_kv, r = shape_kw["n_q"], shape_kw["n_kv"], shape_kw["r_attn"]
+    lo = 0 if window <= 0 else max(0, n - window)
+    near = []
+    for h in range(n_q):
+        th = ref["attn"]["theta"][h]
+        if not np.isfinite(th):
+            continue
+        s = kc[h // (n_q // n_kv), lo:n, :r] @ ref["q"][h, :r]
+        std = float(np.std(s, ddof=1))
+        near += [(h, lo + int(t)) for t in np.flatnonzero(np.abs(s - th) <= BAND * std)]
+    near = near[:4]
+    for combo in range(1, 1 << len(near)):
+        mask = ref["attn"]["mask"].copy()
+        for i, (h, t) in enumerate(near):
+            if combo >> i & 1:
+                mask[h, t] = not mask[h, t]
+        yield O.decoder_layer(h_in, W, kc, vc, n, window=window, attn_mask_override=mask, **shape_kw)

@@ -96,17 +96,27 @@ def run_and_compare(shape, n_layers, B, ctx_len, steps, seed):
             k2 = c["k2c"][:, :, n - 1].float().cpu().numpy()
             v = c["vc"][:, :, n - 1].float().cpu().numpy()
             for b in range(B):
-                ref = O.decoder_layer(H[l][b], st.W[l], st.kc[l][b], st.vc[l][b], n, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd,
-                                      r_attn=sh.r_attn, k_attn=sh.k_attn, r_ff=sh.r_ff, k_ff=sh.k_ff, window=window_of(l, ctx_len))
                 what = f"step {step} layer {l} seq {b}"
+                # the oracle's layer; if a token sits within rounding distance of an attention threshold, also the variants with
+                # that token on the other side (the threshold is discontinuous: the reading taken for the attention tests)
+                last = None
+                for ref in parity.layer_refs_within_band(O, H[l][b], st.W[l], st.kc[l][b], st.vc[l][b], n, window_of(l, ctx_len), n_q=sh.n_q,
+                                                         n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn, k_attn=sh.k_attn, r_ff=sh.r_ff, k_ff=sh.k_ff):
+                    try:
+                        worst = max(worst, parity.check_output(H[l + 1][b], ref["h"], "bf16", what))
+                        parity.check_output(H[l + 1][b] - H[l][b], ref["h"] - H[l][b], "bf16", what + " (update only)")
+                        last = None
+                        break
+                    except AssertionError as e:
+                        last = e
+                if last is not None:
+                    raise last
                 # appended rows: equal up to one bf16 rounding step of an fp32-vs-fp64 difference; with five or more tokens the
                 # projection's inputs are a two-term bf16 split (an absolute error of about 1e-5 of the row's scale before rounding)
                 got_k = np.concatenate([k1[b], k2[b]], axis=-1)
                 atol = 1e-6 if B < 5 else 1e-4 * parity.rms(st.kc[l][b][:, n - 1])
                 np.testing.assert_allclose(got_k, st.kc[l][b][:, n - 1], rtol=2 ** -7, atol=atol, err_msg=what)
                 np.testing.assert_allclose(v[b], st.vc[l][b][:, n - 1], rtol=2 ** -7, atol=atol, err_msg=what)
-                worst = max(worst, parity.check_output(H[l + 1][b], ref["h"], "bf16", what))
-                parity.check_output(H[l + 1][b] - H[l][b], ref["h"] - H[l][b], "bf16", what + " (update only)")
                 # later steps read the rows the GPU stored
                 st.kc[l][b][:, n - 1] = got_k
                 st.vc[l][b][:, n - 1] = v[b]

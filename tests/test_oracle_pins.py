@@ -442,6 +442,30 @@ def test_decoder_layer_composition_against_library_ops():
 
 
 # ---- storage rounding to FP8 E4M3 (used by the quantised-weight FFN; a library routine is the pin) ----------------
+def test_decoder_layer_hands_a_mask_override_to_the_attention():
+    sh = synth.TINY
+    lw = synth.layer_weights(sh, 3, 0)
+    W = {"norm1": lw.norm1, "norm2": lw.norm2, "Wqkv": synth.bf16_bits_to_f32(lw.Wqkv_bits), "Wo": synth.bf16_bits_to_f32(lw.Wo_bits),
+         "K1t": synth.bf16_bits_to_f32(lw.K1t_bits), "K2t": synth.bf16_bits_to_f32(lw.K2t_bits), "Vt": synth.bf16_bits_to_f32(lw.Vt_bits)}
+    kv = synth.attn_inputs(1, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, 128, [100], "bf16", seed=4)
+    kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+    vc = kv.vc[0].astype(np.float64)
+    h = synth.normal_f32((sh.d,), 3, 60)
+    kw = dict(n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn, k_attn=sh.k_attn, r_ff=sh.r_ff, k_ff=sh.k_ff)
+    base = O.decoder_layer(h, W, kc.copy(), vc.copy(), 100, **kw)
+    same = O.decoder_layer(h, W, kc.copy(), vc.copy(), 100, attn_mask_override=base["attn"]["mask"], **kw)
+    assert np.array_equal(same["h"], base["h"])
+    # the override reaches the attention: it gives what spark_attention gives with it, and a toggled token moves the layer output
+    flip = base["attn"]["mask"].copy()
+    flip[0, np.flatnonzero(~flip[0])[0]] = True
+    other = O.decoder_layer(h, W, kc.copy(), vc.copy(), 100, attn_mask_override=flip, **kw)
+    kc2, vc2 = kc.copy(), vc.copy()
+    O.decoder_layer(h, W, kc2, vc2, 100, **kw)                      # leaves the appended row in kc2 / vc2
+    att = O.spark_attention(base["q"], kc2, vc2, 100, sh.k_attn, sh.r_attn, 0, flip)
+    assert np.array_equal(other["attn"]["o"], att["o"])
+    assert not np.array_equal(other["h"], base["h"])
+
+
 def test_e4m3_rounding_matches_the_library_cast_and_known_codes():
     import torch
     from paper_2506_06644_b200 import synth
