@@ -306,33 +306,37 @@ __device__ __noinline__ bool produce_rows(const Ring& rg, RingPos& pos, long lon
                                              RowMap rowmap, volatile int* fail, long long limit, const PhaseTrace& tr) {
     const int lane = threadIdx.x & 31;
     const RowPhase rp = row_phase_of(K, rg.slot_bytes);
-    int spi = 32 / rp.rps;                                     // slots per trip: no two of them the same ring slot
-    if (spi > rg.n_slots / 2) spi = rg.n_slots / 2;
+    int spi = 32;                                              // slots per trip, a lane each
+    if (spi > rg.n_slots - 1) spi = rg.n_slots - 1;
     if (spi > pc.max_inflight) spi = pc.max_inflight;
     const int nslot = cdiv(nrows, rp.rps);
-    const int si = lane / rp.rps, j = lane - si * rp.rps;
-    for (int s0 = 0; s0 < nslot; s0 += spi) {
-        const int sl = s0 + si, row = sl * rp.rps + j;
-        const bool mine = si < spi && sl < nslot && row < nrows;
-        const RingPos my = pos.plus(si < spi ? si : 0, rg.n_slots);
-        const uint32_t bar = rg.full0 + 8u * my.slot;
-        bool ok = true;
-        if (lane == 0) ok = pace_wait(rg, pc, issued, min(spi, nslot - s0), fail, limit);
-        if (__any_sync(kFull, !ok)) return false;
-        if (mine && j == 0) {
-            ok = claim_slot(rg, my, fail, limit);
-            if (ok) mb_expect_tx(bar, static_cast<uint32_t>(min(rp.rps, nrows - sl * rp.rps)) * K * 2u);
-            dbg_stamp(tr, 0, issued + si);
-        }
-        if (__any_sync(kFull, !ok)) return false;              // also: nobody writes into a slot before it is free
-        if (mine)
-            bulk_g2s(rg.base + static_cast<uint32_t>(my.slot) * rg.slot_bytes + j * rp.rstride, W + static_cast<int64_t>(rowmap(row)) * ld,
-                     static_cast<uint32_t>(K) * 2u, bar);
+    bool all_ok = true;
+    for (int s0 = 0; s0 < nslot && all_ok; s0 += spi) {
         const int done = min(spi, nslot - s0);
+        bool ok = true;
+        if (lane == 0) ok = pace_wait(rg, pc, issued, done, fail, limit);
+        if (__any_sync(kFull, !ok)) return false;
+        // A lane claims its slot and issues that slot's copies at once: a lane whose slot is not free yet (its previous use is
+        // still being consumed) must not hold back the copies of the lanes before it -- the consumers may be waiting for those.
+        if (lane < done) {
+            const int sl = s0 + lane;
+            const RingPos my = pos.plus(lane, rg.n_slots);
+            const uint32_t bar = rg.full0 + 8u * my.slot;
+            ok = claim_slot(rg, my, fail, limit);
+            if (ok) {
+                const int n = min(rp.rps, nrows - sl * rp.rps);
+                mb_expect_tx(bar, static_cast<uint32_t>(n) * K * 2u);
+                for (int j = 0; j < n; ++j)
+                    bulk_g2s(rg.base + static_cast<uint32_t>(my.slot) * rg.slot_bytes + j * rp.rstride,
+                             W + static_cast<int64_t>(rowmap(sl * rp.rps + j)) * ld, static_cast<uint32_t>(K) * 2u, bar);
+            }
+            dbg_stamp(tr, 0, issued + lane);
+        }
+        all_ok = !__any_sync(kFull, !ok);
         pos.skip(done, rg.n_slots);
         issued += done;
     }
-    return true;
+    return all_ok;
 }
 
 __device__ __noinline__ void l1_producer(const L1Params& p, const BlockPlan& bp, const Ring& rg, volatile int* fail, long long limit) {
