@@ -99,7 +99,7 @@ __device__ __forceinline__ bool mb_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait on an mbarrier; `fail` is the block's abort flag (set by whoever gives up first, ends everybody's waits).
-__device__ __noinline__ bool mb_wait(uint32_t bar, uint32_t parity, volatile int* fail, long long limit) {
+__device__ __forceinline__ bool mb_wait(uint32_t bar, uint32_t parity, volatile int* fail, long long limit) {
     if (mb_try(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mb_try(bar, parity)) {
@@ -230,7 +230,7 @@ struct RingPos {             // position in the task sequence: slot and the pari
 // Consumer side: wait until use `q.use` of slot `q.slot` has landed.  A parity wait alone is ambiguous when the waiting warp is
 // not the one that consumed the slot's previous use (the barrier may still be a whole phase behind), so the producer first
 // publishes which use it is filling; the parity wait follows.
-__device__ __noinline__ bool wait_full(const Ring& rg, const RingPos& q, volatile int* fail, long long limit) {
+__device__ __forceinline__ bool wait_full(const Ring& rg, const RingPos& q, volatile int* fail, long long limit) {
     if (rg.fillseq[q.slot] != q.use + 1u) {
         const long long t0 = clock64();
         while (rg.fillseq[q.slot] != q.use + 1u) {
@@ -302,7 +302,7 @@ __device__ __forceinline__ void p2_task(const Ring& rg, const RingPos& pos, int 
 // One matrix phase of the producer (all 32 lanes): rows `rowmap(j)` of W (ld elements per row, K of them used).  A lane per row;
 // the lane of a slot's first row waits until the slot is free and announces the bytes.
 template <typename RowMap>
-__device__ __noinline__ bool produce_rows(const Ring& rg, RingPos& pos, long long& issued, Pace& pc, const __nv_bfloat16* W, int64_t ld, int K, int nrows,
+__device__ __forceinline__ bool produce_rows(const Ring& rg, RingPos& pos, long long& issued, Pace& pc, const __nv_bfloat16* W, int64_t ld, int K, int nrows,
                                              RowMap rowmap, volatile int* fail, long long limit, const PhaseTrace& tr) {
     const int lane = threadIdx.x & 31;
     const RowPhase rp = row_phase_of(K, rg.slot_bytes);
@@ -425,7 +425,7 @@ __device__ __forceinline__ unsigned bf16_bits(float x) { return static_cast<unsi
 // The input vector as three bf16 terms (hi + mid + lo = x to fp32 accuracy: 24 significant bits), one row per term,
 // `stride` bytes apart (64 bytes more than a multiple of 128: the fragment loads of the three rows fall on distinct banks).
 // The tensor-core tiles multiply the bf16 weights by each term (products exact in fp32) and the three columns are added.
-__device__ __noinline__ void stage_split3(const ConsCtx& c, const float* xs, int K, unsigned char* xsp, int stride) {
+__device__ __forceinline__ void stage_split3(const ConsCtx& c, const float* xs, int K, unsigned char* xsp, int stride) {
     for (int i = c.tid; i < K / 2; i += kCons) {
         const float2 v = reinterpret_cast<const float2*>(xs)[i];
         unsigned w[3];
@@ -457,7 +457,7 @@ __device__ __forceinline__ int group_parts(int nrows, int K) {
 // columns as long as both operands use it, so a piece feeds two m16n8k16 MMAs; the B operand holds the three terms of the
 // input in columns 0..2.  out[row * 16 + part] receives the partial dot products.  `pos`: ring position of the phase's first
 // slot on entry, of the next phase's first slot on return.
-__device__ __noinline__ bool group_phase(const ConsCtx& c, RingPos& pos, int nrows, int K, const unsigned char* xsp, int xstride, float* out) {
+__device__ __forceinline__ bool group_phase(const ConsCtx& c, RingPos& pos, int nrows, int K, const unsigned char* xsp, int xstride, float* out) {
     dbg_mark(c.tr, c.mk + 14);
     const RowPhase rp = row_phase_of(K, c.rg.slot_bytes);
     const int lrps = 31 - __clz(rp.rps), spg = 16 >> lrps;
@@ -516,7 +516,7 @@ __device__ __noinline__ bool group_phase(const ConsCtx& c, RingPos& pos, int nro
 
 // Grid-wide barrier number `target_gen` (counted since the workspace was reset): one thread adds the block's arrival to its way,
 // sixteen lanes poll the ways until they add up to target_gen x blocks.  Called by all consumer threads.
-__device__ __noinline__ bool grid_barrier(const ConsCtx& c, WsHeader* hdr, unsigned target_gen, int G, int cta) {
+__device__ __forceinline__ bool grid_barrier(const ConsCtx& c, WsHeader* hdr, unsigned target_gen, int G, int cta) {
     dbg_mark(c.tr, c.mk);
     cons_sync();             // everything this block wrote before is ordered before the arrival (bar.sync + release)
     dbg_mark(c.tr, c.mk + 1);
@@ -565,7 +565,7 @@ __device__ __forceinline__ float cons_sum(const ConsCtx& c, float v, float* scra
 
 // x = RMSNorm(h; w) into shared memory as fp32 and as three bf16 terms (all consumer threads; h read past L1: other blocks
 // wrote it; the norm weights are requested together with h: one trip to memory, not two).
-__device__ __noinline__ void stage_rmsnorm(const ConsCtx& c, const L1Params& p, const float* norm_w, float* xs, float* scratch,
+__device__ __forceinline__ void stage_rmsnorm(const ConsCtx& c, const L1Params& p, const float* norm_w, float* xs, float* scratch,
                                               unsigned char* xsp, int xstride) {
     const int d4 = p.d / 4;
     const bool h0 = c.tid < d4, h1 = c.tid + kCons < d4;          // d <= 4096: at most two float4 per thread
@@ -1230,9 +1230,9 @@ int layer1_launch(spark_ctx* ctx, const spark_layer_weights* w, const spark_laye
     if (n_slots > 64) n_slots = 64;
     p.n_slots = n_slots;
     {
-        // bytes in flight per SM that cover bandwidth x latency: about 48 KB (HBM share of an SM x 1 us); SPARK_L1_INFLIGHT (slots)
-        // overrides it for experiments
-        int q = static_cast<int>((48 * 1024 + slot - 1) / slot);
+        // slots in flight at most; measured: any limit below the ring's size only slows the stream down (2 slots: 71 us per
+        // layer, 8: 51, 20: 50.7 at the 2B shape), so the default is the whole ring; SPARK_L1_INFLIGHT overrides it for experiments
+        int q = n_slots - 1;
         if (const char* e = std::getenv("SPARK_L1_INFLIGHT")) q = std::atoi(e);
         if (q < 2) q = 2;
         if (q > n_slots - 1) q = n_slots - 1;
