@@ -216,8 +216,8 @@ int spark_ffn_decode(spark_ctx* ctx, const float* x, int64_t B, const void* K1t,
  * fp32 scale per neuron: row i of K1t / K2t / Vt stands for K1s[i] / K2s[i] / Vs[i] times its stored values
  * (quantised weights are named in the paper's closing section as the natural companion of activation sparsity;
  * the format and the per-neuron scales are this library's choice).  K1t [d_ff][r], K2t [d_ff][d-r], Vt [d_ff][d]
- * uint8 device buffers, 16-byte aligned, r and d multiples of 8; K1s, K2s, Vs [d_ff] fp32.  One token only
- * (B == 1, d <= 4096): SPARK_ERR_UNSUPPORTED otherwise.  Everything else as spark_ffn_decode. */
+ * uint8 device buffers, 16-byte aligned, r and d multiples of 8; K1s, K2s, Vs [d_ff] fp32.  One to four tokens
+ * (B <= 4, d <= 4096): SPARK_ERR_UNSUPPORTED otherwise.  Everything else as spark_ffn_decode. */
 int spark_ffn_decode_fp8(spark_ctx* ctx, const float* x, int64_t B, const void* K1t, const float* K1s, const void* K2t,
                          const float* K2s, const void* Vt, const float* Vs, int64_t d, int64_t d_ff, int64_t r, int64_t k,
                          int flags, float* y, float* theta, int32_t* count, int32_t* idx, void* stream);
@@ -349,6 +349,17 @@ int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark
 int spark_stack_decode(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg,
                        const spark_kv_cache* cache, int64_t n_layers, const int32_t* ctx_len, float* h, int64_t B,
                        float* scratch, void* stream);
+
+/* A prompt through a stack of layers, chunk by chunk (Section 4.3 reports prefill in chunks of 64 tokens; here 1 <= chunk <= 64):
+ * h [n_tokens][d] fp32 holds the prompt's embeddings and is replaced in place by the stack's outputs; the tokens are appended to
+ * every layer's cache at rows start .. start + n_tokens - 1 (start = tokens already cached), every token attending causally to
+ * the rows before it and to itself, later chunks seeing earlier ones through the caches -- what decoding the prompt token by token
+ * gives.  w, cfg, cache: HOST arrays of n_layers structs; every cfg must carry SPARK_SHARED_CACHE (caches [n_kv][cap][.]) and
+ * cap >= start + n_tokens.  len_buf: caller-owned DEVICE buffer of `chunk` int32 (the library writes each chunk's lengths there);
+ * scratch as for spark_layer_decode with B = chunk.  The call only enqueues: one tiny kernel plus n_layers layer calls per chunk. */
+int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg, const spark_kv_cache* cache,
+                  int64_t n_layers, float* h, int64_t n_tokens, int64_t start, int64_t chunk, int32_t* len_buf, float* scratch,
+                  void* stream);
 
 /* Scheduling option (the paper has no counterpart; default off): in layer calls of one to four tokens every kernel asks L2,
  * with a few bulk-prefetch instructions per block, for the weights the NEXT kernel will stream (QKV kernel: Wo; attention:

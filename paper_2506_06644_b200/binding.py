@@ -30,7 +30,7 @@ EXPORTS = [
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
     "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
     "spark_set_wait_limit", "spark_debug_expect_arrivals", "spark_noalloc_status",
-    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch",
+    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill",
 ]
 
 
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         "spark_stack_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64,
                                      vp, vp, i64, vp, vp]),
         "spark_set_fused_layer": (i32, [vp, i32]),
+        "spark_prefill": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64, vp, i64, i64, i64, vp, vp, vp]),
         "spark_set_l2_prefetch": (i32, [vp, i32]),
         "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
                                      vp, vp, i64, vp, vp]),
@@ -323,7 +324,7 @@ def layer_scratch_floats(cfg: dict, B: int) -> int:
 
 
 def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64):
-    """Run a prompt through a stack of layers chunk by chunk (host loop only: every step is spark_layer_decode).
+    """Run a prompt through a stack of layers chunk by chunk (the C entry point of the same name; argument marshalling only).
 
     layers: LayerHandles made with SPARK_SHARED_CACHE in cfg["flags"] and caches [n_kv][cap][.]; h [N][d] fp32 holds the
     prompt's N embeddings and is replaced in place by the stack's outputs; the tokens are appended to each layer's
@@ -332,14 +333,10 @@ def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64):
     if not 1 <= chunk <= 64:
         raise ValueError("chunk must be 1..64")
     N = h.shape[0]
+    stack = make_stack(layers)
     cfg = {k: getattr(layers[0].cfg, k) for k in ("n_q", "n_kv", "hd", "d")}
     scratch = torch.empty(layer_scratch_floats(cfg, min(chunk, N)), dtype=torch.float32, device=h.device)
-    for c0 in range(0, N, chunk):
-        T = min(chunk, N - c0)
-        lens = torch.arange(start + c0 + 1, start + c0 + T + 1, dtype=torch.int32, device=h.device)
-        part = h[c0 : c0 + T]
-        for layer in layers:
-            if not (layer.cfg.flags & SPARK_SHARED_CACHE):
-                raise ValueError("spark_prefill needs layers configured with SPARK_SHARED_CACHE")
-            spark_layer_decode(ctx, layer, lens, part, T, scratch)
+    len_buf = torch.empty(chunk, dtype=torch.int32, device=h.device)
+    _check(lib().spark_prefill(ctx.handle, stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(h), N, start, chunk,
+                               _ptr(len_buf), _ptr(scratch), _stream()), "spark_prefill")
     return h

@@ -405,7 +405,7 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     if (a.y_init == a.y && a.y_init != nullptr) return SPARK_ERR_INVALID_ARG;
     if (a.wdtype != SPARK_F32 && a.wdtype != SPARK_BF16 && a.wdtype != SPARK_FP8_E4M3) return SPARK_ERR_UNSUPPORTED;
     if (a.wdtype == SPARK_FP8_E4M3 && (a.K1s == nullptr || a.K2s == nullptr || a.Vs == nullptr)) return SPARK_ERR_INVALID_ARG;
-    if (a.wdtype == SPARK_FP8_E4M3 && (a.B != 1 || a.d > 4096)) return SPARK_ERR_UNSUPPORTED;      // one token only
+    if (a.wdtype == SPARK_FP8_E4M3 && (a.B > 4 || a.d > 4096)) return SPARK_ERR_UNSUPPORTED;      // one to four tokens
     if ((a.r & 7) != 0 || (a.d & 7) != 0) return SPARK_ERR_UNSUPPORTED;
     if (!aligned16(a.x) || !aligned16(a.K1t) || !aligned16(a.K2t) || !aligned16(a.Vt) || !aligned16(a.y) ||
         !aligned16(a.y_init) || !aligned16(a.norm_w))
@@ -440,7 +440,12 @@ int ffn_launch(spark_ctx* ctx, const FfnArgs& a, cudaStream_t stream) {
     const size_t smem = (static_cast<size_t>(tb) * p.xw + static_cast<size_t>(2) * tb * p.rpc) * sizeof(float) +
                         static_cast<size_t>(p.rpc) * 8;
     if (smem > static_cast<size_t>(ctx->max_smem_optin - 1024)) return SPARK_ERR_UNSUPPORTED;
-    if (a.wdtype == SPARK_FP8_E4M3) return grid <= 512 ? ffn1_launch(ctx, p, a.wdtype, stream) : SPARK_ERR_UNSUPPORTED;
+    if (a.wdtype == SPARK_FP8_E4M3) {
+        if (grid > 512) return SPARK_ERR_UNSUPPORTED;
+        if (a.B == 1) return ffn1_launch(ctx, p, a.wdtype, stream);
+        const int rc = ffn_few_launch(ctx, p, a.wdtype, stream);
+        return rc == SPARK_ERR_WORKSPACE ? SPARK_ERR_UNSUPPORTED : rc;
+    }
     if (a.B == 1 && grid <= 512 && a.d <= 4096) return ffn1_launch(ctx, p, a.wdtype, stream);
     if (a.B >= 2 && a.B <= 4 && grid <= 512) {
         const int rc = ffn_few_launch(ctx, p, a.wdtype, stream);

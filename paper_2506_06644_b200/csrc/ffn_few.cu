@@ -52,6 +52,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_few_kernel(const FfnParams p)
     const WT* K2t = static_cast<const WT*>(p.K2t);
     const WT* Vt = static_cast<const WT*>(p.Vt);
     const int d4 = d / 4, tot4 = NT * d4;
+    constexpr bool kScaled = sizeof(WT) == 1;      // FP8 storage: one fp32 scale per neuron and matrix
+    constexpr unsigned kChunkB = 8 * sizeof(WT);   // bytes of a thread's eight columns of a row of V
 
     // Everything another kernel may have written is read in after_dependency(): with launch overlap after the
     // first batch of K1t loads has been issued, otherwise before them (requests are served in issue order).
@@ -141,7 +143,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_few_kernel(const FfnParams p)
 
     // ---- A: predictor scores s = K1^T x[:r] of this block's neurons, every token -----------------------
     rows_dot<WT, NT, kRows>(K1t, r, row0, nloc, r / 8, xs, d, [&]() { if (p.overlap) after_dependency(); }, prologue,
-                            [&](int j, int t, float v) { s_loc[static_cast<size_t>(t) * rpc + j] = v; });
+                            [&](int j, int t, float v) { s_loc[static_cast<size_t>(t) * rpc + j] = kScaled ? v * __ldg(p.K1s + row0 + j) : v; });
     __syncthreads();
     p.trace.mark(2);
 
@@ -240,7 +242,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_few_kernel(const FfnParams p)
         if (vcol) {
             for (int q = 0; q < ne; ++q) {
                 const WT* src = Vt + static_cast<int64_t>(row0 + ulist[e0 + q]) * d + 8 * tid;
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(vs0 + 16u * static_cast<unsigned>(q * ncd + tid)), "l"(src) : "memory");
+                if constexpr (kScaled)
+                    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(vs0 + kChunkB * static_cast<unsigned>(q * ncd + tid)), "l"(src) : "memory");
+                else
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(vs0 + kChunkB * static_cast<unsigned>(q * ncd + tid)), "l"(src) : "memory");
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
@@ -304,6 +309,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_few_kernel(const FfnParams p)
                     for (int t = 1; t < NT; ++t) tl = lane == t ? tv[h][t] : tl;
                     const float a = s_loc[static_cast<size_t>(lane) * rpc + jm[h]] - (p.identity ? 0.f : theta_s[lane]);
                     u = (p.erf_form ? gelu_erf(a) : gelu_tanh(a)) * tl;
+                    if constexpr (kScaled) u *= __ldg(p.K2s + row0 + jm[h]) * __ldg(p.Vs + row0 + jm[h]);
                 }
                 uval[lane * 32 + warp + 16 * h] = u;
             }
@@ -313,7 +319,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_few_kernel(const FfnParams p)
         if (vcol) {
             for (int q = 0; q < ne; ++q) {
                 Row8<WT> v8;
-                v8.raw = reinterpret_cast<const uint4*>(vstage)[q * ncd + tid];
+                v8.raw = reinterpret_cast<const decltype(v8.raw)*>(vstage)[q * ncd + tid];
                 float wf[8];
                 v8.unpack(wf);
 #pragma unroll
@@ -349,21 +355,24 @@ namespace spark {
 // Serves 2..4 tokens, bf16 weights, with d <= 4096 (a thread owns one 16-byte column chunk of V) and inputs that fit the
 // registers of the prologue; anything else: SPARK_ERR_WORKSPACE (the caller takes the tensor-core kernel).
 int ffn_few_launch(spark_ctx* ctx, FfnParams& p, int wdtype, cudaStream_t stream) {
-    static bool configured[2][64] = {};
+    static bool configured[4][64] = {};
     const int nt = p.B <= 2 ? 2 : 4;
+    const bool f8 = wdtype == SPARK_FP8_E4M3;
     if (p.B < 2 || p.B > 4 || p.d / 8 > kThreads || nt * (p.d / 4) > kXV * kThreads) return SPARK_ERR_WORKSPACE;
-    if (wdtype != SPARK_BF16) return SPARK_ERR_WORKSPACE;        // fp32 weights double the registers per chunk: not served
+    if (wdtype != SPARK_BF16 && wdtype != SPARK_FP8_E4M3) return SPARK_ERR_WORKSPACE;        // fp32 weights double the registers per chunk: not served
     size_t fixed = (static_cast<size_t>(nt) * p.d + static_cast<size_t>(nt) * p.rpc + nt * 32 + 2 * static_cast<size_t>(p.rpc)) * 4;
     fixed = (fixed + 15) & ~static_cast<size_t>(15);
     const size_t limit = static_cast<size_t>(ctx->max_smem_optin - 2048);
-    const size_t rowb = static_cast<size_t>(p.d) * 2;
+    const size_t rowb = static_cast<size_t>(p.d) * (f8 ? 1 : 2);
     if (fixed + 16 * rowb > limit) return SPARK_ERR_WORKSPACE;
     p.vrows = fixed + 32 * rowb <= limit ? 32 : 16;
     p.vstage_off = static_cast<int>(fixed);
     const size_t smem = fixed + static_cast<size_t>(p.vrows) * rowb;
-    const void* kern = nt == 2 ? reinterpret_cast<const void*>(ffn_few_kernel<__nv_bfloat16, 2>)
-                               : reinterpret_cast<const void*>(ffn_few_kernel<__nv_bfloat16, 4>);
-    const int ki = nt == 2 ? 0 : 1;
+    const void* kern = f8 ? (nt == 2 ? reinterpret_cast<const void*>(ffn_few_kernel<__nv_fp8_e4m3, 2>)
+                                     : reinterpret_cast<const void*>(ffn_few_kernel<__nv_fp8_e4m3, 4>))
+                          : (nt == 2 ? reinterpret_cast<const void*>(ffn_few_kernel<__nv_bfloat16, 2>)
+                                     : reinterpret_cast<const void*>(ffn_few_kernel<__nv_bfloat16, 4>));
+    const int ki = (nt == 2 ? 0 : 1) + (f8 ? 2 : 0);
     if (ctx->device >= 0 && ctx->device < 64 && !configured[ki][ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 1024) != cudaSuccess)
             return SPARK_ERR_CUDA;

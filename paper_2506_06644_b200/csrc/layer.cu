@@ -689,3 +689,40 @@ extern "C" int spark_stack_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     }
     return SPARK_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// spark_prefill: a prompt through a stack of layers chunk by chunk (Section 4.3 measures prefill in chunks of 64 tokens).
+// ---------------------------------------------------------------------------------------------
+namespace {
+__global__ void chunk_lengths_kernel(int32_t* len, int n, int first) {      // len[b] = first + b: token b of the chunk sees first + b tokens
+    dep_wait();
+    dep_trigger();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) len[i] = first + i;
+}
+}  // namespace
+
+extern "C" int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const spark_layer_cfg* cfg, const spark_kv_cache* cache,
+                             int64_t n_layers, float* h, int64_t n_tokens, int64_t start, int64_t chunk, int32_t* len_buf, float* scratch,
+                             void* stream) {
+    if (ctx == nullptr || w == nullptr || cfg == nullptr || cache == nullptr || h == nullptr || len_buf == nullptr || scratch == nullptr)
+        return SPARK_ERR_INVALID_ARG;
+    if (n_layers < 1 || n_tokens < 1 || start < 0 || chunk < 1 || chunk > 64) return SPARK_ERR_INVALID_ARG;
+    for (int64_t l = 0; l < n_layers; ++l) {
+        if (!(cfg[l].flags & SPARK_SHARED_CACHE)) return SPARK_ERR_INVALID_ARG;      // the chunk's tokens share one cache
+        if (start + n_tokens > cfg[l].cap || cfg[l].d != cfg[0].d) return SPARK_ERR_INVALID_ARG;
+    }
+    if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int64_t c0 = 0; c0 < n_tokens; c0 += chunk) {
+        const int64_t T = n_tokens - c0 < chunk ? n_tokens - c0 : chunk;
+        int n = static_cast<int>(T), first = static_cast<int>(start + c0 + 1);
+        void* args[] = {&len_buf, &n, &first};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(chunk_lengths_kernel), 1u, 64u, 0, st, false, args) != cudaSuccess) return SPARK_ERR_CUDA;
+        for (int64_t l = 0; l < n_layers; ++l) {
+            const int rc = spark_layer_decode(ctx, w + l, cfg + l, cache + l, len_buf, h + c0 * cfg[0].d, T, scratch, stream);
+            if (rc != SPARK_OK) return rc;
+        }
+    }
+    return SPARK_OK;
+}
