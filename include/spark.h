@@ -78,6 +78,11 @@ enum {
                                 [n_kv][cap][.]; token b is the sequence's token number ctx_len[b]
                                 (1-based) and sees rows [0, ctx_len[b]), so with ctx_len[b] =
                                 L0 + b + 1 the chunk is causal; caches lose their [B] dimension  */
+    SPARK_FFN_FP8 = 16,      /* layer: K1t, K2t, Vt are FP8 E4M3 with the per-neuron scales K1s, K2s, Vs of
+                                spark_layer_weights (as in spark_ffn_decode_fp8; one to four tokens)    */
+    SPARK_K1C_FP8 = 32,      /* layer: the predictor slice of the cache is FP8 E4M3 with one fp32 scale per
+                                cached row in spark_kv_cache.k1s (as in spark_attn_decode_fp8k); the
+                                appended row is stored as e4m3(k / s) with s = max|k| / 448              */
     SPARK_CHECK_FINITE = 8   /* debugging aid: a threshold whose score sums are not finite (a NaN or an
                                 infinity reached the predictor) records SPARK_ERR_NONFINITE in the
                                 device status.  Honoured by the one-token FFN kernel and by the
@@ -312,6 +317,9 @@ typedef struct spark_layer_weights {
     const void* K1t;      /* [d_ff][r_ff]           bf16  */
     const void* K2t;      /* [d_ff][d - r_ff]       bf16  */
     const void* Vt;       /* [d_ff][d]              bf16  */
+    const float* K1s;     /* [d_ff] per-neuron scales of K1t, K2t, Vt: only with SPARK_FFN_FP8 (the three    */
+    const float* K2s;     /*        matrices are then uint8 E4M3 codes), NULL otherwise                   */
+    const float* Vs;
 } spark_layer_weights;
 
 typedef struct spark_layer_cfg {
@@ -328,6 +336,8 @@ typedef struct spark_kv_cache {
     void* k1c;            /* [B][n_kv][cap][r_attn]      bf16, row ctx_len[b]-1 is written */
     void* k2c;            /* [B][n_kv][cap][hd-r_attn]   bf16                              */
     void* vc;             /* [B][n_kv][cap][hd]          bf16                              */
+    float* k1s;           /* [B][n_kv][cap] row scales of k1c: only with SPARK_K1C_FP8 (k1c is then uint8
+                             E4M3 codes; entry ctx_len[b]-1 is written), NULL otherwise             */
 } spark_kv_cache;
 
 /* scratch: B * ((n_q + 2 n_kv) hd + 2 n_q hd + d + 2 + n_q) fp32 values, 16-byte aligned, caller-owned, contents

@@ -324,7 +324,7 @@ def round_to_bf16(a):
 def decoder_layer(h, W, kcache, vcache, ctx_len: int, *, n_q: int, n_kv: int, hd: int,
                   r_attn: int, k_attn: int, r_ff: int, k_ff: int, window: int = 0,
                   gelu_form: str = "tanh", eps: float = 1e-6, cache_bf16: bool = True,
-                  rope_base: float = 10000.0, attn_mask_override=None):
+                  rope_base: float = 10000.0, attn_mask_override=None, k_round=None):
     """One pre-norm decoder layer for one new token of one sequence.
 
         a  = RMSNorm(h; norm1);  [q|k|v] = Wqkv a
@@ -336,7 +336,9 @@ def decoder_layer(h, W, kcache, vcache, ctx_len: int, *, n_q: int, n_kv: int, hd
     W: dict(norm1[d], norm2[d], Wqkv[(n_q+2 n_kv) hd][d], Wo[d][n_q hd],
             K1t[d_ff][r_ff], K2t[d_ff][d-r_ff], Vt[d_ff][d])  (storage-rounded values).
     kcache / vcache: [n_kv][cap][hd] fp64 arrays, modified in place.
-    ctx_len counts the new token.  attn_mask_override, if given, is handed to spark_attention (the
+    ctx_len counts the new token.  k_round, if given, is the storage rounding of the appended key rows
+    ([n_kv][hd] -> the values a quantised cache holds; the rule itself belongs to whoever defines the
+    storage format) and replaces the bf16 rounding of k.  attn_mask_override, if given, is handed to spark_attention (the
     parity harness's way of following the other side's choice for a token within rounding distance of
     the attention threshold).  Returns dict(h, attn, ffn, q).
     """
@@ -351,6 +353,8 @@ def decoder_layer(h, W, kcache, vcache, ctx_len: int, *, n_q: int, n_kv: int, hd
     kn = rope_split(kn, pos, r_attn, rope_base)
     if cache_bf16:
         kn, vn = round_to_bf16(kn), round_to_bf16(vn)
+    if k_round is not None:
+        kn = np.asarray(k_round(rope_split(qkv[n_q * hd:(n_q + n_kv) * hd].reshape(n_kv, hd), pos, r_attn, rope_base)), dtype=F64)
     kcache[:, pos, :] = kn
     vcache[:, pos, :] = vn
     att = spark_attention(q, kcache, vcache, ctx_len, k_attn, r_attn, window, attn_mask_override)

@@ -23,6 +23,7 @@ SPARK_ERR_TIMEOUT, SPARK_ERR_OVERFLOW, SPARK_ERR_NONFINITE = 5, 6, 7
 SPARK_F32, SPARK_BF16, SPARK_FP8_E4M3 = 0, 1, 2
 SPARK_FILL_ZERO, SPARK_FILL_NEGINF = 0, 1
 SPARK_GELU_TANH, SPARK_GELU_ERF, SPARK_DENSE_LOADS, SPARK_SHARED_CACHE, SPARK_CHECK_FINITE = 0, 1, 2, 4, 8
+SPARK_FFN_FP8, SPARK_K1C_FP8 = 16, 32
 
 EXPORTS = [
     "spark_status_string", "spark_normal_upper_quantile", "spark_workspace_bytes", "spark_create",
@@ -41,7 +42,7 @@ class SparkError(RuntimeError):
 
 
 class _LayerWeights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("norm1", "norm2", "Wqkv", "Wo", "K1t", "K2t", "Vt")]
+    _fields_ = [(n, C.c_void_p) for n in ("norm1", "norm2", "Wqkv", "Wo", "K1t", "K2t", "Vt", "K1s", "K2s", "Vs")]
 
 
 class _LayerCfg(C.Structure):
@@ -51,7 +52,7 @@ class _LayerCfg(C.Structure):
 
 
 class _KvCache(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("k1c", "k2c", "vc")]
+    _fields_ = [(n, C.c_void_p) for n in ("k1c", "k2c", "vc", "k1s")]
 
 
 _lib = None
@@ -282,9 +283,9 @@ class LayerHandles:
 
 
 def make_layer(weights: dict, cfg: dict, cache: dict) -> LayerHandles:
-    w = _LayerWeights(**{k: _ptr(weights[k]) for k in ("norm1", "norm2", "Wqkv", "Wo", "K1t", "K2t", "Vt")})
+    w = _LayerWeights(**{k: _ptr(weights.get(k)) for k in ("norm1", "norm2", "Wqkv", "Wo", "K1t", "K2t", "Vt", "K1s", "K2s", "Vs")})
     c = _LayerCfg(**cfg)
-    kv = _KvCache(**{k: _ptr(cache[k]) for k in ("k1c", "k2c", "vc")})
+    kv = _KvCache(**{k: _ptr(cache.get(k)) for k in ("k1c", "k2c", "vc", "k1s")})
     return LayerHandles(w, c, kv, (weights, cache))
 
 

@@ -871,7 +871,9 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.cells = reinterpret_cast<SumCell*>(ctx->scratch);
     p.lsum = lsum != nullptr ? lsum : reinterpret_cast<float*>(ctx->scratch + cells_b);
     p.defer = lsum != nullptr ? 1 : 0;
-    p.pre_stable = p.defer && !shared;      // a chunk's rows are all fresh from the kernel ahead
+    // a chunk's rows are all fresh from the kernel ahead; the FP8 tensor-core pass requests its first tile without holding
+    // the newest row back, so it waits for the kernel ahead first
+    p.pre_stable = p.defer && !shared && k1s == nullptr;
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;

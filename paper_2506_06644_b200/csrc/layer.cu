@@ -312,6 +312,9 @@ struct RopeParams {
     float base, q_scale;
     double* zs;              // [B] out: Q(1 - k_attn / L_b) for the attention kernel that follows
     int window, k_attn;
+    float* k1f32;            // nullable: the rotated predictor part of the new keys goes here in fp32 (element i of KV head g of
+                             // token b at b * k1f32_sb + g * k1f32_sg + i) instead of into k1c: an FP8 slice is quantised by its own kernel
+    int64_t k1f32_sb, k1f32_sg;
     double inv_freq[2][64];  // base^(-2i/m) for the pairs of the first part (m = r) and of the second (m = hd - r)
 };
 
@@ -364,7 +367,11 @@ __global__ void rope_append_kernel(const RopeParams p) {
         } else {
             const int g = h - p.n_q;
             const int64_t rowi = (static_cast<int64_t>(p.shared ? 0 : b) * p.n_kv + g) * p.cap + pos;
-            if (part0 == 0) {
+            if (part0 == 0 && p.k1f32 != nullptr) {
+                float* dst = p.k1f32 + static_cast<int64_t>(b) * p.k1f32_sb + static_cast<int64_t>(g) * p.k1f32_sg;
+                dst[pi] = ra;
+                dst[pi + m / 2] = rb;
+            } else if (part0 == 0) {
                 __nv_bfloat16* dst = p.k1c + rowi * p.r;
                 dst[pi] = __float2bfloat16_rn(ra);
                 dst[pi + m / 2] = __float2bfloat16_rn(rb);
@@ -375,6 +382,45 @@ __global__ void rope_append_kernel(const RopeParams p) {
             }
         }
     }
+}
+
+// The appended row of an FP8 predictor slice: a warp per (token, KV head) takes the fp32 row the projection left, its largest
+// magnitude gives the row's scale s = max|k| / 448 (1 for an all-zero row), the row is stored as e4m3(k / s) (the storage rule of
+// spark_attn_decode_fp8k; format and per-row scales are this library's choice, the paper's closing section only names quantisation).
+struct K1QuantParams {
+    const float* k1f32;
+    int64_t sb, sg;
+    unsigned char* k1c;      // [B or 1][n_kv][cap][r] E4M3 codes
+    float* k1s;              // [B or 1][n_kv][cap]
+    const int32_t* ctx_len;
+    int B, n_kv, r, shared;
+    int64_t cap;
+};
+__global__ void k1_quant_kernel(const K1QuantParams p) {
+    dep_wait();
+    dep_trigger();
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (w >= p.B * p.n_kv) return;
+    const int b = w / p.n_kv, g = w - b * p.n_kv;
+    int n = p.ctx_len[b];
+    n = n < 1 ? 1 : (n > p.cap ? static_cast<int>(p.cap) : n);
+    const float* src = p.k1f32 + static_cast<int64_t>(b) * p.sb + static_cast<int64_t>(g) * p.sg;
+    float v[4], amax = 0.f;                       // r <= 128: four values per lane
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int i = lane * 4 + e;
+        v[e] = i < p.r ? src[i] : 0.f;
+        amax = fmaxf(amax, fabsf(v[e]));
+    }
+    amax = warp_max(amax);
+    const float scale = amax > 0.f ? amax / 448.0f : 1.0f;
+    const int64_t rowi = (static_cast<int64_t>(p.shared ? 0 : b) * p.n_kv + g) * p.cap + (n - 1);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int i = lane * 4 + e;
+        if (i < p.r) p.k1c[rowi * p.r + i] = static_cast<unsigned char>(__nv_cvt_float_to_fp8(v[e] / scale, __NV_SATFINITE, __NV_E4M3));
+    }
+    if (lane == 0) p.k1s[rowi] = scale;
 }
 
 // QKV projection with the rotary encoding and the cache append in its epilogue: a warp computes the
@@ -455,9 +501,15 @@ __global__ void __launch_bounds__(kThreads, 1) qkv_rope_kernel(const QkvRopePara
             } else {
                 const int gk = head - rp.n_q;
                 const int64_t rowi = (static_cast<int64_t>(rp.shared ? 0 : t) * rp.n_kv + gk) * rp.cap + pos;
-                __nv_bfloat16* dst = second ? rp.k2c + rowi * (hd - rp.r) : rp.k1c + rowi * rp.r;
-                dst[pi] = __float2bfloat16_rn(ra);
-                dst[pi + m / 2] = __float2bfloat16_rn(rb);
+                if (!second && rp.k1f32 != nullptr) {
+                    float* dst = rp.k1f32 + static_cast<int64_t>(t) * rp.k1f32_sb + static_cast<int64_t>(gk) * rp.k1f32_sg;
+                    dst[pi] = ra;
+                    dst[pi + m / 2] = rb;
+                } else {
+                    __nv_bfloat16* dst = second ? rp.k2c + rowi * (hd - rp.r) : rp.k1c + rowi * rp.r;
+                    dst[pi] = __float2bfloat16_rn(ra);
+                    dst[pi + m / 2] = __float2bfloat16_rn(rb);
+                }
             }
         });
 }
@@ -562,6 +614,11 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
         cfg->n_kv < 1 || cfg->d < 16)
         return SPARK_ERR_INVALID_ARG;
     if (!aligned16(scratch) || !aligned16(h)) return SPARK_ERR_UNSUPPORTED;
+    const bool ffn_f8 = (cfg->flags & SPARK_FFN_FP8) != 0, k1_f8 = (cfg->flags & SPARK_K1C_FP8) != 0;
+    if (ffn_f8 && (w->K1s == nullptr || w->K2s == nullptr || w->Vs == nullptr)) return SPARK_ERR_INVALID_ARG;
+    if (k1_f8 && cache->k1s == nullptr) return SPARK_ERR_INVALID_ARG;
+    if (ffn_f8 && B > 4) return SPARK_ERR_UNSUPPORTED;          // the chunk kernels take bf16 weights
+    if (k1_f8 && (cfg->flags & SPARK_SHARED_CACHE) && B >= 16) return SPARK_ERR_UNSUPPORTED;      // the chunk attention takes a bf16 slice
     if (!on_device(ctx)) return SPARK_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (B == 1 && ctx->fused) {           // one token: the whole layer as one persistent kernel when it serves the shape
@@ -594,6 +651,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
             rp.inv_freq[part][i] = std::pow(static_cast<double>(cfg->rope_base), -2.0 * static_cast<double>(i) / static_cast<double>(m));
     }
     rp.zs = zs; rp.window = static_cast<int>(cfg->window > 0x7fffffff ? 0x7fffffff : cfg->window);
+    rp.k1f32 = nullptr; rp.k1f32_sb = 0; rp.k1f32_sg = 0;
     rp.k_attn = static_cast<int>(cfg->k_attn > 0x7fffffff ? 0x7fffffff : cfg->k_attn);
     int rc;
     const int tbq = B == 1 ? 1 : (B <= 4 ? 4 : 16);
@@ -602,6 +660,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     // then a small kernel for the rotary encoding and the append
     if (B <= 4 && (cfg->d & 7) == 0 && smem_q <= static_cast<size_t>(ctx->max_smem_optin - 1024) && nqkv / 2 >= 1 &&
         aligned16(w->Wqkv) && aligned16(w->norm1)) {
+        if (k1_f8) { rp.k1f32 = qkv; rp.k1f32_sb = cfg->n_kv * cfg->r_attn; rp.k1f32_sg = cfg->r_attn; }      // the projection buffer is free here
         QkvRopeParams qp;
         qp.g.x = h; qp.g.norm_w = w->norm1; qp.g.eps = cfg->rms_eps; qp.g.Wt = w->Wqkv;
         qp.g.B = static_cast<int>(B); qp.g.n_in = static_cast<int>(cfg->d); qp.g.n_out = static_cast<int>(nqkv);
@@ -623,6 +682,7 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
         g1.pf_ptr = nullptr; g1.pf_bytes = 0;
         rc = gemv_launch(ctx, g1, st);
         if (rc != SPARK_OK) return rc;
+        if (k1_f8) { rp.k1f32 = qkv + cfg->n_q * cfg->hd; rp.k1f32_sb = nqkv; rp.k1f32_sg = cfg->hd; }      // rotated in place
         const int64_t total = B * (cfg->n_q + 2 * cfg->n_kv) * (cfg->hd / 2);
         const int blocks = static_cast<int>((total + 255) / 256);
         void* rargs[] = {&rp};
@@ -630,11 +690,24 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
             return SPARK_ERR_CUDA;
     }
 
+    // 2b. an FP8 predictor slice: the appended rows are quantised (one warp per token and KV head)
+    if (k1_f8) {
+        K1QuantParams kq;
+        kq.k1f32 = rp.k1f32; kq.sb = rp.k1f32_sb; kq.sg = rp.k1f32_sg;
+        kq.k1c = static_cast<unsigned char*>(cache->k1c); kq.k1s = cache->k1s; kq.ctx_len = ctx_len;
+        kq.B = static_cast<int>(B); kq.n_kv = static_cast<int>(cfg->n_kv); kq.r = static_cast<int>(cfg->r_attn);
+        kq.shared = rp.shared; kq.cap = cfg->cap;
+        const unsigned warps = static_cast<unsigned>(B * cfg->n_kv);
+        void* kargs[] = {&kq};
+        if (launch_kernel(ctx, reinterpret_cast<const void*>(k1_quant_kernel), (warps + 7) / 8, 256, 0, st, false, kargs) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+    }
+
     // 3. Spark attention over the cache (the new token included)
     rc = attn_launch(ctx, qr, cache->k1c, cache->k2c, cache->vc, SPARK_BF16, B, cfg->n_q, cfg->n_kv, cfg->hd, cfg->r_attn,
                      cfg->cap, ctx_len, zs, cfg->window, cfg->k_attn, cfg->flags & (SPARK_DENSE_LOADS | SPARK_SHARED_CACHE | SPARK_CHECK_FINITE), ao, lsum, nullptr, nullptr,
-                     nullptr, 0, nullptr, st,
-                     PrefetchSpec{pf_on ? w->K1t : nullptr, static_cast<unsigned long long>(cfg->d_ff) * cfg->r_ff * 2ull});
+                     nullptr, 0, k1_f8 ? cache->k1s : nullptr, st,
+                     PrefetchSpec{pf_on ? w->K1t : nullptr, static_cast<unsigned long long>(cfg->d_ff) * cfg->r_ff * (ffn_f8 ? 1ull : 2ull)});
     if (rc != SPARK_OK) return rc;
 
     // 4. h2 = h + Wo . (attention sums / sums of weights); the projection kernel also clears the
@@ -651,9 +724,9 @@ extern "C" int spark_layer_decode(spark_ctx* ctx, const spark_layer_weights* w, 
     // 5. h = h2 + SparkFFN(RMSNorm(h2; norm2))
     FfnArgs f;
     f.x = h2; f.norm_w = w->norm2; f.rms_eps = cfg->rms_eps;
-    f.K1t = w->K1t; f.K2t = w->K2t; f.Vt = w->Vt; f.wdtype = SPARK_BF16;
-    f.K1s = nullptr; f.K2s = nullptr; f.Vs = nullptr;
-    f.B = B; f.d = cfg->d; f.d_ff = cfg->d_ff; f.r = cfg->r_ff; f.k = cfg->k_ff; f.flags = cfg->flags;
+    f.K1t = w->K1t; f.K2t = w->K2t; f.Vt = w->Vt; f.wdtype = ffn_f8 ? SPARK_FP8_E4M3 : SPARK_BF16;
+    f.K1s = ffn_f8 ? w->K1s : nullptr; f.K2s = ffn_f8 ? w->K2s : nullptr; f.Vs = ffn_f8 ? w->Vs : nullptr;
+    f.B = B; f.d = cfg->d; f.d_ff = cfg->d_ff; f.r = cfg->r_ff; f.k = cfg->k_ff; f.flags = cfg->flags & (SPARK_GELU_ERF | SPARK_DENSE_LOADS | SPARK_CHECK_FINITE);
     f.y_init = h2; f.y = h; f.theta = nullptr; f.count = nullptr; f.idx = nullptr;
     f.pf = PrefetchSpec{pf_on ? ctx->next_wqkv : nullptr, static_cast<unsigned long long>(nqkv) * cfg->d * 2ull};
     return ffn_launch(ctx, f, st);

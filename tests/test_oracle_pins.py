@@ -464,6 +464,12 @@ def test_decoder_layer_hands_a_mask_override_to_the_attention():
     att = O.spark_attention(base["q"], kc2, vc2, 100, sh.k_attn, sh.r_attn, 0, flip)
     assert np.array_equal(other["attn"]["o"], att["o"])
     assert not np.array_equal(other["h"], base["h"])
+    # the storage-rounding hook of the appended key rows: bf16 rounding through it is the default; another rule is what gets stored
+    same2 = O.decoder_layer(h, W, kc.copy(), vc.copy(), 100, k_round=O.round_to_bf16, **kw)
+    assert np.array_equal(same2["h"], base["h"])
+    kc3 = kc.copy()
+    O.decoder_layer(h, W, kc3, vc.copy(), 100, k_round=lambda rows: np.round(rows * 4.0) / 4.0, **kw)
+    assert np.all(kc3[:, 99] * 4.0 == np.round(kc3[:, 99] * 4.0)) and not np.array_equal(kc3[:, 99], kc2[:, 99])
 
 
 def test_e4m3_rounding_matches_the_library_cast_and_known_codes():
