@@ -55,6 +55,7 @@ def parse():
     ap.add_argument("--no-cpu", action="store_true", help="skip the oracle timing")
     ap.add_argument("--overlap", type=int, default=1, help="1 = launch kernels with programmatic stream serialization")
     ap.add_argument("--no-extra", action="store_true", help="skip the other configurations (batched FFN, long-context attention, top-k)")
+    ap.add_argument("--study", default="", choices=["", "batch"], help="batch: where the union of the tokens' active sets stops paying (Appendix B)")
     ap.add_argument("--no-graph", action="store_true", help="launch every kernel from the host instead of replaying a CUDA graph")
     return ap.parse_args()
 
@@ -727,6 +728,49 @@ def other_workloads(torch, S, peak, steps, warmup, with_oracle=True):
                 "dense_loads_us_per_launch": res[1], "speedup_vs_dense_loads": res[1] / res[0]})
     ctx.close()
 
+    # -- the same layers with quantised storage (the paper's closing section: quantisation compounds with activation sparsity):
+    #    FP8 E4M3 predictor slice of the cache with row scales at batch 1 and 8; at batch 1 also FP8 FFN weights with per-neuron scales
+    ctx = S.SparkContext(dev.index, max_batch=8, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
+    ctx.set_launch_overlap(True)
+
+    def q8rows(t):
+        tf = t.float()
+        sc = tf.abs().amax(dim=-1).clamp_min(1e-30) / 448.0
+        return (tf / sc[..., None]).to(torch.float8_e4m3fn).view(torch.uint8), sc
+    for Bq in (1, 8):
+        qlayers = []
+        for l, (_, wts, cache) in enumerate(stacks[0]):
+            k1q, k1s = q8rows(cache["k1c"][:Bq])
+            cq = dict(k1c=k1q.contiguous(), k1s=k1s.contiguous(), k2c=cache["k2c"][:Bq].contiguous(), vc=cache["vc"][:Bq].contiguous())
+            wq = dict(wts)
+            flags = S.SPARK_K1C_FP8
+            if Bq <= 4:
+                flags |= S.SPARK_FFN_FP8
+                for nm, sn in (("K1t", "K1s"), ("K2t", "K2s"), ("Vt", "Vs")):
+                    wq[nm], wq[sn] = q8rows(wts[nm])
+            cfg = dict(d=sh.d, d_ff=sh.d_ff, r_ff=sh.r_ff, k_ff=sh.k_ff, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+                       k_attn=sh.k_attn, window=4096 if l % 2 == 0 else 0, cap=L, rms_eps=1e-6, rope_base=10000.0, flags=flags)
+            cfg_b = dict(cfg, flags=0)
+            cb = dict(k1c=cache["k1c"][:Bq].contiguous(), k2c=cq["k2c"], vc=cq["vc"])
+            qlayers.append((S.make_layer(wq, cfg, cq), S.make_layer(wts, cfg_b, cb), wq, cq, cb))
+        hq = torch.randn(Bq, sh.d, device=dev, generator=gen)
+        clq = torch.full((Bq,), L, dtype=torch.int32, device=dev)
+        scq = torch.empty(S.layer_scratch_floats(dict(n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, d=sh.d), Bq), device=dev)
+        r8 = []
+        for which in (0, 1):
+            def calls():
+                for lay in qlayers:
+                    S.spark_layer_decode(ctx, lay[which], clq, hq, Bq, scq)
+            r8.append(time_graph(calls, nl))
+        assert ctx.device_status() == S.SPARK_OK
+        out.append({"workload": f"spark_layer_decode gemma2-2b shape with quantised storage, batch {Bq}, context {L}, {nl} layers: FP8 predictor "
+                                "slice of the cache" + (" and FP8 FFN weights" if Bq <= 4 else " (FFN weights bf16: the chunk kernels take bf16)") +
+                                "; per layer, beside the bf16 layer on the same inputs",
+                    "us_per_launch": r8[0], "us_per_token_per_layer": r8[0] / Bq, "bf16_us_per_launch": r8[1],
+                    "speedup_vs_bf16_storage": r8[1] / r8[0]})
+        del qlayers
+    ctx.close()
+
     # -- the same eight layers over chunks of a prompt: T consecutive tokens of ONE sequence per call (SPARK_SHARED_CACHE),
     #    appended behind 8192 - T cached tokens, every token attending causally; per-layer caches [n_kv][L][.]
     ctx = S.SparkContext(dev.index, max_batch=64, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
@@ -880,8 +924,75 @@ def cpu_baseline(args, shape):
     return out
 
 
+def batch_study(args):
+    """Spark FFN over 1..64 tokens at the 2B shape, independent and correlated tokens (a common direction plus 30 % individual
+    noise: what a speculative-verify batch looks like), sparse against SPARK_DENSE_LOADS, 8 rotating weight sets, CUDA-graph
+    replay with launch overlap.  From five tokens on the library reads every row (tensor-core chunk kernels), so both columns are
+    the same kernels there.  Prints one JSON line."""
+    import torch
+
+    from paper_2506_06644_b200 import binding as S
+    from paper_2506_06644_b200 import synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7)
+    sh = synth.GEMMA2_2B
+
+    def w(rows, cols):
+        return (torch.randn(rows, cols, device=dev, generator=gen) * sh.d ** -0.5).to(torch.bfloat16)
+    sets = [(w(sh.d_ff, sh.r_ff), w(sh.d_ff, sh.d - sh.r_ff), w(sh.d_ff, sh.d)) for _ in range(8)]
+    rows = []
+    for B in (1, 2, 3, 4, 8, 16, 64):
+        ctx = S.SparkContext(0, max_batch=B, max_dff=sh.d_ff, max_d=sh.d)
+        ctx.set_launch_overlap(True)
+        for kind in ("independent", "correlated"):
+            x = torch.randn(B, sh.d, device=dev, generator=gen)
+            if kind == "correlated":
+                x = torch.randn(1, sh.d, device=dev, generator=gen) + 0.3 * x
+            x = x / x.pow(2).mean(dim=1, keepdim=True).sqrt()
+            y = torch.empty(B, sh.d, device=dev)
+            cnt = torch.zeros(B, dtype=torch.int32, device=dev)
+            idx = torch.zeros(B, sh.d_ff, dtype=torch.int32, device=dev)
+            S.spark_ffn_decode(ctx, x, B, *sets[0], S.SPARK_BF16, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, 0, y, None, cnt, idx)
+            torch.cuda.synchronize()
+            union = int(torch.unique(torch.cat([idx[b, : int(cnt[b])] for b in range(B)])).numel())
+            us = []
+            for flags in (0, S.SPARK_DENSE_LOADS):
+                def calls():
+                    for k1, k2, v in sets:
+                        S.spark_ffn_decode(ctx, x, B, k1, k2, v, S.SPARK_BF16, sh.d, sh.d_ff, sh.r_ff, sh.k_ff, flags, y, None, None, None)
+                side = torch.cuda.Stream()
+                with torch.cuda.stream(side):
+                    calls()
+                    side.synchronize()
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        calls()
+                torch.cuda.synchronize()
+                for _ in range(5):
+                    g.replay()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(30):
+                    g.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                us.append(e0.elapsed_time(e1) * 1e3 / (30 * len(sets)))
+            assert ctx.device_status() == S.SPARK_OK
+            rows.append({"tokens": B, "inputs": kind, "union_rows": union, "union_frac": union / sh.d_ff, "sparse_us": us[0],
+                         "dense_loads_us": us[1], "speedup": us[1] / us[0], "us_per_token": us[0] / B})
+            if B == 1:
+                break
+        ctx.close()
+    print(json.dumps({"study": "batch", "shape": "gemma2-2b FFN (d 2304, d_ff 9216, r 1024, k 737)", "rows": rows}), flush=True)
+
+
 def main():
     args = parse()
+    if args.study == "batch":
+        return batch_study(args)
     if args.impl == "reference":
         run_reference(args)
     else:
