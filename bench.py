@@ -685,8 +685,24 @@ def other_workloads(torch, S, peak, steps, warmup, with_oracle=True):
         assert ctx.device_status() == S.SPARK_OK
         nbytes8 = B * (sh.n_kv * L * (sh.r_attn + 4) + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn) * 2)
         entry(f"spark_attn_decode_fp8k (FP8 predictor slice), context {L}, batch {B}, k_attn {sh.k_attn}", us8, nbytes8)
+        # the whole cache in FP8 E4M3: the gathered rows of the selected tokens are halved too
+        def quant(t):
+            tf = t.float()
+            sc = tf.abs().amax(dim=-1).clamp_min(1e-30) / 448.0
+            return (tf / sc[..., None]).to(torch.float8_e4m3fn).view(torch.uint8), sc
+        q8kv = [(k1q, k1s) + quant(k2c) + quant(vc) for k1q, k1s, k2c, vc in q8c]
+
+        def calls8kv():
+            for rep in range(2):
+                for k1q, k1s, k2q, k2s, vq, vs in q8kv:
+                    S.spark_attn_decode_fp8kv(ctx, q, k1q, k1s, k2q, k2s, vq, vs, B, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, L, cl, 0, sh.k_attn,
+                                              0, o, None, None, None, 0)
+        us8kv = time_graph(calls8kv, 2 * nsets)
+        assert ctx.device_status() == S.SPARK_OK
+        nbytes8kv = B * (sh.n_kv * L * (sh.r_attn + 4) + sh.n_q * sh.k_attn * (2 * sh.hd - sh.r_attn + 8))
+        entry(f"spark_attn_decode_fp8kv (whole cache FP8), context {L}, batch {B}, k_attn {sh.k_attn}", us8kv, nbytes8kv)
         ctx.close()
-        del caches, q8c
+        del caches, q8c, q8kv
 
     # -- eight layers of the decoder at batch 8 (eight sequences, 8192-token synthetic caches each)
     B, L, nl = 8, 8192, 8

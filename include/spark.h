@@ -293,6 +293,14 @@ int spark_attn_decode_fp8k(spark_ctx* ctx, const float* q, const void* k1c, cons
                            const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags, float* o, float* theta,
                            int32_t* count, int32_t* idx, int64_t idx_cap, void* stream);
 
+/* The same with the WHOLE cache in FP8 E4M3: k1c, k2c, vc uint8 with the row scales k1s, k2s, vs [B][n_kv][cap] fp32 each (a cached
+ * row of a tensor stands for its scale times its stored values): the rows gathered for the selected tokens are halved as well.
+ * Not with SPARK_SHARED_CACHE.  Everything else as spark_attn_decode. */
+int spark_attn_decode_fp8kv(spark_ctx* ctx, const float* q, const void* k1c, const float* k1s, const void* k2c, const float* k2s,
+                            const void* vc, const float* vs, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap,
+                            const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags, float* o, float* theta,
+                            int32_t* count, int32_t* idx, int64_t idx_cap, void* stream);
+
 /* ---- dense GEMV (the projections the method leaves dense: Table "FLOPs per token") ----
  * y[b][n_out] = Wt[n_out][n_in] . x[b][n_in] (+ y_add[b][n_out] if y_add != NULL).
  * Wt of dtype wdtype, output-major; n_in % 8 == 0; 1 <= B <= 64.  y_add may equal y. */

@@ -31,7 +31,7 @@ EXPORTS = [
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
     "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
     "spark_set_wait_limit", "spark_debug_expect_arrivals", "spark_noalloc_status",
-    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill",
+    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill", "spark_attn_decode_fp8kv",
 ]
 
 
@@ -92,6 +92,8 @@ def lib() -> C.CDLL:
                                     vp, vp, vp, vp, i64, vp]),
         "spark_attn_decode_fp8k": (i32, [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
                                          vp, vp, vp, vp, i64, vp]),
+        "spark_attn_decode_fp8kv": (i32, [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, vp, i64, i64, i32,
+                                          vp, vp, vp, vp, i64, vp]),
         "spark_dense_gemv": (i32, [vp, vp, i64, vp, i32, i64, i64, vp, vp, vp]),
         "spark_stack_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64,
                                      vp, vp, i64, vp, vp]),
@@ -266,6 +268,13 @@ def spark_attn_decode_fp8k(ctx: SparkContext, q, k1c, k1s, k2c, vc, B, n_q, n_kv
     _check(lib().spark_attn_decode_fp8k(ctx.handle, _ptr(q), _ptr(k1c), _ptr(k1s), _ptr(k2c), _ptr(vc), B, n_q, n_kv, hd, r, cap,
                                         _ptr(ctx_len), window, k_attn, flags, _ptr(o), _ptr(theta), _ptr(count), _ptr(idx), idx_cap,
                                         _stream()), "spark_attn_decode_fp8k")
+
+
+def spark_attn_decode_fp8kv(ctx: SparkContext, q, k1c, k1s, k2c, k2s, vc, vs, B, n_q, n_kv, hd, r, cap, ctx_len, window, k_attn, flags,
+                            o, theta, count, idx, idx_cap):
+    _check(lib().spark_attn_decode_fp8kv(ctx.handle, _ptr(q), _ptr(k1c), _ptr(k1s), _ptr(k2c), _ptr(k2s), _ptr(vc), _ptr(vs), B, n_q, n_kv,
+                                         hd, r, cap, _ptr(ctx_len), window, k_attn, flags, _ptr(o), _ptr(theta), _ptr(count), _ptr(idx),
+                                         idx_cap, _stream()), "spark_attn_decode_fp8kv")
 
 
 def spark_dense_gemv(ctx: SparkContext, x, B, Wt, wdtype, n_in, n_out, y_add, y):

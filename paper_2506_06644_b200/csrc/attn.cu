@@ -59,6 +59,8 @@ struct AttnParams {
     int64_t cap;
     const int32_t* ctx_len;
     const float* k1s;  // nullable: k1c is FP8 E4M3 and k1s[B][n_kv][cap] holds one scale per cached row
+    const float* k2s;  // with KT = FP8 E4M3 (k2c and vc quantised too): their row scales, [B][n_kv][cap] each
+    const float* vs;
     const double* zs;  // nullable: Q(1 - k_attn / L_b) per sequence, precomputed by an earlier kernel
     int window, k_attn, dense;
     int seg_mask;      // cache segment of (sequence b, KV head g) = (b n_kv + g) & seg_mask: all ones, or n_kv - 1 when the B
@@ -589,24 +591,27 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             // the k2c and vc rows of up to four surviving tokens (tk: token inside the window), requested together
             auto gather4 = [&](const int (&tk)[4], const bool (&v)[4], const float (&av)[4]) {
                 Row8<KT> kw[2], vw[4];
+                [[maybe_unused]] float ksc[2] = {1.f, 1.f}, vsc[4] = {1.f, 1.f, 1.f, 1.f};      // row scales of an FP8 cache
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {      // half h reads the k2c rows of entries h and h + 2
                     const bool vv = half ? v[1 + 2 * i] : v[2 * i];
                     const int tt = half ? tk[1 + 2 * i] : tk[2 * i];
                     if (vv && hl < nc2) kw[i].load(k2base + static_cast<int64_t>(lo + tt) * d2, hl);
                     else kw[i].zero();
+                    if constexpr (sizeof(KT) == 1) ksc[i] = vv ? __ldg(p.k2s + cseg(seg) * p.cap + lo + tt) : 1.f;
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (v[i] && lane < ncv) vw[i].load(vbase + static_cast<int64_t>(lo + tk[i]) * hd, lane);
                     else vw[i].zero();
+                    if constexpr (sizeof(KT) == 1) vsc[i] = v[i] ? __ldg(p.vs + cseg(seg) * p.cap + lo + tk[i]) : 1.f;
                 }
                 float gt[4];
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     float wf[8];
                     kw[i].unpack(wf);
-                    const float gate = softplus(half_sum(dot8r(wf, q2)));
+                    const float gate = softplus(sizeof(KT) == 1 ? ksc[i] * half_sum(dot8r(wf, q2)) : half_sum(dot8r(wf, q2)));
                     gt[2 * i] = __shfl_sync(kFull, gate, 0);
                     gt[2 * i + 1] = __shfl_sync(kFull, gate, 16);
                 }
@@ -616,6 +621,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     const float pe = av[i] == -INFINITY ? 0.f : expf(av[i]);
                     l_w += pe;
                     wt[i] = pe * gt[i];         // unselected rows of the dense comparator get weight 0 * gate
+                    if constexpr (sizeof(KT) == 1) wt[i] *= vsc[i];
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
@@ -803,7 +809,7 @@ namespace spark {
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
-                int64_t idx_cap, const float* k1s, cudaStream_t st, PrefetchSpec pf) {
+                int64_t idx_cap, const float* k1s, cudaStream_t st, PrefetchSpec pf, const float* k2s, const float* vs) {
     if (ctx == nullptr || q == nullptr || k1c == nullptr || k2c == nullptr || vc == nullptr || ctx_len == nullptr ||
         o == nullptr)
         return SPARK_ERR_INVALID_ARG;
@@ -883,7 +889,11 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     p.hdr = ctx->hdr;
     p.trace = PhaseTrace{ctx->trace, ctx->trace_cap};
     const size_t smem = smem_fixed + (sel_list ? 3 * sc_bytes : (sc_smem ? sc_bytes : 0));
-    p.k1s = k1s;
+    p.k1s = k1s; p.k2s = k2s; p.vs = vs;
+    if (k2s != nullptr) {          // the whole cache in FP8: predictor slice, gate slice and values
+        if (k1s == nullptr || vs == nullptr) return SPARK_ERR_INVALID_ARG;
+        return launch_gq<__nv_fp8_e4m3, __nv_fp8_e4m3>(ctx, p, static_cast<int>(gq), smem, st);
+    }
     if (k1s != nullptr) return launch_gq<__nv_bfloat16, __nv_fp8_e4m3>(ctx, p, static_cast<int>(gq), smem, st);
     if (kvdtype == SPARK_BF16) return launch_gq<__nv_bfloat16, __nv_bfloat16>(ctx, p, static_cast<int>(gq), smem, st);
     return launch_gq<float, float>(ctx, p, static_cast<int>(gq), smem, st);
@@ -908,4 +918,15 @@ extern "C" int spark_attn_decode_fp8k(spark_ctx* ctx, const float* q, const void
     if (k1s == nullptr) return SPARK_ERR_INVALID_ARG;
     return attn_launch(ctx, q, k1c, k2c, vc, SPARK_BF16, B, n_q, n_kv, hd, r, cap, ctx_len, nullptr, window, k_attn, flags, o,
                        nullptr, theta, count, idx, idx_cap, k1s, static_cast<cudaStream_t>(stream));
+}
+
+// The whole cache in FP8 E4M3 with one fp32 scale per cached row and tensor (k1s, k2s, vs).
+extern "C" int spark_attn_decode_fp8kv(spark_ctx* ctx, const float* q, const void* k1c, const float* k1s, const void* k2c, const float* k2s,
+                                       const void* vc, const float* vs, int64_t B, int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap,
+                                       const int32_t* ctx_len, int64_t window, int64_t k_attn, int flags, float* o, float* theta, int32_t* count,
+                                       int32_t* idx, int64_t idx_cap, void* stream) {
+    if (k1s == nullptr || k2s == nullptr || vs == nullptr) return SPARK_ERR_INVALID_ARG;
+    if (flags & SPARK_SHARED_CACHE) return SPARK_ERR_UNSUPPORTED;
+    return attn_launch(ctx, q, k1c, k2c, vc, SPARK_BF16, B, n_q, n_kv, hd, r, cap, ctx_len, nullptr, window, k_attn, flags, o,
+                       nullptr, theta, count, idx, idx_cap, k1s, static_cast<cudaStream_t>(stream), PrefetchSpec{nullptr, 0}, k2s, vs);
 }

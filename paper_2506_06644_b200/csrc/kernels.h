@@ -58,7 +58,8 @@ int gemm_tc_launch(spark_ctx* ctx, const GemvArgs& a, cudaStream_t stream);
 int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c, const void* vc, int kvdtype, int64_t B,
                 int64_t n_q, int64_t n_kv, int64_t hd, int64_t r, int64_t cap, const int32_t* ctx_len, const double* zs,
                 int64_t window, int64_t k_attn, int flags, float* o, float* lsum, float* theta, int32_t* count, int32_t* idx,
-                int64_t idx_cap, const float* k1s, cudaStream_t st, PrefetchSpec pf = PrefetchSpec{nullptr, 0});
+                int64_t idx_cap, const float* k1s, cudaStream_t st, PrefetchSpec pf = PrefetchSpec{nullptr, 0},
+                const float* k2s = nullptr, const float* vs = nullptr);      // k2s / vs: row scales of an FP8 k2c / vc
 
 // Spark attention for a chunk of a prompt (T consecutive tokens of one sequence over one cache, bf16): predictor scores of
 // the whole chunk as one tcgen05 GEMM per KV head (attn_chunk.cu).  o is written normalised; lsum (nullable) receives 1 per

@@ -56,3 +56,41 @@ def test_fp8_predictor_slice_against_oracle(ctx, B, n_q, n_kv, hd, r, cap, lens,
     dense = run(ctx, a, k_attn, window, flags=S.SPARK_DENSE_LOADS)[1]
     assert np.array_equal(dense[1], out[1]) and np.array_equal(dense[2], out[2])
     np.testing.assert_allclose(dense[0], out[0], rtol=0, atol=2e-5 * max(1e-30, float(np.abs(out[0]).max())))
+
+
+def run_kv(ctx, a, k_attn, window=0, flags=0):
+    """The whole cache quantised: every tensor's rows as e4m3 with a row scale."""
+    B, n_kv, cap, r = a.k1c.shape
+    dev, deq = {}, {}
+    for name in ("k1c", "k2c", "vc"):
+        t = getattr(a, name)
+        bits, scale = synth.quantize_rows_e4m3(t.reshape(-1, t.shape[-1]))
+        deq[name] = (synth.e4m3_bits_to_f32(bits) * scale[:, None]).reshape(t.shape).astype(np.float32)
+        dev[name] = (torch.from_numpy(bits.reshape(t.shape)).cuda(), torch.from_numpy(scale.reshape(t.shape[:-1])).cuda())
+    q = torch.from_numpy(a.q).cuda()
+    cl = torch.from_numpy(a.ctx_len).cuda()
+    idx_cap = int(a.ctx_len.max())
+    o = torch.full((B, a.n_q, a.hd), float("nan"), device="cuda")
+    theta = torch.full((B, a.n_q), 9.0, device="cuda")
+    count = torch.full((B, a.n_q), -3, dtype=torch.int32, device="cuda")
+    idx = torch.full((B, a.n_q, idx_cap), -1, dtype=torch.int32, device="cuda")
+    S.spark_attn_decode_fp8kv(ctx, q, dev["k1c"][0], dev["k1c"][1], dev["k2c"][0], dev["k2c"][1], dev["vc"][0], dev["vc"][1], B, a.n_q, a.n_kv,
+                              a.hd, a.r, a.cap, cl, window, k_attn, flags, o, theta, count, idx, idx_cap)
+    torch.cuda.synchronize()
+    return dataclasses.replace(a, **deq), (o.cpu().numpy(), theta.cpu().numpy(), count.cpu().numpy(), idx.cpu().numpy())
+
+
+@pytest.mark.parametrize("B,n_q,n_kv,hd,r,cap,lens,k_attn,window", [
+    (1, 8, 4, 256, 128, 4096, [4096], 256, 0),
+    (3, 8, 4, 256, 128, 2048, [2048, 700, 33], 256, 512),
+    (8, 16, 8, 256, 128, 1024, [1024, 1000, 900, 512, 300, 100, 17, 1], 64, 0),
+    (2, 4, 4, 64, 32, 300, [300, 150], 16, 0),
+    (2, 16, 4, 256, 128, 500, [500, 77], 32, 128),
+])
+def test_fp8_whole_cache_against_oracle(ctx, B, n_q, n_kv, hd, r, cap, lens, k_attn, window):
+    a = synth.attn_inputs(B, n_q, n_kv, hd, r, cap, lens, "bf16", seed=14)
+    adeq, out = run_kv(ctx, a, k_attn, window)
+    compare(adeq, out, k_attn, window)
+    dense = run_kv(ctx, a, k_attn, window, flags=S.SPARK_DENSE_LOADS)[1]
+    assert np.array_equal(dense[1], out[1]) and np.array_equal(dense[2], out[2])
+    np.testing.assert_allclose(dense[0], out[0], rtol=0, atol=2e-5 * max(1e-30, float(np.abs(out[0]).max())))
