@@ -391,6 +391,16 @@ int spark_set_l2_prefetch(spark_ctx* ctx, int on);
  * critical path is bound by serial bookkeeping and grid-wide barriers).  Host-only setting. */
 int spark_set_fused_layer(spark_ctx* ctx, int on);
 
+/* Prompt chunks (SPARK_SHARED_CACHE with 16 to 64 tokens; Section 4.3 evaluates prompts in chunks): how the attention forms its
+ * output once the predictor scores of the chunk are known.  Either every (token, head) gathers the k2c / vc rows of its own
+ * selection, or -- when a KV head serves 32 or more (token, head) pairs of the chunk and the head sizes fit (hd 128 or 256,
+ * hd - r_attn 64 or 128) -- every cached row is read once per block and the selection of Eq. 7 becomes a mask on dense weights,
+ * both products on the tensor cores.  Same results up to rounding order.  mode 0: always the gather; 1 (default): the dense
+ * form where it measured faster on B200 (up to about 4096 visible rows: the window of a local layer, else the length
+ * spark_prefill knows, else the cache capacity); 2: the dense form wherever it serves the shape.  Host-only setting;
+ * SPARK_ERR_INVALID_ARG for another mode. */
+int spark_set_chunk_dense(spark_ctx* ctx, int mode);
+
 #ifdef __cplusplus
 }
 #endif

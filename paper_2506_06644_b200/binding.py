@@ -31,7 +31,7 @@ EXPORTS = [
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
     "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
     "spark_set_wait_limit", "spark_debug_expect_arrivals", "spark_noalloc_status",
-    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill", "spark_attn_decode_fp8kv",
+    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill", "spark_attn_decode_fp8kv", "spark_set_chunk_dense",
 ]
 
 
@@ -98,6 +98,7 @@ def lib() -> C.CDLL:
         "spark_stack_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64,
                                      vp, vp, i64, vp, vp]),
         "spark_set_fused_layer": (i32, [vp, i32]),
+        "spark_set_chunk_dense": (i32, [vp, i32]),
         "spark_prefill": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64, vp, i64, i64, i64, vp, vp, vp]),
         "spark_set_l2_prefetch": (i32, [vp, i32]),
         "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
@@ -186,11 +187,16 @@ class SparkContext:
         _check(lib().spark_set_wait_limit(self.handle, _stream(), cycles), "spark_set_wait_limit")
 
     def set_fused_layer(self, on: bool):
-        """One-token layer calls: the fused persistent kernel (default) or the kernel-per-step path."""
+        """One-token layer calls: the fused persistent kernel, or the kernel-per-step path (default)."""
         _check(lib().spark_set_fused_layer(self.handle, 1 if on else 0), "spark_set_fused_layer")
 
+    def set_chunk_dense(self, mode: int):
+        """Prompt chunks, second stage of the attention: 0 gather per (token, head), 1 masked dense products on the tensor
+        cores where they measured faster (default), 2 wherever they serve the shape."""
+        _check(lib().spark_set_chunk_dense(self.handle, int(mode)), "spark_set_chunk_dense")
+
     def set_l2_prefetch(self, on: bool):
-        """Kernels of a one-token layer call ask L2 for the next kernel's weights (default on)."""
+        """Kernels of a one-token layer call ask L2 for the next kernel's weights (default off: it measured slower)."""
         _check(lib().spark_set_l2_prefetch(self.handle, 1 if on else 0), "spark_set_l2_prefetch")
 
     def debug_expect_arrivals(self, extra: int):

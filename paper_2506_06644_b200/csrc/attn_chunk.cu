@@ -46,6 +46,12 @@ struct ChunkParams {
     __nv_bfloat16* qlo;
     float* S;                  // [n_kv][kColMax][scap]
     int64_t scap;              // column stride of S: cap + 32, so that the columns' lines do not all fall on the same slices
+    // dense second stage (masked weights x value rows on the tensor cores) only
+    __nv_bfloat16* q2hi;       // [n_kv][kColMax][hd - r]: the gate's query part as two bf16 terms
+    __nv_bfloat16* q2lo;
+    float4* colinfo;           // [n_kv][kColMax] = theta, maximum of the survivors' scores, lo, n (the last two as int bits)
+    float* zsum;               // [T][n_q] sum of exp(s - max) over the survivors
+    int dense;
     WsHeader* hdr;
 };
 
@@ -71,7 +77,7 @@ __global__ void __launch_bounds__(128) attn_chunk_prep_kernel(const ChunkParams 
                                          : (p.k_attn >= L ? 0.0 : -normcdfinv(static_cast<double>(p.k_attn) / static_cast<double>(L)));
         }
     }
-    if (col >= p.ncolp) return;                 // rows the operand boxes never touch
+    if (col >= (p.dense ? ((p.ncol + 63) & ~63) : p.ncolp)) return;                 // rows the operand boxes never touch
     __nv_bfloat16* hi = p.qhi + (static_cast<int64_t>(g) * kColMax + col) * p.r;
     __nv_bfloat16* lo = p.qlo + (static_cast<int64_t>(g) * kColMax + col) * p.r;
     const int t = col / p.gq, hq = col - t * p.gq;
@@ -81,6 +87,18 @@ __global__ void __launch_bounds__(128) attn_chunk_prep_kernel(const ChunkParams 
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         hi[i] = h;
         lo[i] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
+    if (p.dense) {
+        const int d2 = p.hd - p.r;
+        __nv_bfloat16* h2 = p.q2hi + (static_cast<int64_t>(g) * kColMax + col) * d2;
+        __nv_bfloat16* l2 = p.q2lo + (static_cast<int64_t>(g) * kColMax + col) * d2;
+        for (int i = tid; i < d2; i += 128) {
+            float v = 0.f;
+            if (col < p.ncol) v = p.q[(static_cast<int64_t>(t) * p.n_q + g * p.gq + hq) * p.hd + p.r + i];
+            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+            h2[i] = h;
+            l2[i] = __float2bfloat16_rn(v - __bfloat162float(h));
+        }
     }
 }
 
@@ -562,6 +580,449 @@ __global__ void __launch_bounds__(kSelThreads, REGS ? 3 : 4) attn_chunk_select_k
     }
 }
 
+
+// ---- dense second stage ------------------------------------------------------------------------------------------------------
+// With many queries per KV head the union of their selections is most of the cache, and the per-query gather above reads
+// every selected k2c / vc row once per query out of L2.  The dense form reads every cached row once per block instead and
+// leaves the selection to a mask:  o[c] = sum_j w[c][j] v[j] / Z[c],  w[c][j] = [s1 > theta_c] exp(s1 - m_c) softplus(q2_c . k2_j),
+// both products on the tensor cores.  Three kernels:
+//   stats  one block per (token, query head): theta (Eq. 10/11) from the column of predictor scores, the maximum m of the
+//          survivors' scores, Z = sum of exp(s1 - m) over them, their number; clears the column's output row
+//   dense  one block per (KV head, 64 columns, share of the cached rows), per tile of 128 rows:
+//            S2 = k2c . Q2^T                      (tcgen05, M = 128 rows, N = 64 columns, K = hd - r; Q2 as two bf16 terms)
+//            W  = mask . exp(S1 - m) . softplus(S2)   (eight epilogue warps: tensor memory -> registers -> two bf16 terms in
+//                                                  shared memory, written in the swizzled K-major layout the MMA reads)
+//            O^T += V^T . W                       (tcgen05, M = 128 of the hd value columns, N = 64, K = 128 rows; V^T is the vc
+//                                                  tile as it lands, read MN-major)
+//          the accumulated O^T leaves as warp-wide reductions into o (a warp's 32 lanes are 32 consecutive floats of a row)
+//   norm   (only without lsum) o /= Z
+// Cached rows at or beyond the last token of the chunk may hold anything: their weights are zero by selection, and their vc
+// rows are cleared in shared memory before the product (0 x NaN would poison the sum).
+constexpr int kDN = 64;                          // columns per dense block
+constexpr int kDSlotBytes = 32768;               // a k2c tile (<= 2 K chunks x 128 rows x 128 B) or 128 value columns of a vc tile
+constexpr int kDSlots = 4;
+constexpr int kDQBytes = 2 * 2 * kDN * 128;      // Q2: (hi, lo) x K chunks x 64 rows x 128 B
+constexpr int kDWBytes = 2 * 2 * kDN * 128;      // W:  (hi, lo) x 2 chunks of 64 cached rows x 64 rows x 128 B; two such buffers
+constexpr uint32_t kDCols = 256;                 // tensor memory: two S2 accumulators of 64 columns, two O^T tiles of 64
+constexpr int kDEpiWarps = 16;
+constexpr int kDThreads = 64 + kDEpiWarps * 32;  // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..17: weights / output
+
+struct DenseShared {
+    unsigned long long full[kDSlots], empty[kDSlots];
+    unsigned long long q_full, d1_full[2], d1_empty[2], w_full[2], w_empty[2], d2_full;
+    uint32_t tmem;
+    int abort_flag;
+    int lo_min, n_max, n_all, lo_max, n_min;
+    float4 info[kDN];
+    float* orow[kDN];            // output row of each of the block's columns (nullptr: no such column)
+};
+
+__global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams p) {
+    __shared__ double part[8][2];
+    __shared__ float redf[8];
+    __shared__ int redi[8];
+    __shared__ float s_th, s_mx;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t = blockIdx.x / p.n_q, h = blockIdx.x - t * p.n_q;
+    const int g = h / p.gq, col = t * p.gq + (h - g * p.gq);
+    dep_wait();
+    dep_trigger();
+    const int lo = p.range[2 * t], n = p.range[2 * t + 1], L = n - lo;
+    const float* scol = p.S + (static_cast<int64_t>(g) * kColMax + col) * p.scap;
+    if (tid < p.hd) p.o[static_cast<int64_t>(blockIdx.x) * p.hd + tid] = 0.f;       // the dense kernel adds into it
+    constexpr int kKeep = 32;
+    const bool kept = L <= kKeep * 256;
+    float keep[kKeep];
+    if (kept) {
+#pragma unroll
+        for (int u = 0; u < kKeep; ++u) {
+            const int j = lo + 256 * u + tid;
+            keep[u] = j < n ? __ldcg(scol + j) : -INFINITY;
+        }
+    }
+    float th = -INFINITY;
+    if (p.k_attn < L) {
+        // sums around the column's first value (keeps the fp32 partial sums accurate when |mean| >> std); fp64 above
+        const float c0 = __ldcg(scol + lo);
+        float f1 = 0.f, f2 = 0.f;
+        if (kept) {
+#pragma unroll
+            for (int u = 0; u < kKeep; ++u) {
+                const float d = lo + 256 * u + tid < n ? keep[u] - c0 : 0.f;
+                f1 += d;
+                f2 = fmaf(d, d, f2);
+            }
+        } else {
+            for (int j = lo + tid; j < n; j += 256) {
+                const float d = __ldcg(scol + j) - c0;
+                f1 += d;
+                f2 = fmaf(d, d, f2);
+            }
+        }
+        const double s1 = warp_sum_f64(static_cast<double>(f1)), s2 = warp_sum_f64(static_cast<double>(f2));
+        if (lane == 0) {
+            part[warp][0] = s1;
+            part[warp][1] = s2;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            double a = 0.0, b = 0.0;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                a += part[w][0];
+                b += part[w][1];
+            }
+            const double dm = a / static_cast<double>(L);                  // mean - c0
+            const double var = (b - a * dm) / static_cast<double>(L - 1);
+            s_th = static_cast<float>(static_cast<double>(c0) + dm + sqrt(var > 0.0 ? var : 0.0) * p.zt[t]);
+        }
+        __syncthreads();
+        th = s_th;
+    }
+    // the survivors: their number and their maximum, then the sum of their exponentials
+    float mx = -INFINITY;
+    int cnt = 0;
+    if (kept) {
+#pragma unroll
+        for (int u = 0; u < kKeep; ++u)
+            if (keep[u] > th) {
+                mx = fmaxf(mx, keep[u]);
+                ++cnt;
+            }
+    } else {
+        for (int j = lo + tid; j < n; j += 256) {
+            const float v = __ldcg(scol + j);
+            if (v > th) {
+                mx = fmaxf(mx, v);
+                ++cnt;
+            }
+        }
+    }
+    mx = warp_max(mx);
+    cnt = warp_sum_int(cnt);
+    if (lane == 0) {
+        redf[warp] = mx;
+        redi[warp] = cnt;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float m = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) m = fmaxf(m, redf[w]);
+        s_mx = m;
+    }
+    int total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) total += redi[w];
+    __syncthreads();
+    mx = s_mx;
+    float es = 0.f;
+    if (kept) {
+#pragma unroll
+        for (int u = 0; u < kKeep; ++u)
+            if (keep[u] > th) es += __expf(keep[u] - mx);
+    } else {
+        for (int j = lo + tid; j < n; j += 256) {
+            const float v = __ldcg(scol + j);
+            if (v > th) es += __expf(v - mx);
+        }
+    }
+    es = warp_sum(es);
+    if (lane == 0) redf[warp] = es;
+    __syncthreads();
+    if (tid == 0) {
+        float z = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) z += redf[w];
+        p.colinfo[g * kColMax + col] = make_float4(th, mx, __int_as_float(lo), __int_as_float(n));
+        p.zsum[blockIdx.x] = total > 0 ? z : 0.f;
+        if (p.lsum != nullptr) p.lsum[blockIdx.x] = total > 0 ? z : 0.f;
+        if (p.theta != nullptr) p.theta[blockIdx.x] = th;
+        if (p.count != nullptr) p.count[blockIdx.x] = total;
+    }
+}
+
+__global__ void __launch_bounds__(256) attn_chunk_norm_kernel(const ChunkParams p) {
+    dep_wait();
+    dep_trigger();
+    const float z = p.zsum[blockIdx.x];
+    if (threadIdx.x < p.hd) {
+        float* o = p.o + static_cast<int64_t>(blockIdx.x) * p.hd + threadIdx.x;
+        *o = z > 0.f ? *o / z : 0.f;
+    }
+}
+
+__global__ void __launch_bounds__(kDThreads, 1)
+attn_chunk_dense_kernel(const ChunkParams p, const __grid_constant__ CUtensorMap map_k2, const __grid_constant__ CUtensorMap map_v,
+                        const __grid_constant__ CUtensorMap map_q2hi, const __grid_constant__ CUtensorMap map_q2lo, int nsplit) {
+    extern __shared__ unsigned char tc_raw[];
+    __shared__ DenseShared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int d2 = p.hd - p.r, nk2 = d2 / kChunk, nvh = p.hd / 128;
+    const int ncg = (p.ncol + kDN - 1) / kDN;
+    const int grp = blockIdx.x / nsplit, part = blockIdx.x - grp * nsplit;
+    const int g = grp / ncg, cg = grp - g * ncg;
+    const int col0 = cg * kDN;                                  // first column of this block within the KV head
+    if (tid == 0) {
+        for (int s = 0; s < kDSlots; ++s) {
+            mbar_init(smem_addr(&sh.full[s]), 1u);
+            mbar_init(smem_addr(&sh.empty[s]), 1u);
+        }
+        mbar_init(smem_addr(&sh.q_full), 1u);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_addr(&sh.d1_full[b]), 1u);
+            mbar_init(smem_addr(&sh.d1_empty[b]), 1u);
+            mbar_init(smem_addr(&sh.w_full[b]), 1u);
+            mbar_init(smem_addr(&sh.w_empty[b]), 1u);
+        }
+        mbar_init(smem_addr(&sh.d2_full), 1u);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_addr(&sh.tmem), kDCols);
+    dep_wait();                  // everything read here comes from the kernels ahead
+    dep_trigger();
+    if (tid < kDN) {
+        const int col = col0 + tid;
+        sh.info[tid] = col < p.ncol ? p.colinfo[g * kColMax + col] : make_float4(INFINITY, 0.f, __int_as_float(0), __int_as_float(0));
+        const int t = col / p.gq, h = g * p.gq + (col - t * p.gq);
+        sh.orow[tid] = col < p.ncol ? p.o + (static_cast<int64_t>(t) * p.n_q + h) * p.hd : nullptr;
+    }
+    if (tid == 0) {
+        // rows any of this block's columns may see, and the end of what the chunk has written
+        int lo_min = 0x7fffffff, n_max = 0, n_all = 0, lo_max = 0, n_min = 0x7fffffff;
+        for (int t = 0; t < p.T; ++t) n_all = max(n_all, p.range[2 * t + 1]);
+        const int c_end = min(p.ncol, col0 + kDN);
+        for (int t = col0 / p.gq; t <= (c_end - 1) / p.gq; ++t) {
+            lo_min = min(lo_min, p.range[2 * t]);
+            n_max = max(n_max, p.range[2 * t + 1]);
+            lo_max = max(lo_max, p.range[2 * t]);
+            n_min = min(n_min, p.range[2 * t + 1]);
+        }
+        sh.lo_max = lo_max;
+        sh.n_min = n_min;
+        sh.lo_min = lo_min;
+        sh.n_max = n_max;
+        sh.n_all = n_all;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t base = (smem_addr(tc_raw) + 1023u) & ~1023u;
+    const uint32_t qbase = base + kDSlots * kDSlotBytes, wbase = qbase + kDQBytes;
+    unsigned char* wgen = tc_raw + (base - smem_addr(tc_raw)) + kDSlots * kDSlotBytes + kDQBytes;      // W, generic address
+    unsigned char* ring_gen = tc_raw + (base - smem_addr(tc_raw));
+    const uint32_t tmem = sh.tmem;
+    volatile int* abort_flag = &sh.abort_flag;
+    const int tile_lo = sh.lo_min / 128, tile_hi = (sh.n_max + 127) / 128, nt_all = max(0, tile_hi - tile_lo);
+    const int ta = tile_lo + static_cast<int>(static_cast<int64_t>(part) * nt_all / nsplit);
+    const int tb = tile_lo + static_cast<int>(static_cast<int64_t>(part + 1) * nt_all / nsplit);
+    const int n = tb - ta;                                      // this block's tiles
+    // ring items in the order both ends walk them: K(0), then per tile i: K(i + 1) if there is one, V(i, 0..nvh-1)
+    if (warp == 0) {
+        if (lane == 0 && n > 0) {
+            tma_prefetch_desc(&map_k2);
+            tma_prefetch_desc(&map_v);
+            tma_prefetch_desc(&map_q2hi);
+            tma_prefetch_desc(&map_q2lo);
+            {
+                const uint32_t bar = smem_addr(&sh.q_full);
+                mbar_expect_tx(bar, static_cast<uint32_t>(2 * nk2) * kDN * 128);
+                for (int kc = 0; kc < nk2; ++kc) {
+                    tma_load_2d(qbase + kc * (kDN * 128), &map_q2hi, bar, kc * kChunk, g * kColMax + col0);
+                    tma_load_2d(qbase + (nk2 + kc) * (kDN * 128), &map_q2lo, bar, kc * kChunk, g * kColMax + col0);
+                }
+            }
+            int it = 0;
+            bool ok = true;
+            auto slot_for = [&](int item) -> bool {             // waits until the ring slot of `item` is free
+                if (item >= kDSlots && !mbar_wait(smem_addr(&sh.empty[item % kDSlots]), ((item / kDSlots) & 1) ^ 1, abort_flag)) return false;
+                return true;
+            };
+            auto load_k = [&](int i) {
+                if (!(ok = ok && slot_for(it))) return;
+                const uint32_t bar = smem_addr(&sh.full[it % kDSlots]), dst = base + (it % kDSlots) * kDSlotBytes;
+                mbar_expect_tx(bar, static_cast<uint32_t>(nk2) * 128 * 128);
+                for (int kc = 0; kc < nk2; ++kc)
+                    tma_load_2d(dst + kc * (128 * 128), &map_k2, bar, kc * kChunk, static_cast<int>(g * p.cap + (ta + i) * 128));
+                ++it;
+            };
+            auto load_v = [&](int i, int hh) {
+                if (!(ok = ok && slot_for(it))) return;
+                const uint32_t bar = smem_addr(&sh.full[it % kDSlots]), dst = base + (it % kDSlots) * kDSlotBytes;
+                mbar_expect_tx(bar, 2u * 128 * 128);
+                for (int b = 0; b < 2; ++b)
+                    tma_load_2d(dst + b * (128 * 128), &map_v, bar, hh * 128 + b * kChunk, static_cast<int>(g * p.cap + (ta + i) * 128));
+                ++it;
+            };
+            load_k(0);
+            for (int i = 0; i < n && ok; ++i) {
+                if (i + 1 < n) load_k(i + 1);
+                for (int hh = 0; hh < nvh; ++hh) load_v(i, hh);
+            }
+            if (*abort_flag != 0) {            // let the copies in flight land before the block goes
+                for (int i = max(0, it - kDSlots); i < it; ++i) {
+                    const long long c0 = clock64();
+                    while (!mbar_try(smem_addr(&sh.full[i % kDSlots]), (i / kDSlots) & 1))
+                        if (clock64() - c0 > kTcSpinLimit) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && n > 0) {
+            const uint32_t idesc1 = instr_desc(128, kDN, false), idesc2 = instr_desc(128, kDN, true);
+            int it = 0;
+            bool ok = mbar_wait(smem_addr(&sh.q_full), 0u, abort_flag);
+            auto gemm1 = [&](int i) {          // S2 of tile i into accumulator i & 1
+                const int b = i & 1;
+                if (i >= 2) ok = ok && mbar_wait(smem_addr(&sh.d1_empty[b]), ((i >> 1) & 1) ^ 1, abort_flag);
+                ok = ok && mbar_wait(smem_addr(&sh.full[it % kDSlots]), (it / kDSlots) & 1, abort_flag);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t a0 = base + (it % kDSlots) * kDSlotBytes;
+                for (int tt = 0; tt < 2; ++tt)
+                    for (int kc = 0; kc < nk2; ++kc)
+#pragma unroll
+                        for (int j = 0; j < kChunk / 16; ++j)
+                            umma_bf16(tmem + b * kDN, smem_desc(a0 + kc * (128 * 128) + 32 * j, 0u, 1024u),
+                                      smem_desc(qbase + (tt * nk2 + kc) * (kDN * 128) + 32 * j, 0u, 1024u), idesc1,
+                                      (tt == 0 && kc == 0 && j == 0) ? 0u : 1u);
+                umma_commit(smem_addr(&sh.empty[it % kDSlots]));
+                umma_commit(smem_addr(&sh.d1_full[b]));
+                ++it;
+            };
+            gemm1(0);
+            for (int i = 0; i < n && ok; ++i) {
+                if (i + 1 < n) gemm1(i + 1);
+                ok = ok && mbar_wait(smem_addr(&sh.w_full[i & 1]), static_cast<uint32_t>((i >> 1) & 1), abort_flag);
+                for (int hh = 0; hh < nvh && ok; ++hh) {
+                    ok = mbar_wait(smem_addr(&sh.full[it % kDSlots]), (it / kDSlots) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t v0 = base + (it % kDSlots) * kDSlotBytes;
+                    for (int tt = 0; tt < 2; ++tt)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)          // 16 cached rows per step: V^T MN-major (8-row groups 1024 B apart, next 64 columns 16 KB on)
+                            umma_bf16(tmem + 2 * kDN + hh * kDN, smem_desc(v0 + j * 2048, 128 * 128, 1024u),
+                                      smem_desc(wbase + (i & 1) * kDWBytes + (tt * 2 + (j >> 2)) * (kDN * 128) + 32 * (j & 3), 0u, 1024u), idesc2,
+                                      (i == 0 && tt == 0 && j == 0) ? 0u : 1u);
+                    umma_commit(smem_addr(&sh.empty[it % kDSlots]));
+                    ++it;
+                }
+                if (ok) umma_commit(smem_addr(&sh.w_empty[i & 1]));
+            }
+            if (ok) umma_commit(smem_addr(&sh.d2_full));
+        }
+    } else if (n > 0) {
+        // sixteen warps: four per tensor-memory lane quadrant, each with sixteen of the 64 columns
+        const int q = warp & 3, part4 = (warp - 2) >> 2, cbase = 16 * part4;
+        const int n_all = sh.n_all;
+        bool ok = true;
+        const int row = q * 32 + lane;                              // this thread's row of every tile
+        const int etid = tid - 64;                                  // 0..511 among the sixteen warps
+        // predictor scores of the thread's row for its 16 columns, requested one tile ahead
+        float s1n[16];
+        auto request_s1 = [&](int i) {
+            const int tok = (ta + i) * 128 + row;
+            const float* srow = p.S + (static_cast<int64_t>(g) * kColMax + col0 + cbase) * p.scap + tok;
+#pragma unroll
+            for (int c = 0; c < 16; ++c)
+                s1n[c] = (tok < n_all && col0 + cbase + c < p.ncol) ? __ldcg(srow + static_cast<int64_t>(c) * p.scap) : -INFINITY;
+        };
+        request_s1(0);
+        for (int i = 0; i < n && ok; ++i) {
+            const int b = i & 1;
+            const int tok = (ta + i) * 128 + row;
+            float s1[16];
+#pragma unroll
+            for (int c = 0; c < 16; ++c) s1[c] = s1n[c];
+            if (i >= 2) ok = __all_sync(kFull, mbar_wait(smem_addr(&sh.w_empty[b]), static_cast<uint32_t>(((i >> 1) & 1) ^ 1), abort_flag));
+            if (!ok) break;
+            // W starts as zeros (64 bytes per thread); only the rows that pass are written below
+            {
+                uint4* wz = reinterpret_cast<uint4*>(wgen + b * kDWBytes) + etid * 4;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) wz[u] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            ok = __all_sync(kFull, mbar_wait(smem_addr(&sh.d1_full[b]), (i >> 1) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            float s2[16];
+            tmem_ld16(tmem + b * kDN + cbase + (static_cast<uint32_t>(q * 32) << 16), s2);
+            asm volatile("bar.sync 1, %0;" ::"n"(kDEpiWarps * 32) : "memory");      // the zeros are in place
+            // W[column][row] as two bf16 terms, K-major with the 128-byte swizzle: row `c` of a 64-row chunk holds 64 cached
+            // rows; its 16-byte unit u sits at u ^ (c % 8)
+            unsigned char* wchunk = wgen + b * kDWBytes + (row >> 6) * (kDN * 128);
+            const int unit = (row & 63) >> 3, within = (row & 7) * 2;
+            // a tile that every column of the block sees whole needs no range test per element
+            const bool inner = (ta + i) * 128 >= sh.lo_max && (ta + i) * 128 + 128 <= sh.n_min;
+            // no branch per element: the sixteen columns' arithmetic interleaves (a branch per column left every warp waiting
+            // on its own chain of dependent instructions: 2.4 us per tile instead of 1)
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                const float4 ci = sh.info[cbase + c];
+                const bool on = s1[c] > ci.x && (inner || (tok >= __float_as_int(ci.z) && tok < __float_as_int(ci.w)));
+                // softplus(a) = max(a, 0) + log(1 + e), e = exp(-|a|): the hardware logarithm of 1 + e loses e below 1e-4
+                const float e = __expf(-fabsf(s2[c]));
+                const float l1p = e < 1e-4f ? e * (1.f - 0.5f * e) : __logf(1.f + e);
+                const float w = __expf(fminf(s1[c] - ci.y, 0.f)) * (fmaxf(s2[c], 0.f) + l1p);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(w);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(w - __bfloat162float(hi));
+                const int cr = cbase + c;
+                const int off = (cr >> 3) * 1024 + (cr & 7) * 128 + ((unit ^ (cr & 7)) << 4) + within;
+                if (on) {                   // three rows in a hundred
+                    *reinterpret_cast<__nv_bfloat16*>(wchunk + off) = hi;
+                    *reinterpret_cast<__nv_bfloat16*>(wchunk + 2 * (kDN * 128) + off) = lo;
+                }
+            }
+            // value rows nobody has written yet: cleared once they have landed
+            if ((ta + i) * 128 + 128 > n_all && tok >= n_all) {
+                // items before V(i, 0): K(0), and for every earlier tile its K(next) and its nvh value pieces, then K(i + 1)
+                for (int hh = part4; hh < nvh; hh += 4) {
+                    const int item = 1 + i * (1 + nvh) + (i + 1 < n ? 1 : 0) + hh;
+                    if (mbar_wait(smem_addr(&sh.full[item % kDSlots]), (item / kDSlots) & 1, abort_flag)) {
+                        unsigned char* vs = ring_gen + (item % kDSlots) * kDSlotBytes + row * 128;
+#pragma unroll
+                        for (int bx = 0; bx < 2; ++bx)
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) *reinterpret_cast<uint4*>(vs + bx * (128 * 128) + 16 * u) = make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+            }
+            if (i + 1 < n) request_s1(i + 1);          // in flight across the hand-over below and the next tile's waits
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // generic writes -> the tensor core's reads
+            tc_fence_before();
+            asm volatile("bar.sync 1, %0;" ::"n"(kDEpiWarps * 32) : "memory");
+            if (tid == 64) {
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&sh.w_full[b])) : "memory");
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&sh.d1_empty[b])) : "memory");
+            }
+        }
+        // the accumulated O^T: lane = value column; a warp takes sixteen (token, head) columns of one or two value tiles
+        if (ok && __all_sync(kFull, mbar_wait(smem_addr(&sh.d2_full), 0u, abort_flag))) {
+            tc_fence_after();
+            for (int hh = 0; hh < nvh; ++hh) {
+                float v[16];
+                tmem_ld16(tmem + 2 * kDN + hh * kDN + cbase + (static_cast<uint32_t>(q * 32) << 16), v);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    float* orow = sh.orow[cbase + c];
+                    if (orow != nullptr) atomicAdd(orow + hh * 128 + q * 32 + lane, v[c]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_free(tmem, kDCols);
+    }
+    if (tid == 0 && sh.abort_flag != 0) atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_TIMEOUT);
+}
+
 }  // namespace
 
 namespace spark {
@@ -580,6 +1041,18 @@ int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const voi
     const size_t q_b = round_up(static_cast<size_t>(n_kv) * kColMax * r * 2, 1024);
     const size_t s_b = round_up(static_cast<size_t>(n_kv) * kColMax * (cap + 32) * 4, 1024);
     if (ctx->scratch == nullptr || ctx->scratch_bytes < kAttnCellBytes + small_b + 2 * q_b + s_b) return SPARK_ERR_WORKSPACE;
+    // the dense second stage: enough columns per KV head that reading every row once beats gathering per query
+    const size_t q2_b = round_up(static_cast<size_t>(n_kv) * kColMax * d2 * 2, 1024);
+    const size_t info_b = round_up(static_cast<size_t>(n_kv) * kColMax * sizeof(float4) + static_cast<size_t>(T) * n_q * 4, 1024);
+    const size_t smem_dense = static_cast<size_t>(kDSlots) * kDSlotBytes + kDQBytes + 2 * kDWBytes + 1024;
+    // measured at the 2B head shape with 64-token chunks: ahead of the gather up to about 4096 visible rows (31 against 36 us
+    // at 2048), level at 6000, behind beyond (its work grows with the rows, the gather's with k_attn); the caller's hint of
+    // the current length decides, else the capacity
+    int64_t rows_hint = ctx->len_hint > 0 ? ctx->len_hint : cap;
+    if (window > 0 && window + T < rows_hint) rows_hint = window + T;          // a local layer sees no more than its window
+    const bool dense = (ctx->chunk_dense == 2 || (ctx->chunk_dense == 1 && rows_hint <= 4160)) && T * gq >= 32 && (d2 == 64 || d2 == 128) && (hd == 128 || hd == 256) &&
+                       ctx->scratch_bytes >= kAttnCellBytes + small_b + 2 * q_b + s_b + 2 * q2_b + info_b &&
+                       smem_dense + sizeof(DenseShared) + 64 <= static_cast<size_t>(ctx->max_smem_optin);
     const size_t smem_scores = static_cast<size_t>(kChunkStages) * kChunkStageBytes + 1024;
     if (smem_scores + sizeof(ChunkShared) + 64 > static_cast<size_t>(ctx->max_smem_optin)) return SPARK_ERR_WORKSPACE;
 
@@ -600,7 +1073,12 @@ int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const voi
     p.range = reinterpret_cast<int*>(w + static_cast<size_t>(T) * sizeof(double)); w += small_b;
     p.qhi = reinterpret_cast<__nv_bfloat16*>(w); w += q_b;
     p.qlo = reinterpret_cast<__nv_bfloat16*>(w); w += q_b;
-    p.S = reinterpret_cast<float*>(w);
+    p.S = reinterpret_cast<float*>(w); w += s_b;
+    p.dense = dense ? 1 : 0;
+    p.q2hi = reinterpret_cast<__nv_bfloat16*>(w); w += q2_b;
+    p.q2lo = reinterpret_cast<__nv_bfloat16*>(w); w += q2_b;
+    p.colinfo = reinterpret_cast<float4*>(w);
+    p.zsum = reinterpret_cast<float*>(w + static_cast<size_t>(n_kv) * kColMax * sizeof(float4));
     p.hdr = ctx->hdr;
 
     CUtensorMap m_k1, m_qhi, m_qlo;
@@ -620,6 +1098,33 @@ int attn_chunk_launch(spark_ctx* ctx, const float* q, const void* k1c, const voi
         void* args[] = {&p, &m_k1, &m_qhi, &m_qlo};
         if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_scores_kernel), static_cast<unsigned>(ctx->num_sms), kChunkThreads, smem_scores, stream, false, args) != cudaSuccess)
             return SPARK_ERR_CUDA;
+    }
+    if (dense) {
+        CUtensorMap m_k2, m_v, m_q2hi, m_q2lo;
+        if (!make_map(&m_k2, k2c, n_kv * cap, d2, d2, 128, true) || !make_map(&m_v, vc, n_kv * cap, hd, hd, 128, true) ||
+            !make_map(&m_q2hi, p.q2hi, n_kv * kColMax, d2, d2, kDN, false) || !make_map(&m_q2lo, p.q2lo, n_kv * kColMax, d2, d2, kDN, false))
+            return SPARK_ERR_WORKSPACE;
+        if (cudaFuncSetAttribute(attn_chunk_dense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_dense)) != cudaSuccess)
+            return SPARK_ERR_CUDA;
+        {
+            void* args[] = {&p};
+            if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_stats_kernel), static_cast<unsigned>(T * n_q), 256, 0, stream, false, args) != cudaSuccess)
+                return SPARK_ERR_CUDA;
+        }
+        const int groups = static_cast<int>(n_kv) * ((p.ncol + kDN - 1) / kDN);
+        int nsplit = ctx->num_sms / groups;
+        if (nsplit < 1) nsplit = 1;
+        {
+            void* args[] = {&p, &m_k2, &m_v, &m_q2hi, &m_q2lo, &nsplit};
+            if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_dense_kernel), static_cast<unsigned>(groups * nsplit), kDThreads, smem_dense, stream, false, args) != cudaSuccess)
+                return SPARK_ERR_CUDA;
+        }
+        if (lsum == nullptr) {
+            void* args[] = {&p};
+            if (launch_kernel(ctx, reinterpret_cast<const void*>(attn_chunk_norm_kernel), static_cast<unsigned>(T * n_q), 256, 0, stream, false, args) != cudaSuccess)
+                return SPARK_ERR_CUDA;
+        }
+        return SPARK_OK;
     }
     {
         void* args[] = {&p};

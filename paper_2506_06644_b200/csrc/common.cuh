@@ -69,6 +69,8 @@ struct spark_ctx {
     const void* next_wqkv;   // set by spark_stack_decode around a layer call: the QKV matrix of the layer after it (or nullptr)
     int l2_prefetch;         // one-token layer calls ask L2 for the next kernel's weights (spark_set_l2_prefetch)
     int fused;               // one token: take the fused layer kernel when it serves the shape (spark_set_fused_layer)
+    int chunk_dense;         // prompt chunks: second stage of the attention as masked dense products: 0 never, 1 where it measured faster, 2 wherever it serves the shape (spark_set_chunk_dense)
+    int64_t len_hint;        // rows of the cache in use after the current call, when the caller knows them on the host (spark_prefill); 0 = unknown
     int debug_extra_arrivals;   // test hook: the one-token kernels wait for this many arrivals more than blocks exist
 };
 

@@ -559,6 +559,8 @@ extern "C" int spark_ffn_decode_noalloc(const float* x, int64_t B, const void* K
     local.overlap = 0;
     local.wait_kcycles = 0;
     local.fused = 0;
+    local.chunk_dense = 0;
+    local.len_hint = 0;
     local.l2_prefetch = 0;
     local.next_wqkv = nullptr;
     local.debug_extra_arrivals = 0;

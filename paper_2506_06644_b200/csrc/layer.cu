@@ -792,10 +792,15 @@ extern "C" int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const
         int n = static_cast<int>(T), first = static_cast<int>(start + c0 + 1);
         void* args[] = {&len_buf, &n, &first};
         if (launch_kernel(ctx, reinterpret_cast<const void*>(chunk_lengths_kernel), 1u, 64u, 0, st, false, args) != cudaSuccess) return SPARK_ERR_CUDA;
+        ctx->len_hint = start + c0 + T;          // the lengths are known here on the host: the chunk attention picks its second stage by them
         for (int64_t l = 0; l < n_layers; ++l) {
             const int rc = spark_layer_decode(ctx, w + l, cfg + l, cache + l, len_buf, h + c0 * cfg[0].d, T, scratch, stream);
-            if (rc != SPARK_OK) return rc;
+            if (rc != SPARK_OK) {
+                ctx->len_hint = 0;
+                return rc;
+            }
         }
     }
+    ctx->len_hint = 0;
     return SPARK_OK;
 }

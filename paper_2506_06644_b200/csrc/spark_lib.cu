@@ -69,8 +69,9 @@ size_t spark_workspace_bytes(int64_t max_batch, int64_t max_dff, int64_t max_cap
     // tensor-core path, at most n_q KV heads x 128 columns x (max_cap + 32) scores
     size_t need_chunk = 0;
     if (max_batch >= 16)
-        need_chunk = kAttnCellBytes + 4096 + 2 * round_up(static_cast<size_t>(n_q) * 128 * 128 * 2, 1024) +
-                     round_up(static_cast<size_t>(n_q) * 128 * (static_cast<size_t>(max_cap) + 32) * 4, 1024);
+        need_chunk = kAttnCellBytes + 4096 + 4 * round_up(static_cast<size_t>(n_q) * 128 * 128 * 2, 1024) +      // both query parts
+                     round_up(static_cast<size_t>(n_q) * 128 * (static_cast<size_t>(max_cap) + 32) * 4, 1024) +
+                     round_up(static_cast<size_t>(n_q) * (128 * 16 + 64 * 4), 1024) + 1024;                    // column facts of the dense stage
     size_t most = need > need_ffn ? need : need_ffn;
     if (need_chunk > most) most = need_chunk;
     return sizeof(WsHeader) + most + 256;
@@ -105,6 +106,8 @@ int spark_create(spark_ctx** out, int device, void* workspace, size_t workspace_
     c->overlap = 0;
     c->wait_kcycles = 0;
     c->fused = 0;
+    c->chunk_dense = 1;
+    c->len_hint = 0;
     c->l2_prefetch = 0;
     c->next_wqkv = nullptr;
     c->debug_extra_arrivals = 0;
@@ -135,6 +138,12 @@ int spark_grid_size(const spark_ctx* ctx) { return ctx ? ctx->num_sms : 0; }
 int spark_set_l2_prefetch(spark_ctx* ctx, int on) {
     if (ctx == nullptr) return SPARK_ERR_INVALID_ARG;
     ctx->l2_prefetch = on ? 1 : 0;
+    return SPARK_OK;
+}
+
+int spark_set_chunk_dense(spark_ctx* ctx, int mode) {
+    if (ctx == nullptr || mode < 0 || mode > 2) return SPARK_ERR_INVALID_ARG;
+    ctx->chunk_dense = mode;
     return SPARK_OK;
 }
 

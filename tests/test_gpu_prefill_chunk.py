@@ -99,7 +99,9 @@ def test_attention_queries_sharing_one_cache(ctx):
     (32, 8, 2, 256, 128, 256, 0, 16, 0),             # four heads per KV head; the chunk starts the sequence (identity for short rows)
     (12, 8, 4, 256, 128, 512, 400, 64, 0),           # a short chunk: per-query kernel over the shared cache
 ])
-def test_chunk_attention_on_the_tensor_cores(ctx, T, n_q, n_kv, hd, r, cap, L0, k_attn, window):
+@pytest.mark.parametrize("mode", [0, 2])      # second stage: gather per (token, head) / masked dense products where the shape is served
+def test_chunk_attention_on_the_tensor_cores(ctx, mode, T, n_q, n_kv, hd, r, cap, L0, k_attn, window):
+    ctx.set_chunk_dense(mode)
     kv = synth.attn_inputs(1, n_q, n_kv, hd, r, cap, [cap], "bf16", seed=41)
     q = synth.normal_f32((T, n_q, hd), 42, 0) * hd ** -0.5
     lens = [L0 + t + 1 for t in range(T)]
@@ -110,6 +112,7 @@ def test_chunk_attention_on_the_tensor_cores(ctx, T, n_q, n_kv, hd, r, cap, L0, 
                         S.SPARK_BF16, T, n_q, n_kv, hd, r, cap, torch.tensor(lens, dtype=torch.int32, device="cuda"), window, k_attn,
                         S.SPARK_SHARED_CACHE, o, theta, count, None, 0)
     torch.cuda.synchronize()
+    ctx.set_chunk_dense(1)
     kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
     vc = kv.vc[0].astype(np.float64)
     og, thg, cg = o.cpu().numpy(), theta.cpu().numpy(), count.cpu().numpy()
@@ -160,8 +163,10 @@ def test_prefill_loop_over_two_layers_and_ragged_chunks(ctx):
         parity.check_output(got[t], ref[t], "bf16", f"token {t}")
 
 
+@pytest.mark.parametrize("mode", [0, 2])
 @pytest.mark.parametrize("seed", range(6))
-def test_seeded_random_shapes_of_the_chunk_attention(ctx, seed):
+def test_seeded_random_shapes_of_the_chunk_attention(ctx, seed, mode):
+    ctx.set_chunk_dense(mode)
     # head layouts, chunk lengths, cache fill, k and windows drawn from a seeded generator (shapes the tensor-core path serves)
     rng = np.random.default_rng(1000 + seed)
     gq = int(rng.choice([1, 2, 4])); n_kv = int(rng.choice([1, 2, 4])); n_q = gq * n_kv
@@ -177,6 +182,7 @@ def test_seeded_random_shapes_of_the_chunk_attention(ctx, seed):
                         S.SPARK_BF16, T, n_q, n_kv, hd, r, cap, torch.tensor(lens, dtype=torch.int32, device="cuda"), window, k_attn,
                         S.SPARK_SHARED_CACHE, o, theta, None, None, 0)
     torch.cuda.synchronize()
+    ctx.set_chunk_dense(1)
     kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
     vc = kv.vc[0].astype(np.float64)
     og, thg = o.cpu().numpy(), theta.cpu().numpy()
@@ -187,3 +193,37 @@ def test_seeded_random_shapes_of_the_chunk_attention(ctx, seed):
             s = kc[h // gq, lo:lens[t], :r] @ q[t, h, :r].astype(np.float64)
             parity.check_theta(thg[t, h], ref["theta"][h], float(np.std(s, ddof=1)) if s.size > 1 else 1.0, f"token {t} head {h}")
         parity.check_output(og[t].reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"token {t}")
+
+
+@pytest.mark.parametrize("mode", [0, 2])
+def test_rows_behind_the_chunk_may_hold_anything(ctx, mode):
+    # the cache is longer than what has been written: the rows behind the chunk's last token hold NaN bit patterns; and the
+    # 64-token chunk at 4000 cached rows spans several tiles with a ragged last one (8 of its tokens against the oracle)
+    T, n_q, n_kv, hd, r, cap, L0, k_attn = 64, 8, 4, 256, 128, 4200, 4000, 256
+    kv = synth.attn_inputs(1, n_q, n_kv, hd, r, cap, [cap], "bf16", seed=77)
+    q = synth.normal_f32((T, n_q, hd), 78, 0) * hd ** -0.5
+    lens = [L0 + t + 1 for t in range(T)]
+    dev = []
+    for bits in (kv.k1c_bits[0], kv.k2c_bits[0], kv.vc_bits[0]):
+        b = bits.copy()
+        b[:, L0 + T:, :] = 0x7FC0          # bf16 NaN
+        dev.append(bf16_dev(b))
+    ctx.set_chunk_dense(mode)
+    o = torch.full((T, n_q, hd), float("nan"), device="cuda")
+    theta = torch.empty(T, n_q, device="cuda")
+    S.spark_attn_decode(ctx, torch.from_numpy(q).cuda(), dev[0], dev[1], dev[2], S.SPARK_BF16, T, n_q, n_kv, hd, r, cap,
+                        torch.tensor(lens, dtype=torch.int32, device="cuda"), 0, k_attn, S.SPARK_SHARED_CACHE, o, theta, None, None, 0)
+    torch.cuda.synchronize()
+    ctx.set_chunk_dense(1)
+    og = o.cpu().numpy()
+    assert np.all(np.isfinite(og))
+    kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
+    vc = kv.vc[0].astype(np.float64)
+    for t in (0, 1, 17, 31, 32, 47, 62, 63):
+        ref = O.spark_attention(q[t].astype(np.float64), kc, vc, lens[t], k_attn, r, 0)
+        parity.check_output(og[t].reshape(-1), np.asarray(ref["o"]).reshape(-1), "bf16", f"token {t}")
+
+
+def test_chunk_mode_is_checked(ctx):
+    with pytest.raises(S.SparkError):
+        ctx.set_chunk_dense(3)
