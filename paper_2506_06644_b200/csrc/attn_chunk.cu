@@ -617,7 +617,7 @@ struct DenseShared {
     float* orow[kDN];            // output row of each of the block's columns (nullptr: no such column)
 };
 
-__global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams p) {
+__global__ void __launch_bounds__(256, 4) attn_chunk_stats_kernel(const ChunkParams p) {
     __shared__ double part[8][2];
     __shared__ float redf[8];
     __shared__ int redi[8];
@@ -630,14 +630,22 @@ __global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams
     const int lo = p.range[2 * t], n = p.range[2 * t + 1], L = n - lo;
     const float* scol = p.S + (static_cast<int64_t>(g) * kColMax + col) * p.scap;
     if (tid < p.hd) p.o[static_cast<int64_t>(blockIdx.x) * p.hd + tid] = 0.f;       // the dense kernel adds into it
-    constexpr int kKeep = 32;
-    const bool kept = L <= kKeep * 256;
-    float keep[kKeep];
+    // The column's visible part stays in registers between the three sweeps: eight 16-byte loads per thread starting at the
+    // 16-byte boundary at or below lo (rows outside [lo, n) read as -inf); longer columns are swept from L2 three times.
+    constexpr int kKeep4 = 8;
+    const int lo4 = lo & ~3;
+    const bool kept = n - lo4 <= kKeep4 * 4 * 256;
+    float keep[kKeep4][4];
     if (kept) {
 #pragma unroll
-        for (int u = 0; u < kKeep; ++u) {
-            const int j = lo + 256 * u + tid;
-            keep[u] = j < n ? __ldcg(scol + j) : -INFINITY;
+        for (int u = 0; u < kKeep4; ++u) {
+            const int j = lo4 + 4 * (256 * u + tid);
+            float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            if (j < n) v = __ldcg(reinterpret_cast<const float4*>(scol + j));      // the column is padded beyond the capacity
+            keep[u][0] = (j >= lo && j < n) ? v.x : -INFINITY;
+            keep[u][1] = (j + 1 >= lo && j + 1 < n) ? v.y : -INFINITY;
+            keep[u][2] = (j + 2 >= lo && j + 2 < n) ? v.z : -INFINITY;
+            keep[u][3] = (j + 3 >= lo && j + 3 < n) ? v.w : -INFINITY;
         }
     }
     float th = -INFINITY;
@@ -647,11 +655,13 @@ __global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams
         float f1 = 0.f, f2 = 0.f;
         if (kept) {
 #pragma unroll
-            for (int u = 0; u < kKeep; ++u) {
-                const float d = lo + 256 * u + tid < n ? keep[u] - c0 : 0.f;
-                f1 += d;
-                f2 = fmaf(d, d, f2);
-            }
+            for (int u = 0; u < kKeep4; ++u)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float d = keep[u][e] == -INFINITY ? 0.f : keep[u][e] - c0;
+                    f1 += d;
+                    f2 = fmaf(d, d, f2);
+                }
         } else {
             for (int j = lo + tid; j < n; j += 256) {
                 const float d = __ldcg(scol + j) - c0;
@@ -684,10 +694,12 @@ __global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams
     int cnt = 0;
     if (kept) {
 #pragma unroll
-        for (int u = 0; u < kKeep; ++u)
-            if (keep[u] > th) {
-                mx = fmaxf(mx, keep[u]);
-                ++cnt;
+        for (int u = 0; u < kKeep4; ++u)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool on = keep[u][e] > th;
+                mx = fmaxf(mx, on ? keep[u][e] : -INFINITY);
+                cnt += on ? 1 : 0;
             }
     } else {
         for (int j = lo + tid; j < n; j += 256) {
@@ -699,7 +711,7 @@ __global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams
         }
     }
     mx = warp_max(mx);
-    cnt = warp_sum_int(cnt);
+    cnt = __reduce_add_sync(kFull, cnt);
     if (lane == 0) {
         redf[warp] = mx;
         redi[warp] = cnt;
@@ -719,8 +731,9 @@ __global__ void __launch_bounds__(256) attn_chunk_stats_kernel(const ChunkParams
     float es = 0.f;
     if (kept) {
 #pragma unroll
-        for (int u = 0; u < kKeep; ++u)
-            if (keep[u] > th) es += __expf(keep[u] - mx);
+        for (int u = 0; u < kKeep4; ++u)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) es += keep[u][e] > th ? __expf(keep[u][e] - mx) : 0.f;
     } else {
         for (int j = lo + tid; j < n; j += 256) {
             const float v = __ldcg(scol + j);
