@@ -379,6 +379,18 @@ int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const spark_laye
                   int64_t n_layers, float* h, int64_t n_tokens, int64_t start, int64_t chunk, int32_t* len_buf, float* scratch,
                   void* stream);
 
+/* The same with two chunks in flight (scheduling only; the paper has no counterpart): chunk c runs on stream c % 2 with context
+ * c % 2, and layer l of a chunk starts once layer l of the chunk before it has finished, which is all it needs (the caches of
+ * layer l up to its own rows).  The kernels of a chunk layer are short and latency-bound, so the second chunk fills the gaps
+ * the first one leaves.  ctx2: a second context on the same device (two kernels that run at the same time must not share a
+ * workspace); scratch2: a second scratch area like scratch; len_buf: 2 * chunk int32; stream2: a second stream, different from
+ * stream.  The call forks from `stream` and joins back into it: work queued on `stream` before the call is seen by both, work
+ * queued after it sees all of the prefill.  Creates and destroys 2 * n_layers + 2 events (no device memory).  Results equal
+ * spark_prefill's up to the order of floating-point reductions. */
+int spark_prefill_pipelined(spark_ctx* ctx, spark_ctx* ctx2, const spark_layer_weights* w, const spark_layer_cfg* cfg,
+                            const spark_kv_cache* cache, int64_t n_layers, float* h, int64_t n_tokens, int64_t start,
+                            int64_t chunk, int32_t* len_buf, float* scratch, float* scratch2, void* stream, void* stream2);
+
 /* Scheduling option (the paper has no counterpart; default off): in layer calls of one to four tokens every kernel asks L2,
  * with a few bulk-prefetch instructions per block, for the weights the NEXT kernel will stream (QKV kernel: Wo; attention:
  * K1t; FFN, inside spark_stack_decode: the next layer's Wqkv).  Measured on B200 it LOSES (2B layer 30.8 -> 32.0 us, 9B

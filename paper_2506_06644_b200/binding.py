@@ -31,7 +31,7 @@ EXPORTS = [
     "spark_attn_decode", "spark_dense_gemv", "spark_layer_decode", "spark_ffn_decode_noalloc", "spark_ffn_decode_fp8", "spark_attn_decode_fp8k",
     "spark_stat_moments", "spark_stat_merge", "spark_stat_select",
     "spark_set_wait_limit", "spark_debug_expect_arrivals", "spark_noalloc_status",
-    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill", "spark_attn_decode_fp8kv", "spark_set_chunk_dense",
+    "spark_stack_decode", "spark_set_fused_layer", "spark_set_l2_prefetch", "spark_prefill", "spark_attn_decode_fp8kv", "spark_set_chunk_dense", "spark_prefill_pipelined",
 ]
 
 
@@ -100,6 +100,8 @@ def lib() -> C.CDLL:
         "spark_set_fused_layer": (i32, [vp, i32]),
         "spark_set_chunk_dense": (i32, [vp, i32]),
         "spark_prefill": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64, vp, i64, i64, i64, vp, vp, vp]),
+        "spark_prefill_pipelined": (i32, [vp, vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64, vp, i64, i64,
+                                          i64, vp, vp, vp, vp, vp]),
         "spark_set_l2_prefetch": (i32, [vp, i32]),
         "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
                                      vp, vp, i64, vp, vp]),
@@ -339,8 +341,9 @@ def layer_scratch_floats(cfg: dict, B: int) -> int:
     return B * (nqkv + 2 * cfg["n_q"] * cfg["hd"] + cfg["d"] + 2 + cfg["n_q"])
 
 
-def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64):
+def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64, ctx2: SparkContext | None = None, stream2=None):
     """Run a prompt through a stack of layers chunk by chunk (the C entry point of the same name; argument marshalling only).
+    With a second context ctx2 (and optionally a second torch stream) two chunks are in flight: spark_prefill_pipelined.
 
     layers: LayerHandles made with SPARK_SHARED_CACHE in cfg["flags"] and caches [n_kv][cap][.]; h [N][d] fp32 holds the
     prompt's N embeddings and is replaced in place by the stack's outputs; the tokens are appended to each layer's
@@ -352,6 +355,17 @@ def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64):
     stack = make_stack(layers)
     cfg = {k: getattr(layers[0].cfg, k) for k in ("n_q", "n_kv", "hd", "d")}
     scratch = torch.empty(layer_scratch_floats(cfg, min(chunk, N)), dtype=torch.float32, device=h.device)
+    if ctx2 is not None:
+        scratch2 = torch.empty_like(scratch)
+        len_buf = torch.empty(2 * chunk, dtype=torch.int32, device=h.device)
+        s2 = stream2 if stream2 is not None else torch.cuda.Stream(device=h.device)
+        _check(lib().spark_prefill_pipelined(ctx.handle, ctx2.handle, stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(h), N,
+                                             start, chunk, _ptr(len_buf), _ptr(scratch), _ptr(scratch2), _stream(), s2.cuda_stream),
+               "spark_prefill_pipelined")
+        # the temporaries are used on the second stream too: keep the caching allocator from handing them out early
+        for t in (scratch, scratch2, len_buf):
+            t.record_stream(s2)
+        return h
     len_buf = torch.empty(chunk, dtype=torch.int32, device=h.device)
     _check(lib().spark_prefill(ctx.handle, stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(h), N, start, chunk,
                                _ptr(len_buf), _ptr(scratch), _stream()), "spark_prefill")

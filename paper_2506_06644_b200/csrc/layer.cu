@@ -4,6 +4,8 @@
 // not change them (Table "FLOPs per token").
 #include <cmath>
 
+#include <new>
+
 #include "kernels.h"
 #include "mma_rows.cuh"
 #include "rowdot.cuh"
@@ -803,4 +805,63 @@ extern "C" int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const
     }
     ctx->len_hint = 0;
     return SPARK_OK;
+}
+
+// Two chunks in flight: chunk c runs on stream c % 2 with its own context (workspaces must not be shared between kernels that
+// run at the same time); layer l of chunk c waits for layer l of chunk c - 1, which has filled that layer's cache up to the
+// rows chunk c reads -- a wavefront over (chunk, layer).  The kernels of a chunk layer are latency-bound (a dozen launches of
+// 5-10 us, each with an idle boundary): the other stream's kernels fill those gaps.
+extern "C" int spark_prefill_pipelined(spark_ctx* ctx, spark_ctx* ctx2, const spark_layer_weights* w, const spark_layer_cfg* cfg,
+                                       const spark_kv_cache* cache, int64_t n_layers, float* h, int64_t n_tokens, int64_t start,
+                                       int64_t chunk, int32_t* len_buf, float* scratch, float* scratch2, void* stream, void* stream2) {
+    if (ctx == nullptr || ctx2 == nullptr || ctx == ctx2 || w == nullptr || cfg == nullptr || cache == nullptr || h == nullptr ||
+        len_buf == nullptr || scratch == nullptr || scratch2 == nullptr || scratch == scratch2 || stream == stream2)
+        return SPARK_ERR_INVALID_ARG;
+    if (n_layers < 1 || n_layers > 4096 || n_tokens < 1 || start < 0 || chunk < 1 || chunk > 64) return SPARK_ERR_INVALID_ARG;
+    for (int64_t l = 0; l < n_layers; ++l) {
+        if (!(cfg[l].flags & SPARK_SHARED_CACHE)) return SPARK_ERR_INVALID_ARG;
+        if (start + n_tokens > cfg[l].cap || cfg[l].d != cfg[0].d) return SPARK_ERR_INVALID_ARG;
+    }
+    if (!on_device(ctx) || ctx2->device != ctx->device) return SPARK_ERR_INVALID_ARG;
+    spark_ctx* cx[2] = {ctx, ctx2};
+    float* sc[2] = {scratch, scratch2};
+    cudaStream_t st[2] = {static_cast<cudaStream_t>(stream), static_cast<cudaStream_t>(stream2)};
+    // done[s][l]: layer l of the newest chunk on stream s has finished; fork / join around the call
+    const size_t n_ev = 2 * static_cast<size_t>(n_layers) + 2;
+    cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[n_ev];
+    if (ev == nullptr) return SPARK_ERR_CUDA;
+    size_t made = 0;
+    int rc = SPARK_OK;
+    for (; made < n_ev; ++made)
+        if (cudaEventCreateWithFlags(&ev[made], cudaEventDisableTiming) != cudaSuccess) { rc = SPARK_ERR_CUDA; break; }
+    auto done = [&](int s, int64_t l) -> cudaEvent_t& { return ev[2 + static_cast<size_t>(s) * n_layers + l]; };
+    if (rc == SPARK_OK) {
+        // what is queued on the caller's stream (the embeddings) comes before the second stream's first kernel
+        if (cudaEventRecord(ev[0], st[0]) != cudaSuccess || cudaStreamWaitEvent(st[1], ev[0], 0) != cudaSuccess) rc = SPARK_ERR_CUDA;
+    }
+    int64_t c = 0;
+    for (int64_t c0 = 0; c0 < n_tokens && rc == SPARK_OK; c0 += chunk, ++c) {
+        const int s = static_cast<int>(c & 1);
+        const int64_t T = n_tokens - c0 < chunk ? n_tokens - c0 : chunk;
+        int32_t* lens = len_buf + s * chunk;
+        int n = static_cast<int>(T), first = static_cast<int>(start + c0 + 1);
+        void* args[] = {&lens, &n, &first};
+        if (launch_kernel(cx[s], reinterpret_cast<const void*>(chunk_lengths_kernel), 1u, 64u, 0, st[s], false, args) != cudaSuccess) {
+            rc = SPARK_ERR_CUDA;
+            break;
+        }
+        cx[s]->len_hint = start + c0 + T;
+        for (int64_t l = 0; l < n_layers && rc == SPARK_OK; ++l) {
+            if (c > 0 && cudaStreamWaitEvent(st[s], done(1 - s, l), 0) != cudaSuccess) { rc = SPARK_ERR_CUDA; break; }
+            rc = spark_layer_decode(cx[s], w + l, cfg + l, cache + l, lens, h + c0 * cfg[0].d, T, sc[s], st[s]);
+            if (rc == SPARK_OK && cudaEventRecord(done(s, l), st[s]) != cudaSuccess) rc = SPARK_ERR_CUDA;
+        }
+        cx[s]->len_hint = 0;
+    }
+    if (rc == SPARK_OK) {          // the caller's stream continues after both
+        if (cudaEventRecord(ev[1], st[1]) != cudaSuccess || cudaStreamWaitEvent(st[0], ev[1], 0) != cudaSuccess) rc = SPARK_ERR_CUDA;
+    }
+    for (size_t i = 0; i < made; ++i) cudaEventDestroy(ev[i]);      // released once the work that uses them has completed
+    delete[] ev;
+    return rc;
 }
