@@ -281,3 +281,24 @@ def test_two_chunks_in_flight_give_what_one_at_a_time_gives(ctx):
     for la, lb, lc in zip(ca, cb, cc):          # the stored rows likewise
         for k in la:
             assert np.abs(la[k] - lc[k]).mean() <= 3 * np.abs(la[k] - lb[k]).mean() + 1e-4 * np.abs(la[k]).mean()
+
+
+def test_pipelined_prefill_checks_its_arguments(ctx):
+    sh, cap = synth.TINY, 64
+    lw = synth.layer_weights(sh, 3, 0)
+    kv = synth.attn_inputs(1, sh.n_q, sh.n_kv, sh.hd, sh.r_attn, cap, [4], "bf16", seed=4)
+    dev = dict(norm1=torch.from_numpy(lw.norm1).cuda(), norm2=torch.from_numpy(lw.norm2).cuda(), Wqkv=bf16_dev(lw.Wqkv_bits),
+               Wo=bf16_dev(lw.Wo_bits), K1t=bf16_dev(lw.K1t_bits), K2t=bf16_dev(lw.K2t_bits), Vt=bf16_dev(lw.Vt_bits))
+    cache = dict(k1c=bf16_dev(kv.k1c_bits[0]), k2c=bf16_dev(kv.k2c_bits[0]), vc=bf16_dev(kv.vc_bits[0]))
+    cfg = dict(d=sh.d, d_ff=sh.d_ff, r_ff=sh.r_ff, k_ff=sh.k_ff, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
+               k_attn=sh.k_attn, window=0, cap=cap, rms_eps=1e-6, rope_base=10000.0, flags=S.SPARK_SHARED_CACHE)
+    layer = S.make_layer(dev, cfg, cache)
+    h = torch.zeros(8, sh.d, device="cuda")
+    with pytest.raises(S.SparkError) as e:          # one context twice: its workspace would be shared by concurrent kernels
+        S.spark_prefill(ctx, [layer], h, 4, chunk=4, ctx2=ctx)
+    assert e.value.status == S.SPARK_ERR_INVALID_ARG
+    with pytest.raises(S.SparkError) as e:          # the same stream twice
+        S.spark_prefill(ctx, [layer], h, 4, chunk=4, ctx2=S.SparkContext(0, max_batch=8), stream2=torch.cuda.current_stream())
+    assert e.value.status == S.SPARK_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert ctx.device_status() == S.SPARK_OK
