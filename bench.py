@@ -828,24 +828,27 @@ def other_workloads(torch, S, peak, steps, warmup, with_oracle=True):
     out.append({"workload": f"spark_prefill: {Np} tokens from an empty cache through {nl} layers in 64-token chunks (host launches)",
                 "us_per_launch": ms_pre * 1e3 / (Np // 64 * nl), "us_per_token_per_layer": ms_pre * 1e3 / (Np * nl),
                 "prompt_tokens_per_s_per_layer_stack": Np / (ms_pre * 1e-3)})
-    # -- the same prompt with two chunks in flight (spark_prefill_pipelined: two streams, two contexts, a wavefront over
-    #    (chunk, layer)); the caches are overwritten from row 0 again
-    ctx2 = S.SparkContext(dev.index, max_batch=64, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d)
-    ctx2.set_launch_overlap(True)
-    side = torch.cuda.Stream(device=dev)
-    S.spark_prefill(ctx, lay_only, hp[:256].clone(), 0, chunk=64, ctx2=ctx2, stream2=side)          # warm-up
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    S.spark_prefill(ctx, lay_only, hp, 0, chunk=64, ctx2=ctx2, stream2=side)
-    e1.record()
-    torch.cuda.synchronize()
-    assert ctx.device_status() == S.SPARK_OK and ctx2.device_status() == S.SPARK_OK
-    ms_pipe = e0.elapsed_time(e1)
-    out.append({"workload": f"spark_prefill_pipelined: the same {Np}-token prompt, two chunks in flight on two streams (host launches)",
-                "us_per_launch": ms_pipe * 1e3 / (Np // 64 * nl), "us_per_token_per_layer": ms_pipe * 1e3 / (Np * nl),
-                "prompt_tokens_per_s_per_layer_stack": Np / (ms_pipe * 1e-3), "speedup_vs_one_chunk_at_a_time": ms_pre / ms_pipe})
-    ctx2.close()
+    # -- the same prompt with two and three chunks in flight (spark_prefill_pipelined: a stream and a context per chunk in
+    #    flight, a wavefront over (chunk, layer)); the caches are overwritten from row 0 again
+    more = [S.SparkContext(dev.index, max_batch=64, max_dff=sh.d_ff, max_cap=L, n_q=sh.n_q, hd=sh.hd, max_d=sh.d) for _ in range(2)]
+    sides = [torch.cuda.Stream(device=dev) for _ in more]
+    for c in more:
+        c.set_launch_overlap(True)
+    for n_in in (2, 3):
+        S.spark_prefill(ctx, lay_only, hp[:256].clone(), 0, chunk=64, more_ctx=more[:n_in - 1], more_streams=sides[:n_in - 1])      # warm-up
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        S.spark_prefill(ctx, lay_only, hp, 0, chunk=64, more_ctx=more[:n_in - 1], more_streams=sides[:n_in - 1])
+        e1.record()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == S.SPARK_OK and all(c.device_status() == S.SPARK_OK for c in more)
+        ms_pipe = e0.elapsed_time(e1)
+        out.append({"workload": f"spark_prefill_pipelined: the same {Np}-token prompt, {n_in} chunks in flight on {n_in} streams (host launches)",
+                    "us_per_launch": ms_pipe * 1e3 / (Np // 64 * nl), "us_per_token_per_layer": ms_pipe * 1e3 / (Np * nl),
+                    "prompt_tokens_per_s_per_layer_stack": Np / (ms_pipe * 1e-3), "speedup_vs_one_chunk_at_a_time": ms_pre / ms_pipe})
+    for c in more:
+        c.close()
     ctx.close()
     del stacks, chunk_layers
 

@@ -379,17 +379,17 @@ int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const spark_laye
                   int64_t n_layers, float* h, int64_t n_tokens, int64_t start, int64_t chunk, int32_t* len_buf, float* scratch,
                   void* stream);
 
-/* The same with two chunks in flight (scheduling only; the paper has no counterpart): chunk c runs on stream c % 2 with context
- * c % 2, and layer l of a chunk starts once layer l of the chunk before it has finished, which is all it needs (the caches of
- * layer l up to its own rows).  The kernels of a chunk layer are short and latency-bound, so the second chunk fills the gaps
- * the first one leaves.  ctx2: a second context on the same device (two kernels that run at the same time must not share a
- * workspace); scratch2: a second scratch area like scratch; len_buf: 2 * chunk int32; stream2: a second stream, different from
- * stream.  The call forks from `stream` and joins back into it: work queued on `stream` before the call is seen by both, work
- * queued after it sees all of the prefill.  Creates and destroys 2 * n_layers + 2 events (no device memory).  Results equal
- * spark_prefill's up to the order of floating-point reductions. */
-int spark_prefill_pipelined(spark_ctx* ctx, spark_ctx* ctx2, const spark_layer_weights* w, const spark_layer_cfg* cfg,
-                            const spark_kv_cache* cache, int64_t n_layers, float* h, int64_t n_tokens, int64_t start,
-                            int64_t chunk, int32_t* len_buf, float* scratch, float* scratch2, void* stream, void* stream2);
+/* The same with several chunks in flight (scheduling only; the paper has no counterpart): chunk c runs on stream c % n_inflight
+ * with context c % n_inflight, and layer l of a chunk starts once layer l of the chunk before it has finished, which is all it
+ * needs (the caches of layer l up to its own rows).  The kernels of a chunk layer are short and latency-bound, so the other
+ * chunks fill the gaps each one leaves.  ctxs, scratches, streams: HOST arrays of n_inflight (2 to 8) distinct contexts on one
+ * device (kernels that run at the same time must not share a workspace), scratch areas like spark_prefill's, and streams;
+ * len_buf: n_inflight * chunk int32.  The call forks from streams[0] and joins back into it: work queued there before the call
+ * is seen by all, work queued after it sees all of the prefill.  Creates and destroys n_inflight * (n_layers + 1) + 1 events
+ * (no device memory).  Results equal spark_prefill's up to the order of floating-point reductions. */
+int spark_prefill_pipelined(spark_ctx* const* ctxs, float* const* scratches, void* const* streams, int64_t n_inflight,
+                            const spark_layer_weights* w, const spark_layer_cfg* cfg, const spark_kv_cache* cache,
+                            int64_t n_layers, float* h, int64_t n_tokens, int64_t start, int64_t chunk, int32_t* len_buf);
 
 /* Scheduling option (the paper has no counterpart; default off): in layer calls of one to four tokens every kernel asks L2,
  * with a few bulk-prefetch instructions per block, for the weights the NEXT kernel will stream (QKV kernel: Wo; attention:

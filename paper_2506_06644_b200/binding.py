@@ -100,8 +100,8 @@ def lib() -> C.CDLL:
         "spark_set_fused_layer": (i32, [vp, i32]),
         "spark_set_chunk_dense": (i32, [vp, i32]),
         "spark_prefill": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64, vp, i64, i64, i64, vp, vp, vp]),
-        "spark_prefill_pipelined": (i32, [vp, vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache), i64, vp, i64, i64,
-                                          i64, vp, vp, vp, vp, vp]),
+        "spark_prefill_pipelined": (i32, [C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), i64, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg),
+                                          C.POINTER(_KvCache), i64, vp, i64, i64, i64, vp]),
         "spark_set_l2_prefetch": (i32, [vp, i32]),
         "spark_layer_decode": (i32, [vp, C.POINTER(_LayerWeights), C.POINTER(_LayerCfg), C.POINTER(_KvCache),
                                      vp, vp, i64, vp, vp]),
@@ -341,9 +341,10 @@ def layer_scratch_floats(cfg: dict, B: int) -> int:
     return B * (nqkv + 2 * cfg["n_q"] * cfg["hd"] + cfg["d"] + 2 + cfg["n_q"])
 
 
-def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64, ctx2: SparkContext | None = None, stream2=None):
+def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64, more_ctx=(), more_streams=None):
     """Run a prompt through a stack of layers chunk by chunk (the C entry point of the same name; argument marshalling only).
-    With a second context ctx2 (and optionally a second torch stream) two chunks are in flight: spark_prefill_pipelined.
+    With further contexts in more_ctx (and optionally as many further torch streams) that many more chunks are in flight at
+    a time: spark_prefill_pipelined.
 
     layers: LayerHandles made with SPARK_SHARED_CACHE in cfg["flags"] and caches [n_kv][cap][.]; h [N][d] fp32 holds the
     prompt's N embeddings and is replaced in place by the stack's outputs; the tokens are appended to each layer's
@@ -355,16 +356,22 @@ def spark_prefill(ctx: SparkContext, layers, h, start: int, chunk: int = 64, ctx
     stack = make_stack(layers)
     cfg = {k: getattr(layers[0].cfg, k) for k in ("n_q", "n_kv", "hd", "d")}
     scratch = torch.empty(layer_scratch_floats(cfg, min(chunk, N)), dtype=torch.float32, device=h.device)
-    if ctx2 is not None:
-        scratch2 = torch.empty_like(scratch)
-        len_buf = torch.empty(2 * chunk, dtype=torch.int32, device=h.device)
-        s2 = stream2 if stream2 is not None else torch.cuda.Stream(device=h.device)
-        _check(lib().spark_prefill_pipelined(ctx.handle, ctx2.handle, stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(h), N,
-                                             start, chunk, _ptr(len_buf), _ptr(scratch), _ptr(scratch2), _stream(), s2.cuda_stream),
-               "spark_prefill_pipelined")
-        # the temporaries are used on the second stream too: keep the caching allocator from handing them out early
-        for t in (scratch, scratch2, len_buf):
-            t.record_stream(s2)
+    more_ctx = list(more_ctx) if not isinstance(more_ctx, SparkContext) else [more_ctx]
+    if more_ctx:
+        n = 1 + len(more_ctx)
+        ctxs = [ctx] + more_ctx
+        scratches = [scratch] + [torch.empty_like(scratch) for _ in more_ctx]
+        side = list(more_streams) if more_streams is not None else [torch.cuda.Stream(device=h.device) for _ in more_ctx]
+        streams = [_stream()] + [s.cuda_stream for s in side]
+        len_buf = torch.empty(n * chunk, dtype=torch.int32, device=h.device)
+        arr = lambda vals: (C.c_void_p * n)(*vals)
+        _check(lib().spark_prefill_pipelined(arr([c.handle.value for c in ctxs]), arr([_ptr(t) for t in scratches]), arr(streams), n,
+                                             stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(h), N, start, chunk,
+                                             _ptr(len_buf)), "spark_prefill_pipelined")
+        # the temporaries are used on the other streams too: keep the caching allocator from handing them out early
+        for s in side:
+            for t in scratches + [len_buf]:
+                t.record_stream(s)
         return h
     len_buf = torch.empty(chunk, dtype=torch.int32, device=h.device)
     _check(lib().spark_prefill(ctx.handle, stack.weights, stack.cfgs, stack.caches, stack.n_layers, _ptr(h), N, start, chunk,

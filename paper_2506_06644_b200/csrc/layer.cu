@@ -807,59 +807,69 @@ extern "C" int spark_prefill(spark_ctx* ctx, const spark_layer_weights* w, const
     return SPARK_OK;
 }
 
-// Two chunks in flight: chunk c runs on stream c % 2 with its own context (workspaces must not be shared between kernels that
-// run at the same time); layer l of chunk c waits for layer l of chunk c - 1, which has filled that layer's cache up to the
-// rows chunk c reads -- a wavefront over (chunk, layer).  The kernels of a chunk layer are latency-bound (a dozen launches of
-// 5-10 us, each with an idle boundary): the other stream's kernels fill those gaps.
-extern "C" int spark_prefill_pipelined(spark_ctx* ctx, spark_ctx* ctx2, const spark_layer_weights* w, const spark_layer_cfg* cfg,
-                                       const spark_kv_cache* cache, int64_t n_layers, float* h, int64_t n_tokens, int64_t start,
-                                       int64_t chunk, int32_t* len_buf, float* scratch, float* scratch2, void* stream, void* stream2) {
-    if (ctx == nullptr || ctx2 == nullptr || ctx == ctx2 || w == nullptr || cfg == nullptr || cache == nullptr || h == nullptr ||
-        len_buf == nullptr || scratch == nullptr || scratch2 == nullptr || scratch == scratch2 || stream == stream2)
+// Several chunks in flight: chunk c runs on stream c % n with its own context (workspaces must not be shared between kernels
+// that run at the same time); layer l of chunk c waits for layer l of chunk c - 1, which has filled that layer's cache up to
+// the rows chunk c reads -- a wavefront over (chunk, layer).  The kernels of a chunk layer are latency-bound (a dozen launches
+// of 5-10 us, each with an idle boundary): the other streams' kernels fill those gaps.
+extern "C" int spark_prefill_pipelined(spark_ctx* const* ctxs, float* const* scratches, void* const* streams, int64_t n_inflight,
+                                       const spark_layer_weights* w, const spark_layer_cfg* cfg, const spark_kv_cache* cache,
+                                       int64_t n_layers, float* h, int64_t n_tokens, int64_t start, int64_t chunk, int32_t* len_buf) {
+    constexpr int kMaxInflight = 8;
+    if (ctxs == nullptr || scratches == nullptr || streams == nullptr || n_inflight < 2 || n_inflight > kMaxInflight || w == nullptr ||
+        cfg == nullptr || cache == nullptr || h == nullptr || len_buf == nullptr)
         return SPARK_ERR_INVALID_ARG;
+    const int n = static_cast<int>(n_inflight);
+    for (int i = 0; i < n; ++i) {
+        if (ctxs[i] == nullptr || scratches[i] == nullptr) return SPARK_ERR_INVALID_ARG;
+        for (int j = 0; j < i; ++j)
+            if (ctxs[i] == ctxs[j] || scratches[i] == scratches[j] || streams[i] == streams[j]) return SPARK_ERR_INVALID_ARG;
+        if (ctxs[i]->device != ctxs[0]->device) return SPARK_ERR_INVALID_ARG;
+    }
     if (n_layers < 1 || n_layers > 4096 || n_tokens < 1 || start < 0 || chunk < 1 || chunk > 64) return SPARK_ERR_INVALID_ARG;
     for (int64_t l = 0; l < n_layers; ++l) {
         if (!(cfg[l].flags & SPARK_SHARED_CACHE)) return SPARK_ERR_INVALID_ARG;
         if (start + n_tokens > cfg[l].cap || cfg[l].d != cfg[0].d) return SPARK_ERR_INVALID_ARG;
     }
-    if (!on_device(ctx) || ctx2->device != ctx->device) return SPARK_ERR_INVALID_ARG;
-    spark_ctx* cx[2] = {ctx, ctx2};
-    float* sc[2] = {scratch, scratch2};
-    cudaStream_t st[2] = {static_cast<cudaStream_t>(stream), static_cast<cudaStream_t>(stream2)};
-    // done[s][l]: layer l of the newest chunk on stream s has finished; fork / join around the call
-    const size_t n_ev = 2 * static_cast<size_t>(n_layers) + 2;
+    if (!on_device(ctxs[0])) return SPARK_ERR_INVALID_ARG;
+    cudaStream_t st[kMaxInflight];
+    for (int i = 0; i < n; ++i) st[i] = static_cast<cudaStream_t>(streams[i]);
+    // done[s][l]: layer l of the newest chunk on stream s has finished; fork and join around the call
+    const size_t n_ev = static_cast<size_t>(n) * static_cast<size_t>(n_layers) + 1 + static_cast<size_t>(n);
     cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[n_ev];
     if (ev == nullptr) return SPARK_ERR_CUDA;
     size_t made = 0;
     int rc = SPARK_OK;
     for (; made < n_ev; ++made)
         if (cudaEventCreateWithFlags(&ev[made], cudaEventDisableTiming) != cudaSuccess) { rc = SPARK_ERR_CUDA; break; }
-    auto done = [&](int s, int64_t l) -> cudaEvent_t& { return ev[2 + static_cast<size_t>(s) * n_layers + l]; };
+    auto done = [&](int s, int64_t l) -> cudaEvent_t& { return ev[1 + n + static_cast<size_t>(s) * n_layers + l]; };
     if (rc == SPARK_OK) {
-        // what is queued on the caller's stream (the embeddings) comes before the second stream's first kernel
-        if (cudaEventRecord(ev[0], st[0]) != cudaSuccess || cudaStreamWaitEvent(st[1], ev[0], 0) != cudaSuccess) rc = SPARK_ERR_CUDA;
+        // what is queued on the caller's stream (the embeddings) comes before the other streams' first kernels
+        if (cudaEventRecord(ev[0], st[0]) != cudaSuccess) rc = SPARK_ERR_CUDA;
+        for (int i = 1; i < n && rc == SPARK_OK; ++i)
+            if (cudaStreamWaitEvent(st[i], ev[0], 0) != cudaSuccess) rc = SPARK_ERR_CUDA;
     }
     int64_t c = 0;
     for (int64_t c0 = 0; c0 < n_tokens && rc == SPARK_OK; c0 += chunk, ++c) {
-        const int s = static_cast<int>(c & 1);
+        const int s = static_cast<int>(c % n), prev = static_cast<int>((c + n - 1) % n);
         const int64_t T = n_tokens - c0 < chunk ? n_tokens - c0 : chunk;
         int32_t* lens = len_buf + s * chunk;
-        int n = static_cast<int>(T), first = static_cast<int>(start + c0 + 1);
-        void* args[] = {&lens, &n, &first};
-        if (launch_kernel(cx[s], reinterpret_cast<const void*>(chunk_lengths_kernel), 1u, 64u, 0, st[s], false, args) != cudaSuccess) {
+        int nt = static_cast<int>(T), first = static_cast<int>(start + c0 + 1);
+        void* args[] = {&lens, &nt, &first};
+        if (launch_kernel(ctxs[s], reinterpret_cast<const void*>(chunk_lengths_kernel), 1u, 64u, 0, st[s], false, args) != cudaSuccess) {
             rc = SPARK_ERR_CUDA;
             break;
         }
-        cx[s]->len_hint = start + c0 + T;
+        ctxs[s]->len_hint = start + c0 + T;
         for (int64_t l = 0; l < n_layers && rc == SPARK_OK; ++l) {
-            if (c > 0 && cudaStreamWaitEvent(st[s], done(1 - s, l), 0) != cudaSuccess) { rc = SPARK_ERR_CUDA; break; }
-            rc = spark_layer_decode(cx[s], w + l, cfg + l, cache + l, lens, h + c0 * cfg[0].d, T, sc[s], st[s]);
+            if (c > 0 && cudaStreamWaitEvent(st[s], done(prev, l), 0) != cudaSuccess) { rc = SPARK_ERR_CUDA; break; }
+            rc = spark_layer_decode(ctxs[s], w + l, cfg + l, cache + l, lens, h + c0 * cfg[0].d, T, scratches[s], st[s]);
             if (rc == SPARK_OK && cudaEventRecord(done(s, l), st[s]) != cudaSuccess) rc = SPARK_ERR_CUDA;
         }
-        cx[s]->len_hint = 0;
+        ctxs[s]->len_hint = 0;
     }
-    if (rc == SPARK_OK) {          // the caller's stream continues after both
-        if (cudaEventRecord(ev[1], st[1]) != cudaSuccess || cudaStreamWaitEvent(st[0], ev[1], 0) != cudaSuccess) rc = SPARK_ERR_CUDA;
+    if (rc == SPARK_OK) {          // the caller's stream continues after all of them
+        for (int i = 1; i < n && rc == SPARK_OK; ++i)
+            if (cudaEventRecord(ev[i], st[i]) != cudaSuccess || cudaStreamWaitEvent(st[0], ev[i], 0) != cudaSuccess) rc = SPARK_ERR_CUDA;
     }
     for (size_t i = 0; i < made; ++i) cudaEventDestroy(ev[i]);      // released once the work that uses them has completed
     delete[] ev;

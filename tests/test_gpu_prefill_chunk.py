@@ -148,7 +148,7 @@ def test_prefill_loop_over_two_layers_and_ragged_chunks(ctx, chunk, pipelined):
         keep.append((dev, cache))
     h = torch.from_numpy(h0).cuda()
     ctx2 = S.SparkContext(0, max_batch=64) if pipelined else None
-    S.spark_prefill(ctx, layers, h, L0, chunk=chunk, ctx2=ctx2)
+    S.spark_prefill(ctx, layers, h, L0, chunk=chunk, more_ctx=[ctx2] if ctx2 is not None else [])
     torch.cuda.synchronize()
     if ctx2 is not None:
         assert ctx2.device_status() == S.SPARK_OK
@@ -235,7 +235,7 @@ def test_chunk_mode_is_checked(ctx):
         ctx.set_chunk_dense(3)
 
 
-def test_two_chunks_in_flight_give_what_one_at_a_time_gives(ctx):
+def test_chunks_in_flight_give_what_one_at_a_time_gives(ctx):
     # many chunks through four layers (alternating local / global) on two streams against the plain loop: outputs and caches
     sh, N, L0, cap, n_layers, chunk = synth.GEMMA2_2B, 640, 17, 704, 4, 64
     gen = torch.Generator(device="cuda")
@@ -261,12 +261,12 @@ def test_two_chunks_in_flight_give_what_one_at_a_time_gives(ctx):
     for pipelined in (False, False, True):
         layers, keep = make()
         h = torch.from_numpy(h0).cuda()
-        ctx2 = S.SparkContext(0, max_batch=64) if pipelined else None
-        S.spark_prefill(ctx, layers, h, L0, chunk=chunk, ctx2=ctx2)
+        more = [S.SparkContext(0, max_batch=64) for _ in range(2)] if pipelined else []          # three chunks in flight
+        S.spark_prefill(ctx, layers, h, L0, chunk=chunk, more_ctx=more)
         torch.cuda.synchronize()
-        if ctx2 is not None:
-            assert ctx2.device_status() == S.SPARK_OK
-            ctx2.close()
+        for c in more:
+            assert c.device_status() == S.SPARK_OK
+            c.close()
         outs.append((h.cpu().numpy(), [{k: v.float().cpu().numpy() for k, v in c.items()} for _, c in keep]))
     (ha, ca), (hb, cb), (hc, cc) = outs
     assert np.all(np.isfinite(hc))
@@ -295,10 +295,10 @@ def test_pipelined_prefill_checks_its_arguments(ctx):
     layer = S.make_layer(dev, cfg, cache)
     h = torch.zeros(8, sh.d, device="cuda")
     with pytest.raises(S.SparkError) as e:          # one context twice: its workspace would be shared by concurrent kernels
-        S.spark_prefill(ctx, [layer], h, 4, chunk=4, ctx2=ctx)
+        S.spark_prefill(ctx, [layer], h, 4, chunk=4, more_ctx=[ctx])
     assert e.value.status == S.SPARK_ERR_INVALID_ARG
     with pytest.raises(S.SparkError) as e:          # the same stream twice
-        S.spark_prefill(ctx, [layer], h, 4, chunk=4, ctx2=S.SparkContext(0, max_batch=8), stream2=torch.cuda.current_stream())
+        S.spark_prefill(ctx, [layer], h, 4, chunk=4, more_ctx=[S.SparkContext(0, max_batch=8)], more_streams=[torch.cuda.current_stream()])
     assert e.value.status == S.SPARK_ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert ctx.device_status() == S.SPARK_OK
