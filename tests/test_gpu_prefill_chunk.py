@@ -31,6 +31,9 @@ def ctx():
     (synth.GEMMA2_2B, 64, 100, 256, 0),         # the largest chunk a layer call takes
     (synth.TINY, 20, 10, 64, 0),                # more than sixteen tokens on the fallback kernels (shape not served by the GEMMs)
     (synth.GEMMA2_9B, 16, 40, 128, 0),          # 9B shape: 16 query / 8 KV heads, d 3584, d_ff 14336 on every tensor-core path
+    (synth.GEMMA2_2B, 64, 8128, 8192, 0),       # the benchmarked chunk: 64 tokens behind 8128, global layer (gather stage) ...
+    (synth.GEMMA2_2B, 64, 8128, 8192, 4096),    # ... and local layer (window 4096: dense stage)
+    (synth.GEMMA2_2B, 64, 3000, 3072, 0),       # a short cache: dense stage over all rows, ragged last tile
 ])
 def test_chunk_of_a_prompt_equals_token_by_token_decoding(ctx, shape, T, L0, cap, window):
     sh = shape
@@ -58,10 +61,20 @@ def test_chunk_of_a_prompt_equals_token_by_token_decoding(ctx, shape, T, L0, cap
     kc = np.concatenate([kv.k1c[0], kv.k2c[0]], axis=-1).astype(np.float64)
     vc = kv.vc[0].astype(np.float64)
     for t in range(T):                           # the oracle appends token t's row before token t + 1 reads the cache
-        ref = O.decoder_layer(h0[t], W, kc, vc, L0 + t + 1, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd, r_attn=sh.r_attn,
-                              k_attn=sh.k_attn, r_ff=sh.r_ff, k_ff=sh.k_ff, window=window)
-        parity.check_output(got[t], ref["h"], "bf16", f"token {t}")
-        parity.check_output(got[t] - h0[t], ref["h"] - h0[t], "bf16", f"token {t} (update only)")
+        # the oracle's layer, or -- when a cached token sits within rounding distance of a head's threshold -- its variant
+        # with that token on the other side (the reading taken for the attention tests: either is a correct result)
+        last = None
+        for ref in parity.layer_refs_within_band(O, h0[t], W, kc, vc, L0 + t + 1, window, n_q=sh.n_q, n_kv=sh.n_kv, hd=sh.hd,
+                                                 r_attn=sh.r_attn, k_attn=sh.k_attn, r_ff=sh.r_ff, k_ff=sh.k_ff):
+            try:
+                parity.check_output(got[t], ref["h"], "bf16", f"token {t}")
+                parity.check_output(got[t] - h0[t], ref["h"] - h0[t], "bf16", f"token {t} (update only)")
+                last = None
+                break
+            except AssertionError as e:
+                last = e
+        if last is not None:
+            raise last
     # the chunk's rows are in the one cache, the prompt's rows untouched
     k1 = cache["k1c"].float().cpu().numpy()
     v = cache["vc"].float().cpu().numpy()
