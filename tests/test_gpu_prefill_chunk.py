@@ -111,6 +111,8 @@ def test_attention_queries_sharing_one_cache(ctx):
     (40, 4, 4, 128, 64, 512, 300, 40, 100),          # one head per KV head, r = 64, a window sliding over the chunk
     (32, 8, 2, 256, 128, 256, 0, 16, 0),             # four heads per KV head; the chunk starts the sequence (identity for short rows)
     (12, 8, 4, 256, 128, 512, 400, 64, 0),           # a short chunk: per-query kernel over the shared cache
+    (64, 16, 8, 256, 128, 900, 800, 48, 0),          # 9B head layout: eight KV heads, sixteen (KV head, 64 columns) groups
+    (48, 16, 2, 128, 64, 700, 600, 24, 250),         # eight heads per KV head: falls back (more than 128 columns per KV head)
 ])
 @pytest.mark.parametrize("mode", [0, 2])      # second stage: gather per (token, head) / masked dense products where the shape is served
 def test_chunk_attention_on_the_tensor_cores(ctx, mode, T, n_q, n_kv, hd, r, cap, L0, k_attn, window):
