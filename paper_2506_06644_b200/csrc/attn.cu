@@ -353,11 +353,16 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     __syncthreads();
                 }
             }
-            float qreg[GQ][8];
+            // Heads in groups of at most four: with eight heads per KV head the query fragments and the partial products of all
+            // of them at once do not fit the register file (the group's fragments are then re-read from shared memory per step).
+            constexpr int HG = GQ > 4 ? 4 : GQ;
+            float qreg[HG][8];
+            if constexpr (GQ <= 4) {
 #pragma unroll
-            for (int hq = 0; hq < GQ; ++hq)
+                for (int hq = 0; hq < GQ; ++hq)
 #pragma unroll
-                for (int e = 0; e < 8; ++e) qreg[hq][e] = hl < nc1 ? qs[hq * hd + hl * 8 + e] : 0.f;
+                    for (int e = 0; e < 8; ++e) qreg[hq][e] = hl < nc1 ? qs[hq * hd + hl * 8 + e] : 0.f;
+            }
             double s1[GQ], s2[GQ];
             float mx[GQ];
 #pragma unroll
@@ -450,50 +455,59 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                         else w[j].zero();
                     }
                 }
-                float pj[8][GQ];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float wf[8];
-                    w[j].unpack(wf);
-#pragma unroll
-                    for (int hq = 0; hq < GQ; ++hq) pj[j][hq] = dot8r(wf, qreg[hq]);
-                }
-                // butterfly over the 16 lanes of the half-warp: 8 tokens -> 4 -> 2 -> 1 per lane
-                float a4[4][GQ], a2[2][GQ], a1[GQ];
                 const bool b8 = hl & 8, b4 = hl & 4, b2 = hl & 2;
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj)
-#pragma unroll
-                    for (int hq = 0; hq < GQ; ++hq) {
-                        const float keep = b8 ? pj[jj + 4][hq] : pj[jj][hq];
-                        const float send = b8 ? pj[jj][hq] : pj[jj + 4][hq];
-                        a4[jj][hq] = keep + __shfl_xor_sync(kFull, send, 8);
-                    }
-#pragma unroll
-                for (int jj = 0; jj < 2; ++jj)
-#pragma unroll
-                    for (int hq = 0; hq < GQ; ++hq) {
-                        const float keep = b4 ? a4[jj + 2][hq] : a4[jj][hq];
-                        const float send = b4 ? a4[jj][hq] : a4[jj + 2][hq];
-                        a2[jj][hq] = keep + __shfl_xor_sync(kFull, send, 4);
-                    }
-#pragma unroll
-                for (int hq = 0; hq < GQ; ++hq) {
-                    const float keep = b2 ? a2[1][hq] : a2[0][hq];
-                    const float send = b2 ? a2[0][hq] : a2[1][hq];
-                    a1[hq] = keep + __shfl_xor_sync(kFull, send, 2);
-                    a1[hq] += __shfl_xor_sync(kFull, a1[hq], 1);
-                    if constexpr (sizeof(K1T) == 1) a1[hq] *= ksc;
-                }
                 const int t = tok0 + jidx;
-                if ((hl & 1) == 0 && t < w1) {
 #pragma unroll
-                    for (int hq = 0; hq < GQ; ++hq) {
-                        sc[static_cast<size_t>(hq) * ntok + off + t] = a1[hq];
-                        const double v = static_cast<double>(a1[hq]);
-                        s1[hq] += v;
-                        s2[hq] = fma(v, v, s2[hq]);
-                        mx[hq] = fmaxf(mx[hq], a1[hq]);
+                for (int h0 = 0; h0 < GQ; h0 += HG) {
+                    if constexpr (GQ > 4) {
+#pragma unroll
+                        for (int hq = 0; hq < HG; ++hq)
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) qreg[hq][e] = hl < nc1 ? qs[(h0 + hq) * hd + hl * 8 + e] : 0.f;
+                    }
+                    float pj[8][HG];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float wf[8];
+                        w[j].unpack(wf);
+#pragma unroll
+                        for (int hq = 0; hq < HG; ++hq) pj[j][hq] = dot8r(wf, qreg[hq]);
+                    }
+                    // butterfly over the 16 lanes of the half-warp: 8 tokens -> 4 -> 2 -> 1 per lane
+                    float a4[4][HG], a2[2][HG], a1[HG];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                        for (int hq = 0; hq < HG; ++hq) {
+                            const float keep = b8 ? pj[jj + 4][hq] : pj[jj][hq];
+                            const float send = b8 ? pj[jj][hq] : pj[jj + 4][hq];
+                            a4[jj][hq] = keep + __shfl_xor_sync(kFull, send, 8);
+                        }
+#pragma unroll
+                    for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+                        for (int hq = 0; hq < HG; ++hq) {
+                            const float keep = b4 ? a4[jj + 2][hq] : a4[jj][hq];
+                            const float send = b4 ? a4[jj][hq] : a4[jj + 2][hq];
+                            a2[jj][hq] = keep + __shfl_xor_sync(kFull, send, 4);
+                        }
+#pragma unroll
+                    for (int hq = 0; hq < HG; ++hq) {
+                        const float keep = b2 ? a2[1][hq] : a2[0][hq];
+                        const float send = b2 ? a2[0][hq] : a2[1][hq];
+                        a1[hq] = keep + __shfl_xor_sync(kFull, send, 2);
+                        a1[hq] += __shfl_xor_sync(kFull, a1[hq], 1);
+                        if constexpr (sizeof(K1T) == 1) a1[hq] *= ksc;
+                    }
+                    if ((hl & 1) == 0 && t < w1) {
+#pragma unroll
+                        for (int hq = 0; hq < HG; ++hq) {
+                            sc[static_cast<size_t>(h0 + hq) * ntok + off + t] = a1[hq];
+                            const double v = static_cast<double>(a1[hq]);
+                            s1[h0 + hq] += v;
+                            s2[h0 + hq] = fma(v, v, s2[h0 + hq]);
+                            mx[h0 + hq] = fmaxf(mx[h0 + hq], a1[hq]);
+                        }
                     }
                 }
             }
