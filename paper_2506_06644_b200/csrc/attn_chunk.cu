@@ -10,6 +10,9 @@
 //   select  one block per (token, query head): sums of its column over the rows it may see -> theta (Eq. 10/11),
 //           survivors, softmax over the survivors, softplus gate from the k2c rows, weighted sum of the vc rows
 //           (only the survivors' rows are read)
+// or, in place of select when a KV head serves many (token, head) pairs and the rows are few thousand (see "dense second
+// stage" below): stats (theta, maximum, sum of exponentials per column) and dense (every row read once per block; gate and
+// weighted value sum as two more tensor-core products under the selection mask).
 // Same pipeline skeleton and bounded waits as the other tensor-core kernels (tc_common.cuh).
 #include <cstddef>
 
