@@ -39,6 +39,16 @@ constexpr int kPartPad = 8;           // floats in front of a partial accumulato
 // 4 h + i, scaled by qsc[4 h + i]; each term carries four significant bits, 16 in all).  q8 row stride 160 bytes:
 // the 8-byte fragment reads of a half warp fall on distinct banks.
 constexpr int kQ8Stride = 160;
+// bf16 predictor slice on the tensor cores, for blocks with a long share of the slice (the scalar pass is half issue-bound
+// there): 16 cached rows are the M dimension of mma.m16n8k16 bf16 tiles, the query enters as three bf16 terms per head
+// (exact to fp32) in columns 4 h .. 4 h + 2.  q16 row stride 320 bytes: the 16-byte fragment reads of a quarter warp fall on
+// distinct banks.
+constexpr int kQ16Stride = 320;
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void mma_e4m3_16832(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0, unsigned b1) {
     asm volatile("mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
@@ -80,6 +90,7 @@ struct AttnParams {
     int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
     PrefetchSpec pf;   // weights of the kernel after this one, asked into L2 once the first predictor rows are in flight
     int check_finite;  // SPARK_CHECK_FINITE: non-finite score sums are reported in the device status
+    int mma_pass;      // 1: bf16 predictor pass on the tensor cores (long shares; r = 128, at most two heads per KV head)
     int pre_stable;    // 1: the kernel directly before this one writes neither ctx_len nor cache rows other than each
                        //    sequence's newest, so lengths and older rows may be read before dep_wait()
     WsHeader* hdr;
@@ -101,7 +112,7 @@ __device__ __forceinline__ float half_sum(float v) {   // sum over the 16 lanes 
 // MODE 0: flat cut of the token space; 1: segment-aligned cut (the host asks for it when the batch has enough segments);
 // 2: flat cut, all queries read one shared cache (a chunk of a prompt).
 // K1T: storage of the predictor slice k1c (KT, or FP8 E4M3 with one fp32 scale per cached row in p.k1s).
-template <typename KT, typename K1T, int GQ, int MODE>
+template <typename KT, typename K1T, int GQ, int MODE, bool M16 = false>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     constexpr bool AL = MODE == 1;      // segment-aligned cut
     constexpr bool SH = MODE == 2;      // one cache shared by all queries (flat cut)
@@ -121,7 +132,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     __shared__ double zcache[kZc];
     __shared__ double s_z;
     __shared__ int s_last, s_fail, s_aligned;
-    __shared__ __align__(16) unsigned char q8[sizeof(K1T) == 1 ? 8 * kQ8Stride : 16];   // FP8 tensor-core pass 1: query terms
+    __shared__ __align__(16) unsigned char q8[sizeof(K1T) == 1 ? 8 * kQ8Stride : (M16 ? 8 * kQ16Stride : 16)];   // tensor-core pass 1: query terms
     __shared__ float qsc[8];                                                             //   and their scales, per column
     __shared__ int segblk[AL ? kMaxAlignedSegs + 1 : 1];   // first block of every segment (aligned cut)
 
@@ -131,6 +142,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     const int nc1 = r / 8, nc2 = d2 / 8, ncv = hd / 8;
     const int pstride = hd + kPartPad;
     const bool mma8 = sizeof(K1T) == 1 && GQ <= 2 && r == 128;          // FP8 tensor-core pass 1
+    constexpr bool mma16 = M16;                                         // bf16 tensor-core pass 1 (the host checks r = 128)
     const int mg = lane >> 2, mt = lane & 3;                            // fragment row group and column pair
     const K1T* k1c = static_cast<const K1T*>(p.k1c);
     const KT* k2c = static_cast<const KT*>(p.k2c);
@@ -155,6 +167,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     if (tid == 32) s_fail = 0;
     if constexpr (sizeof(K1T) == 1)
         for (int i = tid; i < 8 * kQ8Stride / 4; i += kThreads) reinterpret_cast<unsigned*>(q8)[i] = 0u;
+    if constexpr (M16)
+        for (int i = tid; i < 8 * kQ16Stride / 4; i += kThreads) reinterpret_cast<unsigned*>(q8)[i] = 0u;
     if (warp == 0) {
         int run = 0;
         for (int s0 = 0; s0 < NS; s0 += 32) {
@@ -277,7 +291,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                                                   : make_uint4(0u, 0u, 0u, 0u);
                 }
                 have_pre = true;
-            } else if (w0 < w1) {
+            } else if (w0 < w1 && !mma16) {
                 const int tok0 = w0 + half * 8;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -356,6 +370,30 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             // Heads in groups of at most four: with eight heads per KV head the query fragments and the partial products of all
             // of them at once do not fit the register file (the group's fragments are then re-read from shared memory per step).
             constexpr int HG = GQ > 4 ? 4 : GQ;
+            if constexpr (M16) {
+                {
+                    // The query as three bf16 terms per head (hi + mid + lo = the fp32 value to its last bit but one): a warp per
+                    // head, four values per lane, term i of head h in row 4 h + i of q16.
+                    if (warp < GQ) {
+#pragma unroll
+                        for (int i = 0; i < 3; ++i) {
+                            unsigned packed[2];
+#pragma unroll
+                            for (int e2 = 0; e2 < 2; ++e2) {
+                                float a = qs[warp * hd + lane * 4 + 2 * e2], b = qs[warp * hd + lane * 4 + 2 * e2 + 1];
+                                for (int k = 0; k < i; ++k) {          // what the earlier terms left
+                                    a -= __bfloat162float(__float2bfloat16_rn(a));
+                                    b -= __bfloat162float(__float2bfloat16_rn(b));
+                                }
+                                const __nv_bfloat162 hb = __floats2bfloat162_rn(a, b);
+                                packed[e2] = *reinterpret_cast<const unsigned*>(&hb);
+                            }
+                            *reinterpret_cast<uint2*>(q8 + (4 * warp + i) * kQ16Stride + lane * 8) = make_uint2(packed[0], packed[1]);
+                        }
+                    }
+                    __syncthreads();
+                }
+            }
             float qreg[HG][8];
             if constexpr (GQ <= 4) {
 #pragma unroll
@@ -434,6 +472,58 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     tm = fmaxf(tm, __shfl_xor_sync(kFull, tm, o));
                 }
                 if (owner && mg == 0) { red[warp][myh][0] = t1; red[warp][myh][1] = t2; redm[warp][myh] = tm; }
+            } else if constexpr (M16) {
+                {
+                    const int myh = mt >> 1;                                  // the head whose terms this lane's two columns hold
+                    const bool owner = (mt & 1) == 0 && myh < GQ;              // ... and the lane that ends up with its scores
+                    double t1 = 0.0, t2 = 0.0;
+                    float tm = -INFINITY;
+#pragma unroll 1
+                    for (int base = w0; base < w1; base += 16) {               // a 16-row tile per trip: eight 16-byte loads in flight per lane
+                        // A lane takes the 16-byte pieces mt, mt + 4, mt + 8, mt + 12 of rows mg and mg + 8: the k-slots of an MMA
+                        // may be any permutation of the columns as long as both operands use it, so a piece feeds two MMAs.
+                        uint4 w[2][4];
+#pragma unroll
+                        for (int hrow = 0; hrow < 2; ++hrow) {
+                            const int t = base + mg + 8 * hrow;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                w[hrow][j] = t < w1 ? ld_stream16(reinterpret_cast<const uint4*>(kbase + static_cast<int64_t>(t) * r) + mt + 4 * j)
+                                                    : make_uint4(0u, 0u, 0u, 0u);
+                        }
+                        float dd[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 qb = *reinterpret_cast<const uint4*>(q8 + mg * kQ16Stride + 16 * (mt + 4 * j));
+                            mma_bf16_16816(dd, w[0][j].x, w[1][j].x, w[0][j].y, w[1][j].y, qb.x, qb.y);
+                            mma_bf16_16816(dd, w[0][j].z, w[1][j].z, w[0][j].w, w[1][j].w, qb.z, qb.w);
+                        }
+                        float sa = dd[0] + dd[1], sb2 = dd[2] + dd[3];       // the head's four columns sit in this lane and its neighbour
+                        sa += __shfl_xor_sync(kFull, sa, 1);
+                        sb2 += __shfl_xor_sync(kFull, sb2, 1);
+                        if (owner) {
+                            const int ta = base + mg, tb2 = ta + 8;
+                            if (ta < w1) {
+                                sc[static_cast<size_t>(myh) * ntok + off + ta] = sa;
+                                const double v = static_cast<double>(sa);
+                                t1 += v; t2 = fma(v, v, t2); tm = fmaxf(tm, sa);
+                            }
+                            if (tb2 < w1) {
+                                sc[static_cast<size_t>(myh) * ntok + off + tb2] = sb2;
+                                const double v = static_cast<double>(sb2);
+                                t1 += v; t2 = fma(v, v, t2); tm = fmaxf(tm, sb2);
+                            }
+                        }
+                    }
+                    // sums over the eight row groups (lane bits 2..4); lanes with mg == 0 hold a head's totals
+#pragma unroll
+                    for (int o = 4; o < 32; o <<= 1) {
+                        t1 += __shfl_xor_sync(kFull, t1, o);
+                        t2 += __shfl_xor_sync(kFull, t2, o);
+                        tm = fmaxf(tm, __shfl_xor_sync(kFull, tm, o));
+                    }
+                    if (owner && mg == 0) { red[warp][myh][0] = t1; red[warp][myh][1] = t2; redm[warp][myh] = tm; }
+                }
             } else {
 #pragma unroll 1
             for (int base = w0; base < w1; base += 16) {
@@ -779,10 +869,10 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
     p.trace.mark(3);
 }
 
-template <typename KT, typename K1T, int GQ, int MODE>
+template <typename KT, typename K1T, int GQ, int MODE, bool M16 = false>
 int launch_al(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) {
     static bool configured[64] = {};
-    auto kern = attn_kernel<KT, K1T, GQ, MODE>;
+    auto kern = attn_kernel<KT, K1T, GQ, MODE, M16>;
     if (ctx->device >= 0 && ctx->device < 64 && !configured[ctx->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ctx->max_smem_optin - 8192) != cudaSuccess)
             return SPARK_ERR_CUDA;
@@ -799,9 +889,16 @@ int launch_one(spark_ctx* ctx, AttnParams& p, size_t smem, cudaStream_t stream) 
     // gives the segments 1/(blocks per segment) uneven shares of the streaming pass: worth it while a block's
     // share of that pass is short.
     const int ns = p.B * p.n_kv;
+    const bool aligned = p.al_ok && ns >= kMinAlignedSegs && ns <= ctx->num_sms && ns <= kMaxAlignedSegs;
+    if constexpr (sizeof(KT) == 2 && sizeof(K1T) == 2 && GQ <= 2) {      // long shares: the predictor pass on the tensor cores
+        if (p.mma_pass && p.r == 128) {
+            if (p.seg_mask != -1) return launch_al<KT, K1T, GQ, 2, true>(ctx, p, smem, stream);
+            if (aligned) return launch_al<KT, K1T, GQ, 1, true>(ctx, p, smem, stream);
+            return launch_al<KT, K1T, GQ, 0, true>(ctx, p, smem, stream);
+        }
+    }
     if (p.seg_mask != -1) return launch_al<KT, K1T, GQ, 2>(ctx, p, smem, stream);
-    if (p.al_ok && ns >= kMinAlignedSegs && ns <= ctx->num_sms && ns <= kMaxAlignedSegs)
-        return launch_al<KT, K1T, GQ, 1>(ctx, p, smem, stream);
+    if (aligned) return launch_al<KT, K1T, GQ, 1>(ctx, p, smem, stream);
     return launch_al<KT, K1T, GQ, 0>(ctx, p, smem, stream);
 }
 
@@ -894,6 +991,10 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     // a chunk's rows are all fresh from the kernel ahead; the FP8 tensor-core pass requests its first tile without holding
     // the newest row back, so it waits for the kernel ahead first
     p.pre_stable = p.defer && !shared && k1s == nullptr;
+    // measured: the tensor-core pass wins from about 450 tokens a block on (16384 tokens, one sequence: 16.3 -> 15.5 us; eight
+    // sequences x 32768: 77.2 -> 71.9) but gives up the rows requested before the kernel ahead has finished, which a layer
+    // call of one 9B-shaped sequence (443 tokens a block) still wants: from 800 tokens a block
+    p.mma_pass = (kvdtype == SPARK_BF16 && k1s == nullptr && ntok >= 800) ? 1 : 0;
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;

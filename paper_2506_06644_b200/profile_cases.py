@@ -224,7 +224,7 @@ def case_layer_ab(shape_name="2b", n_layers=12, ctx_len=8192):
     print(f"  G1 -> G6 (a layer minus its P1): median {np.median(dl):6.2f}")
 
 
-CASES = {"layer_ab": case_layer_ab, "chunk64": case_chunk, "chunk64_4k": lambda: case_chunk(ctx_len=4096), "layer8": lambda: case_layer(n_layers=4, B=8, steps=2), "ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
+CASES = {"layer_ab": case_layer_ab, "chunk64": case_chunk, "chunk64_4k": lambda: case_chunk(ctx_len=4096), "attn8x32k": lambda: case_attn(B=8, ctx_len=32768, sets=3), "layer8": lambda: case_layer(n_layers=4, B=8, steps=2), "ffn": case_ffn, "ffn4": lambda: case_ffn(B=4, sets=12), "ffn16": lambda: case_ffn(B=16, sets=12), "ffn64": lambda: case_ffn(B=64, sets=12), "attn": case_attn, "topk": case_topk, "layer": case_layer}
 
 if __name__ == "__main__":
     name = sys.argv[1] if len(sys.argv) > 1 else ""
