@@ -737,6 +737,72 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             };
             int* ltok = sel_tok + static_cast<size_t>(hq) * ntok;
             float* la = sel_a + static_cast<size_t>(hq) * ntok;
+            bool listed = false;
+            if constexpr (M16) {
+            if (p.sel_list) {
+                listed = true;
+                // Two sweeps over the warp's scores, four 32-token steps per trip with their loads issued together (a step per
+                // trip left every warp waiting on its own chain of load, compare and vote: 0.3 us per step).  The first sweep
+                // counts what the warp will list; a single shared-memory atomic reserves that many entries of the head's list.
+                int mine = 0;
+#pragma unroll 1
+                for (int base = w0; base < w1; base += 128) {
+                    float sv[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = base + 32 * u + lane;
+                        sv[u] = t < w1 ? srow[t] : -INFINITY;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const bool valid = base + 32 * u + lane < w1;
+                        mine += __popc(__ballot_sync(kFull, valid && (p.dense || ident || sv[u] > th)));
+                    }
+                }
+                int lpos = 0;
+                if (lane == 0 && mine > 0) lpos = atomicAdd(&sel_n[hq], mine);
+                lpos = __shfl_sync(kFull, lpos, 0);
+#pragma unroll 1
+                for (int base = w0; base < w1; base += 128) {
+                    float sv[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = base + 32 * u + lane;
+                        sv[u] = t < w1 ? srow[t] : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = base + 32 * u + lane;
+                        const bool valid = t < w1;
+                        const float s = sv[u];
+                        const bool sel = valid && (ident || s > th);
+                        const float a = sel ? s - smax : -INFINITY;        // softmax is shift-invariant: the head's largest score is the reference
+                        const unsigned bsel = __ballot_sync(kFull, sel);
+                        const unsigned bal = p.dense ? __ballot_sync(kFull, valid) : bsel;
+                        if (p.count != nullptr && bsel != 0u) {
+                            int cbase = 0;
+                            if (lane == 0) cbase = atomicAdd(&p.count[bh], __popc(bsel));
+                            cbase = __shfl_sync(kFull, cbase, 0);
+                            if (sel && p.idx != nullptr) {
+                                const int64_t pos = static_cast<int64_t>(cbase) + __popc(bsel & ((1u << lane) - 1u));
+                                if (pos < p.idx_cap) p.idx[static_cast<int64_t>(bh) * p.idx_cap + pos] = lo + t;
+                                else atomicCAS(&p.hdr->status, SPARK_OK, SPARK_ERR_OVERFLOW);
+                            }
+                        }
+                        // The survivors of the whole piece go to one list per head, from which the head's warps then take four
+                        // entries each: a warp that found many does not make the block wait for a second round of loads while
+                        // others found none.
+                        if ((bal >> lane) & 1u) {
+                            const int pos = lpos + __popc(bal & ((1u << lane) - 1u));
+                            ltok[pos] = t;
+                            la[pos] = a;
+                        }
+                        lpos += __popc(bal);
+                    }
+                }
+            }
+            }
+            if (!listed) {
 #pragma unroll 1
             for (int base = w0; base < w1; base += 32) {
                 const int t = base + lane;
@@ -787,6 +853,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
                     }
                     gather4(tk, v, av);
                 }
+            }
             }
             if (p.sel_list) {
                 __syncthreads();
