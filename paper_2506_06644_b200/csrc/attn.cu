@@ -90,6 +90,7 @@ struct AttnParams {
     int defer;         // 1: leave o unnormalised and the cells for the next kernel to clear
     PrefetchSpec pf;   // weights of the kernel after this one, asked into L2 once the first predictor rows are in flight
     int check_finite;  // SPARK_CHECK_FINITE: non-finite score sums are reported in the device status
+    int long_share;    // 1: a block owns 800 or more tokens of the slice
     int mma_pass;      // 1: bf16 predictor pass on the tensor cores (long shares; r = 128, at most two heads per KV head)
     int pre_stable;    // 1: the kernel directly before this one writes neither ctx_len nor cache rows other than each
                        //    sequence's newest, so lengths and older rows may be read before dep_wait()
@@ -738,8 +739,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const AttnParams p) {
             int* ltok = sel_tok + static_cast<size_t>(hq) * ntok;
             float* la = sel_a + static_cast<size_t>(hq) * ntok;
             bool listed = false;
-            if constexpr (M16) {
-            if (p.sel_list) {
+            if constexpr (M16 || sizeof(K1T) == 1) {
+            if (p.sel_list && (M16 || p.long_share)) {
                 listed = true;
                 // Two sweeps over the warp's scores, four 32-token steps per trip with their loads issued together (a step per
                 // trip left every warp waiting on its own chain of load, compare and vote: 0.3 us per step).  The first sweep
@@ -1061,7 +1062,8 @@ int attn_launch(spark_ctx* ctx, const float* q, const void* k1c, const void* k2c
     // measured: the tensor-core pass wins from about 450 tokens a block on (16384 tokens, one sequence: 16.3 -> 15.5 us; eight
     // sequences x 32768: 77.2 -> 71.9) but gives up the rows requested before the kernel ahead has finished, which a layer
     // call of one 9B-shaped sequence (443 tokens a block) still wants: from 800 tokens a block
-    p.mma_pass = (kvdtype == SPARK_BF16 && k1s == nullptr && ntok >= 800) ? 1 : 0;
+    p.long_share = ntok >= 800 ? 1 : 0;
+    p.mma_pass = (kvdtype == SPARK_BF16 && k1s == nullptr && p.long_share) ? 1 : 0;
     p.scores = reinterpret_cast<float*>(ctx->scratch + cells_b + part_b);
     p.ntok = static_cast<int>(ntok);
     p.sc_smem = sc_smem ? 1 : 0;
